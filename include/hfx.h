@@ -1,0 +1,266 @@
+/*
+ * hfx.h -- C ABI of the multi-SLO scheduler hot path (one GPU, sm_100a).
+ *
+ * The library evaluates, for a whole request table at once, the decision
+ * primitives of the paper's dispatcher (Sec. 3.3.1 "Dispatching Mechanism and
+ * Policy"): the latency predictor E_p / E_d, the safe token budget (Eq. 3),
+ * slack and the priority key, the per-replica priority order, the budgeted
+ * greedy admission ("most urgent requests that fit", dispatching step 3) and
+ * the maturity-time update (dispatching step 4).  hfx_sim_run steps many
+ * independent replicas through that scheduler over arrival traces and reports
+ * the attainment metric (Eq. 2) and latency percentiles.
+ *
+ * Conventions
+ *   - Every time is an int64 count of nanoseconds.  There is no floating point
+ *     anywhere in the library.
+ *   - "device" pointers are CUDA device pointers of the current device, each
+ *     16-byte aligned; "host" pointers are ordinary host memory.
+ *   - The caller owns every table, state and output buffer.  The library owns
+ *     only the workspace it allocates in hfx_sched_create.
+ *   - Calls are asynchronous on the stream given at create; only
+ *     hfx_sched_status synchronises.
+ *   - Return value: HFX_OK (0) or a negative HFX_E_* code.  Argument errors are
+ *     reported before anything is launched.  Bad data found on the device (an
+ *     id out of range, a length outside the domain) never traps: the row is
+ *     treated as inactive and a bit is set in a sticky status word that
+ *     hfx_sched_status returns.
+ *   - There is no CPU fallback: without a CUDA device every entry point that
+ *     would launch work returns HFX_E_CUDA.
+ *
+ * Domain (checked at create for the configuration, per row on the device for
+ * lengths and ids; timestamps are not checked):
+ *   rows            1 .. 2^27 per call (0 rows is a no-op)
+ *   replicas        1 .. 65536, classes 1 .. 64
+ *   prompt_len, gen 0 .. 2^24      token_cap 1 .. 2^24
+ *   c0, d0 0 .. 2^40   c1, d1 0 .. 2^30   c2 0 .. 2^12   d2 0 .. 2^8
+ *   ttft_slo <= 2^44, tpot_slo <= 2^34 (<= 0 means unbounded), prio 0 .. 62
+ *   timestamps      -2^56 .. 2^56
+ */
+#ifndef HFX_H
+#define HFX_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes --------------------------------------------------------- */
+#define HFX_OK            0
+#define HFX_E_ARG        -1   /* NULL or out-of-domain argument              */
+#define HFX_E_ALIGN      -2   /* a device pointer is not 16-byte aligned     */
+#define HFX_E_CAPACITY   -3   /* more rows / replicas than created for       */
+#define HFX_E_CUDA       -4   /* a CUDA runtime call failed (no device, ...) */
+#define HFX_E_TIMEOUT    -5   /* a bounded device-side wait ran out          */
+#define HFX_E_NOMEM      -6   /* workspace allocation failed                 */
+
+/* bits of the sticky device status word */
+#define HFX_ST_BAD_REPLICA  1u  /* replica_id outside [0, n_replicas)         */
+#define HFX_ST_BAD_CLASS    2u  /* class_id >= n_classes                      */
+#define HFX_ST_BAD_LEN      4u  /* prompt_len or gen outside [0, 2^24]        */
+#define HFX_ST_TIMEOUT      8u  /* a device-side wait gave up                 */
+
+/* request states (column `state`) */
+#define HFX_QUEUED    0
+#define HFX_RUNNING   1
+#define HFX_DONE      2
+#define HFX_REJECTED  3
+
+/* replica modes */
+#define HFX_COLOCATED 0   /* prefill and decode share the instance            */
+#define HFX_PREFILL   1   /* P-stage instance of the disaggregated mode       */
+#define HFX_DECODE    2   /* D-stage instance of the disaggregated mode       */
+
+/* budget modes */
+#define HFX_BUDGET_SAFE      0  /* Eq. 3 (generalised to the quadratic E_p)   */
+#define HFX_BUDGET_CAP_ONLY  1  /* capacity caps only, no SLO-derived bound   */
+
+/* hfx_sched_step flags */
+#define HFX_COMMIT 1u           /* apply the admitted batch to the table      */
+
+#define HFX_INF        INT64_MAX              /* "unbounded" budget / minimum */
+#define HFX_TIME_MAX   (INT64_C(1) << 62)     /* saturation of maturity       */
+#define HFX_SLACK_MAX  ((INT64_C(1) << 39) - 1)
+#define HFX_SLACK_MIN  (-(INT64_C(1) << 39))
+#define HFX_MAX_TOKENS (1 << 24)
+
+typedef struct hfx_sched hfx_sched; /* opaque */
+
+/* Latency predictor (Sec. 3.3.1: E_p of a prefill batch of t tokens, E_d of one
+ * decode iteration of a running batch; the quadratic term of the cited
+ * prefill model is kept as c2, the paper's linear model is c2 = 0):
+ *   E_p(t)     = c0 + c1*t + c2*t*t
+ *   E_d(b, kv) = d0 + d1*b + d2*kv     b = batch size, kv = sum of context
+ *                                       lengths (prompt_len + gen) of the batch */
+typedef struct hfx_latency_model { int64_t c0, c1, c2, d0, d1, d2; } hfx_latency_model;
+
+/* One SLO class: TTFT and TPOT targets (Problem Definition: each request
+ * carries heterogeneous SLOs) and the class priority, 0 = highest
+ * (Sec. 3.3.2, "Priority as input"). */
+typedef struct hfx_slo_class {
+  int64_t ttft_slo_ns;  /* <= 0 : no TTFT bound */
+  int64_t tpot_slo_ns;  /* <= 0 : no TPOT bound */
+  int32_t prio;         /* 0 .. 62 */
+  int32_t reserved;
+} hfx_slo_class;
+
+typedef struct hfx_replica_cfg {
+  int32_t mode;       /* HFX_COLOCATED / HFX_PREFILL / HFX_DECODE           */
+  int32_t token_cap;  /* tokens one iteration can take                       */
+  int32_t batch_cap;  /* sequences in the running batch; 0 = unlimited       */
+} hfx_replica_cfg;
+
+typedef struct hfx_options {
+  int32_t  budget_mode; /* HFX_BUDGET_*                                       */
+  int32_t  weight_max;  /* 0: prio = class prio; >0: prio = clamp(weight_max -
+                           weight, 0, 62) and the table's `weight` is read    */
+  uint32_t flags;       /* reserved, 0                                        */
+  uint32_t reserved;
+} hfx_options;
+
+/* Request table, structure of arrays, all columns device pointers of n_rows
+ * elements (Problem Definition: a request has an arrival timestamp, a prompt,
+ * an output length and TTFT / TPOT SLOs).  Columns the call does not need may
+ * be NULL: `weight` unless weight_max > 0; `output_len`, `last_token_ns`,
+ * `finish_ns` unless HFX_COMMIT is given or the call is hfx_sim_run. */
+typedef struct hfx_table {
+  int64_t        n_rows;
+  const int32_t *replica_id;     /* instance the request is bound to          */
+  const uint8_t *class_id;       /* index into the SLO class table            */
+  uint8_t       *state;          /* HFX_QUEUED .. HFX_REJECTED (written by
+                                    COMMIT and by hfx_sim_run)                */
+  const int32_t *prompt_len;     /* tokens                                    */
+  const int32_t *output_len;     /* true output length; read only to detect
+                                    completion, never by the scheduler        */
+  int32_t       *gen;            /* decode steps completed after the first
+                                    token                                     */
+  const int64_t *arrival_ns;
+  int64_t       *first_token_ns; /* valid once RUNNING (and for QUEUED rows of
+                                    a DECODE replica, which are prefilled)    */
+  int64_t       *last_token_ns;
+  int64_t       *finish_ns;
+  const int32_t *req_id;         /* unique; final tie-break of the order      */
+  const int32_t *weight;         /* priority weight, higher = served first    */
+} hfx_table;
+
+/* Per-replica clock and maturity time (Sec. 3.3.1: the earliest time an
+ * instance may take new load), device arrays of n_replicas elements.  Read by
+ * every step; written only by HFX_COMMIT (clock advanced, maturity replaced by
+ * maturity_next).  Without HFX_COMMIT a step changes neither the table nor
+ * this state. */
+typedef struct hfx_replica_state {
+  int64_t *now_ns;
+  int64_t *maturity_ns;
+} hfx_replica_state;
+
+/* Outputs of one step.  Device pointers.  Required: order, seg_off, admit,
+ * slack_ns, budget, adm_cost, adm_count, maturity_next.  Optional (NULL =
+ * skip): the rest. */
+typedef struct hfx_step_out {
+  int64_t  *slack_ns;      /* [n_rows] remaining SLO budget, unclamped; 0 for
+                              inactive rows                                   */
+  int64_t  *pred_ttft_ns;  /* [n_rows] optional                               */
+  int64_t  *pred_tpot_ns;  /* [n_rows] optional                               */
+  uint64_t *key;           /* [n_rows] optional: replica<16> | phase<2> |
+                              prio<6> | (clamp(slack)+2^39)<40>               */
+  int32_t  *order;         /* [n_rows] row indices, replica-major, each
+                              replica's rows ascending by (key, req_id); rows
+                              with a bad replica_id follow seg_off[R], by
+                              req_id                                          */
+  int32_t  *seg_off;       /* [n_replicas+1] start of each replica in order   */
+  uint8_t  *admit;         /* [n_rows] 1 = in the next batch (running rows and
+                              admitted queued rows)                           */
+  int32_t  *admitted_rows; /* [n_rows] optional: for replica r the first
+                              adm_count[r] entries after seg_off[r] are the
+                              newly admitted rows in priority order, the rest
+                              of the replica's range is -1                    */
+  int64_t  *budget;        /* [n_replicas] tokens (COLOCATED, PREFILL) or ns
+                              of decode-step latency (DECODE); HFX_INF if
+                              unbounded                                       */
+  int64_t  *e_d_ns;        /* [n_replicas] optional: decode-iteration latency
+                              of the current running batch                    */
+  int32_t  *n_run;         /* [n_replicas] optional                           */
+  int64_t  *sum_kv;        /* [n_replicas] optional                           */
+  int64_t  *adm_cost;      /* [n_replicas] total cost of newly admitted rows  */
+  int32_t  *adm_count;     /* [n_replicas] number of newly admitted rows      */
+  int64_t  *maturity_next; /* [n_replicas] maturity time after this dispatch
+                              (dispatching step 4); the old one if nothing
+                              was admitted                                    */
+} hfx_step_out;
+
+/* Outputs of the simulator, device arrays of n_traces elements; all required
+ * except now_ns. */
+typedef struct hfx_sim_out {
+  int32_t *iters_executed; /* iterations that did work or advanced the clock  */
+  int32_t *finished;       /* rows that ended DONE                            */
+  int32_t *rejected;       /* rows that ended REJECTED                        */
+  int32_t *attained;       /* DONE rows that met both SLOs (numerator of
+                              Eq. 2; the denominator is the trace length)     */
+  int64_t *ttft_p50_ns;    /* nearest-rank percentiles; -1 if no sample       */
+  int64_t *ttft_p99_ns;
+  int64_t *tpot_p50_ns;
+  int64_t *tpot_p99_ns;
+  int64_t *now_ns;         /* optional: final clock of the trace              */
+} hfx_sim_out;
+
+/* Create a scheduler.  `model`, `classes[n_classes]`, `replicas[n_replicas]`
+ * and `opts` are host pointers, copied.  `max_rows` bounds n_rows of later
+ * calls and sizes the workspace (about 40 bytes per row plus 64 bytes per
+ * replica of device memory).  `cuda_stream` is a cudaStream_t (NULL = the
+ * default stream).  Errors: HFX_E_ARG (NULL pointer, value outside the domain
+ * above), HFX_E_CUDA, HFX_E_NOMEM.  On error *out is NULL. */
+int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
+                     const hfx_slo_class *classes, int n_classes,
+                     const hfx_replica_cfg *replicas, int n_replicas,
+                     int64_t max_rows, const hfx_options *opts,
+                     void *cuda_stream);
+
+/* One scheduling iteration over the whole table (dispatching steps 2-4 of
+ * Sec. 3.3.1 for every replica at once, and its P-stage / D-stage variants of
+ * the paragraph "Disaggregated Mode"): per-replica aggregates of the running
+ * batch, E_d, the safe budget (Eq. 3), per-row predicted TTFT / TPOT, slack and
+ * key, the per-replica order, admission under the budget by a segmented prefix
+ * sum, the new maturity time.  With HFX_COMMIT the admitted batch is applied:
+ * admitted rows become RUNNING with their first-token time, running rows
+ * advance one decode step, finished rows become DONE, oversize prompts become
+ * REJECTED, and the replica clock advances by the iteration's latency (or, when
+ * the replica is idle, to its next event).
+ * `table`, `state`, `out` are host structs holding device pointers.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_CUDA. */
+int hfx_sched_step(hfx_sched *s, const hfx_table *table,
+                   const hfx_replica_state *state, const hfx_step_out *out,
+                   uint32_t flags);
+
+/* Trace-driven simulation (events are request arrivals and iteration
+ * completions, Problem Definition; metrics are Eq. 2 and the TTFT / TPOT
+ * definitions).  `table` holds n_traces traces back to back, trace j being
+ * rows trace_off[j] .. trace_off[j+1]-1 (device int32 array of n_traces+1
+ * offsets), sorted by arrival within a trace; trace j runs on replica j of the
+ * scheduler, which must be COLOCATED.  replica_id is not read.  Every trace
+ * starts at time 0 with all rows QUEUED (the incoming state, gen and time
+ * columns are overwritten) and runs `iters` iterations of step + commit, or
+ * until nothing is left to happen.  Written: state, gen, first_token_ns,
+ * last_token_ns, finish_ns and `out`.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY (n_traces > n_replicas, or a
+ * trace longer than 8192 rows), HFX_E_CUDA. */
+int hfx_sim_run(hfx_sched *s, const hfx_table *table, const int32_t *trace_off,
+                int32_t n_traces, int32_t iters, const hfx_sim_out *out);
+
+/* Synchronise the scheduler's stream and return the sticky status word
+ * (HFX_ST_* bits) in *status_word (host pointer); the word is then cleared.
+ * Returns HFX_E_TIMEOUT if HFX_ST_TIMEOUT was set, HFX_E_CUDA if the stream
+ * reports an error, else HFX_OK. */
+int hfx_sched_status(hfx_sched *s, uint32_t *status_word);
+
+/* Number of kernels the library has launched on behalf of `s` so far. */
+int64_t hfx_sched_launch_count(const hfx_sched *s);
+
+void hfx_sched_destroy(hfx_sched *s);
+
+/* Static, never NULL. */
+const char *hfx_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HFX_H */

@@ -1,0 +1,188 @@
+"""CPU oracle of the scheduler hot path -- TEST INFRASTRUCTURE, not the product.
+
+`hfx_oracle.c` is the oracle (plain single-threaded C written from the paper);
+this module compiles it with gcc on first use and wraps it with ctypes + numpy.
+Only the tests, the smoke check and the benchmark's CPU-baseline leg import it.
+It shares nothing with the CUDA library and never imports it.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hfx_oracle.c")
+_SO = os.path.join(_HERE, "libhfx_oracle.so")
+_lib = None
+
+INF = (1 << 63) - 1
+TIME_MAX = 1 << 62
+SLACK_MAX = (1 << 39) - 1
+SLACK_MIN = -(1 << 39)
+CM_WORKED, CM_JUMPED, CM_STUCK = 0, 1, 2
+FLAG_COMMIT = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C11, -O2).  Returns the .so path."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-std=gnu11", "-O2", "-fPIC", "-shared", "-Wall", "-o", tmp, _SRC])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+class _Model(C.Structure):
+    _fields_ = [(k, C.c_int64) for k in ("c0", "c1", "c2", "d0", "d1", "d2")]
+
+
+class _Class(C.Structure):
+    _fields_ = [("ttft", C.c_int64), ("tpot", C.c_int64), ("prio", C.c_int32), ("pad", C.c_int32)]
+
+
+class _Replica(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("token_cap", C.c_int32), ("batch_cap", C.c_int32)]
+
+
+class _Config(C.Structure):
+    _fields_ = [("model", _Model), ("classes", C.POINTER(_Class)), ("n_classes", C.c_int32),
+                ("replicas", C.POINTER(_Replica)), ("n_replicas", C.c_int32),
+                ("budget_mode", C.c_int32), ("weight_max", C.c_int32)]
+
+
+_TABLE_COLS = ["replica_id", "class_id", "state", "prompt_len", "output_len", "gen", "arrival_ns",
+               "first_token_ns", "last_token_ns", "finish_ns", "req_id", "weight"]
+
+
+class _Table(C.Structure):
+    _fields_ = [("n", C.c_int64)] + [(k, C.c_void_p) for k in _TABLE_COLS]
+
+
+_STEP_OUT = [("slack", np.int64, "n"), ("pred_ttft", np.int64, "n"), ("pred_tpot", np.int64, "n"),
+             ("key", np.uint64, "n"), ("order", np.int32, "n"), ("seg_off", np.int32, "R1"),
+             ("admit", np.uint8, "n"), ("admitted_rows", np.int32, "n"), ("budget", np.int64, "R"),
+             ("e_d", np.int64, "R"), ("n_run", np.int32, "R"), ("sum_kv", np.int64, "R"),
+             ("adm_cost", np.int64, "R"), ("adm_count", np.int32, "R"),
+             ("maturity_next", np.int64, "R"), ("epmax", np.int64, "R"), ("n_safe", np.int64, "R")]
+
+
+class _StepOut(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k, _, _ in _STEP_OUT]
+
+
+_SIM_OUT = [("iters_executed", np.int32), ("finished", np.int32), ("rejected", np.int32),
+            ("attained", np.int32), ("ttft_p50", np.int64), ("ttft_p99", np.int64),
+            ("tpot_p50", np.int64), ("tpot_p99", np.int64), ("now", np.int64)]
+
+
+class _SimOut(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k, _ in _SIM_OUT]
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.ora_Ep.restype = C.c_int64
+        L.ora_Ep.argtypes = [C.POINTER(_Model), C.c_int64]
+        L.ora_Ed.restype = C.c_int64
+        L.ora_Ed.argtypes = [C.POINTER(_Model), C.c_int64, C.c_int64]
+        L.ora_key.restype = C.c_uint64
+        L.ora_key.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int64]
+        L.ora_epmax.restype = C.c_int64
+        L.ora_epmax.argtypes = [C.c_int64, C.c_int, C.c_int64, C.c_int64]
+        L.ora_nsafe.restype = C.c_int64
+        L.ora_nsafe.argtypes = [C.POINTER(_Model), C.c_int64, C.c_int64]
+        L.ora_step.restype = C.c_uint32
+        L.ora_step.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p, C.c_void_p,
+                               C.POINTER(_StepOut), C.c_uint32]
+        L.ora_sim.restype = C.c_uint32
+        L.ora_sim.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p, C.c_int32, C.c_int32,
+                              C.c_int32, C.POINTER(_SimOut)]
+        _lib = L
+    return _lib
+
+
+def _model(m) -> _Model:
+    return _Model(*[int(x) for x in m])
+
+
+def Ep(model, t: int) -> int:
+    return int(lib().ora_Ep(C.byref(_model(model)), int(t)))
+
+
+def Ed(model, b: int, kv: int) -> int:
+    return int(lib().ora_Ed(C.byref(_model(model)), int(b), int(kv)))
+
+
+def key(replica: int, phase: int, prio: int, slack: int) -> int:
+    return int(lib().ora_key(replica, phase, prio, slack))
+
+
+def epmax(min_ttft: int, decoding: bool, min_tpot: int, e_d: int) -> int:
+    return int(lib().ora_epmax(min_ttft, int(decoding), min_tpot, e_d))
+
+
+def nsafe(model, epmax_: int, token_cap: int) -> int:
+    return int(lib().ora_nsafe(C.byref(_model(model)), epmax_, token_cap))
+
+
+class _Ctx:
+    """Keeps the ctypes structs and the arrays they point to alive together."""
+
+    def __init__(self, wl):
+        self.keep = []
+        cls = (_Class * len(wl.classes))(*[_Class(int(a), int(b), int(p), 0) for a, b, p in wl.classes])
+        reps = (_Replica * wl.n_replicas)(*[_Replica(int(r[0]), int(r[1]), int(r[2])) for r in wl.replicas])
+        self.keep += [cls, reps]
+        self.cfg = _Config(_model(wl.model), cls, len(wl.classes), reps, wl.n_replicas,
+                           int(wl.budget_mode), int(wl.weight_max))
+        self.table = _Table()
+        self.table.n = wl.n_rows
+        for k in _TABLE_COLS:
+            a = wl.table[k]
+            assert a.flags["C_CONTIGUOUS"]
+            setattr(self.table, k, a.ctypes.data)
+
+
+def step(wl, commit: bool = False) -> Dict[str, np.ndarray]:
+    """One scheduling iteration over wl (in place on wl.table / wl.now / wl.maturity
+    when commit=True).  Returns every output as numpy arrays plus 'status'."""
+    L = lib()
+    ctx = _Ctx(wl)
+    n, R = wl.n_rows, wl.n_replicas
+    out = {}
+    so = _StepOut()
+    for k, dt, dim in _STEP_OUT:
+        size = {"n": n, "R": R, "R1": R + 1}[dim]
+        out[k] = np.zeros(size, dt)
+        setattr(so, k, out[k].ctypes.data)
+    now = wl.now if commit else wl.now.copy()
+    mat = wl.maturity if commit else wl.maturity.copy()
+    st = L.ora_step(C.byref(ctx.cfg), C.byref(ctx.table), now.ctypes.data, mat.ctypes.data,
+                    C.byref(so), FLAG_COMMIT if commit else 0)
+    out["status"] = int(st)
+    return out
+
+
+def sim(wl, iters: Optional[int] = None, j0: int = 0, j1: Optional[int] = None) -> Dict[str, np.ndarray]:
+    """Simulate traces [j0, j1) of wl in place (state, gen and time columns of wl.table
+    are overwritten).  Returns per-trace metrics (arrays of n_traces; only [j0, j1) filled)."""
+    L = lib()
+    ctx = _Ctx(wl)
+    T = wl.trace_off.shape[0] - 1
+    j1 = T if j1 is None else j1
+    out = {}
+    so = _SimOut()
+    for k, dt in _SIM_OUT:
+        out[k] = np.zeros(T, dt)
+        setattr(so, k, out[k].ctypes.data)
+    off = np.ascontiguousarray(wl.trace_off, np.int32)
+    st = L.ora_sim(C.byref(ctx.cfg), C.byref(ctx.table), off.ctypes.data, j0, j1,
+                   int(wl.sim_iters if iters is None else iters), C.byref(so))
+    out["status"] = int(st)
+    return out

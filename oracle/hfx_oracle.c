@@ -1,0 +1,559 @@
+/*
+ * hfx_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, single-threaded statement of what the scheduler hot path
+ * computes, written from the paper's Sec. 3.3.1 (dispatching steps 2-4, slack,
+ * maturity time, Eq. 3, the P-stage / D-stage variants) and the Problem
+ * Definition (events, Eq. 2).  The paper's Algorithm 1 is not printed in the
+ * paper body, so the steps below follow its prose in the paper's order and
+ * notation; every reading of a point the paper leaves open is marked
+ * "reading:".  Integer nanoseconds throughout, one 128-bit product, a library
+ * qsort on explicit tuples, no blocking or fusion.
+ *
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg use this
+ * file.  It shares no code, header, table or constant with the CUDA library.
+ *
+ * Parity status: the arithmetic below is pinned by hand-worked values, the
+ * closed form of Eq. 3 in exact rationals, invariants, brute force on tiny
+ * inputs and a pure-Python restatement (tests/test_oracle_*.py).  Against the
+ * behaviour of the paper's own system it is "parity unpinned": the paper
+ * prints no scheduler trace or worked numeric example.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef __int128 i128;
+
+#define ORA_INF INT64_MAX
+#define ORA_TIME_MAX ((int64_t)1 << 62)
+#define ORA_SLACK_MAX (((int64_t)1 << 39) - 1)
+#define ORA_SLACK_MIN (-((int64_t)1 << 39))
+#define ORA_MAX_LEN (1 << 24)
+
+enum { ST_QUEUED = 0, ST_RUNNING = 1, ST_DONE = 2, ST_REJECTED = 3 };
+enum { MODE_COLOCATED = 0, MODE_PREFILL = 1, MODE_DECODE = 2 };
+enum { BUDGET_SAFE = 0, BUDGET_CAP_ONLY = 1 };
+enum { PH_RUNNING = 0, PH_QUEUED = 1, PH_INACTIVE = 3 };
+enum { BAD_REPLICA = 1, BAD_CLASS = 2, BAD_LEN = 4 };
+enum { FLAG_COMMIT = 1 };
+
+typedef struct { int64_t c0, c1, c2, d0, d1, d2; } ora_model;
+typedef struct { int64_t ttft, tpot; int32_t prio, pad; } ora_class;
+typedef struct { int32_t mode, token_cap, batch_cap; } ora_replica;
+
+typedef struct {
+  ora_model model;
+  const ora_class *classes;
+  int32_t n_classes;
+  const ora_replica *replicas;
+  int32_t n_replicas;
+  int32_t budget_mode;
+  int32_t weight_max;
+} ora_config;
+
+typedef struct {
+  int64_t n;
+  const int32_t *replica_id;
+  const uint8_t *class_id;
+  uint8_t *state;
+  const int32_t *prompt_len;
+  const int32_t *output_len;
+  int32_t *gen;
+  const int64_t *arrival;
+  int64_t *first_token;
+  int64_t *last_token;
+  int64_t *finish;
+  const int32_t *req_id;
+  const int32_t *weight;
+} ora_table;
+
+typedef struct {
+  int64_t *slack;      /* [n] */
+  int64_t *pred_ttft;  /* [n] */
+  int64_t *pred_tpot;  /* [n] */
+  uint64_t *key;       /* [n] */
+  int32_t *order;      /* [n] */
+  int32_t *seg_off;    /* [R+1] */
+  uint8_t *admit;      /* [n] */
+  int32_t *admitted_rows; /* [n] */
+  int64_t *budget;     /* [R] */
+  int64_t *e_d;        /* [R] */
+  int32_t *n_run;      /* [R] */
+  int64_t *sum_kv;     /* [R] */
+  int64_t *adm_cost;   /* [R] */
+  int32_t *adm_count;  /* [R] */
+  int64_t *maturity_next; /* [R] */
+  /* extra, for the pins */
+  int64_t *epmax;      /* [R] largest safe prefill latency (ORA_INF, or -1)  */
+  int64_t *n_safe;     /* [R] */
+} ora_step_out;
+
+/* ---- latency predictor (Sec. 3.3.1; quadratic prefill model of the cited
+ *      work, linear when c2 = 0; decode latency from the running batch) ------ */
+int64_t ora_Ep(const ora_model *m, int64_t t) { return m->c0 + m->c1 * t + m->c2 * t * t; }
+int64_t ora_Ed(const ora_model *m, int64_t b, int64_t kv) { return m->d0 + m->d1 * b + m->d2 * kv; }
+
+static int64_t clamp_slack(int64_t s) {
+  if (s < ORA_SLACK_MIN) return ORA_SLACK_MIN;
+  if (s > ORA_SLACK_MAX) return ORA_SLACK_MAX;
+  return s;
+}
+
+/* 64-bit priority key: replica<16> | phase<2> | prio<6> | (clamp(slack)+2^39)<40>.
+ * Smaller = more urgent (in-flight first, priority 0 highest, least remaining
+ * SLO budget first). */
+uint64_t ora_key(int32_t replica, int32_t phase, int32_t prio, int64_t slack) {
+  uint64_t f = (uint64_t)(clamp_slack(slack) + ((int64_t)1 << 39));
+  return ((uint64_t)replica << 48) | ((uint64_t)phase << 46) | ((uint64_t)prio << 40) | f;
+}
+
+/* Largest prefill latency E_p that keeps the worst-case TTFT bound of
+ * Sec. 3.3.1: a request arriving right after this dispatch waits one maturity
+ * time plus its own prefill, 2*E_p + k*E_d <= TTFT with k = E_p/(TPOT - E_d)
+ * real, i.e. E_p*(2*TPOT - E_d)/(TPOT - E_d) <= TTFT.  Returns ORA_INF when no
+ * TTFT bound applies, -1 when TPOT <= E_d (no slack can accumulate; reading:
+ * nothing is safe). `decoding` = the instance has a running batch with a
+ * bounded TPOT. */
+int64_t ora_epmax(int64_t min_ttft, int decoding, int64_t min_tpot, int64_t e_d) {
+  if (min_ttft == ORA_INF) return ORA_INF;
+  if (!decoding) return min_ttft / 2;            /* E_d = 0: 2*E_p <= TTFT    */
+  if (min_tpot <= e_d) return -1;
+  i128 num = (i128)min_ttft * (i128)(min_tpot - e_d);
+  i128 den = (i128)2 * min_tpot - e_d;
+  return (int64_t)(num / den);
+}
+
+/* Eq. 3 solved on the general E_p: the largest n in [0, token_cap] with
+ * E_p(n) <= epmax, 0 if there is none.  E_p is non-decreasing for non-negative
+ * coefficients, so a binary search finds it. */
+int64_t ora_nsafe(const ora_model *m, int64_t epmax, int64_t token_cap) {
+  if (epmax == ORA_INF) return token_cap;
+  if (ora_Ep(m, 0) > epmax) return 0;
+  int64_t lo = 0, hi = token_cap;              /* E_p(lo) <= epmax always      */
+  while (lo < hi) {
+    int64_t mid = lo + (hi - lo + 1) / 2;
+    if (ora_Ep(m, mid) <= epmax) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+typedef struct {
+  int32_t phase, prio;
+  int64_t cslack;     /* clamped slack */
+  int32_t req_id;
+  int64_t row;        /* global row index */
+} sort_tuple;
+
+static int cmp_tuple(const void *pa, const void *pb) {
+  const sort_tuple *a = (const sort_tuple *)pa, *b = (const sort_tuple *)pb;
+  if (a->phase != b->phase) return a->phase < b->phase ? -1 : 1;
+  if (a->prio != b->prio) return a->prio < b->prio ? -1 : 1;
+  if (a->cslack != b->cslack) return a->cslack < b->cslack ? -1 : 1;
+  if (a->req_id != b->req_id) return a->req_id < b->req_id ? -1 : 1;
+  return 0;
+}
+
+static int cmp_i64(const void *pa, const void *pb) {
+  int64_t a = *(const int64_t *)pa, b = *(const int64_t *)pb;
+  return a < b ? -1 : (a > b ? 1 : 0);
+}
+
+static int row_valid(const ora_config *c, const ora_table *t, int64_t i, uint32_t *status) {
+  int ok = 1;
+  if (t->class_id[i] >= c->n_classes) { *status |= BAD_CLASS; ok = 0; }
+  if (t->prompt_len[i] < 0 || t->prompt_len[i] > ORA_MAX_LEN || t->gen[i] < 0 || t->gen[i] > ORA_MAX_LEN) {
+    *status |= BAD_LEN; ok = 0;
+  }
+  return ok;
+}
+
+/* result of the commit of one replica */
+enum { CM_WORKED = 0, CM_JUMPED = 1, CM_STUCK = 2 };
+
+/*
+ * One scheduling iteration of one replica over the rows `rows[0..m)` (global
+ * row indices).  `r` selects the replica configuration; `key_replica` is the
+ * replica field of the key; `order_base` is where this replica's order starts.
+ * Steps are numbered as the dispatching steps of Sec. 3.3.1 are refined here.
+ */
+static int step_replica(const ora_config *c, const ora_table *t, int32_t r, int32_t key_replica,
+                        const int64_t *rows, int64_t m, int64_t order_base, int64_t *now_p,
+                        int64_t *mat_p, const ora_step_out *o, uint32_t flags, uint32_t *status) {
+  const ora_model *M = &c->model;
+  const ora_replica *cfg = &c->replicas[r];
+  const int64_t now = *now_p, mat = *mat_p;
+  int32_t *phase = (int32_t *)malloc(sizeof(int32_t) * (size_t)(m + 1));
+  int64_t *cost = (int64_t *)malloc(sizeof(int64_t) * (size_t)(m + 1));
+  sort_tuple *tup = (sort_tuple *)malloc(sizeof(sort_tuple) * (size_t)(m + 1));
+
+  /* 1. visibility and phase: a request exists for the scheduler once it has
+   *    arrived; in-flight requests are phase 0, the visible queue phase 1. */
+  for (int64_t j = 0; j < m; j++) {
+    int64_t i = rows[j];
+    int ph = PH_INACTIVE;
+    if (row_valid(c, t, i, status)) {
+      if (t->state[i] == ST_RUNNING) ph = PH_RUNNING;
+      else if (t->state[i] == ST_QUEUED && t->arrival[i] <= now) ph = PH_QUEUED;
+    }
+    phase[j] = ph;
+  }
+
+  /* 2. aggregates of the running batch and the strictest SLOs ("use current
+   *    running batch to estimate a constant E_d"; strictest TTFT of the queue;
+   *    strictest TPOT among in-flight).  reading: sum_kv = sum of prompt_len +
+   *    gen over running rows; classes without a bound are skipped in a minimum. */
+  int64_t n_run = 0, sum_kv = 0, min_tpot = ORA_INF, min_ttft = ORA_INF, min_tpot_q = ORA_INF;
+  for (int64_t j = 0; j < m; j++) {
+    int64_t i = rows[j];
+    if (phase[j] == PH_RUNNING) {
+      const ora_class *k = &c->classes[t->class_id[i]];
+      n_run += 1;
+      sum_kv += (int64_t)t->prompt_len[i] + t->gen[i];
+      if (k->tpot > 0 && k->tpot < min_tpot) min_tpot = k->tpot;
+    } else if (phase[j] == PH_QUEUED) {
+      const ora_class *k = &c->classes[t->class_id[i]];
+      if (k->ttft > 0 && k->ttft < min_ttft) min_ttft = k->ttft;
+      if (k->tpot > 0 && k->tpot < min_tpot_q) min_tpot_q = k->tpot;
+    }
+  }
+  /* a P-stage instance starts from an empty instance: it has no decode batch */
+  const int64_t n_eff = cfg->mode == MODE_PREFILL ? 0 : n_run;
+  const int64_t kv_eff = cfg->mode == MODE_PREFILL ? 0 : sum_kv;
+  const int64_t tpot_eff = cfg->mode == MODE_PREFILL ? ORA_INF : min_tpot;
+  const int64_t e_d = n_eff > 0 ? ora_Ed(M, n_eff, kv_eff) : 0;
+
+  /* 3. safe budget (dispatching step 2).  Before maturity the instance is
+   *    protected: budget 0. */
+  int64_t epmax = ORA_INF, n_safe = 0, budget = 0;
+  const int64_t cap_left = cfg->token_cap - n_eff > 0 ? cfg->token_cap - n_eff : 0;
+  if (cfg->mode == MODE_DECODE) {
+    /* D-stage: strictest TPOT among in-flight, else of the queue of prefilled
+     * requests.  reading: the budget is the decode-step latency still
+     * available, E_d(batch) <= TPOT, and a request costs d1 + d2*kv of it. */
+    int64_t T = (n_run > 0 && min_tpot < ORA_INF) ? min_tpot : min_tpot_q;
+    if (c->budget_mode == BUDGET_CAP_ONLY || T == ORA_INF) budget = ORA_INF;
+    else {
+      int64_t room = T - ora_Ed(M, n_run, sum_kv);
+      budget = room > 0 ? room : 0;
+    }
+    epmax = ORA_INF; n_safe = 0;
+  } else {
+    if (c->budget_mode == BUDGET_CAP_ONLY) { epmax = ORA_INF; n_safe = cfg->token_cap; }
+    else {
+      epmax = ora_epmax(min_ttft, n_eff > 0 && tpot_eff < ORA_INF, tpot_eff, e_d);
+      n_safe = ora_nsafe(M, epmax, cfg->token_cap);
+    }
+    budget = n_safe < cap_left ? n_safe : cap_left;
+  }
+  if (now < mat) budget = 0;
+
+  /* 4. per-row predicted TTFT / TPOT, slack ("remaining SLO budget"), cost;
+   * 5. priority and key. */
+  const int64_t start = now > mat ? now : mat;
+  for (int64_t j = 0; j < m; j++) {
+    int64_t i = rows[j];
+    int64_t sl = 0, pt = 0, pp = 0, cst = 0;
+    int32_t prio = 63;
+    if (phase[j] != PH_INACTIVE) {
+      const ora_class *k = &c->classes[t->class_id[i]];
+      const int64_t kv_i = (int64_t)t->prompt_len[i] + t->gen[i];
+      if (c->weight_max > 0) {
+        int64_t p = (int64_t)c->weight_max - t->weight[i];
+        prio = (int32_t)(p < 0 ? 0 : (p > 62 ? 62 : p));
+      } else prio = k->prio;
+      if (phase[j] == PH_RUNNING) {
+        /* accumulated slack of an in-flight request, net of the coming step:
+         * its next-token deadline is first_token + (gen+1)*TPOT */
+        pp = e_d;
+        pt = t->first_token[i] - t->arrival[i];
+        sl = k->tpot > 0 ? t->first_token[i] + ((int64_t)t->gen[i] + 1) * k->tpot - now - e_d : ORA_SLACK_MAX;
+        cst = 0;
+      } else if (cfg->mode == MODE_DECODE) {
+        /* prefilled request waiting to be migrated to this D-stage instance */
+        pp = ora_Ed(M, n_eff + 1, kv_eff + kv_i);
+        pt = t->first_token[i] - t->arrival[i];
+        sl = k->tpot > 0 ? t->first_token[i] + ((int64_t)t->gen[i] + 1) * k->tpot - start - pp : ORA_SLACK_MAX;
+        cst = M->d1 + M->d2 * kv_i;
+      } else {
+        /* queued request: earliest start is max(now, maturity) */
+        pt = (start - t->arrival[i]) + ora_Ep(M, t->prompt_len[i]);
+        pp = ora_Ed(M, n_eff + 1, kv_eff + kv_i);
+        sl = k->ttft > 0 ? k->ttft - pt : ORA_SLACK_MAX;
+        cst = t->prompt_len[i];
+      }
+    }
+    cost[j] = cst;
+    o->slack[i] = sl;
+    if (o->pred_ttft) o->pred_ttft[i] = pt;
+    if (o->pred_tpot) o->pred_tpot[i] = pp;
+    tup[j].phase = phase[j];
+    tup[j].prio = prio;
+    tup[j].cslack = phase[j] == PH_INACTIVE ? ORA_SLACK_MAX : clamp_slack(sl);
+    tup[j].req_id = t->req_id[i];
+    tup[j].row = j; /* local index for now */
+    if (o->key) o->key[i] = ora_key(key_replica, phase[j], prio, tup[j].cslack);
+  }
+
+  /* order within the replica: in-flight first, then by priority, then by
+   * remaining slack; reading: req_id breaks ties, inactive rows last. */
+  qsort(tup, (size_t)m, sizeof(sort_tuple), cmp_tuple);
+
+  /* 6. admission (dispatching step 3): the most urgent requests that fit.
+   *    reading: a request that could not fit even alone is skipped; among the
+   *    rest admission is the longest prefix whose running totals stay within
+   *    the budget and the batch cap (totals keep growing after a failure). */
+  int64_t s_cost = 0, s_count = 0, adm_cost = 0, adm_count = 0, adm_kv = 0;
+  for (int64_t q = 0; q < m; q++) {
+    int64_t j = tup[q].row, i = rows[j];
+    o->order[order_base + q] = (int32_t)i;
+    if (o->admitted_rows) o->admitted_rows[order_base + q] = -1;
+    uint8_t a = 0;
+    if (phase[j] == PH_RUNNING) a = 1;
+    else if (phase[j] == PH_QUEUED && cost[j] <= budget) {
+      s_cost += cost[j];
+      s_count += 1;
+      if (s_cost <= budget && (cfg->batch_cap == 0 || n_eff + s_count <= cfg->batch_cap)) {
+        a = 1;
+        if (o->admitted_rows) o->admitted_rows[order_base + adm_count] = (int32_t)i;
+        adm_cost += cost[j];
+        adm_count += 1;
+        adm_kv += (int64_t)t->prompt_len[i] + t->gen[i];
+      }
+    }
+    o->admit[i] = a;
+  }
+
+  /* 7. maturity time after the dispatch (dispatching step 4). */
+  int64_t mat_next = mat;
+  int64_t lp = 0;
+  if (cfg->mode == MODE_DECODE) {
+    /* end of the next decode iteration of the enlarged batch; reading: before
+     * maturity an iteration is still in flight and its end stands */
+    if (now >= mat && n_run + adm_count > 0) mat_next = now + ora_Ed(M, n_run + adm_count, sum_kv + adm_kv);
+  } else if (adm_count > 0) {
+    lp = ora_Ep(M, adm_cost);   /* reading: E_p of a batch = model at its total tokens */
+    if (cfg->mode == MODE_PREFILL) mat_next = now + lp;  /* completion of the batch */
+    else {
+      /* Maturity = E_p + k*E_d, k decode iterations accumulate E_p of slack;
+       * reading: k is rounded up here, and is 0 without a bounded running batch */
+      i128 k = 0;
+      if (n_eff > 0 && tpot_eff < ORA_INF && tpot_eff > e_d) k = ((i128)lp + (tpot_eff - e_d) - 1) / (tpot_eff - e_d);
+      i128 v = (i128)now + lp + k * e_d;
+      mat_next = v > ORA_TIME_MAX ? ORA_TIME_MAX : (int64_t)v;
+    }
+  }
+
+  o->budget[r] = budget;
+  if (o->e_d) o->e_d[r] = e_d;
+  if (o->n_run) o->n_run[r] = (int32_t)n_run;
+  if (o->sum_kv) o->sum_kv[r] = sum_kv;
+  o->adm_cost[r] = adm_cost;
+  o->adm_count[r] = (int32_t)adm_count;
+  o->maturity_next[r] = mat_next;
+  if (o->epmax) o->epmax[r] = epmax;
+  if (o->n_safe) o->n_safe[r] = n_safe;
+
+  /* 8. commit: the iteration happens.  Colocated: the new prefill batch runs
+   *    first (prefill preempts ongoing decoding), then one decode iteration of
+   *    the batch that was running. */
+  int result = CM_WORKED;
+  if (flags & FLAG_COMMIT) {
+    int worked;
+    int64_t t1 = now, t2 = now;
+    if (cfg->mode == MODE_COLOCATED) {
+      worked = adm_count > 0 || n_run > 0;
+      t1 = now + (adm_count > 0 ? lp : 0);
+      t2 = t1 + (n_run > 0 ? e_d : 0);
+    } else if (cfg->mode == MODE_PREFILL) {
+      worked = adm_count > 0;
+      t1 = t2 = now + (adm_count > 0 ? lp : 0);
+    } else {
+      worked = now >= mat && n_run + adm_count > 0;
+      t1 = now;
+      t2 = worked ? mat_next : now;
+    }
+    int64_t next_arrival = ORA_INF;
+    for (int64_t j = 0; j < m; j++) {
+      int64_t i = rows[j];
+      if (phase[j] == PH_RUNNING) {
+        if (cfg->mode == MODE_PREFILL) continue;   /* a P-stage instance does not decode */
+        if (cfg->mode == MODE_DECODE && !worked) continue;
+        t->gen[i] += 1;
+        t->last_token[i] = t2;
+        if ((int64_t)t->gen[i] + 1 >= t->output_len[i]) { t->state[i] = ST_DONE; t->finish[i] = t2; }
+      } else if (phase[j] == PH_QUEUED) {
+        if (o->admit[i]) {
+          t->state[i] = ST_RUNNING;
+          if (cfg->mode == MODE_DECODE) {
+            t->gen[i] += 1;
+            t->last_token[i] = t2;
+            if ((int64_t)t->gen[i] + 1 >= t->output_len[i]) { t->state[i] = ST_DONE; t->finish[i] = t2; }
+          } else {
+            t->gen[i] = 0;
+            t->first_token[i] = t1;
+            t->last_token[i] = t1;
+            if (t->output_len[i] <= 1) { t->state[i] = ST_DONE; t->finish[i] = t1; }
+          }
+        } else if (cfg->mode != MODE_DECODE && t->prompt_len[i] > cfg->token_cap) {
+          t->state[i] = ST_REJECTED;   /* reading: an oversize prompt can never be served */
+        }
+      } else if (t->state[i] == ST_QUEUED && t->arrival[i] > now && row_valid(c, t, i, status)) {
+        if (t->arrival[i] < next_arrival) next_arrival = t->arrival[i];
+      }
+    }
+    if (worked) { *now_p = t2; result = CM_WORKED; }
+    else {
+      /* idle: jump to the next event (maturity or the next arrival), if any */
+      int64_t ev = ORA_INF;
+      if (mat > now) ev = mat;
+      if (next_arrival < ev) ev = next_arrival;
+      if (ev == ORA_INF) result = CM_STUCK;
+      else { *now_p = ev; result = CM_JUMPED; }
+    }
+    *mat_p = mat_next;
+  }
+  free(phase); free(cost); free(tup);
+  return result;
+}
+
+/*
+ * One scheduling iteration over the whole table.  now[R], maturity[R] are read,
+ * and written when flags has FLAG_COMMIT.  Returns the status bits.
+ */
+uint32_t ora_step(const ora_config *c, const ora_table *t, int64_t *now, int64_t *maturity,
+                  const ora_step_out *o, uint32_t flags) {
+  const int32_t R = c->n_replicas;
+  uint32_t status = 0;
+  int64_t *cnt = (int64_t *)calloc((size_t)R + 2, sizeof(int64_t));
+  for (int64_t i = 0; i < t->n; i++) {
+    int32_t r = t->replica_id[i];
+    if (r < 0 || r >= R) { status |= BAD_REPLICA; r = R; }
+    cnt[r + 1]++;
+  }
+  for (int32_t r = 0; r <= R; r++) cnt[r + 1] += cnt[r];
+  for (int32_t r = 0; r <= R; r++) o->seg_off[r] = (int32_t)cnt[r];
+  int64_t *rows = (int64_t *)malloc(sizeof(int64_t) * (size_t)(t->n + 1));
+  int64_t *fill = (int64_t *)malloc(sizeof(int64_t) * ((size_t)R + 2));
+  memcpy(fill, cnt, sizeof(int64_t) * ((size_t)R + 2));
+  for (int64_t i = 0; i < t->n; i++) {
+    int32_t r = t->replica_id[i];
+    if (r < 0 || r >= R) r = R;
+    rows[fill[r]++] = i;
+  }
+  for (int32_t r = 0; r < R; r++)
+    step_replica(c, t, r, r, rows + cnt[r], cnt[r + 1] - cnt[r], cnt[r], &now[r], &maturity[r], o, flags, &status);
+  /* rows bound to no replica: inactive, listed after every replica by req_id */
+  {
+    int64_t m = cnt[R + 1] - cnt[R];
+    sort_tuple *tup = (sort_tuple *)malloc(sizeof(sort_tuple) * (size_t)(m + 1));
+    for (int64_t j = 0; j < m; j++) {
+      int64_t i = rows[cnt[R] + j];
+      tup[j].phase = PH_INACTIVE; tup[j].prio = 63; tup[j].cslack = ORA_SLACK_MAX;
+      tup[j].req_id = t->req_id[i]; tup[j].row = i;
+      o->slack[i] = 0;
+      if (o->pred_ttft) o->pred_ttft[i] = 0;
+      if (o->pred_tpot) o->pred_tpot[i] = 0;
+      if (o->key) o->key[i] = ora_key(R & 0xFFFF, PH_INACTIVE, 63, ORA_SLACK_MAX);
+      o->admit[i] = 0;
+    }
+    qsort(tup, (size_t)m, sizeof(sort_tuple), cmp_tuple);
+    for (int64_t j = 0; j < m; j++) {
+      o->order[cnt[R] + j] = (int32_t)tup[j].row;
+      if (o->admitted_rows) o->admitted_rows[cnt[R] + j] = -1;
+    }
+    free(tup);
+  }
+  free(cnt); free(rows); free(fill);
+  return status;
+}
+
+typedef struct {
+  int32_t *iters_executed, *finished, *rejected, *attained;
+  int64_t *ttft_p50, *ttft_p99, *tpot_p50, *tpot_p99, *now;
+} ora_sim_out;
+
+static int64_t nearest_rank(int64_t *v, int64_t n, int p) {
+  if (n == 0) return -1;
+  qsort(v, (size_t)n, sizeof(int64_t), cmp_i64);
+  int64_t k = (p * n + 99) / 100;   /* ceil(p*n/100) */
+  if (k < 1) k = 1;
+  return v[k - 1];
+}
+
+/*
+ * Discrete-event simulation of traces [j0, j1): trace j = rows trace_off[j] ..
+ * trace_off[j+1]-1 on replica j (colocated).  Events are arrivals and iteration
+ * completions (Problem Definition).  Each iteration is one step + commit at
+ * the replica's clock.  Metrics: attainment numerator (Eq. 2; unfinished and
+ * rejected requests count as misses), TTFT = first token - arrival, TPOT =
+ * floor((last token - first token)/(output_len - 1)), nearest-rank percentiles.
+ */
+uint32_t ora_sim(const ora_config *c, const ora_table *t, const int32_t *trace_off, int32_t j0,
+                 int32_t j1, int32_t iters, const ora_sim_out *so) {
+  uint32_t status = 0;
+  int64_t max_m = 0;
+  for (int32_t j = j0; j < j1; j++) {
+    int64_t m = trace_off[j + 1] - trace_off[j];
+    if (m > max_m) max_m = m;
+  }
+  int64_t *rows = (int64_t *)malloc(sizeof(int64_t) * (size_t)(max_m + 1));
+  int64_t *va = (int64_t *)malloc(sizeof(int64_t) * (size_t)(max_m + 1));
+  int64_t *vb = (int64_t *)malloc(sizeof(int64_t) * (size_t)(max_m + 1));
+  /* scratch outputs of the step, indexed by global row / by replica */
+  ora_step_out o;
+  memset(&o, 0, sizeof(o));
+  const int32_t R = c->n_replicas;
+  o.slack = (int64_t *)malloc(sizeof(int64_t) * (size_t)(t->n + 1));
+  o.order = (int32_t *)malloc(sizeof(int32_t) * (size_t)(t->n + 1));
+  o.admit = (uint8_t *)malloc((size_t)(t->n + 1));
+  o.budget = (int64_t *)malloc(sizeof(int64_t) * (size_t)R);
+  o.adm_cost = (int64_t *)malloc(sizeof(int64_t) * (size_t)R);
+  o.adm_count = (int32_t *)malloc(sizeof(int32_t) * (size_t)R);
+  o.maturity_next = (int64_t *)malloc(sizeof(int64_t) * (size_t)R);
+  for (int32_t j = j0; j < j1; j++) {
+    const int64_t b = trace_off[j], m = trace_off[j + 1] - trace_off[j];
+    for (int64_t q = 0; q < m; q++) {
+      int64_t i = b + q;
+      rows[q] = i;
+      t->state[i] = ST_QUEUED; t->gen[i] = 0;
+      t->first_token[i] = -1; t->last_token[i] = -1; t->finish[i] = -1;
+    }
+    int64_t now = 0, mat = 0;
+    int32_t executed = 0;
+    for (int32_t it = 0; it < iters; it++) {
+      int res = step_replica(c, t, j, j, rows, m, b, &now, &mat, &o, FLAG_COMMIT, &status);
+      if (res == CM_STUCK) break;
+      executed++;
+    }
+    int32_t fin = 0, rej = 0, att = 0;
+    int64_t na = 0, nb = 0;
+    for (int64_t q = 0; q < m; q++) {
+      int64_t i = b + q;
+      if (t->class_id[i] >= c->n_classes) continue;
+      const ora_class *k = &c->classes[t->class_id[i]];
+      if (t->state[i] == ST_REJECTED) rej++;
+      if (t->state[i] == ST_RUNNING || t->state[i] == ST_DONE) va[na++] = t->first_token[i] - t->arrival[i];
+      if (t->state[i] == ST_DONE) {
+        fin++;
+        int64_t ttft = t->first_token[i] - t->arrival[i];
+        int64_t tpot = t->output_len[i] > 1 ? (t->last_token[i] - t->first_token[i]) / (t->output_len[i] - 1) : 0;
+        if (t->output_len[i] > 1) vb[nb++] = tpot;
+        if ((k->ttft <= 0 || ttft <= k->ttft) && (k->tpot <= 0 || tpot <= k->tpot)) att++;
+      }
+    }
+    so->iters_executed[j] = executed;
+    so->finished[j] = fin;
+    so->rejected[j] = rej;
+    so->attained[j] = att;
+    so->ttft_p50[j] = nearest_rank(va, na, 50);
+    so->ttft_p99[j] = nearest_rank(va, na, 99);
+    so->tpot_p50[j] = nearest_rank(vb, nb, 50);
+    so->tpot_p99[j] = nearest_rank(vb, nb, 99);
+    if (so->now) so->now[j] = now;
+  }
+  free(rows); free(va); free(vb);
+  free(o.slack); free(o.order); free(o.admit); free(o.budget); free(o.adm_cost); free(o.adm_count);
+  free(o.maturity_next);
+  return status;
+}

@@ -1,0 +1,246 @@
+"""The oracle against what the paper and the mathematics fix: hand-worked values
+(tests/golden/pins.txt), the closed form of Eq. 3 in exact rationals, single-request
+closed forms of the simulator and a two-request case worked out by hand."""
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from helpers import MS, load_pins, make_wl
+
+PINS = load_pins()
+M = gen.DEFAULT_MODEL
+C200 = [(200 * MS, 30 * MS, 0)]
+
+
+def test_prefill_model_values():
+    for t in (16, 1000, 8192, 32768, 131072, 1281, 1282):
+        assert oracle.Ep(M, t) == PINS[f"Ep_{t}"]
+    assert oracle.Ed(M, 80, 64000) == PINS["Ed_80_64000"]
+
+
+def test_key_layout():
+    assert oracle.key(3, 1, 0, PINS["slack_queued"]) == PINS["key_queued"]
+    assert oracle.key(0, 0, 0, -1) & ((1 << 40) - 1) == PINS["key_low40_slack_minus1"]
+    # saturation of the 40-bit slack field
+    assert oracle.key(0, 0, 0, -(1 << 50)) & ((1 << 40) - 1) == 0
+    assert oracle.key(0, 0, 0, 1 << 50) & ((1 << 40) - 1) == (1 << 40) - 1
+    # field order: replica > phase > prio > slack
+    assert oracle.key(1, 0, 0, oracle.SLACK_MIN) > oracle.key(0, 3, 63, oracle.SLACK_MAX)
+    assert oracle.key(0, 1, 0, oracle.SLACK_MIN) > oracle.key(0, 0, 62, oracle.SLACK_MAX)
+    assert oracle.key(0, 1, 1, oracle.SLACK_MIN) > oracle.key(0, 1, 0, oracle.SLACK_MAX)
+
+
+def test_epmax_and_nsafe_pins():
+    ed = PINS["Ed_80_64000"]
+    ep = oracle.epmax(200 * MS, True, 30 * MS, ed)
+    assert ep == PINS["Epmax_busy"]
+    assert oracle.nsafe(M, ep, 8192) == PINS["nsafe_busy"]
+    lin = (M[0], M[1], 0) + M[3:]
+    assert oracle.nsafe(lin, ep, 8192) == PINS["nsafe_linear"]
+    assert oracle.epmax(200 * MS, False, oracle.INF, 0) == PINS["Epmax_idle"]
+    assert oracle.nsafe(M, PINS["Epmax_idle"], 8192) == PINS["nsafe_idle"]
+    # no TTFT bound in the queue -> capacity only; TPOT <= E_d -> nothing is safe
+    assert oracle.epmax(oracle.INF, True, 30 * MS, ed) == oracle.INF
+    assert oracle.nsafe(M, oracle.INF, 777) == 777
+    assert oracle.epmax(200 * MS, True, ed, ed) == -1
+    assert oracle.nsafe(M, -1, 8192) == 0
+    assert oracle.nsafe(M, M[0] - 1, 8192) == 0 and oracle.nsafe(M, M[0], 8192) == 0
+    assert oracle.nsafe(M, oracle.Ep(M, 1), 8192) == 1
+
+
+def test_eq3_closed_form_in_exact_rationals():
+    """With the paper's linear model E_p = a + b n, the budget must equal floor(Eq. 3)."""
+    rng = np.random.default_rng(7)
+    for _ in range(3000):
+        a = int(rng.integers(0, 20_000_000))
+        b = int(rng.integers(1, 200_000))
+        lin = (a, b, 0, 8_000_000, 100_000, 20)
+        tpot = int(rng.integers(1 * MS, 300 * MS))
+        ttft = int(rng.integers(1 * MS, 20_000 * MS))
+        ed = int(rng.integers(0, tpot))          # TPOT > E_d
+        cap = 1 << 24
+        rhs = Fraction((tpot - ed) * ttft, (2 * tpot - ed) * b) - Fraction(a, b)   # Eq. 3
+        ep = oracle.epmax(ttft, True, tpot, ed)
+        got = oracle.nsafe(lin, ep, cap)
+        want = max(0, min(cap, rhs.numerator // rhs.denominator)) if rhs >= 0 else 0
+        assert got == want, (a, b, tpot, ttft, ed)
+
+
+def test_eq3_quadratic_generalisation_brackets():
+    rng = np.random.default_rng(8)
+    for _ in range(500):
+        tpot = int(rng.integers(10 * MS, 300 * MS)); ttft = int(rng.integers(50 * MS, 20_000 * MS))
+        ed = int(rng.integers(0, tpot))
+        ep = oracle.epmax(ttft, True, tpot, ed)
+        # E_p (2 TPOT - E_d)/(TPOT - E_d) <= TTFT holds at ep and fails at ep + 1
+        assert Fraction(ep * (2 * tpot - ed), tpot - ed) <= ttft < Fraction((ep + 1) * (2 * tpot - ed), tpot - ed)
+        n = oracle.nsafe(M, ep, 16384)
+        if n == 0:
+            assert oracle.Ep(M, 1) > ep
+        else:
+            assert oracle.Ep(M, n) <= ep
+        if n < 16384:
+            assert oracle.Ep(M, n + 1) > ep
+
+
+def test_queued_slack_closed_form_single_row():
+    wl = make_wl([dict(prompt_len=1000, arrival_ns=0)], C200, replicas=[(gen.COLOCATED, 8192, 0)] * 4,
+                 now=[10 * MS] * 4, maturity=[0] * 4)
+    wl.table["replica_id"][0] = 3
+    o = oracle.step(wl)
+    assert o["slack"][0] == PINS["slack_queued"]
+    assert o["key"][0] == PINS["key_queued"]
+    assert o["pred_ttft"][0] == 10 * MS + PINS["Ep_1000"]
+    assert o["pred_tpot"][0] == 8_000_000 + 100_000 + 20 * 1000
+    assert list(o["seg_off"]) == [0, 0, 0, 0, 1]
+    # maturity in the future delays the earliest start
+    wl.maturity[3] = 25 * MS
+    o = oracle.step(wl)
+    assert o["slack"][0] == 200 * MS - 25 * MS - PINS["Ep_1000"]
+    assert o["admit"][0] == 0 and o["budget"][3] == 0 and o["adm_count"][3] == 0
+
+
+def _busy_replica(queued_prompt):
+    rows = [dict(state=gen.RUNNING, prompt_len=700, gen=100, first_token_ns=0, arrival_ns=-MS, req_id=i)
+            for i in range(80)]                      # n_run = 80, sum_kv = 80 * 800 = 64000
+    rows.append(dict(prompt_len=queued_prompt, arrival_ns=0, req_id=1000))
+    return make_wl(rows, C200, now=[5 * MS], maturity=[0])
+
+
+def test_busy_replica_budget_and_maturity():
+    wl = _busy_replica(1281)
+    o = oracle.step(wl)
+    assert o["n_run"][0] == 80 and o["sum_kv"][0] == 64000
+    assert o["e_d"][0] == PINS["Ed_80_64000"]
+    assert o["epmax"][0] == PINS["Epmax_busy"] and o["n_safe"][0] == PINS["nsafe_busy"]
+    assert o["budget"][0] == PINS["nsafe_busy"]
+    assert o["admit"][80] == 1 and o["adm_count"][0] == 1 and o["adm_cost"][0] == 1281
+    assert o["maturity_next"][0] - wl.now[0] == PINS["maturity_busy_delta"]
+    # one token more does not fit
+    o = oracle.step(_busy_replica(1282))
+    assert o["admit"][80] == 0 and o["adm_count"][0] == 0 and o["maturity_next"][0] == 0
+    # running rows: slack = first_token + (gen+1) TPOT - now - E_d
+    assert o["slack"][0] == 0 + 101 * 30 * MS - 5 * MS - PINS["Ed_80_64000"]
+    assert o["pred_tpot"][0] == PINS["Ed_80_64000"] and o["pred_ttft"][0] == MS
+    assert all(o["admit"][:80] == 1)
+
+
+def test_idle_replica_budget():
+    wl = make_wl([dict(prompt_len=2144, arrival_ns=0), dict(prompt_len=2145, arrival_ns=0, req_id=1)],
+                 C200, now=[0])
+    o = oracle.step(wl)
+    assert o["epmax"][0] == PINS["Epmax_idle"] and o["budget"][0] == PINS["nsafe_idle"]
+    # equal slack order: shorter prompt has more slack, so the 2145-token row is more urgent but
+    # cannot fit alone and is skipped; the 2144-token row is admitted
+    assert list(o["order"]) == [1, 0]
+    assert list(o["admit"]) == [1, 0]
+    assert o["maturity_next"][0] == oracle.Ep(M, 2144)   # k = 0 without a running batch
+
+
+def test_simulator_single_request_closed_form():
+    wl = make_wl([dict(prompt_len=1000, output_len=101, arrival_ns=0)], C200, trace_off=[0, 1], sim_iters=500)
+    s = oracle.sim(wl)
+    t = wl.table
+    assert t["first_token_ns"][0] == PINS["sim1_ttft"]
+    assert t["finish_ns"][0] == PINS["sim1_finish"] == PINS["sim1_ttft"] + PINS["sim1_decode_sum"]
+    assert t["last_token_ns"][0] == PINS["sim1_finish"]
+    assert t["state"][0] == gen.DONE and t["gen"][0] == 100
+    assert s["iters_executed"][0] == PINS["sim1_iters"]
+    assert s["tpot_p50"][0] == s["tpot_p99"][0] == PINS["sim1_tpot"]
+    assert s["ttft_p50"][0] == PINS["sim1_ttft"]
+    assert s["attained"][0] == 1 and s["finished"][0] == 1 and s["rejected"][0] == 0
+    assert s["now"][0] == PINS["sim1_finish"]
+
+
+def test_simulator_iteration_limit_and_late_arrival():
+    # the request arrives at 1 s: iteration 0 only advances the clock
+    wl = make_wl([dict(prompt_len=1000, output_len=101, arrival_ns=1000 * MS)], C200, trace_off=[0, 1], sim_iters=50)
+    s = oracle.sim(wl)
+    assert s["iters_executed"][0] == 50
+    assert wl.table["state"][0] == gen.RUNNING and wl.table["gen"][0] == 48   # 1 jump + 1 prefill + 48 decodes
+    assert wl.table["first_token_ns"][0] == 1000 * MS + PINS["sim1_ttft"]
+    assert s["finished"][0] == 0 and s["attained"][0] == 0
+    assert s["ttft_p50"][0] == PINS["sim1_ttft"] and s["tpot_p50"][0] == -1
+
+
+def test_simulator_two_requests_hand_worked():
+    rows = [dict(prompt_len=1000, output_len=3, arrival_ns=0, req_id=0),
+            dict(prompt_len=500, output_len=2, arrival_ns=10 * MS, req_id=1)]
+    # replay iteration by iteration with step+commit to check the intermediate values
+    wl = make_wl(rows, C200, now=[0], maturity=[0])
+    o = oracle.step(wl, commit=True)
+    assert list(o["admit"]) == [1, 0] and wl.now[0] == 47 * MS and wl.maturity[0] == 47 * MS
+    o = oracle.step(wl, commit=True)
+    assert o["epmax"][0] == PINS["sim2_epmax_it1"] and o["n_safe"][0] == PINS["sim2_nsafe_it1"]
+    assert o["slack"][1] == PINS["sim2_slackB_it1"] and o["slack"][0] == PINS["sim2_slackA_it1"]
+    assert list(o["order"]) == [0, 1] and list(o["admit"]) == [1, 1]
+    assert wl.maturity[0] == PINS["sim2_maturity_it1"] and wl.now[0] == PINS["sim2_now_after_it1"]
+    assert wl.table["first_token_ns"][1] == 72_500_000 and wl.table["gen"][0] == 1
+    o = oracle.step(wl, commit=True)
+    assert o["e_d"][0] == 8_230_020 and wl.now[0] == PINS["sim2_finish"]
+    assert list(wl.table["state"]) == [gen.DONE, gen.DONE]
+    # and the same through the simulator
+    wl = make_wl(rows, C200, trace_off=[0, 2], sim_iters=100)
+    s = oracle.sim(wl)
+    t = wl.table
+    assert list(t["finish_ns"]) == [PINS["sim2_finish"]] * 2
+    assert t["first_token_ns"][0] - t["arrival_ns"][0] == PINS["sim2_ttft_A"]
+    assert t["first_token_ns"][1] - t["arrival_ns"][1] == PINS["sim2_ttft_B"]
+    assert s["iters_executed"][0] == PINS["sim2_iters"]
+    assert s["ttft_p50"][0] == PINS["sim2_ttft_A"] and s["ttft_p99"][0] == PINS["sim2_ttft_B"]
+    assert s["tpot_p50"][0] == PINS["sim2_tpot_B"] and s["tpot_p99"][0] == PINS["sim2_tpot_A"]
+    assert s["attained"][0] == 2 and s["finished"][0] == 2
+
+
+def test_prefill_and_decode_stage_budgets():
+    # P-stage: budget from the strictest TTFT of the queue alone (E_d = 0), running rows ignored
+    rows = [dict(state=gen.RUNNING, prompt_len=4000, gen=3, first_token_ns=0, class_id=0, req_id=9),
+            dict(prompt_len=100, class_id=1, req_id=1), dict(prompt_len=100, class_id=0, req_id=2)]
+    cls = [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)]
+    wl = make_wl(rows, cls, replicas=[(gen.PREFILL, 32768, 0)], now=[MS])
+    o = oracle.step(wl)
+    assert o["epmax"][0] == 100 * MS and o["budget"][0] == 2144 and o["e_d"][0] == 0
+    assert o["adm_count"][0] == 2 and o["maturity_next"][0] == MS + oracle.Ep(M, 200)
+    # D-stage: budget = strictest in-flight TPOT - E_d(batch), in ns; cost of a request d1 + d2 kv
+    rows = [dict(state=gen.RUNNING, prompt_len=900, gen=100, first_token_ns=0, class_id=1, req_id=9),
+            dict(prompt_len=500, gen=0, first_token_ns=0, class_id=0, req_id=1),
+            dict(prompt_len=2000, gen=0, first_token_ns=0, class_id=0, req_id=2)]
+    wl = make_wl(rows, cls, replicas=[(gen.DECODE, 32768, 2)], now=[MS])
+    o = oracle.step(wl)
+    ed1 = 8_000_000 + 100_000 + 20 * 1000
+    assert o["e_d"][0] == ed1 and o["budget"][0] == 50 * MS - ed1
+    assert o["adm_count"][0] == 1          # batch cap 2: one running + one migrated
+    # the longer prefilled request predicts the larger TPOT, so it has less slack and goes first
+    assert list(o["order"]) == [0, 2, 1]
+    assert o["adm_cost"][0] == 100_000 + 20 * 2000
+    assert o["maturity_next"][0] == MS + 8_000_000 + 2 * 100_000 + 20 * 3000
+    # idle D-stage instance: strictest TPOT of the prefilled queue
+    rows[0]["state"] = gen.DONE
+    wl = make_wl(rows, cls, replicas=[(gen.DECODE, 32768, 0)], now=[MS])
+    o = oracle.step(wl)
+    assert o["budget"][0] == 30 * MS - 8_000_000 and o["adm_count"][0] == 2
+    assert o["maturity_next"][0] == MS + 8_000_000 + 2 * 100_000 + 20 * 2500
+
+
+def test_cap_only_mode_and_batch_cap():
+    rows = [dict(prompt_len=3000, req_id=i, arrival_ns=i) for i in range(5)]
+    wl = make_wl(rows, C200, replicas=[(gen.COLOCATED, 8192, 2)], now=[MS], budget_mode=gen.BUDGET_CAP_ONLY)
+    o = oracle.step(wl)
+    assert o["budget"][0] == 8192 and o["adm_count"][0] == 2 and o["adm_cost"][0] == 6000
+    wl = make_wl(rows, C200, replicas=[(gen.COLOCATED, 8192, 0)], now=[MS], budget_mode=gen.BUDGET_CAP_ONLY)
+    o = oracle.step(wl)
+    assert o["adm_count"][0] == 2          # third request would make 9000 > 8192
+
+
+def test_oversize_prompt_rejected_on_commit_and_bad_rows_flagged():
+    rows = [dict(prompt_len=9000, req_id=0), dict(prompt_len=100, req_id=1, output_len=5), dict(prompt_len=100, class_id=7, req_id=2),
+            dict(prompt_len=-5, req_id=3), dict(prompt_len=10, req_id=4, replica_id=5)]
+    wl = make_wl(rows, C200, now=[MS])
+    o = oracle.step(wl, commit=True)
+    assert o["status"] == 1 | 2 | 4
+    assert list(wl.table["state"]) == [gen.REJECTED, gen.RUNNING, gen.QUEUED, gen.QUEUED, gen.QUEUED]
+    assert list(o["seg_off"]) == [0, 4] and o["order"][4] == 4
+    assert list(o["admit"]) == [0, 1, 0, 0, 0]

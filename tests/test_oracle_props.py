@@ -1,0 +1,260 @@
+"""Invariants, brute force and permutation tests of the oracle (CPU only)."""
+import itertools
+
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from helpers import MS, SEC, make_wl, permute_rows
+
+MODES3 = (gen.COLOCATED, gen.PREFILL, gen.DECODE)
+
+
+def _cases():
+    for seed in range(12):
+        yield gen.random_table(seed, 300 + 37 * seed, 1 + seed % 5, modes=MODES3, tie_heavy=seed % 3 == 0,
+                               batch_cap=(0, 7)[seed % 2], weight_max=(0, 16)[seed % 4 == 1],
+                               budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 2])
+
+
+@pytest.mark.parametrize("wl", list(_cases()), ids=lambda w: w.name)
+def test_step_invariants(wl):
+    o = oracle.step(wl)
+    t = wl.table
+    R = wl.n_replicas
+    assert o["status"] == 0
+    assert o["seg_off"][0] == 0 and o["seg_off"][R] == wl.n_rows
+    assert sorted(o["order"]) == list(range(wl.n_rows))            # a permutation
+    ttft = np.array([c[0] for c in wl.classes]); tpot = np.array([c[1] for c in wl.classes])
+    for r in range(R):
+        rows = o["order"][o["seg_off"][r]:o["seg_off"][r + 1]]
+        assert np.all(t["replica_id"][rows] == r)
+        mode, cap, bcap = wl.replicas[r]
+        running = t["state"][rows] == gen.RUNNING
+        visible = (t["state"][rows] == gen.QUEUED) & (t["arrival_ns"][rows] <= wl.now[r])
+        # in-flight requests are protected: always in the batch, and ordered first
+        assert np.all(o["admit"][rows][running] == 1)
+        nrun = int(running.sum())
+        assert np.all(running[:nrun]) and o["n_run"][r] == nrun
+        assert np.all(visible[nrun:nrun + int(visible.sum())])
+        inactive = ~(running | visible)
+        assert np.all(o["admit"][rows][inactive] == 0) and np.all(o["slack"][rows][inactive] == 0)
+        assert o["sum_kv"][r] == int((t["prompt_len"][rows][running].astype(np.int64) + t["gen"][rows][running]).sum())
+        # the order is ascending in (key, req_id)
+        keys = [(int(k), int(q)) for k, q in zip(o["key"][rows], t["req_id"][rows])]
+        assert keys == sorted(keys)
+        assert all((k >> 48) == r for k, _ in keys)
+        # admitted tokens never exceed the budget; the batch cap holds
+        newly = visible & (o["admit"][rows] == 1)
+        n_eff = 0 if mode == gen.PREFILL else nrun
+        if mode == gen.DECODE:
+            cost = wl.model[4] + wl.model[5] * (t["prompt_len"][rows].astype(np.int64) + t["gen"][rows])
+        else:
+            cost = t["prompt_len"][rows].astype(np.int64)
+            assert o["budget"][r] <= max(0, cap - n_eff)
+        assert o["adm_cost"][r] == int(cost[newly].sum()) <= o["budget"][r]
+        assert o["adm_count"][r] == int(newly.sum())
+        if bcap:
+            assert o["adm_count"][r] == 0 or n_eff + o["adm_count"][r] <= bcap
+        # before maturity the instance is protected
+        if wl.now[r] < wl.maturity[r]:
+            assert o["budget"][r] == 0 and o["adm_count"][r] == 0
+            assert o["maturity_next"][r] == wl.maturity[r]
+        # admission is prefix-closed among the rows that fit alone
+        elig = visible & (cost <= o["budget"][r])
+        adm_seq = o["admit"][rows][elig]
+        assert list(adm_seq) == sorted(adm_seq, reverse=True)
+        # the compacted admitted list
+        lst = o["admitted_rows"][o["seg_off"][r]:o["seg_off"][r + 1]]
+        assert list(lst[:o["adm_count"][r]]) == list(rows[newly]) and np.all(lst[o["adm_count"][r]:] == -1)
+        # slack of a visible queued row with a TTFT bound on a colocated / prefill replica
+        if mode != gen.DECODE:
+            start = max(wl.now[r], wl.maturity[r])
+            for i in rows[visible][:20]:
+                c = t["class_id"][i]
+                want = (ttft[c] - (start - t["arrival_ns"][i]) - oracle.Ep(wl.model, int(t["prompt_len"][i]))
+                        if ttft[c] > 0 else oracle.SLACK_MAX)
+                assert o["slack"][i] == want
+                assert o["pred_ttft"][i] == start - t["arrival_ns"][i] + oracle.Ep(wl.model, int(t["prompt_len"][i]))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_outputs_invariant_under_row_permutation(seed):
+    wl = gen.random_table(seed + 50, 400, 3, modes=MODES3, tie_heavy=seed % 2 == 0)
+    o1 = oracle.step(wl)
+    perm = np.random.default_rng(seed).permutation(wl.n_rows)
+    wl2 = permute_rows(wl, perm)
+    o2 = oracle.step(wl2)
+    for k in ("budget", "e_d", "n_run", "sum_kv", "adm_cost", "adm_count", "maturity_next", "seg_off"):
+        assert np.array_equal(o1[k], o2[k]), k
+    # per-request outputs keyed by req_id
+    id1, id2 = wl.table["req_id"], wl2.table["req_id"]
+    for k in ("slack", "admit", "key", "pred_ttft", "pred_tpot"):
+        a = dict(zip(id1.tolist(), o1[k].tolist())); b = dict(zip(id2.tolist(), o2[k].tolist()))
+        assert a == b, k
+    assert id1[o1["order"]].tolist() == id2[o2["order"]].tolist()
+
+
+def _brute_force_best_prefix(costs, budget, count_room):
+    """Over all subsets of the rows (given in priority order) that are prefix-closed among the
+    rows that fit alone and feasible, the largest one."""
+    elig = [j for j, c in enumerate(costs) if c <= budget]
+    best = []
+    for k in range(len(elig) + 1):
+        sub = elig[:k]
+        if sum(costs[j] for j in sub) <= budget and (count_room is None or len(sub) <= count_room):
+            best = sub
+        # feasibility is monotone in k for non-negative costs, but do not assume it here
+    return best
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_admission_against_brute_force(seed):
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(1, 9))
+    rows = [dict(prompt_len=int(rng.integers(1, 1500)), arrival_ns=int(rng.integers(0, 50 * MS)), req_id=i,
+                 class_id=int(rng.integers(0, 2))) for i in range(n)]
+    bcap = int(rng.integers(0, 4))
+    wl = make_wl(rows, [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)],
+                 replicas=[(gen.COLOCATED, 8192, bcap)], now=[60 * MS])
+    o = oracle.step(wl)
+    order = list(o["order"])
+    costs = [rows[i]["prompt_len"] for i in order]
+    best = _brute_force_best_prefix(costs, int(o["budget"][0]), bcap if bcap else None)
+    assert sorted(order[j] for j in best) == sorted(np.nonzero(o["admit"])[0].tolist())
+    # with equal costs the greedy set also has the maximum count over all feasible subsets
+    for r in rows:
+        r["prompt_len"] = 300
+    wl = make_wl(rows, [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)],
+                 replicas=[(gen.COLOCATED, 8192, bcap)], now=[60 * MS])
+    o = oracle.step(wl)
+    b = int(o["budget"][0])
+    best_count = 0
+    for mask in itertools.product([0, 1], repeat=n):
+        k = sum(mask)
+        if 300 * k <= b and (not bcap or k <= bcap):
+            best_count = max(best_count, k)
+    assert o["adm_count"][0] == best_count
+
+
+def test_budget_monotone_in_load():
+    cls = [(200 * MS, 30 * MS, 0)]
+    prev = None
+    for n_run in range(0, 240, 7):
+        rows = [dict(state=gen.RUNNING, prompt_len=300, gen=10, first_token_ns=0, req_id=i) for i in range(n_run)]
+        rows.append(dict(prompt_len=16, req_id=10_000))
+        o = oracle.step(make_wl(rows, cls, now=[MS]))
+        if prev is not None:
+            assert o["budget"][0] <= prev
+        prev = o["budget"][0]
+    assert prev == 0            # E_d has passed the TPOT SLO: nothing is safe
+    prev = None
+    for kv in range(0, 900_000, 50_000):
+        rows = [dict(state=gen.RUNNING, prompt_len=kv // 4, gen=0, first_token_ns=0, req_id=i) for i in range(4)]
+        rows.append(dict(prompt_len=16, req_id=10_000))
+        o = oracle.step(make_wl(rows, cls, now=[MS], replicas=[(gen.COLOCATED, 1 << 20, 0)]))
+        if prev is not None:
+            assert o["budget"][0] <= prev
+        prev = o["budget"][0]
+
+
+def test_queued_slack_falls_one_for_one_with_time():
+    wl = gen.random_table(99, 200, 1, inflight=0.0, done=0.0, future=0.0)
+    wl.maturity[:] = 0
+    o1 = oracle.step(wl)
+    wl.now += 12345
+    o2 = oracle.step(wl)
+    bounded = np.array([wl.classes[c][0] > 0 for c in wl.table["class_id"]])
+    assert np.all((o1["slack"] - o2["slack"])[bounded] == 12345)
+    assert np.all(o2["slack"][~bounded] == oracle.SLACK_MAX)
+
+
+def test_larger_batch_later_maturity():
+    cls = [(5000 * MS, 100 * MS, 0)]
+    base = [dict(state=gen.RUNNING, prompt_len=300, gen=10, first_token_ns=0, req_id=i) for i in range(8)]
+    prev = 0
+    for p in (16, 64, 256, 1024, 4096):
+        o = oracle.step(make_wl(base + [dict(prompt_len=p, req_id=100)], cls, now=[MS]))
+        assert o["adm_count"][0] == 1 and o["maturity_next"][0] > prev
+        prev = o["maturity_next"][0]
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_simulator_conservation(seed):
+    wl = gen.random_traces(seed, 6, 0, 120, iters=3000)
+    s = oracle.sim(wl)
+    t = wl.table
+    for j in range(6):
+        a, b = wl.trace_off[j], wl.trace_off[j + 1]
+        st = t["state"][a:b]
+        assert np.all(st <= 3)
+        done = st == gen.DONE
+        assert s["finished"][j] == int(done.sum()) and s["rejected"][j] == int((st == gen.REJECTED).sum())
+        assert s["attained"][j] <= s["finished"][j]
+        # a finished request emitted exactly output_len tokens; times are ordered
+        assert np.all(t["gen"][a:b][done] + 1 == t["output_len"][a:b][done])
+        served = (st == gen.DONE) | (st == gen.RUNNING)
+        assert np.all(t["first_token_ns"][a:b][served] >= t["arrival_ns"][a:b][served])
+        assert np.all(t["last_token_ns"][a:b][served] >= t["first_token_ns"][a:b][served])
+        assert np.all(t["finish_ns"][a:b][done] == t["last_token_ns"][a:b][done])
+        assert np.all(t["first_token_ns"][a:b][~served] == -1)
+        assert np.all(t["prompt_len"][a:b][st == gen.REJECTED] > 8192)
+        assert 0 <= s["iters_executed"][j] <= 3000
+        if b > a and s["iters_executed"][j] < 3000:     # ran to completion: nothing is left waiting
+            assert not np.any(st == gen.RUNNING)
+            left = np.nonzero(st == gen.QUEUED)[0] + a
+            if left.size:
+                # what is left could never fit: the idle budget set by the strictest TTFT still
+                # waiting is smaller than every waiting prompt
+                ttfts = [wl.classes[c][0] for c in t["class_id"][left] if wl.classes[c][0] > 0]
+                assert ttfts
+                n_safe = oracle.nsafe(wl.model, min(ttfts) // 2, 8192)
+                assert np.all(t["prompt_len"][left] > n_safe)
+        if b == a:
+            assert s["iters_executed"][j] == 0 and s["ttft_p50"][j] == -1
+
+
+def test_simulator_equals_repeated_step_commit():
+    wl = gen.random_traces(11, 1, 60, 60, iters=400)
+    w1 = wl.copy()
+    s = oracle.sim(w1)
+    w2 = wl.copy()
+    t = w2.table
+    t["state"][:] = 0; t["gen"][:] = 0
+    for k in ("first_token_ns", "last_token_ns", "finish_ns"):
+        t[k][:] = -1
+    clocks = []
+    for it in range(int(s["iters_executed"][0])):
+        oracle.step(w2, commit=True)
+        clocks.append(int(w2.now[0]))
+    assert clocks == sorted(clocks)
+    for k in ("state", "gen", "first_token_ns", "last_token_ns", "finish_ns"):
+        assert np.array_equal(w1.table[k], t[k]), k
+    assert s["now"][0] == w2.now[0]
+
+
+def test_percentiles_nearest_rank_against_numpy():
+    wl = gen.random_traces(5, 3, 100, 200, iters=20000)
+    s = oracle.sim(wl)
+    t = wl.table
+    for j in range(3):
+        a, b = wl.trace_off[j], wl.trace_off[j + 1]
+        served = (t["state"][a:b] == gen.DONE) | (t["state"][a:b] == gen.RUNNING)
+        v = np.sort((t["first_token_ns"][a:b] - t["arrival_ns"][a:b])[served])
+        for p, k in ((50, "ttft_p50"), (99, "ttft_p99")):
+            want = np.percentile(v, p, method="inverted_cdf") if v.size else -1
+            assert s[k][j] == want
+
+
+def test_configs_smoke():
+    for wl in (gen.config1(), gen.config2(R=4, rows_per=256), gen.config3(R=4, rows_per=512),
+               gen.config4(R=8, n=4096), gen.config2(R=4, rows_per=256, inflight=0.02)):
+        o = oracle.step(wl)
+        assert o["status"] == 0 and sorted(o["order"]) == list(range(wl.n_rows))
+    wl = gen.config5(traces=2, rows_per=256, iters=3000)
+    s = oracle.sim(wl)
+    assert np.all(s["finished"] > 0)
+    full = gen.config5(traces=3, rows_per=64, iters=10)
+    part = gen.config5(traces=1, rows_per=64, iters=10, first_trace=2)
+    assert np.array_equal(full.table["arrival_ns"][128:], part.table["arrival_ns"])
