@@ -234,15 +234,15 @@ int hfx_sched_step(hfx_sched *s, const hfx_table *table,
 /* Trace-driven simulation (events are request arrivals and iteration
  * completions, Problem Definition; metrics are Eq. 2 and the TTFT / TPOT
  * definitions).  `table` holds n_traces traces back to back, trace j being
- * rows trace_off[j] .. trace_off[j+1]-1 (device int32 array of n_traces+1
- * offsets), sorted by arrival within a trace; trace j runs on replica j of the
- * scheduler, which must be COLOCATED.  replica_id is not read.  Every trace
+ * rows trace_off[j] .. trace_off[j+1]-1 (HOST int32 array of n_traces+1
+ * offsets, copied before the call returns), sorted by arrival within a trace;
+ * trace j runs on replica j of the scheduler, which must be COLOCATED.  replica_id is not read.  Every trace
  * starts at time 0 with all rows QUEUED (the incoming state, gen and time
  * columns are overwritten) and runs `iters` iterations of step + commit, or
  * until nothing is left to happen.  Written: state, gen, first_token_ns,
  * last_token_ns, finish_ns and `out`.
  * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY (n_traces > n_replicas, or a
- * trace longer than 8192 rows), HFX_E_CUDA. */
+ * trace longer than 4096 rows), HFX_E_CUDA. */
 int hfx_sim_run(hfx_sched *s, const hfx_table *table, const int32_t *trace_off,
                 int32_t n_traces, int32_t iters, const hfx_sim_out *out);
 

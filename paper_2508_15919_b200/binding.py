@@ -1,0 +1,259 @@
+"""ctypes binding of libhfx.so (argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libhfx.so")
+_lib = None
+
+COMMIT = 1
+QUEUED, RUNNING, DONE, REJECTED = 0, 1, 2, 3
+COLOCATED, PREFILL, DECODE = 0, 1, 2
+BUDGET_SAFE, BUDGET_CAP_ONLY = 0, 1
+ST_BAD_REPLICA, ST_BAD_CLASS, ST_BAD_LEN, ST_TIMEOUT = 1, 2, 4, 8
+E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
+
+EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
+                    "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror"]
+
+
+class HfxError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {load_library().hfx_strerror(code).decode()} ({code})")
+
+
+class _Model(C.Structure):
+    _fields_ = [(k, C.c_int64) for k in ("c0", "c1", "c2", "d0", "d1", "d2")]
+
+
+class _SloClass(C.Structure):
+    _fields_ = [("ttft_slo_ns", C.c_int64), ("tpot_slo_ns", C.c_int64), ("prio", C.c_int32), ("reserved", C.c_int32)]
+
+
+class _ReplicaCfg(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("token_cap", C.c_int32), ("batch_cap", C.c_int32)]
+
+
+class _Options(C.Structure):
+    _fields_ = [("budget_mode", C.c_int32), ("weight_max", C.c_int32), ("flags", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+TABLE_COLUMNS = ["replica_id", "class_id", "state", "prompt_len", "output_len", "gen", "arrival_ns",
+                 "first_token_ns", "last_token_ns", "finish_ns", "req_id", "weight"]
+TABLE_DTYPES = {"replica_id": torch.int32, "class_id": torch.uint8, "state": torch.uint8, "prompt_len": torch.int32,
+                "output_len": torch.int32, "gen": torch.int32, "arrival_ns": torch.int64,
+                "first_token_ns": torch.int64, "last_token_ns": torch.int64, "finish_ns": torch.int64,
+                "req_id": torch.int32, "weight": torch.int32}
+
+
+class _Table(C.Structure):
+    _fields_ = [("n_rows", C.c_int64)] + [(k, C.c_void_p) for k in TABLE_COLUMNS]
+
+
+class _ReplicaState(C.Structure):
+    _fields_ = [("now_ns", C.c_void_p), ("maturity_ns", C.c_void_p)]
+
+
+STEP_OUT_FIELDS = [("slack_ns", torch.int64, "n"), ("pred_ttft_ns", torch.int64, "n"), ("pred_tpot_ns", torch.int64, "n"),
+                   ("key", torch.int64, "n"), ("order", torch.int32, "n"), ("seg_off", torch.int32, "R1"),
+                   ("admit", torch.uint8, "n"), ("admitted_rows", torch.int32, "n"), ("budget", torch.int64, "R"),
+                   ("e_d_ns", torch.int64, "R"), ("n_run", torch.int32, "R"), ("sum_kv", torch.int64, "R"),
+                   ("adm_cost", torch.int64, "R"), ("adm_count", torch.int32, "R"), ("maturity_next", torch.int64, "R")]
+STEP_OUT_OPTIONAL = {"pred_ttft_ns", "pred_tpot_ns", "key", "admitted_rows", "e_d_ns", "n_run", "sum_kv"}
+
+
+class _StepOut(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k, _, _ in STEP_OUT_FIELDS]
+
+
+SIM_OUT_FIELDS = [("iters_executed", torch.int32), ("finished", torch.int32), ("rejected", torch.int32),
+                  ("attained", torch.int32), ("ttft_p50_ns", torch.int64), ("ttft_p99_ns", torch.int64),
+                  ("tpot_p50_ns", torch.int64), ("tpot_p99_ns", torch.int64), ("now_ns", torch.int64)]
+
+
+class _SimOut(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k, _ in SIM_OUT_FIELDS]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Load libhfx.so.  There is no fallback: a missing library is an error."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2508_15919_b200.build` "
+                          "(nvcc, sm_100a); there is no CPU fallback")
+    L = C.CDLL(_LIB_PATH)
+    L.hfx_sched_create.restype = C.c_int
+    L.hfx_sched_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(_Model), C.POINTER(_SloClass), C.c_int,
+                                   C.POINTER(_ReplicaCfg), C.c_int, C.c_int64, C.POINTER(_Options), C.c_void_p]
+    L.hfx_sched_step.restype = C.c_int
+    L.hfx_sched_step.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_ReplicaState), C.POINTER(_StepOut), C.c_uint32]
+    L.hfx_sim_run.restype = C.c_int
+    L.hfx_sim_run.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_SimOut)]
+    L.hfx_sched_status.restype = C.c_int
+    L.hfx_sched_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
+    L.hfx_sched_launch_count.restype = C.c_int64
+    L.hfx_sched_launch_count.argtypes = [C.c_void_p]
+    L.hfx_sched_destroy.restype = None
+    L.hfx_sched_destroy.argtypes = [C.c_void_p]
+    L.hfx_strerror.restype = C.c_char_p
+    L.hfx_strerror.argtypes = [C.c_int]
+    _lib = L
+    return L
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+class DeviceTable:
+    """The request table as torch tensors on the GPU (structure of arrays)."""
+
+    def __init__(self, cols: Dict[str, torch.Tensor]):
+        self.cols = cols
+        self.n_rows = int(cols["class_id"].shape[0])
+        for k, t in cols.items():
+            if t is not None:
+                assert t.is_cuda and t.is_contiguous() and t.dtype == TABLE_DTYPES[k], k
+
+    @staticmethod
+    def from_numpy(cols: Dict[str, np.ndarray], device="cuda") -> "DeviceTable":
+        out = {}
+        for k in TABLE_COLUMNS:
+            a = cols.get(k)
+            out[k] = None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(device)
+        return DeviceTable(out)
+
+    def to_numpy(self) -> Dict[str, np.ndarray]:
+        return {k: v.cpu().numpy() for k, v in self.cols.items() if v is not None}
+
+    def c_struct(self) -> _Table:
+        s = _Table()
+        s.n_rows = self.n_rows
+        for k in TABLE_COLUMNS:
+            setattr(s, k, _ptr(self.cols.get(k)))
+        return s
+
+
+class StepOut:
+    """Output buffers of one step (allocated once, reused)."""
+
+    def __init__(self, n_rows: int, n_replicas: int, device="cuda", optional: bool = True):
+        self.t: Dict[str, Optional[torch.Tensor]] = {}
+        for k, dt, dim in STEP_OUT_FIELDS:
+            size = {"n": max(n_rows, 1), "R": n_replicas, "R1": n_replicas + 1}[dim]
+            self.t[k] = None if (k in STEP_OUT_OPTIONAL and not optional) else torch.zeros(size, dtype=dt, device=device)
+        self.n_rows = n_rows
+
+    def c_struct(self) -> _StepOut:
+        s = _StepOut()
+        for k, _, _ in STEP_OUT_FIELDS:
+            setattr(s, k, _ptr(self.t[k]))
+        return s
+
+    def to_numpy(self) -> Dict[str, np.ndarray]:
+        out = {}
+        for k, v in self.t.items():
+            if v is None:
+                continue
+            a = v.cpu().numpy()
+            if k == "key":
+                a = a.view(np.uint64)
+            if k in ("slack_ns", "pred_ttft_ns", "pred_tpot_ns", "key", "order", "admit", "admitted_rows"):
+                a = a[:self.n_rows]
+            out[k] = a
+        return out
+
+
+class SimOut:
+    def __init__(self, n_traces: int, device="cuda"):
+        self.t = {k: torch.zeros(max(n_traces, 1), dtype=dt, device=device) for k, dt in SIM_OUT_FIELDS}
+        self.n_traces = n_traces
+
+    def c_struct(self) -> _SimOut:
+        s = _SimOut()
+        for k, _ in SIM_OUT_FIELDS:
+            setattr(s, k, _ptr(self.t[k]))
+        return s
+
+    def to_numpy(self) -> Dict[str, np.ndarray]:
+        return {k: v.cpu().numpy()[:self.n_traces] for k, v in self.t.items()}
+
+
+class Scheduler:
+    """hfx_sched_create / hfx_sched_step / hfx_sim_run / hfx_sched_status on torch tensors."""
+
+    def __init__(self, model: Sequence[int], classes: Sequence[Sequence[int]], replicas, max_rows: int,
+                 budget_mode: int = BUDGET_SAFE, weight_max: int = 0, stream: Optional[torch.cuda.Stream] = None):
+        L = load_library()
+        self._L = L
+        self._h = C.c_void_p()
+        m = _Model(*[int(x) for x in model])
+        cls = (_SloClass * len(classes))(*[_SloClass(int(a), int(b), int(p), 0) for a, b, p in classes])
+        reps_np = np.asarray(replicas, np.int32).reshape(-1, 3)
+        reps = (_ReplicaCfg * reps_np.shape[0])(*[_ReplicaCfg(int(r[0]), int(r[1]), int(r[2])) for r in reps_np])
+        opts = _Options(int(budget_mode), int(weight_max), 0, 0)
+        self.n_replicas = reps_np.shape[0]
+        self.stream = stream
+        if stream is not None:
+            sp = C.c_void_p(stream.cuda_stream)
+        elif torch.cuda.is_available():
+            sp = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+        else:
+            sp = C.c_void_p()      # no device: the library reports HFX_E_CUDA
+        rc = L.hfx_sched_create(C.byref(self._h), C.byref(m), cls, len(classes), reps, self.n_replicas, int(max_rows),
+                                C.byref(opts), sp)
+        if rc != 0:
+            self._h = C.c_void_p()
+            raise HfxError(rc, "hfx_sched_create")
+
+    def step(self, table: DeviceTable, now: torch.Tensor, maturity: torch.Tensor, out: StepOut, commit: bool = False):
+        ts, os_ = table.c_struct(), out.c_struct()
+        st = _ReplicaState(now.data_ptr(), maturity.data_ptr())
+        rc = self._L.hfx_sched_step(self._h, C.byref(ts), C.byref(st), C.byref(os_), COMMIT if commit else 0)
+        if rc != 0:
+            raise HfxError(rc, "hfx_sched_step")
+
+    def step_raw(self, ts: _Table, st: _ReplicaState, os_: _StepOut, flags: int) -> int:
+        """The bare call on prebuilt structs (what a latency-sensitive caller keeps around)."""
+        return self._L.hfx_sched_step(self._h, C.byref(ts), C.byref(st), C.byref(os_), flags)
+
+    def sim_run(self, table: DeviceTable, trace_off: np.ndarray, iters: int, out: SimOut):
+        off = np.ascontiguousarray(trace_off, np.int32)
+        ts, os_ = table.c_struct(), out.c_struct()
+        rc = self._L.hfx_sim_run(self._h, C.byref(ts), off.ctypes.data, int(off.shape[0] - 1), int(iters), C.byref(os_))
+        if rc != 0:
+            raise HfxError(rc, "hfx_sim_run")
+
+    def status(self) -> int:
+        w = C.c_uint32(0)
+        rc = self._L.hfx_sched_status(self._h, C.byref(w))
+        if rc not in (0, E_TIMEOUT):
+            raise HfxError(rc, "hfx_sched_status")
+        return int(w.value)
+
+    def launch_count(self) -> int:
+        return int(self._L.hfx_sched_launch_count(self._h))
+
+    def close(self):
+        if self._h:
+            self._L.hfx_sched_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

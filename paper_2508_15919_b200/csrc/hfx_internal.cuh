@@ -1,0 +1,222 @@
+// Internal declarations shared by the kernels of the scheduler library.
+// Integer nanoseconds everywhere; nothing here is floating point.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hfx.h"
+
+#define HFX_MAX_CLASSES 64
+#define HFX_MAX_REPLICAS 65536
+#define HFX_MAX_ROWS (INT64_C(1) << 27)
+
+// phases of the key (2 bits)
+#define PH_RUNNING 0
+#define PH_QUEUED 1
+#define PH_INACTIVE 3
+
+// kinds of a regrouped record
+#define KIND_RUNNING 0  // in flight
+#define KIND_QUEUED 1   // arrived and waiting
+#define KIND_FUTURE 2   // QUEUED but not arrived yet (only matters for the idle clock jump)
+#define KIND_DEAD 3     // DONE, REJECTED or a row with bad data
+
+// "no bound" marker of a slack base
+#define BASE_UNBOUNDED INT64_MAX
+
+// Scheduler constants, passed by value to every kernel (lives in the constant bank).
+struct HfxParams {
+  int64_t c0, c1, c2, d0, d1, d2;
+  int64_t ttft[HFX_MAX_CLASSES];
+  int64_t tpot[HFX_MAX_CLASSES];
+  uint8_t prio[HFX_MAX_CLASSES];
+  int32_t n_classes;
+  int32_t n_replicas;
+  int32_t budget_mode;
+  int32_t weight_max;
+};
+
+// One row after regrouping by replica: everything the per-replica kernel needs, 32 bytes
+// (one L2 sector), so that kernel never goes back to the table for reads.
+struct __align__(16) HfxRec {
+  int64_t base;      // slack before the per-replica shift; arrival for KIND_FUTURE
+  int32_t req_id;
+  int32_t row;
+  int32_t prompt;
+  int32_t gen;
+  int32_t output_len;
+  uint8_t cls, kind, prio, pad;
+};
+static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
+
+struct hfx_sched {
+  HfxParams p;
+  hfx_options opts;
+  int64_t max_rows;
+  int n_sm;
+  cudaStream_t stream;
+  int64_t launches;
+  // device
+  hfx_replica_cfg *d_cfg;   // [R]
+  uint32_t *d_status;       // sticky status word
+  uint32_t *d_seg_count;    // [R+2] rows per replica (+ the bad-replica bucket R)
+  uint32_t *d_seg_begin;    // [R+2] exclusive prefix
+  uint32_t *d_cursor;       // [R+2] fill cursors of the regroup pass
+  int32_t *d_list;          // [3][R+1] replicas by segment-size class
+  uint32_t *d_list_n;       // [4]
+  HfxRec *d_rec;            // [max_rows]
+  uint64_t *d_big_hi;       // sort scratch of oversize segments
+  uint32_t *d_big_lo;
+  uint32_t *d_barrier;      // grid barrier words of the oversize path
+};
+
+// ---- latency predictor -------------------------------------------------------------------
+__device__ __forceinline__ int64_t dev_Ep(const HfxParams &p, int64_t t) { return p.c0 + p.c1 * t + p.c2 * t * t; }
+__device__ __forceinline__ int64_t dev_Ed(const HfxParams &p, int64_t b, int64_t kv) { return p.d0 + p.d1 * b + p.d2 * kv; }
+
+__device__ __forceinline__ int64_t dev_clamp_slack(int64_t s) {
+  return s < HFX_SLACK_MIN ? HFX_SLACK_MIN : (s > HFX_SLACK_MAX ? HFX_SLACK_MAX : s);
+}
+
+// phase<2> | prio<6> | (clamp(slack) + 2^39)<40>  -- the low 48 bits of the key
+__device__ __forceinline__ uint64_t dev_key48(int phase, int prio, int64_t slack) {
+  return ((uint64_t)phase << 46) | ((uint64_t)prio << 40) | (uint64_t)(dev_clamp_slack(slack) + (INT64_C(1) << 39));
+}
+
+// Per-replica quantities of one step, computed once per replica.
+struct ReplicaPlan {
+  int64_t now, mat, start;
+  int64_t n_run, sum_kv, n_eff, kv_eff;
+  int64_t tpot_eff;   // strictest TPOT of the running batch (HFX_INF if none)
+  int64_t e_d;
+  int64_t budget;
+  int64_t shift_run;  // slack of a running row   = base - shift_run
+  int64_t shift_dq;   // slack of a decode-queued = base - shift_dq
+  int32_t mode, token_cap, batch_cap;
+};
+
+// Largest E_p with 2 E_p + k E_d <= TTFT, k = E_p / (TPOT - E_d)  (worst-case TTFT bound
+// behind Eq. 3).  HFX_INF without a TTFT bound, -1 when TPOT <= E_d.
+__device__ inline int64_t dev_epmax(int64_t min_ttft, bool decoding, int64_t min_tpot, int64_t e_d) {
+  if (min_ttft == HFX_INF) return HFX_INF;
+  if (!decoding) return min_ttft / 2;
+  if (min_tpot <= e_d) return -1;
+  unsigned __int128 num = (unsigned __int128)(uint64_t)min_ttft * (uint64_t)(min_tpot - e_d);
+  uint64_t den = (uint64_t)(2 * min_tpot - e_d);
+  return (int64_t)(num / den);
+}
+
+// Largest n in [0, cap] with E_p(n) <= epmax (Eq. 3 on the general prefill model), 0 if none.
+__device__ inline int64_t dev_nsafe(const HfxParams &p, int64_t epmax, int64_t cap) {
+  if (epmax == HFX_INF) return cap;
+  if (dev_Ep(p, 0) > epmax) return 0;
+  int64_t lo = 0, hi = cap;
+  while (lo < hi) {
+    int64_t mid = lo + (hi - lo + 1) / 2;
+    if (dev_Ep(p, mid) <= epmax) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ inline int64_t dev_min_over_mask(const int64_t *v, uint64_t mask) {
+  int64_t m = HFX_INF;
+  while (mask) {
+    int c = __ffsll((long long)mask) - 1;
+    mask &= mask - 1;
+    if (v[c] > 0 && v[c] < m) m = v[c];
+  }
+  return m;
+}
+
+// Dispatching step 2 for one replica: E_d of the running batch and the safe budget.
+__device__ inline void dev_plan(const HfxParams &p, const hfx_replica_cfg &cfg, int64_t now, int64_t mat,
+                                int64_t n_run, int64_t sum_kv, uint64_t mask_run, uint64_t mask_q,
+                                ReplicaPlan &pl) {
+  pl.now = now; pl.mat = mat; pl.start = now > mat ? now : mat;
+  pl.mode = cfg.mode; pl.token_cap = cfg.token_cap; pl.batch_cap = cfg.batch_cap;
+  pl.n_run = n_run; pl.sum_kv = sum_kv;
+  const int64_t min_tpot = dev_min_over_mask(p.tpot, mask_run);
+  const int64_t min_ttft = dev_min_over_mask(p.ttft, mask_q);
+  const int64_t min_tpot_q = dev_min_over_mask(p.tpot, mask_q);
+  const bool prefill = cfg.mode == HFX_PREFILL;
+  pl.n_eff = prefill ? 0 : n_run;
+  pl.kv_eff = prefill ? 0 : sum_kv;
+  pl.tpot_eff = prefill ? HFX_INF : min_tpot;
+  pl.e_d = pl.n_eff > 0 ? dev_Ed(p, pl.n_eff, pl.kv_eff) : 0;
+  int64_t budget;
+  if (cfg.mode == HFX_DECODE) {
+    const int64_t T = (n_run > 0 && min_tpot < HFX_INF) ? min_tpot : min_tpot_q;
+    if (p.budget_mode == HFX_BUDGET_CAP_ONLY || T == HFX_INF) budget = HFX_INF;
+    else {
+      const int64_t room = T - dev_Ed(p, n_run, sum_kv);
+      budget = room > 0 ? room : 0;
+    }
+  } else {
+    const int64_t cap_left = cfg.token_cap - pl.n_eff > 0 ? cfg.token_cap - pl.n_eff : 0;
+    int64_t n_safe;
+    if (p.budget_mode == HFX_BUDGET_CAP_ONLY) n_safe = cfg.token_cap;
+    else n_safe = dev_nsafe(p, dev_epmax(min_ttft, pl.n_eff > 0 && pl.tpot_eff < HFX_INF, pl.tpot_eff, pl.e_d), cfg.token_cap);
+    budget = n_safe < cap_left ? n_safe : cap_left;
+  }
+  if (now < mat) budget = 0;
+  pl.budget = budget;
+  pl.shift_run = pl.e_d;
+  pl.shift_dq = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
+}
+
+// Dispatching step 4: maturity time after admitting adm_count requests of adm_cost in total.
+__device__ inline int64_t dev_maturity_next(const HfxParams &p, const ReplicaPlan &pl, int64_t adm_count,
+                                            int64_t adm_cost, int64_t adm_kv, int64_t *lp_out) {
+  int64_t lp = 0, mat_next = pl.mat;
+  if (pl.mode == HFX_DECODE) {
+    if (pl.now >= pl.mat && pl.n_run + adm_count > 0)
+      mat_next = pl.now + dev_Ed(p, pl.n_run + adm_count, pl.sum_kv + adm_kv);
+  } else if (adm_count > 0) {
+    lp = dev_Ep(p, adm_cost);
+    if (pl.mode == HFX_PREFILL) mat_next = pl.now + lp;
+    else {
+      unsigned __int128 k = 0;
+      if (pl.n_eff > 0 && pl.tpot_eff < HFX_INF && pl.tpot_eff > pl.e_d) {
+        const uint64_t d = (uint64_t)(pl.tpot_eff - pl.e_d);
+        k = ((uint64_t)lp + d - 1) / d;
+      }
+      __int128 v = (__int128)pl.now + lp + (__int128)(k * (uint64_t)pl.e_d);
+      mat_next = v > (__int128)HFX_TIME_MAX ? HFX_TIME_MAX : (int64_t)v;
+    }
+  }
+  *lp_out = lp;
+  return mat_next;
+}
+
+// ---- warp / block primitives ----------------------------------------------------------------
+__device__ __forceinline__ int64_t warp_sum_i64(int64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int64_t warp_min_i64(int64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { int64_t w = __shfl_xor_sync(0xffffffffu, v, o); v = w < v ? w : v; }
+  return v;
+}
+__device__ __forceinline__ uint64_t warp_or_u64(uint64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v |= __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int64_t warp_incl_scan_i64(int64_t v, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { int64_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+  return v;
+}
+__device__ __forceinline__ int32_t warp_incl_scan_i32(int32_t v, int lane) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { int32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+  return v;
+}
+
+// host-side launchers implemented in the .cu files
+int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o, uint32_t flags);
+int hfx_launch_sim(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
+                   const hfx_sim_out *o);

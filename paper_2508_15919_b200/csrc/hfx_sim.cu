@@ -1,0 +1,412 @@
+// hfx_sim_run: batched trace-driven simulation, one persistent thread block per trace.
+//
+// A trace is staged once into shared memory; then the block runs the scheduler iteration
+// (visible set, aggregates of the running batch, E_d, safe budget, most-urgent-first admission,
+// maturity, commit, clock advance) `iters` times without leaving the chip.  Work per iteration
+// scales with the live set (queue + running batch), not with the trace length:
+//   - rows are sorted by arrival, so the visible queue grows from a head pointer;
+//   - the running batch and the strictest SLOs are kept as incremental counters;
+//   - a running request's completion iteration is fixed at admission (every iteration with a
+//     running batch advances each of its requests by one token);
+//   - admission extracts the most urgent eligible request repeatedly (block-wide arg-min on
+//     (prio, clamp(slack), req_id)) and stops at the first one that does not fit, which is
+//     exactly the prefix-closed rule of the sorted formulation.
+#include "hfx_internal.cuh"
+
+#define SIM_THREADS 128
+#define SIM_WARPS (SIM_THREADS / 32)
+#define SIM_MAX_ROWS 4096
+#define SIM_BYTES_PER_ROW 44
+
+#define ROW_INVALID 0xff
+
+struct SimArgs {
+  const uint8_t *class_id; const int32_t *prompt_len; const int32_t *output_len; const int64_t *arrival;
+  const int32_t *req_id; const int32_t *weight;
+  uint8_t *state; int32_t *gen; int64_t *first_token; int64_t *last_token; int64_t *finish;
+  const int32_t *trace_off; const hfx_replica_cfg *cfg;
+  int32_t n_traces, iters, cap_rows;
+  // outputs
+  int32_t *iters_executed, *finished, *rejected, *attained;
+  int64_t *ttft_p50, *ttft_p99, *tpot_p50, *tpot_p99, *now_out;
+};
+
+struct SimShared {
+  ReplicaPlan plan;
+  int64_t now, mat, sum_kv;
+  int64_t t1, t2, lp, mat_next;
+  int64_t d_kv;                 // change of sum_kv collected during commit
+  int32_t cnt_run[HFX_MAX_CLASSES], cnt_q[HFX_MAX_CLASSES];
+  int32_t head, nq, nr, nr_next, na, no, arrived;
+  int32_t worked, stop, trace, zero_prompt;
+  // arg-min scratch, double buffered
+  uint64_t best_key[2][SIM_WARPS];
+  uint32_t best_id[2][SIM_WARPS];
+  int32_t best_slot[2][SIM_WARPS];
+  // end-of-trace counters
+  int32_t n_fin, n_rej, n_att, n_a, n_b;
+};
+
+__device__ __forceinline__ void sort_i64(int64_t *v, int n) {
+  int n_pad = 1;
+  while (n_pad < n) n_pad <<= 1;
+  const int half = n_pad >> 1;
+  for (int k = 2; k <= n_pad; k <<= 1) {
+    const int hk = k >> 1;
+    for (int t = threadIdx.x; t < half; t += blockDim.x) {
+      const int blk = t / hk, off = t - blk * hk;
+      const int i = blk * k + off, j = blk * k + k - 1 - off;
+      if (j < n) { const int64_t x = v[i], y = v[j]; if (x > y) { v[i] = y; v[j] = x; } }
+    }
+    __syncthreads();
+    for (int j = k >> 2; j > 0; j >>= 1) {
+      for (int t = threadIdx.x; t < half; t += blockDim.x) {
+        const int i = 2 * t - (t & (j - 1));
+        if (i + j < n) { const int64_t x = v[i], y = v[i + j]; if (x > y) { v[i] = y; v[i + j] = x; } }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+__device__ __forceinline__ int64_t nearest_rank(const int64_t *sorted, int n, int pct) {
+  if (n == 0) return -1;
+  int64_t k = ((int64_t)pct * n + 99) / 100;
+  if (k < 1) k = 1;
+  return sorted[k - 1];
+}
+
+__global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const SimArgs a, uint32_t *__restrict__ work_counter,
+                                                     uint32_t *__restrict__ status) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int cap = a.cap_rows;
+  int64_t *s_arr = reinterpret_cast<int64_t *>(smem_raw);              // arrival; later TTFT samples
+  int64_t *s_dst = s_arr + cap;                                        // ttft_slo + arrival - E_p(prompt); later TPOT samples
+  int32_t *s_prompt = reinterpret_cast<int32_t *>(s_dst + cap);
+  int32_t *s_outlen = s_prompt + cap;
+  int32_t *s_admit_it = s_outlen + cap;
+  uint32_t *s_reqid = reinterpret_cast<uint32_t *>(s_admit_it + cap);
+  uint16_t *s_q = reinterpret_cast<uint16_t *>(s_reqid + cap);         // visible queue (row indices, unordered)
+  uint16_t *s_run = s_q + cap;                                         // running batch, ping
+  uint16_t *s_run2 = s_run + cap;                                      // running batch, pong
+  uint16_t *s_adm = s_run2 + cap;                                      // admitted this iteration; oversize rows from the top
+  uint8_t *s_cls = reinterpret_cast<uint8_t *>(s_adm + cap);
+  uint8_t *s_prio = s_cls + cap;
+  uint8_t *s_state = s_prio + cap;
+  __shared__ SimShared S;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (;;) {
+    __syncthreads();
+    if (tid == 0) S.trace = (int32_t)atomicAdd(work_counter, 1u);
+    __syncthreads();
+    const int j = S.trace;
+    if (j >= a.n_traces) return;
+    const int32_t b = a.trace_off[j];
+    const int m = a.trace_off[j + 1] - b;
+    const hfx_replica_cfg cfg = a.cfg[j];
+
+    // ---- stage the trace ----------------------------------------------------------------
+    if (tid == 0) {
+      S.now = 0; S.mat = 0; S.sum_kv = 0; S.head = 0; S.nq = 0; S.nr = 0; S.stop = 0;
+      S.n_fin = 0; S.n_rej = 0; S.n_att = 0; S.n_a = 0; S.n_b = 0; S.zero_prompt = 0;
+    }
+    __syncthreads();
+    for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; }
+    uint32_t bad = 0;
+    bool unsorted = false;
+    for (int i = tid; i < m; i += SIM_THREADS) {
+      const int64_t g = (int64_t)b + i;
+      const uint32_t cls = a.class_id[g];
+      const int32_t prompt = a.prompt_len[g];
+      const int64_t arr = a.arrival[g];
+      bool ok = true;
+      if (cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
+      if (prompt < 0 || prompt > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }
+      if (i + 1 < m && a.arrival[g + 1] < arr) unsorted = true;
+      s_arr[i] = arr;
+      s_prompt[i] = prompt;
+      if (prompt == 0) S.zero_prompt = 1;   // a zero-token prompt fits a zero budget
+      s_outlen[i] = a.output_len[g];
+      s_reqid[i] = (uint32_t)a.req_id[g] ^ 0x80000000u;
+      s_admit_it[i] = -1;
+      s_cls[i] = ok ? (uint8_t)cls : ROW_INVALID;
+      s_state[i] = HFX_QUEUED;
+      int prio = 63;
+      int64_t d = BASE_UNBOUNDED;
+      if (ok) {
+        if (p.weight_max > 0) {
+          const int64_t w = (int64_t)p.weight_max - a.weight[g];
+          prio = (int)(w < 0 ? 0 : (w > 62 ? 62 : w));
+        } else prio = p.prio[cls];
+        const int64_t ttft = p.ttft[cls];
+        if (ttft > 0) d = ttft + arr - dev_Ep(p, prompt);
+      }
+      s_prio[i] = (uint8_t)prio;
+      s_dst[i] = d;
+      a.first_token[g] = -1; a.last_token[g] = -1; a.finish[g] = -1;
+    }
+    if (bad) atomicOr(status, bad);
+    // reading: an unsorted trace is a caller error; it is simulated as given (the head pointer
+    // stops at the first row that has not arrived), no fault can result
+    (void)unsorted;
+    __syncthreads();
+
+    int executed = 0;
+    uint16_t *run_cur = s_run, *run_nxt = s_run2;
+    for (int it = 0; it < a.iters; it++) {
+      // ---- 1. arrivals: rows [head, head + k) with arrival <= now join the queue -----------
+      if (tid == 0) { S.arrived = 0; S.no = 0; S.na = 0; S.nr_next = 0; S.d_kv = 0; }
+      __syncthreads();
+      {
+        const int64_t now = S.now;
+        const int head = S.head;
+        int local = 0;
+        for (int i = head + tid; i < m && s_arr[i] <= now; i += SIM_THREADS) {
+          local++;
+          const uint8_t cls = s_cls[i];
+          if (cls == ROW_INVALID) continue;
+          atomicAdd(&S.cnt_q[cls], 1);
+          if (s_prompt[i] > cfg.token_cap) {
+            // can never be served: visible for this one iteration, rejected at its commit
+            const int slot = atomicAdd(&S.no, 1);
+            s_adm[cap - 1 - slot] = (uint16_t)i;
+          } else {
+            const int slot = atomicAdd(&S.nq, 1);
+            s_q[slot] = (uint16_t)i;
+          }
+        }
+        if (local) atomicAdd(&S.arrived, local);
+      }
+      __syncthreads();
+
+      // ---- 2. plan: E_d of the running batch and the safe budget (one thread) -------------
+      if (tid == 0) {
+        S.head += S.arrived;
+        uint64_t m_run = 0, m_q = 0;
+        for (int c = 0; c < p.n_classes; c++) {
+          if (S.cnt_run[c] > 0) m_run |= 1ull << c;
+          if (S.cnt_q[c] > 0) m_q |= 1ull << c;
+        }
+        dev_plan(p, cfg, S.now, S.mat, S.nr, S.sum_kv, m_run, m_q, S.plan);
+      }
+      __syncthreads();
+      const int64_t budget = S.plan.budget, start = S.plan.start;
+      const int nr = S.nr;
+
+      // ---- 3. admission: extract the most urgent request that fits alone, until one fails ----
+      int64_t s_cost = 0, adm_cost = 0;
+      int s_cnt = 0, adm_cnt = 0;
+      int nq = S.nq;
+      if (budget > 0 || S.zero_prompt) {
+        int buf = 0;
+        for (;;) {
+          uint64_t bk = ~0ull; uint32_t bid = ~0u; int bslot = -1;
+          for (int s = tid; s < nq; s += SIM_THREADS) {
+            const int i = s_q[s];
+            if ((int64_t)s_prompt[i] > budget) continue;
+            const int64_t d = s_dst[i];
+            const int64_t sl = d == BASE_UNBOUNDED ? HFX_SLACK_MAX : dev_clamp_slack(d - start);
+            const uint64_t k = ((uint64_t)s_prio[i] << 40) | (uint64_t)(sl + (INT64_C(1) << 39));
+            const uint32_t id = s_reqid[i];
+            if (k < bk || (k == bk && id < bid)) { bk = k; bid = id; bslot = s; }
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const uint64_t k2 = __shfl_xor_sync(0xffffffffu, bk, o);
+            const uint32_t i2 = __shfl_xor_sync(0xffffffffu, bid, o);
+            const int s2 = __shfl_xor_sync(0xffffffffu, bslot, o);
+            if (k2 < bk || (k2 == bk && i2 < bid)) { bk = k2; bid = i2; bslot = s2; }
+          }
+          if (lane == 0) { S.best_key[buf][warp] = bk; S.best_id[buf][warp] = bid; S.best_slot[buf][warp] = bslot; }
+          __syncthreads();
+          bk = S.best_key[buf][0]; bid = S.best_id[buf][0]; bslot = S.best_slot[buf][0];
+#pragma unroll
+          for (int w = 1; w < SIM_WARPS; w++) {
+            const uint64_t k2 = S.best_key[buf][w]; const uint32_t i2 = S.best_id[buf][w];
+            if (k2 < bk || (k2 == bk && i2 < bid)) { bk = k2; bid = i2; bslot = S.best_slot[buf][w]; }
+          }
+          buf ^= 1;
+          if (bslot < 0) break;                       // no eligible request left
+          const int i = s_q[bslot];
+          s_cost += s_prompt[i]; s_cnt += 1;
+          if (!(s_cost <= budget && (cfg.batch_cap == 0 || nr + s_cnt <= cfg.batch_cap))) break;
+          adm_cost += s_prompt[i]; adm_cnt += 1;
+          __syncthreads();                            // everyone has read s_q[bslot]
+          if (tid == 0) { s_adm[adm_cnt - 1] = (uint16_t)i; s_q[bslot] = s_q[nq - 1]; }
+          nq -= 1;
+          __syncthreads();
+        }
+      }
+
+      // ---- 4. maturity and the iteration's clock -------------------------------------------
+      if (tid == 0) {
+        int64_t lp = 0;
+        const int64_t mat_next = dev_maturity_next(p, S.plan, adm_cnt, adm_cost, 0, &lp);
+        const int worked = adm_cnt > 0 || nr > 0;
+        S.t1 = S.now + (adm_cnt > 0 ? lp : 0);
+        S.t2 = S.t1 + (nr > 0 ? S.plan.e_d : 0);
+        S.worked = worked; S.mat_next = mat_next; S.nq = nq; S.na = adm_cnt;
+      }
+      __syncthreads();
+      const int64_t t1 = S.t1, t2 = S.t2;
+
+      // ---- 5. commit ---------------------------------------------------------------------------
+      int64_t d_kv = 0;
+      // running batch: one more token each; a request finishes when gen + 1 reaches output_len
+      for (int s = tid; s < nr; s += SIM_THREADS) {
+        const int i = run_cur[s];
+        const int gen_new = it - s_admit_it[i];
+        if ((int64_t)gen_new + 1 >= s_outlen[i]) {
+          s_state[i] = HFX_DONE;
+          a.finish[(int64_t)b + i] = t2;
+          atomicSub(&S.cnt_run[s_cls[i]], 1);
+          d_kv -= (int64_t)s_prompt[i] + gen_new - 1;     // leaves with the context it had before this step
+        } else {
+          run_nxt[atomicAdd(&S.nr_next, 1)] = (uint16_t)i;
+          d_kv += 1;
+        }
+      }
+      // admitted requests: first token at t1
+      for (int s = tid; s < adm_cnt; s += SIM_THREADS) {
+        const int i = s_adm[s];
+        a.first_token[(int64_t)b + i] = t1;
+        s_admit_it[i] = it;
+        atomicSub(&S.cnt_q[s_cls[i]], 1);
+        if (s_outlen[i] <= 1) {
+          s_state[i] = HFX_DONE;
+          a.finish[(int64_t)b + i] = t1;
+        } else {
+          s_state[i] = HFX_RUNNING;
+          run_nxt[atomicAdd(&S.nr_next, 1)] = (uint16_t)i;
+          atomicAdd(&S.cnt_run[s_cls[i]], 1);
+          d_kv += s_prompt[i];
+        }
+      }
+      // oversize prompts seen for the first time
+      {
+        const int no = S.no;
+        for (int s = tid; s < no; s += SIM_THREADS) {
+          const int i = s_adm[cap - 1 - s];
+          s_state[i] = HFX_REJECTED;
+          atomicSub(&S.cnt_q[s_cls[i]], 1);
+        }
+      }
+      d_kv = warp_sum_i64(d_kv);
+      if (lane == 0 && d_kv) atomicAdd(reinterpret_cast<unsigned long long *>(&S.d_kv), (unsigned long long)d_kv);
+      __syncthreads();
+      if (tid == 0) {
+        S.sum_kv += S.d_kv;
+        S.nr = S.nr_next;
+        S.mat = S.mat_next;
+        if (S.worked) S.now = t2;
+        else {
+          int64_t ev = HFX_INF;
+          if (S.plan.mat > S.plan.now) ev = S.plan.mat;
+          int h = S.head;
+          while (h < m && s_cls[h] == ROW_INVALID) h++;     // rows with bad data never arrive
+          if (h < m && s_arr[h] < ev) ev = s_arr[h];
+          if (ev == HFX_INF) S.stop = 1; else S.now = ev;
+        }
+      }
+      { uint16_t *x = run_cur; run_cur = run_nxt; run_nxt = x; }
+      __syncthreads();
+      if (S.stop) break;
+      executed++;
+    }
+
+    // ---- per-request outputs and per-trace metrics ------------------------------------------
+    __syncthreads();
+    const int64_t now_final = S.now;
+    int fin = 0, rej = 0, att = 0;
+    for (int i = tid; i < m; i += SIM_THREADS) {
+      const int64_t g = (int64_t)b + i;
+      const int st = s_state[i];
+      int32_t gen = 0;
+      int64_t first = -1, last = -1;
+      if (st == HFX_RUNNING || st == HFX_DONE) {
+        first = a.first_token[g];
+        if (st == HFX_DONE) { gen = s_outlen[i] > 1 ? s_outlen[i] - 1 : 0; last = a.finish[g]; }
+        else { gen = executed - 1 - s_admit_it[i]; last = gen > 0 ? now_final : first; }
+        a.last_token[g] = last;
+      }
+      a.state[g] = (uint8_t)st;
+      a.gen[g] = gen;
+      const int64_t arr = s_arr[i];
+      const uint8_t cls = s_cls[i];
+      int64_t ttft = -1, tpot = -1;
+      if (cls != ROW_INVALID) {
+        if (st == HFX_REJECTED) rej++;
+        if (st == HFX_RUNNING || st == HFX_DONE) ttft = first - arr;
+        if (st == HFX_DONE) {
+          fin++;
+          const int64_t tp = s_outlen[i] > 1 ? (last - first) / (s_outlen[i] - 1) : 0;
+          if (s_outlen[i] > 1) tpot = tp;
+          const int64_t ttft_slo = p.ttft[cls], tpot_slo = p.tpot[cls];
+          if ((ttft_slo <= 0 || ttft <= ttft_slo) && (tpot_slo <= 0 || tp <= tpot_slo)) att++;
+        }
+      }
+      // park the samples; compaction follows
+      s_arr[i] = ttft;
+      s_dst[i] = tpot;
+    }
+    fin = (int)warp_sum_i64(fin); rej = (int)warp_sum_i64(rej); att = (int)warp_sum_i64(att);
+    if (lane == 0) { atomicAdd(&S.n_fin, fin); atomicAdd(&S.n_rej, rej); atomicAdd(&S.n_att, att); }
+    __syncthreads();
+    // compact the samples (order is irrelevant before the sort): negative = no sample.
+    // In-place compaction by one warp-synchronous pass per array would need care; the arrays are
+    // small, so let thread 0 of each of two warps do it serially.
+    if (tid == 0) { int k = 0; for (int i = 0; i < m; i++) { const int64_t v = s_arr[i]; if (v >= 0) s_arr[k++] = v; } S.n_a = k; }
+    if (tid == 32) { int k = 0; for (int i = 0; i < m; i++) { const int64_t v = s_dst[i]; if (v >= 0) s_dst[k++] = v; } S.n_b = k; }
+    __syncthreads();
+    const int na = S.n_a, nb = S.n_b;
+    sort_i64(s_arr, na);
+    sort_i64(s_dst, nb);
+    __syncthreads();
+    if (tid == 0) {
+      a.iters_executed[j] = executed;
+      a.finished[j] = S.n_fin;
+      a.rejected[j] = S.n_rej;
+      a.attained[j] = S.n_att;
+      a.ttft_p50[j] = nearest_rank(s_arr, na, 50);
+      a.ttft_p99[j] = nearest_rank(s_arr, na, 99);
+      a.tpot_p50[j] = nearest_rank(s_dst, nb, 50);
+      a.tpot_p99[j] = nearest_rank(s_dst, nb, 99);
+      if (a.now_out) a.now_out[j] = now_final;
+    }
+  }
+}
+
+int hfx_sim_configure() {
+  if (cudaFuncSetAttribute(k_sim, cudaFuncAttributeMaxDynamicSharedMemorySize, SIM_MAX_ROWS * SIM_BYTES_PER_ROW) != cudaSuccess)
+    return HFX_E_CUDA;
+  return HFX_OK;
+}
+
+// `trace_off` is already on the device (copied by the caller of this launcher); max_rows is the
+// longest trace, known on the host.
+int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_trace_off, int32_t n_traces,
+                          int32_t max_trace_rows, int32_t iters, const hfx_sim_out *o, uint32_t *d_work_counter) {
+  SimArgs a;
+  a.class_id = t->class_id; a.prompt_len = t->prompt_len; a.output_len = t->output_len; a.arrival = t->arrival_ns;
+  a.req_id = t->req_id; a.weight = s->p.weight_max > 0 ? t->weight : nullptr;
+  a.state = t->state; a.gen = t->gen; a.first_token = t->first_token_ns; a.last_token = t->last_token_ns;
+  a.finish = t->finish_ns; a.trace_off = d_trace_off; a.cfg = s->d_cfg;
+  a.n_traces = n_traces; a.iters = iters;
+  int cap = (max_trace_rows + 15) & ~15;
+  if (cap < 16) cap = 16;
+  a.cap_rows = cap;
+  a.iters_executed = o->iters_executed; a.finished = o->finished; a.rejected = o->rejected; a.attained = o->attained;
+  a.ttft_p50 = o->ttft_p50_ns; a.ttft_p99 = o->ttft_p99_ns; a.tpot_p50 = o->tpot_p50_ns; a.tpot_p99 = o->tpot_p99_ns;
+  a.now_out = o->now_ns;
+  const size_t smem = (size_t)cap * SIM_BYTES_PER_ROW;
+  if (cudaMemsetAsync(d_work_counter, 0, sizeof(uint32_t), s->stream) != cudaSuccess) return HFX_E_CUDA;
+  int per_sm = (int)((200 * 1024) / (smem + 2048));
+  if (per_sm < 1) per_sm = 1;
+  if (per_sm > 8) per_sm = 8;
+  int grid = s->n_sm * per_sm;
+  if (grid > n_traces) grid = n_traces;
+  k_sim<<<grid, SIM_THREADS, smem, s->stream>>>(s->p, a, d_work_counter, s->d_status);
+  s->launches++;
+  return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
+}

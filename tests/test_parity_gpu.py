@@ -1,0 +1,223 @@
+"""Parity of the CUDA path with the oracle, bit for bit, through the C ABI (needs a GPU)."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+from helpers import MS, SEC, make_wl
+from gpu_helpers import assert_step_parity, assert_sim_parity, make_sched, run_sim_gpu
+
+pytestmark = pytest.mark.gpu
+MODES3 = (gen.COLOCATED, gen.PREFILL, gen.DECODE)
+
+
+# ---- the five configurations ---------------------------------------------------------------------
+def test_config1_step_and_simulation():
+    wl = gen.config1()
+    assert_step_parity(wl)
+    assert_step_parity(wl, steps=5, commit=True)
+    assert_sim_parity(wl)
+
+
+@pytest.mark.parametrize("mode", [gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY])
+@pytest.mark.parametrize("inflight", [0.6, 0.02])
+def test_config2_full(mode, inflight):
+    g = assert_step_parity(gen.config2(inflight=inflight, budget_mode=mode))
+    if mode == gen.BUDGET_CAP_ONLY or inflight < 0.1:
+        assert g["adm_count"].sum() > 0
+
+
+def test_config2_committed_steps():
+    assert_step_parity(gen.config2(R=16, rows_per=4096, inflight=0.02), steps=4, commit=True)
+
+
+def test_config3_full():
+    g = assert_step_parity(gen.config3(), optional=False)
+    assert g["adm_count"][:128].sum() > 0 and g["adm_count"][128:].sum() > 0
+
+
+def test_config3_small_committed():
+    assert_step_parity(gen.config3(R=8, rows_per=3000), steps=4, commit=True)
+
+
+def test_config4_full_ten_committed_steps():
+    wl = gen.config4()
+    g = assert_step_parity(wl, steps=wl.steps, commit=True, optional=False)
+
+
+def test_config4_small_all_outputs():
+    assert_step_parity(gen.config4(R=32, n=50_001, steps=3), steps=3, commit=True)
+
+
+def test_config5_subset_of_traces():
+    wl = gen.config5(traces=6)
+    assert_sim_parity(wl)
+
+
+# ---- random and adversarial step cases -----------------------------------------------------------
+@pytest.mark.parametrize("seed", range(16))
+def test_random_tables(seed):
+    wl = gen.random_table(seed, 1000 + 997 * seed, 1 + (seed * 7) % 23, modes=MODES3, tie_heavy=seed % 3 == 0,
+                          batch_cap=(0, 7)[seed % 2], weight_max=(0, 16)[seed % 4 == 1],
+                          budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 2], grouped=seed % 4 == 3)
+    assert_step_parity(wl, steps=3, commit=True)
+    assert_step_parity(wl)
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 5, 255, 257, 2047, 2048, 2049, 4099])
+def test_ragged_sizes_single_replica(n):
+    wl = gen.random_table(100 + n, n, 1, modes=(gen.COLOCATED,))
+    assert_step_parity(wl, steps=2, commit=True)
+
+
+def test_medium_and_oversize_segments():
+    # 2048 < rows <= 16384: medium path; > 16384: global-sort path
+    assert_step_parity(gen.random_table(7, 9000, 1, tie_heavy=True), steps=2, commit=True)
+    assert_step_parity(gen.random_table(8, 16384 + 16385 + 100, 3, grouped=True, modes=MODES3), steps=2, commit=True)
+    wl = gen.random_table(9, 40_001, 1)
+    assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_table(10, 70_000, 2, tie_heavy=True, modes=(gen.DECODE, gen.COLOCATED))
+    assert_step_parity(wl)
+
+
+def test_empty_replicas_and_all_inactive():
+    wl = gen.random_table(11, 500, 40)
+    wl.table["replica_id"][:] = wl.table["replica_id"] % 3 * 13        # most replicas have no rows
+    assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_table(12, 700, 4)
+    wl.table["state"][:] = gen.DONE
+    assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_table(13, 700, 4)
+    wl.table["arrival_ns"][:] = wl.now.max() + SEC                     # everything in the future
+    wl.table["state"][:] = gen.QUEUED
+    assert_step_parity(wl, steps=3, commit=True)
+
+
+def test_bad_rows_are_flagged_not_fatal():
+    wl = gen.random_table(14, 3000, 5, modes=MODES3)
+    t = wl.table
+    t["replica_id"][::17] = 5
+    t["replica_id"][5::31] = -1
+    t["class_id"][3::29] = 200
+    t["prompt_len"][7::37] = -1
+    t["gen"][11::41] = (1 << 24) + 1
+    g = assert_step_parity(wl, steps=2, commit=True)
+    sched = make_sched(wl)
+    assert sched.status() == 0
+    sched.close()
+
+
+def test_ties_in_every_key_field():
+    rows = []
+    for i in range(600):
+        rows.append(dict(prompt_len=64, arrival_ns=0, class_id=i % 2, req_id=(i * 7919) % 600 - 300,
+                         state=gen.RUNNING if i % 3 == 0 else gen.QUEUED, first_token_ns=MS, gen=2))
+    wl = make_wl(rows, [(200 * MS, 30 * MS, 1), (200 * MS, 30 * MS, 1)], now=[50 * MS],
+                 replicas=[(gen.COLOCATED, 8192, 0)])
+    assert_step_parity(wl, steps=2, commit=True)
+
+
+def test_slack_saturation_and_budget_zero():
+    # waits far beyond 2^39 ns saturate the key's slack field: order falls back to req_id
+    rows = [dict(prompt_len=100 + i, arrival_ns=-(i % 5) * 700 * SEC, req_id=1000 - i, class_id=i % 3) for i in range(300)]
+    cls = [(200 * MS, 30 * MS, 0), (0, 0, 0), (1 << 44, 1 << 34, 0)]
+    wl = make_wl(rows, cls, now=[5 * SEC])
+    g = assert_step_parity(wl, steps=2, commit=True)
+    # TPOT <= E_d: nothing is safe
+    rows = [dict(state=gen.RUNNING, prompt_len=4000, gen=50, first_token_ns=0, req_id=i, output_len=900) for i in range(260)]
+    rows += [dict(prompt_len=16, req_id=500 + i) for i in range(50)]
+    g = assert_step_parity(make_wl(rows, [(200 * MS, 30 * MS, 0)], now=[SEC]), steps=2, commit=True)
+    assert g["budget"][0] == 0 and g["adm_count"][0] == 0
+    # zero-token prompts fit a zero budget
+    rows += [dict(prompt_len=0, req_id=900 + i) for i in range(3)]
+    g = assert_step_parity(make_wl(rows, [(200 * MS, 30 * MS, 0)], now=[SEC]), steps=2, commit=True)
+
+
+def test_oversize_prompts_and_batch_cap():
+    wl = gen.random_table(15, 2500, 6, token_cap=512, batch_cap=3, modes=MODES3)
+    assert_step_parity(wl, steps=4, commit=True)
+
+
+def test_scheduler_reuse_and_capacity():
+    wl = gen.random_table(16, 1200, 4)
+    sched = make_sched(wl, max_rows=5000)
+    assert_step_parity(wl, sched=sched)
+    wl2 = gen.random_table(17, 4999, 4)
+    wl2.classes, wl2.replicas = wl.classes, wl.replicas
+    assert_step_parity(wl2, steps=2, commit=True, sched=sched)
+    assert sched.launch_count() > 0
+    sched.close()
+
+
+# ---- simulator ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(4))
+def test_simulator_ragged_traces(seed):
+    wl = gen.random_traces(seed, 40, 0, 300, iters=4000, token_cap=(8192, 600)[seed % 2])
+    assert_sim_parity(wl)
+
+
+def test_simulator_iteration_limits():
+    wl = gen.random_traces(20, 12, 50, 200, iters=0)
+    for iters in (0, 1, 7, 150):
+        assert_sim_parity(wl, iters=iters)
+
+
+def test_simulator_long_trace_and_weights():
+    wl = gen.random_traces(21, 3, 3000, 4096, iters=6000, rate=60.0)
+    wl.weight_max = 8
+    wl.table["weight"][:] = np.random.default_rng(0).integers(0, 12, wl.n_rows).astype(np.int32)
+    assert_sim_parity(wl)
+
+
+def test_simulator_saturated_slack_and_zero_prompts():
+    # a slow model makes waits exceed the 40-bit slack field; zero-token prompts are admitted at budget 0
+    model = (200 * SEC, 40_000, 2, 8_000_000, 100_000, 20)
+    cls = [(1 << 44, 30 * MS, 0), (200 * MS, 30 * MS, 0), (0, 0, 0)]
+    wl = gen.random_traces(22, 6, 20, 60, iters=3000, model=model, classes=cls, out_hi=8)
+    wl.table["prompt_len"][::9] = 0
+    assert_sim_parity(wl)
+
+
+def test_simulator_bad_rows():
+    wl = gen.random_traces(23, 5, 50, 100, iters=2000)
+    wl.table["class_id"][::13] = 99
+    wl.table["prompt_len"][5::17] = -3
+    res, cols, st = run_sim_gpu(wl)
+    assert st == 2 | 4
+    assert_sim_parity(wl)
+
+
+# ---- argument errors ---------------------------------------------------------------------------------
+def test_argument_errors():
+    import paper_2508_15919_b200 as hfx
+    wl = gen.random_table(30, 64, 2)
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    now = torch.from_numpy(wl.now).cuda(); mat = torch.from_numpy(wl.maturity).cuda()
+    out = hfx.StepOut(64, 2)
+    bad = hfx.StepOut(64, 2)
+    bad.t["order"] = torch.zeros(65, dtype=torch.int32, device="cuda")[1:]
+    with pytest.raises(hfx.HfxError) as e:
+        sched.step(tab, now, mat, bad)
+    assert e.value.code == -2
+    bad = hfx.StepOut(64, 2)
+    bad.t["admit"] = None
+    with pytest.raises(hfx.HfxError) as e:
+        sched.step(tab, now, mat, bad)
+    assert e.value.code == -1
+    big = hfx.DeviceTable.from_numpy(gen.random_table(31, 65, 2).table)
+    with pytest.raises(hfx.HfxError) as e:
+        sched.step(big, now, mat, out)
+    assert e.value.code == -3
+    tab.cols["output_len"] = None
+    with pytest.raises(hfx.HfxError) as e:
+        sched.step(tab, now, mat, out, commit=True)
+    assert e.value.code == -1
+    sched.step(tab, now, mat, out)          # still usable, and output_len is optional without commit
+    assert sched.status() == 0
+    with pytest.raises(hfx.HfxError):
+        hfx.Scheduler((1, 1, 1 << 13, 1, 1, 1), wl.classes, wl.replicas, 10)
+    with pytest.raises(hfx.HfxError):
+        hfx.Scheduler(wl.model, wl.classes, [(3, 100, 0)], 10)
+    sched.close()
