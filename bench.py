@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the scheduler hot path: requests scheduled per second per hfx_sched_step on the
+1,048,576-request / 1024-replica shared-queue workload (rows interleaved across replicas, committed
+steps with in-flight state carried over), plus simulated scheduler iterations per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-sim] [--no-cpu]
+
+One "step" is one hfx_sched_step(COMMIT) over the whole table: per-replica aggregates, E_d, safe
+budget, per-row slack and key, per-replica sort, segmented-scan admission, maturity update, commit.
+Steps are timed one by one with CUDA events on the launching stream; between steps L2 is flushed by
+writing a 256 MiB buffer (outside the events), and the table is restored to its initial state every
+10 steps (outside the events) so that the workload stays the one the configuration names.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "requests_scheduled_per_sec_per_hfx_sched_step"
+UNIT = "requests/s"
+ALGO_BYTES_PER_ROW = 51            # 38 B read (incl. priority weight) + 13 B written per row and step
+# algorithmic bytes per row of each kernel (what that kernel must move once)
+KERNEL_BYTES_PER_ROW = {"k_count": 4, "k_regroup": 42, "k_segment(small)": 13, "k_segment(medium)": 13,
+                        "k_big": 13, "k_step_fused": 51}
+STEPS_PER_EPISODE = 10
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel on this workload,
+# taken from the ncu capture summarised under profiles/; absent = no capture of the current kernel
+NCU_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _workload(rank: int, args):
+    return gen.config4(seed=4 + rank, R=args.replicas, n=args.rows, steps=STEPS_PER_EPISODE)
+
+
+def _workload_name(n, R):
+    return ("config4: shared queue, %d requests over %d replicas (rows interleaved), 5 SLO tiers, priority "
+            "weights, Pareto prompts, committed steps with in-flight state carried over" % (n, R))
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: one step = one oracle step (with commit) over
+    the same table.  Rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    wl0 = _workload(0, args)
+    wl = wl0.copy()
+    times = []
+    for s in range(args.warmup + args.steps):
+        if s % STEPS_PER_EPISODE == 0:
+            wl = wl0.copy()
+        t0 = time.perf_counter()
+        oracle.step(wl, commit=True)
+        dt = time.perf_counter() - t0
+        if s >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    val = wl0.n_rows / (ms * 1e-3)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int64", "data": "synthetic",
+            "config": {"workload": _workload_name(wl0.n_rows, wl0.n_replicas),
+                       "note": "CPU oracle (plain single-threaded C), one oracle step per bench step, full table"},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": "%d full-table committed steps of the %d-row workload" % (args.steps, wl0.n_rows)},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2508_15919_b200 as hfx
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the scheduler library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    hfx.load_library()
+    wl = _workload(rank, args)
+    n, R = wl.n_rows, wl.n_replicas
+    sched = hfx.Scheduler(wl.model, wl.classes, wl.replicas, n, budget_mode=wl.budget_mode, weight_max=wl.weight_max)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    init = {k: v.clone() for k, v in tab.cols.items()}
+    now0 = torch.from_numpy(wl.now).cuda(); mat0 = torch.from_numpy(wl.maturity).cuda()
+    now = now0.clone(); mat = mat0.clone()
+    out = hfx.StepOut(n, R, optional=False)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def restore():
+        for k in ("state", "gen", "first_token_ns", "last_token_ns", "finish_ns"):
+            tab.cols[k].copy_(init[k])
+        now.copy_(now0); mat.copy_(mat0)
+
+    def timed_pass(steps, warmup, profile=False):
+        """Per-step device times (ms) of `steps` steps after `warmup` untimed ones."""
+        evs = []
+        sched.set_profiling(False)
+        for s in range(warmup + steps):
+            if s == warmup:
+                sched.get_profile()
+                sched.set_profiling(profile)
+            if s % STEPS_PER_EPISODE == 0:
+                restore()
+            flush.fill_(s & 0xff)                       # L2 flush, outside the events
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            sched.step(tab, now, mat, out, commit=True)
+            b.record(stream)
+            if s >= warmup:
+                evs.append((a, b))
+        torch.cuda.synchronize()
+        sched.set_profiling(False)
+        return [a.elapsed_time(b) for a, b in evs]
+
+    # ---- device-resident timing: K steps bracketed by barrier + synchronize -----------------------
+    timed_pass(0, max(args.warmup, 3))
+    clocks = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        clocks.start()
+    launches0 = sched.launch_count()
+    t_wall0 = time.perf_counter()
+    times = timed_pass(args.steps, 0)
+    barrier()
+    wall = time.perf_counter() - t_wall0
+    launches = sched.launch_count() - launches0
+    clk = clocks.stop() if rank == 0 else None
+    status = sched.status()
+    step_ms = float(np.sum(times)) / args.steps
+    t = torch.tensor([step_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    step_ms_max = float(t.item())
+    value = world * n / (step_ms_max * 1e-3)
+
+    # ---- per-kernel times over the same K steps (events inside the library) ------------------------
+    timed_pass(args.steps, 1, profile=True)
+    prof = sched.get_profile()
+
+    # ---- end to end: host buffers in, results out, through the C ABI --------------------------------
+    in_cols = ["replica_id", "class_id", "state", "prompt_len", "output_len", "gen", "arrival_ns", "first_token_ns",
+               "req_id", "weight"]
+    pinned = {k: init[k].cpu().pin_memory() for k in in_cols}
+    pin_now = now0.cpu().pin_memory(); pin_mat = mat0.cpu().pin_memory()
+    res_host = {k: torch.empty_like(out.t[k], device="cpu").pin_memory()
+                for k in ("admit", "order", "seg_off", "budget", "adm_cost", "adm_count", "maturity_next")}
+    h2d = sum(v.numel() * v.element_size() for v in pinned.values()) + 2 * pin_now.numel() * 8
+    d2h = sum(v.numel() * v.element_size() for v in res_host.values())
+
+    def e2e_step():
+        for k in in_cols:
+            tab.cols[k].copy_(pinned[k], non_blocking=True)
+        now.copy_(pin_now, non_blocking=True); mat.copy_(pin_mat, non_blocking=True)
+        sched.step(tab, now, mat, out, commit=True)
+        for k, v in res_host.items():
+            v.copy_(out.t[k], non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e_evs = []
+    for _ in range(e2e_steps):
+        flush.fill_(1)
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(stream); e2e_step(); b.record(stream)
+        e_evs.append((a, b))
+    barrier()
+    e2e_ms = float(np.mean([a.elapsed_time(b) for a, b in e_evs]))
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms_max = float(t.item())
+    e2e_value = world * n / (e2e_ms_max * 1e-3)
+
+    # ---- simulator: scheduler iterations per second (rank 0, outside the timed steps) --------------
+    sim = None
+    if rank == 0 and not args.no_sim:
+        swl = gen.config5(traces=args.sim_traces, iters=args.sim_iters)
+        ssched = hfx.Scheduler(swl.model, swl.classes, swl.replicas, swl.n_rows)
+        stab = hfx.DeviceTable.from_numpy(swl.table)
+        sout = hfx.SimOut(args.sim_traces)
+        ssched.sim_run(stab, swl.trace_off, 50, sout)           # warm-up
+        torch.cuda.synchronize()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(stream); ssched.sim_run(stab, swl.trace_off, swl.sim_iters, sout); b.record(stream)
+        torch.cuda.synchronize()
+        sim_ms = a.elapsed_time(b)
+        so = sout.to_numpy()
+        iters_total = int(so["iters_executed"].sum())
+        sim = {"workload": "config5: %d traces x 2048 requests, %d iterations" % (args.sim_traces, args.sim_iters),
+               "sched_iters_per_sec": iters_total / (sim_ms * 1e-3), "ms": sim_ms, "iterations_executed": iters_total,
+               "mean_attainment": float((so["attained"] / 2048.0).mean()), "status": ssched.status()}
+        ssched.close()
+
+    # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only -----------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        import oracle
+        oracle.build()
+        cw = wl.copy()
+        k_cpu = 0
+        t0 = time.perf_counter()
+        while k_cpu < STEPS_PER_EPISODE and (time.perf_counter() - t0 < 12 or k_cpu < 2):
+            oracle.step(cw, commit=True)
+            k_cpu += 1
+        cpu_s = (time.perf_counter() - t0) / k_cpu
+        cpu = {"value": n / cpu_s, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "%d committed steps of the full %d-row table" % (k_cpu, n)}
+
+    if rank == 0:
+        peak, peak_kind = _peaks()
+        dom = max(prof.items(), key=lambda kv: kv[1]["ms"])[0] if prof else None
+        roof = None
+        if dom:
+            per_launch_ms = prof[dom]["ms"] / prof[dom]["launches"]
+            bpr = KERNEL_BYTES_PER_ROW.get(dom, ALGO_BYTES_PER_ROW)
+            achieved = bpr * n / (per_launch_ms * 1e-3) / 1e9
+            step_gbs = ALGO_BYTES_PER_ROW * n / (step_ms_max * 1e-3) / 1e9
+            tot = sum(x["ms"] for x in prof.values())
+            roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES.get(dom),
+                    "algorithmic_bytes_per_launch": bpr * n, "ms_per_launch": per_launch_ms,
+                    "step": {"algorithmic_bytes": ALGO_BYTES_PER_ROW * n, "achieved": step_gbs,
+                             "frac": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / 8000.0},
+                    "kernels": {k: {"ms_per_launch": v["ms"] / v["launches"], "launches": v["launches"],
+                                    "share": v["ms"] / tot} for k, v in prof.items()}}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+                "config": {"workload": _workload_name(n, R),
+                           "rows_per_gpu": n, "replicas_per_gpu": R, "parallelism": "replica shards, no collective",
+                           "l2": "flushed between steps (256 MiB write, outside the per-step events)",
+                           "episode": "table restored every %d steps, outside the events" % STEPS_PER_EPISODE,
+                           "wall_s_timed_region": wall},
+                "clocks": clk, "gpu_launches": launches, "device_status": status,
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "ms_per_step": e2e_ms_max},
+                "roofline": roof, "cpu_baseline": cpu, "sim": sim}
+        print(json.dumps(line))
+    sched.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="hfx", choices=["hfx", "reference"])
+    ap.add_argument("--rows", type=int, default=1 << 20)
+    ap.add_argument("--replicas", type=int, default=1024)
+    ap.add_argument("--sim-traces", type=int, default=4096)
+    ap.add_argument("--sim-iters", type=int, default=10000)
+    ap.add_argument("--no-sim", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -255,6 +255,22 @@ int hfx_sched_status(hfx_sched *s, uint32_t *status_word);
 /* Number of kernels the library has launched on behalf of `s` so far. */
 int64_t hfx_sched_launch_count(const hfx_sched *s);
 
+/* Per-kernel timing (a measurement aid; the paper has no counterpart).  While
+ * profiling is on, every kernel the library launches is bracketed by CUDA
+ * events on the scheduler's stream.  hfx_sched_get_profile synchronises the
+ * stream, adds the elapsed times of all brackets recorded since the last call
+ * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 offsets,
+ * 2 regroup, 3 segment (small), 4 segment (medium), 5 oversize path,
+ * 6 simulator; hfx_kernel_name gives the name of a slot (NULL past the end). */
+#define HFX_N_KERNELS 8
+typedef struct hfx_profile {
+  double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
+  int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */
+} hfx_profile;
+int hfx_sched_set_profiling(hfx_sched *s, int on);
+int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out);
+const char *hfx_kernel_name(int slot);
+
 void hfx_sched_destroy(hfx_sched *s);
 
 /* Static, never NULL. */

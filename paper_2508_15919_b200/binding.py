@@ -20,7 +20,9 @@ ST_BAD_REPLICA, ST_BAD_CLASS, ST_BAD_LEN, ST_TIMEOUT = 1, 2, 4, 8
 E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
-                    "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror"]
+                    "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
+                    "hfx_sched_get_profile", "hfx_kernel_name"]
+N_KERNELS = 8
 
 
 class HfxError(RuntimeError):
@@ -78,6 +80,10 @@ SIM_OUT_FIELDS = [("iters_executed", torch.int32), ("finished", torch.int32), ("
                   ("tpot_p50_ns", torch.int64), ("tpot_p99_ns", torch.int64), ("now_ns", torch.int64)]
 
 
+class _Profile(C.Structure):
+    _fields_ = [("ms", C.c_double * 8), ("launches", C.c_int64 * 8)]
+
+
 class _SimOut(C.Structure):
     _fields_ = [(k, C.c_void_p) for k, _ in SIM_OUT_FIELDS]
 
@@ -108,6 +114,12 @@ def load_library():
     L.hfx_sched_launch_count.argtypes = [C.c_void_p]
     L.hfx_sched_destroy.restype = None
     L.hfx_sched_destroy.argtypes = [C.c_void_p]
+    L.hfx_sched_set_profiling.restype = C.c_int
+    L.hfx_sched_set_profiling.argtypes = [C.c_void_p, C.c_int]
+    L.hfx_sched_get_profile.restype = C.c_int
+    L.hfx_sched_get_profile.argtypes = [C.c_void_p, C.POINTER(_Profile)]
+    L.hfx_kernel_name.restype = C.c_char_p
+    L.hfx_kernel_name.argtypes = [C.c_int]
     L.hfx_strerror.restype = C.c_char_p
     L.hfx_strerror.argtypes = [C.c_int]
     _lib = L
@@ -243,6 +255,24 @@ class Scheduler:
         if rc not in (0, E_TIMEOUT):
             raise HfxError(rc, "hfx_sched_status")
         return int(w.value)
+
+    def set_profiling(self, on: bool):
+        rc = self._L.hfx_sched_set_profiling(self._h, int(on))
+        if rc != 0:
+            raise HfxError(rc, "hfx_sched_set_profiling")
+
+    def get_profile(self) -> Dict[str, Dict[str, float]]:
+        """Per-kernel device time (ms) and launches recorded since the last call."""
+        pr = _Profile()
+        rc = self._L.hfx_sched_get_profile(self._h, C.byref(pr))
+        if rc != 0:
+            raise HfxError(rc, "hfx_sched_get_profile")
+        out = {}
+        for i in range(N_KERNELS):
+            name = self._L.hfx_kernel_name(i)
+            if name and pr.launches[i]:
+                out[name.decode()] = {"ms": float(pr.ms[i]), "launches": int(pr.launches[i])}
+        return out
 
     def launch_count(self) -> int:
         return int(self._L.hfx_sched_launch_count(self._h))

@@ -83,6 +83,8 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   s->opts = *opts; s->max_rows = max_rows; s->n_sm = n_sm;
   s->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   s->launches = 0;
+  s->profiling = 0;
+  s->brackets = new (std::nothrow) std::vector<HfxBracket>();
 
   const size_t R2 = (size_t)n_replicas + 2;
   bool ok = true;
@@ -126,6 +128,10 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();
+  if (s->brackets) {
+    for (HfxBracket &b : *s->brackets) { cudaEventDestroy(b.a); cudaEventDestroy(b.b); }
+    delete s->brackets;
+  }
   delete[] h->h_cfg;
   delete h;
 }
@@ -205,3 +211,31 @@ extern "C" int hfx_sched_status(hfx_sched *s, uint32_t *status_word) {
 }
 
 extern "C" int64_t hfx_sched_launch_count(const hfx_sched *s) { return s ? s->launches : 0; }
+
+extern "C" int hfx_sched_set_profiling(hfx_sched *s, int on) {
+  if (!s) return HFX_E_ARG;
+  s->profiling = on ? 1 : 0;
+  return HFX_OK;
+}
+
+extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
+  if (!s || !out) return HFX_E_ARG;
+  if (cudaStreamSynchronize(s->stream) != cudaSuccess) { cudaGetLastError(); return HFX_E_CUDA; }
+  if (!s->brackets) return HFX_OK;
+  for (HfxBracket &b : *s->brackets) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, b.a, b.b) == cudaSuccess && b.slot >= 0 && b.slot < HFX_N_KERNELS) {
+      out->ms[b.slot] += ms;
+      out->launches[b.slot] += 1;
+    }
+    cudaEventDestroy(b.a); cudaEventDestroy(b.b);
+  }
+  s->brackets->clear();
+  cudaGetLastError();
+  return HFX_OK;
+}
+
+extern "C" const char *hfx_kernel_name(int slot) {
+  static const char *names[] = {"k_count", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)", "k_big", "k_sim"};
+  return (slot >= 0 && slot < 7) ? names[slot] : nullptr;
+}

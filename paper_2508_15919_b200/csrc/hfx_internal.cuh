@@ -50,6 +50,12 @@ struct __align__(16) HfxRec {
 };
 static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
+#include <vector>
+
+enum { KSLOT_COUNT = 0, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM };
+
+struct HfxBracket { cudaEvent_t a, b; int slot; };
+
 struct hfx_sched {
   HfxParams p;
   hfx_options opts;
@@ -57,6 +63,8 @@ struct hfx_sched {
   int n_sm;
   cudaStream_t stream;
   int64_t launches;
+  int profiling;
+  std::vector<HfxBracket> *brackets;
   // device
   hfx_replica_cfg *d_cfg;   // [R]
   uint32_t *d_status;       // sticky status word
@@ -215,6 +223,24 @@ __device__ __forceinline__ int32_t warp_incl_scan_i32(int32_t v, int lane) {
   for (int o = 1; o < 32; o <<= 1) { int32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
   return v;
 }
+
+// Brackets one kernel launch with events when profiling is on; counts the launch either way.
+struct KernelScope {
+  hfx_sched *s; HfxBracket br; bool on;
+  KernelScope(hfx_sched *s_, int slot) : s(s_), on(false) {
+    s->launches++;
+    if (s->profiling && s->brackets) {
+      br.slot = slot;
+      if (cudaEventCreate(&br.a) == cudaSuccess && cudaEventCreate(&br.b) == cudaSuccess) {
+        cudaEventRecord(br.a, s->stream);
+        on = true;
+      }
+    }
+  }
+  ~KernelScope() {
+    if (on) { cudaEventRecord(br.b, s->stream); s->brackets->push_back(br); }
+  }
+};
 
 // host-side launchers implemented in the .cu files
 int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o, uint32_t flags);

@@ -114,7 +114,6 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     __syncthreads();
     for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; }
     uint32_t bad = 0;
-    bool unsorted = false;
     for (int i = tid; i < m; i += SIM_THREADS) {
       const int64_t g = (int64_t)b + i;
       const uint32_t cls = a.class_id[g];
@@ -123,7 +122,6 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       bool ok = true;
       if (cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
       if (prompt < 0 || prompt > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }
-      if (i + 1 < m && a.arrival[g + 1] < arr) unsorted = true;
       s_arr[i] = arr;
       s_prompt[i] = prompt;
       if (prompt == 0) S.zero_prompt = 1;   // a zero-token prompt fits a zero budget
@@ -147,9 +145,8 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       a.first_token[g] = -1; a.last_token[g] = -1; a.finish[g] = -1;
     }
     if (bad) atomicOr(status, bad);
-    // reading: an unsorted trace is a caller error; it is simulated as given (the head pointer
-    // stops at the first row that has not arrived), no fault can result
-    (void)unsorted;
+    // A trace that is not sorted by arrival is a caller error; it is simulated as given (the head
+    // pointer stops at the first row that has not arrived) and cannot fault.
     __syncthreads();
 
     int executed = 0;
@@ -406,7 +403,9 @@ int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_tra
   if (per_sm > 8) per_sm = 8;
   int grid = s->n_sm * per_sm;
   if (grid > n_traces) grid = n_traces;
-  k_sim<<<grid, SIM_THREADS, smem, s->stream>>>(s->p, a, d_work_counter, s->d_status);
-  s->launches++;
+  {
+    KernelScope ks(s, KSLOT_SIM);
+    k_sim<<<grid, SIM_THREADS, smem, s->stream>>>(s->p, a, d_work_counter, s->d_status);
+  }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }

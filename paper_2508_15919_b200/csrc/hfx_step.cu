@@ -799,8 +799,6 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-static inline bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
-
 int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o,
                     uint32_t flags) {
   const int R = s->p.n_replicas;
@@ -813,19 +811,21 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
   const int grid_stream = s->n_sm * 4;
   {
     const size_t sm = (R + 1 <= HIST_SMEM_MAX) ? sizeof(uint32_t) * (R + 1) : 0;
+    KernelScope ks(s, KSLOT_COUNT);
     k_count<<<grid_stream, 512, sm, stream>>>(t->replica_id, n, R, s->d_seg_count, s->d_status);
-    s->launches++;
   }
-  k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, R, s->d_seg_begin, s->d_cursor, o->seg_off, s->d_list, s->d_list_n);
-  s->launches++;
+  {
+    KernelScope ks(s, KSLOT_OFFSETS);
+    k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, R, s->d_seg_begin, s->d_cursor, o->seg_off, s->d_list, s->d_list_n);
+  }
   {
     RegroupArgs a;
     a.replica_id = t->replica_id; a.class_id = t->class_id; a.state = t->state; a.prompt_len = t->prompt_len;
     a.output_len = t->output_len; a.gen = t->gen; a.arrival = t->arrival_ns; a.first_token = t->first_token_ns;
     a.req_id = t->req_id; a.weight = s->p.weight_max > 0 ? t->weight : nullptr;
     a.now = st->now_ns; a.mat = st->maturity_ns; a.cfg = s->d_cfg; a.pred_ttft = o->pred_ttft_ns; a.n = n;
+    KernelScope ks(s, KSLOT_REGROUP);
     k_regroup<<<s->n_sm * 8, 256, 0, stream>>>(s->p, a, s->d_cursor, s->d_rec, s->d_status);
-    s->launches++;
   }
   SegArgs sa;
   sa.state = t->state; sa.gen = t->gen; sa.first_token = t->first_token_ns; sa.last_token = t->last_token_ns;
@@ -836,15 +836,15 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
   sa.flags = flags;
   {
     const int grid = R + 1 < s->n_sm * 8 ? R + 1 : s->n_sm * 8;
+    KernelScope ks(s, KSLOT_SEG_SMALL);
     k_segment<<<grid, THREADS_SMALL, SEG_SMALL * 12, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_list,
                                                                 s->d_list_n, SEG_SMALL);
-    s->launches++;
   }
   if (n > SEG_SMALL) {
     const int grid = R + 1 < s->n_sm ? R + 1 : s->n_sm;
+    KernelScope ks(s, KSLOT_SEG_MED);
     k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_list + (R + 1),
                                                             s->d_list_n + 1, SEG_MED);
-    s->launches++;
   }
   if (n > SEG_MED) {
     const int32_t *list = s->d_list + 2 * (size_t)(R + 1);
@@ -854,9 +854,9 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
     void *args[] = {(void *)&s->p, (void *)&sa, (void *)&s->d_rec, (void *)&s->d_seg_begin, (void *)&list,
                     (void *)&list_n, (void *)&s->d_big_hi, (void *)&s->d_big_lo, (void *)&big_idx,
                     (void *)&s->d_barrier, (void *)&s->d_status};
+    KernelScope ks(s, KSLOT_BIG);
     if (cudaLaunchCooperativeKernel((void *)k_big, dim3(s->n_sm), dim3(512), args, 0, stream) != cudaSuccess)
       return HFX_E_CUDA;
-    s->launches++;
   }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }
