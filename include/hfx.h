@@ -273,6 +273,31 @@ const char *hfx_kernel_name(int slot);
 
 void hfx_sched_destroy(hfx_sched *s);
 
+/* Rows per replica without any allocation (the paper has no counterpart; this
+ * is a service entry for callers that cannot call cudaMalloc: a process whose
+ * device memory is owned entirely by a framework's allocator, a plugin inside
+ * another component's memory budget, a path where an allocation's implicit
+ * synchronisation is not acceptable).  It needs no hfx_sched.
+ * Computes what hfx_sched_step returns in seg_off: seg_off[r] is the number of
+ * rows whose replica_id is below r (the start of replica r in a replica-major
+ * order) for r = 0 .. n_replicas, so seg_off[n_replicas] counts the rows with a
+ * valid id; *n_bad (optional) receives the number of rows whose id is outside
+ * [0, n_replicas).  `replica_id` [n_rows], `seg_off` [n_replicas+1] and `n_bad`
+ * are device pointers (4-byte aligned) owned by the caller; the call is
+ * asynchronous on `cuda_stream`.
+ * The counters live in a fixed 16 KiB array inside the library image, held by
+ * every GPU that loads the library until the process exits; hence the limit
+ * n_replicas <= HFX_NOALLOC_MAX_REPLICAS (HFX_E_CAPACITY beyond it, and for
+ * n_rows > 2^27).  The first call on each device looks up the array's device
+ * address (make that first call outside any stream capture); no call allocates
+ * or frees memory.  All calls on a device share the array and each call clears
+ * what it uses, so two calls whose kernels overlap on the GPU (different
+ * streams, different threads) race: serialise them.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_CUDA. */
+#define HFX_NOALLOC_MAX_REPLICAS 4096
+int hfx_count_rows_noalloc(const int32_t *replica_id, int64_t n_rows, int32_t n_replicas,
+                           int32_t *seg_off, uint32_t *n_bad, void *cuda_stream);
+
 /* Static, never NULL. */
 const char *hfx_strerror(int code);
 

@@ -21,7 +21,8 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_kernel_name"]
+                    "hfx_sched_get_profile", "hfx_kernel_name", "hfx_count_rows_noalloc"]
+NOALLOC_MAX_REPLICAS = 4096
 N_KERNELS = 8
 
 
@@ -120,6 +121,8 @@ def load_library():
     L.hfx_sched_get_profile.argtypes = [C.c_void_p, C.POINTER(_Profile)]
     L.hfx_kernel_name.restype = C.c_char_p
     L.hfx_kernel_name.argtypes = [C.c_int]
+    L.hfx_count_rows_noalloc.restype = C.c_int
+    L.hfx_count_rows_noalloc.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     L.hfx_strerror.restype = C.c_char_p
     L.hfx_strerror.argtypes = [C.c_int]
     _lib = L
@@ -128,6 +131,21 @@ def load_library():
 
 def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else t.data_ptr()
+
+
+def count_rows_noalloc(replica_id: torch.Tensor, n_replicas: int, seg_off: torch.Tensor,
+                       n_bad: Optional[torch.Tensor] = None) -> None:
+    """hfx_count_rows_noalloc on the current stream: fills seg_off (int32, n_replicas + 1) with the
+    start of every replica in a replica-major order, using no device allocation of its own (the
+    caller passes every buffer; the counters are a fixed array inside the library).  For callers
+    that may not allocate; at most NOALLOC_MAX_REPLICAS replicas."""
+    L = load_library()
+    assert replica_id.dtype == torch.int32 and seg_off.dtype == torch.int32 and seg_off.numel() >= n_replicas + 1
+    rc = L.hfx_count_rows_noalloc(_ptr(replica_id) if replica_id.numel() else None, int(replica_id.numel()),
+                                  int(n_replicas), _ptr(seg_off), _ptr(n_bad),
+                                  C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if rc != 0:
+        raise HfxError(rc, "hfx_count_rows_noalloc")
 
 
 class DeviceTable:
