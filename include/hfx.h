@@ -259,9 +259,10 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * profiling is on, every kernel the library launches is bracketed by CUDA
  * events on the scheduler's stream.  hfx_sched_get_profile synchronises the
  * stream, adds the elapsed times of all brackets recorded since the last call
- * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 offsets,
- * 2 regroup, 3 segment (small), 4 segment (medium), 5 oversize path,
- * 6 simulator; hfx_kernel_name gives the name of a slot (NULL past the end). */
+ * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
+ * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
+ * 6 oversize path, 7 simulator; hfx_kernel_name gives the name of a slot
+ * (NULL past the end). */
 #define HFX_N_KERNELS 8
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */

@@ -4,7 +4,8 @@
 
 #include "hfx_internal.cuh"
 
-int hfx_step_configure();
+int hfx_regroup_configure();
+int hfx_segment_configure();
 int hfx_sim_configure();
 int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_trace_off, int32_t n_traces,
                           int32_t max_trace_rows, int32_t iters, const hfx_sim_out *o, uint32_t *d_work_counter);
@@ -65,7 +66,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     cudaGetLastError();
     return HFX_E_CUDA;
   }
-  if (hfx_step_configure() != HFX_OK || hfx_sim_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
+  if (hfx_regroup_configure() != HFX_OK || hfx_segment_configure() != HFX_OK || hfx_sim_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
 
   hfx_sched_host *h = new (std::nothrow) hfx_sched_host();
   if (!h) return HFX_E_NOMEM;
@@ -93,8 +94,17 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   ok = ok && cudaMalloc(&s->d_seg_count, sizeof(uint32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_seg_begin, sizeof(uint32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_cursor, sizeof(uint32_t) * R2) == cudaSuccess;
-  ok = ok && cudaMalloc(&s->d_list, sizeof(int32_t) * 3 * R2) == cudaSuccess;
-  ok = ok && cudaMalloc(&s->d_list_n, 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_flags, 256) == cudaSuccess;
+  {
+    int32_t tile_rows = 0, n_tiles = 0;
+    hfx_tile_shape(max_rows, &tile_rows, &n_tiles);
+    if (n_tiles < HFX_TILE_BLOCKS) n_tiles = HFX_TILE_BLOCKS;
+    s->tile_blocks_max = 0;
+    if (n_replicas <= HFX_TILE_REPLICAS_MAX && (int64_t)n_tiles * (n_replicas + 1) <= HFX_TILE_MATRIX_MAX) {
+      ok = ok && cudaMalloc(&s->d_tile_hist, sizeof(uint32_t) * (size_t)n_tiles * ((size_t)n_replicas + 1)) == cudaSuccess;
+      s->tile_blocks_max = n_tiles;
+    }
+  }
   ok = ok && cudaMalloc(&s->d_rec, sizeof(HfxRec) * (size_t)max_rows) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_barrier, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&h->d_trace_off, sizeof(int32_t) * R2) == cudaSuccess;
@@ -124,7 +134,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   hfx_sched_host *h = reinterpret_cast<hfx_sched_host *>(s);
   cudaStreamSynchronize(s->stream);
   cudaFree(s->d_cfg); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
-  cudaFree(s->d_cursor); cudaFree(s->d_list); cudaFree(s->d_list_n); cudaFree(s->d_rec);
+  cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
   cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();
@@ -236,6 +246,7 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 }
 
 extern "C" const char *hfx_kernel_name(int slot) {
-  static const char *names[] = {"k_count", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)", "k_big", "k_sim"};
-  return (slot >= 0 && slot < 7) ? names[slot] : nullptr;
+  static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
+                                "k_big", "k_sim"};
+  return (slot >= 0 && slot < 8) ? names[slot] : nullptr;
 }

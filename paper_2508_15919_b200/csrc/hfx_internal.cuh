@@ -52,7 +52,13 @@ static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
 #include <vector>
 
-enum { KSLOT_COUNT = 0, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM };
+enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM };
+
+// tiling of the streaming passes: about this many tiles (2 per SM), each at most this many rows
+#define HFX_TILE_BLOCKS 296
+#define HFX_TILE_ROWS_MAX 8192
+#define HFX_TILE_MATRIX_MAX (INT64_C(8) << 20)   // entries of the tile-histogram matrix (32 MiB)
+#define HFX_TILE_REPLICAS_MAX 8191               // replicas whose counters fit in shared memory
 
 struct HfxBracket { cudaEvent_t a, b; int slot; };
 
@@ -71,8 +77,9 @@ struct hfx_sched {
   uint32_t *d_seg_count;    // [R+2] rows per replica (+ the bad-replica bucket R)
   uint32_t *d_seg_begin;    // [R+2] exclusive prefix
   uint32_t *d_cursor;       // [R+2] fill cursors of the regroup pass
-  int32_t *d_list;          // [3][R+1] replicas by segment-size class
-  uint32_t *d_list_n;       // [4]
+  uint32_t *d_tile_hist;    // [tile_blocks_max][R+1] per-tile histograms (nullptr: atomic mode only)
+  int32_t tile_blocks_max;
+  uint32_t *d_flags;        // [0] records in req_id order, [1] largest segment
   HfxRec *d_rec;            // [max_rows]
   uint64_t *d_big_hi;       // sort scratch of oversize segments
   uint32_t *d_big_lo;
@@ -242,7 +249,32 @@ struct KernelScope {
   }
 };
 
+// ---- kernel argument blocks ------------------------------------------------------------------
+struct RegroupArgs {
+  const int32_t *replica_id; const uint8_t *class_id; const uint8_t *state; const int32_t *prompt_len;
+  const int32_t *output_len; const int32_t *gen; const int64_t *arrival; const int64_t *first_token;
+  const int32_t *req_id; const int32_t *weight;
+  const int64_t *now; const int64_t *mat; const hfx_replica_cfg *cfg;
+  int64_t *pred_ttft;    // optional output
+  int64_t n;
+};
+
+struct SegArgs {
+  // table columns written by COMMIT
+  uint8_t *state; int32_t *gen; int64_t *first_token; int64_t *last_token; int64_t *finish;
+  // replica state
+  int64_t *now; int64_t *mat; const hfx_replica_cfg *cfg;
+  // outputs
+  int64_t *slack; int64_t *pred_tpot; uint64_t *key; int32_t *order; uint8_t *admit; int32_t *admitted_rows;
+  int64_t *budget; int64_t *e_d; int32_t *n_run; int64_t *sum_kv; int64_t *adm_cost; int32_t *adm_count;
+  int64_t *maturity_next;
+  uint32_t flags;
+};
+
 // host-side launchers implemented in the .cu files
+void hfx_tile_shape(int64_t n, int32_t *tile_rows, int32_t *n_tiles);
+int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off);
+int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n);
 int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o, uint32_t flags);
 int hfx_launch_sim(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
                    const hfx_sim_out *o);

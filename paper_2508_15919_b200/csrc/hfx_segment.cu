@@ -1,0 +1,624 @@
+// Per-replica work after the regroup: aggregates of the running batch, E_d, the safe budget
+// (Eq. 3), final slack and key, the sort, segmented-scan admission, maturity, commit.
+//   k_segment  one block per replica whose rows fit in shared memory (two size classes)
+//   k_big      cooperative kernel for larger replicas (global sort with bounded grid barriers)
+#include "hfx_internal.cuh"
+
+#define SEG_SMALL 2048    // rows a small-segment block sorts in shared memory
+#define SEG_MED 16384     // rows a medium-segment block sorts in shared memory
+#define THREADS_SMALL 256
+#define THREADS_MED 1024
+
+struct BlockShared {
+  int64_t red_a[32], red_b[32], red_c[32];
+  uint64_t red_m0[32], red_m1[32];
+  int32_t red_n[32];
+  ReplicaPlan plan;
+  int64_t carry_cost;
+  int32_t carry_count, carry_act, carry_inact;
+  int64_t adm_cost, adm_kv, t1, t2, next_arrival;
+  int32_t adm_count, worked, n_act;
+};
+
+// Compare-exchange of sort items, ascending: `hi` alone (items carry their tie-break in the low
+// bits) or the 96-bit pair (hi, lo).
+template <bool WIDE>
+__device__ __forceinline__ void cmp_swap(uint64_t *hi, uint32_t *lo, int i, int j) {
+  const uint64_t hi_i = hi[i], hi_j = hi[j];
+  if (WIDE) {
+    const uint32_t lo_i = lo[i], lo_j = lo[j];
+    if (hi_i > hi_j || (hi_i == hi_j && lo_i > lo_j)) { hi[i] = hi_j; hi[j] = hi_i; lo[i] = lo_j; lo[j] = lo_i; }
+  } else if (hi_i > hi_j) { hi[i] = hi_j; hi[j] = hi_i; }
+}
+
+// Bitonic sorting network with ascending comparators only (mirrored first sub-stage), so the virtual
+// +inf padding beyond n never moves: any n, in place.  Items are distinct, so the result is unique.
+// Each warp owns a contiguous chunk of E items; stages whose pairs stay inside a chunk need only a
+// warp barrier, the others a block barrier.  Callers synchronise the block before the call; the
+// block is synchronised on return.
+template <bool WIDE>
+__device__ void block_sort(uint64_t *hi, uint32_t *lo, int n) {
+  if (n > 1) {
+    int n_pad = 2;
+    while (n_pad < n) n_pad <<= 1;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    int E = n_pad / nwarp;
+    if (E < 64) E = 64;
+    if (E > n_pad) E = n_pad;
+    const int c0 = warp * E;
+    const bool has_chunk = c0 < n_pad;
+    const int half = n_pad >> 1;
+    bool local = true;    // the previous stage was chunk-local (or there was none)
+    for (int k = 2; k <= n_pad; k <<= 1) {
+      const int hk = k >> 1;
+      if (k <= E) {   // mirrored sub-stage of merge size k, inside the chunk
+        if (has_chunk)
+          for (int t = lane; t < (E >> 1); t += 32) {
+            const int blk = t / hk, off = t - blk * hk;
+            const int i = c0 + blk * k + off, j = c0 + blk * k + k - 1 - off;
+            if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
+          }
+        __syncwarp();
+      } else {
+        if (local) { __syncthreads(); local = false; }
+        for (int t = threadIdx.x; t < half; t += blockDim.x) {
+          const int blk = t / hk, off = t - blk * hk;
+          const int i = blk * k + off, j = blk * k + k - 1 - off;
+          if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
+        }
+        __syncthreads();
+      }
+      for (int j = k >> 2; j > 0; j >>= 1) {
+        if (2 * j <= E) {   // pairs (i, i+j) stay inside an aligned block of 2j <= E items
+          local = true;
+          if (has_chunk)
+            for (int t = lane; t < (E >> 1); t += 32) {
+              const int i = c0 + 2 * t - (t & (j - 1));
+              if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
+            }
+          __syncwarp();
+        } else {
+          if (local) { __syncthreads(); local = false; }
+          for (int t = threadIdx.x; t < half; t += blockDim.x) {
+            const int i = 2 * t - (t & (j - 1));
+            if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
+          }
+          __syncthreads();
+        }
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// what a record says about its row once the replica's plan is known
+struct RowEval { int64_t slack, pred_tpot; uint64_t k48; int phase; };
+
+__device__ __forceinline__ RowEval eval_row(const HfxParams &p, const ReplicaPlan &pl, int64_t base, int kind, int prio,
+                                            int32_t prompt, int32_t gen) {
+  RowEval e;
+  e.slack = 0; e.pred_tpot = 0; e.phase = PH_INACTIVE;
+  int kprio = 63;
+  int64_t kslack = HFX_SLACK_MAX;
+  if (kind == KIND_RUNNING) {
+    e.phase = PH_RUNNING; kprio = prio;
+    e.slack = base == BASE_UNBOUNDED ? HFX_SLACK_MAX : base - pl.shift_run;
+    e.pred_tpot = pl.e_d; kslack = e.slack;
+  } else if (kind == KIND_QUEUED) {
+    e.phase = PH_QUEUED; kprio = prio;
+    e.pred_tpot = pl.shift_dq + p.d2 * ((int64_t)prompt + gen);
+    if (pl.mode == HFX_DECODE) e.slack = base == BASE_UNBOUNDED ? HFX_SLACK_MAX : base - pl.shift_dq;
+    else e.slack = base == BASE_UNBOUNDED ? HFX_SLACK_MAX : base;
+    kslack = e.slack;
+  }
+  e.k48 = dev_key48(e.phase, kprio, kslack);
+  return e;
+}
+
+// iteration clock of a replica once its admission is known (the commit rules)
+__device__ __forceinline__ void iteration_clock(const ReplicaPlan &pl, int32_t adm_count, int64_t lp, int64_t mat_next,
+                                                int &worked, int64_t &t1, int64_t &t2) {
+  t1 = pl.now; t2 = pl.now;
+  if (pl.mode == HFX_COLOCATED) {
+    worked = adm_count > 0 || pl.n_run > 0;
+    t1 = pl.now + (adm_count > 0 ? lp : 0);
+    t2 = t1 + (pl.n_run > 0 ? pl.e_d : 0);
+  } else if (pl.mode == HFX_PREFILL) {
+    worked = adm_count > 0;
+    t1 = t2 = pl.now + (adm_count > 0 ? lp : 0);
+  } else {
+    worked = pl.now >= pl.mat && pl.n_run + adm_count > 0;
+    t2 = worked ? mat_next : pl.now;
+  }
+}
+
+__device__ __forceinline__ void write_replica_outputs(const SegArgs &a, int r, const ReplicaPlan &pl, int64_t adm_cost,
+                                                      int32_t adm_count, int64_t mat_next, int worked, int64_t t2,
+                                                      int64_t next_arrival) {
+  a.budget[r] = pl.budget;
+  if (a.e_d) a.e_d[r] = pl.e_d;
+  if (a.n_run) a.n_run[r] = (int32_t)pl.n_run;
+  if (a.sum_kv) a.sum_kv[r] = pl.sum_kv;
+  a.adm_cost[r] = adm_cost;
+  a.adm_count[r] = adm_count;
+  a.maturity_next[r] = mat_next;
+  if (a.flags & HFX_COMMIT) {
+    int64_t now_next = pl.now;
+    if (worked) now_next = t2;
+    else {   // idle: jump to the next event, if any
+      int64_t ev = HFX_INF;
+      if (pl.mat > pl.now) ev = pl.mat;
+      if (next_arrival < ev) ev = next_arrival;
+      if (ev != HFX_INF) now_next = ev;
+    }
+    a.now[r] = now_next;
+    a.mat[r] = mat_next;
+  }
+}
+
+// the table update of one row at commit
+__device__ __forceinline__ void commit_row(const SegArgs &a, const ReplicaPlan &pl, int kind, bool adm, int worked,
+                                           int64_t t1, int64_t t2, int32_t row, int32_t prompt, int32_t gen, int32_t out_len) {
+  if (kind == KIND_RUNNING) {
+    if (pl.mode == HFX_PREFILL || (pl.mode == HFX_DECODE && !worked)) return;
+    a.gen[row] = gen + 1;
+    a.last_token[row] = t2;
+    if ((int64_t)gen + 2 >= out_len) { a.state[row] = HFX_DONE; a.finish[row] = t2; }
+  } else if (kind == KIND_QUEUED) {
+    if (adm) {
+      uint8_t st = HFX_RUNNING;
+      if (pl.mode == HFX_DECODE) {
+        a.gen[row] = gen + 1;
+        a.last_token[row] = t2;
+        if ((int64_t)gen + 2 >= out_len) { st = HFX_DONE; a.finish[row] = t2; }
+      } else {
+        a.gen[row] = 0;
+        a.first_token[row] = t1;
+        a.last_token[row] = t1;
+        if (out_len <= 1) { st = HFX_DONE; a.finish[row] = t1; }
+      }
+      a.state[row] = st;
+    } else if (pl.mode != HFX_DECODE && prompt > pl.token_cap) {
+      a.state[row] = HFX_REJECTED;
+    }
+  }
+}
+
+// aggregates of one segment into the block's plan (all threads call; result in sh.plan)
+__device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &a, const HfxRec *seg, int64_t n, int r,
+                                             bool real, BlockShared &sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  int64_t n_run = 0, sum_kv = 0, next_arr = HFX_INF;
+  uint64_t m_run = 0, m_q = 0;
+  int32_t n_act = 0;
+  for (int64_t q = threadIdx.x; q < n; q += blockDim.x) {
+    const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);   // prompt, gen, output_len, bytes
+    const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
+    if (kind == KIND_RUNNING) { n_run++; n_act++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
+    else if (kind == KIND_QUEUED) { n_act++; m_q |= 1ull << cls; }
+    else if (kind == KIND_FUTURE) { const int64_t arr = seg[q].base; next_arr = arr < next_arr ? arr : next_arr; }
+  }
+  n_run = warp_sum_i64(n_run); sum_kv = warp_sum_i64(sum_kv); next_arr = warp_min_i64(next_arr);
+  m_run = warp_or_u64(m_run); m_q = warp_or_u64(m_q); n_act = (int32_t)warp_sum_i64(n_act);
+  if (lane == 0) {
+    sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_c[warp] = next_arr; sh.red_m0[warp] = m_run;
+    sh.red_m1[warp] = m_q; sh.red_n[warp] = n_act;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int k = 1; k < nwarp; k++) {
+      n_run += sh.red_a[k]; sum_kv += sh.red_b[k]; n_act += sh.red_n[k];
+      next_arr = sh.red_c[k] < next_arr ? sh.red_c[k] : next_arr;
+      m_run |= sh.red_m0[k]; m_q |= sh.red_m1[k];
+    }
+    hfx_replica_cfg cfg; cfg.mode = HFX_COLOCATED; cfg.token_cap = 1; cfg.batch_cap = 0;
+    int64_t now = 0, mat = 0;
+    if (real) { cfg = a.cfg[r]; now = a.now[r]; mat = a.mat[r]; }
+    dev_plan(p, cfg, now, mat, n_run, sum_kv, m_run, m_q, sh.plan);
+    sh.next_arrival = next_arr; sh.n_act = n_act;
+    sh.carry_cost = 0; sh.carry_count = 0; sh.carry_act = 0; sh.carry_inact = 0;
+    sh.adm_cost = 0; sh.adm_kv = 0; sh.adm_count = 0;
+  }
+  __syncthreads();
+}
+
+// Block-wide admission over the sorted items s_lo[0..n_sorted) (low 16 bits = position of the
+// record inside the segment): writes order, admit and the compacted admitted list, keeps each
+// decision in bit 16 of s_lo, accumulates the totals in sh.
+__device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs &a, const ReplicaPlan &pl,
+                                              const HfxRec *seg, uint32_t b, uint32_t *s_lo, int n_sorted,
+                                              BlockShared &sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  for (int tile = 0; tile < n_sorted; tile += blockDim.x) {
+    const int q = tile + threadIdx.x;
+    int64_t cost = 0, kv = 0;
+    int32_t cnt = 0, row = -1, kind = KIND_DEAD;
+    if (q < n_sorted) {
+      const int li = s_lo[q] & 0xffff;
+      const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
+      const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
+      row = (int32_t)w0.w;
+      kind = (w1.w >> 8) & 0xff;
+      if (kind == KIND_QUEUED) {
+        kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
+        const int64_t c = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
+        if (c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
+      }
+      a.order[b + q] = row;
+    }
+    // block-wide inclusive scan of (cost, cnt) with carry
+    int64_t sc = warp_incl_scan_i64(cost, lane);
+    int32_t sn = warp_incl_scan_i32(cnt, lane);
+    if (lane == 31) { sh.red_a[warp] = sc; sh.red_b[warp] = sn; }
+    __syncthreads();
+    if (warp == 0) {
+      int64_t x = lane < nwarp ? sh.red_a[lane] : 0;
+      int32_t y = lane < nwarp ? (int32_t)sh.red_b[lane] : 0;
+      x = warp_incl_scan_i64(x, lane); y = warp_incl_scan_i32(y, lane);
+      sh.red_a[lane] = x; sh.red_b[lane] = y;
+    }
+    __syncthreads();
+    sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
+    sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
+    bool adm = false;
+    if (cnt) adm = sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap);
+    if (q < n_sorted) {
+      a.admit[row] = (uint8_t)((kind == KIND_RUNNING || adm) ? 1 : 0);
+      if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
+      s_lo[q] = (s_lo[q] & 0xffffu) | (adm ? 0x10000u : 0u);
+    }
+    // totals over admitted rows (admission is prefix-closed, so a block reduction suffices)
+    int64_t ac = adm ? cost : 0, ak = adm ? kv : 0;
+    int32_t an = adm ? 1 : 0;
+    ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)warp_sum_i64(an);
+    __syncthreads();     // everyone has read red_a / red_b / carry
+    if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_c[warp] = an; }
+    if (threadIdx.x == blockDim.x - 1) { sh.carry_cost = sc; sh.carry_count = sn; }
+    __syncthreads();
+    if (threadIdx.x == 0)
+      for (int k = 0; k < nwarp; k++) { sh.adm_cost += sh.red_a[k]; sh.adm_kv += sh.red_b[k]; sh.adm_count += (int32_t)sh.red_c[k]; }
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegArgs a, const HfxRec *__restrict__ rec,
+                                                  const uint32_t *__restrict__ seg_begin,
+                                                  const uint32_t *__restrict__ flags, int seg_min, int seg_cap) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint64_t *s_hi = reinterpret_cast<uint64_t *>(smem_raw);
+  uint32_t *s_lo = reinterpret_cast<uint32_t *>(smem_raw + (size_t)seg_cap * 8);
+  __shared__ BlockShared sh;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const int R = p.n_replicas;
+  if (flags[1] < (uint32_t)seg_min) return;     // no segment of this kernel's size class exists
+  const bool ordered = flags[0] != 0;
+
+  for (int r = blockIdx.x; r <= R; r += gridDim.x) {
+    const uint32_t b = seg_begin[r];
+    const int n = (int)(seg_begin[r + 1] - b);
+    if (n < seg_min || n > seg_cap) continue;
+    if (r == R && n == 0) continue;
+    const HfxRec *seg = rec + b;
+    const bool real = r < R;    // bucket R holds rows bound to no replica
+
+    segment_plan(p, a, seg, n, r, real, sh);
+    const ReplicaPlan pl = sh.plan;
+    int n_sorted;
+
+    if (ordered) {
+      // ---- records are in req_id order: only rows in flight or in the queue are sorted, by
+      //      (key48, position); inactive rows keep their order behind them ---------------------
+      n_sorted = sh.n_act;
+      const int n_active = n_sorted;
+      for (int tile = 0; tile < n; tile += blockDim.x) {
+        const int q = tile + threadIdx.x;
+        int act = 0, inact = 0;
+        int32_t row = -1;
+        uint64_t k48 = 0;
+        if (q < n) {
+          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
+          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
+          const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
+          row = (int32_t)w0.w;
+          const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
+          const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+          k48 = e.k48;
+          act = e.phase != PH_INACTIVE; inact = !act;
+          a.slack[row] = e.slack;
+          if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
+          if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+          if (inact) a.admit[row] = 0;
+        }
+        const uint32_t bal = __ballot_sync(0xffffffffu, act);
+        const uint32_t bal_in = __ballot_sync(0xffffffffu, inact);
+        const uint32_t lt = (1u << lane) - 1u;
+        if (lane == 0) { sh.red_a[warp] = __popc(bal); sh.red_b[warp] = __popc(bal_in); }
+        __syncthreads();
+        int pre_a = sh.carry_act, pre_i = sh.carry_inact, tot_a = 0, tot_i = 0;
+        for (int k = 0; k < nwarp; k++) {
+          const int ca = (int)sh.red_a[k], ci = (int)sh.red_b[k];
+          if (k < warp) { pre_a += ca; pre_i += ci; }
+          tot_a += ca; tot_i += ci;
+        }
+        if (act) s_hi[pre_a + __popc(bal & lt)] = (k48 << 16) | (uint32_t)q;
+        if (inact) a.order[b + n_active + pre_i + __popc(bal_in & lt)] = row;
+        __syncthreads();
+        if (threadIdx.x == 0) { sh.carry_act += tot_a; sh.carry_inact += tot_i; }
+      }
+      __syncthreads();
+      block_sort<false>(s_hi, nullptr, n_sorted);
+      for (int q = threadIdx.x; q < n_sorted; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+    } else {
+      // ---- general case: every row takes part, the tie-break req_id travels with the item -----
+      n_sorted = n;
+      for (int q = threadIdx.x; q < n; q += blockDim.x) {
+        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
+        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
+        const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
+        const int32_t req_id = (int32_t)w0.z, row = (int32_t)w0.w;
+        const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
+        const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+        const uint32_t uid = (uint32_t)req_id ^ 0x80000000u;      // signed order as unsigned
+        s_hi[q] = (e.k48 << 16) | (uid >> 16);
+        s_lo[q] = (uid << 16) | (uint32_t)q;
+        a.slack[row] = e.slack;
+        if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
+        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+      }
+      __syncthreads();
+      block_sort<true>(s_hi, s_lo, n);
+      for (int q = threadIdx.x; q < n; q += blockDim.x) s_lo[q] &= 0xffffu;
+    }
+    __syncthreads();
+
+    segment_admit(p, a, pl, seg, b, s_lo, n_sorted, sh);
+
+    // ---- maturity, per-replica outputs, commit decisions --------------------------------
+    if (threadIdx.x == 0) {
+      int64_t lp = 0;
+      const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
+      int worked; int64_t t1, t2;
+      iteration_clock(pl, sh.adm_count, lp, mat_next, worked, t1, t2);
+      sh.worked = worked; sh.t1 = t1; sh.t2 = t2;
+      if (real) write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, t2, sh.next_arrival);
+    }
+    __syncthreads();
+
+    // ---- second pass: padding of the compacted list, commit ------------------------------
+    if (a.admitted_rows)
+      for (int q = sh.adm_count + threadIdx.x; q < n; q += blockDim.x) a.admitted_rows[b + q] = -1;
+    if (real && (a.flags & HFX_COMMIT)) {
+      const int worked = sh.worked;
+      const int64_t t1 = sh.t1, t2 = sh.t2;
+      for (int q = threadIdx.x; q < n_sorted; q += blockDim.x) {
+        const uint32_t lo = s_lo[q];
+        const int li = lo & 0xffff;
+        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
+        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
+        commit_row(a, pl, (w1.w >> 8) & 0xff, (lo & 0x10000u) != 0, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x,
+                   (int32_t)w1.y, (int32_t)w1.z);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Oversize segments (more rows than a block can sort in shared memory): one cooperative kernel.
+// All blocks walk the replicas in the same order and share the work of each oversize one: keys
+// spread over the grid, a global bitonic network with bounded grid barriers, admission by block 0
+// walking the order with a carried prefix, commit by the grid.  Slow but exact; it only exists so
+// that any table is handled.
+// ------------------------------------------------------------------------------------------------
+
+// Bounded grid barrier (all blocks of a cooperative launch are resident).  Returns false if the
+// wait ran out; the caller then leaves, and HFX_ST_TIMEOUT is raised.
+__device__ bool grid_barrier(uint32_t *bar, uint32_t *status, uint32_t &epoch) {
+  __shared__ int ok_s;
+  __syncthreads();
+  epoch++;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const uint32_t target = epoch * gridDim.x;
+    atomicAdd(bar, 1u);
+    int ok = 0;
+    for (long long spin = 0; spin < (1ll << 26); spin++) {
+      if (*((volatile uint32_t *)bar) >= target) { ok = 1; break; }
+      if (*((volatile uint32_t *)status) & HFX_ST_TIMEOUT) break;
+      __nanosleep(64);
+    }
+    if (!ok) atomicOr(status, HFX_ST_TIMEOUT);
+    __threadfence();
+    ok_s = ok;
+  }
+  __syncthreads();
+  return ok_s != 0;
+}
+
+__device__ __forceinline__ void global_cmp_swap(uint64_t *hi, uint32_t *lo, uint32_t *idx, int64_t i, int64_t j) {
+  const uint64_t hi_i = hi[i], hi_j = hi[j];
+  const uint32_t lo_i = lo[i], lo_j = lo[j];
+  if (hi_i > hi_j || (hi_i == hi_j && lo_i > lo_j)) {
+    hi[i] = hi_j; hi[j] = hi_i; lo[i] = lo_j; lo[j] = lo_i;
+    const uint32_t x = idx[i]; idx[i] = idx[j]; idx[j] = x;
+  }
+}
+
+__global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a, const HfxRec *__restrict__ rec,
+                                             const uint32_t *__restrict__ seg_begin, const uint32_t *__restrict__ flags,
+                                             uint64_t *__restrict__ g_hi, uint32_t *__restrict__ g_lo,
+                                             uint32_t *__restrict__ g_idx, uint32_t *bar, uint32_t *status) {
+  __shared__ BlockShared sh;
+  if (flags[1] <= SEG_MED) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const int R = p.n_replicas;
+  uint32_t epoch = 0;
+  const int64_t gtid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t gsize = (int64_t)gridDim.x * blockDim.x;
+  volatile int64_t *mail = reinterpret_cast<volatile int64_t *>(bar + 4);
+
+  for (int r = 0; r <= R; r++) {
+    const uint32_t b = seg_begin[r];
+    const int64_t n = (int64_t)(seg_begin[r + 1] - b);
+    if (n <= SEG_MED) continue;
+    const HfxRec *seg = rec + b;
+    const bool real = r < R;
+    uint64_t *hi = g_hi + b;
+    uint32_t *lo = g_lo + b, *idx = g_idx + b;
+
+    // every block computes the aggregates redundantly (reads come from L2 after the first)
+    segment_plan(p, a, seg, n, r, real, sh);
+    const ReplicaPlan pl = sh.plan;
+
+    // keys, spread over the grid
+    for (int64_t q = gtid; q < n; q += gsize) {
+      const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
+      const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
+      const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
+      const int32_t req_id = (int32_t)w0.z, row = (int32_t)w0.w;
+      const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
+      const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+      hi[q] = e.k48;
+      lo[q] = (uint32_t)req_id ^ 0x80000000u;
+      idx[q] = (uint32_t)q;
+      a.slack[row] = e.slack;
+      if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
+      if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+    }
+    if (!grid_barrier(bar, status, epoch)) return;
+
+    // global bitonic network (ascending comparators, virtual padding), idx travels with the item
+    int64_t n_pad = 1;
+    while (n_pad < n) n_pad <<= 1;
+    const int64_t half = n_pad >> 1;
+    for (int64_t k = 2; k <= n_pad; k <<= 1) {
+      const int64_t hk = k >> 1;
+      for (int64_t t = gtid; t < half; t += gsize) {
+        const int64_t blk = t / hk, off = t - blk * hk;
+        const int64_t i = blk * k + off, j = blk * k + k - 1 - off;
+        if (j < n) global_cmp_swap(hi, lo, idx, i, j);
+      }
+      if (!grid_barrier(bar, status, epoch)) return;
+      for (int64_t j = k >> 2; j > 0; j >>= 1) {
+        for (int64_t t = gtid; t < half; t += gsize) {
+          const int64_t i = 2 * t - (t & (j - 1));
+          if (i + j < n) global_cmp_swap(hi, lo, idx, i, i + j);
+        }
+        if (!grid_barrier(bar, status, epoch)) return;
+      }
+    }
+
+    // admission walk by block 0 with a carried prefix, then commit by the whole grid
+    if (blockIdx.x == 0) {
+      for (int64_t tile = 0; tile < n; tile += blockDim.x) {
+        const int64_t q = tile + threadIdx.x;
+        int64_t cost = 0, kv = 0;
+        int32_t cnt = 0, row = -1, kind = KIND_DEAD;
+        if (q < n) {
+          const uint32_t li = idx[q];
+          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
+          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
+          row = (int32_t)w0.w;
+          kind = (w1.w >> 8) & 0xff;
+          if (kind == KIND_QUEUED) {
+            kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
+            const int64_t c = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
+            if (c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
+          }
+          a.order[b + q] = row;
+        }
+        int64_t sc = warp_incl_scan_i64(cost, lane);
+        int32_t sn = warp_incl_scan_i32(cnt, lane);
+        if (lane == 31) { sh.red_a[warp] = sc; sh.red_b[warp] = sn; }
+        __syncthreads();
+        if (warp == 0) {
+          int64_t x = lane < nwarp ? sh.red_a[lane] : 0;
+          int32_t y = lane < nwarp ? (int32_t)sh.red_b[lane] : 0;
+          x = warp_incl_scan_i64(x, lane); y = warp_incl_scan_i32(y, lane);
+          sh.red_a[lane] = x; sh.red_b[lane] = y;
+        }
+        __syncthreads();
+        sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
+        sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
+        bool adm = false;
+        if (cnt) adm = sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap);
+        if (q < n) {
+          a.admit[row] = (uint8_t)((kind == KIND_RUNNING || adm) ? 1 : 0);
+          if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
+          lo[q] = adm ? 1u : 0u;      // the sort is over: lo now carries the decision
+        }
+        int64_t ac = adm ? cost : 0, ak = adm ? kv : 0;
+        int32_t an = adm ? 1 : 0;
+        ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)warp_sum_i64(an);
+        __syncthreads();
+        if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_c[warp] = an; }
+        if (threadIdx.x == blockDim.x - 1) { sh.carry_cost = sc; sh.carry_count = sn; }
+        __syncthreads();
+        if (threadIdx.x == 0)
+          for (int k = 0; k < nwarp; k++) { sh.adm_cost += sh.red_a[k]; sh.adm_kv += sh.red_b[k]; sh.adm_count += (int32_t)sh.red_c[k]; }
+        __syncthreads();
+      }
+      if (threadIdx.x == 0) {
+        int64_t lp = 0;
+        const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
+        int worked; int64_t t1, t2;
+        iteration_clock(pl, sh.adm_count, lp, mat_next, worked, t1, t2);
+        mail[0] = t1; mail[1] = t2; mail[2] = worked; mail[3] = sh.adm_count;   // for the other blocks
+        if (real) write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, t2, sh.next_arrival);
+      }
+    }
+    if (!grid_barrier(bar, status, epoch)) return;
+    {
+      const int64_t t1 = mail[0], t2 = mail[1];
+      const int worked = (int)mail[2], adm_count = (int)mail[3];
+      const bool commit = real && (a.flags & HFX_COMMIT);
+      for (int64_t q = gtid; q < n; q += gsize) {
+        if (a.admitted_rows && q >= adm_count) a.admitted_rows[b + q] = -1;
+        if (!commit) continue;
+        const uint32_t li = idx[q];
+        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
+        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
+        commit_row(a, pl, (w1.w >> 8) & 0xff, lo[q] != 0, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x, (int32_t)w1.y,
+                   (int32_t)w1.z);
+      }
+    }
+    if (!grid_barrier(bar, status, epoch)) return;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
+  const int R1 = s->p.n_replicas + 1;
+  cudaStream_t stream = s->stream;
+  {
+    KernelScope ks(s, KSLOT_SEG_SMALL);
+    const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
+    k_segment<<<grid, THREADS_SMALL, SEG_SMALL * 12, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_flags, 0,
+                                                                SEG_SMALL);
+  }
+  if (n > SEG_SMALL) {
+    KernelScope ks(s, KSLOT_SEG_MED);
+    const int grid = R1 < s->n_sm ? R1 : s->n_sm;
+    k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_flags, SEG_SMALL + 1,
+                                                            SEG_MED);
+  }
+  if (n > SEG_MED) {
+    uint32_t *big_idx = reinterpret_cast<uint32_t *>(s->d_big_lo + s->max_rows);
+    if (cudaMemsetAsync(s->d_barrier, 0, 64, stream) != cudaSuccess) return HFX_E_CUDA;
+    void *args[] = {(void *)&s->p, (void *)&sa, (void *)&s->d_rec, (void *)&s->d_seg_begin, (void *)&s->d_flags,
+                    (void *)&s->d_big_hi, (void *)&s->d_big_lo, (void *)&big_idx, (void *)&s->d_barrier,
+                    (void *)&s->d_status};
+    KernelScope ks(s, KSLOT_BIG);
+    if (cudaLaunchCooperativeKernel((void *)k_big, dim3(s->n_sm), dim3(512), args, 0, stream) != cudaSuccess)
+      return HFX_E_CUDA;
+  }
+  return HFX_OK;
+}
+
+int hfx_segment_configure() {
+  if (cudaFuncSetAttribute(k_segment, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_MED * 12) != cudaSuccess)
+    return HFX_E_CUDA;
+  return HFX_OK;
+}

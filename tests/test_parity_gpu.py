@@ -81,6 +81,23 @@ def test_medium_and_oversize_segments():
     assert_step_parity(wl)
 
 
+def test_many_replicas_atomic_regroup_and_natural_ids():
+    # more replicas than fit the shared-memory counters: global-counter regroup
+    wl = gen.random_table(40, 30_000, 9000, modes=MODES3)
+    assert_step_parity(wl, steps=2, commit=True)
+    # request ids rising with the row index, interleaved replicas: the order of equal keys comes from positions
+    for R, n in ((300, 40_000), (3, 5000), (64, 20_000)):
+        wl = gen.random_table(41 + R, n, R, modes=MODES3, permute_ids=False, tie_heavy=R == 64)
+        assert_step_parity(wl, steps=3, commit=True)
+    # one id out of order anywhere must switch every replica to the general order
+    wl = gen.random_table(44, 20_000, 50, permute_ids=False)
+    wl.table["req_id"][12_345] = -5
+    assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_table(45, 20_001, 50, permute_ids=False, grouped=True)
+    wl.table["req_id"][20_000] = 7
+    assert_step_parity(wl)
+
+
 def test_empty_replicas_and_all_inactive():
     wl = gen.random_table(11, 500, 40)
     wl.table["replica_id"][:] = wl.table["replica_id"] % 3 * 13        # most replicas have no rows
