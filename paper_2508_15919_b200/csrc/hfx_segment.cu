@@ -8,6 +8,7 @@
 #define SEG_MED 16384     // rows a medium-segment block sorts in shared memory
 #define THREADS_SMALL 256
 #define THREADS_MED 1024
+#define SMEM_SMALL (SEG_SMALL * 20 + (2 * 1024 + 8) * 4)   // sort items, their order, scatter buffer, bins
 
 struct BlockShared {
   int64_t red_a[32], red_b[32], red_c[32];
@@ -89,6 +90,70 @@ __device__ void block_sort(uint64_t *hi, uint32_t *lo, int n) {
     }
   }
   __syncthreads();
+}
+
+// Distribution sort of distinct 64-bit items for small segments: items are binned by their offset
+// from the smallest item (a shift makes at most SORT_BINS bins, so bins are in key order), scattered
+// bin by bin, and ranked inside their bin by counting smaller items.  Writes the low 16 bits of the
+// items, in ascending item order, to s_lo.  Returns false (uniformly, nothing written) when a bin is
+// too crowded for the counting to pay; the caller then runs the sorting network instead.
+// Needs blockDim.x <= SORT_BINS and SORT_BINS % blockDim.x == 0.  Block-synchronised on entry by the
+// caller and on return.
+#define SORT_BINS 1024
+#define SORT_BIN_MAX 48
+__device__ bool block_bucket_order(const uint64_t *s_hi, uint64_t *s_tmp, uint32_t *s_lo, uint32_t *s_bin,
+                                   uint32_t *s_cur, int n, BlockShared &sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  uint64_t mn = ~0ull, mx = 0;
+  for (int q = threadIdx.x; q < n; q += blockDim.x) { const uint64_t v = s_hi[q]; mn = v < mn ? v : mn; mx = v > mx ? v : mx; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const uint64_t a = __shfl_xor_sync(0xffffffffu, mn, o), b = __shfl_xor_sync(0xffffffffu, mx, o);
+    mn = a < mn ? a : mn; mx = b > mx ? b : mx;
+  }
+  if (lane == 0) { sh.red_m0[warp] = mn; sh.red_m1[warp] = mx; }
+  for (int i = threadIdx.x; i <= SORT_BINS; i += blockDim.x) s_bin[i] = 0;
+  __syncthreads();
+  for (int k = 0; k < nwarp; k++) { const uint64_t a = sh.red_m0[k], b = sh.red_m1[k]; mn = a < mn ? a : mn; mx = b > mx ? b : mx; }
+  const uint64_t range = mx - mn;
+  int sft = 0;
+  if (range >> 10) sft = 64 - __clzll((long long)range) - 10;     // (range >> sft) < SORT_BINS
+  for (int q = threadIdx.x; q < n; q += blockDim.x) atomicAdd(&s_bin[(uint32_t)((s_hi[q] - mn) >> sft)], 1u);
+  __syncthreads();
+  // exclusive scan of the bin counts; the largest bin
+  const int per = SORT_BINS / blockDim.x;
+  const int i0 = threadIdx.x * per;
+  uint32_t sum = 0, big = 0;
+  for (int i = 0; i < per; i++) { const uint32_t c = s_bin[i0 + i]; sum += c; big = c > big ? c : big; }
+  uint32_t v = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { const uint32_t x = __shfl_xor_sync(0xffffffffu, big, o); big = x > big ? x : big; }
+  if (lane == 31) sh.red_n[warp] = (int32_t)v;
+  if (lane == 0) sh.red_a[warp] = big;
+  __syncthreads();
+  uint32_t pre = 0, bigall = 0;
+  for (int k = 0; k < nwarp; k++) { if (k < warp) pre += (uint32_t)sh.red_n[k]; const uint32_t x = (uint32_t)sh.red_a[k]; bigall = x > bigall ? x : bigall; }
+  if (bigall > SORT_BIN_MAX) { __syncthreads(); return false; }
+  uint32_t run = pre + v - sum;
+  for (int i = 0; i < per; i++) { const uint32_t c = s_bin[i0 + i]; s_bin[i0 + i] = run; s_cur[i0 + i] = run; run += c; }
+  __syncthreads();
+  for (int q = threadIdx.x; q < n; q += blockDim.x) {
+    const uint64_t x = s_hi[q];
+    s_tmp[atomicAdd(&s_cur[(uint32_t)((x - mn) >> sft)], 1u)] = x;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < n; e += blockDim.x) {
+    const uint64_t x = s_tmp[e];
+    const uint32_t b = (uint32_t)((x - mn) >> sft);
+    const uint32_t g0 = s_bin[b], g1 = s_cur[b];
+    uint32_t rank = 0;
+    for (uint32_t g = g0; g < g1; g++) rank += s_tmp[g] < x ? 1u : 0u;
+    s_lo[g0 + rank] = (uint32_t)(x & 0xffffu);
+  }
+  __syncthreads();
+  return true;
 }
 
 // what a record says about its row once the replica's plan is known
@@ -283,10 +348,15 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
 
 __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegArgs a, const HfxRec *__restrict__ rec,
                                                   const uint32_t *__restrict__ seg_begin,
-                                                  const uint32_t *__restrict__ flags, int seg_min, int seg_cap) {
+                                                  const uint32_t *__restrict__ flags, int seg_min, int seg_cap,
+                                                  int bucket) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint64_t *s_hi = reinterpret_cast<uint64_t *>(smem_raw);
   uint32_t *s_lo = reinterpret_cast<uint32_t *>(smem_raw + (size_t)seg_cap * 8);
+  // only with `bucket`: scratch of the distribution sort
+  uint64_t *s_tmp = reinterpret_cast<uint64_t *>(smem_raw + (size_t)seg_cap * 12);
+  uint32_t *s_bin = reinterpret_cast<uint32_t *>(smem_raw + (size_t)seg_cap * 20);
+  uint32_t *s_cur = s_bin + SORT_BINS + 4;
   __shared__ BlockShared sh;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const int R = p.n_replicas;
@@ -346,8 +416,10 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
         if (threadIdx.x == 0) { sh.carry_act += tot_a; sh.carry_inact += tot_i; }
       }
       __syncthreads();
-      block_sort<false>(s_hi, nullptr, n_sorted);
-      for (int q = threadIdx.x; q < n_sorted; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+      if (!(bucket && n_sorted > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_sorted, sh))) {
+        block_sort<false>(s_hi, nullptr, n_sorted);
+        for (int q = threadIdx.x; q < n_sorted; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+      }
     } else {
       // ---- general case: every row takes part, the tie-break req_id travels with the item -----
       n_sorted = n;
@@ -595,14 +667,13 @@ int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
   {
     KernelScope ks(s, KSLOT_SEG_SMALL);
     const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
-    k_segment<<<grid, THREADS_SMALL, SEG_SMALL * 12, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_flags, 0,
-                                                                SEG_SMALL);
+    k_segment<<<grid, THREADS_SMALL, SMEM_SMALL, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_flags, 0, SEG_SMALL, 1);
   }
   if (n > SEG_SMALL) {
     KernelScope ks(s, KSLOT_SEG_MED);
     const int grid = R1 < s->n_sm ? R1 : s->n_sm;
     k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_flags, SEG_SMALL + 1,
-                                                            SEG_MED);
+                                                            SEG_MED, 0);
   }
   if (n > SEG_MED) {
     uint32_t *big_idx = reinterpret_cast<uint32_t *>(s->d_big_lo + s->max_rows);
