@@ -93,15 +93,20 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   ok = ok && cudaMalloc(&s->d_status, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_seg_count, sizeof(uint32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_seg_begin, sizeof(uint32_t) * R2) == cudaSuccess;
-  ok = ok && cudaMalloc(&s->d_cursor, sizeof(uint32_t) * R2) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_cursor, sizeof(uint32_t) * 2 * R2) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_act_count, sizeof(uint32_t) * R2) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_rowflag, (size_t)max_rows + 16) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_flags, 256) == cudaSuccess;
   {
     int32_t tile_rows = 0, n_tiles = 0;
     hfx_tile_shape(max_rows, &tile_rows, &n_tiles);
     if (n_tiles < HFX_TILE_BLOCKS) n_tiles = HFX_TILE_BLOCKS;
     s->tile_blocks_max = 0;
-    if (n_replicas <= HFX_TILE_REPLICAS_MAX && (int64_t)n_tiles * (n_replicas + 1) <= HFX_TILE_MATRIX_MAX) {
-      ok = ok && cudaMalloc(&s->d_tile_hist, sizeof(uint32_t) * (size_t)n_tiles * ((size_t)n_replicas + 1)) == cudaSuccess;
+    if (n_replicas <= HFX_TILE_REPLICAS_MAX && 2 * (int64_t)n_tiles * (n_replicas + 1) <= HFX_TILE_MATRIX_MAX) {
+      const size_t cells = (size_t)n_tiles * ((size_t)n_replicas + 1);
+      ok = ok && cudaMalloc(&s->d_tile_hist, sizeof(uint32_t) * 2 * cells) == cudaSuccess;
+      ok = ok && cudaMalloc(&s->d_tile_fmin, sizeof(int64_t) * cells) == cudaSuccess;
+      ok = ok && cudaMalloc(&s->d_tile_mode, (size_t)n_tiles + 16) == cudaSuccess;
       s->tile_blocks_max = n_tiles;
     }
   }
@@ -119,6 +124,8 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     memcpy(h->h_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas);
     ok = ok && cudaMemcpy(s->d_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemset(s->d_status, 0, 256) == cudaSuccess;
+    const uint32_t init_flags[4] = {1u, 1u, 0u, 0u};
+    ok = ok && cudaMemcpy(s->d_flags, init_flags, sizeof(init_flags), cudaMemcpyHostToDevice) == cudaSuccess;
   }
   if (!ok) {
     cudaGetLastError();
@@ -135,6 +142,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   cudaStreamSynchronize(s->stream);
   cudaFree(s->d_cfg); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
+  cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_fmin); cudaFree(s->d_tile_mode);
   cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();

@@ -22,6 +22,13 @@
 #define KIND_FUTURE 2   // QUEUED but not arrived yet (only matters for the idle clock jump)
 #define KIND_DEAD 3     // DONE, REJECTED or a row with bad data
 
+#define ROWFLAG_BADREP 4  // row bound to no replica (bucket R)
+
+// how a tile's rows get their rank inside their (replica, class) group, in row order
+#define TILE_SORTED 0     // tile already sorted by replica: ranks from positions
+#define TILE_GROUPS 1     // small groups: counting sort of the tile, rank by scanning the group
+#define TILE_ANY 2        // large unsorted groups: any order (clears "ordered")
+
 // "no bound" marker of a slack base
 #define BASE_UNBOUNDED INT64_MAX
 
@@ -58,7 +65,7 @@ enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_S
 #define HFX_TILE_BLOCKS 296
 #define HFX_TILE_ROWS_MAX 8192
 #define HFX_TILE_MATRIX_MAX (INT64_C(8) << 20)   // entries of the tile-histogram matrix (32 MiB)
-#define HFX_TILE_REPLICAS_MAX 8191               // replicas whose counters fit in shared memory
+#define HFX_TILE_REPLICAS_MAX 4095               // replicas whose counters fit in shared memory
 
 struct HfxBracket { cudaEvent_t a, b; int slot; };
 
@@ -75,11 +82,17 @@ struct hfx_sched {
   hfx_replica_cfg *d_cfg;   // [R]
   uint32_t *d_status;       // sticky status word
   uint32_t *d_seg_count;    // [R+2] rows per replica (+ the bad-replica bucket R)
-  uint32_t *d_seg_begin;    // [R+2] exclusive prefix
-  uint32_t *d_cursor;       // [R+2] fill cursors of the regroup pass
-  uint32_t *d_tile_hist;    // [tile_blocks_max][R+1] per-tile histograms (nullptr: atomic mode only)
+  uint32_t *d_act_count;    // [R+2] active rows (in flight or in the visible queue) per replica
+  uint32_t *d_seg_begin;    // [R+2] exclusive prefix of d_seg_count
+  uint32_t *d_cursor;       // [2][R+2] fill cursors of the atomic regroup (active, inactive)
+  uint32_t *d_tile_hist;    // [tile_blocks_max][2][R+1] per-tile histograms: all rows, active rows
+                            // (nullptr: atomic mode only)
+  uint8_t *d_tile_mode;     // [tile_blocks_max] how ranks inside a tile are found (TILE_*)
+  int64_t *d_tile_fmin;     // [tile_blocks_max][R+1] earliest arrival among a tile's not-yet-arrived rows
+  uint8_t *d_rowflag;       // [max_rows] kind of every row (KIND_*), ROWFLAG_BADREP for a bad replica id
   int32_t tile_blocks_max;
-  uint32_t *d_flags;        // [0] records in req_id order, [1] largest segment
+  uint32_t step_parity;     // which of the two `ordered` words this step uses
+  uint32_t *d_flags;        // [0],[1] "ordered" (by step parity), [2] largest sort size of a replica
   HfxRec *d_rec;            // [max_rows]
   uint64_t *d_big_hi;       // sort scratch of oversize segments
   uint32_t *d_big_lo;
@@ -257,6 +270,9 @@ struct RegroupArgs {
   const int64_t *now; const int64_t *mat; const hfx_replica_cfg *cfg;
   int64_t *pred_ttft;    // optional output
   int64_t n;
+  // outputs of inactive rows, written by the regroup itself when the step is "ordered"
+  int64_t *slack; int64_t *pred_tpot; uint64_t *key; int32_t *order; uint8_t *admit; int32_t *admitted_rows;
+  uint32_t commit;
 };
 
 struct SegArgs {
@@ -274,6 +290,7 @@ struct SegArgs {
 // host-side launchers implemented in the .cu files
 void hfx_tile_shape(int64_t n, int32_t *tile_rows, int32_t *n_tiles);
 int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off);
+size_t hfx_regroup_smem(int R1, int tile_rows);
 int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n);
 int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o, uint32_t flags);
 int hfx_launch_sim(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,

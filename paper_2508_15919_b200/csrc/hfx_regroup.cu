@@ -1,111 +1,188 @@
-// Grouping the request table by replica: count, scan, and the one streaming pass that turns every
-// row into a 32-byte record inside its replica's range.
+// Grouping the request table by replica: classify and count, scan, and the one streaming pass that
+// turns every row the scheduler has to look at into a 32-byte record inside its replica's range.
 //
-// Matrix mode (default): the table is cut into tiles; k_count writes one histogram row per tile,
-// k_colscan turns the columns into exclusive prefixes, and k_regroup places each row at
-//   seg_begin[replica] + (rows of that replica in earlier tiles) + (rank inside the tile, row order)
-// which is a stable partition without a single global atomic.
-// Atomic mode (very many replicas, so the tile matrix would be too large): global counters and
-// global fill cursors; rows land in any order inside a replica's range, which the sort repairs.
+// A row is ACTIVE when it is in flight or in the visible queue; everything else (not yet arrived,
+// finished, rejected, bad data) is inactive: it only needs a place at the end of its replica's
+// order.  Each replica's range [seg_begin[r], seg_begin[r+1]) holds its active rows first.
+//
+// Matrix mode (default): the table is cut into tiles; k_count classifies every row once (one flag
+// byte per row) and writes two histogram rows per tile (all rows, active rows); k_colscan turns the
+// columns into exclusive prefixes; k_regroup places each row at
+//   range start + (rows of its replica and class in earlier tiles) + (rank inside the tile, row order)
+// which is a stable partition without a single global atomic.  When additionally req_id rises with
+// the row index (the step is then "ordered"), inactive rows need no record at all: the regroup
+// writes their outputs and their place in the order directly.
+// Atomic mode (very many replicas, so the tile matrices would be too large): global counters and
+// global fill cursors; rows land in any order inside their class, which the sort repairs.
 #include "hfx_internal.cuh"
 
 #define THREADS_TILE 512
 #define GROUP_MAX 64      // largest same-replica group of an unsorted tile that is ranked by scanning
 
+__device__ __forceinline__ int bucket_of(int rid, int R) { return (rid < 0 || rid >= R) ? R : rid; }
+
+// Kind of a row (KIND_*), with ROWFLAG_BADREP for a row bound to no replica; raises status bits.
+__device__ __forceinline__ uint32_t classify_row(const HfxParams &p, int32_t rid, uint32_t cls, uint32_t st, int32_t prompt,
+                                                 int32_t gen, int64_t arrival, const int64_t *now, uint32_t &bad) {
+  if (rid < 0 || rid >= p.n_replicas) { bad |= HFX_ST_BAD_REPLICA; return KIND_DEAD | ROWFLAG_BADREP; }
+  bool ok = true;
+  if (cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
+  if (prompt < 0 || prompt > HFX_MAX_TOKENS || gen < 0 || gen > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }
+  if (!ok) return KIND_DEAD;
+  if (st == HFX_RUNNING) return KIND_RUNNING;
+  if (st == HFX_QUEUED) return arrival <= __ldg(now + rid) ? KIND_QUEUED : KIND_FUTURE;
+  return KIND_DEAD;
+}
+
 // ------------------------------------------------------------------------------------------------
-// k_count: rows per replica of one tile.  Bad replica ids go to bucket R and raise a status bit.
-// M != nullptr: M[tile][0..R] = the tile's histogram (plain stores).  M == nullptr: global counters.
+// k_count: classify the rows of one tile, count them per replica (all / active), note how the
+// regroup will rank the tile's rows, and whether the step can be "ordered".
+// Matrix mode: M[tile][0][0..R] = all rows, M[tile][1][0..R] = active rows (plain stores).
+// Atomic mode (M == nullptr): global counters tot_all / tot_act; never ordered.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(THREADS_TILE) k_count(const int32_t *__restrict__ replica_id, int64_t n, int32_t R,
-                                                        int32_t tile_rows, uint32_t *__restrict__ M,
-                                                        uint32_t *__restrict__ seg_count, uint32_t *__restrict__ status) {
-  extern __shared__ uint32_t hist[];
-  const int R1 = R + 1;
-  const bool use_smem = M != nullptr;
-  if (use_smem) {
-    for (int i = threadIdx.x; i < R1; i += blockDim.x) hist[i] = 0;
+struct CountArgs {
+  const int32_t *replica_id; const uint8_t *class_id; const uint8_t *state; const int32_t *prompt_len;
+  const int32_t *gen; const int64_t *arrival; const int32_t *req_id; const int64_t *now;
+  int64_t n; int32_t tile_rows;
+  uint32_t *M; uint8_t *tile_mode; uint32_t *tot_all; uint32_t *tot_act;
+  uint8_t *rowflag; uint32_t *status; uint32_t *ordered;
+};
+
+__global__ void __launch_bounds__(THREADS_TILE) k_count(const HfxParams p, const CountArgs a) {
+  extern __shared__ uint32_t s_hist[];    // [2][R1]
+  const int R = p.n_replicas, R1 = R + 1;
+  const bool matrix = a.M != nullptr;
+  uint32_t *h_all = s_hist, *h_act = s_hist + R1;
+  if (matrix) {
+    for (int i = threadIdx.x; i < 2 * R1; i += blockDim.x) s_hist[i] = 0;
     __syncthreads();
   }
-  const int64_t lo = (int64_t)blockIdx.x * tile_rows;
-  const int64_t hi = lo + tile_rows < n ? lo + tile_rows : n;
+  const int64_t lo = (int64_t)blockIdx.x * a.tile_rows;
+  const int64_t hi = lo + a.tile_rows < a.n ? lo + a.tile_rows : a.n;
+  const int nt = hi > lo ? (int)(hi - lo) : 0;
+  const int nvec = nt >> 2;
+  const int64_t v0 = lo >> 2;
   uint32_t bad = 0;
-  const int64_t nvec = hi > lo ? (hi - lo) >> 2 : 0;
-  const int4 *rid4 = reinterpret_cast<const int4 *>(replica_id + lo);
-  for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
-    const int4 r = __ldg(rid4 + v);
-    const int rr[4] = {r.x, r.y, r.z, r.w};
+  int sorted = 1, rising = 1;
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+    const int64_t gv = v0 + v;
+    const int4 rid = __ldg(reinterpret_cast<const int4 *>(a.replica_id) + gv);
+    const uchar4 cls = __ldg(reinterpret_cast<const uchar4 *>(a.class_id) + gv);
+    const uchar4 st = __ldg(reinterpret_cast<const uchar4 *>(a.state) + gv);
+    const int4 pr = __ldg(reinterpret_cast<const int4 *>(a.prompt_len) + gv);
+    const int4 ge = __ldg(reinterpret_cast<const int4 *>(a.gen) + gv);
+    const int4 id = __ldg(reinterpret_cast<const int4 *>(a.req_id) + gv);
+    const longlong2 ar0 = __ldg(reinterpret_cast<const longlong2 *>(a.arrival) + 2 * gv);
+    const longlong2 ar1 = __ldg(reinterpret_cast<const longlong2 *>(a.arrival) + 2 * gv + 1);
+    const int rr[4] = {rid.x, rid.y, rid.z, rid.w};
+    const uint32_t cc[4] = {cls.x, cls.y, cls.z, cls.w}, ss[4] = {st.x, st.y, st.z, st.w};
+    const int pp[4] = {pr.x, pr.y, pr.z, pr.w}, gg[4] = {ge.x, ge.y, ge.z, ge.w};
+    const int64_t aa[4] = {ar0.x, ar0.y, ar1.x, ar1.y};
+    uint32_t fl[4];
+    int b[5];
 #pragma unroll
     for (int k = 0; k < 4; k++) {
-      int b = rr[k];
-      if (b < 0 || b >= R) { b = R; bad = 1; }
-      if (use_smem) atomicAdd(&hist[b], 1u); else atomicAdd(&seg_count[b], 1u);
+      fl[k] = classify_row(p, rr[k], cc[k], ss[k], pp[k], gg[k], aa[k], a.now, bad);
+      b[k] = bucket_of(rr[k], R);
+      if (matrix) { atomicAdd(&h_all[b[k]], 1u); if (fl[k] <= KIND_QUEUED) atomicAdd(&h_act[b[k]], 1u); }
+      else { atomicAdd(&a.tot_all[b[k]], 1u); if (fl[k] <= KIND_QUEUED) atomicAdd(&a.tot_act[b[k]], 1u); }
     }
+    *reinterpret_cast<uchar4 *>(a.rowflag + (gv << 2)) = make_uchar4(fl[0], fl[1], fl[2], fl[3]);
+    // sorted by replica inside the tile?  req_id rising along the table (also across tiles)?
+    const int64_t nxt = (gv << 2) + 4;
+    b[4] = nxt < hi ? bucket_of(__ldg(a.replica_id + nxt), R) : b[3];
+    if (b[0] > b[1] || b[1] > b[2] || b[2] > b[3] || b[3] > b[4]) sorted = 0;
+    if (!(id.x < id.y && id.y < id.z && id.z < id.w && (nxt >= a.n || id.w < __ldg(a.req_id + nxt)))) rising = 0;
   }
-  for (int64_t i = lo + (nvec << 2) + threadIdx.x; i < hi; i += blockDim.x) {
-    int b = replica_id[i];
-    if (b < 0 || b >= R) { b = R; bad = 1; }
-    if (use_smem) atomicAdd(&hist[b], 1u); else atomicAdd(&seg_count[b], 1u);
+  for (int i = (nvec << 2) + threadIdx.x; i < nt; i += blockDim.x) {
+    const int64_t g = lo + i;
+    const int32_t rid = a.replica_id[g];
+    const uint32_t fl = classify_row(p, rid, a.class_id[g], a.state[g], a.prompt_len[g], a.gen[g], a.arrival[g], a.now, bad);
+    const int b = bucket_of(rid, R);
+    if (matrix) { atomicAdd(&h_all[b], 1u); if (fl <= KIND_QUEUED) atomicAdd(&h_act[b], 1u); }
+    else { atomicAdd(&a.tot_all[b], 1u); if (fl <= KIND_QUEUED) atomicAdd(&a.tot_act[b], 1u); }
+    a.rowflag[g] = (uint8_t)fl;
+    if (g + 1 < hi && b > bucket_of(a.replica_id[g + 1], R)) sorted = 0;
+    if (g + 1 < a.n && !(a.req_id[g] < a.req_id[g + 1])) rising = 0;
   }
-  if (bad) atomicOr(status, HFX_ST_BAD_REPLICA);
-  if (use_smem) {
-    __syncthreads();
-    uint32_t *row = M + (size_t)blockIdx.x * R1;
-    for (int i = threadIdx.x; i < R1; i += blockDim.x) row[i] = hist[i];
+  if (bad) atomicOr(a.status, bad);
+  if (!matrix) return;
+  sorted = __syncthreads_and(sorted);      // also orders the histogram updates before the reads below
+  rising = __syncthreads_and(rising);
+  uint32_t *row = a.M + (size_t)blockIdx.x * 2 * R1;
+  uint32_t mx = 0;
+  for (int i = threadIdx.x; i < 2 * R1; i += blockDim.x) {
+    const uint32_t c = s_hist[i];
+    row[i] = c;
+    if (i < R1) mx = c > mx ? c : mx;
+  }
+  const int small_groups = __syncthreads_and(mx <= GROUP_MAX);
+  if (threadIdx.x == 0) {
+    const int mode = sorted ? TILE_SORTED : (small_groups ? TILE_GROUPS : TILE_ANY);
+    a.tile_mode[blockIdx.x] = (uint8_t)mode;
+    if (mode == TILE_ANY || !rising) *a.ordered = 0;
   }
 }
 
 // ------------------------------------------------------------------------------------------------
-// k_colscan: for each replica (column) the exclusive prefix of its counts over the tiles, in place,
-// and the column total.  Block = 32 columns x 32 chunks of tiles.
+// k_colscan: for each column of the tile matrix (2 x (R+1) columns: all rows, active rows) the
+// exclusive prefix of its counts over the tiles, in place, and the column total.
+// Block = 32 columns x 32 chunks of tiles.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) k_colscan(uint32_t *__restrict__ M, int32_t n_tiles, int32_t R1,
-                                                  uint32_t *__restrict__ tot) {
+                                                  uint32_t *__restrict__ tot_all, uint32_t *__restrict__ tot_act) {
   __shared__ uint32_t part[32][33];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int C = 2 * R1;
   const int col = blockIdx.x * 32 + lane;
   const int cb = (n_tiles + 31) / 32;
   const int t0 = w * cb < n_tiles ? w * cb : n_tiles;
   const int t1 = (t0 + cb < n_tiles) ? t0 + cb : n_tiles;
   uint32_t sum = 0;
-  if (col < R1)
-    for (int t = t0; t < t1; t++) sum += M[(size_t)t * R1 + col];
+  if (col < C)
+    for (int t = t0; t < t1; t++) sum += M[(size_t)t * C + col];
   part[w][lane] = sum;
   __syncthreads();
   uint32_t pre = 0;
   for (int k = 0; k < w; k++) pre += part[k][lane];
-  if (col < R1) {
+  if (col < C) {
     uint32_t run = pre;
     for (int t = t0; t < t1; t++) {
-      const size_t idx = (size_t)t * R1 + col;
+      const size_t idx = (size_t)t * C + col;
       const uint32_t v = M[idx];
       M[idx] = run;
       run += v;
     }
-    if (w == 31) tot[col] = pre + sum;
+    if (w == 31) { if (col < R1) tot_all[col] = pre + sum; else tot_act[col - R1] = pre + sum; }
   }
 }
 
 // ------------------------------------------------------------------------------------------------
-// k_offsets: exclusive scan of the per-replica totals (one block) -> seg_begin, the user-visible
-// seg_off, the fill cursors of the atomic mode, and the step's flags:
-// flags[0] = 1 says "records of a replica are in row order and req_id rises with the row index"
-// (k_regroup clears it when it finds otherwise); flags[1] = largest segment.
+// k_offsets: exclusive scan of the per-replica totals (one block) -> seg_begin and the user-visible
+// seg_off; zeroes the fill cursors of the atomic mode; flags[2] = the largest number of items any
+// replica has to sort (its active rows; without "ordered" also its inactive rows); re-arms the
+// "ordered" word of the next step.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) k_offsets(const uint32_t *__restrict__ tot, int32_t R,
-                                                  uint32_t *__restrict__ seg_begin, uint32_t *__restrict__ cursor,
+__global__ void __launch_bounds__(1024) k_offsets(const uint32_t *__restrict__ tot_all, const uint32_t *__restrict__ tot_act,
+                                                  int32_t R, uint32_t *__restrict__ seg_begin, uint32_t *__restrict__ cursor,
                                                   int32_t *__restrict__ seg_off, uint32_t *__restrict__ flags,
-                                                  uint32_t ordered_init) {
+                                                  uint32_t parity, uint32_t force_unordered) {
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t carry_s, max_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) { carry_s = 0; max_s = 0; }
+  if (threadIdx.x == 0) { carry_s = 0; max_s = 0; if (force_unordered) flags[parity] = 0; }
   __syncthreads();
+  const bool ordered = flags[parity] != 0;
   const int total = R + 1;  // buckets 0..R
   uint32_t mx = 0;
   for (int base = 0; base < total; base += blockDim.x) {
     const int i = base + threadIdx.x;
-    const uint32_t c = i < total ? tot[i] : 0;
-    mx = c > mx ? c : mx;
+    const uint32_t c = i < total ? tot_all[i] : 0;
+    if (i < total) {
+      const uint32_t act = tot_act[i];
+      const uint32_t need = ordered ? act : (act > c - act ? act : c - act);
+      mx = need > mx ? need : mx;
+    }
     uint32_t v = c;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
@@ -121,7 +198,8 @@ __global__ void __launch_bounds__(1024) k_offsets(const uint32_t *__restrict__ t
     const uint32_t excl = carry_s + (warp ? warp_tot[warp - 1] : 0) + v - c;
     if (i < total) {
       seg_begin[i] = excl;
-      cursor[i] = excl;
+      cursor[i] = 0;
+      cursor[R + 2 + i] = 0;
       seg_off[i] = (int32_t)excl;   // seg_off[R] = number of rows bound to a valid replica
     }
     __syncthreads();
@@ -132,7 +210,7 @@ __global__ void __launch_bounds__(1024) k_offsets(const uint32_t *__restrict__ t
   for (int o = 16; o > 0; o >>= 1) { const uint32_t x = __shfl_xor_sync(0xffffffffu, mx, o); mx = x > mx ? x : mx; }
   if (lane == 0) atomicMax(&max_s, mx);
   __syncthreads();
-  if (threadIdx.x == 0) { seg_begin[total] = carry_s; flags[0] = ordered_init; flags[1] = max_s; }
+  if (threadIdx.x == 0) { seg_begin[total] = carry_s; flags[2] = max_s; flags[parity ^ 1u] = 1u; }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -141,54 +219,42 @@ __global__ void __launch_bounds__(1024) k_offsets(const uint32_t *__restrict__ t
 // ------------------------------------------------------------------------------------------------
 struct RowIn {
   int32_t rid, prompt, gen, req_id, weight, out_len;
-  uint32_t cls, st;
+  uint32_t cls, kind;      // kind: the row's flag byte from k_count
   int64_t arrival, first_token;
 };
 
-__device__ __forceinline__ void make_record(const HfxParams &p, const RegroupArgs &a, const int64_t *s_ttft,
-                                            const int64_t *s_tpot, const uint8_t *s_prio, int64_t i, const RowIn &in,
-                                            HfxRec &r, uint32_t &bad) {
-  const int32_t R = p.n_replicas;
+// Fills the record of a row of kind in.kind; returns the row's predicted TTFT (0 if inactive).
+__device__ __forceinline__ int64_t make_record(const HfxParams &p, const RegroupArgs &a, const int64_t *s_ttft,
+                                               const int64_t *s_tpot, const uint8_t *s_prio, int64_t i, const RowIn &in,
+                                               HfxRec &r) {
   r.req_id = in.req_id; r.row = (int32_t)i; r.prompt = in.prompt; r.gen = in.gen; r.output_len = in.out_len;
-  r.cls = (uint8_t)in.cls; r.kind = KIND_DEAD; r.prio = 63; r.pad = 0; r.base = 0;
+  r.cls = (uint8_t)in.cls; r.kind = (uint8_t)(in.kind & 3u); r.prio = 63; r.pad = 0; r.base = 0;
   int64_t pred_ttft = 0;
-  if (in.rid >= 0 && in.rid < R) {   // a bad replica id was flagged by k_count
-    bool ok = true;
-    if (in.cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
-    if (in.prompt < 0 || in.prompt > HFX_MAX_TOKENS || in.gen < 0 || in.gen > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }
-    if (ok) {
-      const int64_t now = __ldg(a.now + in.rid), mat = __ldg(a.mat + in.rid);
-      const int32_t mode = __ldg(&a.cfg[in.rid].mode);
-      const int64_t start = now > mat ? now : mat;
-      int prio;
-      if (p.weight_max > 0) {
-        const int64_t w = (int64_t)p.weight_max - in.weight;
-        prio = (int)(w < 0 ? 0 : (w > 62 ? 62 : w));
-      } else prio = s_prio[in.cls];
-      const int64_t ttft = s_ttft[in.cls], tpot = s_tpot[in.cls];
-      if (in.st == HFX_RUNNING) {
-        r.kind = KIND_RUNNING; r.prio = (uint8_t)prio;
-        r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot - now : BASE_UNBOUNDED;
-        pred_ttft = in.first_token - in.arrival;
-      } else if (in.st == HFX_QUEUED) {
-        if (in.arrival <= now) {
-          r.kind = KIND_QUEUED; r.prio = (uint8_t)prio;
-          if (mode == HFX_DECODE) {
-            r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot - start - p.d2 * ((int64_t)in.prompt + in.gen)
-                              : BASE_UNBOUNDED;
-            pred_ttft = in.first_token - in.arrival;
-          } else {
-            pred_ttft = (start - in.arrival) + dev_Ep(p, in.prompt);
-            r.base = ttft > 0 ? ttft - pred_ttft : BASE_UNBOUNDED;
-          }
-        } else {
-          r.kind = KIND_FUTURE;
-          r.base = in.arrival;
-        }
-      }
+  if (in.kind == KIND_FUTURE) r.base = in.arrival;
+  else if (in.kind <= KIND_QUEUED) {
+    const int64_t now = __ldg(a.now + in.rid), mat = __ldg(a.mat + in.rid);
+    const int32_t mode = __ldg(&a.cfg[in.rid].mode);
+    const int64_t start = now > mat ? now : mat;
+    int prio;
+    if (p.weight_max > 0) {
+      const int64_t w = (int64_t)p.weight_max - in.weight;
+      prio = (int)(w < 0 ? 0 : (w > 62 ? 62 : w));
+    } else prio = s_prio[in.cls];
+    r.prio = (uint8_t)prio;
+    const int64_t ttft = s_ttft[in.cls], tpot = s_tpot[in.cls];
+    if (in.kind == KIND_RUNNING) {
+      r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot - now : BASE_UNBOUNDED;
+      pred_ttft = in.first_token - in.arrival;
+    } else if (mode == HFX_DECODE) {
+      r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot - start - p.d2 * ((int64_t)in.prompt + in.gen)
+                        : BASE_UNBOUNDED;
+      pred_ttft = in.first_token - in.arrival;
+    } else {
+      pred_ttft = (start - in.arrival) + dev_Ep(p, in.prompt);
+      r.base = ttft > 0 ? ttft - pred_ttft : BASE_UNBOUNDED;
     }
   }
-  if (a.pred_ttft) a.pred_ttft[i] = pred_ttft;
+  return pred_ttft;
 }
 
 __device__ __forceinline__ void store_record(HfxRec *rec, uint32_t pos, const HfxRec &r) {
@@ -199,10 +265,10 @@ __device__ __forceinline__ void store_record(HfxRec *rec, uint32_t pos, const Hf
 }
 
 // rows 4v .. 4v+3 with 16-byte loads
-__device__ __forceinline__ void load_rows4(const RegroupArgs &a, int64_t v, RowIn in[4]) {
+__device__ __forceinline__ void load_rows4(const RegroupArgs &a, const uint8_t *rowflag, int64_t v, RowIn in[4]) {
   const int4 rid = __ldg(reinterpret_cast<const int4 *>(a.replica_id) + v);
   const uchar4 cls = __ldg(reinterpret_cast<const uchar4 *>(a.class_id) + v);
-  const uchar4 st = __ldg(reinterpret_cast<const uchar4 *>(a.state) + v);
+  const uchar4 kd = __ldg(reinterpret_cast<const uchar4 *>(rowflag) + v);
   const int4 pr = __ldg(reinterpret_cast<const int4 *>(a.prompt_len) + v);
   const int4 ge = __ldg(reinterpret_cast<const int4 *>(a.gen) + v);
   const int4 id = __ldg(reinterpret_cast<const int4 *>(a.req_id) + v);
@@ -213,15 +279,15 @@ __device__ __forceinline__ void load_rows4(const RegroupArgs &a, int64_t v, RowI
   int4 we = make_int4(0, 0, 0, 0), ol = make_int4(0, 0, 0, 0);
   if (a.weight) we = __ldg(reinterpret_cast<const int4 *>(a.weight) + v);
   if (a.output_len) ol = __ldg(reinterpret_cast<const int4 *>(a.output_len) + v);
-  in[0] = {rid.x, pr.x, ge.x, id.x, we.x, ol.x, cls.x, st.x, ar0.x, ft0.x};
-  in[1] = {rid.y, pr.y, ge.y, id.y, we.y, ol.y, cls.y, st.y, ar0.y, ft0.y};
-  in[2] = {rid.z, pr.z, ge.z, id.z, we.z, ol.z, cls.z, st.z, ar1.x, ft1.x};
-  in[3] = {rid.w, pr.w, ge.w, id.w, we.w, ol.w, cls.w, st.w, ar1.y, ft1.y};
+  in[0] = {rid.x, pr.x, ge.x, id.x, we.x, ol.x, cls.x, kd.x, ar0.x, ft0.x};
+  in[1] = {rid.y, pr.y, ge.y, id.y, we.y, ol.y, cls.y, kd.y, ar0.y, ft0.y};
+  in[2] = {rid.z, pr.z, ge.z, id.z, we.z, ol.z, cls.z, kd.z, ar1.x, ft1.x};
+  in[3] = {rid.w, pr.w, ge.w, id.w, we.w, ol.w, cls.w, kd.w, ar1.y, ft1.y};
 }
 
-__device__ __forceinline__ void load_row1(const RegroupArgs &a, int64_t i, RowIn &in) {
+__device__ __forceinline__ void load_row1(const RegroupArgs &a, const uint8_t *rowflag, int64_t i, RowIn &in) {
   in = {a.replica_id[i], a.prompt_len[i], a.gen[i], a.req_id[i], a.weight ? a.weight[i] : 0,
-        a.output_len ? a.output_len[i] : 0, a.class_id[i], a.state[i], a.arrival[i], a.first_token[i]};
+        a.output_len ? a.output_len[i] : 0, a.class_id[i], rowflag[i], a.arrival[i], a.first_token[i]};
 }
 
 __device__ __forceinline__ void stage_classes(const HfxParams &p, int64_t *s_ttft, int64_t *s_tpot, uint8_t *s_prio) {
@@ -232,185 +298,213 @@ __device__ __forceinline__ void stage_classes(const HfxParams &p, int64_t *s_ttf
   }
 }
 
-// atomic mode: positions from global fill cursors (any order inside a replica's range)
-__global__ void __launch_bounds__(256) k_regroup_atomic(const HfxParams p, const RegroupArgs a, uint32_t *__restrict__ cursor,
-                                                        HfxRec *__restrict__ rec, uint32_t *__restrict__ status) {
+// the outputs of an inactive row, written by the regroup of an ordered step
+__device__ __forceinline__ void write_inactive(const RegroupArgs &a, int64_t i, uint32_t opos, int bkt) {
+  a.order[opos] = (int32_t)i;
+  a.slack[i] = 0;
+  a.admit[i] = 0;
+  if (a.pred_tpot) a.pred_tpot[i] = 0;
+  if (a.key) a.key[i] = ((uint64_t)(bkt & 0xffff) << 48) | dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
+}
+
+// atomic mode: positions from global fill cursors (any order inside a replica's two classes)
+__global__ void __launch_bounds__(256) k_regroup_atomic(const HfxParams p, const RegroupArgs a, const uint8_t *__restrict__ rowflag,
+                                                        const uint32_t *__restrict__ seg_begin,
+                                                        const uint32_t *__restrict__ tot_act, uint32_t *__restrict__ cursor,
+                                                        HfxRec *__restrict__ rec) {
   __shared__ int64_t s_ttft[HFX_MAX_CLASSES], s_tpot[HFX_MAX_CLASSES];
   __shared__ uint8_t s_prio[HFX_MAX_CLASSES];
   stage_classes(p, s_ttft, s_tpot, s_prio);
   __syncthreads();
-  uint32_t bad = 0;
   const int R = p.n_replicas;
+  auto emit = [&](int64_t i, const RowIn &in) {
+    HfxRec r;
+    const int64_t pt = make_record(p, a, s_ttft, s_tpot, s_prio, i, in, r);
+    if (a.pred_ttft) a.pred_ttft[i] = pt;
+    const int bkt = bucket_of(in.rid, R);
+    const uint32_t pos = in.kind <= KIND_QUEUED ? seg_begin[bkt] + atomicAdd(&cursor[bkt], 1u)
+                                                : seg_begin[bkt] + tot_act[bkt] + atomicAdd(&cursor[R + 2 + bkt], 1u);
+    store_record(rec, pos, r);
+  };
   const int64_t n4 = a.n >> 2;
   for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < n4; v += (int64_t)gridDim.x * blockDim.x) {
     RowIn in[4];
-    load_rows4(a, v, in);
+    load_rows4(a, rowflag, v, in);
 #pragma unroll
-    for (int k = 0; k < 4; k++) {
-      HfxRec r;
-      make_record(p, a, s_ttft, s_tpot, s_prio, (v << 2) + k, in[k], r, bad);
-      const int bucket = (in[k].rid < 0 || in[k].rid >= R) ? R : in[k].rid;
-      store_record(rec, atomicAdd(&cursor[bucket], 1u), r);
-    }
+    for (int k = 0; k < 4; k++) emit((v << 2) + k, in[k]);
   }
   if (blockIdx.x == 0) {
     for (int64_t i = (n4 << 2) + threadIdx.x; i < a.n; i += blockDim.x) {
-      RowIn in; HfxRec r;
-      load_row1(a, i, in);
-      make_record(p, a, s_ttft, s_tpot, s_prio, i, in, r, bad);
-      const int bucket = (in.rid < 0 || in.rid >= R) ? R : in.rid;
-      store_record(rec, atomicAdd(&cursor[bucket], 1u), r);
+      RowIn in;
+      load_row1(a, rowflag, i, in);
+      emit(i, in);
     }
   }
-  if (bad) atomicOr(status, bad);
 }
 
-// clamp of a replica id to its bucket (bad ids share bucket R)
-__device__ __forceinline__ int bucket_of(int rid, int R) { return (rid < 0 || rid >= R) ? R : rid; }
+// matrix mode: see the head of this file
+struct TileArgs {
+  const uint32_t *M; const uint8_t *tile_mode; const uint32_t *seg_begin; const uint32_t *tot_act;
+  const uint8_t *rowflag; const uint32_t *ordered; int64_t *fmin; HfxRec *rec; int32_t tile_rows;
+};
 
-// matrix mode: tile t writes its rows of replica r at seg_begin[r] + M[t][r] + (rank of the row
-// among the tile's rows of r, in row order).  The rank comes from the tile being sorted by replica
-// already (grouped tables), or from a small shared-memory counting sort of the tile.
-__global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, const RegroupArgs a, int32_t tile_rows,
-                                                          const uint32_t *__restrict__ M,
-                                                          const uint32_t *__restrict__ seg_begin, HfxRec *__restrict__ rec,
-                                                          uint32_t *__restrict__ status, uint32_t *__restrict__ flags) {
+__global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, const RegroupArgs a, const TileArgs ta) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int R = p.n_replicas, R1 = R + 1;
-  uint32_t *s_cnt = reinterpret_cast<uint32_t *>(smem_raw);           // [R1]   rows of each replica in the tile
-  uint32_t *s_off = s_cnt + R1;                                        // [R1+1] exclusive prefix of s_cnt
-  uint32_t *s_base = s_off + R1 + 1;                                   // [R1]   global position of the tile's first row of r
-  uint16_t *s_stage = reinterpret_cast<uint16_t *>(s_base + R1);       // [tile_rows] tile rows grouped by replica
+  const int R = p.n_replicas, R1 = R + 1, T = ta.tile_rows;
+  int64_t *s_fmin = reinterpret_cast<int64_t *>(smem_raw);           // [R1] earliest not-yet-arrived row per replica
+  uint32_t *s_cnt = reinterpret_cast<uint32_t *>(s_fmin + R1);       // [R1]   rows of each replica in the tile / cursors
+  uint32_t *s_off = s_cnt + R1;                                      // [R1+1] exclusive prefix of s_cnt / cursors
+  uint32_t *s_bact = s_off + R1 + 1;                                 // [R1]   where the tile's active rows of r start
+  uint32_t *s_bin = s_bact + R1;                                     // [R1]   where its inactive rows start
+  uint16_t *s_stage = reinterpret_cast<uint16_t *>(s_bin + R1);      // [T]    tile rows grouped by replica (+ class bit)
+  uint16_t *s_P = s_stage + T;                                       // [T+1]  active rows before each tile position
   __shared__ int64_t s_ttft[HFX_MAX_CLASSES], s_tpot[HFX_MAX_CLASSES];
   __shared__ uint8_t s_prio[HFX_MAX_CLASSES];
   __shared__ uint32_t s_warp[32];
-  __shared__ uint32_t s_maxcnt;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
+  const int mode = ta.tile_mode[blockIdx.x];
+  const bool ordered = *ta.ordered != 0;
+  const bool use_fmin = ordered && a.commit;
 
   stage_classes(p, s_ttft, s_tpot, s_prio);
-  for (int i = tid; i < R1; i += blockDim.x) s_cnt[i] = 0;
-  if (tid == 0) s_maxcnt = 0;
+  for (int i = tid; i < R1; i += blockDim.x) { s_cnt[i] = 0; s_off[i] = 0; if (use_fmin) s_fmin[i] = HFX_INF; }
   __syncthreads();
 
-  const int64_t lo = (int64_t)blockIdx.x * tile_rows;
-  const int64_t hi = lo + tile_rows < a.n ? lo + tile_rows : a.n;
+  const int64_t lo = (int64_t)blockIdx.x * T;
+  const int64_t hi = lo + T < a.n ? lo + T : a.n;
   const int nt = hi > lo ? (int)(hi - lo) : 0;
   const int nvec = nt >> 2;
-  const int4 *rid4 = reinterpret_cast<const int4 *>(a.replica_id + lo);
-  const uint32_t *Mrow = M + (size_t)blockIdx.x * R1;
+  const int64_t v0 = lo >> 2;
+  const size_t mrow = (size_t)blockIdx.x * 2 * R1;
 
-  // ---- A: histogram of the tile; is the tile already sorted by replica? ----------------------------
-  int sorted = 1;
-  for (int v = tid; v < nvec; v += blockDim.x) {
-    const int4 r4 = __ldg(rid4 + v);
-    int b[5] = {bucket_of(r4.x, R), bucket_of(r4.y, R), bucket_of(r4.z, R), bucket_of(r4.w, R), 0};
-#pragma unroll
-    for (int k = 0; k < 4; k++) atomicAdd(&s_cnt[b[k]], 1u);
-    const int nxt = 4 * v + 4;
-    b[4] = nxt < nt ? bucket_of(__ldg(a.replica_id + lo + nxt), R) : b[3];
-    if (b[0] > b[1] || b[1] > b[2] || b[2] > b[3] || b[3] > b[4]) sorted = 0;
-  }
-  for (int i = (nvec << 2) + tid; i < nt; i += blockDim.x) {
-    const int x = bucket_of(a.replica_id[lo + i], R);
-    atomicAdd(&s_cnt[x], 1u);
-    if (i + 1 < nt && x > bucket_of(a.replica_id[lo + i + 1], R)) sorted = 0;
-  }
-  sorted = __syncthreads_and(sorted);
-
-  // ---- B: exclusive scan of the histogram; global bases; largest group ---------------------------
-  {
-    const int per = (R1 + blockDim.x - 1) / blockDim.x;
-    const int i0 = tid * per < R1 ? tid * per : R1, i1 = (i0 + per < R1) ? i0 + per : R1;
-    uint32_t sum = 0, mx = 0;
-    for (int i = i0; i < i1; i++) { const uint32_t c = s_cnt[i]; sum += c; mx = c > mx ? c : mx; }
-    uint32_t v = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) { const uint32_t x = __shfl_xor_sync(0xffffffffu, mx, o); mx = x > mx ? x : mx; }
-    if (lane == 31) s_warp[warp] = v;
-    if (lane == 0) atomicMax(&s_maxcnt, mx);
-    __syncthreads();
-    if (warp == 0) {
-      uint32_t w = lane < nwarp ? s_warp[lane] : 0;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += x; }
-      s_warp[lane] = w;
+  if (mode != TILE_ANY) {
+    // ---- A: histogram of the tile; active flag of every position ------------------------------------
+    for (int v = tid; v < nvec; v += blockDim.x) {
+      const int4 r4 = __ldg(reinterpret_cast<const int4 *>(a.replica_id) + v0 + v);
+      const uchar4 k4 = __ldg(reinterpret_cast<const uchar4 *>(ta.rowflag) + v0 + v);
+      atomicAdd(&s_cnt[bucket_of(r4.x, R)], 1u); atomicAdd(&s_cnt[bucket_of(r4.y, R)], 1u);
+      atomicAdd(&s_cnt[bucket_of(r4.z, R)], 1u); atomicAdd(&s_cnt[bucket_of(r4.w, R)], 1u);
+      s_P[4 * v] = k4.x <= KIND_QUEUED; s_P[4 * v + 1] = k4.y <= KIND_QUEUED;
+      s_P[4 * v + 2] = k4.z <= KIND_QUEUED; s_P[4 * v + 3] = k4.w <= KIND_QUEUED;
+    }
+    for (int i = (nvec << 2) + tid; i < nt; i += blockDim.x) {
+      atomicAdd(&s_cnt[bucket_of(a.replica_id[lo + i], R)], 1u);
+      s_P[i] = ta.rowflag[lo + i] <= KIND_QUEUED;
     }
     __syncthreads();
-    uint32_t run = (warp ? s_warp[warp - 1] : 0) + v - sum;
-    for (int i = i0; i < i1; i++) { s_off[i] = run; run += s_cnt[i]; }
-    if (tid == 0) s_off[R1] = (uint32_t)nt;
-    for (int i = tid; i < R1; i += blockDim.x) s_base[i] = seg_begin[i] + Mrow[i];
-  }
-  __syncthreads();
-  // how the rank of a row inside its (tile, replica) group is found:
-  // 0 by position (tile sorted by replica), 1 by scanning the group, 2 any order (huge groups)
-  const int mode = sorted ? 0 : (s_maxcnt <= GROUP_MAX ? 1 : 2);
-  if (mode != 0) {
-    for (int i = tid; i < R1; i += blockDim.x) s_cnt[i] = 0;
-    __syncthreads();
-    if (mode == 1) {
-      // ---- C: tile rows grouped by replica (counting sort of the local indices) ----------------
-      for (int v = tid; v < nvec; v += blockDim.x) {
-        const int4 r4 = __ldg(rid4 + v);
-        const int b[4] = {bucket_of(r4.x, R), bucket_of(r4.y, R), bucket_of(r4.z, R), bucket_of(r4.w, R)};
+    // ---- B: exclusive scan of the histogram ---------------------------------------------------------
+    {
+      const int per = (R1 + blockDim.x - 1) / blockDim.x;
+      const int i0 = tid * per < R1 ? tid * per : R1, i1 = (i0 + per < R1) ? i0 + per : R1;
+      uint32_t sum = 0;
+      for (int i = i0; i < i1; i++) sum += s_cnt[i];
+      uint32_t v = sum;
 #pragma unroll
-        for (int k = 0; k < 4; k++) s_stage[s_off[b[k]] + atomicAdd(&s_cnt[b[k]], 1u)] = (uint16_t)(4 * v + k);
-      }
-      for (int i = (nvec << 2) + tid; i < nt; i += blockDim.x) {
-        const int x = bucket_of(a.replica_id[lo + i], R);
-        s_stage[s_off[x] + atomicAdd(&s_cnt[x], 1u)] = (uint16_t)i;
+      for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+      if (lane == 31) s_warp[warp] = v;
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t w = lane < nwarp ? s_warp[lane] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += x; }
+        s_warp[lane] = w;
       }
       __syncthreads();
+      uint32_t run = (warp ? s_warp[warp - 1] : 0) + v - sum;
+      for (int i = i0; i < i1; i++) { s_off[i] = run; run += s_cnt[i]; }
+      if (tid == 0) s_off[R1] = (uint32_t)nt;
+    }
+    __syncthreads();
+    if (mode == TILE_SORTED) {
+      // ---- C0: s_P := number of active rows before each position (exclusive scan, in place) -----------
+      const int per = (nt + blockDim.x - 1) / blockDim.x;
+      const int i0 = tid * per < nt ? tid * per : nt, i1 = (i0 + per < nt) ? i0 + per : nt;
+      uint32_t sum = 0;
+      for (int i = i0; i < i1; i++) sum += s_P[i];
+      uint32_t v = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+      if (lane == 31) s_warp[warp] = v;
+      __syncthreads();
+      if (warp == 0) {
+        uint32_t w = lane < nwarp ? s_warp[lane] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += x; }
+        s_warp[lane] = w;
+      }
+      __syncthreads();
+      uint32_t run = (warp ? s_warp[warp - 1] : 0) + v - sum;
+      for (int i = i0; i < i1; i++) { const uint32_t f = s_P[i]; s_P[i] = (uint16_t)run; run += f; }
+      if (i1 == nt && i0 < nt) s_P[nt] = (uint16_t)run;
+      if (nt == 0 && tid == 0) s_P[0] = 0;
+    } else {
+      // ---- C1: tile rows grouped by replica (counting sort of local indices, class in bit 15) ---------
+      for (int i = tid; i < R1; i += blockDim.x) s_cnt[i] = 0;
+      __syncthreads();
+      for (int i = tid; i < nt; i += blockDim.x) {
+        const int b = bucket_of(__ldg(a.replica_id + lo + i), R);
+        s_stage[s_off[b] + atomicAdd(&s_cnt[b], 1u)] = (uint16_t)(i | (s_P[i] ? 0x8000 : 0));
+      }
     }
   }
+  for (int i = tid; i < R1; i += blockDim.x) {
+    const uint32_t m_all = ta.M[mrow + i], m_act = ta.M[mrow + R1 + i], sb = ta.seg_begin[i];
+    s_bact[i] = sb + m_act;
+    s_bin[i] = sb + ta.tot_act[i] + (m_all - m_act);
+  }
+  __syncthreads();
 
-  // ---- D: records -----------------------------------------------------------------------------------
-  uint32_t bad = 0;
-  int ordered = mode != 2;
-  auto place = [&](int rid, int il) -> uint32_t {
-    const int bkt = bucket_of(rid, R);
+  // ---- D: records of active rows; inactive rows: their outputs (ordered) or their records ----------
+  auto emit = [&](int64_t i, int il, const RowIn &in) {
+    const int bkt = bucket_of(in.rid, R);
+    const bool act = in.kind <= KIND_QUEUED;
     uint32_t rank;
-    if (mode == 0) rank = (uint32_t)il - s_off[bkt];
-    else if (mode == 1) {
+    if (mode == TILE_SORTED) {
+      const uint32_t o = s_off[bkt];
+      const uint32_t ra = (uint32_t)s_P[il] - (uint32_t)s_P[o];
+      rank = act ? ra : (uint32_t)il - o - ra;
+    } else if (mode == TILE_GROUPS) {
       rank = 0;
       const uint32_t g0 = s_off[bkt], g1 = s_off[bkt + 1];
-      for (uint32_t g = g0; g < g1; g++) rank += s_stage[g] < (uint32_t)il ? 1u : 0u;
-    } else rank = atomicAdd(&s_cnt[bkt], 1u);
-    return s_base[bkt] + rank;
+      const uint32_t me = (uint32_t)il | (act ? 0x8000u : 0u);
+      for (uint32_t g = g0; g < g1; g++) { const uint32_t e = s_stage[g]; rank += ((e ^ me) < 0x8000u && e < me) ? 1u : 0u; }
+    } else rank = atomicAdd(act ? &s_cnt[bkt] : &s_off[bkt], 1u);
+    if (act || !ordered) {
+      HfxRec r;
+      const int64_t pt = make_record(p, a, s_ttft, s_tpot, s_prio, i, in, r);
+      if (a.pred_ttft) a.pred_ttft[i] = pt;
+      store_record(ta.rec, (act ? s_bact[bkt] : s_bin[bkt]) + rank, r);
+    } else {
+      if (a.pred_ttft) a.pred_ttft[i] = 0;
+      write_inactive(a, i, s_bin[bkt] + rank, bkt);
+      if (use_fmin && in.kind == KIND_FUTURE) atomicMin(reinterpret_cast<long long *>(&s_fmin[bkt]), (long long)in.arrival);
+    }
   };
-  const int64_t v0 = lo >> 2;
   for (int v = tid; v < nvec; v += blockDim.x) {
     RowIn in[4];
-    load_rows4(a, v0 + v, in);
-    // req_id must rise with the row index for the order of equal keys to come for free
-    const int64_t nxt = lo + 4 * (int64_t)v + 4;
-    const bool has_next = nxt < a.n;
-    const int32_t id_next = has_next ? __ldg(a.req_id + nxt) : 0;
-    if (!(in[0].req_id < in[1].req_id && in[1].req_id < in[2].req_id && in[2].req_id < in[3].req_id &&
-          (!has_next || in[3].req_id < id_next))) ordered = 0;
+    load_rows4(a, ta.rowflag, v0 + v, in);
 #pragma unroll
-    for (int k = 0; k < 4; k++) {
-      HfxRec r;
-      make_record(p, a, s_ttft, s_tpot, s_prio, lo + 4 * (int64_t)v + k, in[k], r, bad);
-      store_record(rec, place(in[k].rid, 4 * v + k), r);
-    }
+    for (int k = 0; k < 4; k++) emit(lo + 4 * (int64_t)v + k, 4 * v + k, in[k]);
   }
   for (int i = (nvec << 2) + tid; i < nt; i += blockDim.x) {
-    RowIn in; HfxRec r;
-    load_row1(a, lo + i, in);
-    if (lo + i + 1 < a.n && !(in.req_id < a.req_id[lo + i + 1])) ordered = 0;
-    make_record(p, a, s_ttft, s_tpot, s_prio, lo + i, in, r, bad);
-    store_record(rec, place(in.rid, i), r);
+    RowIn in;
+    load_row1(a, ta.rowflag, lo + i, in);
+    emit(lo + i, i, in);
   }
-  if (bad) atomicOr(status, bad);
-  if (!ordered) flags[0] = 0;
+  if (use_fmin) {
+    __syncthreads();
+    int64_t *frow = ta.fmin + (size_t)blockIdx.x * R1;
+    for (int i = tid; i < R1; i += blockDim.x) frow[i] = s_fmin[i];
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
+size_t hfx_regroup_smem(int R1, int tile_rows) {
+  return sizeof(int64_t) * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) + 32;
+}
+
 int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
   const int R = s->p.n_replicas, R1 = R + 1;
   const int64_t n = ra.n;
@@ -418,46 +512,57 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
   int32_t tile_rows, n_tiles;
   hfx_tile_shape(n, &tile_rows, &n_tiles);
   const bool matrix = s->d_tile_hist != nullptr && n_tiles <= s->tile_blocks_max;
+  uint32_t *ordered = s->d_flags + s->step_parity;
+  CountArgs ca;
+  ca.replica_id = ra.replica_id; ca.class_id = ra.class_id; ca.state = ra.state; ca.prompt_len = ra.prompt_len;
+  ca.gen = ra.gen; ca.arrival = ra.arrival; ca.req_id = ra.req_id; ca.now = ra.now; ca.n = n; ca.tile_rows = tile_rows;
+  ca.M = matrix ? s->d_tile_hist : nullptr; ca.tile_mode = s->d_tile_mode; ca.tot_all = s->d_seg_count;
+  ca.tot_act = s->d_act_count; ca.rowflag = s->d_rowflag; ca.status = s->d_status; ca.ordered = ordered;
   if (matrix) {
     {
       KernelScope ks(s, KSLOT_COUNT);
-      k_count<<<n_tiles, THREADS_TILE, sizeof(uint32_t) * R1, stream>>>(ra.replica_id, n, R, tile_rows, s->d_tile_hist,
-                                                                          nullptr, s->d_status);
+      k_count<<<n_tiles, THREADS_TILE, sizeof(uint32_t) * 2 * R1, stream>>>(s->p, ca);
     }
     {
       KernelScope ks(s, KSLOT_COLSCAN);
-      k_colscan<<<(R1 + 31) / 32, 1024, 0, stream>>>(s->d_tile_hist, n_tiles, R1, s->d_seg_count);
+      k_colscan<<<(2 * R1 + 31) / 32, 1024, 0, stream>>>(s->d_tile_hist, n_tiles, R1, s->d_seg_count, s->d_act_count);
     }
     {
       KernelScope ks(s, KSLOT_OFFSETS);
-      k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags, 1u);
+      k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, s->d_act_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags,
+                                        s->step_parity, 0u);
     }
     {
       KernelScope ks(s, KSLOT_REGROUP);
-      const size_t sm = sizeof(uint32_t) * (3 * (size_t)R1 + 1) + sizeof(uint16_t) * (size_t)tile_rows + 16;
-      k_regroup<<<n_tiles, THREADS_TILE, sm, stream>>>(s->p, ra, tile_rows, s->d_tile_hist, s->d_seg_begin, s->d_rec,
-                                                        s->d_status, s->d_flags);
+      TileArgs ta;
+      ta.M = s->d_tile_hist; ta.tile_mode = s->d_tile_mode; ta.seg_begin = s->d_seg_begin; ta.tot_act = s->d_act_count;
+      ta.rowflag = s->d_rowflag; ta.ordered = ordered; ta.fmin = s->d_tile_fmin; ta.rec = s->d_rec; ta.tile_rows = tile_rows;
+      k_regroup<<<n_tiles, THREADS_TILE, hfx_regroup_smem(R1, tile_rows), stream>>>(s->p, ra, ta);
     }
   } else {
-    if (cudaMemsetAsync(s->d_seg_count, 0, sizeof(uint32_t) * (R + 2), stream) != cudaSuccess) return HFX_E_CUDA;
+    if (cudaMemsetAsync(s->d_seg_count, 0, sizeof(uint32_t) * (R + 2), stream) != cudaSuccess ||
+        cudaMemsetAsync(s->d_act_count, 0, sizeof(uint32_t) * (R + 2), stream) != cudaSuccess)
+      return HFX_E_CUDA;
     {
       KernelScope ks(s, KSLOT_COUNT);
-      k_count<<<n_tiles, THREADS_TILE, 0, stream>>>(ra.replica_id, n, R, tile_rows, nullptr, s->d_seg_count, s->d_status);
+      k_count<<<n_tiles, THREADS_TILE, 0, stream>>>(s->p, ca);
     }
     {
       KernelScope ks(s, KSLOT_OFFSETS);
-      k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags, 0u);
+      k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, s->d_act_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags,
+                                        s->step_parity, 1u);
     }
     {
       KernelScope ks(s, KSLOT_REGROUP);
-      k_regroup_atomic<<<s->n_sm * 8, 256, 0, stream>>>(s->p, ra, s->d_cursor, s->d_rec, s->d_status);
+      k_regroup_atomic<<<s->n_sm * 8, 256, 0, stream>>>(s->p, ra, s->d_rowflag, s->d_seg_begin, s->d_act_count, s->d_cursor,
+                                                        s->d_rec);
     }
   }
   return HFX_OK;
 }
 
 int hfx_regroup_configure() {
-  if (cudaFuncSetAttribute(k_regroup, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_regroup, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }

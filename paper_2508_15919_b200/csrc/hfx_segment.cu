@@ -249,42 +249,63 @@ __device__ __forceinline__ void commit_row(const SegArgs &a, const ReplicaPlan &
   }
 }
 
-// aggregates of one segment into the block's plan (all threads call; result in sh.plan)
-__device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &a, const HfxRec *seg, int64_t n, int r,
+// where a kernel finds the regrouped table
+struct SegCtx {
+  const HfxRec *rec; const uint32_t *seg_begin; const uint32_t *tot_act; const uint32_t *flags;
+  const int64_t *fmin; int32_t n_tiles; uint32_t parity;
+};
+
+// aggregates of a replica's active records into the block's plan (all threads call; result in
+// sh.plan; sh.next_arrival is left at "none")
+__device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &a, const HfxRec *seg, int64_t n_act, int r,
                                              bool real, BlockShared &sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  int64_t n_run = 0, sum_kv = 0, next_arr = HFX_INF;
+  int64_t n_run = 0, sum_kv = 0;
   uint64_t m_run = 0, m_q = 0;
-  int32_t n_act = 0;
-  for (int64_t q = threadIdx.x; q < n; q += blockDim.x) {
+  for (int64_t q = threadIdx.x; q < n_act; q += blockDim.x) {
     const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);   // prompt, gen, output_len, bytes
     const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
-    if (kind == KIND_RUNNING) { n_run++; n_act++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
-    else if (kind == KIND_QUEUED) { n_act++; m_q |= 1ull << cls; }
-    else if (kind == KIND_FUTURE) { const int64_t arr = seg[q].base; next_arr = arr < next_arr ? arr : next_arr; }
+    if (kind == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
+    else m_q |= 1ull << cls;
   }
-  n_run = warp_sum_i64(n_run); sum_kv = warp_sum_i64(sum_kv); next_arr = warp_min_i64(next_arr);
-  m_run = warp_or_u64(m_run); m_q = warp_or_u64(m_q); n_act = (int32_t)warp_sum_i64(n_act);
-  if (lane == 0) {
-    sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_c[warp] = next_arr; sh.red_m0[warp] = m_run;
-    sh.red_m1[warp] = m_q; sh.red_n[warp] = n_act;
-  }
+  n_run = warp_sum_i64(n_run); sum_kv = warp_sum_i64(sum_kv);
+  m_run = warp_or_u64(m_run); m_q = warp_or_u64(m_q);
+  if (lane == 0) { sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_m0[warp] = m_run; sh.red_m1[warp] = m_q; }
   __syncthreads();
   if (threadIdx.x == 0) {
-    for (int k = 1; k < nwarp; k++) {
-      n_run += sh.red_a[k]; sum_kv += sh.red_b[k]; n_act += sh.red_n[k];
-      next_arr = sh.red_c[k] < next_arr ? sh.red_c[k] : next_arr;
-      m_run |= sh.red_m0[k]; m_q |= sh.red_m1[k];
-    }
+    for (int k = 1; k < nwarp; k++) { n_run += sh.red_a[k]; sum_kv += sh.red_b[k]; m_run |= sh.red_m0[k]; m_q |= sh.red_m1[k]; }
     hfx_replica_cfg cfg; cfg.mode = HFX_COLOCATED; cfg.token_cap = 1; cfg.batch_cap = 0;
     int64_t now = 0, mat = 0;
     if (real) { cfg = a.cfg[r]; now = a.now[r]; mat = a.mat[r]; }
     dev_plan(p, cfg, now, mat, n_run, sum_kv, m_run, m_q, sh.plan);
-    sh.next_arrival = next_arr; sh.n_act = n_act;
-    sh.carry_cost = 0; sh.carry_count = 0; sh.carry_act = 0; sh.carry_inact = 0;
+    sh.next_arrival = HFX_INF;
+    sh.carry_cost = 0; sh.carry_count = 0;
     sh.adm_cost = 0; sh.adm_kv = 0; sh.adm_count = 0;
   }
   __syncthreads();
+}
+
+// block-wide minimum into sh.next_arrival (all threads call)
+__device__ __forceinline__ void block_min_arrival(int64_t v, BlockShared &sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  v = warp_min_i64(v);
+  __syncthreads();
+  if (lane == 0) sh.red_c[warp] = v;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int64_t m = sh.next_arrival;
+    for (int k = 0; k < nwarp; k++) m = sh.red_c[k] < m ? sh.red_c[k] : m;
+    sh.next_arrival = m;
+  }
+  __syncthreads();
+}
+
+// the outputs of an inactive row (when the regroup has not written them already)
+__device__ __forceinline__ void write_inactive_row(const SegArgs &a, int32_t row, int r) {
+  a.slack[row] = 0;
+  a.admit[row] = 0;
+  if (a.pred_tpot) a.pred_tpot[row] = 0;
+  if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
 }
 
 // Block-wide admission over the sorted items s_lo[0..n_sorted) (low 16 bits = position of the
@@ -346,10 +367,8 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
   }
 }
 
-__global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegArgs a, const HfxRec *__restrict__ rec,
-                                                  const uint32_t *__restrict__ seg_begin,
-                                                  const uint32_t *__restrict__ flags, int seg_min, int seg_cap,
-                                                  int bucket) {
+__global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegArgs a, const SegCtx c, int seg_min,
+                                                  int seg_cap, int bucket) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint64_t *s_hi = reinterpret_cast<uint64_t *>(smem_raw);
   uint32_t *s_lo = reinterpret_cast<uint32_t *>(smem_raw + (size_t)seg_cap * 8);
@@ -358,111 +377,106 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
   uint32_t *s_bin = reinterpret_cast<uint32_t *>(smem_raw + (size_t)seg_cap * 20);
   uint32_t *s_cur = s_bin + SORT_BINS + 4;
   __shared__ BlockShared sh;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const int R = p.n_replicas;
-  if (flags[1] < (uint32_t)seg_min) return;     // no segment of this kernel's size class exists
-  const bool ordered = flags[0] != 0;
+  if (c.flags[2] < (uint32_t)seg_min) return;     // no replica of this kernel's size class exists
+  const bool ordered = c.flags[c.parity] != 0;
 
   for (int r = blockIdx.x; r <= R; r += gridDim.x) {
-    const uint32_t b = seg_begin[r];
-    const int n = (int)(seg_begin[r + 1] - b);
-    if (n < seg_min || n > seg_cap) continue;
+    const uint32_t b = c.seg_begin[r];
+    const int n = (int)(c.seg_begin[r + 1] - b);
+    const int n_act = (int)c.tot_act[r];
+    const int n_in = n - n_act;
+    const int need = ordered ? n_act : (n_act > n_in ? n_act : n_in);
+    if (need < seg_min || need > seg_cap) continue;
     if (r == R && n == 0) continue;
-    const HfxRec *seg = rec + b;
+    const HfxRec *seg = c.rec + b;
     const bool real = r < R;    // bucket R holds rows bound to no replica
 
-    segment_plan(p, a, seg, n, r, real, sh);
-    const ReplicaPlan pl = sh.plan;
-    int n_sorted;
-
-    if (ordered) {
-      // ---- records are in req_id order: only rows in flight or in the queue are sorted, by
-      //      (key48, position); inactive rows keep their order behind them ---------------------
-      n_sorted = sh.n_act;
-      const int n_active = n_sorted;
-      for (int tile = 0; tile < n; tile += blockDim.x) {
-        const int q = tile + threadIdx.x;
-        int act = 0, inact = 0;
-        int32_t row = -1;
-        uint64_t k48 = 0;
-        if (q < n) {
-          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
-          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
-          const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
-          row = (int32_t)w0.w;
-          const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
-          const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
-          k48 = e.k48;
-          act = e.phase != PH_INACTIVE; inact = !act;
-          a.slack[row] = e.slack;
-          if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-          if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
-          if (inact) a.admit[row] = 0;
-        }
-        const uint32_t bal = __ballot_sync(0xffffffffu, act);
-        const uint32_t bal_in = __ballot_sync(0xffffffffu, inact);
-        const uint32_t lt = (1u << lane) - 1u;
-        if (lane == 0) { sh.red_a[warp] = __popc(bal); sh.red_b[warp] = __popc(bal_in); }
-        __syncthreads();
-        int pre_a = sh.carry_act, pre_i = sh.carry_inact, tot_a = 0, tot_i = 0;
-        for (int k = 0; k < nwarp; k++) {
-          const int ca = (int)sh.red_a[k], ci = (int)sh.red_b[k];
-          if (k < warp) { pre_a += ca; pre_i += ci; }
-          tot_a += ca; tot_i += ci;
-        }
-        if (act) s_hi[pre_a + __popc(bal & lt)] = (k48 << 16) | (uint32_t)q;
-        if (inact) a.order[b + n_active + pre_i + __popc(bal_in & lt)] = row;
-        __syncthreads();
-        if (threadIdx.x == 0) { sh.carry_act += tot_a; sh.carry_inact += tot_i; }
+    // ---- inactive rows of a step that is not ordered: listed by req_id behind the active ones ----
+    if (!ordered && n_in > 0) {
+      const HfxRec *sin = seg + n_act;
+      int64_t next_arr = HFX_INF;
+      for (int q = threadIdx.x; q < n_in; q += blockDim.x) {
+        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
+        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
+        if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); next_arr = arr < next_arr ? arr : next_arr; }
+        s_hi[q] = ((uint64_t)(w0.z ^ 0x80000000u) << 16) | (uint32_t)q;     // signed req_id order, then position
+        write_inactive_row(a, (int32_t)w0.w, r);
       }
       __syncthreads();
-      if (!(bucket && n_sorted > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_sorted, sh))) {
-        block_sort<false>(s_hi, nullptr, n_sorted);
-        for (int q = threadIdx.x; q < n_sorted; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+      if (!(bucket && n_in > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_in, sh))) {
+        block_sort<false>(s_hi, nullptr, n_in);
+        for (int q = threadIdx.x; q < n_in; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+        __syncthreads();
       }
+      for (int q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = sin[s_lo[q]].row;
+      __syncthreads();
+      segment_plan(p, a, seg, n_act, r, real, sh);
+      block_min_arrival(next_arr, sh);
     } else {
-      // ---- general case: every row takes part, the tie-break req_id travels with the item -----
-      n_sorted = n;
-      for (int q = threadIdx.x; q < n; q += blockDim.x) {
-        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
-        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
-        const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
-        const int32_t req_id = (int32_t)w0.z, row = (int32_t)w0.w;
-        const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
-        const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
-        const uint32_t uid = (uint32_t)req_id ^ 0x80000000u;      // signed order as unsigned
+      segment_plan(p, a, seg, n_act, r, real, sh);
+    }
+    const ReplicaPlan pl = sh.plan;
+
+    // ---- sort items of the active rows ---------------------------------------------------------------
+    for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
+      const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
+      const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
+      const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
+      const int32_t row = (int32_t)w0.w;
+      const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
+      const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+      if (ordered) s_hi[q] = (e.k48 << 16) | (uint32_t)q;     // records are in req_id order: position breaks ties
+      else {
+        const uint32_t uid = w0.z ^ 0x80000000u;               // signed req_id order as unsigned
         s_hi[q] = (e.k48 << 16) | (uid >> 16);
         s_lo[q] = (uid << 16) | (uint32_t)q;
-        a.slack[row] = e.slack;
-        if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
       }
-      __syncthreads();
-      block_sort<true>(s_hi, s_lo, n);
-      for (int q = threadIdx.x; q < n; q += blockDim.x) s_lo[q] &= 0xffffu;
+      a.slack[row] = e.slack;
+      if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
+      if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+    }
+    __syncthreads();
+    if (ordered) {
+      if (!(bucket && n_act > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_act, sh))) {
+        block_sort<false>(s_hi, nullptr, n_act);
+        for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+      }
+    } else {
+      block_sort<true>(s_hi, s_lo, n_act);
+      for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] &= 0xffffu;
     }
     __syncthreads();
 
-    segment_admit(p, a, pl, seg, b, s_lo, n_sorted, sh);
+    segment_admit(p, a, pl, seg, b, s_lo, n_act, sh);
 
-    // ---- maturity, per-replica outputs, commit decisions --------------------------------
+    // ---- maturity, iteration clock ------------------------------------------------------------------
     if (threadIdx.x == 0) {
       int64_t lp = 0;
       const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
       int worked; int64_t t1, t2;
       iteration_clock(pl, sh.adm_count, lp, mat_next, worked, t1, t2);
-      sh.worked = worked; sh.t1 = t1; sh.t2 = t2;
-      if (real) write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, t2, sh.next_arrival);
+      sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
     }
     __syncthreads();
+    const bool commit = real && (a.flags & HFX_COMMIT);
+    const int worked = sh.worked;
+    const int64_t mat_next = sh.red_c[0];
+    if (commit && !worked && ordered) {
+      // idle replica of an ordered step: its next arrival comes from the regroup's per-tile minima
+      int64_t v = HFX_INF;
+      for (int t = threadIdx.x; t < c.n_tiles; t += blockDim.x) { const int64_t x = c.fmin[(size_t)t * (R + 1) + r]; v = x < v ? x : v; }
+      block_min_arrival(v, sh);
+    }
+    if (threadIdx.x == 0 && real)
+      write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
 
-    // ---- second pass: padding of the compacted list, commit ------------------------------
+    // ---- padding of the compacted list, commit ----------------------------------------------------
     if (a.admitted_rows)
       for (int q = sh.adm_count + threadIdx.x; q < n; q += blockDim.x) a.admitted_rows[b + q] = -1;
-    if (real && (a.flags & HFX_COMMIT)) {
-      const int worked = sh.worked;
+    if (commit) {
       const int64_t t1 = sh.t1, t2 = sh.t2;
-      for (int q = threadIdx.x; q < n_sorted; q += blockDim.x) {
+      for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
         const uint32_t lo = s_lo[q];
         const int li = lo & 0xffff;
         const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
@@ -476,7 +490,7 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
 }
 
 // ------------------------------------------------------------------------------------------------
-// Oversize segments (more rows than a block can sort in shared memory): one cooperative kernel.
+// Oversize replicas (more items than a block can sort in shared memory): one cooperative kernel.
 // All blocks walk the replicas in the same order and share the work of each oversize one: keys
 // spread over the grid, a global bitonic network with bounded grid barriers, admission by block 0
 // walking the order with a carried prefix, commit by the grid.  Slow but exact; it only exists so
@@ -516,12 +530,40 @@ __device__ __forceinline__ void global_cmp_swap(uint64_t *hi, uint32_t *lo, uint
   }
 }
 
-__global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a, const HfxRec *__restrict__ rec,
-                                             const uint32_t *__restrict__ seg_begin, const uint32_t *__restrict__ flags,
+// Global bitonic network over n items (hi, lo) with idx travelling along: ascending comparators,
+// virtual padding.  The items must be visible grid-wide on entry (a grid barrier precedes it).
+__device__ bool grid_sort(uint64_t *hi, uint32_t *lo, uint32_t *idx, int64_t n, uint32_t *bar, uint32_t *status,
+                          uint32_t &epoch) {
+  const int64_t gtid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t gsize = (int64_t)gridDim.x * blockDim.x;
+  int64_t n_pad = 1;
+  while (n_pad < n) n_pad <<= 1;
+  const int64_t half = n_pad >> 1;
+  for (int64_t k = 2; k <= n_pad; k <<= 1) {
+    const int64_t hk = k >> 1;
+    for (int64_t t = gtid; t < half; t += gsize) {
+      const int64_t blk = t / hk, off = t - blk * hk;
+      const int64_t i = blk * k + off, j = blk * k + k - 1 - off;
+      if (j < n) global_cmp_swap(hi, lo, idx, i, j);
+    }
+    if (!grid_barrier(bar, status, epoch)) return false;
+    for (int64_t j = k >> 2; j > 0; j >>= 1) {
+      for (int64_t t = gtid; t < half; t += gsize) {
+        const int64_t i = 2 * t - (t & (j - 1));
+        if (i + j < n) global_cmp_swap(hi, lo, idx, i, i + j);
+      }
+      if (!grid_barrier(bar, status, epoch)) return false;
+    }
+  }
+  return true;
+}
+
+__global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a, const SegCtx c,
                                              uint64_t *__restrict__ g_hi, uint32_t *__restrict__ g_lo,
                                              uint32_t *__restrict__ g_idx, uint32_t *bar, uint32_t *status) {
   __shared__ BlockShared sh;
-  if (flags[1] <= SEG_MED) return;
+  if (c.flags[2] <= SEG_MED) return;
+  const bool ordered = c.flags[c.parity] != 0;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const int R = p.n_replicas;
   uint32_t epoch = 0;
@@ -530,63 +572,60 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
   volatile int64_t *mail = reinterpret_cast<volatile int64_t *>(bar + 4);
 
   for (int r = 0; r <= R; r++) {
-    const uint32_t b = seg_begin[r];
-    const int64_t n = (int64_t)(seg_begin[r + 1] - b);
-    if (n <= SEG_MED) continue;
-    const HfxRec *seg = rec + b;
+    const uint32_t b = c.seg_begin[r];
+    const int64_t n = (int64_t)(c.seg_begin[r + 1] - b);
+    const int64_t n_act = c.tot_act[r], n_in = n - n_act;
+    const int64_t need = ordered ? n_act : (n_act > n_in ? n_act : n_in);
+    if (need <= SEG_MED) continue;
+    const HfxRec *seg = c.rec + b;
     const bool real = r < R;
+
+    // ---- inactive rows of a step that is not ordered: by req_id behind the active ones -----------
+    if (!ordered && n_in > 0) {
+      const HfxRec *sin = seg + n_act;
+      uint64_t *hi = g_hi + b + n_act;
+      uint32_t *lo = g_lo + b + n_act, *idx = g_idx + b + n_act;
+      for (int64_t q = gtid; q < n_in; q += gsize) {
+        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
+        hi[q] = w0.z ^ 0x80000000u; lo[q] = 0; idx[q] = (uint32_t)q;
+        write_inactive_row(a, (int32_t)w0.w, r);
+      }
+      if (!grid_barrier(bar, status, epoch)) return;
+      if (!grid_sort(hi, lo, idx, n_in, bar, status, epoch)) return;
+      for (int64_t q = gtid; q < n_in; q += gsize) a.order[b + n_act + q] = sin[idx[q]].row;
+    }
+
+    // every block computes the aggregates redundantly (reads come from L2 after the first)
+    segment_plan(p, a, seg, n_act, r, real, sh);
+    const ReplicaPlan pl = sh.plan;
     uint64_t *hi = g_hi + b;
     uint32_t *lo = g_lo + b, *idx = g_idx + b;
 
-    // every block computes the aggregates redundantly (reads come from L2 after the first)
-    segment_plan(p, a, seg, n, r, real, sh);
-    const ReplicaPlan pl = sh.plan;
-
-    // keys, spread over the grid
-    for (int64_t q = gtid; q < n; q += gsize) {
+    // keys of the active rows, spread over the grid
+    for (int64_t q = gtid; q < n_act; q += gsize) {
       const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
       const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
       const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
-      const int32_t req_id = (int32_t)w0.z, row = (int32_t)w0.w;
+      const int32_t row = (int32_t)w0.w;
       const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
       const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
       hi[q] = e.k48;
-      lo[q] = (uint32_t)req_id ^ 0x80000000u;
+      lo[q] = w0.z ^ 0x80000000u;
       idx[q] = (uint32_t)q;
       a.slack[row] = e.slack;
       if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
       if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
     }
     if (!grid_barrier(bar, status, epoch)) return;
-
-    // global bitonic network (ascending comparators, virtual padding), idx travels with the item
-    int64_t n_pad = 1;
-    while (n_pad < n) n_pad <<= 1;
-    const int64_t half = n_pad >> 1;
-    for (int64_t k = 2; k <= n_pad; k <<= 1) {
-      const int64_t hk = k >> 1;
-      for (int64_t t = gtid; t < half; t += gsize) {
-        const int64_t blk = t / hk, off = t - blk * hk;
-        const int64_t i = blk * k + off, j = blk * k + k - 1 - off;
-        if (j < n) global_cmp_swap(hi, lo, idx, i, j);
-      }
-      if (!grid_barrier(bar, status, epoch)) return;
-      for (int64_t j = k >> 2; j > 0; j >>= 1) {
-        for (int64_t t = gtid; t < half; t += gsize) {
-          const int64_t i = 2 * t - (t & (j - 1));
-          if (i + j < n) global_cmp_swap(hi, lo, idx, i, i + j);
-        }
-        if (!grid_barrier(bar, status, epoch)) return;
-      }
-    }
+    if (!grid_sort(hi, lo, idx, n_act, bar, status, epoch)) return;
 
     // admission walk by block 0 with a carried prefix, then commit by the whole grid
     if (blockIdx.x == 0) {
-      for (int64_t tile = 0; tile < n; tile += blockDim.x) {
+      for (int64_t tile = 0; tile < n_act; tile += blockDim.x) {
         const int64_t q = tile + threadIdx.x;
         int64_t cost = 0, kv = 0;
         int32_t cnt = 0, row = -1, kind = KIND_DEAD;
-        if (q < n) {
+        if (q < n_act) {
           const uint32_t li = idx[q];
           const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
           const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
@@ -594,8 +633,8 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
           kind = (w1.w >> 8) & 0xff;
           if (kind == KIND_QUEUED) {
             kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
-            const int64_t c = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-            if (c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
+            const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
+            if (cc <= pl.budget) { cost = cc; cnt = 1; } else kv = 0;
           }
           a.order[b + q] = row;
         }
@@ -614,7 +653,7 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
         sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
         bool adm = false;
         if (cnt) adm = sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap);
-        if (q < n) {
+        if (q < n_act) {
           a.admit[row] = (uint8_t)((kind == KIND_RUNNING || adm) ? 1 : 0);
           if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
           lo[q] = adm ? 1u : 0u;      // the sort is over: lo now carries the decision
@@ -630,6 +669,19 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
           for (int k = 0; k < nwarp; k++) { sh.adm_cost += sh.red_a[k]; sh.adm_kv += sh.red_b[k]; sh.adm_count += (int32_t)sh.red_c[k]; }
         __syncthreads();
       }
+      // the replica's next arrival, should it turn out idle
+      int64_t v = HFX_INF;
+      if (ordered) {
+        for (int t = threadIdx.x; t < c.n_tiles; t += blockDim.x) { const int64_t x = c.fmin[(size_t)t * (R + 1) + r]; v = x < v ? x : v; }
+      } else {
+        const HfxRec *sin = seg + n_act;
+        for (int64_t q = threadIdx.x; q < n_in; q += blockDim.x) {
+          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
+          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
+          if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); v = arr < v ? arr : v; }
+        }
+      }
+      block_min_arrival(v, sh);
       if (threadIdx.x == 0) {
         int64_t lp = 0;
         const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
@@ -644,15 +696,16 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
       const int64_t t1 = mail[0], t2 = mail[1];
       const int worked = (int)mail[2], adm_count = (int)mail[3];
       const bool commit = real && (a.flags & HFX_COMMIT);
-      for (int64_t q = gtid; q < n; q += gsize) {
-        if (a.admitted_rows && q >= adm_count) a.admitted_rows[b + q] = -1;
-        if (!commit) continue;
-        const uint32_t li = idx[q];
-        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
-        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
-        commit_row(a, pl, (w1.w >> 8) & 0xff, lo[q] != 0, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x, (int32_t)w1.y,
-                   (int32_t)w1.z);
-      }
+      if (a.admitted_rows)
+        for (int64_t q = adm_count + gtid; q < n; q += gsize) a.admitted_rows[b + q] = -1;
+      if (commit)
+        for (int64_t q = gtid; q < n_act; q += gsize) {
+          const uint32_t li = idx[q];
+          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
+          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
+          commit_row(a, pl, (w1.w >> 8) & 0xff, lo[q] != 0, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x, (int32_t)w1.y,
+                     (int32_t)w1.z);
+        }
     }
     if (!grid_barrier(bar, status, epoch)) return;
   }
@@ -664,23 +717,26 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
 int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
   const int R1 = s->p.n_replicas + 1;
   cudaStream_t stream = s->stream;
+  SegCtx c;
+  c.rec = s->d_rec; c.seg_begin = s->d_seg_begin; c.tot_act = s->d_act_count; c.flags = s->d_flags;
+  c.fmin = s->d_tile_fmin; c.parity = s->step_parity;
+  int32_t tile_rows;
+  hfx_tile_shape(n, &tile_rows, &c.n_tiles);
   {
     KernelScope ks(s, KSLOT_SEG_SMALL);
     const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
-    k_segment<<<grid, THREADS_SMALL, SMEM_SMALL, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_flags, 0, SEG_SMALL, 1);
+    k_segment<<<grid, THREADS_SMALL, SMEM_SMALL, stream>>>(s->p, sa, c, 0, SEG_SMALL, 1);
   }
   if (n > SEG_SMALL) {
     KernelScope ks(s, KSLOT_SEG_MED);
     const int grid = R1 < s->n_sm ? R1 : s->n_sm;
-    k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, s->d_rec, s->d_seg_begin, s->d_flags, SEG_SMALL + 1,
-                                                            SEG_MED, 0);
+    k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, c, SEG_SMALL + 1, SEG_MED, 0);
   }
   if (n > SEG_MED) {
     uint32_t *big_idx = reinterpret_cast<uint32_t *>(s->d_big_lo + s->max_rows);
     if (cudaMemsetAsync(s->d_barrier, 0, 64, stream) != cudaSuccess) return HFX_E_CUDA;
-    void *args[] = {(void *)&s->p, (void *)&sa, (void *)&s->d_rec, (void *)&s->d_seg_begin, (void *)&s->d_flags,
-                    (void *)&s->d_big_hi, (void *)&s->d_big_lo, (void *)&big_idx, (void *)&s->d_barrier,
-                    (void *)&s->d_status};
+    void *args[] = {(void *)&s->p, (void *)&sa, (void *)&c, (void *)&s->d_big_hi, (void *)&s->d_big_lo, (void *)&big_idx,
+                    (void *)&s->d_barrier, (void *)&s->d_status};
     KernelScope ks(s, KSLOT_BIG);
     if (cudaLaunchCooperativeKernel((void *)k_big, dim3(s->n_sm), dim3(512), args, 0, stream) != cudaSuccess)
       return HFX_E_CUDA;

@@ -33,6 +33,8 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
   ra.output_len = t->output_len; ra.gen = t->gen; ra.arrival = t->arrival_ns; ra.first_token = t->first_token_ns;
   ra.req_id = t->req_id; ra.weight = s->p.weight_max > 0 ? t->weight : nullptr;
   ra.now = st->now_ns; ra.mat = st->maturity_ns; ra.cfg = s->d_cfg; ra.pred_ttft = o->pred_ttft_ns; ra.n = t->n_rows;
+  ra.slack = o->slack_ns; ra.pred_tpot = o->pred_tpot_ns; ra.key = o->key; ra.order = o->order; ra.admit = o->admit;
+  ra.admitted_rows = o->admitted_rows; ra.commit = flags & HFX_COMMIT;
   int rc = hfx_launch_regroup(s, ra, o->seg_off);
   if (rc != HFX_OK) return rc;
 
@@ -44,6 +46,7 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
   sa.sum_kv = o->sum_kv; sa.adm_cost = o->adm_cost; sa.adm_count = o->adm_count; sa.maturity_next = o->maturity_next;
   sa.flags = flags;
   rc = hfx_launch_segments(s, sa, t->n_rows);
+  s->step_parity ^= 1u;
   if (rc != HFX_OK) return rc;
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }
