@@ -130,9 +130,9 @@ __device__ inline int64_t dev_epmax(int64_t min_ttft, bool decoding, int64_t min
   if (min_ttft == HFX_INF) return HFX_INF;
   if (!decoding) return min_ttft / 2;
   if (min_tpot <= e_d) return -1;
-  unsigned __int128 num = (unsigned __int128)(uint64_t)min_ttft * (uint64_t)(min_tpot - e_d);
-  uint64_t den = (uint64_t)(2 * min_tpot - e_d);
-  return (int64_t)(num / den);
+  const uint64_t x = (uint64_t)min_ttft, y = (uint64_t)(min_tpot - e_d), den = (uint64_t)(2 * min_tpot - e_d);
+  if (__umul64hi(x, y) == 0) return (int64_t)((x * y) / den);     // the product fits 64 bits (the usual case)
+  return (int64_t)(((unsigned __int128)x * y) / den);
 }
 
 // Largest n in [0, cap] with E_p(n) <= epmax (Eq. 3 on the general prefill model), 0 if none.
@@ -193,6 +193,71 @@ __device__ inline void dev_plan(const HfxParams &p, const hfx_replica_cfg &cfg, 
   pl.shift_dq = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
 }
 
+// The same plan computed by a whole warp (all 32 lanes call with the same arguments and get the same
+// result): class minima by lanes, and the largest safe n by a 32-way search instead of a bisection.
+__device__ inline int64_t warp_min_over_mask(const int64_t *v, uint64_t mask, int lane) {
+  int64_t m = HFX_INF;
+#pragma unroll
+  for (int c = lane; c < HFX_MAX_CLASSES; c += 32)
+    if ((mask >> c) & 1ull) { const int64_t x = v[c]; if (x > 0 && x < m) m = x; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { const int64_t w = __shfl_xor_sync(0xffffffffu, m, o); m = w < m ? w : m; }
+  return m;
+}
+
+__device__ inline int64_t warp_nsafe(const HfxParams &p, int64_t epmax, int64_t cap, int lane) {
+  if (epmax == HFX_INF) return cap;
+  if (dev_Ep(p, 0) > epmax) return 0;
+  int64_t lo = 0, hi = cap;          // E_p(lo) <= epmax; the answer lies in [lo, hi]
+  while (lo < hi) {
+    const int64_t step = (hi - lo + 31) / 32;
+    int64_t cand = lo + (int64_t)(lane + 1) * step;
+    const bool in = cand <= hi;
+    const bool ok = in && dev_Ep(p, cand) <= epmax;
+    const int m = __popc(__ballot_sync(0xffffffffu, ok));       // E_p is monotone: the ok lanes are a prefix
+    const int64_t nlo = lo + (int64_t)m * step;
+    int64_t nhi = lo + (int64_t)(m + 1) * step - 1;
+    if (nhi > hi) nhi = hi;
+    lo = nlo; hi = nhi;
+  }
+  return lo;
+}
+
+__device__ inline void warp_plan(const HfxParams &p, const hfx_replica_cfg &cfg, int64_t now, int64_t mat,
+                                 int64_t n_run, int64_t sum_kv, uint64_t mask_run, uint64_t mask_q, ReplicaPlan &pl,
+                                 int lane) {
+  pl.now = now; pl.mat = mat; pl.start = now > mat ? now : mat;
+  pl.mode = cfg.mode; pl.token_cap = cfg.token_cap; pl.batch_cap = cfg.batch_cap;
+  pl.n_run = n_run; pl.sum_kv = sum_kv;
+  const int64_t min_tpot = warp_min_over_mask(p.tpot, mask_run, lane);
+  const int64_t min_ttft = warp_min_over_mask(p.ttft, mask_q, lane);
+  const int64_t min_tpot_q = warp_min_over_mask(p.tpot, mask_q, lane);
+  const bool prefill = cfg.mode == HFX_PREFILL;
+  pl.n_eff = prefill ? 0 : n_run;
+  pl.kv_eff = prefill ? 0 : sum_kv;
+  pl.tpot_eff = prefill ? HFX_INF : min_tpot;
+  pl.e_d = pl.n_eff > 0 ? dev_Ed(p, pl.n_eff, pl.kv_eff) : 0;
+  int64_t budget;
+  if (cfg.mode == HFX_DECODE) {
+    const int64_t T = (n_run > 0 && min_tpot < HFX_INF) ? min_tpot : min_tpot_q;
+    if (p.budget_mode == HFX_BUDGET_CAP_ONLY || T == HFX_INF) budget = HFX_INF;
+    else {
+      const int64_t room = T - dev_Ed(p, n_run, sum_kv);
+      budget = room > 0 ? room : 0;
+    }
+  } else {
+    const int64_t cap_left = cfg.token_cap - pl.n_eff > 0 ? cfg.token_cap - pl.n_eff : 0;
+    int64_t n_safe;
+    if (p.budget_mode == HFX_BUDGET_CAP_ONLY) n_safe = cfg.token_cap;
+    else n_safe = warp_nsafe(p, dev_epmax(min_ttft, pl.n_eff > 0 && pl.tpot_eff < HFX_INF, pl.tpot_eff, pl.e_d), cfg.token_cap, lane);
+    budget = n_safe < cap_left ? n_safe : cap_left;
+  }
+  if (now < mat) budget = 0;
+  pl.budget = budget;
+  pl.shift_run = pl.e_d;
+  pl.shift_dq = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
+}
+
 // Dispatching step 4: maturity time after admitting adm_count requests of adm_cost in total.
 __device__ inline int64_t dev_maturity_next(const HfxParams &p, const ReplicaPlan &pl, int64_t adm_count,
                                             int64_t adm_cost, int64_t adm_kv, int64_t *lp_out) {
@@ -204,13 +269,16 @@ __device__ inline int64_t dev_maturity_next(const HfxParams &p, const ReplicaPla
     lp = dev_Ep(p, adm_cost);
     if (pl.mode == HFX_PREFILL) mat_next = pl.now + lp;
     else {
-      unsigned __int128 k = 0;
+      uint64_t k = 0;
       if (pl.n_eff > 0 && pl.tpot_eff < HFX_INF && pl.tpot_eff > pl.e_d) {
         const uint64_t d = (uint64_t)(pl.tpot_eff - pl.e_d);
         k = ((uint64_t)lp + d - 1) / d;
       }
-      __int128 v = (__int128)pl.now + lp + (__int128)(k * (uint64_t)pl.e_d);
-      mat_next = v > (__int128)HFX_TIME_MAX ? HFX_TIME_MAX : (int64_t)v;
+      // now + lp + k * e_d, saturating at HFX_TIME_MAX (the product may need more than 64 bits)
+      const uint64_t ed = (uint64_t)pl.e_d, prod = k * ed;
+      const int64_t t = pl.now + lp;                              // |now| <= 2^56, lp < 2^61
+      if (__umul64hi(k, ed) != 0 || prod >= (UINT64_C(1) << 63)) mat_next = HFX_TIME_MAX;
+      else mat_next = (int64_t)prod > HFX_TIME_MAX - t ? HFX_TIME_MAX : t + (int64_t)prod;
     }
   }
   *lp_out = lp;

@@ -7,6 +7,7 @@
 #define SEG_SMALL 2048    // rows a small-segment block sorts in shared memory
 #define SEG_MED 16384     // rows a medium-segment block sorts in shared memory
 #define THREADS_SMALL 256
+#define TINY_BLOCKS_PER_SM 4
 #define THREADS_MED 1024
 #define SMEM_SMALL (SEG_SMALL * 20 + (2 * 1024 + 8) * 4)   // sort items, their order, scatter buffer, bins
 
@@ -490,6 +491,277 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
 }
 
 // ------------------------------------------------------------------------------------------------
+// k_segment_small: replicas with at most SEG_TINY items to sort.  What later passes need of the
+// replica's active records (lengths, kind, row) is staged once into shared memory; sort items live
+// in registers until they are scattered into their bins.
+// ------------------------------------------------------------------------------------------------
+#define SEG_TINY 768
+#define TINY_IPT ((SEG_TINY + THREADS_SMALL - 1) / THREADS_SMALL)     // items per thread
+#define TINY_BINS 512
+#define TINY_BIN_MAX 48
+#define SMEM_TINY (SEG_TINY * (16 + 4 + 8 + 4) + (2 * TINY_BINS + 8) * 4)
+
+__global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_small(const HfxParams p, const SegArgs a, const SegCtx c) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint4 *s_w1 = reinterpret_cast<uint4 *>(smem_raw);                                   // [SEG_TINY] prompt, gen, output_len, bytes
+  uint64_t *s_key = reinterpret_cast<uint64_t *>(smem_raw + (size_t)SEG_TINY * 16);    // [SEG_TINY] sort items, binned
+  int32_t *s_row = reinterpret_cast<int32_t *>(s_key + SEG_TINY);                      // [SEG_TINY]
+  uint32_t *s_lo = reinterpret_cast<uint32_t *>(s_row + SEG_TINY);                     // [SEG_TINY] order (+ tie-break words)
+  uint32_t *s_bin = s_lo + SEG_TINY;                                                   // [TINY_BINS + 4]
+  uint32_t *s_cur = s_bin + TINY_BINS + 4;                                             // [TINY_BINS]
+  __shared__ BlockShared sh;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const int R = p.n_replicas;
+  const bool ordered = c.flags[c.parity] != 0;
+
+  for (int r = blockIdx.x; r <= R; r += gridDim.x) {
+    const uint32_t b = c.seg_begin[r];
+    const int n = (int)(c.seg_begin[r + 1] - b);
+    const int n_act = (int)c.tot_act[r];
+    const int n_in = n - n_act;
+    const int need = ordered ? n_act : (n_act > n_in ? n_act : n_in);
+    if (need > SEG_TINY) continue;
+    if (r == R && n == 0) continue;
+    const HfxRec *seg = c.rec + b;
+    const bool real = r < R;    // bucket R holds rows bound to no replica
+
+    int64_t next_arr = HFX_INF;
+    if (!ordered && n_in > 0) {
+      // inactive rows of a step that is not ordered: listed by req_id behind the active ones
+      const HfxRec *sin = seg + n_act;
+      for (int q = threadIdx.x; q < n_in; q += blockDim.x) {
+        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
+        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
+        if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); next_arr = arr < next_arr ? arr : next_arr; }
+        s_key[q] = ((uint64_t)(w0.z ^ 0x80000000u) << 16) | (uint32_t)q;
+        write_inactive_row(a, (int32_t)w0.w, r);
+      }
+      __syncthreads();
+      block_sort<false>(s_key, nullptr, n_in);
+      for (int q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = sin[s_key[q] & 0xffffu].row;
+      __syncthreads();
+    }
+
+    // ---- stage what later passes need of the active records; aggregates --------------------------
+    uint4 w0r[TINY_IPT];
+    {
+      int64_t n_run = 0, sum_kv = 0;
+      uint64_t m_run = 0, m_q = 0;
+#pragma unroll
+      for (int k = 0; k < TINY_IPT; k++) {
+        const int q = threadIdx.x + k * THREADS_SMALL;
+        if (q < n_act) {
+          w0r[k] = __ldg(reinterpret_cast<const uint4 *>(seg + q));
+          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
+          s_w1[q] = w1;
+          s_row[q] = (int32_t)w0r[k].w;
+          const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
+          if (kind == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
+          else m_q |= 1ull << cls;
+        }
+      }
+      n_run = warp_sum_i64(n_run); sum_kv = warp_sum_i64(sum_kv); next_arr = warp_min_i64(next_arr);
+      m_run = warp_or_u64(m_run); m_q = warp_or_u64(m_q);
+      if (lane == 0) { sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_c[warp] = next_arr; sh.red_m0[warp] = m_run; sh.red_m1[warp] = m_q; }
+      for (int i = threadIdx.x; i <= TINY_BINS; i += blockDim.x) s_bin[i] = 0;
+      __syncthreads();
+      if (warp == 0) {     // the whole first warp finishes the reduction and plans
+        const bool has = lane < nwarp;
+        n_run = warp_sum_i64(has ? sh.red_a[lane] : 0); sum_kv = warp_sum_i64(has ? sh.red_b[lane] : 0);
+        next_arr = warp_min_i64(has ? sh.red_c[lane] : HFX_INF);
+        m_run = warp_or_u64(has ? sh.red_m0[lane] : 0); m_q = warp_or_u64(has ? sh.red_m1[lane] : 0);
+        hfx_replica_cfg cfg; cfg.mode = HFX_COLOCATED; cfg.token_cap = 1; cfg.batch_cap = 0;
+        int64_t now = 0, mat = 0;
+        if (real) { cfg = a.cfg[r]; now = a.now[r]; mat = a.mat[r]; }
+        ReplicaPlan pl0;
+        warp_plan(p, cfg, now, mat, n_run, sum_kv, m_run, m_q, pl0, lane);
+        if (lane == 0) { sh.plan = pl0; sh.next_arrival = next_arr; }
+      }
+      __syncthreads();
+    }
+    const ReplicaPlan pl = sh.plan;
+
+    // ---- keys (in registers), their range ---------------------------------------------------------
+    uint64_t item[TINY_IPT];
+    uint64_t mn = ~0ull, mx = 0;
+#pragma unroll
+    for (int k = 0; k < TINY_IPT; k++) {
+      const int q = threadIdx.x + k * THREADS_SMALL;
+      item[k] = ~0ull;
+      if (q < n_act) {
+        const uint4 w0 = w0r[k], w1 = s_w1[q];
+        const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
+        const int32_t row = (int32_t)w0.w;
+        const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
+        const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+        if (ordered) {
+          item[k] = (e.k48 << 16) | (uint32_t)q;     // records are in req_id order: position breaks ties
+          mn = item[k] < mn ? item[k] : mn; mx = item[k] > mx ? item[k] : mx;
+        } else {
+          const uint32_t uid = w0.z ^ 0x80000000u;
+          s_key[q] = (e.k48 << 16) | (uid >> 16);
+          s_lo[q] = (uid << 16) | (uint32_t)q;
+        }
+        a.slack[row] = e.slack;
+        if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
+        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+      }
+    }
+    bool sorted_done = false;
+    if (ordered && n_act > 0) {
+      // ---- distribution sort: bins by offset from the smallest item, rank inside the bin by counting ----
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const uint64_t x = __shfl_xor_sync(0xffffffffu, mn, o), y = __shfl_xor_sync(0xffffffffu, mx, o);
+        mn = x < mn ? x : mn; mx = y > mx ? y : mx;
+      }
+      if (lane == 0) { sh.red_m0[warp] = mn; sh.red_m1[warp] = mx; }
+      __syncthreads();
+      for (int k = 0; k < nwarp; k++) { const uint64_t x = sh.red_m0[k], y = sh.red_m1[k]; mn = x < mn ? x : mn; mx = y > mx ? y : mx; }
+      const uint64_t range = mx - mn;
+      int sft = 0;
+      if (range >= TINY_BINS) sft = 64 - __clzll((long long)range) - 9;     // (range >> sft) < TINY_BINS
+#pragma unroll
+      for (int k = 0; k < TINY_IPT; k++)
+        if (threadIdx.x + k * THREADS_SMALL < n_act) atomicAdd(&s_bin[(uint32_t)((item[k] - mn) >> sft)], 1u);
+      __syncthreads();
+      if (warp == 0) {     // exclusive scan of the bin counts by one warp; the largest bin
+        const int per = TINY_BINS / 32;
+        uint32_t cnt[TINY_BINS / 32];
+        uint32_t sum = 0, big = 0;
+#pragma unroll
+        for (int i = 0; i < per; i++) { cnt[i] = s_bin[lane * per + i]; sum += cnt[i]; big = cnt[i] > big ? cnt[i] : big; }
+        uint32_t v = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { const uint32_t x = __shfl_xor_sync(0xffffffffu, big, o); big = x > big ? x : big; }
+        uint32_t run = v - sum;
+#pragma unroll
+        for (int i = 0; i < per; i++) { s_bin[lane * per + i] = run; s_cur[lane * per + i] = run; run += cnt[i]; }
+        if (lane == 0) sh.red_n[0] = (int32_t)big;
+      }
+      __syncthreads();
+      if (sh.red_n[0] <= TINY_BIN_MAX) {
+#pragma unroll
+        for (int k = 0; k < TINY_IPT; k++)
+          if (threadIdx.x + k * THREADS_SMALL < n_act) s_key[atomicAdd(&s_cur[(uint32_t)((item[k] - mn) >> sft)], 1u)] = item[k];
+        __syncthreads();
+        for (int e = threadIdx.x; e < n_act; e += blockDim.x) {
+          const uint64_t x = s_key[e];
+          const uint32_t bi = (uint32_t)((x - mn) >> sft);
+          const uint32_t g0 = s_bin[bi], g1 = s_cur[bi];
+          uint32_t rank = 0;
+          for (uint32_t g = g0; g < g1; g++) rank += s_key[g] < x ? 1u : 0u;
+          s_lo[g0 + rank] = (uint32_t)(x & 0xffffu);
+        }
+        sorted_done = true;
+      } else {
+#pragma unroll
+        for (int k = 0; k < TINY_IPT; k++) { const int q = threadIdx.x + k * THREADS_SMALL; if (q < n_act) s_key[q] = item[k]; }
+      }
+    }
+    __syncthreads();
+    if (!sorted_done) {
+      if (ordered) {
+        block_sort<false>(s_key, nullptr, n_act);
+        for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] = (uint32_t)(s_key[q] & 0xffffu);
+      } else {
+        block_sort<true>(s_key, s_lo, n_act);
+        for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] &= 0xffffu;
+      }
+      __syncthreads();
+    }
+
+    // ---- admission: each thread walks TINY_IPT consecutive places of the order ---------------------
+    const int q0 = threadIdx.x * TINY_IPT;
+    int64_t cost[TINY_IPT], kvs[TINY_IPT];
+    int32_t rows[TINY_IPT], kinds[TINY_IPT];
+    int64_t my_cost = 0;
+    int32_t my_cnt = 0;
+#pragma unroll
+    for (int k = 0; k < TINY_IPT; k++) {
+      const int q = q0 + k;
+      cost[k] = -1; kvs[k] = 0; rows[k] = -1; kinds[k] = KIND_DEAD;
+      if (q < n_act) {
+        const int li = s_lo[q];
+        const uint4 w1 = s_w1[li];
+        rows[k] = s_row[li];
+        kinds[k] = (w1.w >> 8) & 0xff;
+        if (kinds[k] == KIND_QUEUED) {
+          const int64_t kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
+          const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
+          if (cc <= pl.budget) { cost[k] = cc; kvs[k] = kv; my_cost += cc; my_cnt++; }
+        }
+        a.order[b + q] = rows[k];
+      }
+    }
+    int64_t sc = warp_incl_scan_i64(my_cost, lane);
+    int32_t sn = warp_incl_scan_i32(my_cnt, lane);
+    if (lane == 31) { sh.red_a[warp] = sc; sh.red_n[warp] = sn; }
+    __syncthreads();
+    int64_t run_c = sc - my_cost;
+    int32_t run_n = sn - my_cnt;
+    for (int k = 0; k < warp; k++) { run_c += sh.red_a[k]; run_n += sh.red_n[k]; }
+    int64_t ac = 0, ak = 0;
+    int32_t an = 0;
+#pragma unroll
+    for (int k = 0; k < TINY_IPT; k++) {
+      const int q = q0 + k;
+      if (q < n_act) {
+        bool adm = false;
+        if (cost[k] >= 0) {
+          run_c += cost[k]; run_n += 1;
+          adm = run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap);
+          if (adm) { ac += cost[k]; ak += kvs[k]; an++; if (a.admitted_rows) a.admitted_rows[b + run_n - 1] = rows[k]; }
+        }
+        a.admit[rows[k]] = (uint8_t)((kinds[k] == KIND_RUNNING || adm) ? 1 : 0);
+        s_lo[q] = (s_lo[q] & 0xffffu) | (adm ? 0x10000u : 0u);
+      }
+    }
+    ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)warp_sum_i64(an);
+    __syncthreads();
+    if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_n[warp] = an; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int64_t adm_cost = 0, adm_kv = 0; int32_t adm_count = 0;
+      for (int k = 0; k < nwarp; k++) { adm_cost += sh.red_a[k]; adm_kv += sh.red_b[k]; adm_count += sh.red_n[k]; }
+      int64_t lp = 0;
+      const int64_t mat_next = dev_maturity_next(p, pl, adm_count, adm_cost, adm_kv, &lp);
+      int worked; int64_t t1, t2;
+      iteration_clock(pl, adm_count, lp, mat_next, worked, t1, t2);
+      sh.adm_cost = adm_cost; sh.adm_count = adm_count;
+      sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
+    }
+    __syncthreads();
+    const bool commit = real && (a.flags & HFX_COMMIT);
+    const int worked = sh.worked;
+    const int64_t mat_next = sh.red_c[0];
+    if (commit && !worked && ordered) {
+      // idle replica of an ordered step: its next arrival comes from the regroup's per-tile minima
+      int64_t v = HFX_INF;
+      for (int t = threadIdx.x; t < c.n_tiles; t += blockDim.x) { const int64_t x = c.fmin[(size_t)t * (R + 1) + r]; v = x < v ? x : v; }
+      block_min_arrival(v, sh);
+    }
+    if (threadIdx.x == 0 && real)
+      write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
+    if (a.admitted_rows)
+      for (int q = sh.adm_count + threadIdx.x; q < n; q += blockDim.x) a.admitted_rows[b + q] = -1;
+    if (commit) {
+      const int64_t t1 = sh.t1, t2 = sh.t2;
+      for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
+        const uint32_t lo = s_lo[q];
+        const int li = lo & 0xffff;
+        const uint4 w1 = s_w1[li];
+        commit_row(a, pl, (w1.w >> 8) & 0xff, (lo & 0x10000u) != 0, worked, t1, t2, s_row[li], (int32_t)w1.x,
+                   (int32_t)w1.y, (int32_t)w1.z);
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Oversize replicas (more items than a block can sort in shared memory): one cooperative kernel.
 // All blocks walk the replicas in the same order and share the work of each oversize one: keys
 // spread over the grid, a global bitonic network with bounded grid barriers, admission by block 0
@@ -725,12 +997,12 @@ int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
   {
     KernelScope ks(s, KSLOT_SEG_SMALL);
     const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
-    k_segment<<<grid, THREADS_SMALL, SMEM_SMALL, stream>>>(s->p, sa, c, 0, SEG_SMALL, 1);
+    k_segment_small<<<grid, THREADS_SMALL, SMEM_TINY, stream>>>(s->p, sa, c);
   }
-  if (n > SEG_SMALL) {
+  if (n > SEG_TINY) {
     KernelScope ks(s, KSLOT_SEG_MED);
     const int grid = R1 < s->n_sm ? R1 : s->n_sm;
-    k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, c, SEG_SMALL + 1, SEG_MED, 0);
+    k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, c, SEG_TINY + 1, SEG_MED, 0);
   }
   if (n > SEG_MED) {
     uint32_t *big_idx = reinterpret_cast<uint32_t *>(s->d_big_lo + s->max_rows);
@@ -745,7 +1017,8 @@ int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
 }
 
 int hfx_segment_configure() {
-  if (cudaFuncSetAttribute(k_segment, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_MED * 12) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_segment, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_MED * 12) != cudaSuccess ||
+      cudaFuncSetAttribute(k_segment_small, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TINY) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }

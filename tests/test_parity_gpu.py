@@ -151,6 +151,23 @@ def test_slack_saturation_and_budget_zero():
     g = assert_step_parity(make_wl(rows, [(200 * MS, 30 * MS, 0)], now=[SEC]), steps=2, commit=True)
 
 
+def test_maturity_saturates():
+    # k * E_d beyond 64 bits: one running request whose TPOT leaves 1 ns of slack per step, a slow prefill
+    model = (1 << 40, 40_000, 2, 1 << 33, 100_000, 20)
+    tpot = (1 << 33) + 100_000 + 20 * 1000 + 1
+    rows = [dict(state=gen.RUNNING, prompt_len=1000, gen=0, first_token_ns=0, req_id=0, output_len=50),
+            dict(prompt_len=64, req_id=1, output_len=50)]
+    wl = make_wl(rows, [(1 << 44, tpot, 0)], now=[SEC], model=model, budget_mode=gen.BUDGET_CAP_ONLY)
+    g = assert_step_parity(wl, steps=2, commit=True)
+    wl = make_wl(rows, [(1 << 44, tpot, 0)], now=[SEC], model=model, budget_mode=gen.BUDGET_CAP_ONLY)
+    g = assert_step_parity(wl)
+    assert g["maturity_next"][0] == 1 << 62 and g["adm_count"][0] == 1
+    # and just below the 64-bit product limit / the saturation point
+    for c0 in (1 << 20, 1 << 28, 1 << 29, 1 << 30):
+        wl = make_wl(rows, [(1 << 44, tpot, 0)], now=[SEC], model=(c0,) + model[1:], budget_mode=gen.BUDGET_CAP_ONLY)
+        assert_step_parity(wl)
+
+
 def test_oversize_prompts_and_batch_cap():
     wl = gen.random_table(15, 2500, 6, token_cap=512, batch_cap=3, modes=MODES3)
     assert_step_parity(wl, steps=4, commit=True)
