@@ -89,6 +89,9 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
 
   const size_t R2 = (size_t)n_replicas + 2;
   bool ok = true;
+  ok = ok && cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_cfg, sizeof(hfx_replica_cfg) * n_replicas) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_status, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_seg_count, sizeof(uint32_t) * R2) == cudaSuccess;
@@ -140,6 +143,9 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   if (!s) return;
   hfx_sched_host *h = reinterpret_cast<hfx_sched_host *>(s);
   cudaStreamSynchronize(s->stream);
+  if (s->side) { cudaStreamSynchronize(s->side); cudaStreamDestroy(s->side); }
+  if (s->ev_fork) cudaEventDestroy(s->ev_fork);
+  if (s->ev_join) cudaEventDestroy(s->ev_join);
   cudaFree(s->d_cfg); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
   cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_fmin); cudaFree(s->d_tile_mode);

@@ -75,6 +75,8 @@ struct hfx_sched {
   int64_t max_rows;
   int n_sm;
   cudaStream_t stream;
+  cudaStream_t side;        // second stream: the (usually empty) kernels of larger replicas run beside the main one
+  cudaEvent_t ev_fork, ev_join;
   int64_t launches;
   int profiling;
   std::vector<HfxBracket> *brackets;
@@ -314,19 +316,19 @@ __device__ __forceinline__ int32_t warp_incl_scan_i32(int32_t v, int lane) {
 
 // Brackets one kernel launch with events when profiling is on; counts the launch either way.
 struct KernelScope {
-  hfx_sched *s; HfxBracket br; bool on;
-  KernelScope(hfx_sched *s_, int slot) : s(s_), on(false) {
+  hfx_sched *s; HfxBracket br; bool on; cudaStream_t st;
+  KernelScope(hfx_sched *s_, int slot, cudaStream_t stream = nullptr) : s(s_), on(false), st(stream ? stream : s_->stream) {
     s->launches++;
     if (s->profiling && s->brackets) {
       br.slot = slot;
       if (cudaEventCreate(&br.a) == cudaSuccess && cudaEventCreate(&br.b) == cudaSuccess) {
-        cudaEventRecord(br.a, s->stream);
+        cudaEventRecord(br.a, st);
         on = true;
       }
     }
   }
   ~KernelScope() {
-    if (on) { cudaEventRecord(br.b, s->stream); s->brackets->push_back(br); }
+    if (on) { cudaEventRecord(br.b, st); s->brackets->push_back(br); }
   }
 };
 

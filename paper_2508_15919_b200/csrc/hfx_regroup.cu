@@ -125,61 +125,37 @@ __global__ void __launch_bounds__(THREADS_TILE) k_count(const HfxParams p, const
 }
 
 // ------------------------------------------------------------------------------------------------
-// k_colscan: for each column of the tile matrix (2 x (R+1) columns: all rows, active rows) the
-// exclusive prefix of its counts over the tiles, in place, and the column total.
-// Block = 32 columns x 32 chunks of tiles.
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) k_colscan(uint32_t *__restrict__ M, int32_t n_tiles, int32_t R1,
-                                                  uint32_t *__restrict__ tot_all, uint32_t *__restrict__ tot_act) {
-  __shared__ uint32_t part[32][33];
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int C = 2 * R1;
-  const int col = blockIdx.x * 32 + lane;
-  const int cb = (n_tiles + 31) / 32;
-  const int t0 = w * cb < n_tiles ? w * cb : n_tiles;
-  const int t1 = (t0 + cb < n_tiles) ? t0 + cb : n_tiles;
-  uint32_t sum = 0;
-  if (col < C)
-    for (int t = t0; t < t1; t++) sum += M[(size_t)t * C + col];
-  part[w][lane] = sum;
-  __syncthreads();
-  uint32_t pre = 0;
-  for (int k = 0; k < w; k++) pre += part[k][lane];
-  if (col < C) {
-    uint32_t run = pre;
-    for (int t = t0; t < t1; t++) {
-      const size_t idx = (size_t)t * C + col;
-      const uint32_t v = M[idx];
-      M[idx] = run;
-      run += v;
-    }
-    if (w == 31) { if (col < R1) tot_all[col] = pre + sum; else tot_act[col - R1] = pre + sum; }
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
 // k_offsets: exclusive scan of the per-replica totals (one block) -> seg_begin and the user-visible
 // seg_off; zeroes the fill cursors of the atomic mode; flags[2] = the largest number of items any
 // replica has to sort (its active rows; without "ordered" also its inactive rows); re-arms the
 // "ordered" word of the next step.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) k_offsets(const uint32_t *__restrict__ tot_all, const uint32_t *__restrict__ tot_act,
-                                                  int32_t R, uint32_t *__restrict__ seg_begin, uint32_t *__restrict__ cursor,
-                                                  int32_t *__restrict__ seg_off, uint32_t *__restrict__ flags,
-                                                  uint32_t parity, uint32_t force_unordered) {
+struct OffsetArgs {
+  const uint32_t *tot_all; const uint32_t *tot_act; int32_t R; uint32_t *seg_begin; uint32_t *cursor; int32_t *seg_off;
+  uint32_t *flags; uint32_t parity; uint32_t force_unordered;
+};
+
+// one block of 1024 threads
+__device__ void offsets_block(const OffsetArgs &oa) {
+  const uint32_t *__restrict__ tot_all = oa.tot_all; const uint32_t *__restrict__ tot_act = oa.tot_act;
+  const int32_t R = oa.R;
+  uint32_t *__restrict__ seg_begin = oa.seg_begin; uint32_t *__restrict__ cursor = oa.cursor;
+  int32_t *__restrict__ seg_off = oa.seg_off; uint32_t *__restrict__ flags = oa.flags;
+  const uint32_t parity = oa.parity, force_unordered = oa.force_unordered;
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t carry_s, max_s;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (threadIdx.x == 0) { carry_s = 0; max_s = 0; if (force_unordered) flags[parity] = 0; }
   __syncthreads();
-  const bool ordered = flags[parity] != 0;
+  const bool ordered = __ldcg(flags + parity) != 0;
   const int total = R + 1;  // buckets 0..R
   uint32_t mx = 0;
   for (int base = 0; base < total; base += blockDim.x) {
     const int i = base + threadIdx.x;
-    const uint32_t c = i < total ? tot_all[i] : 0;
+    // (L2 loads: in the fused kernel other blocks wrote these totals a moment ago)
+    const uint32_t c = i < total ? __ldcg(tot_all + i) : 0;
     if (i < total) {
-      const uint32_t act = tot_act[i];
+      const uint32_t act = __ldcg(tot_act + i);
       const uint32_t need = ordered ? act : (act > c - act ? act : c - act);
       mx = need > mx ? need : mx;
     }
@@ -212,6 +188,54 @@ __global__ void __launch_bounds__(1024) k_offsets(const uint32_t *__restrict__ t
   __syncthreads();
   if (threadIdx.x == 0) { seg_begin[total] = carry_s; flags[2] = max_s; flags[parity ^ 1u] = 1u; }
 }
+
+__global__ void __launch_bounds__(1024) k_offsets(const OffsetArgs oa) { offsets_block(oa); }
+
+// ------------------------------------------------------------------------------------------------
+// k_colscan: for each column of the tile matrix (2 x (R+1) columns: all rows, active rows) the
+// exclusive prefix of its counts over the tiles, in place, and the column total.
+// Block = 32 columns x 32 chunks of tiles.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) k_colscan(uint32_t *__restrict__ M, int32_t n_tiles, int32_t R1,
+                                                  uint32_t *__restrict__ tot_all, uint32_t *__restrict__ tot_act,
+                                                  uint32_t *__restrict__ done, const OffsetArgs oa) {
+  __shared__ uint32_t part[32][33];
+  __shared__ uint32_t s_last;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int C = 2 * R1;
+  const int col = blockIdx.x * 32 + lane;
+  const int cb = (n_tiles + 31) / 32;
+  const int t0 = w * cb < n_tiles ? w * cb : n_tiles;
+  const int t1 = (t0 + cb < n_tiles) ? t0 + cb : n_tiles;
+  uint32_t sum = 0;
+  if (col < C)
+    for (int t = t0; t < t1; t++) sum += M[(size_t)t * C + col];
+  part[w][lane] = sum;
+  __syncthreads();
+  uint32_t pre = 0;
+  for (int k = 0; k < w; k++) pre += part[k][lane];
+  if (col < C) {
+    uint32_t run = pre;
+    for (int t = t0; t < t1; t++) {
+      const size_t idx = (size_t)t * C + col;
+      const uint32_t v = M[idx];
+      M[idx] = run;
+      run += v;
+    }
+    if (w == 31) { if (col < R1) tot_all[col] = pre + sum; else tot_act[col - R1] = pre + sum; }
+  }
+  // the block that finishes last turns the totals into offsets (no block waits for another)
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(done, 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (s_last) {
+    __threadfence();
+    offsets_block(oa);
+    if (threadIdx.x == 0) *done = 0;
+  }
+}
+
 
 // ------------------------------------------------------------------------------------------------
 // Per-row work of the streaming pass: what does not depend on the replica's aggregates (prefill
@@ -525,12 +549,10 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
     }
     {
       KernelScope ks(s, KSLOT_COLSCAN);
-      k_colscan<<<(2 * R1 + 31) / 32, 1024, 0, stream>>>(s->d_tile_hist, n_tiles, R1, s->d_seg_count, s->d_act_count);
-    }
-    {
-      KernelScope ks(s, KSLOT_OFFSETS);
-      k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, s->d_act_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags,
-                                        s->step_parity, 0u);
+      const OffsetArgs oa = {s->d_seg_count, s->d_act_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags,
+                             s->step_parity, 0u};
+      k_colscan<<<(2 * R1 + 31) / 32, 1024, 0, stream>>>(s->d_tile_hist, n_tiles, R1, s->d_seg_count, s->d_act_count,
+                                                          s->d_flags + 3, oa);
     }
     {
       KernelScope ks(s, KSLOT_REGROUP);
@@ -549,8 +571,9 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
     }
     {
       KernelScope ks(s, KSLOT_OFFSETS);
-      k_offsets<<<1, 1024, 0, stream>>>(s->d_seg_count, s->d_act_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags,
-                                        s->step_parity, 1u);
+      const OffsetArgs oa = {s->d_seg_count, s->d_act_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags,
+                             s->step_parity, 1u};
+      k_offsets<<<1, 1024, 0, stream>>>(oa);
     }
     {
       KernelScope ks(s, KSLOT_REGROUP);

@@ -994,23 +994,41 @@ int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
   c.fmin = s->d_tile_fmin; c.parity = s->step_parity;
   int32_t tile_rows;
   hfx_tile_shape(n, &tile_rows, &c.n_tiles);
-  {
+  // Replicas too large for the small kernel are rare; their kernels (which leave at once when there is
+  // nothing for them) run on a second stream beside the small-replica kernel, forked and joined by events.
+  const bool larger = n > SEG_TINY;
+  const bool beside = larger && !s->profiling;
+  cudaStream_t st2 = beside ? s->side : stream;
+  if (beside) {
+    if (cudaEventRecord(s->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(s->side, s->ev_fork, 0) != cudaSuccess)
+      return HFX_E_CUDA;
+  }
+  if (!beside) {
     KernelScope ks(s, KSLOT_SEG_SMALL);
     const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
     k_segment_small<<<grid, THREADS_SMALL, SMEM_TINY, stream>>>(s->p, sa, c);
   }
-  if (n > SEG_TINY) {
-    KernelScope ks(s, KSLOT_SEG_MED);
+  if (larger) {
+    KernelScope ks(s, KSLOT_SEG_MED, st2);
     const int grid = R1 < s->n_sm ? R1 : s->n_sm;
-    k_segment<<<grid, THREADS_MED, SEG_MED * 12, stream>>>(s->p, sa, c, SEG_TINY + 1, SEG_MED, 0);
+    k_segment<<<grid, THREADS_MED, SEG_MED * 12, st2>>>(s->p, sa, c, SEG_TINY + 1, SEG_MED, 0);
   }
   if (n > SEG_MED) {
     uint32_t *big_idx = reinterpret_cast<uint32_t *>(s->d_big_lo + s->max_rows);
-    if (cudaMemsetAsync(s->d_barrier, 0, 64, stream) != cudaSuccess) return HFX_E_CUDA;
+    if (cudaMemsetAsync(s->d_barrier, 0, 64, st2) != cudaSuccess) return HFX_E_CUDA;
     void *args[] = {(void *)&s->p, (void *)&sa, (void *)&c, (void *)&s->d_big_hi, (void *)&s->d_big_lo, (void *)&big_idx,
                     (void *)&s->d_barrier, (void *)&s->d_status};
-    KernelScope ks(s, KSLOT_BIG);
-    if (cudaLaunchCooperativeKernel((void *)k_big, dim3(s->n_sm), dim3(512), args, 0, stream) != cudaSuccess)
+    KernelScope ks(s, KSLOT_BIG, st2);
+    if (cudaLaunchCooperativeKernel((void *)k_big, dim3(s->n_sm), dim3(512), args, 0, st2) != cudaSuccess)
+      return HFX_E_CUDA;
+  }
+  if (beside) {
+    {
+      KernelScope ks(s, KSLOT_SEG_SMALL);
+      const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
+      k_segment_small<<<grid, THREADS_SMALL, SMEM_TINY, stream>>>(s->p, sa, c);
+    }
+    if (cudaEventRecord(s->ev_join, s->side) != cudaSuccess || cudaStreamWaitEvent(stream, s->ev_join, 0) != cudaSuccess)
       return HFX_E_CUDA;
   }
   return HFX_OK;
