@@ -94,6 +94,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   ok = ok && cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_cfg, sizeof(hfx_replica_cfg) * n_replicas) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_status, 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_mode, (size_t)n_replicas + 16) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_seg_count, sizeof(uint32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_seg_begin, sizeof(uint32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_cursor, sizeof(uint32_t) * 2 * R2) == cudaSuccess;
@@ -127,6 +128,11 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     memcpy(h->h_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas);
     ok = ok && cudaMemcpy(s->d_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemset(s->d_status, 0, 256) == cudaSuccess;
+    {
+      std::vector<uint8_t> modes((size_t)n_replicas);
+      for (int r = 0; r < n_replicas; r++) modes[r] = (uint8_t)replicas[r].mode;
+      ok = ok && cudaMemcpy(s->d_mode, modes.data(), (size_t)n_replicas, cudaMemcpyHostToDevice) == cudaSuccess;
+    }
     const uint32_t init_flags[4] = {1u, 1u, 0u, 0u};
     ok = ok && cudaMemcpy(s->d_flags, init_flags, sizeof(init_flags), cudaMemcpyHostToDevice) == cudaSuccess;
   }
@@ -146,7 +152,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   if (s->side) { cudaStreamSynchronize(s->side); cudaStreamDestroy(s->side); }
   if (s->ev_fork) cudaEventDestroy(s->ev_fork);
   if (s->ev_join) cudaEventDestroy(s->ev_join);
-  cudaFree(s->d_cfg); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
+  cudaFree(s->d_cfg); cudaFree(s->d_mode); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
   cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_fmin); cudaFree(s->d_tile_mode);
   cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier);

@@ -46,8 +46,8 @@ struct HfxParams {
 
 // One row after regrouping by replica: everything the per-replica kernel needs, 32 bytes
 // (one L2 sector), so that kernel never goes back to the table for reads.
-struct __align__(16) HfxRec {
-  int64_t base;      // slack before the per-replica shift; arrival for KIND_FUTURE
+struct __align__(32) HfxRec {
+  int64_t base;      // slack before the per-replica shift (see ReplicaPlan); arrival for KIND_FUTURE
   int32_t req_id;
   int32_t row;
   int32_t prompt;
@@ -82,6 +82,7 @@ struct hfx_sched {
   std::vector<HfxBracket> *brackets;
   // device
   hfx_replica_cfg *d_cfg;   // [R]
+  uint8_t *d_mode;          // [R] replica modes, one byte each
   uint32_t *d_status;       // sticky status word
   uint32_t *d_seg_count;    // [R+2] rows per replica (+ the bad-replica bucket R)
   uint32_t *d_act_count;    // [R+2] active rows (in flight or in the visible queue) per replica
@@ -121,8 +122,9 @@ struct ReplicaPlan {
   int64_t tpot_eff;   // strictest TPOT of the running batch (HFX_INF if none)
   int64_t e_d;
   int64_t budget;
-  int64_t shift_run;  // slack of a running row   = base - shift_run
-  int64_t shift_dq;   // slack of a decode-queued = base - shift_dq
+  int64_t shift_run;  // slack of a running row = base - shift_run      (now + E_d)
+  int64_t shift_q;    // slack of a queued row  = base - shift_q        (earliest start; + predicted TPOT base on DECODE)
+  int64_t tpot_q0;    // predicted TPOT of a queued row = tpot_q0 + d2 * (prompt_len + gen)
   int32_t mode, token_cap, batch_cap;
 };
 
@@ -191,8 +193,9 @@ __device__ inline void dev_plan(const HfxParams &p, const hfx_replica_cfg &cfg, 
   }
   if (now < mat) budget = 0;
   pl.budget = budget;
-  pl.shift_run = pl.e_d;
-  pl.shift_dq = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
+  pl.tpot_q0 = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
+  pl.shift_run = now + pl.e_d;
+  pl.shift_q = pl.start + (cfg.mode == HFX_DECODE ? pl.tpot_q0 : 0);
 }
 
 // The same plan computed by a whole warp (all 32 lanes call with the same arguments and get the same
@@ -256,8 +259,9 @@ __device__ inline void warp_plan(const HfxParams &p, const hfx_replica_cfg &cfg,
   }
   if (now < mat) budget = 0;
   pl.budget = budget;
-  pl.shift_run = pl.e_d;
-  pl.shift_dq = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
+  pl.tpot_q0 = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
+  pl.shift_run = now + pl.e_d;
+  pl.shift_q = pl.start + (cfg.mode == HFX_DECODE ? pl.tpot_q0 : 0);
 }
 
 // Dispatching step 4: maturity time after admitting adm_count requests of adm_cost in total.
@@ -337,7 +341,7 @@ struct RegroupArgs {
   const int32_t *replica_id; const uint8_t *class_id; const uint8_t *state; const int32_t *prompt_len;
   const int32_t *output_len; const int32_t *gen; const int64_t *arrival; const int64_t *first_token;
   const int32_t *req_id; const int32_t *weight;
-  const int64_t *now; const int64_t *mat; const hfx_replica_cfg *cfg;
+  const int64_t *now; const int64_t *mat; const hfx_replica_cfg *cfg; const uint8_t *mode;
   int64_t *pred_ttft;    // optional output
   int64_t n;
   // outputs of inactive rows, written by the regroup itself when the step is "ordered"

@@ -247,18 +247,18 @@ struct RowIn {
   int64_t arrival, first_token;
 };
 
-// Fills the record of a row of kind in.kind; returns the row's predicted TTFT (0 if inactive).
-__device__ __forceinline__ int64_t make_record(const HfxParams &p, const RegroupArgs &a, const int64_t *s_ttft,
-                                               const int64_t *s_tpot, const uint8_t *s_prio, int64_t i, const RowIn &in,
-                                               HfxRec &r) {
+// Fills the record of a row of kind in.kind.  The slack base is free of per-replica quantities (the
+// replica's clock, earliest start and E_d are subtracted later, once per replica):
+//   in flight                base = first_token + (gen+1) * tpot_slo              (next-token deadline)
+//   queued, colocated/prefill base = ttft_slo + arrival - E_p(prompt_len)
+//   queued on a decode replica base = first_token + (gen+1) * tpot_slo - d2 * (prompt_len + gen)
+//   not yet arrived          base = arrival
+__device__ __forceinline__ void make_record(const HfxParams &p, const int64_t *s_ttft, const int64_t *s_tpot,
+                                            const uint8_t *s_prio, int64_t i, const RowIn &in, int mode, HfxRec &r) {
   r.req_id = in.req_id; r.row = (int32_t)i; r.prompt = in.prompt; r.gen = in.gen; r.output_len = in.out_len;
   r.cls = (uint8_t)in.cls; r.kind = (uint8_t)(in.kind & 3u); r.prio = 63; r.pad = 0; r.base = 0;
-  int64_t pred_ttft = 0;
   if (in.kind == KIND_FUTURE) r.base = in.arrival;
   else if (in.kind <= KIND_QUEUED) {
-    const int64_t now = __ldg(a.now + in.rid), mat = __ldg(a.mat + in.rid);
-    const int32_t mode = __ldg(&a.cfg[in.rid].mode);
-    const int64_t start = now > mat ? now : mat;
     int prio;
     if (p.weight_max > 0) {
       const int64_t w = (int64_t)p.weight_max - in.weight;
@@ -266,26 +266,26 @@ __device__ __forceinline__ int64_t make_record(const HfxParams &p, const Regroup
     } else prio = s_prio[in.cls];
     r.prio = (uint8_t)prio;
     const int64_t ttft = s_ttft[in.cls], tpot = s_tpot[in.cls];
-    if (in.kind == KIND_RUNNING) {
-      r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot - now : BASE_UNBOUNDED;
-      pred_ttft = in.first_token - in.arrival;
-    } else if (mode == HFX_DECODE) {
-      r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot - start - p.d2 * ((int64_t)in.prompt + in.gen)
-                        : BASE_UNBOUNDED;
-      pred_ttft = in.first_token - in.arrival;
-    } else {
-      pred_ttft = (start - in.arrival) + dev_Ep(p, in.prompt);
-      r.base = ttft > 0 ? ttft - pred_ttft : BASE_UNBOUNDED;
-    }
+    if (in.kind == KIND_RUNNING) r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot : BASE_UNBOUNDED;
+    else if (mode == HFX_DECODE)
+      r.base = tpot > 0 ? in.first_token + ((int64_t)in.gen + 1) * tpot - p.d2 * ((int64_t)in.prompt + in.gen) : BASE_UNBOUNDED;
+    else r.base = ttft > 0 ? ttft + in.arrival - dev_Ep(p, in.prompt) : BASE_UNBOUNDED;
   }
-  return pred_ttft;
 }
 
+// predicted TTFT of a row (optional output; the one place that needs the replica's clock here)
+__device__ __forceinline__ int64_t row_pred_ttft(const HfxParams &p, const RegroupArgs &a, const RowIn &in, int mode) {
+  if (in.kind > KIND_QUEUED) return 0;
+  if (in.kind == KIND_RUNNING || mode == HFX_DECODE) return in.first_token - in.arrival;
+  const int64_t now = __ldg(a.now + in.rid), mat = __ldg(a.mat + in.rid);
+  return ((now > mat ? now : mat) - in.arrival) + dev_Ep(p, in.prompt);
+}
+
+// One 32-byte store per record: a whole L2 sector at once (two 16-byte stores would each be a
+// partial-sector write).
 __device__ __forceinline__ void store_record(HfxRec *rec, uint32_t pos, const HfxRec &r) {
-  uint4 *dst = reinterpret_cast<uint4 *>(rec + pos);
-  const uint4 *src = reinterpret_cast<const uint4 *>(&r);
-  dst[0] = src[0];
-  dst[1] = src[1];
+  const uint64_t *w = reinterpret_cast<const uint64_t *>(&r);
+  asm volatile("st.global.v4.b64 [%0], {%1, %2, %3, %4};" ::"l"(rec + pos), "l"(w[0]), "l"(w[1]), "l"(w[2]), "l"(w[3]) : "memory");
 }
 
 // rows 4v .. 4v+3 with 16-byte loads
@@ -322,9 +322,25 @@ __device__ __forceinline__ void stage_classes(const HfxParams &p, int64_t *s_ttf
   }
 }
 
-// the outputs of an inactive row, written by the regroup of an ordered step
-__device__ __forceinline__ void write_inactive(const RegroupArgs &a, int64_t i, uint32_t opos, int bkt) {
-  a.order[opos] = (int32_t)i;
+// Default outputs of rows 4v .. 4v+3 (slack 0, admit 0, ...), written with vector stores for every
+// row of an ordered step; the replica kernels overwrite them for the active rows afterwards.
+__device__ __forceinline__ void write_defaults4(const RegroupArgs &a, int64_t v, const int bkt[4]) {
+  longlong2 *sl = reinterpret_cast<longlong2 *>(a.slack) + 2 * v;
+  sl[0] = make_longlong2(0, 0); sl[1] = make_longlong2(0, 0);
+  reinterpret_cast<uint32_t *>(a.admit)[v] = 0u;
+  if (a.pred_tpot) {
+    longlong2 *pt = reinterpret_cast<longlong2 *>(a.pred_tpot) + 2 * v;
+    pt[0] = make_longlong2(0, 0); pt[1] = make_longlong2(0, 0);
+  }
+  if (a.key) {
+    const uint64_t k = dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
+    ulonglong2 *kp = reinterpret_cast<ulonglong2 *>(a.key) + 2 * v;
+    kp[0] = make_ulonglong2(((uint64_t)(bkt[0] & 0xffff) << 48) | k, ((uint64_t)(bkt[1] & 0xffff) << 48) | k);
+    kp[1] = make_ulonglong2(((uint64_t)(bkt[2] & 0xffff) << 48) | k, ((uint64_t)(bkt[3] & 0xffff) << 48) | k);
+  }
+}
+
+__device__ __forceinline__ void write_defaults1(const RegroupArgs &a, int64_t i, int bkt) {
   a.slack[i] = 0;
   a.admit[i] = 0;
   if (a.pred_tpot) a.pred_tpot[i] = 0;
@@ -343,9 +359,10 @@ __global__ void __launch_bounds__(256) k_regroup_atomic(const HfxParams p, const
   const int R = p.n_replicas;
   auto emit = [&](int64_t i, const RowIn &in) {
     HfxRec r;
-    const int64_t pt = make_record(p, a, s_ttft, s_tpot, s_prio, i, in, r);
-    if (a.pred_ttft) a.pred_ttft[i] = pt;
     const int bkt = bucket_of(in.rid, R);
+    const int mode = bkt < R ? __ldg(a.mode + bkt) : 0;
+    make_record(p, s_ttft, s_tpot, s_prio, i, in, mode, r);
+    if (a.pred_ttft) a.pred_ttft[i] = row_pred_ttft(p, a, in, mode);
     const uint32_t pos = in.kind <= KIND_QUEUED ? seg_begin[bkt] + atomicAdd(&cursor[bkt], 1u)
                                                 : seg_begin[bkt] + tot_act[bkt] + atomicAdd(&cursor[R + 2 + bkt], 1u);
     store_record(rec, pos, r);
@@ -382,6 +399,7 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   uint32_t *s_bin = s_bact + R1;                                     // [R1]   where its inactive rows start
   uint16_t *s_stage = reinterpret_cast<uint16_t *>(s_bin + R1);      // [T]    tile rows grouped by replica (+ class bit)
   uint16_t *s_P = s_stage + T;                                       // [T+1]  active rows before each tile position
+  uint8_t *s_mode = reinterpret_cast<uint8_t *>(s_P + T + 1);        // [R1]   replica modes
   __shared__ int64_t s_ttft[HFX_MAX_CLASSES], s_tpot[HFX_MAX_CLASSES];
   __shared__ uint8_t s_prio[HFX_MAX_CLASSES];
   __shared__ uint32_t s_warp[32];
@@ -391,7 +409,10 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   const bool use_fmin = ordered && a.commit;
 
   stage_classes(p, s_ttft, s_tpot, s_prio);
-  for (int i = tid; i < R1; i += blockDim.x) { s_cnt[i] = 0; s_off[i] = 0; if (use_fmin) s_fmin[i] = HFX_INF; }
+  for (int i = tid; i < R1; i += blockDim.x) {
+    s_cnt[i] = 0; s_off[i] = 0; s_mode[i] = i < R ? a.mode[i] : 0;
+    if (use_fmin) s_fmin[i] = HFX_INF;
+  }
   __syncthreads();
 
   const int64_t lo = (int64_t)blockIdx.x * T;
@@ -493,26 +514,31 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
       const uint32_t me = (uint32_t)il | (act ? 0x8000u : 0u);
       for (uint32_t g = g0; g < g1; g++) { const uint32_t e = s_stage[g]; rank += ((e ^ me) < 0x8000u && e < me) ? 1u : 0u; }
     } else rank = atomicAdd(act ? &s_cnt[bkt] : &s_off[bkt], 1u);
+    const int rmode = s_mode[bkt];
+    if (a.pred_ttft) a.pred_ttft[i] = row_pred_ttft(p, a, in, rmode);
     if (act || !ordered) {
       HfxRec r;
-      const int64_t pt = make_record(p, a, s_ttft, s_tpot, s_prio, i, in, r);
-      if (a.pred_ttft) a.pred_ttft[i] = pt;
+      make_record(p, s_ttft, s_tpot, s_prio, i, in, rmode, r);
       store_record(ta.rec, (act ? s_bact[bkt] : s_bin[bkt]) + rank, r);
     } else {
-      if (a.pred_ttft) a.pred_ttft[i] = 0;
-      write_inactive(a, i, s_bin[bkt] + rank, bkt);
+      a.order[s_bin[bkt] + rank] = (int32_t)i;
       if (use_fmin && in.kind == KIND_FUTURE) atomicMin(reinterpret_cast<long long *>(&s_fmin[bkt]), (long long)in.arrival);
     }
   };
   for (int v = tid; v < nvec; v += blockDim.x) {
     RowIn in[4];
     load_rows4(a, ta.rowflag, v0 + v, in);
+    if (ordered) {
+      const int bk[4] = {bucket_of(in[0].rid, R), bucket_of(in[1].rid, R), bucket_of(in[2].rid, R), bucket_of(in[3].rid, R)};
+      write_defaults4(a, v0 + v, bk);
+    }
 #pragma unroll
     for (int k = 0; k < 4; k++) emit(lo + 4 * (int64_t)v + k, 4 * v + k, in[k]);
   }
   for (int i = (nvec << 2) + tid; i < nt; i += blockDim.x) {
     RowIn in;
     load_row1(a, ta.rowflag, lo + i, in);
+    if (ordered) write_defaults1(a, lo + i, bucket_of(in.rid, R));
     emit(lo + i, i, in);
   }
   if (use_fmin) {
@@ -526,7 +552,8 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
 // host side
 // ------------------------------------------------------------------------------------------------
 size_t hfx_regroup_smem(int R1, int tile_rows) {
-  return sizeof(int64_t) * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) + 32;
+  return sizeof(int64_t) * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) +
+         (size_t)R1 + 32;
 }
 
 int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {

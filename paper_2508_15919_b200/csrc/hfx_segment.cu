@@ -172,9 +172,8 @@ __device__ __forceinline__ RowEval eval_row(const HfxParams &p, const ReplicaPla
     e.pred_tpot = pl.e_d; kslack = e.slack;
   } else if (kind == KIND_QUEUED) {
     e.phase = PH_QUEUED; kprio = prio;
-    e.pred_tpot = pl.shift_dq + p.d2 * ((int64_t)prompt + gen);
-    if (pl.mode == HFX_DECODE) e.slack = base == BASE_UNBOUNDED ? HFX_SLACK_MAX : base - pl.shift_dq;
-    else e.slack = base == BASE_UNBOUNDED ? HFX_SLACK_MAX : base;
+    e.pred_tpot = pl.tpot_q0 + p.d2 * ((int64_t)prompt + gen);
+    e.slack = base == BASE_UNBOUNDED ? HFX_SLACK_MAX : base - pl.shift_q;
     kslack = e.slack;
   }
   e.k48 = dev_key48(e.phase, kprio, kslack);

@@ -32,7 +32,7 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
   ra.replica_id = t->replica_id; ra.class_id = t->class_id; ra.state = t->state; ra.prompt_len = t->prompt_len;
   ra.output_len = t->output_len; ra.gen = t->gen; ra.arrival = t->arrival_ns; ra.first_token = t->first_token_ns;
   ra.req_id = t->req_id; ra.weight = s->p.weight_max > 0 ? t->weight : nullptr;
-  ra.now = st->now_ns; ra.mat = st->maturity_ns; ra.cfg = s->d_cfg; ra.pred_ttft = o->pred_ttft_ns; ra.n = t->n_rows;
+  ra.now = st->now_ns; ra.mat = st->maturity_ns; ra.cfg = s->d_cfg; ra.mode = s->d_mode; ra.pred_ttft = o->pred_ttft_ns; ra.n = t->n_rows;
   ra.slack = o->slack_ns; ra.pred_tpot = o->pred_tpot_ns; ra.key = o->key; ra.order = o->order; ra.admit = o->admit;
   ra.admitted_rows = o->admitted_rows; ra.commit = flags & HFX_COMMIT;
   int rc = hfx_launch_regroup(s, ra, o->seg_off);
