@@ -273,12 +273,11 @@ __device__ __forceinline__ void make_record(const HfxParams &p, const int64_t *s
   }
 }
 
-// predicted TTFT of a row (optional output; the one place that needs the replica's clock here)
-__device__ __forceinline__ int64_t row_pred_ttft(const HfxParams &p, const RegroupArgs &a, const RowIn &in, int mode) {
+// predicted TTFT of a row (optional output)
+__device__ __forceinline__ int64_t row_pred_ttft(const HfxParams &p, const RowIn &in, int mode, int64_t start) {
   if (in.kind > KIND_QUEUED) return 0;
   if (in.kind == KIND_RUNNING || mode == HFX_DECODE) return in.first_token - in.arrival;
-  const int64_t now = __ldg(a.now + in.rid), mat = __ldg(a.mat + in.rid);
-  return ((now > mat ? now : mat) - in.arrival) + dev_Ep(p, in.prompt);
+  return (start - in.arrival) + dev_Ep(p, in.prompt);
 }
 
 // One 32-byte store per record: a whole L2 sector at once (two 16-byte stores would each be a
@@ -322,29 +321,45 @@ __device__ __forceinline__ void stage_classes(const HfxParams &p, int64_t *s_ttf
   }
 }
 
-// Default outputs of rows 4v .. 4v+3 (slack 0, admit 0, ...), written with vector stores for every
-// row of an ordered step; the replica kernels overwrite them for the active rows afterwards.
-__device__ __forceinline__ void write_defaults4(const RegroupArgs &a, int64_t v, const int bkt[4]) {
+// Per-row outputs that the regroup can finish by itself: slack 0 / admit 0 / inactive key for rows
+// the scheduler does not look at, and the final slack and key of queued rows on colocated and
+// prefill replicas (slack = base - earliest start needs nothing from the running batch).  Rows in
+// flight and queued rows of decode replicas get their slack from the replica kernels afterwards;
+// those kernels also set admit = 1 where it applies.
+struct RowOut { int64_t slack; uint64_t k48; };
+
+__device__ __forceinline__ RowOut row_out(const HfxRec &r, int mode, int64_t start) {
+  RowOut o;
+  o.slack = 0;
+  o.k48 = dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
+  if (r.kind == KIND_QUEUED && mode != HFX_DECODE) {
+    o.slack = r.base == BASE_UNBOUNDED ? HFX_SLACK_MAX : r.base - start;
+    o.k48 = dev_key48(PH_QUEUED, r.prio, o.slack);
+  }
+  return o;
+}
+
+// rows 4v .. 4v+3 with vector stores
+__device__ __forceinline__ void write_outputs4(const RegroupArgs &a, int64_t v, const int bkt[4], const RowOut o[4]) {
   longlong2 *sl = reinterpret_cast<longlong2 *>(a.slack) + 2 * v;
-  sl[0] = make_longlong2(0, 0); sl[1] = make_longlong2(0, 0);
+  sl[0] = make_longlong2(o[0].slack, o[1].slack); sl[1] = make_longlong2(o[2].slack, o[3].slack);
   reinterpret_cast<uint32_t *>(a.admit)[v] = 0u;
   if (a.pred_tpot) {
     longlong2 *pt = reinterpret_cast<longlong2 *>(a.pred_tpot) + 2 * v;
     pt[0] = make_longlong2(0, 0); pt[1] = make_longlong2(0, 0);
   }
   if (a.key) {
-    const uint64_t k = dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
     ulonglong2 *kp = reinterpret_cast<ulonglong2 *>(a.key) + 2 * v;
-    kp[0] = make_ulonglong2(((uint64_t)(bkt[0] & 0xffff) << 48) | k, ((uint64_t)(bkt[1] & 0xffff) << 48) | k);
-    kp[1] = make_ulonglong2(((uint64_t)(bkt[2] & 0xffff) << 48) | k, ((uint64_t)(bkt[3] & 0xffff) << 48) | k);
+    kp[0] = make_ulonglong2(((uint64_t)(bkt[0] & 0xffff) << 48) | o[0].k48, ((uint64_t)(bkt[1] & 0xffff) << 48) | o[1].k48);
+    kp[1] = make_ulonglong2(((uint64_t)(bkt[2] & 0xffff) << 48) | o[2].k48, ((uint64_t)(bkt[3] & 0xffff) << 48) | o[3].k48);
   }
 }
 
-__device__ __forceinline__ void write_defaults1(const RegroupArgs &a, int64_t i, int bkt) {
-  a.slack[i] = 0;
+__device__ __forceinline__ void write_outputs1(const RegroupArgs &a, int64_t i, int bkt, const RowOut &o) {
+  a.slack[i] = o.slack;
   a.admit[i] = 0;
   if (a.pred_tpot) a.pred_tpot[i] = 0;
-  if (a.key) a.key[i] = ((uint64_t)(bkt & 0xffff) << 48) | dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
+  if (a.key) a.key[i] = ((uint64_t)(bkt & 0xffff) << 48) | o.k48;
 }
 
 // atomic mode: positions from global fill cursors (any order inside a replica's two classes)
@@ -360,9 +375,16 @@ __global__ void __launch_bounds__(256) k_regroup_atomic(const HfxParams p, const
   auto emit = [&](int64_t i, const RowIn &in) {
     HfxRec r;
     const int bkt = bucket_of(in.rid, R);
-    const int mode = bkt < R ? __ldg(a.mode + bkt) : 0;
+    int mode = 0;
+    int64_t start = 0;
+    if (bkt < R) {
+      mode = __ldg(a.mode + bkt);
+      const int64_t now = __ldg(a.now + bkt), mat = __ldg(a.mat + bkt);
+      start = now > mat ? now : mat;
+    }
     make_record(p, s_ttft, s_tpot, s_prio, i, in, mode, r);
-    if (a.pred_ttft) a.pred_ttft[i] = row_pred_ttft(p, a, in, mode);
+    if (a.pred_ttft) a.pred_ttft[i] = row_pred_ttft(p, in, mode, start);
+    write_outputs1(a, i, bkt, row_out(r, mode, start));
     const uint32_t pos = in.kind <= KIND_QUEUED ? seg_begin[bkt] + atomicAdd(&cursor[bkt], 1u)
                                                 : seg_begin[bkt] + tot_act[bkt] + atomicAdd(&cursor[R + 2 + bkt], 1u);
     store_record(rec, pos, r);
@@ -393,12 +415,13 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int R = p.n_replicas, R1 = R + 1, T = ta.tile_rows;
   int64_t *s_fmin = reinterpret_cast<int64_t *>(smem_raw);           // [R1] earliest not-yet-arrived row per replica
-  uint32_t *s_cnt = reinterpret_cast<uint32_t *>(s_fmin + R1);       // [R1]   rows of each replica in the tile / cursors
+  uint32_t *s_cnt = reinterpret_cast<uint32_t *>(s_fmin + 2 * R1);   // [R1]   rows of each replica in the tile / cursors
   uint32_t *s_off = s_cnt + R1;                                      // [R1+1] exclusive prefix of s_cnt / cursors
   uint32_t *s_bact = s_off + R1 + 1;                                 // [R1]   where the tile's active rows of r start
   uint32_t *s_bin = s_bact + R1;                                     // [R1]   where its inactive rows start
   uint16_t *s_stage = reinterpret_cast<uint16_t *>(s_bin + R1);      // [T]    tile rows grouped by replica (+ class bit)
   uint16_t *s_P = s_stage + T;                                       // [T+1]  active rows before each tile position
+  int64_t *s_start = s_fmin + R1;                                    // [R1]   earliest start max(now, maturity)
   uint8_t *s_mode = reinterpret_cast<uint8_t *>(s_P + T + 1);        // [R1]   replica modes
   __shared__ int64_t s_ttft[HFX_MAX_CLASSES], s_tpot[HFX_MAX_CLASSES];
   __shared__ uint8_t s_prio[HFX_MAX_CLASSES];
@@ -411,6 +434,7 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   stage_classes(p, s_ttft, s_tpot, s_prio);
   for (int i = tid; i < R1; i += blockDim.x) {
     s_cnt[i] = 0; s_off[i] = 0; s_mode[i] = i < R ? a.mode[i] : 0;
+    { int64_t st = 0; if (i < R) { const int64_t nw = a.now[i], mt = a.mat[i]; st = nw > mt ? nw : mt; } s_start[i] = st; }
     if (use_fmin) s_fmin[i] = HFX_INF;
   }
   __syncthreads();
@@ -500,7 +524,7 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   __syncthreads();
 
   // ---- D: records of active rows; inactive rows: their outputs (ordered) or their records ----------
-  auto emit = [&](int64_t i, int il, const RowIn &in) {
+  auto emit = [&](int64_t i, int il, const RowIn &in) -> RowOut {
     const int bkt = bucket_of(in.rid, R);
     const bool act = in.kind <= KIND_QUEUED;
     uint32_t rank;
@@ -515,31 +539,35 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
       for (uint32_t g = g0; g < g1; g++) { const uint32_t e = s_stage[g]; rank += ((e ^ me) < 0x8000u && e < me) ? 1u : 0u; }
     } else rank = atomicAdd(act ? &s_cnt[bkt] : &s_off[bkt], 1u);
     const int rmode = s_mode[bkt];
-    if (a.pred_ttft) a.pred_ttft[i] = row_pred_ttft(p, a, in, rmode);
+    const int64_t start = s_start[bkt];
+    if (a.pred_ttft) a.pred_ttft[i] = row_pred_ttft(p, in, rmode, start);
+    RowOut o;
+    o.slack = 0; o.k48 = dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
     if (act || !ordered) {
       HfxRec r;
       make_record(p, s_ttft, s_tpot, s_prio, i, in, rmode, r);
+      o = row_out(r, rmode, start);
       store_record(ta.rec, (act ? s_bact[bkt] : s_bin[bkt]) + rank, r);
     } else {
       a.order[s_bin[bkt] + rank] = (int32_t)i;
       if (use_fmin && in.kind == KIND_FUTURE) atomicMin(reinterpret_cast<long long *>(&s_fmin[bkt]), (long long)in.arrival);
     }
+    return o;
   };
   for (int v = tid; v < nvec; v += blockDim.x) {
     RowIn in[4];
     load_rows4(a, ta.rowflag, v0 + v, in);
-    if (ordered) {
-      const int bk[4] = {bucket_of(in[0].rid, R), bucket_of(in[1].rid, R), bucket_of(in[2].rid, R), bucket_of(in[3].rid, R)};
-      write_defaults4(a, v0 + v, bk);
-    }
+    const int bk[4] = {bucket_of(in[0].rid, R), bucket_of(in[1].rid, R), bucket_of(in[2].rid, R), bucket_of(in[3].rid, R)};
+    RowOut o[4];
 #pragma unroll
-    for (int k = 0; k < 4; k++) emit(lo + 4 * (int64_t)v + k, 4 * v + k, in[k]);
+    for (int k = 0; k < 4; k++) o[k] = emit(lo + 4 * (int64_t)v + k, 4 * v + k, in[k]);
+    write_outputs4(a, v0 + v, bk, o);
   }
   for (int i = (nvec << 2) + tid; i < nt; i += blockDim.x) {
     RowIn in;
     load_row1(a, ta.rowflag, lo + i, in);
-    if (ordered) write_defaults1(a, lo + i, bucket_of(in.rid, R));
-    emit(lo + i, i, in);
+    const RowOut o = emit(lo + i, i, in);
+    write_outputs1(a, lo + i, bucket_of(in.rid, R), o);
   }
   if (use_fmin) {
     __syncthreads();
@@ -552,7 +580,7 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
 // host side
 // ------------------------------------------------------------------------------------------------
 size_t hfx_regroup_smem(int R1, int tile_rows) {
-  return sizeof(int64_t) * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) +
+  return sizeof(int64_t) * 2 * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) +
          (size_t)R1 + 32;
 }
 
@@ -612,7 +640,7 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
 }
 
 int hfx_regroup_configure() {
-  if (cudaFuncSetAttribute(k_regroup, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_regroup, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }

@@ -300,13 +300,6 @@ __device__ __forceinline__ void block_min_arrival(int64_t v, BlockShared &sh) {
   __syncthreads();
 }
 
-// the outputs of an inactive row (when the regroup has not written them already)
-__device__ __forceinline__ void write_inactive_row(const SegArgs &a, int32_t row, int r) {
-  a.slack[row] = 0;
-  a.admit[row] = 0;
-  if (a.pred_tpot) a.pred_tpot[row] = 0;
-  if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | dev_key48(PH_INACTIVE, 63, HFX_SLACK_MAX);
-}
 
 // Block-wide admission over the sorted items s_lo[0..n_sorted) (low 16 bits = position of the
 // record inside the segment): writes order, admit and the compacted admitted list, keeps each
@@ -349,7 +342,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     bool adm = false;
     if (cnt) adm = sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap);
     if (q < n_sorted) {
-      a.admit[row] = (uint8_t)((kind == KIND_RUNNING || adm) ? 1 : 0);
+      if (kind == KIND_RUNNING || adm) a.admit[row] = 1;
       if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
       s_lo[q] = (s_lo[q] & 0xffffu) | (adm ? 0x10000u : 0u);
     }
@@ -401,7 +394,6 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
         const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
         if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); next_arr = arr < next_arr ? arr : next_arr; }
         s_hi[q] = ((uint64_t)(w0.z ^ 0x80000000u) << 16) | (uint32_t)q;     // signed req_id order, then position
-        write_inactive_row(a, (int32_t)w0.w, r);
       }
       __syncthreads();
       if (!(bucket && n_in > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_in, sh))) {
@@ -432,9 +424,11 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
         s_hi[q] = (e.k48 << 16) | (uid >> 16);
         s_lo[q] = (uid << 16) | (uint32_t)q;
       }
-      a.slack[row] = e.slack;
+      if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the regroup wrote the slack of the other queued rows)
+        a.slack[row] = e.slack;
+        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+      }
       if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-      if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
     }
     __syncthreads();
     if (ordered) {
@@ -533,7 +527,6 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
         const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
         if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); next_arr = arr < next_arr ? arr : next_arr; }
         s_key[q] = ((uint64_t)(w0.z ^ 0x80000000u) << 16) | (uint32_t)q;
-        write_inactive_row(a, (int32_t)w0.w, r);
       }
       __syncthreads();
       block_sort<false>(s_key, nullptr, n_in);
@@ -601,9 +594,11 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
           s_key[q] = (e.k48 << 16) | (uid >> 16);
           s_lo[q] = (uid << 16) | (uint32_t)q;
         }
-        a.slack[row] = e.slack;
+        if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the regroup wrote the slack of the other queued rows)
+          a.slack[row] = e.slack;
+          if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+        }
         if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
       }
     }
     bool sorted_done = false;
@@ -714,7 +709,7 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
           adm = run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap);
           if (adm) { ac += cost[k]; ak += kvs[k]; an++; if (a.admitted_rows) a.admitted_rows[b + run_n - 1] = rows[k]; }
         }
-        a.admit[rows[k]] = (uint8_t)((kinds[k] == KIND_RUNNING || adm) ? 1 : 0);
+        if (kinds[k] == KIND_RUNNING || adm) a.admit[rows[k]] = 1;
         s_lo[q] = (s_lo[q] & 0xffffu) | (adm ? 0x10000u : 0u);
       }
     }
@@ -859,7 +854,6 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
       for (int64_t q = gtid; q < n_in; q += gsize) {
         const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
         hi[q] = w0.z ^ 0x80000000u; lo[q] = 0; idx[q] = (uint32_t)q;
-        write_inactive_row(a, (int32_t)w0.w, r);
       }
       if (!grid_barrier(bar, status, epoch)) return;
       if (!grid_sort(hi, lo, idx, n_in, bar, status, epoch)) return;
@@ -883,9 +877,11 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
       hi[q] = e.k48;
       lo[q] = w0.z ^ 0x80000000u;
       idx[q] = (uint32_t)q;
-      a.slack[row] = e.slack;
+      if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the regroup wrote the slack of the other queued rows)
+        a.slack[row] = e.slack;
+        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+      }
       if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-      if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
     }
     if (!grid_barrier(bar, status, epoch)) return;
     if (!grid_sort(hi, lo, idx, n_act, bar, status, epoch)) return;
@@ -925,7 +921,7 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
         bool adm = false;
         if (cnt) adm = sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap);
         if (q < n_act) {
-          a.admit[row] = (uint8_t)((kind == KIND_RUNNING || adm) ? 1 : 0);
+          if (kind == KIND_RUNNING || adm) a.admit[row] = 1;
           if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
           lo[q] = adm ? 1u : 0u;      // the sort is over: lo now carries the decision
         }
