@@ -177,15 +177,16 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       }
       __syncthreads();
 
-      // ---- 2. plan: E_d of the running batch and the safe budget (one thread) -------------
-      if (tid == 0) {
-        S.head += S.arrived;
-        uint64_t m_run = 0, m_q = 0;
-        for (int c = 0; c < p.n_classes; c++) {
-          if (S.cnt_run[c] > 0) m_run |= 1ull << c;
-          if (S.cnt_q[c] > 0) m_q |= 1ull << c;
-        }
-        dev_plan(p, cfg, S.now, S.mat, S.nr, S.sum_kv, m_run, m_q, S.plan);
+      // ---- 2. plan: E_d of the running batch and the safe budget (the first warp) ----------------
+      if (warp == 0) {
+        if (lane == 0) S.head += S.arrived;
+        const uint32_t r0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_run[lane] > 0);
+        const uint32_t r1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && S.cnt_run[lane + 32] > 0);
+        const uint32_t q0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_q[lane] > 0);
+        const uint32_t q1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && S.cnt_q[lane + 32] > 0);
+        ReplicaPlan pl0;
+        warp_plan(p, cfg, S.now, S.mat, S.nr, S.sum_kv, ((uint64_t)r1 << 32) | r0, ((uint64_t)q1 << 32) | q0, pl0, lane);
+        if (lane == 0) S.plan = pl0;
       }
       __syncthreads();
       const int64_t budget = S.plan.budget, start = S.plan.start;
