@@ -235,29 +235,31 @@ __device__ inline void warp_plan(const HfxParams &p, const hfx_replica_cfg &cfg,
   pl.mode = cfg.mode; pl.token_cap = cfg.token_cap; pl.batch_cap = cfg.batch_cap;
   pl.n_run = n_run; pl.sum_kv = sum_kv;
   const int64_t min_tpot = warp_min_over_mask(p.tpot, mask_run, lane);
-  const int64_t min_ttft = warp_min_over_mask(p.ttft, mask_q, lane);
-  const int64_t min_tpot_q = warp_min_over_mask(p.tpot, mask_q, lane);
   const bool prefill = cfg.mode == HFX_PREFILL;
   pl.n_eff = prefill ? 0 : n_run;
   pl.kv_eff = prefill ? 0 : sum_kv;
   pl.tpot_eff = prefill ? HFX_INF : min_tpot;
   pl.e_d = pl.n_eff > 0 ? dev_Ed(p, pl.n_eff, pl.kv_eff) : 0;
-  int64_t budget;
-  if (cfg.mode == HFX_DECODE) {
-    const int64_t T = (n_run > 0 && min_tpot < HFX_INF) ? min_tpot : min_tpot_q;
-    if (p.budget_mode == HFX_BUDGET_CAP_ONLY || T == HFX_INF) budget = HFX_INF;
-    else {
-      const int64_t room = T - dev_Ed(p, n_run, sum_kv);
-      budget = room > 0 ? room : 0;
+  int64_t budget = 0;
+  if (now >= mat) {      // before maturity the instance is protected: no budget to work out
+    if (cfg.mode == HFX_DECODE) {
+      const int64_t T = (n_run > 0 && min_tpot < HFX_INF) ? min_tpot : warp_min_over_mask(p.tpot, mask_q, lane);
+      if (p.budget_mode == HFX_BUDGET_CAP_ONLY || T == HFX_INF) budget = HFX_INF;
+      else {
+        const int64_t room = T - dev_Ed(p, n_run, sum_kv);
+        budget = room > 0 ? room : 0;
+      }
+    } else {
+      const int64_t cap_left = cfg.token_cap - pl.n_eff > 0 ? cfg.token_cap - pl.n_eff : 0;
+      int64_t n_safe;
+      if (p.budget_mode == HFX_BUDGET_CAP_ONLY) n_safe = cfg.token_cap;
+      else {
+        const int64_t min_ttft = warp_min_over_mask(p.ttft, mask_q, lane);
+        n_safe = warp_nsafe(p, dev_epmax(min_ttft, pl.n_eff > 0 && pl.tpot_eff < HFX_INF, pl.tpot_eff, pl.e_d), cfg.token_cap, lane);
+      }
+      budget = n_safe < cap_left ? n_safe : cap_left;
     }
-  } else {
-    const int64_t cap_left = cfg.token_cap - pl.n_eff > 0 ? cfg.token_cap - pl.n_eff : 0;
-    int64_t n_safe;
-    if (p.budget_mode == HFX_BUDGET_CAP_ONLY) n_safe = cfg.token_cap;
-    else n_safe = warp_nsafe(p, dev_epmax(min_ttft, pl.n_eff > 0 && pl.tpot_eff < HFX_INF, pl.tpot_eff, pl.e_d), cfg.token_cap, lane);
-    budget = n_safe < cap_left ? n_safe : cap_left;
   }
-  if (now < mat) budget = 0;
   pl.budget = budget;
   pl.tpot_q0 = dev_Ed(p, pl.n_eff + 1, pl.kv_eff);
   pl.shift_run = now + pl.e_d;
