@@ -205,8 +205,8 @@ typedef struct hfx_sim_out {
 
 /* Create a scheduler.  `model`, `classes[n_classes]`, `replicas[n_replicas]`
  * and `opts` are host pointers, copied.  `max_rows` bounds n_rows of later
- * calls and sizes the workspace (about 40 bytes per row plus 64 bytes per
- * replica of device memory).  `cuda_stream` is a cudaStream_t (NULL = the
+ * calls and sizes the workspace (about 50 bytes per row of device memory, plus
+ * per-replica tables of a few KB per replica for up to 4095 replicas).  `cuda_stream` is a cudaStream_t (NULL = the
  * default stream).  Errors: HFX_E_ARG (NULL pointer, value outside the domain
  * above), HFX_E_CUDA, HFX_E_NOMEM.  On error *out is NULL. */
 int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
