@@ -17,6 +17,7 @@
 #include "hfx_internal.cuh"
 
 #define THREADS_TILE 512
+#define COLSCAN_REG 16
 #define GROUP_MAX 64      // largest same-replica group of an unsorted tile that is ranked by scanning
 
 __device__ __forceinline__ int bucket_of(int rid, int R) { return (rid < 0 || rid >= R) ? R : rid; }
@@ -207,20 +208,38 @@ __global__ void __launch_bounds__(1024) k_colscan(uint32_t *__restrict__ M, int3
   const int cb = (n_tiles + 31) / 32;
   const int t0 = w * cb < n_tiles ? w * cb : n_tiles;
   const int t1 = (t0 + cb < n_tiles) ? t0 + cb : n_tiles;
+  // Up to COLSCAN_REG tiles per thread are held in registers (independent loads, one pass);
+  // longer chunks take the two-pass loop.
+  uint32_t v[COLSCAN_REG];
+  const bool in_regs = cb <= COLSCAN_REG;
   uint32_t sum = 0;
-  if (col < C)
-    for (int t = t0; t < t1; t++) sum += M[(size_t)t * C + col];
+  if (col < C) {
+    if (in_regs) {
+#pragma unroll
+      for (int k = 0; k < COLSCAN_REG; k++) v[k] = t0 + k < t1 ? M[(size_t)(t0 + k) * C + col] : 0u;
+#pragma unroll
+      for (int k = 0; k < COLSCAN_REG; k++) sum += v[k];
+    } else {
+      for (int t = t0; t < t1; t++) sum += M[(size_t)t * C + col];
+    }
+  }
   part[w][lane] = sum;
   __syncthreads();
   uint32_t pre = 0;
   for (int k = 0; k < w; k++) pre += part[k][lane];
   if (col < C) {
     uint32_t run = pre;
-    for (int t = t0; t < t1; t++) {
-      const size_t idx = (size_t)t * C + col;
-      const uint32_t v = M[idx];
-      M[idx] = run;
-      run += v;
+    if (in_regs) {
+#pragma unroll
+      for (int k = 0; k < COLSCAN_REG; k++)
+        if (t0 + k < t1) { M[(size_t)(t0 + k) * C + col] = run; run += v[k]; }
+    } else {
+      for (int t = t0; t < t1; t++) {
+        const size_t idx = (size_t)t * C + col;
+        const uint32_t x = M[idx];
+        M[idx] = run;
+        run += x;
+      }
     }
     if (w == 31) { if (col < R1) tot_all[col] = pre + sum; else tot_act[col - R1] = pre + sum; }
   }
