@@ -55,6 +55,16 @@ def test_config5_subset_of_traces():
     assert_sim_parity(wl)
 
 
+def test_config5_full_batch_sampled_traces():
+    # the whole 4096-trace batch in one call (the launch the benchmark times); four traces spread over
+    # the batch are checked against the oracle, the rest through properties that hold for every trace
+    wl = gen.config5()
+    res = assert_sim_parity(wl, traces=[0, 1365, 2730, 4095])
+    assert np.all(res["iters_executed"] <= wl.sim_iters) and np.all(res["iters_executed"] > 0)
+    assert np.all(res["attained"] <= res["finished"]) and np.all(res["finished"] + res["rejected"] <= 2048)
+    assert np.all(res["ttft_p50_ns"] <= res["ttft_p99_ns"]) and np.all(res["tpot_p50_ns"] <= res["tpot_p99_ns"])
+
+
 # ---- random and adversarial step cases -----------------------------------------------------------
 @pytest.mark.parametrize("seed", range(16))
 def test_random_tables(seed):
