@@ -196,7 +196,7 @@ extern "C" int hfx_sim_run(hfx_sched *s, const hfx_table *t, const int32_t *trac
                            const hfx_sim_out *o) {
   if (!s || !t || !trace_off || !o) return HFX_E_ARG;
   hfx_sched_host *h = reinterpret_cast<hfx_sched_host *>(s);
-  if (n_traces < 0 || iters < 0) return HFX_E_ARG;
+  if (n_traces < 0 || iters < 0 || iters > (1 << 29)) return HFX_E_ARG;
   if (n_traces > s->p.n_replicas) return HFX_E_CAPACITY;
   const void *need[] = {t->class_id, t->state, t->prompt_len, t->output_len, t->gen, t->arrival_ns, t->first_token_ns,
                         t->last_token_ns, t->finish_ns, t->req_id, o->iters_executed, o->finished, o->rejected,

@@ -16,7 +16,8 @@
 #define SIM_THREADS 128
 #define SIM_WARPS (SIM_THREADS / 32)
 #define SIM_MAX_ROWS 4096
-#define SIM_BYTES_PER_ROW 44
+#define SIM_BYTES_PER_ROW 28
+#define SIM_OUTLEN_CAP (1 << 30)   // output lengths are clamped here when the finish iteration is formed
 
 #define ROW_INVALID 0xff
 
@@ -45,6 +46,7 @@ struct SimShared {
   int32_t best_slot[2][SIM_WARPS];
   // end-of-trace counters
   int32_t n_fin, n_rej, n_att, n_a, n_b;
+  int64_t ttft[HFX_MAX_CLASSES];   // TTFT SLO per class
 };
 
 __device__ __forceinline__ void sort_i64(int64_t *v, int n) {
@@ -80,13 +82,10 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
                                                      uint32_t *__restrict__ status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int cap = a.cap_rows;
-  int64_t *s_arr = reinterpret_cast<int64_t *>(smem_raw);              // arrival; later TTFT samples
-  int64_t *s_dst = s_arr + cap;                                        // ttft_slo + arrival - E_p(prompt); later TPOT samples
-  int32_t *s_prompt = reinterpret_cast<int32_t *>(s_dst + cap);
-  int32_t *s_outlen = s_prompt + cap;
-  int32_t *s_admit_it = s_outlen + cap;
-  uint32_t *s_reqid = reinterpret_cast<uint32_t *>(s_admit_it + cap);
-  uint16_t *s_q = reinterpret_cast<uint16_t *>(s_reqid + cap);         // visible queue (row indices, unordered)
+  int64_t *s_arr = reinterpret_cast<int64_t *>(smem_raw);              // arrival; later the TTFT, then the TPOT samples
+  int32_t *s_prompt = reinterpret_cast<int32_t *>(s_arr + cap);
+  int32_t *s_fin = s_prompt + cap;                                     // iteration at which a running row emits its last token
+  uint16_t *s_q = reinterpret_cast<uint16_t *>(s_fin + cap);           // visible queue (row indices, unordered)
   uint16_t *s_run = s_q + cap;                                         // running batch, ping
   uint16_t *s_run2 = s_run + cap;                                      // running batch, pong
   uint16_t *s_adm = s_run2 + cap;                                      // admitted this iteration; oversize rows from the top
@@ -112,7 +111,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       S.n_fin = 0; S.n_rej = 0; S.n_att = 0; S.n_a = 0; S.n_b = 0; S.zero_prompt = 0;
     }
     __syncthreads();
-    for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; }
+    for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; S.ttft[c] = c < p.n_classes ? p.ttft[c] : 0; }
     uint32_t bad = 0;
     for (int i = tid; i < m; i += SIM_THREADS) {
       const int64_t g = (int64_t)b + i;
@@ -125,23 +124,17 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       s_arr[i] = arr;
       s_prompt[i] = prompt;
       if (prompt == 0) S.zero_prompt = 1;   // a zero-token prompt fits a zero budget
-      s_outlen[i] = a.output_len[g];
-      s_reqid[i] = (uint32_t)a.req_id[g] ^ 0x80000000u;
-      s_admit_it[i] = -1;
+      s_fin[i] = -1;
       s_cls[i] = ok ? (uint8_t)cls : ROW_INVALID;
       s_state[i] = HFX_QUEUED;
       int prio = 63;
-      int64_t d = BASE_UNBOUNDED;
       if (ok) {
         if (p.weight_max > 0) {
           const int64_t w = (int64_t)p.weight_max - a.weight[g];
           prio = (int)(w < 0 ? 0 : (w > 62 ? 62 : w));
         } else prio = p.prio[cls];
-        const int64_t ttft = p.ttft[cls];
-        if (ttft > 0) d = ttft + arr - dev_Ep(p, prompt);
       }
       s_prio[i] = (uint8_t)prio;
-      s_dst[i] = d;
       a.first_token[g] = -1; a.last_token[g] = -1; a.finish[g] = -1;
     }
     if (bad) atomicOr(status, bad);
@@ -203,17 +196,26 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           for (int s = tid; s < nq; s += SIM_THREADS) {
             const int i = s_q[s];
             if ((int64_t)s_prompt[i] > budget) continue;
-            const int64_t d = s_dst[i];
-            const int64_t sl = d == BASE_UNBOUNDED ? HFX_SLACK_MAX : dev_clamp_slack(d - start);
+            // slack of a queued request: ttft_slo - (start - arrival) - E_p(prompt_len)
+            const int64_t ttft = S.ttft[s_cls[i]];
+            const int64_t sl = ttft > 0 ? dev_clamp_slack(ttft + s_arr[i] - dev_Ep(p, s_prompt[i]) - start) : HFX_SLACK_MAX;
             const uint64_t k = ((uint64_t)s_prio[i] << 40) | (uint64_t)(sl + (INT64_C(1) << 39));
-            const uint32_t id = s_reqid[i];
-            if (k < bk || (k == bk && id < bid)) { bk = k; bid = id; bslot = s; }
+            if (k < bk) { bk = k; bslot = s; bid = ~0u; }
+            else if (k == bk) {      // equal keys are rare: only then fetch the request ids that break the tie
+              if (bid == ~0u) bid = (uint32_t)__ldg(a.req_id + b + s_q[bslot]) ^ 0x80000000u;
+              const uint32_t id = (uint32_t)__ldg(a.req_id + b + i) ^ 0x80000000u;
+              if (id < bid) { bid = id; bslot = s; }
+            }
           }
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) {
             const uint64_t k2 = __shfl_xor_sync(0xffffffffu, bk, o);
-            const uint32_t i2 = __shfl_xor_sync(0xffffffffu, bid, o);
+            uint32_t i2 = __shfl_xor_sync(0xffffffffu, bid, o);
             const int s2 = __shfl_xor_sync(0xffffffffu, bslot, o);
+            if (k2 == bk && bslot >= 0 && s2 >= 0 && s2 != bslot) {
+              if (bid == ~0u) bid = (uint32_t)__ldg(a.req_id + b + s_q[bslot]) ^ 0x80000000u;
+              if (i2 == ~0u) i2 = (uint32_t)__ldg(a.req_id + b + s_q[s2]) ^ 0x80000000u;
+            }
             if (k2 < bk || (k2 == bk && i2 < bid)) { bk = k2; bid = i2; bslot = s2; }
           }
           if (lane == 0) { S.best_key[buf][warp] = bk; S.best_id[buf][warp] = bid; S.best_slot[buf][warp] = bslot; }
@@ -221,8 +223,13 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           bk = S.best_key[buf][0]; bid = S.best_id[buf][0]; bslot = S.best_slot[buf][0];
 #pragma unroll
           for (int w = 1; w < SIM_WARPS; w++) {
-            const uint64_t k2 = S.best_key[buf][w]; const uint32_t i2 = S.best_id[buf][w];
-            if (k2 < bk || (k2 == bk && i2 < bid)) { bk = k2; bid = i2; bslot = S.best_slot[buf][w]; }
+            const uint64_t k2 = S.best_key[buf][w]; uint32_t i2 = S.best_id[buf][w];
+            const int s2 = S.best_slot[buf][w];
+            if (k2 == bk && bslot >= 0 && s2 >= 0) {
+              if (bid == ~0u) bid = (uint32_t)__ldg(a.req_id + b + s_q[bslot]) ^ 0x80000000u;
+              if (i2 == ~0u) i2 = (uint32_t)__ldg(a.req_id + b + s_q[s2]) ^ 0x80000000u;
+            }
+            if (k2 < bk || (k2 == bk && i2 < bid)) { bk = k2; bid = i2; bslot = s2; }
           }
           buf ^= 1;
           if (bslot < 0) break;                       // no eligible request left
@@ -254,12 +261,12 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       // running batch: one more token each; a request finishes when gen + 1 reaches output_len
       for (int s = tid; s < nr; s += SIM_THREADS) {
         const int i = run_cur[s];
-        const int gen_new = it - s_admit_it[i];
-        if ((int64_t)gen_new + 1 >= s_outlen[i]) {
+        if (it >= s_fin[i]) {       // gen + 1 reaches output_len in this iteration
           s_state[i] = HFX_DONE;
           a.finish[(int64_t)b + i] = t2;
           atomicSub(&S.cnt_run[s_cls[i]], 1);
-          d_kv -= (int64_t)s_prompt[i] + gen_new - 1;     // leaves with the context it had before this step
+          const int32_t outlen = __ldg(a.output_len + b + i);
+          d_kv -= (int64_t)s_prompt[i] + outlen - 2;       // leaves with the context it had before this step
         } else {
           run_nxt[atomicAdd(&S.nr_next, 1)] = (uint16_t)i;
           d_kv += 1;
@@ -269,9 +276,10 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       for (int s = tid; s < adm_cnt; s += SIM_THREADS) {
         const int i = s_adm[s];
         a.first_token[(int64_t)b + i] = t1;
-        s_admit_it[i] = it;
+        const int32_t outlen = __ldg(a.output_len + b + i);
+        s_fin[i] = it + (outlen < SIM_OUTLEN_CAP ? outlen : SIM_OUTLEN_CAP) - 1;
         atomicSub(&S.cnt_q[s_cls[i]], 1);
-        if (s_outlen[i] <= 1) {
+        if (outlen <= 1) {
           s_state[i] = HFX_DONE;
           a.finish[(int64_t)b + i] = t1;
         } else {
@@ -320,56 +328,70 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     for (int i = tid; i < m; i += SIM_THREADS) {
       const int64_t g = (int64_t)b + i;
       const int st = s_state[i];
+      const int32_t outlen = a.output_len[g];
       int32_t gen = 0;
       int64_t first = -1, last = -1;
       if (st == HFX_RUNNING || st == HFX_DONE) {
         first = a.first_token[g];
-        if (st == HFX_DONE) { gen = s_outlen[i] > 1 ? s_outlen[i] - 1 : 0; last = a.finish[g]; }
-        else { gen = executed - 1 - s_admit_it[i]; last = gen > 0 ? now_final : first; }
+        if (st == HFX_DONE) { gen = outlen > 1 ? outlen - 1 : 0; last = a.finish[g]; }
+        else {
+          const int admit_it = s_fin[i] - (outlen < SIM_OUTLEN_CAP ? outlen : SIM_OUTLEN_CAP) + 1;
+          gen = executed - 1 - admit_it;
+          last = gen > 0 ? now_final : first;
+        }
         a.last_token[g] = last;
       }
       a.state[g] = (uint8_t)st;
       a.gen[g] = gen;
       const int64_t arr = s_arr[i];
       const uint8_t cls = s_cls[i];
-      int64_t ttft = -1, tpot = -1;
+      int64_t ttft = -1;
       if (cls != ROW_INVALID) {
         if (st == HFX_REJECTED) rej++;
         if (st == HFX_RUNNING || st == HFX_DONE) ttft = first - arr;
         if (st == HFX_DONE) {
           fin++;
-          const int64_t tp = s_outlen[i] > 1 ? (last - first) / (s_outlen[i] - 1) : 0;
-          if (s_outlen[i] > 1) tpot = tp;
+          const int64_t tp = outlen > 1 ? (last - first) / (outlen - 1) : 0;
           const int64_t ttft_slo = p.ttft[cls], tpot_slo = p.tpot[cls];
           if ((ttft_slo <= 0 || ttft <= ttft_slo) && (tpot_slo <= 0 || tp <= tpot_slo)) att++;
         }
       }
-      // park the samples; compaction follows
-      s_arr[i] = ttft;
-      s_dst[i] = tpot;
+      s_arr[i] = ttft;     // park the TTFT sample; negative = none
     }
     fin = (int)warp_sum_i64(fin); rej = (int)warp_sum_i64(rej); att = (int)warp_sum_i64(att);
     if (lane == 0) { atomicAdd(&S.n_fin, fin); atomicAdd(&S.n_rej, rej); atomicAdd(&S.n_att, att); }
     __syncthreads();
-    // compact the samples (order is irrelevant before the sort): negative = no sample.
-    // In-place compaction by one warp-synchronous pass per array would need care; the arrays are
-    // small, so let thread 0 of each of two warps do it serially.
+    // Compact the samples (their order is irrelevant before the sort), sort, take the ranks; then the
+    // same array takes the TPOT samples.  The arrays are small: one thread compacts serially.
     if (tid == 0) { int k = 0; for (int i = 0; i < m; i++) { const int64_t v = s_arr[i]; if (v >= 0) s_arr[k++] = v; } S.n_a = k; }
-    if (tid == 32) { int k = 0; for (int i = 0; i < m; i++) { const int64_t v = s_dst[i]; if (v >= 0) s_dst[k++] = v; } S.n_b = k; }
     __syncthreads();
-    const int na = S.n_a, nb = S.n_b;
+    const int na = S.n_a;
     sort_i64(s_arr, na);
-    sort_i64(s_dst, nb);
+    if (tid == 0) { S.t1 = nearest_rank(s_arr, na, 50); S.t2 = nearest_rank(s_arr, na, 99); }
     __syncthreads();
+    for (int i = tid; i < m; i += SIM_THREADS) {
+      const int64_t g = (int64_t)b + i;
+      int64_t tpot = -1;
+      if (s_state[i] == HFX_DONE && s_cls[i] != ROW_INVALID) {
+        const int32_t outlen = a.output_len[g];
+        if (outlen > 1) tpot = (a.finish[g] - a.first_token[g]) / (outlen - 1);
+      }
+      s_arr[i] = tpot;
+    }
+    __syncthreads();
+    if (tid == 0) { int k = 0; for (int i = 0; i < m; i++) { const int64_t v = s_arr[i]; if (v >= 0) s_arr[k++] = v; } S.n_b = k; }
+    __syncthreads();
+    const int nb = S.n_b;
+    sort_i64(s_arr, nb);
     if (tid == 0) {
       a.iters_executed[j] = executed;
       a.finished[j] = S.n_fin;
       a.rejected[j] = S.n_rej;
       a.attained[j] = S.n_att;
-      a.ttft_p50[j] = nearest_rank(s_arr, na, 50);
-      a.ttft_p99[j] = nearest_rank(s_arr, na, 99);
-      a.tpot_p50[j] = nearest_rank(s_dst, nb, 50);
-      a.tpot_p99[j] = nearest_rank(s_dst, nb, 99);
+      a.ttft_p50[j] = S.t1;
+      a.ttft_p99[j] = S.t2;
+      a.tpot_p50[j] = nearest_rank(s_arr, nb, 50);
+      a.tpot_p99[j] = nearest_rank(s_arr, nb, 99);
       if (a.now_out) a.now_out[j] = now_final;
     }
   }
@@ -399,7 +421,7 @@ int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_tra
   a.now_out = o->now_ns;
   const size_t smem = (size_t)cap * SIM_BYTES_PER_ROW;
   if (cudaMemsetAsync(d_work_counter, 0, sizeof(uint32_t), s->stream) != cudaSuccess) return HFX_E_CUDA;
-  int per_sm = (int)((200 * 1024) / (smem + 2048));
+  int per_sm = (int)((224 * 1024) / (smem + 2560));
   if (per_sm < 1) per_sm = 1;
   if (per_sm > 8) per_sm = 8;
   int grid = s->n_sm * per_sm;
