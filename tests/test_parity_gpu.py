@@ -108,6 +108,42 @@ def test_many_replicas_atomic_regroup_and_natural_ids():
     assert_step_parity(wl)
 
 
+@pytest.mark.parametrize("R", [4095, 4096])
+def test_replica_count_at_the_counter_limit(R):
+    # 4095 replicas still use the tile histograms, 4096 the global counters
+    for ids in (True, False):
+        wl = gen.random_table(60 + R % 7, 60_000, R, modes=MODES3, permute_ids=ids)
+        assert_step_parity(wl, steps=2, commit=True)
+
+
+@pytest.mark.parametrize("n", [1023, 1024, 1025, 296 * 1024 - 1, 296 * 1024, 296 * 1024 + 5])
+def test_sizes_at_tile_boundaries(n):
+    wl = gen.config4(seed=n % 100, R=64, n=n, steps=2)
+    assert_step_parity(wl, steps=2, commit=True, optional=n < 5000)
+
+
+def test_scheduler_on_its_own_stream():
+    import paper_2508_15919_b200 as hfx
+    wl = gen.config4(seed=77, R=32, n=30_000, steps=3)
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        sched = hfx.Scheduler(wl.model, wl.classes, wl.replicas, wl.n_rows, budget_mode=wl.budget_mode,
+                              weight_max=wl.weight_max, stream=st)
+        assert_step_parity(wl, steps=3, commit=True, sched=sched)
+        sched.close()
+    st.synchronize()
+
+
+def test_two_schedulers_interleaved():
+    a = gen.config4(seed=78, R=16, n=20_000, steps=2)
+    b = gen.random_table(79, 5000, 7, modes=MODES3)
+    sa, sb = make_sched(a), make_sched(b)
+    assert_step_parity(a, steps=1, commit=True, sched=sa)
+    assert_step_parity(b, steps=2, commit=True, sched=sb)
+    assert_step_parity(a, steps=2, commit=True, sched=sa)
+    sa.close(); sb.close()
+
+
 def test_empty_replicas_and_all_inactive():
     wl = gen.random_table(11, 500, 40)
     wl.table["replica_id"][:] = wl.table["replica_id"] % 3 * 13        # most replicas have no rows
