@@ -14,8 +14,8 @@
  * file.  It shares no code, header, table or constant with the CUDA library.
  *
  * Parity status: the arithmetic below is pinned by hand-worked values, the
- * closed form of Eq. 3 in exact rationals, invariants, brute force on tiny
- * inputs and a pure-Python restatement (tests/test_oracle_*.py).  Against the
+ * closed form of Eq. 3 in exact rationals, closed forms of the simulator,
+ * invariants and brute force on tiny inputs (tests/test_oracle_*.py).  Against the
  * behaviour of the paper's own system it is "parity unpinned": the paper
  * prints no scheduler trace or worked numeric example.
  */
