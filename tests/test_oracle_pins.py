@@ -244,3 +244,43 @@ def test_oversize_prompt_rejected_on_commit_and_bad_rows_flagged():
     assert list(wl.table["state"]) == [gen.REJECTED, gen.RUNNING, gen.QUEUED, gen.QUEUED, gen.QUEUED]
     assert list(o["seg_off"]) == [0, 4] and o["order"][4] == 4
     assert list(o["admit"]) == [0, 1, 0, 0, 0]
+
+
+def test_commit_of_the_disaggregated_stages_hand_worked():
+    cls = [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)]
+    # D-stage: the enlarged batch advances one token; t2 = now + E_d(2, 1000 + 2000)
+    rows = [dict(state=gen.RUNNING, prompt_len=900, gen=100, first_token_ns=0, class_id=1, req_id=9, output_len=102),
+            dict(prompt_len=500, gen=0, first_token_ns=0, class_id=0, req_id=1, output_len=5),
+            dict(prompt_len=2000, gen=0, first_token_ns=0, class_id=0, req_id=2, output_len=5)]
+    wl = make_wl(rows, cls, replicas=[(gen.DECODE, 32768, 2)], now=[MS])
+    oracle.step(wl, commit=True)
+    t2 = MS + 8_000_000 + 2 * 100_000 + 20 * 3000
+    t = wl.table
+    assert list(t["state"]) == [gen.DONE, gen.QUEUED, gen.RUNNING]
+    assert list(t["gen"]) == [101, 0, 1] and t["finish_ns"][0] == t2
+    assert t["last_token_ns"][0] == t2 and t["last_token_ns"][2] == t2 and t["first_token_ns"][2] == 0
+    assert wl.now[0] == t2 and wl.maturity[0] == t2
+    # P-stage: the admitted batch completes at t1 = now + E_p(200); the instance does not decode
+    rows = [dict(state=gen.RUNNING, prompt_len=4000, gen=3, first_token_ns=0, class_id=0, req_id=9, output_len=50),
+            dict(prompt_len=100, class_id=1, req_id=1, output_len=1), dict(prompt_len=100, class_id=0, req_id=2, output_len=3)]
+    wl = make_wl(rows, cls, replicas=[(gen.PREFILL, 32768, 0)], now=[MS])
+    oracle.step(wl, commit=True)
+    t1 = MS + 5_000_000 + 40_000 * 200 + 2 * 200 * 200
+    t = wl.table
+    assert list(t["state"]) == [gen.RUNNING, gen.DONE, gen.RUNNING] and list(t["gen"]) == [3, 0, 0]
+    assert t["finish_ns"][1] == t1 and t["first_token_ns"][2] == t1 and t["last_token_ns"][2] == t1
+    assert wl.now[0] == t1 and wl.maturity[0] == t1
+
+
+def test_idle_replica_jumps_to_its_next_event():
+    rows = [dict(prompt_len=10, arrival_ns=900 * MS, req_id=0), dict(prompt_len=10, arrival_ns=700 * MS, req_id=1),
+            dict(prompt_len=10, arrival_ns=100 * MS, req_id=2, state=gen.DONE)]
+    wl = make_wl(rows, C200, now=[500 * MS], maturity=[0])
+    o = oracle.step(wl, commit=True)
+    assert wl.now[0] == 700 * MS and o["adm_count"][0] == 0 and list(wl.table["state"]) == [0, 0, gen.DONE]
+    wl = make_wl(rows, C200, now=[500 * MS], maturity=[600 * MS])
+    oracle.step(wl, commit=True)
+    assert wl.now[0] == 600 * MS and wl.maturity[0] == 600 * MS
+    wl = make_wl(rows[2:], C200, now=[500 * MS], maturity=[0])       # nothing left to happen: the clock stays
+    oracle.step(wl, commit=True)
+    assert wl.now[0] == 500 * MS
