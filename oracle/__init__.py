@@ -83,6 +83,21 @@ class _SimOut(C.Structure):
     _fields_ = [(k, C.c_void_p) for k, _ in _SIM_OUT]
 
 
+class _ScaleParams(C.Structure):
+    _fields_ = [("window", C.c_int64), ("block_tokens", C.c_int32), ("min_samples", C.c_int32),
+                ("eps_out_num", C.c_int32), ("eps_out_den", C.c_int32), ("eps_in_num", C.c_int32),
+                ("eps_in_den", C.c_int32), ("eps_wait_num", C.c_int32), ("eps_wait_den", C.c_int32)]
+
+
+class _ScaleOut(C.Structure):
+    _fields_ = [("counts", C.c_void_p), ("used_blocks", C.c_void_p), ("decision", C.c_void_p)]
+
+
+# defaults of the paper: 10 s window, eps_out 0.7, eps_in 1.1, eps_wait 1/4
+SCALE_DEFAULTS = dict(window=10_000_000_000, block_tokens=16, min_samples=10, eps_out=(7, 10), eps_in=(11, 10),
+                      eps_wait=(1, 4))
+
+
 def lib():
     global _lib
     if _lib is None:
@@ -103,6 +118,9 @@ def lib():
         L.ora_sim.restype = C.c_uint32
         L.ora_sim.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p, C.c_int32, C.c_int32,
                               C.c_int32, C.POINTER(_SimOut)]
+        L.ora_scale.restype = C.c_uint32
+        L.ora_scale.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_ScaleParams),
+                                C.POINTER(_ScaleOut)]
         _lib = L
     return _lib
 
@@ -185,4 +203,19 @@ def sim(wl, iters: Optional[int] = None, j0: int = 0, j1: Optional[int] = None) 
     st = L.ora_sim(C.byref(ctx.cfg), C.byref(ctx.table), off.ctypes.data, j0, j1,
                    int(wl.sim_iters if iters is None else iters), C.byref(so))
     out["status"] = int(st)
+    return out
+
+
+def scale_tick(wl, now: int, total_blocks: np.ndarray, **kw) -> Dict[str, np.ndarray]:
+    """Scaling indicators f1, f2, f3 and the threshold decision per pool at time `now`."""
+    L = lib()
+    ctx = _Ctx(wl)
+    prm = dict(SCALE_DEFAULTS); prm.update(kw)
+    sp = _ScaleParams(int(prm["window"]), int(prm["block_tokens"]), int(prm["min_samples"]), *prm["eps_out"],
+                      *prm["eps_in"], *prm["eps_wait"])
+    out = {"counts": np.zeros((3, 4), np.int64), "used_blocks": np.zeros(wl.n_replicas, np.int64),
+           "decision": np.zeros((3, 2), np.int32)}
+    so = _ScaleOut(out["counts"].ctypes.data, out["used_blocks"].ctypes.data, out["decision"].ctypes.data)
+    tb = np.ascontiguousarray(total_blocks, np.int32)
+    out["status"] = int(L.ora_scale(C.byref(ctx.cfg), C.byref(ctx.table), int(now), tb.ctypes.data, C.byref(sp), C.byref(so)))
     return out

@@ -557,3 +557,78 @@ uint32_t ora_sim(const ora_config *c, const ora_table *t, const int32_t *trace_o
   free(o.maturity_next);
   return status;
 }
+
+/* ---- scaling indicators and the threshold policy (Sec. 3.3.3 "Scaling Mechanism and Policy") -------
+ * At a tick at time `now` the Scaler computes, per pool of instances (colocated, prefill, decode; the
+ * paper evaluates the stages of the disaggregated mode independently):
+ *   f1 = lambda_out / lambda_in over the window (now - W, now]: arrivals in and completions in the
+ *        window (the window length cancels); used only once enough arrivals were seen;
+ *   f2 = (1/N) * sum over queued requests of waiting_time / SLO;
+ *   f3 = used_blocks / total_blocks per instance: KV blocks of in-flight requests plus blocks
+ *        reserved for the requests waiting in the instance's queue.
+ * f1 < eps_out or f2 > eps_wait -> scale out; else f1 > eps_in with more than one active instance ->
+ * scale in, removing the instance with the smallest f3.
+ * reading: waiting time is measured against the TTFT SLO, requests without one are left out of N;
+ * each ratio waiting/SLO is taken in 16.16 fixed point (floor), saturated at 2^15; thresholds are
+ * rationals num/den compared by cross-multiplication; an instance with total_blocks <= 0 is not
+ * active; ties for the smallest f3 go to the lowest instance id. */
+typedef struct {
+  int64_t window;
+  int32_t block_tokens, min_samples;
+  int32_t eps_out_num, eps_out_den, eps_in_num, eps_in_den, eps_wait_num, eps_wait_den;
+} ora_scale_params;
+
+typedef struct {
+  int64_t *counts;       /* [3][4]: per pool n_in, n_out, n_queue, sum of waiting/SLO in 16.16 */
+  int64_t *used_blocks;  /* [R] */
+  int32_t *decision;     /* [3][2]: per pool action (+1 out, -1 in, 0 hold), instance to remove or -1 */
+} ora_scale_out;
+
+uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const int32_t *total_blocks,
+                   const ora_scale_params *sp, const ora_scale_out *o) {
+  const int32_t R = c->n_replicas;
+  uint32_t status = 0;
+  for (int k = 0; k < 12; k++) o->counts[k] = 0;
+  for (int32_t r = 0; r < R; r++) o->used_blocks[r] = 0;
+  const int64_t B = sp->block_tokens;
+  for (int64_t i = 0; i < t->n; i++) {
+    const int32_t r = t->replica_id[i];
+    if (r < 0 || r >= R) { status |= BAD_REPLICA; continue; }
+    if (!row_valid(c, t, i, &status)) continue;
+    int64_t *cnt = o->counts + 4 * c->replicas[r].mode;
+    const ora_class *k = &c->classes[t->class_id[i]];
+    if (t->arrival[i] > now - sp->window && t->arrival[i] <= now) cnt[0] += 1;               /* enqueued in the window */
+    if (t->state[i] == ST_DONE && t->finish[i] > now - sp->window && t->finish[i] <= now) cnt[1] += 1;  /* completed in it */
+    if (t->state[i] == ST_RUNNING) o->used_blocks[r] += ((int64_t)t->prompt_len[i] + t->gen[i] + B - 1) / B;
+    if (t->state[i] == ST_QUEUED && t->arrival[i] <= now) {
+      o->used_blocks[r] += ((int64_t)t->prompt_len[i] + B - 1) / B;
+      if (k->ttft > 0) {
+        const int64_t wait = now - t->arrival[i];
+        i128 q = ((i128)wait << 16) / k->ttft;
+        if (q > ((i128)1 << 31)) q = (i128)1 << 31;
+        cnt[2] += 1;
+        cnt[3] += (int64_t)q;
+      }
+    }
+  }
+  for (int pool = 0; pool < 3; pool++) {
+    const int64_t *cnt = o->counts + 4 * pool;
+    int32_t n_active = 0, victim = -1;
+    for (int32_t r = 0; r < R; r++) {
+      if (c->replicas[r].mode != pool || total_blocks[r] <= 0) continue;
+      n_active++;
+      /* smallest used/total: compare by cross-multiplication */
+      if (victim < 0 || (i128)o->used_blocks[r] * total_blocks[victim] < (i128)o->used_blocks[victim] * total_blocks[r]) victim = r;
+    }
+    const int f1_valid = cnt[0] >= sp->min_samples;
+    int action = 0;
+    if ((f1_valid && (i128)sp->eps_out_den * cnt[1] < (i128)sp->eps_out_num * cnt[0]) ||
+        (cnt[2] > 0 && (i128)sp->eps_wait_den * cnt[3] > ((i128)sp->eps_wait_num * cnt[2] << 16)))
+      action = 1;
+    else if (f1_valid && (i128)sp->eps_in_den * cnt[1] > (i128)sp->eps_in_num * cnt[0] && n_active > 1)
+      action = -1;
+    o->decision[2 * pool] = action;
+    o->decision[2 * pool + 1] = action == -1 ? victim : -1;
+  }
+  return status;
+}

@@ -284,3 +284,42 @@ def test_idle_replica_jumps_to_its_next_event():
     wl = make_wl(rows[2:], C200, now=[500 * MS], maturity=[0])       # nothing left to happen: the clock stays
     oracle.step(wl, commit=True)
     assert wl.now[0] == 500 * MS
+
+
+def test_scaling_indicators_hand_worked():
+    # two colocated instances, tick at 20 s, 10 s window, 16-token KV blocks (Sec. 3.3.3)
+    S = 1000 * MS
+    rows = [dict(replica_id=0, arrival_ns=5 * S, state=gen.DONE, finish_ns=12 * S, req_id=0),      # completed in the window
+            dict(replica_id=1, arrival_ns=11 * S, state=gen.DONE, finish_ns=19 * S, req_id=1),     # arrived and completed in it
+            dict(replica_id=0, arrival_ns=15 * S, state=gen.RUNNING, prompt_len=100, gen=28, req_id=2),
+            dict(replica_id=1, arrival_ns=20 * S - 100 * MS, prompt_len=33, req_id=3),             # waits 100 ms of 200 ms
+            dict(replica_id=1, arrival_ns=20 * S - 20 * MS, prompt_len=16, req_id=4),              # waits 20 ms of 200 ms
+            dict(replica_id=0, arrival_ns=25 * S, prompt_len=500, req_id=5)]                       # not arrived yet
+    wl = make_wl(rows, C200, replicas=[(gen.COLOCATED, 8192, 0)] * 2, now=[0, 0], maturity=[0, 0])
+    o = oracle.scale_tick(wl, 20 * S, np.array([100, 100]), min_samples=2)
+    assert list(o["counts"][0]) == [4, 2, 2, 32768 + 6553]        # 0.5 and floor(0.1 * 65536) in 16.16
+    assert list(o["used_blocks"]) == [8, 3 + 1]                   # ceil(128/16); ceil(33/16) + ceil(16/16)
+    assert list(o["decision"][0]) == [1, -1]                      # f1 = 2/4 < 0.7 (and f2 = 0.3 > 1/4): scale out
+    assert np.all(o["counts"][1:] == 0) and np.all(o["decision"][1:] == [0, -1])
+    # too few arrivals seen: f1 is suppressed, f2 alone decides (0.3 > 1/4 still scales out; 1/2 does not)
+    assert list(oracle.scale_tick(wl, 20 * S, np.array([100, 100]), min_samples=5)["decision"][0]) == [1, -1]
+    assert list(oracle.scale_tick(wl, 20 * S, np.array([100, 100]), min_samples=5, eps_wait=(1, 2))["decision"][0]) == [0, -1]
+    # completions outpace arrivals and nobody waits: scale in, removing the emptier instance
+    for r in rows[3:5]:
+        r.update(state=gen.DONE, finish_ns=20 * S - 1)
+    wl = make_wl(rows, C200, replicas=[(gen.COLOCATED, 8192, 0)] * 2, now=[0, 0], maturity=[0, 0])
+    o = oracle.scale_tick(wl, 20 * S, np.array([100, 100]), min_samples=2)
+    assert list(o["counts"][0]) == [4, 4, 0, 0] and list(o["used_blocks"]) == [8, 0]
+    assert list(o["decision"][0]) == [0, -1]                      # f1 = 1.0: between the thresholds, hold
+    rows[2].update(state=gen.DONE, finish_ns=18 * S)
+    rows.append(dict(replica_id=0, arrival_ns=2 * S, state=gen.DONE, finish_ns=17 * S, req_id=6))
+    rows.append(dict(replica_id=0, arrival_ns=3 * S, state=gen.RUNNING, prompt_len=40, gen=0, req_id=7))
+    wl = make_wl(rows, C200, replicas=[(gen.COLOCATED, 8192, 0)] * 2, now=[0, 0], maturity=[0, 0])
+    o = oracle.scale_tick(wl, 20 * S, np.array([100, 100]), min_samples=2)
+    assert list(o["counts"][0]) == [4, 6, 0, 0] and list(o["decision"][0]) == [-1, 1]     # f1 = 1.5 > 1.1; instance 1 holds 0 blocks
+    o = oracle.scale_tick(wl, 20 * S, np.array([100, 0]), min_samples=2)
+    assert list(o["decision"][0]) == [0, -1]                      # a single active instance is never removed
+    o = oracle.scale_tick(wl, 20 * S, np.array([1, 100]), min_samples=2)
+    assert list(o["decision"][0]) == [-1, 1]
+    o = oracle.scale_tick(wl, 20 * S, np.array([1000, 100]), min_samples=2)     # 3/1000 vs 0/100: still instance 1
+    assert list(o["used_blocks"]) == [3, 0] and list(o["decision"][0]) == [-1, 1]
