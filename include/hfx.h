@@ -246,6 +246,37 @@ int hfx_sched_step(hfx_sched *s, const hfx_table *table,
 int hfx_sim_run(hfx_sched *s, const hfx_table *table, const int32_t *trace_off,
                 int32_t n_traces, int32_t iters, const hfx_sim_out *out);
 
+/* Scaling indicators and threshold policy of one Scaler tick (Sec. 3.3.3 "Scaling Mechanism and
+ * Policy"), evaluated per pool of instances (0 colocated, 1 prefill, 2 decode) over the whole
+ * table at time now_ns:
+ *   f1 = completions / arrivals inside the window (now - window_ns, now]   (used once at least
+ *        min_samples arrivals were seen),
+ *   f2 = mean over visible queued requests with a TTFT SLO of waiting_time / TTFT SLO, each ratio
+ *        in 16.16 fixed point (floor), saturated at 2^15,
+ *   f3 = used_blocks / total_blocks per instance: ceil((prompt_len + gen) / block_tokens) of every
+ *        in-flight request plus ceil(prompt_len / block_tokens) of every visible queued one.
+ * Decision per pool: scale out (+1) if f1 < eps_out or f2 > eps_wait; else scale in (-1) if
+ * f1 > eps_in and more than one instance of the pool is active (total_blocks > 0), removing the
+ * active instance with the smallest f3 (lowest id on ties); else hold (0).  Thresholds are the
+ * rationals num/den; the paper's defaults are window 10 s, 7/10, 11/10 and 1/4.
+ * `total_blocks` [n_replicas] and the outputs are device pointers; `params` is a host pointer.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_CUDA. */
+typedef struct hfx_scale_params {
+  int64_t window_ns;
+  int32_t block_tokens;   /* tokens per KV block, > 0 */
+  int32_t min_samples;
+  int32_t eps_out_num, eps_out_den, eps_in_num, eps_in_den, eps_wait_num, eps_wait_den;   /* > 0 */
+} hfx_scale_params;
+
+typedef struct hfx_scale_out {
+  int64_t *counts;       /* [3][4] per pool: arrivals, completions, queued requests, sum of 16.16 ratios */
+  int64_t *used_blocks;  /* [n_replicas] */
+  int32_t *decision;     /* [3][2] per pool: action, instance to remove (-1 unless scaling in) */
+} hfx_scale_out;
+
+int hfx_scale_tick(hfx_sched *s, const hfx_table *table, int64_t now_ns, const int32_t *total_blocks,
+                   const hfx_scale_params *params, const hfx_scale_out *out);
+
 /* Synchronise the scheduler's stream and return the sticky status word
  * (HFX_ST_* bits) in *status_word (host pointer); the word is then cleared.
  * Returns HFX_E_TIMEOUT if HFX_ST_TIMEOUT was set, HFX_E_CUDA if the stream
@@ -261,9 +292,9 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * stream, adds the elapsed times of all brackets recorded since the last call
  * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
  * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
- * 6 oversize path, 7 simulator; hfx_kernel_name gives the name of a slot
- * (NULL past the end). */
-#define HFX_N_KERNELS 8
+ * 6 oversize path, 7 simulator, 8 scaler tick; hfx_kernel_name gives the name of a
+ * slot (NULL past the end). */
+#define HFX_N_KERNELS 10
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
   int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */

@@ -21,9 +21,9 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_kernel_name", "hfx_count_rows_noalloc"]
+                    "hfx_sched_get_profile", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick"]
 NOALLOC_MAX_REPLICAS = 4096
-N_KERNELS = 8
+N_KERNELS = 10
 
 
 class HfxError(RuntimeError):
@@ -82,7 +82,17 @@ SIM_OUT_FIELDS = [("iters_executed", torch.int32), ("finished", torch.int32), ("
 
 
 class _Profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 8), ("launches", C.c_int64 * 8)]
+    _fields_ = [("ms", C.c_double * 10), ("launches", C.c_int64 * 10)]
+
+
+class _ScaleParams(C.Structure):
+    _fields_ = [("window_ns", C.c_int64), ("block_tokens", C.c_int32), ("min_samples", C.c_int32),
+                ("eps_out_num", C.c_int32), ("eps_out_den", C.c_int32), ("eps_in_num", C.c_int32),
+                ("eps_in_den", C.c_int32), ("eps_wait_num", C.c_int32), ("eps_wait_den", C.c_int32)]
+
+
+class _ScaleOut(C.Structure):
+    _fields_ = [("counts", C.c_void_p), ("used_blocks", C.c_void_p), ("decision", C.c_void_p)]
 
 
 class _SimOut(C.Structure):
@@ -123,6 +133,9 @@ def load_library():
     L.hfx_kernel_name.argtypes = [C.c_int]
     L.hfx_count_rows_noalloc.restype = C.c_int
     L.hfx_count_rows_noalloc.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.hfx_scale_tick.restype = C.c_int
+    L.hfx_scale_tick.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_ScaleParams),
+                                 C.POINTER(_ScaleOut)]
     L.hfx_strerror.restype = C.c_char_p
     L.hfx_strerror.argtypes = [C.c_int]
     _lib = L
@@ -266,6 +279,17 @@ class Scheduler:
         rc = self._L.hfx_sim_run(self._h, C.byref(ts), off.ctypes.data, int(off.shape[0] - 1), int(iters), C.byref(os_))
         if rc != 0:
             raise HfxError(rc, "hfx_sim_run")
+
+    def scale_tick(self, table: DeviceTable, now_ns: int, total_blocks: torch.Tensor, counts: torch.Tensor,
+                   used_blocks: torch.Tensor, decision: torch.Tensor, window_ns: int = 10_000_000_000,
+                   block_tokens: int = 16, min_samples: int = 10, eps_out=(7, 10), eps_in=(11, 10), eps_wait=(1, 4)):
+        """hfx_scale_tick: counts int64 [3, 4], used_blocks int64 [n_replicas], decision int32 [3, 2] (device)."""
+        ts = table.c_struct()
+        sp = _ScaleParams(int(window_ns), int(block_tokens), int(min_samples), *eps_out, *eps_in, *eps_wait)
+        so = _ScaleOut(counts.data_ptr(), used_blocks.data_ptr(), decision.data_ptr())
+        rc = self._L.hfx_scale_tick(self._h, C.byref(ts), int(now_ns), total_blocks.data_ptr(), C.byref(sp), C.byref(so))
+        if rc != 0:
+            raise HfxError(rc, "hfx_scale_tick")
 
     def status(self) -> int:
         w = C.c_uint32(0)

@@ -267,6 +267,6 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 
 extern "C" const char *hfx_kernel_name(int slot) {
   static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
-                                "k_big", "k_sim"};
-  return (slot >= 0 && slot < 8) ? names[slot] : nullptr;
+                                "k_big", "k_sim", "k_scale"};
+  return (slot >= 0 && slot < 9) ? names[slot] : nullptr;
 }

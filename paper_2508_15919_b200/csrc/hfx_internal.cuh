@@ -59,7 +59,7 @@ static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
 #include <vector>
 
-enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM };
+enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE };
 
 // tiling of the streaming passes: about this many tiles (2 per SM), each at most this many rows
 #define HFX_TILE_BLOCKS 296

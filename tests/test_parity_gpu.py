@@ -301,3 +301,51 @@ def test_argument_errors():
     with pytest.raises(hfx.HfxError):
         hfx.Scheduler(wl.model, wl.classes, [(3, 100, 0)], 10)
     sched.close()
+
+
+# ---- scaler tick -----------------------------------------------------------------------------------------
+def _scale_parity(wl, now, total_blocks, **kw):
+    import paper_2508_15919_b200 as hfx
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    tb = torch.from_numpy(np.ascontiguousarray(total_blocks, np.int32)).cuda()
+    counts = torch.full((3, 4), -1, dtype=torch.int64, device="cuda")
+    used = torch.full((wl.n_replicas,), -1, dtype=torch.int64, device="cuda")
+    dec = torch.full((3, 2), 9, dtype=torch.int32, device="cuda")
+    for _ in range(2):      # twice: the outputs must not accumulate
+        sched.scale_tick(tab, now, tb, counts, used, dec, **{("window_ns" if k == "window" else k): v for k, v in kw.items()})
+    st = sched.status()
+    c = oracle.scale_tick(wl, now, total_blocks, **kw)
+    assert st == c["status"]
+    assert np.array_equal(counts.cpu().numpy(), c["counts"]), (counts.cpu().numpy(), c["counts"])
+    assert np.array_equal(used.cpu().numpy(), c["used_blocks"])
+    assert np.array_equal(dec.cpu().numpy(), c["decision"]), (dec.cpu().numpy(), c["decision"])
+    sched.close()
+    return c
+
+
+def test_scaler_tick_parity():
+    rng = np.random.default_rng(3)
+    wl = gen.config4(R=64, n=200_001, steps=1)
+    wl.table["state"][::7] = gen.DONE
+    wl.table["finish_ns"][::7] = wl.table["arrival_ns"][::7] + rng.integers(0, 20 * SEC, wl.table["finish_ns"][::7].shape)
+    tb = rng.integers(0, 4000, 64)
+    seen = set()
+    for now, kw in ((30 * SEC, {}), (12 * SEC, dict(min_samples=100_000)),
+                    (30 * SEC, dict(eps_out=(1, 1000), eps_wait=(1000, 1), eps_in=(1, 100))),
+                    (30 * SEC, dict(eps_out=(1, 1000), eps_wait=(1000, 1), eps_in=(1000, 1))),
+                    (30 * SEC, dict(window=SEC, block_tokens=1, eps_out=(1, 1000)))):
+        c = _scale_parity(wl, now, tb, **kw)
+        seen.add(int(c["decision"][0][0]))
+    assert seen == {1, 0, -1}
+    # all three pools, bad rows, ties for the emptiest instance, more replicas than fit the shared counters
+    wl = gen.random_table(5, 30_000, 40, modes=MODES3, future=0.1, done=0.4)
+    wl.table["finish_ns"][:] = wl.now.max() - rng.integers(0, 3 * SEC, wl.n_rows)
+    wl.table["replica_id"][::31] = 77
+    wl.table["class_id"][5::29] = 200
+    tb = np.full(40, 1000); tb[::5] = 0
+    _scale_parity(wl, int(wl.now.max()), tb, window=2 * SEC, eps_in=(1, 50), eps_wait=(50, 1), min_samples=1)
+    wl = gen.random_table(6, 20_000, 9000)
+    _scale_parity(wl, int(wl.now.max()), np.full(9000, 5), window=2 * SEC)
+    wl = gen.random_table(7, 0, 3)
+    _scale_parity(wl, 5, np.full(3, 5))
