@@ -109,7 +109,6 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     if (n_replicas <= HFX_TILE_REPLICAS_MAX && 2 * (int64_t)n_tiles * (n_replicas + 1) <= HFX_TILE_MATRIX_MAX) {
       const size_t cells = (size_t)n_tiles * ((size_t)n_replicas + 1);
       ok = ok && cudaMalloc(&s->d_tile_hist, sizeof(uint32_t) * 2 * cells) == cudaSuccess;
-      ok = ok && cudaMalloc(&s->d_tile_fmin, sizeof(int64_t) * cells) == cudaSuccess;
       ok = ok && cudaMalloc(&s->d_tile_mode, (size_t)n_tiles + 16) == cudaSuccess;
       s->tile_blocks_max = n_tiles;
     }
@@ -154,7 +153,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   if (s->ev_join) cudaEventDestroy(s->ev_join);
   cudaFree(s->d_cfg); cudaFree(s->d_mode); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
-  cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_fmin); cudaFree(s->d_tile_mode);
+  cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_mode);
   cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();

@@ -91,7 +91,6 @@ struct hfx_sched {
   uint32_t *d_tile_hist;    // [tile_blocks_max][2][R+1] per-tile histograms: all rows, active rows
                             // (nullptr: atomic mode only)
   uint8_t *d_tile_mode;     // [tile_blocks_max] how ranks inside a tile are found (TILE_*)
-  int64_t *d_tile_fmin;     // [tile_blocks_max][R+1] earliest arrival among a tile's not-yet-arrived rows
   uint8_t *d_rowflag;       // [max_rows] kind of every row (KIND_*), ROWFLAG_BADREP for a bad replica id
   int32_t tile_blocks_max;
   uint32_t step_parity;     // which of the two `ordered` words this step uses
@@ -352,6 +351,7 @@ struct RegroupArgs {
 };
 
 struct SegArgs {
+  const int64_t *arrival;   // read-only table column (next arrival of an idle replica)
   // table columns written by COMMIT
   uint8_t *state; int32_t *gen; int64_t *first_token; int64_t *last_token; int64_t *finish;
   // replica state

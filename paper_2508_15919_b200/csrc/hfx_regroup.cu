@@ -427,20 +427,19 @@ __global__ void __launch_bounds__(256) k_regroup_atomic(const HfxParams p, const
 // matrix mode: see the head of this file
 struct TileArgs {
   const uint32_t *M; const uint8_t *tile_mode; const uint32_t *seg_begin; const uint32_t *tot_act;
-  const uint8_t *rowflag; const uint32_t *ordered; int64_t *fmin; HfxRec *rec; int32_t tile_rows;
+  const uint8_t *rowflag; const uint32_t *ordered; HfxRec *rec; int32_t tile_rows;
 };
 
 __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, const RegroupArgs a, const TileArgs ta) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int R = p.n_replicas, R1 = R + 1, T = ta.tile_rows;
-  int64_t *s_fmin = reinterpret_cast<int64_t *>(smem_raw);           // [R1] earliest not-yet-arrived row per replica
-  uint32_t *s_cnt = reinterpret_cast<uint32_t *>(s_fmin + 2 * R1);   // [R1]   rows of each replica in the tile / cursors
+  int64_t *s_start = reinterpret_cast<int64_t *>(smem_raw);          // [R1]   earliest start max(now, maturity)
+  uint32_t *s_cnt = reinterpret_cast<uint32_t *>(s_start + R1);      // [R1]   rows of each replica in the tile / cursors
   uint32_t *s_off = s_cnt + R1;                                      // [R1+1] exclusive prefix of s_cnt / cursors
   uint32_t *s_bact = s_off + R1 + 1;                                 // [R1]   where the tile's active rows of r start
   uint32_t *s_bin = s_bact + R1;                                     // [R1]   where its inactive rows start
   uint16_t *s_stage = reinterpret_cast<uint16_t *>(s_bin + R1);      // [T]    tile rows grouped by replica (+ class bit)
   uint16_t *s_P = s_stage + T;                                       // [T+1]  active rows before each tile position
-  int64_t *s_start = s_fmin + R1;                                    // [R1]   earliest start max(now, maturity)
   uint8_t *s_mode = reinterpret_cast<uint8_t *>(s_P + T + 1);        // [R1]   replica modes
   __shared__ int64_t s_ttft[HFX_MAX_CLASSES], s_tpot[HFX_MAX_CLASSES];
   __shared__ uint8_t s_prio[HFX_MAX_CLASSES];
@@ -448,13 +447,11 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
   const int mode = ta.tile_mode[blockIdx.x];
   const bool ordered = *ta.ordered != 0;
-  const bool use_fmin = ordered && a.commit;
 
   stage_classes(p, s_ttft, s_tpot, s_prio);
   for (int i = tid; i < R1; i += blockDim.x) {
     s_cnt[i] = 0; s_off[i] = 0; s_mode[i] = i < R ? a.mode[i] : 0;
     { int64_t st = 0; if (i < R) { const int64_t nw = a.now[i], mt = a.mat[i]; st = nw > mt ? nw : mt; } s_start[i] = st; }
-    if (use_fmin) s_fmin[i] = HFX_INF;
   }
   __syncthreads();
 
@@ -569,7 +566,6 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
       store_record(ta.rec, (act ? s_bact[bkt] : s_bin[bkt]) + rank, r);
     } else {
       a.order[s_bin[bkt] + rank] = (int32_t)i;
-      if (use_fmin && in.kind == KIND_FUTURE) atomicMin(reinterpret_cast<long long *>(&s_fmin[bkt]), (long long)in.arrival);
     }
     return o;
   };
@@ -588,18 +584,13 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
     const RowOut o = emit(lo + i, i, in);
     write_outputs1(a, lo + i, bucket_of(in.rid, R), o);
   }
-  if (use_fmin) {
-    __syncthreads();
-    int64_t *frow = ta.fmin + (size_t)blockIdx.x * R1;
-    for (int i = tid; i < R1; i += blockDim.x) frow[i] = s_fmin[i];
-  }
 }
 
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
 size_t hfx_regroup_smem(int R1, int tile_rows) {
-  return sizeof(int64_t) * 2 * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) +
+  return sizeof(int64_t) * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) +
          (size_t)R1 + 32;
 }
 
@@ -632,7 +623,7 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
       KernelScope ks(s, KSLOT_REGROUP);
       TileArgs ta;
       ta.M = s->d_tile_hist; ta.tile_mode = s->d_tile_mode; ta.seg_begin = s->d_seg_begin; ta.tot_act = s->d_act_count;
-      ta.rowflag = s->d_rowflag; ta.ordered = ordered; ta.fmin = s->d_tile_fmin; ta.rec = s->d_rec; ta.tile_rows = tile_rows;
+      ta.rowflag = s->d_rowflag; ta.ordered = ordered; ta.rec = s->d_rec; ta.tile_rows = tile_rows;
       k_regroup<<<n_tiles, THREADS_TILE, hfx_regroup_smem(R1, tile_rows), stream>>>(s->p, ra, ta);
     }
   } else {

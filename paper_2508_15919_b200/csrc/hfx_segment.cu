@@ -252,8 +252,21 @@ __device__ __forceinline__ void commit_row(const SegArgs &a, const ReplicaPlan &
 // where a kernel finds the regrouped table
 struct SegCtx {
   const HfxRec *rec; const uint32_t *seg_begin; const uint32_t *tot_act; const uint32_t *flags;
-  const int64_t *fmin; int32_t n_tiles; uint32_t parity;
+  const uint8_t *rowflag; uint32_t parity;
 };
+
+// Earliest arrival among a replica's rows that have not arrived yet, for the clock jump of an idle
+// replica in an ordered step: the regroup has listed the replica's inactive rows in
+// order[b + n_act .. b + n); their kind bytes say which of them are still to come.
+__device__ __forceinline__ int64_t next_arrival_listed(const SegArgs &a, const SegCtx &c, uint32_t b, int64_t n_act, int64_t n,
+                                                       int64_t first, int64_t stride) {
+  int64_t v = HFX_INF;
+  for (int64_t q = n_act + first; q < n; q += stride) {
+    const int32_t row = a.order[b + q];
+    if (c.rowflag[row] == KIND_FUTURE) { const int64_t x = a.arrival[row]; v = x < v ? x : v; }
+  }
+  return v;
+}
 
 // aggregates of a replica's active records into the block's plan (all threads call; result in
 // sh.plan; sh.next_arrival is left at "none")
@@ -457,10 +470,8 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
     const int worked = sh.worked;
     const int64_t mat_next = sh.red_c[0];
     if (commit && !worked && ordered) {
-      // idle replica of an ordered step: its next arrival comes from the regroup's per-tile minima
-      int64_t v = HFX_INF;
-      for (int t = threadIdx.x; t < c.n_tiles; t += blockDim.x) { const int64_t x = c.fmin[(size_t)t * (R + 1) + r]; v = x < v ? x : v; }
-      block_min_arrival(v, sh);
+      // idle replica of an ordered step: its next arrival is looked up among its listed inactive rows
+      block_min_arrival(next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x), sh);
     }
     if (threadIdx.x == 0 && real)
       write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
@@ -732,10 +743,8 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
     const int worked = sh.worked;
     const int64_t mat_next = sh.red_c[0];
     if (commit && !worked && ordered) {
-      // idle replica of an ordered step: its next arrival comes from the regroup's per-tile minima
-      int64_t v = HFX_INF;
-      for (int t = threadIdx.x; t < c.n_tiles; t += blockDim.x) { const int64_t x = c.fmin[(size_t)t * (R + 1) + r]; v = x < v ? x : v; }
-      block_min_arrival(v, sh);
+      // idle replica of an ordered step: its next arrival is looked up among its listed inactive rows
+      block_min_arrival(next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x), sh);
     }
     if (threadIdx.x == 0 && real)
       write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
@@ -939,7 +948,7 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
       // the replica's next arrival, should it turn out idle
       int64_t v = HFX_INF;
       if (ordered) {
-        for (int t = threadIdx.x; t < c.n_tiles; t += blockDim.x) { const int64_t x = c.fmin[(size_t)t * (R + 1) + r]; v = x < v ? x : v; }
+        v = next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x);
       } else {
         const HfxRec *sin = seg + n_act;
         for (int64_t q = threadIdx.x; q < n_in; q += blockDim.x) {
@@ -986,9 +995,7 @@ int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
   cudaStream_t stream = s->stream;
   SegCtx c;
   c.rec = s->d_rec; c.seg_begin = s->d_seg_begin; c.tot_act = s->d_act_count; c.flags = s->d_flags;
-  c.fmin = s->d_tile_fmin; c.parity = s->step_parity;
-  int32_t tile_rows;
-  hfx_tile_shape(n, &tile_rows, &c.n_tiles);
+  c.rowflag = s->d_rowflag; c.parity = s->step_parity;
   // Replicas too large for the small kernel are rare; their kernels (which leave at once when there is
   // nothing for them) run on a second stream beside the small-replica kernel, forked and joined by events.
   const bool larger = n > SEG_TINY;

@@ -39,7 +39,7 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
   if (rc != HFX_OK) return rc;
 
   SegArgs sa;
-  sa.state = t->state; sa.gen = t->gen; sa.first_token = t->first_token_ns; sa.last_token = t->last_token_ns;
+  sa.arrival = t->arrival_ns; sa.state = t->state; sa.gen = t->gen; sa.first_token = t->first_token_ns; sa.last_token = t->last_token_ns;
   sa.finish = t->finish_ns; sa.now = st->now_ns; sa.mat = st->maturity_ns; sa.cfg = s->d_cfg;
   sa.slack = o->slack_ns; sa.pred_tpot = o->pred_tpot_ns; sa.key = o->key; sa.order = o->order; sa.admit = o->admit;
   sa.admitted_rows = o->admitted_rows; sa.budget = o->budget; sa.e_d = o->e_d_ns; sa.n_run = o->n_run;
