@@ -198,27 +198,38 @@ __device__ inline void dev_plan(const HfxParams &p, const hfx_replica_cfg &cfg, 
 }
 
 // The same plan computed by a whole warp (all 32 lanes call with the same arguments and get the same
-// result): class minima by lanes, and the largest safe n by a 32-way search instead of a bisection.
-__device__ inline int64_t warp_min_over_mask(const int64_t *v, uint64_t mask, int lane) {
+// result).  The class minima are taken by lanes from a copy of the class tables in shared memory
+// (cls_ttft / cls_tpot, HFX_MAX_CLASSES entries each); the largest safe n comes from a 128-way search
+// on the bound itself, E_p(n) * (2 TPOT - E_d) <= TTFT * (TPOT - E_d), compared in 128 bits: for
+// integer E_p that is the same set of n as E_p(n) <= floor(TTFT (TPOT - E_d) / (2 TPOT - E_d)), and no
+// division is needed.
+__device__ inline int64_t warp_min_over_mask(const int64_t *cls_v, uint64_t mask, int lane) {
   int64_t m = HFX_INF;
 #pragma unroll
   for (int c = lane; c < HFX_MAX_CLASSES; c += 32)
-    if ((mask >> c) & 1ull) { const int64_t x = v[c]; if (x > 0 && x < m) m = x; }
+    if ((mask >> c) & 1ull) { const int64_t x = cls_v[c]; if (x > 0 && x < m) m = x; }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) { const int64_t w = __shfl_xor_sync(0xffffffffu, m, o); m = w < m ? w : m; }
   return m;
 }
 
-__device__ inline int64_t warp_nsafe(const HfxParams &p, int64_t epmax, int64_t cap, int lane) {
-  if (epmax == HFX_INF) return cap;
-  if (dev_Ep(p, 0) > epmax) return 0;
-  int64_t lo = 0, hi = cap;          // E_p(lo) <= epmax; the answer lies in [lo, hi]
+// Largest n in [0, cap] with E_p(n) * den <= num (num = nh:nl as 128 bits, den > 0), 0 if none.
+__device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t nl, uint64_t den, int64_t cap, int lane) {
+  auto fits = [&](int64_t n) {
+    const uint64_t ep = (uint64_t)dev_Ep(p, n);
+    const uint64_t ph = __umul64hi(ep, den), pl = ep * den;
+    return ph < nh || (ph == nh && pl <= nl);
+  };
+  if (!fits(0)) return 0;
+  int64_t lo = 0, hi = cap;          // fits(lo); the answer lies in [lo, hi]
   while (lo < hi) {
-    const int64_t step = (hi - lo + 31) / 32;
-    int64_t cand = lo + (int64_t)(lane + 1) * step;
-    const bool in = cand <= hi;
-    const bool ok = in && dev_Ep(p, cand) <= epmax;
-    const int m = __popc(__ballot_sync(0xffffffffu, ok));       // E_p is monotone: the ok lanes are a prefix
+    const int64_t step = (int64_t)(((uint64_t)(hi - lo) + 127u) >> 7);
+    int m = 0;
+#pragma unroll
+    for (int j = 0; j < 4; j++) {    // candidate index j * 32 + lane: E_p is monotone, so the ones that fit are a prefix
+      const int64_t cand = lo + (int64_t)(j * 32 + lane + 1) * step;
+      m += __popc(__ballot_sync(0xffffffffu, cand <= hi && fits(cand)));
+    }
     const int64_t nlo = lo + (int64_t)m * step;
     int64_t nhi = lo + (int64_t)(m + 1) * step - 1;
     if (nhi > hi) nhi = hi;
@@ -227,13 +238,13 @@ __device__ inline int64_t warp_nsafe(const HfxParams &p, int64_t epmax, int64_t 
   return lo;
 }
 
-__device__ inline void warp_plan(const HfxParams &p, const hfx_replica_cfg &cfg, int64_t now, int64_t mat,
-                                 int64_t n_run, int64_t sum_kv, uint64_t mask_run, uint64_t mask_q, ReplicaPlan &pl,
-                                 int lane) {
+__device__ inline void warp_plan(const HfxParams &p, const int64_t *cls_ttft, const int64_t *cls_tpot,
+                                 const hfx_replica_cfg &cfg, int64_t now, int64_t mat, int64_t n_run, int64_t sum_kv,
+                                 uint64_t mask_run, uint64_t mask_q, ReplicaPlan &pl, int lane) {
   pl.now = now; pl.mat = mat; pl.start = now > mat ? now : mat;
   pl.mode = cfg.mode; pl.token_cap = cfg.token_cap; pl.batch_cap = cfg.batch_cap;
   pl.n_run = n_run; pl.sum_kv = sum_kv;
-  const int64_t min_tpot = warp_min_over_mask(p.tpot, mask_run, lane);
+  const int64_t min_tpot = warp_min_over_mask(cls_tpot, mask_run, lane);
   const bool prefill = cfg.mode == HFX_PREFILL;
   pl.n_eff = prefill ? 0 : n_run;
   pl.kv_eff = prefill ? 0 : sum_kv;
@@ -242,7 +253,7 @@ __device__ inline void warp_plan(const HfxParams &p, const hfx_replica_cfg &cfg,
   int64_t budget = 0;
   if (now >= mat) {      // before maturity the instance is protected: no budget to work out
     if (cfg.mode == HFX_DECODE) {
-      const int64_t T = (n_run > 0 && min_tpot < HFX_INF) ? min_tpot : warp_min_over_mask(p.tpot, mask_q, lane);
+      const int64_t T = (n_run > 0 && min_tpot < HFX_INF) ? min_tpot : warp_min_over_mask(cls_tpot, mask_q, lane);
       if (p.budget_mode == HFX_BUDGET_CAP_ONLY || T == HFX_INF) budget = HFX_INF;
       else {
         const int64_t room = T - dev_Ed(p, n_run, sum_kv);
@@ -253,8 +264,15 @@ __device__ inline void warp_plan(const HfxParams &p, const hfx_replica_cfg &cfg,
       int64_t n_safe;
       if (p.budget_mode == HFX_BUDGET_CAP_ONLY) n_safe = cfg.token_cap;
       else {
-        const int64_t min_ttft = warp_min_over_mask(p.ttft, mask_q, lane);
-        n_safe = warp_nsafe(p, dev_epmax(min_ttft, pl.n_eff > 0 && pl.tpot_eff < HFX_INF, pl.tpot_eff, pl.e_d), cfg.token_cap, lane);
+        const int64_t min_ttft = warp_min_over_mask(cls_ttft, mask_q, lane);
+        const bool decoding = pl.n_eff > 0 && pl.tpot_eff < HFX_INF;
+        if (min_ttft == HFX_INF) n_safe = cfg.token_cap;
+        else if (!decoding) n_safe = warp_nsafe(p, 0, (uint64_t)min_ttft, 2, cfg.token_cap, lane);     // 2 E_p <= TTFT
+        else if (pl.tpot_eff <= pl.e_d) n_safe = 0;
+        else {
+          const uint64_t x = (uint64_t)min_ttft, y = (uint64_t)(pl.tpot_eff - pl.e_d);
+          n_safe = warp_nsafe(p, __umul64hi(x, y), x * y, (uint64_t)(2 * pl.tpot_eff - pl.e_d), cfg.token_cap, lane);
+        }
       }
       budget = n_safe < cap_left ? n_safe : cap_left;
     }

@@ -514,9 +514,14 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
   uint32_t *s_bin = s_lo + SEG_TINY;                                                   // [TINY_BINS + 4]
   uint32_t *s_cur = s_bin + TINY_BINS + 4;                                             // [TINY_BINS]
   __shared__ BlockShared sh;
+  __shared__ int64_t s_cls_ttft[HFX_MAX_CLASSES], s_cls_tpot[HFX_MAX_CLASSES];     // class tables for the planning warp
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const int R = p.n_replicas;
   const bool ordered = c.flags[c.parity] != 0;
+  for (int k = threadIdx.x; k < HFX_MAX_CLASSES; k += blockDim.x) {
+    s_cls_ttft[k] = k < p.n_classes ? p.ttft[k] : 0;
+    s_cls_tpot[k] = k < p.n_classes ? p.tpot[k] : 0;
+  }
 
   for (int r = blockIdx.x; r <= R; r += gridDim.x) {
     const uint32_t b = c.seg_begin[r];
@@ -577,7 +582,7 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
         int64_t now = 0, mat = 0;
         if (real) { cfg = a.cfg[r]; now = a.now[r]; mat = a.mat[r]; }
         ReplicaPlan pl0;
-        warp_plan(p, cfg, now, mat, n_run, sum_kv, m_run, m_q, pl0, lane);
+        warp_plan(p, s_cls_ttft, s_cls_tpot, cfg, now, mat, n_run, sum_kv, m_run, m_q, pl0, lane);
         if (lane == 0) { sh.plan = pl0; sh.next_arrival = next_arr; }
       }
       __syncthreads();

@@ -47,6 +47,7 @@ struct SimShared {
   // end-of-trace counters
   int32_t n_fin, n_rej, n_att, n_a, n_b;
   int64_t ttft[HFX_MAX_CLASSES];   // TTFT SLO per class
+  int64_t tpot[HFX_MAX_CLASSES];   // TPOT SLO per class
 };
 
 __device__ __forceinline__ void sort_i64(int64_t *v, int n) {
@@ -111,7 +112,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       S.n_fin = 0; S.n_rej = 0; S.n_att = 0; S.n_a = 0; S.n_b = 0; S.zero_prompt = 0;
     }
     __syncthreads();
-    for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; S.ttft[c] = c < p.n_classes ? p.ttft[c] : 0; }
+    for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; S.ttft[c] = c < p.n_classes ? p.ttft[c] : 0; S.tpot[c] = c < p.n_classes ? p.tpot[c] : 0; }
     uint32_t bad = 0;
     for (int i = tid; i < m; i += SIM_THREADS) {
       const int64_t g = (int64_t)b + i;
@@ -178,7 +179,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
         const uint32_t q0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_q[lane] > 0);
         const uint32_t q1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && S.cnt_q[lane + 32] > 0);
         ReplicaPlan pl0;
-        warp_plan(p, cfg, S.now, S.mat, S.nr, S.sum_kv, ((uint64_t)r1 << 32) | r0, ((uint64_t)q1 << 32) | q0, pl0, lane);
+        warp_plan(p, S.ttft, S.tpot, cfg, S.now, S.mat, S.nr, S.sum_kv, ((uint64_t)r1 << 32) | r0, ((uint64_t)q1 << 32) | q0, pl0, lane);
         if (lane == 0) S.plan = pl0;
       }
       __syncthreads();
