@@ -33,7 +33,7 @@ METRIC = "requests_scheduled_per_sec_per_hfx_sched_step"
 UNIT = "requests/s"
 ALGO_BYTES_PER_ROW = 51            # 38 B read (incl. priority weight) + 13 B written per row and step
 # algorithmic bytes per row of each kernel (what that kernel must move once)
-KERNEL_BYTES_PER_ROW = {"k_count": 26, "k_colscan": 0, "k_regroup": 51, "k_segment(small)": 13,
+KERNEL_BYTES_PER_ROW = {"k_front": 51, "k_count": 26, "k_colscan": 0, "k_regroup": 51, "k_segment(small)": 13,
                         "k_segment(medium)": 13, "k_big": 13}
 STEPS_PER_EPISODE = 10
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel on this workload,

@@ -292,14 +292,22 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * stream, adds the elapsed times of all brackets recorded since the last call
  * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
  * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
- * 6 oversize path, 7 simulator, 8 scaler tick; hfx_kernel_name gives the name of a
- * slot (NULL past the end). */
+ * 6 oversize path, 7 simulator, 8 scaler tick, 9 fused front end; hfx_kernel_name
+ * gives the name of a slot (NULL past the end). */
 #define HFX_N_KERNELS 10
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
   int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */
 } hfx_profile;
 int hfx_sched_set_profiling(hfx_sched *s, int on);
+/* The front end of a step (row kinds and per-tile counts, their column scan,
+ * the offsets, the regroup into per-replica ranges) normally runs as one
+ * cooperative kernel, k_front, when every tile's block can be resident at once
+ * (slot 9); `on` = 0 makes the following steps use the separate kernels k_count,
+ * k_colscan and k_regroup instead, which is also what larger tables fall back
+ * to.  Results are identical either way.  Host call, takes effect at the next
+ * hfx_sched_step.  The paper has no counterpart (an execution switch). */
+int hfx_sched_set_fused_front(hfx_sched *s, int on);
 int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out);
 const char *hfx_kernel_name(int slot);
 

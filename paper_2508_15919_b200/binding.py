@@ -21,7 +21,7 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick"]
+                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick"]
 NOALLOC_MAX_REPLICAS = 4096
 N_KERNELS = 10
 
@@ -127,6 +127,8 @@ def load_library():
     L.hfx_sched_destroy.argtypes = [C.c_void_p]
     L.hfx_sched_set_profiling.restype = C.c_int
     L.hfx_sched_set_profiling.argtypes = [C.c_void_p, C.c_int]
+    L.hfx_sched_set_fused_front.restype = C.c_int
+    L.hfx_sched_set_fused_front.argtypes = [C.c_void_p, C.c_int]
     L.hfx_sched_get_profile.restype = C.c_int
     L.hfx_sched_get_profile.argtypes = [C.c_void_p, C.POINTER(_Profile)]
     L.hfx_kernel_name.restype = C.c_char_p
@@ -302,6 +304,13 @@ class Scheduler:
         rc = self._L.hfx_sched_set_profiling(self._h, int(on))
         if rc != 0:
             raise HfxError(rc, "hfx_sched_set_profiling")
+
+    def set_fused_front(self, on: bool):
+        """Run the front end of the following steps as one cooperative kernel (default) or as
+        separate kernels; the results are the same."""
+        rc = self._L.hfx_sched_set_fused_front(self._h, int(on))
+        if rc != 0:
+            raise HfxError(rc, "hfx_sched_set_fused_front")
 
     def get_profile(self) -> Dict[str, Dict[str, float]]:
         """Per-kernel device time (ms) and launches recorded since the last call."""

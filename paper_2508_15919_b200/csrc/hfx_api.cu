@@ -115,6 +115,8 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   }
   ok = ok && cudaMalloc(&s->d_rec, sizeof(HfxRec) * (size_t)max_rows) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_barrier, 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_front_bar, 256) == cudaSuccess;
+  s->front_enabled = 1; s->front_arrivals = 0; s->front_smem_cached = 0; s->front_capacity = 0;
   ok = ok && cudaMalloc(&h->d_trace_off, sizeof(int32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&h->d_work_counter, 256) == cudaSuccess;
   if (ok && max_rows > 16384) {   // scratch of the global sort: only tables that can hold an oversize segment
@@ -127,6 +129,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     memcpy(h->h_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas);
     ok = ok && cudaMemcpy(s->d_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemset(s->d_status, 0, 256) == cudaSuccess;
+    ok = ok && cudaMemset(s->d_front_bar, 0, 256) == cudaSuccess;
     {
       std::vector<uint8_t> modes((size_t)n_replicas);
       for (int r = 0; r < n_replicas; r++) modes[r] = (uint8_t)replicas[r].mode;
@@ -154,7 +157,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   cudaFree(s->d_cfg); cudaFree(s->d_mode); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
   cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_mode);
-  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier);
+  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier); cudaFree(s->d_front_bar);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();
   if (s->brackets) {
@@ -247,6 +250,12 @@ extern "C" int hfx_sched_set_profiling(hfx_sched *s, int on) {
   return HFX_OK;
 }
 
+extern "C" int hfx_sched_set_fused_front(hfx_sched *s, int on) {
+  if (!s) return HFX_E_ARG;
+  s->front_enabled = on ? 1 : 0;
+  return HFX_OK;
+}
+
 extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
   if (!s || !out) return HFX_E_ARG;
   if (cudaStreamSynchronize(s->stream) != cudaSuccess) { cudaGetLastError(); return HFX_E_CUDA; }
@@ -266,6 +275,6 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 
 extern "C" const char *hfx_kernel_name(int slot) {
   static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
-                                "k_big", "k_sim", "k_scale"};
-  return (slot >= 0 && slot < 9) ? names[slot] : nullptr;
+                                "k_big", "k_sim", "k_scale", "k_front"};
+  return (slot >= 0 && slot < 10) ? names[slot] : nullptr;
 }

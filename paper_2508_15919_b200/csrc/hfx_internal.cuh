@@ -59,7 +59,7 @@ static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
 #include <vector>
 
-enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE };
+enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT };
 
 // tiling of the streaming passes: about this many tiles (2 per SM), each at most this many rows
 #define HFX_TILE_BLOCKS 296
@@ -99,6 +99,12 @@ struct hfx_sched {
   uint64_t *d_big_hi;       // sort scratch of oversize segments
   uint32_t *d_big_lo;
   uint32_t *d_barrier;      // grid barrier words of the oversize path
+  // fused front end (count + column scan + offsets + regroup as one cooperative kernel)
+  unsigned long long *d_front_bar;     // arrivals at its grid barriers, only ever grows
+  unsigned long long front_arrivals;   // host copy of what that word holds once every launch so far is done
+  int front_enabled;
+  size_t front_smem_cached;            // shared-memory size the capacity below was asked for
+  int front_capacity;                  // blocks of the fused kernel that can be resident at once
 };
 
 // ---- latency predictor -------------------------------------------------------------------

@@ -17,6 +17,13 @@
 #include "hfx_internal.cuh"
 
 #define THREADS_TILE 512
+
+// dynamic shared memory of the regroup's arrays (multiple of 16 bytes)
+__host__ __device__ inline size_t hfx_regroup_smem_dev(int R1, int tile_rows) {
+  const size_t b = sizeof(int64_t) * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) +
+                   sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) + (size_t)R1 + 32;
+  return (b + 15) & ~(size_t)15;
+}
 #define COLSCAN_REG 16
 #define GROUP_MAX 64      // largest same-replica group of an unsorted tile that is ranked by scanning
 
@@ -49,8 +56,8 @@ struct CountArgs {
   uint8_t *rowflag; uint32_t *status; uint32_t *ordered;
 };
 
-__global__ void __launch_bounds__(THREADS_TILE) k_count(const HfxParams p, const CountArgs a) {
-  extern __shared__ uint32_t s_hist[];    // [2][R1]
+// s_hist: [2][R1] words of shared memory (matrix mode only)
+__device__ __forceinline__ void count_tile(const HfxParams &p, const CountArgs &a, uint32_t *s_hist) {
   const int R = p.n_replicas, R1 = R + 1;
   const bool matrix = a.M != nullptr;
   uint32_t *h_all = s_hist, *h_act = s_hist + R1;
@@ -123,6 +130,11 @@ __global__ void __launch_bounds__(THREADS_TILE) k_count(const HfxParams p, const
     a.tile_mode[blockIdx.x] = (uint8_t)mode;
     if (mode == TILE_ANY || !rising) *a.ordered = 0;
   }
+}
+
+__global__ void __launch_bounds__(THREADS_TILE) k_count(const HfxParams p, const CountArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  count_tile(p, a, reinterpret_cast<uint32_t *>(smem_raw));
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -310,7 +322,7 @@ __device__ __forceinline__ void store_record(HfxRec *rec, uint32_t pos, const Hf
 __device__ __forceinline__ void load_rows4(const RegroupArgs &a, const uint8_t *rowflag, int64_t v, RowIn in[4]) {
   const int4 rid = __ldg(reinterpret_cast<const int4 *>(a.replica_id) + v);
   const uchar4 cls = __ldg(reinterpret_cast<const uchar4 *>(a.class_id) + v);
-  const uchar4 kd = __ldg(reinterpret_cast<const uchar4 *>(rowflag) + v);
+  const uchar4 kd = reinterpret_cast<const uchar4 *>(rowflag)[v];     // (not a read-only load: the fused kernel wrote it)
   const int4 pr = __ldg(reinterpret_cast<const int4 *>(a.prompt_len) + v);
   const int4 ge = __ldg(reinterpret_cast<const int4 *>(a.gen) + v);
   const int4 id = __ldg(reinterpret_cast<const int4 *>(a.req_id) + v);
@@ -430,8 +442,8 @@ struct TileArgs {
   const uint8_t *rowflag; const uint32_t *ordered; HfxRec *rec; int32_t tile_rows;
 };
 
-__global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, const RegroupArgs a, const TileArgs ta) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+// ta.seg_begin and ta.tot_act may point to shared memory (the fused kernel keeps its own copy there).
+__device__ __forceinline__ void regroup_tile(const HfxParams &p, const RegroupArgs &a, const TileArgs &ta, unsigned char *smem_raw) {
   const int R = p.n_replicas, R1 = R + 1, T = ta.tile_rows;
   int64_t *s_start = reinterpret_cast<int64_t *>(smem_raw);          // [R1]   earliest start max(now, maturity)
   uint32_t *s_cnt = reinterpret_cast<uint32_t *>(s_start + R1);      // [R1]   rows of each replica in the tile / cursors
@@ -446,7 +458,7 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   __shared__ uint32_t s_warp[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
   const int mode = ta.tile_mode[blockIdx.x];
-  const bool ordered = *ta.ordered != 0;
+  const bool ordered = __ldcg(ta.ordered) != 0;
 
   stage_classes(p, s_ttft, s_tpot, s_prio);
   for (int i = tid; i < R1; i += blockDim.x) {
@@ -466,7 +478,7 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
     // ---- A: histogram of the tile; active flag of every position ------------------------------------
     for (int v = tid; v < nvec; v += blockDim.x) {
       const int4 r4 = __ldg(reinterpret_cast<const int4 *>(a.replica_id) + v0 + v);
-      const uchar4 k4 = __ldg(reinterpret_cast<const uchar4 *>(ta.rowflag) + v0 + v);
+      const uchar4 k4 = reinterpret_cast<const uchar4 *>(ta.rowflag)[v0 + v];
       atomicAdd(&s_cnt[bucket_of(r4.x, R)], 1u); atomicAdd(&s_cnt[bucket_of(r4.y, R)], 1u);
       atomicAdd(&s_cnt[bucket_of(r4.z, R)], 1u); atomicAdd(&s_cnt[bucket_of(r4.w, R)], 1u);
       s_P[4 * v] = k4.x <= KIND_QUEUED; s_P[4 * v + 1] = k4.y <= KIND_QUEUED;
@@ -533,7 +545,7 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
     }
   }
   for (int i = tid; i < R1; i += blockDim.x) {
-    const uint32_t m_all = ta.M[mrow + i], m_act = ta.M[mrow + R1 + i], sb = ta.seg_begin[i];
+    const uint32_t m_all = __ldcg(ta.M + mrow + i), m_act = __ldcg(ta.M + mrow + R1 + i), sb = ta.seg_begin[i];
     s_bact[i] = sb + m_act;
     s_bin[i] = sb + ta.tot_act[i] + (m_all - m_act);
   }
@@ -586,12 +598,157 @@ __global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, 
   }
 }
 
+__global__ void __launch_bounds__(THREADS_TILE, 2) k_regroup(const HfxParams p, const RegroupArgs a, const TileArgs ta) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  regroup_tile(p, a, ta, smem_raw);
+}
+
+// ------------------------------------------------------------------------------------------------
+// k_front: count, column scan, offsets and regroup as ONE cooperative kernel (one block per tile,
+// all blocks resident), separated by two grid barriers.  The barriers count arrivals on a 64-bit
+// word that only ever grows: the host passes the value it must reach, so nothing is reset
+// between launches.  Every wait is bounded; a block whose wait runs out raises HFX_ST_TIMEOUT and
+// leaves.
+// ------------------------------------------------------------------------------------------------
+__device__ bool front_barrier(unsigned long long *bar, unsigned long long target, uint32_t *status) {
+  __shared__ int ok_s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(bar, 1ull);
+    int ok = 0;
+    for (int spin = 0; spin < (1 << 22); spin++) {
+      if (*((volatile unsigned long long *)bar) >= target) { ok = 1; break; }
+      if (spin > 64) __nanosleep(spin > 4096 ? 256 : 20);
+    }
+    if (!ok) atomicOr(status, HFX_ST_TIMEOUT);
+    __threadfence();
+    ok_s = ok;
+  }
+  __syncthreads();
+  return ok_s != 0;
+}
+
+// Column scan of the tile matrix by the whole grid.  A block takes 8 neighbouring columns (one
+// 32-byte sector of every matrix row): its 16 warps load them for all tiles (a lane = one of 4 tiles
+// x 8 columns, so every load instruction reads whole sectors), the block transposes them through
+// shared memory, one warp per column scans its tiles, and the prefixes go back the way they came.
+// M was written by other blocks of this kernel: L2 loads.  At most FRONT_TILES_MAX tiles.
+#define FRONT_TILES_MAX 512
+#define FRONT_LD (FRONT_TILES_MAX / (THREADS_TILE / 8))     // loads per thread
+__device__ __forceinline__ void colscan_grid(uint32_t *M, int32_t n_tiles, int32_t R1, uint32_t *tot_all, uint32_t *tot_act,
+                                             uint32_t *s_t /* [n_tiles][9] */) {
+  const int C = 2 * R1;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = threadIdx.x & 7, tsub = threadIdx.x >> 3;          // tsub in [0, 64)
+  for (int g = blockIdx.x; g * 8 < C; g += gridDim.x) {
+    const int col = g * 8 + c;
+    uint32_t x[FRONT_LD];
+#pragma unroll
+    for (int k = 0; k < FRONT_LD; k++) {
+      const int t = tsub + 64 * k;
+      x[k] = (t < n_tiles && col < C) ? __ldcg(M + (size_t)t * C + col) : 0u;
+    }
+#pragma unroll
+    for (int k = 0; k < FRONT_LD; k++) { const int t = tsub + 64 * k; if (t < n_tiles) s_t[t * 9 + c] = x[k]; }
+    __syncthreads();
+    if (warp < 8) {       // warp = column of the group; a lane scans a run of consecutive tiles
+      const int per = (n_tiles + 31) / 32;
+      const int t0 = lane * per < n_tiles ? lane * per : n_tiles, t1 = (t0 + per < n_tiles) ? t0 + per : n_tiles;
+      uint32_t sum = 0;
+      for (int t = t0; t < t1; t++) sum += s_t[t * 9 + warp];
+      uint32_t v = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+      uint32_t run = v - sum;
+      for (int t = t0; t < t1; t++) { const uint32_t y = s_t[t * 9 + warp]; s_t[t * 9 + warp] = run; run += y; }
+      const int wc = g * 8 + warp;
+      if (lane == 31 && wc < C) { if (wc < R1) tot_all[wc] = v; else tot_act[wc - R1] = v; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < FRONT_LD; k++) {
+      const int t = tsub + 64 * k;
+      if (t < n_tiles && col < C) M[(size_t)t * C + col] = s_t[t * 9 + c];
+    }
+    __syncthreads();
+  }
+}
+
+// Exclusive scan of the per-replica totals into shared memory (every block computes its own copy);
+// block 0 also publishes what the replica kernels and the caller read: seg_begin, seg_off, the
+// largest sort size, and it re-arms the next step's "ordered" word.
+__device__ __forceinline__ void offsets_local(const OffsetArgs &oa, uint32_t *s_segb /* [R+2] */, uint32_t *s_act /* [R+1] */) {
+  __shared__ uint32_t warp_tot[32], warp_max[32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const bool pub = blockIdx.x == 0;
+  const bool ordered = __ldcg(oa.flags + oa.parity) != 0;
+  const int total = oa.R + 1;
+  // each thread owns a run of consecutive replicas
+  const int per = (total + blockDim.x - 1) / blockDim.x;
+  const int i0 = threadIdx.x * per < total ? threadIdx.x * per : total, i1 = (i0 + per < total) ? i0 + per : total;
+  for (int i = threadIdx.x; i < total; i += blockDim.x) { s_segb[i] = __ldcg(oa.tot_all + i); s_act[i] = __ldcg(oa.tot_act + i); }
+  __syncthreads();
+  uint32_t sum = 0, mx = 0;
+  for (int i = i0; i < i1; i++) {
+    const uint32_t c = s_segb[i], act = s_act[i];
+    sum += c;
+    const uint32_t need = ordered ? act : (act > c - act ? act : c - act);
+    mx = need > mx ? need : mx;
+  }
+  uint32_t v = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { const uint32_t x = __shfl_xor_sync(0xffffffffu, mx, o); mx = x > mx ? x : mx; }
+  if (lane == 31) warp_tot[warp] = v;
+  if (lane == 0) warp_max[warp] = mx;
+  __syncthreads();
+  uint32_t run = v - sum, all = 0, mxall = 0;
+  for (int k = 0; k < nwarp; k++) { const uint32_t w = warp_tot[k]; if (k < warp) run += w; all += w; mxall = warp_max[k] > mxall ? warp_max[k] : mxall; }
+  for (int i = i0; i < i1; i++) {
+    const uint32_t c = s_segb[i];
+    s_segb[i] = run;
+    if (pub) { oa.seg_begin[i] = run; oa.seg_off[i] = (int32_t)run; }
+    run += c;
+  }
+  if (threadIdx.x == 0) {
+    s_segb[total] = all;
+    if (pub) { oa.seg_begin[total] = all; oa.flags[2] = mxall; oa.flags[oa.parity ^ 1u] = 1u; }
+  }
+  __syncthreads();
+}
+
+struct FrontArgs { unsigned long long *bar; unsigned long long target; uint32_t *status; int32_t n_tiles; };
+
+__global__ void __launch_bounds__(THREADS_TILE, 2) k_front(const HfxParams p, const CountArgs ca, const OffsetArgs oa,
+                                                           const RegroupArgs ra, const TileArgs ta0, const FrontArgs fa) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int R1 = p.n_replicas + 1;
+  count_tile(p, ca, reinterpret_cast<uint32_t *>(smem_raw));
+  if (!front_barrier(fa.bar, fa.target, fa.status)) return;
+  colscan_grid(ca.M, fa.n_tiles, R1, ca.tot_all, ca.tot_act, reinterpret_cast<uint32_t *>(smem_raw));
+  if (!front_barrier(fa.bar, fa.target + gridDim.x, fa.status)) return;
+  // the block's own copy of the range starts and active counts sits behind the regroup's arrays
+  uint32_t *s_segb = reinterpret_cast<uint32_t *>(smem_raw + hfx_regroup_smem_dev(R1, ta0.tile_rows));
+  uint32_t *s_act = s_segb + R1 + 1;
+  offsets_local(oa, s_segb, s_act);
+  TileArgs ta = ta0;
+  ta.seg_begin = s_segb; ta.tot_act = s_act;
+  regroup_tile(p, ra, ta, smem_raw);
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-size_t hfx_regroup_smem(int R1, int tile_rows) {
-  return sizeof(int64_t) * (size_t)R1 + sizeof(uint32_t) * (4 * (size_t)R1 + 1) + sizeof(uint16_t) * (2 * (size_t)tile_rows + 1) +
-         (size_t)R1 + 32;
+size_t hfx_regroup_smem(int R1, int tile_rows) { return hfx_regroup_smem_dev(R1, tile_rows); }
+
+// shared memory of the fused kernel: the regroup's arrays (the count's histograms reuse their space)
+// plus the block's copy of the offsets, or the column scan's slab if that is larger
+static size_t hfx_front_smem(int R1, int tile_rows, int n_tiles) {
+  const size_t regroup = hfx_regroup_smem_dev(R1, tile_rows) + sizeof(uint32_t) * (2 * (size_t)R1 + 2);
+  const size_t colscan = sizeof(uint32_t) * 9 * (size_t)n_tiles;      // the transposed 8-column slab of the column scan
+  return regroup > colscan ? regroup : colscan;
 }
 
 int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
@@ -607,7 +764,30 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
   ca.gen = ra.gen; ca.arrival = ra.arrival; ca.req_id = ra.req_id; ca.now = ra.now; ca.n = n; ca.tile_rows = tile_rows;
   ca.M = matrix ? s->d_tile_hist : nullptr; ca.tile_mode = s->d_tile_mode; ca.tot_all = s->d_seg_count;
   ca.tot_act = s->d_act_count; ca.rowflag = s->d_rowflag; ca.status = s->d_status; ca.ordered = ordered;
-  if (matrix) {
+  const size_t front_smem = hfx_front_smem(R1, tile_rows, n_tiles);
+  bool fused = matrix && s->front_enabled && front_smem <= 200 * 1024 && n_tiles <= FRONT_TILES_MAX;
+  if (fused) {     // every tile's block must be resident at once
+    if (s->front_smem_cached != front_smem) {
+      int per_sm = 0;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_front, THREADS_TILE, front_smem) != cudaSuccess) per_sm = 0;
+      s->front_smem_cached = front_smem;
+      s->front_capacity = per_sm * s->n_sm;
+    }
+    fused = n_tiles <= s->front_capacity;
+  }
+  if (fused) {
+    OffsetArgs oa = {s->d_seg_count, s->d_act_count, R, s->d_seg_begin, s->d_cursor, seg_off, s->d_flags, s->step_parity, 0u};
+    TileArgs ta;
+    ta.M = s->d_tile_hist; ta.tile_mode = s->d_tile_mode; ta.seg_begin = nullptr; ta.tot_act = nullptr;
+    ta.rowflag = s->d_rowflag; ta.ordered = ordered; ta.rec = s->d_rec; ta.tile_rows = tile_rows;
+    FrontArgs fa;
+    fa.bar = s->d_front_bar; fa.target = s->front_arrivals + (unsigned long long)n_tiles; fa.status = s->d_status; fa.n_tiles = n_tiles;
+    s->front_arrivals += 2ull * (unsigned long long)n_tiles;
+    void *args[] = {(void *)&s->p, (void *)&ca, (void *)&oa, (void *)&ra, (void *)&ta, (void *)&fa};
+    KernelScope ks(s, KSLOT_FRONT);
+    if (cudaLaunchCooperativeKernel((void *)k_front, dim3(n_tiles), dim3(THREADS_TILE), args, front_smem, stream) != cudaSuccess)
+      return HFX_E_CUDA;
+  } else if (matrix) {
     {
       KernelScope ks(s, KSLOT_COUNT);
       k_count<<<n_tiles, THREADS_TILE, sizeof(uint32_t) * 2 * R1, stream>>>(s->p, ca);
@@ -650,7 +830,8 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off) {
 }
 
 int hfx_regroup_configure() {
-  if (cudaFuncSetAttribute(k_regroup, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_regroup, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(k_front, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }

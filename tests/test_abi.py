@@ -48,7 +48,7 @@ def test_strerror_and_argument_checks_without_a_device():
     lib = hfx.load_library()
     assert lib.hfx_strerror(0) == b"ok" and b"aligned" in lib.hfx_strerror(-2)
     assert lib.hfx_strerror(-99) == b"unknown error"
-    assert lib.hfx_kernel_name(3) == b"k_regroup" and lib.hfx_kernel_name(9) is None
+    assert lib.hfx_kernel_name(3) == b"k_regroup" and lib.hfx_kernel_name(9) == b"k_front" and lib.hfx_kernel_name(10) is None
     import torch
     if not torch.cuda.is_available():
         # no device: the product path fails loudly, it never falls back to the CPU

@@ -81,6 +81,25 @@ def test_ragged_sizes_single_replica(n):
     assert_step_parity(wl, steps=2, commit=True)
 
 
+@pytest.mark.parametrize("seed", [0, 3, 5, 9])
+def test_separate_front_end_kernels(seed):
+    # the front end as separate kernels (what tables with more tiles than resident blocks use) gives
+    # the same results as the fused cooperative kernel that the other tests run
+    wl = gen.random_table(seed, 1000 + 997 * seed, 1 + (seed * 7) % 23, modes=MODES3, tie_heavy=seed % 3 == 0,
+                          batch_cap=(0, 7)[seed % 2], weight_max=(0, 16)[seed % 4 == 1], grouped=seed % 4 == 3)
+    sched = make_sched(wl)
+    sched.set_fused_front(False)
+    assert_step_parity(wl, steps=3, commit=True, sched=sched)
+    sched.set_fused_front(True)
+    assert_step_parity(wl, steps=2, commit=True, sched=sched)
+    sched.close()
+    wl = gen.config4(R=64, n=200_000, steps=3)
+    sched = make_sched(wl)
+    sched.set_fused_front(False)
+    assert_step_parity(wl, steps=3, commit=True, optional=False, sched=sched)
+    sched.close()
+
+
 def test_medium_and_oversize_segments():
     # 2048 < rows <= 16384: medium path; > 16384: global-sort path
     assert_step_parity(gen.random_table(7, 9000, 1, tie_heavy=True), steps=2, commit=True)
