@@ -89,6 +89,16 @@ class _ScaleParams(C.Structure):
                 ("eps_in_den", C.c_int32), ("eps_wait_num", C.c_int32), ("eps_wait_den", C.c_int32)]
 
 
+_DISPATCH_OUT = [("assign", np.int32, "n"), ("queue_order", np.int32, "n"), ("n_queue", np.int32, "1"),
+                 ("inst_order", np.int32, "R"), ("n_mature", np.int32, "1"), ("slack", np.int64, "n"),
+                 ("budget", np.int64, "R"), ("e_d", np.int64, "R"), ("n_run", np.int32, "R"), ("sum_kv", np.int64, "R"),
+                 ("adm_cost", np.int64, "R"), ("adm_count", np.int32, "R"), ("maturity_next", np.int64, "R")]
+
+
+class _DispatchOut(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k, _, _ in _DISPATCH_OUT]
+
+
 class _ScaleOut(C.Structure):
     _fields_ = [("counts", C.c_void_p), ("used_blocks", C.c_void_p), ("decision", C.c_void_p)]
 
@@ -118,6 +128,8 @@ def lib():
         L.ora_sim.restype = C.c_uint32
         L.ora_sim.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p, C.c_int32, C.c_int32,
                               C.c_int32, C.POINTER(_SimOut)]
+        L.ora_dispatch.restype = C.c_uint32
+        L.ora_dispatch.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_DispatchOut)]
         L.ora_scale.restype = C.c_uint32
         L.ora_scale.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_ScaleParams),
                                 C.POINTER(_ScaleOut)]
@@ -202,6 +214,26 @@ def sim(wl, iters: Optional[int] = None, j0: int = 0, j1: Optional[int] = None) 
     off = np.ascontiguousarray(wl.trace_off, np.int32)
     st = L.ora_sim(C.byref(ctx.cfg), C.byref(ctx.table), off.ctypes.data, j0, j1,
                    int(wl.sim_iters if iters is None else iters), C.byref(so))
+    out["status"] = int(st)
+    return out
+
+
+def dispatch(wl, now: int) -> Dict[str, np.ndarray]:
+    """The dispatching steps over the shared global queue at time `now`: every instance of wl whose
+    maturity (wl.maturity) has come takes its turn once, in maturity order.  Nothing in wl changes."""
+    L = lib()
+    ctx = _Ctx(wl)
+    n, R = wl.n_rows, wl.n_replicas
+    out = {}
+    so = _DispatchOut()
+    for k, dt, dim in _DISPATCH_OUT:
+        out[k] = np.zeros({"n": max(n, 1), "R": R, "1": 1}[dim], dt)
+        setattr(so, k, out[k].ctypes.data)
+    mat = np.ascontiguousarray(wl.maturity, np.int64)
+    st = L.ora_dispatch(C.byref(ctx.cfg), C.byref(ctx.table), int(now), mat.ctypes.data, C.byref(so))
+    for k, dt, dim in _DISPATCH_OUT:
+        if dim == "n":
+            out[k] = out[k][:n]
     out["status"] = int(st)
     return out
 

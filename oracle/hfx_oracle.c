@@ -632,3 +632,159 @@ uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const i
   }
   return status;
 }
+
+/* ==========================================================================
+ * Dispatching over a shared global queue (Sec. 3.3.1, colocated mode, the four
+ * dispatching steps as the paper lists them): (1) take the instance whose
+ * maturity time arrives first, (2) compute its safe token budget, (3) scan the
+ * global request queue for the most urgent requests that fit within it,
+ * (4) dispatch them and update the instance's maturity time; repeat with the
+ * next instance.  Here one call makes the decisions that are due at time `now`:
+ * every instance that has matured takes its turn once, in maturity order.
+ *
+ * reading: a request belongs to the global queue while it is QUEUED and has
+ *   arrived (its replica_id is not looked at); in-flight requests count for the
+ *   instance they run on.
+ * reading: the queue is ordered by (priority, remaining slack, req_id) with
+ *   slack = TTFT - (now - arrival) - E_p(prompt_len), the request starting at
+ *   once on an instance that has matured.
+ * reading: the TTFT of Eq. 3 is the strictest TTFT in the queue as it stands
+ *   when the call begins; the TPOT is the strictest among the instance's
+ *   in-flight requests.
+ * reading: "requests that fit" -- each instance takes the run of consecutive
+ *   queue entries, from where the previous instance stopped, whose total stays
+ *   within its budget and batch cap, and stops at the first that does not fit
+ *   (that request waits at the head for the next instance).  A prompt longer
+ *   than every instance's token cap can never be served and is left out of the
+ *   queue.
+ * reading: instances tie on maturity in index order.
+ * ========================================================================== */
+typedef struct {
+  int32_t *assign;        /* [n] instance a queued row is dispatched to, else -1         */
+  int32_t *queue_order;   /* [n] rows of the queue, most urgent first; -1 past n_queue   */
+  int32_t *n_queue;       /* [1]                                                         */
+  int32_t *inst_order;    /* [R] matured instances in dispatch order; -1 past n_mature   */
+  int32_t *n_mature;      /* [1]                                                         */
+  int64_t *slack;         /* [n] slack of queue rows, 0 elsewhere                        */
+  int64_t *budget;        /* [R] safe token budget (0 for an instance not matured)       */
+  int64_t *e_d;           /* [R] */
+  int32_t *n_run;         /* [R] */
+  int64_t *sum_kv;        /* [R] */
+  int64_t *adm_cost;      /* [R] tokens dispatched to the instance                       */
+  int32_t *adm_count;     /* [R] requests dispatched to the instance                     */
+  int64_t *maturity_next; /* [R] */
+} ora_dispatch_out;
+
+typedef struct { int64_t mat; int32_t id; } inst_tuple;
+static int cmp_inst(const void *pa, const void *pb) {
+  const inst_tuple *a = (const inst_tuple *)pa, *b = (const inst_tuple *)pb;
+  if (a->mat != b->mat) return a->mat < b->mat ? -1 : 1;
+  return a->id < b->id ? -1 : (a->id > b->id ? 1 : 0);
+}
+
+uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, const int64_t *maturity,
+                      const ora_dispatch_out *o) {
+  const ora_model *M = &c->model;
+  const int32_t R = c->n_replicas;
+  const int64_t n = t->n;
+  uint32_t status = 0;
+  int64_t *n_run = (int64_t *)calloc((size_t)R + 1, sizeof(int64_t));
+  int64_t *sum_kv = (int64_t *)calloc((size_t)R + 1, sizeof(int64_t));
+  int64_t *min_tpot = (int64_t *)malloc(sizeof(int64_t) * ((size_t)R + 1));
+  sort_tuple *q = (sort_tuple *)malloc(sizeof(sort_tuple) * (size_t)(n + 1));
+  inst_tuple *inst = (inst_tuple *)malloc(sizeof(inst_tuple) * ((size_t)R + 1));
+  int32_t cap_max = 0;
+  for (int32_t r = 0; r < R; r++) {
+    min_tpot[r] = ORA_INF;
+    if (c->replicas[r].token_cap > cap_max) cap_max = c->replicas[r].token_cap;
+  }
+
+  /* in-flight requests: the running batch of each instance; the queue */
+  int64_t nq = 0, min_ttft = ORA_INF;
+  for (int64_t i = 0; i < n; i++) {
+    o->assign[i] = -1;
+    o->slack[i] = 0;
+    o->queue_order[i] = -1;
+    if (!row_valid(c, t, i, &status)) continue;
+    const ora_class *k = &c->classes[t->class_id[i]];
+    if (t->state[i] == ST_RUNNING) {
+      const int32_t r = t->replica_id[i];
+      if (r < 0 || r >= R) { status |= BAD_REPLICA; continue; }
+      n_run[r] += 1;
+      sum_kv[r] += (int64_t)t->prompt_len[i] + t->gen[i];
+      if (k->tpot > 0 && k->tpot < min_tpot[r]) min_tpot[r] = k->tpot;
+    } else if (t->state[i] == ST_QUEUED && t->arrival[i] <= now && t->prompt_len[i] <= cap_max) {
+      const int64_t pred_ttft = (now - t->arrival[i]) + ora_Ep(M, t->prompt_len[i]);
+      const int64_t sl = k->ttft > 0 ? k->ttft - pred_ttft : ORA_SLACK_MAX;
+      int32_t prio;
+      if (c->weight_max > 0) {
+        int64_t p = (int64_t)c->weight_max - t->weight[i];
+        prio = (int32_t)(p < 0 ? 0 : (p > 62 ? 62 : p));
+      } else prio = k->prio;
+      o->slack[i] = sl;
+      q[nq].phase = PH_QUEUED; q[nq].prio = prio; q[nq].cslack = clamp_slack(sl);
+      q[nq].req_id = t->req_id[i]; q[nq].row = i;
+      nq++;
+      if (k->ttft > 0 && k->ttft < min_ttft) min_ttft = k->ttft;
+    }
+  }
+  qsort(q, (size_t)nq, sizeof(sort_tuple), cmp_tuple);
+  for (int64_t j = 0; j < nq; j++) o->queue_order[j] = (int32_t)q[j].row;
+  *o->n_queue = (int32_t)nq;
+
+  /* step 2 for every instance that has matured; step 1: their order */
+  int32_t nm = 0;
+  for (int32_t r = 0; r < R; r++) {
+    const ora_replica *cfg = &c->replicas[r];
+    const int64_t e_d = n_run[r] > 0 ? ora_Ed(M, n_run[r], sum_kv[r]) : 0;
+    int64_t budget = 0;
+    if (maturity[r] <= now) {
+      int64_t n_safe;
+      if (c->budget_mode == BUDGET_CAP_ONLY) n_safe = cfg->token_cap;
+      else n_safe = ora_nsafe(M, ora_epmax(min_ttft, n_run[r] > 0 && min_tpot[r] < ORA_INF, min_tpot[r], e_d), cfg->token_cap);
+      const int64_t cap_left = cfg->token_cap - n_run[r] > 0 ? cfg->token_cap - n_run[r] : 0;
+      budget = n_safe < cap_left ? n_safe : cap_left;
+      inst[nm].mat = maturity[r]; inst[nm].id = r; nm++;
+    }
+    o->budget[r] = budget;
+    o->e_d[r] = e_d;
+    o->n_run[r] = (int32_t)n_run[r];
+    o->sum_kv[r] = sum_kv[r];
+    o->adm_cost[r] = 0;
+    o->adm_count[r] = 0;
+    o->maturity_next[r] = maturity[r];
+    o->inst_order[r] = -1;
+  }
+  qsort(inst, (size_t)nm, sizeof(inst_tuple), cmp_inst);
+  for (int32_t k = 0; k < nm; k++) o->inst_order[k] = inst[k].id;
+  *o->n_mature = nm;
+
+  /* steps 3 and 4, instance by instance */
+  int64_t cursor = 0;
+  for (int32_t k = 0; k < nm; k++) {
+    const int32_t r = inst[k].id;
+    const ora_replica *cfg = &c->replicas[r];
+    int64_t cost = 0, count = 0;
+    while (cursor < nq) {
+      const int64_t i = q[cursor].row;
+      if (cost + t->prompt_len[i] > o->budget[r]) break;
+      if (cfg->batch_cap != 0 && n_run[r] + count + 1 > cfg->batch_cap) break;
+      cost += t->prompt_len[i];
+      count += 1;
+      o->assign[i] = r;
+      cursor++;
+    }
+    o->adm_cost[r] = cost;
+    o->adm_count[r] = (int32_t)count;
+    if (count > 0) {
+      /* Maturity = E_p + k*E_d as in the per-instance step */
+      const int64_t lp = ora_Ep(M, cost), e_d = o->e_d[r];
+      i128 kk = 0;
+      if (n_run[r] > 0 && min_tpot[r] < ORA_INF && min_tpot[r] > e_d) kk = ((i128)lp + (min_tpot[r] - e_d) - 1) / (min_tpot[r] - e_d);
+      i128 v = (i128)now + lp + kk * e_d;
+      o->maturity_next[r] = v > ORA_TIME_MAX ? ORA_TIME_MAX : (int64_t)v;
+    }
+  }
+  free(n_run); free(sum_kv); free(min_tpot); free(q); free(inst);
+  return status;
+}

@@ -323,3 +323,49 @@ def test_scaling_indicators_hand_worked():
     assert list(o["decision"][0]) == [-1, 1]
     o = oracle.scale_tick(wl, 20 * S, np.array([1000, 100]), min_samples=2)     # 3/1000 vs 0/100: still instance 1
     assert list(o["used_blocks"]) == [3, 0] and list(o["decision"][0]) == [-1, 1]
+
+
+# ---- dispatching over the shared global queue -------------------------------------------------------
+def _dispatch_hand_case():
+    now = 1000 * MS
+    classes = [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)]
+    rows = [dict(state=1, replica_id=0, prompt_len=800, gen=0, output_len=500, arrival_ns=0, first_token_ns=now - 30 * MS)
+            for _ in range(80)]
+    rows += [dict(replica_id=-1, class_id=0, prompt_len=1000, arrival_ns=now - 10 * MS),    # q1  row 80
+             dict(replica_id=-1, class_id=0, prompt_len=1144, arrival_ns=now - 50 * MS),    # q2  row 81
+             dict(replica_id=-1, class_id=1, prompt_len=281, arrival_ns=now - 900 * MS),    # q3  row 82
+             dict(replica_id=-1, class_id=0, prompt_len=16, arrival_ns=now - 1 * MS),       # q4  row 83
+             dict(replica_id=-1, class_id=1, prompt_len=2000, arrival_ns=now - 100 * MS),   # q5  row 84
+             dict(replica_id=-1, class_id=0, prompt_len=16, arrival_ns=now + 1)]            # not arrived yet
+    wl = make_wl(rows, classes, replicas=[(gen.COLOCATED, 8192, 0)] * 3, now=[now] * 3,
+                 maturity=[now - 5, now - 10, now + 1])
+    return wl, now
+
+
+def test_dispatch_global_queue_hand_worked():
+    wl, now = _dispatch_hand_case()
+    o = oracle.dispatch(wl, now)
+    assert o["status"] == 0
+    assert o["n_queue"][0] == 5 and list(o["queue_order"][:5]) == [81, 80, 83, 82, 84] and o["queue_order"][5] == -1
+    assert o["slack"][80] == PINS["slack_queued"] and o["slack"][81] == PINS["disp_slack_q2"]
+    assert o["slack"][82] == PINS["disp_slack_q3"] and o["slack"][83] == PINS["disp_slack_q4"]
+    assert o["slack"][84] == PINS["disp_slack_q5"] and o["slack"][85] == 0 and o["slack"][0] == 0
+    assert o["n_mature"][0] == 2 and list(o["inst_order"]) == [1, 0, -1]
+    assert list(o["budget"]) == [PINS["nsafe_busy"], PINS["nsafe_idle"], 0]
+    assert list(o["n_run"]) == [80, 0, 0] and o["e_d"][0] == PINS["Ed_80_64000"] and o["e_d"][1] == 0
+    assert list(o["assign"][80:86]) == [1, 1, 0, 0, -1, -1] and np.all(o["assign"][:80] == -1)
+    assert list(o["adm_cost"]) == [297, 2144, 0] and list(o["adm_count"]) == [2, 2, 0]
+    assert o["maturity_next"][1] - now == PINS["disp_mat1_delta"]
+    assert o["maturity_next"][0] - now == PINS["disp_mat0_delta"]
+    assert o["maturity_next"][2] == now + 1
+
+
+def test_dispatch_batch_cap_stops_a_run_and_oversize_prompts_leave_the_queue():
+    wl, now = _dispatch_hand_case()
+    wl.replicas[1, 2] = 1                      # the idle instance may hold one request
+    wl.table["prompt_len"][84] = 9000          # longer than every token cap: can never be served
+    o = oracle.dispatch(wl, now)
+    assert o["n_queue"][0] == 4 and list(o["queue_order"][:4]) == [81, 80, 83, 82]
+    # instance 1 takes q2 and is full; instance 0 (budget 1281) takes q1 + q4 = 1016, q3 would make 1297
+    assert list(o["assign"][80:86]) == [0, 1, -1, 0, -1, -1]
+    assert list(o["adm_cost"]) == [1016, 1144, 0] and list(o["adm_count"]) == [2, 1, 0]

@@ -258,3 +258,79 @@ def test_configs_smoke():
     full = gen.config5(traces=3, rows_per=64, iters=10)
     part = gen.config5(traces=1, rows_per=64, iters=10, first_trace=2)
     assert np.array_equal(full.table["arrival_ns"][128:], part.table["arrival_ns"])
+
+
+# ---- dispatching over the shared global queue -------------------------------------------------------
+def _dispatch_case(seed, **kw):
+    wl = gen.random_table(seed, 60 + 37 * seed, 1 + seed % 6, modes=(gen.COLOCATED,), token_cap=(4096, 600)[seed % 2], **kw)
+    return wl, int(wl.now.max())
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_dispatch_invariants(seed):
+    wl, now = _dispatch_case(seed, batch_cap=(0, 12)[seed % 3 == 1], tie_heavy=seed % 4 == 2,
+                             budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 3])
+    o = oracle.dispatch(wl, now)
+    t, R = wl.table, wl.n_replicas
+    nq, nm = int(o["n_queue"][0]), int(o["n_mature"][0])
+    cap_max = int(wl.replicas[:, 1].max())
+    queue = o["queue_order"][:nq]
+    # the queue is exactly the visible, valid, servable QUEUED rows
+    vis = (t["state"] == 0) & (t["arrival_ns"] <= now) & (t["prompt_len"] <= cap_max) & (t["class_id"] < len(wl.classes))
+    assert sorted(queue.tolist()) == np.nonzero(vis)[0].tolist() and np.all(o["queue_order"][nq:] == -1)
+    # instances take their turn in maturity order, only once matured
+    mature = np.nonzero(wl.maturity <= now)[0]
+    assert nm == mature.size and sorted(o["inst_order"][:nm].tolist()) == mature.tolist()
+    mo = wl.maturity[o["inst_order"][:nm]]
+    assert np.all(np.diff(mo) >= 0)
+    # consecutive runs of the queue, in instance order; each within budget and batch cap, each maximal
+    cursor = 0
+    for r in o["inst_order"][:nm]:
+        cnt, cost = int(o["adm_count"][r]), int(o["adm_cost"][r])
+        rows = queue[cursor:cursor + cnt]
+        assert np.all(o["assign"][rows] == r) and int(t["prompt_len"][rows].sum()) == cost
+        assert cost <= o["budget"][r] <= wl.replicas[r, 1]
+        cap = int(wl.replicas[r, 2])
+        assert cap == 0 or cnt == 0 or o["n_run"][r] + cnt <= cap
+        cursor += cnt
+        if cursor < nq:
+            nxt = int(t["prompt_len"][queue[cursor]])
+            assert cost + nxt > o["budget"][r] or (cap != 0 and o["n_run"][r] + cnt + 1 > cap)
+        assert (o["maturity_next"][r] > now) == (cnt > 0) or cnt == 0
+    assert np.all(o["assign"][queue[cursor:]] == -1)
+    for r in range(R):
+        if wl.maturity[r] > now:
+            assert o["budget"][r] == 0 and o["adm_count"][r] == 0 and o["maturity_next"][r] == wl.maturity[r]
+    assert np.count_nonzero(o["assign"] >= 0) == int(o["adm_count"].sum())
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_dispatch_invariant_under_row_permutation(seed):
+    wl, now = _dispatch_case(seed, tie_heavy=seed % 2 == 1)
+    a = oracle.dispatch(wl, now)
+    perm = np.random.default_rng(100 + seed).permutation(wl.n_rows)
+    wp = permute_rows(wl, perm)
+    b = oracle.dispatch(wp, now)
+    ida, idb = wl.table["req_id"], wp.table["req_id"]
+    nq = int(a["n_queue"][0])
+    assert nq == int(b["n_queue"][0]) and np.array_equal(ida[a["queue_order"][:nq]], idb[b["queue_order"][:nq]])
+    assert dict(zip(ida.tolist(), a["assign"].tolist())) == dict(zip(idb.tolist(), b["assign"].tolist()))
+    assert dict(zip(ida.tolist(), a["slack"].tolist())) == dict(zip(idb.tolist(), b["slack"].tolist()))
+    for k in ("budget", "adm_cost", "adm_count", "maturity_next", "inst_order", "n_run", "sum_kv", "e_d"):
+        assert np.array_equal(a[k], b[k]), k
+
+
+def test_dispatch_single_instance_equals_the_per_replica_step_without_skips():
+    # one matured instance, every queued prompt small enough to fit alone, all rows bound to it:
+    # the per-replica step admits the same prefix of the same order with the same budget and maturity
+    wl = gen.random_table(5, 300, 1, modes=(gen.COLOCATED,), token_cap=4096)
+    wl.table["prompt_len"][:] = np.minimum(wl.table["prompt_len"], 40)
+    wl.maturity[:] = wl.now - 1
+    now = int(wl.now[0])
+    d = oracle.dispatch(wl, now)
+    s = oracle.step(wl)
+    assert d["budget"][0] == s["budget"][0] and d["adm_count"][0] == s["adm_count"][0] > 0
+    assert d["adm_cost"][0] == s["adm_cost"][0] and d["maturity_next"][0] == s["maturity_next"][0]
+    queued = (wl.table["state"] == 0) & (wl.table["arrival_ns"] <= now)
+    assert np.array_equal(d["assign"][queued] == 0, s["admit"][queued] == 1)
+    assert np.array_equal(d["slack"][queued], s["slack"][queued])
