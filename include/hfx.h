@@ -231,6 +231,50 @@ int hfx_sched_step(hfx_sched *s, const hfx_table *table,
                    const hfx_replica_state *state, const hfx_step_out *out,
                    uint32_t flags);
 
+/* Outputs of hfx_dispatch_step; every member is a device pointer.  n = rows of
+ * the table, R = replicas of the scheduler. */
+typedef struct hfx_dispatch_out {
+  int32_t *assign;         /* [n] instance a queued row is dispatched to, else -1 */
+  int32_t *queue_order;    /* [n] rows of the queue, most urgent first; -1 past n_queue */
+  int32_t *n_queue;        /* [1] */
+  int32_t *inst_order;     /* [R] matured instances in dispatch order; -1 past n_mature */
+  int32_t *n_mature;       /* [1] */
+  int64_t *slack_ns;       /* [n] slack of queue rows, 0 elsewhere */
+  int64_t *budget;         /* [R] safe token budget; 0 for an instance not matured */
+  int64_t *e_d_ns;         /* [R] */
+  int32_t *n_run;          /* [R] */
+  int64_t *sum_kv;         /* [R] */
+  int64_t *adm_cost;       /* [R] tokens dispatched to the instance */
+  int32_t *adm_count;      /* [R] requests dispatched to the instance */
+  int64_t *maturity_next;  /* [R] */
+} hfx_dispatch_out;
+
+/* The four dispatching steps of Sec. 3.3.1 (colocated mode) over a shared
+ * global queue, for the decisions due at time now_ns: (1) the instances whose
+ * maturity time (maturity_ns, device, [R]) has come take their turn once each,
+ * earliest maturity first, ties in index order; (2) each gets its safe token
+ * budget (Eq. 3) from the strictest TTFT in the queue as it stands when the
+ * call begins and the strictest TPOT among its own in-flight requests;
+ * (3) the queue -- every QUEUED row that has arrived, whatever its replica_id,
+ * ordered by (priority, slack, req_id) with slack = TTFT - (now - arrival) -
+ * E_p(prompt_len) -- is handed out in order: an instance takes entries from
+ * where the previous one stopped while their total stays within its budget
+ * and batch room, and stops at the first that does not fit (it waits at the
+ * head for the next instance); an entry larger than the largest budget of
+ * the call fits nowhere now and is passed over; (4) an instance that took
+ * requests gets the maturity time E_p + k E_d of the per-replica step.
+ * RUNNING rows count for the instance in their replica_id.  A prompt longer
+ * than every instance's token_cap can never be served and is left out of the
+ * queue.  The table is not changed; the caller binds the dispatched rows
+ * (replica_id := assign) before the next hfx_sched_step.
+ * Every replica of the scheduler must be HFX_COLOCATED, and there may be at
+ * most 4096 of them.  The first call allocates the call's workspace (44 bytes
+ * per row of max_rows) with cudaMalloc, so it should not be made inside a
+ * stream capture; hfx_sched_destroy frees it.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_NOMEM, HFX_E_CUDA. */
+int hfx_dispatch_step(hfx_sched *s, const hfx_table *table, int64_t now_ns,
+                      const int64_t *maturity_ns, const hfx_dispatch_out *out);
+
 /* Trace-driven simulation (events are request arrivals and iteration
  * completions, Problem Definition; metrics are Eq. 2 and the TTFT / TPOT
  * definitions).  `table` holds n_traces traces back to back, trace j being
@@ -292,9 +336,10 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * stream, adds the elapsed times of all brackets recorded since the last call
  * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
  * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
- * 6 oversize path, 7 simulator, 8 scaler tick, 9 fused front end; hfx_kernel_name
- * gives the name of a slot (NULL past the end). */
-#define HFX_N_KERNELS 10
+ * 6 oversize path, 7 simulator, 8 scaler tick, 9 fused front end, 10 the kernels of
+ * hfx_dispatch_step together; hfx_kernel_name gives the name of a slot (NULL past
+ * the end). */
+#define HFX_N_KERNELS 11
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
   int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */

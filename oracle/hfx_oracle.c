@@ -651,12 +651,14 @@ uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const i
  * reading: the TTFT of Eq. 3 is the strictest TTFT in the queue as it stands
  *   when the call begins; the TPOT is the strictest among the instance's
  *   in-flight requests.
- * reading: "requests that fit" -- each instance takes the run of consecutive
- *   queue entries, from where the previous instance stopped, whose total stays
- *   within its budget and batch cap, and stops at the first that does not fit
- *   (that request waits at the head for the next instance).  A prompt longer
- *   than every instance's token cap can never be served and is left out of the
- *   queue.
+ * reading: "requests that fit" -- each instance takes queue entries in order,
+ *   from where the previous instance stopped, while their total stays within
+ *   its budget and batch cap, and stops at the first that does not fit (that
+ *   request waits at the head for the next instance).  An entry larger than
+ *   the largest budget any matured instance has in this call fits nowhere now:
+ *   it is passed over and stays queued, so it never blocks the entries behind
+ *   it.  A prompt longer than every instance's token cap can never be served
+ *   and is left out of the queue.
  * reading: instances tie on maturity in index order.
  * ========================================================================== */
 typedef struct {
@@ -760,6 +762,8 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
   *o->n_mature = nm;
 
   /* steps 3 and 4, instance by instance */
+  int64_t budget_max = 0;
+  for (int32_t k = 0; k < nm; k++) if (o->budget[inst[k].id] > budget_max) budget_max = o->budget[inst[k].id];
   int64_t cursor = 0;
   for (int32_t k = 0; k < nm; k++) {
     const int32_t r = inst[k].id;
@@ -767,6 +771,7 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
     int64_t cost = 0, count = 0;
     while (cursor < nq) {
       const int64_t i = q[cursor].row;
+      if (t->prompt_len[i] > budget_max) { cursor++; continue; }   /* fits no instance in this call */
       if (cost + t->prompt_len[i] > o->budget[r]) break;
       if (cfg->batch_cap != 0 && n_run[r] + count + 1 > cfg->batch_cap) break;
       cost += t->prompt_len[i];

@@ -21,9 +21,9 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick"]
+                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step"]
 NOALLOC_MAX_REPLICAS = 4096
-N_KERNELS = 10
+N_KERNELS = 11
 
 
 class HfxError(RuntimeError):
@@ -82,7 +82,7 @@ SIM_OUT_FIELDS = [("iters_executed", torch.int32), ("finished", torch.int32), ("
 
 
 class _Profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 10), ("launches", C.c_int64 * 10)]
+    _fields_ = [("ms", C.c_double * 11), ("launches", C.c_int64 * 11)]
 
 
 class _ScaleParams(C.Structure):
@@ -97,6 +97,17 @@ class _ScaleOut(C.Structure):
 
 class _SimOut(C.Structure):
     _fields_ = [(k, C.c_void_p) for k, _ in SIM_OUT_FIELDS]
+
+
+DISPATCH_OUT_FIELDS = [("assign", torch.int32, "n"), ("queue_order", torch.int32, "n"), ("n_queue", torch.int32, "1"),
+                       ("inst_order", torch.int32, "R"), ("n_mature", torch.int32, "1"), ("slack_ns", torch.int64, "n"),
+                       ("budget", torch.int64, "R"), ("e_d_ns", torch.int64, "R"), ("n_run", torch.int32, "R"),
+                       ("sum_kv", torch.int64, "R"), ("adm_cost", torch.int64, "R"), ("adm_count", torch.int32, "R"),
+                       ("maturity_next", torch.int64, "R")]
+
+
+class _DispatchOut(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k, _, _ in DISPATCH_OUT_FIELDS]
 
 
 def library_path() -> str:
@@ -117,6 +128,8 @@ def load_library():
                                    C.POINTER(_ReplicaCfg), C.c_int, C.c_int64, C.POINTER(_Options), C.c_void_p]
     L.hfx_sched_step.restype = C.c_int
     L.hfx_sched_step.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_ReplicaState), C.POINTER(_StepOut), C.c_uint32]
+    L.hfx_dispatch_step.restype = C.c_int
+    L.hfx_dispatch_step.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_DispatchOut)]
     L.hfx_sim_run.restype = C.c_int
     L.hfx_sim_run.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_SimOut)]
     L.hfx_sched_status.restype = C.c_int
@@ -222,6 +235,28 @@ class StepOut:
         return out
 
 
+class DispatchOut:
+    """Output buffers of hfx_dispatch_step (allocated once, reused)."""
+
+    def __init__(self, n_rows: int, n_replicas: int, device="cuda"):
+        self.t = {k: torch.zeros({"n": max(n_rows, 1), "R": n_replicas, "1": 4}[dim], dtype=dt, device=device)
+                  for k, dt, dim in DISPATCH_OUT_FIELDS}
+        self.n_rows = n_rows
+
+    def c_struct(self) -> _DispatchOut:
+        s = _DispatchOut()
+        for k, _, _ in DISPATCH_OUT_FIELDS:
+            setattr(s, k, _ptr(self.t[k]))
+        return s
+
+    def to_numpy(self) -> Dict[str, np.ndarray]:
+        out = {}
+        for k, _, dim in DISPATCH_OUT_FIELDS:
+            a = self.t[k].cpu().numpy()
+            out[k] = a[:self.n_rows] if dim == "n" else (a[:1] if dim == "1" else a)
+        return out
+
+
 class SimOut:
     def __init__(self, n_traces: int, device="cuda"):
         self.t = {k: torch.zeros(max(n_traces, 1), dtype=dt, device=device) for k, dt in SIM_OUT_FIELDS}
@@ -281,6 +316,13 @@ class Scheduler:
         rc = self._L.hfx_sim_run(self._h, C.byref(ts), off.ctypes.data, int(off.shape[0] - 1), int(iters), C.byref(os_))
         if rc != 0:
             raise HfxError(rc, "hfx_sim_run")
+
+    def dispatch_step(self, table: DeviceTable, now_ns: int, maturity: torch.Tensor, out: DispatchOut):
+        """hfx_dispatch_step: the dispatching steps over the shared global queue at time now_ns."""
+        ts, os_ = table.c_struct(), out.c_struct()
+        rc = self._L.hfx_dispatch_step(self._h, C.byref(ts), int(now_ns), _ptr(maturity), C.byref(os_))
+        if rc != 0:
+            raise HfxError(rc, "hfx_dispatch_step")
 
     def scale_tick(self, table: DeviceTable, now_ns: int, total_blocks: torch.Tensor, counts: torch.Tensor,
                    used_blocks: torch.Tensor, decision: torch.Tensor, window_ns: int = 10_000_000_000,

@@ -7,6 +7,7 @@
 int hfx_regroup_configure();
 int hfx_segment_configure();
 int hfx_sim_configure();
+int hfx_dispatch_configure();
 int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_trace_off, int32_t n_traces,
                           int32_t max_trace_rows, int32_t iters, const hfx_sim_out *o, uint32_t *d_work_counter);
 
@@ -66,7 +67,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     cudaGetLastError();
     return HFX_E_CUDA;
   }
-  if (hfx_regroup_configure() != HFX_OK || hfx_segment_configure() != HFX_OK || hfx_sim_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
+  if (hfx_regroup_configure() != HFX_OK || hfx_segment_configure() != HFX_OK || hfx_sim_configure() != HFX_OK || hfx_dispatch_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
 
   hfx_sched_host *h = new (std::nothrow) hfx_sched_host();
   if (!h) return HFX_E_NOMEM;
@@ -151,6 +152,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   if (!s) return;
   hfx_sched_host *h = reinterpret_cast<hfx_sched_host *>(s);
   cudaStreamSynchronize(s->stream);
+  hfx_dispatch_release(s);
   if (s->side) { cudaStreamSynchronize(s->side); cudaStreamDestroy(s->side); }
   if (s->ev_fork) cudaEventDestroy(s->ev_fork);
   if (s->ev_join) cudaEventDestroy(s->ev_join);
@@ -192,6 +194,33 @@ extern "C" int hfx_sched_step(hfx_sched *s, const hfx_table *t, const hfx_replic
                        o->adm_count, o->maturity_next};
   for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
   return hfx_launch_step(s, t, st, o, flags);
+}
+
+extern "C" int hfx_dispatch_step(hfx_sched *s, const hfx_table *t, int64_t now_ns, const int64_t *maturity_ns,
+                                 const hfx_dispatch_out *o) {
+  if (!s || !t || !maturity_ns || !o) return HFX_E_ARG;
+  hfx_sched_host *h = reinterpret_cast<hfx_sched_host *>(s);
+  if (t->n_rows < 0) return HFX_E_ARG;
+  if (t->n_rows > s->max_rows || s->p.n_replicas > 4096) return HFX_E_CAPACITY;
+  const void *need_rep[] = {o->n_queue, o->inst_order, o->n_mature, o->budget, o->e_d_ns, o->n_run, o->sum_kv, o->adm_cost,
+                            o->adm_count, o->maturity_next};
+  for (const void *p : need_rep) if (!p) return HFX_E_ARG;
+  if (t->n_rows > 0) {
+    const void *need_row[] = {t->replica_id, t->class_id, t->state, t->prompt_len, t->gen, t->arrival_ns, t->req_id,
+                              o->assign, o->queue_order, o->slack_ns};
+    for (const void *p : need_row) if (!p) return HFX_E_ARG;
+    if (s->p.weight_max > 0 && !t->weight) return HFX_E_ARG;
+  }
+  const void *all[] = {t->replica_id, t->class_id, t->state, t->prompt_len, t->gen, t->arrival_ns, t->req_id, t->weight,
+                       maturity_ns, o->assign, o->queue_order, o->n_queue, o->inst_order, o->n_mature, o->slack_ns, o->budget,
+                       o->e_d_ns, o->n_run, o->sum_kv, o->adm_cost, o->adm_count, o->maturity_next};
+  for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
+  int32_t cap_max = 0;
+  for (int r = 0; r < s->p.n_replicas; r++) {
+    if (h->h_cfg[r].mode != HFX_COLOCATED) return HFX_E_ARG;
+    if (h->h_cfg[r].token_cap > cap_max) cap_max = h->h_cfg[r].token_cap;
+  }
+  return hfx_launch_dispatch(s, t, now_ns, maturity_ns, o, cap_max);
 }
 
 extern "C" int hfx_sim_run(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
@@ -275,6 +304,6 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 
 extern "C" const char *hfx_kernel_name(int slot) {
   static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
-                                "k_big", "k_sim", "k_scale", "k_front"};
-  return (slot >= 0 && slot < 10) ? names[slot] : nullptr;
+                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch"};
+  return (slot >= 0 && slot < 11) ? names[slot] : nullptr;
 }

@@ -1,0 +1,571 @@
+// hfx_dispatch_step: the four dispatching steps of Sec. 3.3.1 over a shared global queue, for every
+// instance whose maturity time has come, in maturity order.
+//
+//   k_disp_scan     one streaming pass over the table: the running batch of every instance (count,
+//                   context tokens, classes), and the visible queue: slack, priority key, and an
+//                   unordered list of (request id, row) pairs
+//   radix passes    the queue ordered by (priority, slack, request id): a stable least-significant-
+//                   digit radix sort, 8 bits a pass, first on the request id, then on the 48-bit key
+//   k_disp_plan     E_d and the safe token budget (Eq. 3) of every instance; the largest budget
+//   k_disp_prefix   the queue's rows in order, and the running totals (tokens, entries) of those that
+//                   fit some instance; larger entries are passed over
+//   k_disp_chain    matured instances sorted by (maturity, index); one warp hands consecutive runs of
+//                   the queue to them, each run found by a search on the running totals
+//   k_disp_assign   the request -> instance binding of every dispatched row
+#include <new>
+#include <string.h>
+
+#include "hfx_internal.cuh"
+
+#define DISP_THREADS 256
+#define RADIX_ITEMS 8                               // items a thread holds in the scatter pass
+#define RADIX_TILE (DISP_THREADS * RADIX_ITEMS)     // 2048
+#define DISP_MAX_INSTANCES 4096                     // instances the chain kernel orders in shared memory
+
+struct DispWork {
+  // queue, ping-pong
+  uint64_t *key[2]; uint32_t *val[2];
+  uint64_t *rowkey;          // [rows] the 48-bit key of a queue row, by row
+  int64_t *prefix;           // [rows] running total of prompt lengths along the queue (entries that fit some instance)
+  int32_t *prefix_cnt;       // [rows] running count of those entries
+  uint32_t *hist;            // [256][tiles] digit counts of the current pass, then their exclusive prefix
+  int64_t *tile_sum;         // [2][tiles] totals of the prefix pass: tokens, entries
+  uint32_t *n_run;           // [R]
+  unsigned long long *sum_kv;    // [R]
+  unsigned long long *mask_run;  // [R]
+  unsigned long long *ctl;   // [0] classes present in the queue  [1] queue length  [2], [3] last-block counters
+                             // [4] largest budget among the matured instances
+  ReplicaPlan *plan;         // [R]
+  int32_t *run_start;        // [R] where an instance's run starts in the queue
+  int32_t *run_len;          // [R] queue positions the run covers (passed-over entries included)
+  int64_t max_rows; int32_t R;
+};
+
+struct DispArgs {
+  const int32_t *replica_id; const uint8_t *class_id; const uint8_t *state; const int32_t *prompt_len; const int32_t *gen;
+  const int64_t *arrival; const int32_t *req_id; const int32_t *weight;
+  int64_t n; int64_t now; int32_t cap_max;
+  const int64_t *maturity; const hfx_replica_cfg *cfg;
+  // outputs
+  int32_t *assign; int32_t *queue_order; int32_t *n_queue; int32_t *inst_order; int32_t *n_mature; int64_t *slack;
+  int64_t *budget; int64_t *e_d; int32_t *n_run; int64_t *sum_kv; int64_t *adm_cost; int32_t *adm_count; int64_t *maturity_next;
+  uint32_t *status;
+};
+
+// ------------------------------------------------------------------------------------------------
+// k_disp_scan
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, const DispArgs a, const DispWork w) {
+  __shared__ int64_t s_ttft[HFX_MAX_CLASSES];
+  __shared__ uint8_t s_prio[HFX_MAX_CLASSES];
+  for (int c = threadIdx.x; c < HFX_MAX_CLASSES; c += blockDim.x) {
+    s_ttft[c] = c < p.n_classes ? p.ttft[c] : 0;
+    s_prio[c] = c < p.n_classes ? p.prio[c] : 63;
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  uint32_t bad = 0;
+  unsigned long long qmask = 0;
+  const int64_t n_round = (a.n + 31) & ~INT64_C(31);       // whole warps stay together for the ballot
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += (int64_t)gridDim.x * blockDim.x) {
+    bool in_queue = false;
+    uint64_t k48 = 0;
+    uint32_t uid = 0;
+    if (i < a.n) {
+      const uint32_t cls = a.class_id[i], st = a.state[i];
+      const int32_t prompt = a.prompt_len[i], gen = a.gen[i];
+      bool ok = true;
+      if (cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
+      if (prompt < 0 || prompt > HFX_MAX_TOKENS || gen < 0 || gen > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }
+      int64_t slack = 0;
+      if (ok && st == HFX_RUNNING) {
+        const int32_t r = a.replica_id[i];
+        if (r < 0 || r >= p.n_replicas) bad |= HFX_ST_BAD_REPLICA;
+        else {
+          atomicAdd(&w.n_run[r], 1u);
+          atomicAdd(&w.sum_kv[r], (unsigned long long)((int64_t)prompt + gen));
+          atomicOr(&w.mask_run[r], 1ull << cls);
+        }
+      } else if (ok && st == HFX_QUEUED && a.arrival[i] <= a.now && prompt <= a.cap_max) {
+        const int64_t ttft = s_ttft[cls];
+        slack = ttft > 0 ? ttft - ((a.now - a.arrival[i]) + dev_Ep(p, prompt)) : HFX_SLACK_MAX;
+        int prio;
+        if (p.weight_max > 0) {
+          const int64_t x = (int64_t)p.weight_max - a.weight[i];
+          prio = (int)(x < 0 ? 0 : (x > 62 ? 62 : x));
+        } else prio = s_prio[cls];
+        k48 = dev_key48(PH_QUEUED, prio, slack);
+        uid = (uint32_t)a.req_id[i] ^ 0x80000000u;         // signed order as unsigned
+        qmask |= 1ull << cls;
+        in_queue = true;
+      }
+      a.slack[i] = slack;
+      a.assign[i] = -1;
+      a.queue_order[i] = -1;
+    }
+    // append to the queue list: one counter update per warp
+    const uint32_t m = __ballot_sync(0xffffffffu, in_queue);
+    if (m) {
+      unsigned long long base = 0;
+      if (lane == 0) base = atomicAdd(&w.ctl[1], (unsigned long long)__popc(m));
+      base = __shfl_sync(0xffffffffu, base, 0);
+      if (in_queue) {
+        const uint64_t pos = base + __popc(m & ((1u << lane) - 1u));
+        w.key[0][pos] = uid;
+        w.val[0][pos] = (uint32_t)i;
+        w.rowkey[i] = k48;
+      }
+    }
+  }
+  qmask = warp_or_u64(qmask);
+  if (lane == 0 && qmask) atomicOr(&w.ctl[0], qmask);
+  if (bad) atomicOr(a.status, bad);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Radix sort pass, 8 bits: k_radix_hist counts the digits of every tile (hist[digit][tile]); the
+// block that finishes last turns the whole array into its exclusive prefix, which is where each
+// tile's items of each digit go.  k_radix_scatter orders a tile by the digit (eight stable one-bit
+// splits of packed (digit, position) words in shared memory) and writes the items out.
+// The item count lives on the device (ctl[1]); tiles beyond it leave at once.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DISP_THREADS) k_radix_hist(const uint64_t *__restrict__ keys, const unsigned long long *ctl_n,
+                                                             int shift, uint32_t *__restrict__ hist, int32_t tiles_max,
+                                                             unsigned long long *done) {
+  __shared__ uint32_t s_h[256];
+  __shared__ uint32_t s_warp[32];
+  __shared__ uint32_t s_last, s_carry;
+  const int64_t n = (int64_t)*ctl_n;
+  const int32_t tiles = (int32_t)((n + RADIX_TILE - 1) / RADIX_TILE);
+  const int tile = blockIdx.x;
+  if (tile < tiles) {
+    s_h[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t lo = (int64_t)tile * RADIX_TILE;
+    const int64_t hi = lo + RADIX_TILE < n ? lo + RADIX_TILE : n;
+    for (int64_t j = lo + threadIdx.x; j < hi; j += DISP_THREADS) atomicAdd(&s_h[(uint32_t)(keys[j] >> shift) & 255u], 1u);
+    __syncthreads();
+    hist[(size_t)threadIdx.x * tiles_max + tile] = s_h[threadIdx.x];
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(done, 1ull) == (unsigned long long)gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // exclusive scan of hist[d][t], d-major, over the tiles in use (entries of unused tiles are skipped)
+  if (threadIdx.x == 0) { s_carry = 0; *done = 0; }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t total = (int64_t)256 * tiles;
+  for (int64_t base = 0; base < total; base += DISP_THREADS * 4) {
+    uint32_t v[4], sum = 0;
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int64_t e = base + (int64_t)threadIdx.x * 4 + k;
+      v[k] = 0;
+      if (e < total) { const int64_t d = e / tiles, t = e - d * tiles; v[k] = __ldcg(hist + (size_t)d * tiles_max + t); }
+      sum += v[k];
+    }
+    uint32_t inc = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += x; }
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    uint32_t run = s_carry + inc - sum;
+    for (int k = 0; k < warp; k++) run += s_warp[k];
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int64_t e = base + (int64_t)threadIdx.x * 4 + k;
+      if (e < total) { const int64_t d = e / tiles, t = e - d * tiles; hist[(size_t)d * tiles_max + t] = run; }
+      run += v[k];
+    }
+    __syncthreads();
+    if (threadIdx.x == DISP_THREADS - 1) s_carry = run;
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(DISP_THREADS) k_radix_scatter(const uint64_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in,
+                                                                uint64_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out,
+                                                                const unsigned long long *ctl_n, int shift,
+                                                                const uint32_t *__restrict__ hist, int32_t tiles_max) {
+  __shared__ uint64_t s_key[RADIX_TILE];
+  __shared__ uint32_t s_val[RADIX_TILE];
+  __shared__ uint32_t s_item[2][RADIX_TILE];     // digit << 16 | position in the tile
+  __shared__ uint32_t s_start[257];              // where each digit starts in the ordered tile
+  __shared__ uint32_t s_warp[32];
+  const int64_t n = (int64_t)*ctl_n;
+  const int32_t tiles = (int32_t)((n + RADIX_TILE - 1) / RADIX_TILE);
+  const int tile = blockIdx.x;
+  if (tile >= tiles) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t lo = (int64_t)tile * RADIX_TILE;
+  const int nt = (int)((lo + RADIX_TILE < n ? lo + RADIX_TILE : n) - lo);
+  for (int q = threadIdx.x; q < RADIX_TILE; q += DISP_THREADS) {
+    uint32_t item = (256u << 16) | (uint32_t)q;           // padding sorts behind every digit
+    if (q < nt) {
+      const uint64_t k = keys_in[lo + q];
+      s_key[q] = k; s_val[q] = vals_in[lo + q];
+      item = (((uint32_t)(k >> shift) & 255u) << 16) | (uint32_t)q;
+    }
+    s_item[0][q] = item;
+  }
+  __syncthreads();
+  int src = 0;
+  for (int bit = 16; bit < 25; bit++) {                    // 8 digit bits and the padding bit
+    uint32_t it[RADIX_ITEMS];
+    uint32_t zeros = 0;
+#pragma unroll
+    for (int k = 0; k < RADIX_ITEMS; k++) { it[k] = s_item[src][threadIdx.x * RADIX_ITEMS + k]; zeros += ((it[k] >> bit) & 1u) ^ 1u; }
+    uint32_t inc = zeros;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += x; }
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    uint32_t zbase = inc - zeros, ztotal = 0;
+    for (int k = 0; k < DISP_THREADS / 32; k++) { const uint32_t x = s_warp[k]; if (k < warp) zbase += x; ztotal += x; }
+    uint32_t obase = ztotal + (uint32_t)threadIdx.x * RADIX_ITEMS - zbase;
+#pragma unroll
+    for (int k = 0; k < RADIX_ITEMS; k++) {
+      if ((it[k] >> bit) & 1u) s_item[src ^ 1][obase++] = it[k];
+      else s_item[src ^ 1][zbase++] = it[k];
+    }
+    src ^= 1;
+    __syncthreads();
+  }
+  // digit starts inside the ordered tile: first position of each digit
+  for (int d = threadIdx.x; d <= 256; d += DISP_THREADS) s_start[d] = (uint32_t)nt;
+  __syncthreads();
+  for (int q = threadIdx.x; q < nt; q += DISP_THREADS) {
+    const uint32_t d = s_item[src][q] >> 16;
+    if (q == 0 || (s_item[src][q - 1] >> 16) != d) s_start[d] = (uint32_t)q;
+  }
+  __syncthreads();
+  for (int q = threadIdx.x; q < nt; q += DISP_THREADS) {
+    const uint32_t item = s_item[src][q];
+    const uint32_t d = item >> 16, from = item & 0xffffu;
+    const uint32_t pos = hist[(size_t)d * tiles_max + tile] + ((uint32_t)q - s_start[d]);
+    keys_out[pos] = s_key[from];
+    vals_out[pos] = s_val[from];
+  }
+}
+
+// after the request-id passes: the 48-bit key of every queue entry, in the order reached so far
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_gather(uint64_t *__restrict__ keys, const uint32_t *__restrict__ vals,
+                                                              const uint64_t *__restrict__ rowkey, const unsigned long long *ctl_n) {
+  const int64_t n = (int64_t)*ctl_n;
+  for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (int64_t)gridDim.x * blockDim.x)
+    keys[j] = rowkey[vals[j]];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Running total of prompt lengths along the ordered queue: per-tile totals, the last block scans
+// them; then every tile scans its own items on top of its offset and lists the queue's rows.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_tilesum(const uint32_t *__restrict__ vals, const int32_t *__restrict__ prompt_len,
+                                                               const unsigned long long *ctl, int64_t *__restrict__ tile_sum,
+                                                               int32_t tiles_max, unsigned long long *done) {
+  __shared__ int64_t s_red[32], s_redc[32];
+  __shared__ uint32_t s_last;
+  const int64_t n = (int64_t)ctl[1];
+  const int64_t bmax = (int64_t)ctl[4];
+  const int32_t tiles = (int32_t)((n + RADIX_TILE - 1) / RADIX_TILE);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if ((int)blockIdx.x < tiles) {
+    const int64_t lo = (int64_t)blockIdx.x * RADIX_TILE;
+    const int64_t hi = lo + RADIX_TILE < n ? lo + RADIX_TILE : n;
+    int64_t s = 0, c = 0;
+    for (int64_t j = lo + threadIdx.x; j < hi; j += DISP_THREADS) { const int64_t x = prompt_len[vals[j]]; if (x <= bmax) { s += x; c += 1; } }
+    s = warp_sum_i64(s); c = warp_sum_i64(c);
+    if (lane == 0) { s_red[warp] = s; s_redc[warp] = c; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int64_t t = 0, u = 0;
+      for (int k = 0; k < DISP_THREADS / 32; k++) { t += s_red[k]; u += s_redc[k]; }
+      tile_sum[blockIdx.x] = t;
+      tile_sum[tiles_max + blockIdx.x] = u;
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(done, 1ull) == (unsigned long long)gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (threadIdx.x == 0) {       // exclusive scan of the tile totals (a few hundred entries at most)
+    int64_t run = 0, runc = 0;
+    for (int32_t t = 0; t < tiles; t++) {
+      const int64_t x = __ldcg(tile_sum + t), y = __ldcg(tile_sum + tiles_max + t);
+      tile_sum[t] = run; tile_sum[tiles_max + t] = runc;
+      run += x; runc += y;
+    }
+    *done = 0;
+  }
+}
+
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_prefix(const uint32_t *__restrict__ vals, const int32_t *__restrict__ prompt_len,
+                                                              const unsigned long long *ctl, const int64_t *__restrict__ tile_sum,
+                                                              int32_t tiles_max, int64_t *__restrict__ prefix,
+                                                              int32_t *__restrict__ prefix_cnt, int32_t *__restrict__ queue_order,
+                                                              int32_t *__restrict__ n_queue) {
+  __shared__ int64_t s_warp[32];
+  __shared__ int32_t s_warpc[32];
+  const int64_t n = (int64_t)ctl[1];
+  const int64_t bmax = (int64_t)ctl[4];
+  const int32_t tiles = (int32_t)((n + RADIX_TILE - 1) / RADIX_TILE);
+  if (blockIdx.x == 0 && threadIdx.x == 0) *n_queue = (int32_t)n;
+  if ((int)blockIdx.x >= tiles) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t lo = (int64_t)blockIdx.x * RADIX_TILE + (int64_t)threadIdx.x * RADIX_ITEMS;
+  int64_t c[RADIX_ITEMS], sum = 0;
+  int32_t e[RADIX_ITEMS], cnt = 0;
+#pragma unroll
+  for (int k = 0; k < RADIX_ITEMS; k++) {
+    c[k] = 0; e[k] = 0;
+    if (lo + k < n) {
+      const uint32_t row = vals[lo + k];
+      const int64_t x = prompt_len[row];
+      if (x <= bmax) { c[k] = x; e[k] = 1; }      // larger than every budget of this call: passed over
+      queue_order[lo + k] = (int32_t)row;
+    }
+    sum += c[k]; cnt += e[k];
+  }
+  const int64_t inc = warp_incl_scan_i64(sum, lane);
+  const int32_t incc = warp_incl_scan_i32(cnt, lane);
+  if (lane == 31) { s_warp[warp] = inc; s_warpc[warp] = incc; }
+  __syncthreads();
+  int64_t run = tile_sum[blockIdx.x] + inc - sum;
+  int32_t runc = (int32_t)tile_sum[tiles_max + blockIdx.x] + incc - cnt;
+  for (int k = 0; k < warp; k++) { run += s_warp[k]; runc += s_warpc[k]; }
+#pragma unroll
+  for (int k = 0; k < RADIX_ITEMS; k++) {     // inclusive
+    run += c[k]; runc += e[k];
+    if (lo + k < n) { prefix[lo + k] = run; prefix_cnt[lo + k] = runc; }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// k_disp_plan: dispatching step 2 for every instance (E_d of its running batch, the safe budget from
+// the strictest TTFT in the queue and the strictest TPOT in flight); resets the per-instance results.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_plan(const HfxParams p, const DispArgs a, const DispWork w) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= p.n_replicas) return;
+  ReplicaPlan pl;
+  dev_plan(p, a.cfg[r], a.now, a.maturity[r], (int64_t)w.n_run[r], (int64_t)w.sum_kv[r], w.mask_run[r], w.ctl[0], pl);
+  w.plan[r] = pl;
+  a.budget[r] = pl.budget;
+  a.e_d[r] = pl.e_d;
+  a.n_run[r] = (int32_t)pl.n_run;
+  a.sum_kv[r] = pl.sum_kv;
+  a.adm_cost[r] = 0;
+  a.adm_count[r] = 0;
+  a.maturity_next[r] = pl.mat;
+  a.inst_order[r] = -1;
+  w.run_start[r] = 0;
+  w.run_len[r] = 0;
+  if (pl.now >= pl.mat && pl.budget > 0) atomicMax(&w.ctl[4], (unsigned long long)pl.budget);
+}
+
+// ------------------------------------------------------------------------------------------------
+// k_disp_chain: one block.  Dispatching step 1: the matured instances ordered by (maturity, index)
+// in shared memory.  Steps 3 and 4: the first warp walks them; each takes the longest run of queue
+// entries, from where the previous one stopped, whose total stays within its budget and batch room
+// (a gallop and a 32-way search on the running totals), then gets its new maturity time.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const DispArgs a, const DispWork w) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int R = p.n_replicas;
+  uint64_t *s_mat = reinterpret_cast<uint64_t *>(smem_raw);     // [R] maturity, biased to unsigned order
+  uint32_t *s_id = reinterpret_cast<uint32_t *>(s_mat + R);     // [R]
+  __shared__ int32_t s_nm;
+  if (threadIdx.x == 0) s_nm = 0;
+  __syncthreads();
+  for (int r = threadIdx.x; r < R; r += blockDim.x)
+    if (a.maturity[r] <= a.now) {
+      const int k = atomicAdd(&s_nm, 1);
+      s_mat[k] = (uint64_t)a.maturity[r] ^ (1ull << 63);
+      s_id[k] = (uint32_t)r;
+    }
+  __syncthreads();
+  const int nm = s_nm;
+  block_sort<true>(s_mat, s_id, nm);
+  for (int k = threadIdx.x; k < nm; k += blockDim.x) a.inst_order[k] = (int32_t)s_id[k];
+  if (threadIdx.x == 0) *a.n_mature = nm;
+  if (threadIdx.x >= 32) return;
+  const int lane = threadIdx.x;
+  const int64_t nq = (int64_t)w.ctl[1];
+  int64_t cursor = 0, base = 0, base_cnt = 0;         // queue position; running totals before it
+  for (int k = 0; k < nm && cursor < nq; k++) {
+    const int r = (int)s_id[k];
+    const ReplicaPlan pl = w.plan[r];
+    const int64_t span = nq - cursor;
+    int64_t room = span;                              // entries the batch cap still allows
+    if (pl.batch_cap != 0) {
+      const int64_t left = (int64_t)pl.batch_cap - pl.n_run;
+      room = left < room ? (left > 0 ? left : 0) : room;
+    }
+    // longest stretch m in [0, span] of queue positions whose entries that count stay within the budget
+    // and the batch room (both running totals never decrease)
+    const int64_t limit = base + pl.budget, limit_cnt = base_cnt + room;
+    auto fits = [&](int64_t m) { return w.prefix[cursor + m - 1] <= limit && (int64_t)w.prefix_cnt[cursor + m - 1] <= limit_cnt; };
+    int64_t lo = 0, hi = span;                        // fits(lo); the answer lies in [lo, hi]
+    {   // gallop: lane l tries m = 2^l
+      const int64_t m = INT64_C(1) << lane;
+      const bool ok = m <= span && fits(m);
+      const uint32_t b = __ballot_sync(0xffffffffu, ok);
+      const int f = __popc(b);                        // the lanes that fit are a prefix
+      if (f > 0) lo = INT64_C(1) << (f - 1);
+      if (f < 32) { const int64_t t = (INT64_C(1) << f) - 1; hi = t < hi ? t : hi; }
+    }
+    while (lo < hi) {
+      const int64_t step = (hi - lo + 31) / 32;
+      const int64_t cand = lo + (int64_t)(lane + 1) * step;
+      const bool ok = cand <= hi && fits(cand);
+      const int f = __popc(__ballot_sync(0xffffffffu, ok));
+      const int64_t nlo = lo + (int64_t)f * step;
+      int64_t nhi = lo + (int64_t)(f + 1) * step - 1;
+      if (nhi > hi) nhi = hi;
+      lo = nlo; hi = nhi;
+    }
+    const int64_t m = lo;
+    if (m > 0) {
+      const int64_t cost = w.prefix[cursor + m - 1] - base;
+      const int64_t cnt = (int64_t)w.prefix_cnt[cursor + m - 1] - base_cnt;
+      if (lane == 0) {
+        w.run_start[r] = (int32_t)cursor;
+        w.run_len[r] = (int32_t)m;
+        if (cnt > 0) {
+          int64_t lp = 0;
+          a.adm_cost[r] = cost;
+          a.adm_count[r] = (int32_t)cnt;
+          a.maturity_next[r] = dev_maturity_next(p, pl, cnt, cost, 0, &lp);
+        }
+      }
+      cursor += m;
+      base += cost;
+      base_cnt += cnt;
+    }
+  }
+}
+
+// the request -> instance binding of every dispatched row: one block per instance
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_assign(const DispArgs a, const DispWork w, int slot) {
+  const int r = blockIdx.x;
+  const int32_t m = w.run_len[r], s0 = w.run_start[r];
+  const int64_t bmax = (int64_t)w.ctl[4];
+  for (int32_t q = threadIdx.x; q < m; q += blockDim.x) {
+    const uint32_t row = w.val[slot][s0 + q];
+    if (a.prompt_len[row] <= bmax) a.assign[row] = r;       // the others were passed over
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+struct hfx_dispatch_ws { DispWork w; int ready; };
+
+int hfx_dispatch_configure() {
+  if (cudaFuncSetAttribute(k_disp_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, 12 * DISP_MAX_INSTANCES) != cudaSuccess)
+    return HFX_E_CUDA;
+  return HFX_OK;
+}
+
+static void disp_free(DispWork &w) {
+  cudaFree(w.key[0]); cudaFree(w.key[1]); cudaFree(w.val[0]); cudaFree(w.val[1]); cudaFree(w.rowkey); cudaFree(w.prefix);
+  cudaFree(w.hist); cudaFree(w.tile_sum); cudaFree(w.n_run); cudaFree(w.sum_kv); cudaFree(w.mask_run); cudaFree(w.ctl);
+  cudaFree(w.plan); cudaFree(w.run_start); cudaFree(w.run_len); cudaFree(w.prefix_cnt);
+  cudaGetLastError();
+}
+
+void hfx_dispatch_release(hfx_sched *s) {
+  if (!s->dispatch_ws) return;
+  hfx_dispatch_ws *d = reinterpret_cast<hfx_dispatch_ws *>(s->dispatch_ws);
+  disp_free(d->w);
+  delete d;
+  s->dispatch_ws = nullptr;
+}
+
+static int disp_workspace(hfx_sched *s, hfx_dispatch_ws **out) {
+  if (s->dispatch_ws) { *out = reinterpret_cast<hfx_dispatch_ws *>(s->dispatch_ws); return HFX_OK; }
+  hfx_dispatch_ws *d = new (std::nothrow) hfx_dispatch_ws();
+  if (!d) return HFX_E_NOMEM;
+  memset(d, 0, sizeof(*d));
+  DispWork &w = d->w;
+  const size_t rows = (size_t)s->max_rows, R = (size_t)s->p.n_replicas;
+  const size_t tiles = (rows + RADIX_TILE - 1) / RADIX_TILE;
+  w.max_rows = s->max_rows; w.R = s->p.n_replicas;
+  bool ok = true;
+  for (int k = 0; k < 2; k++) {
+    ok = ok && cudaMalloc(&w.key[k], sizeof(uint64_t) * rows) == cudaSuccess;
+    ok = ok && cudaMalloc(&w.val[k], sizeof(uint32_t) * rows) == cudaSuccess;
+  }
+  ok = ok && cudaMalloc(&w.rowkey, sizeof(uint64_t) * rows) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.prefix, sizeof(int64_t) * rows) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.hist, sizeof(uint32_t) * 256 * tiles) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.tile_sum, sizeof(int64_t) * 2 * tiles) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.prefix_cnt, sizeof(int32_t) * rows) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.n_run, sizeof(uint32_t) * R) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.sum_kv, sizeof(unsigned long long) * R) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.mask_run, sizeof(unsigned long long) * R) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.ctl, 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.plan, sizeof(ReplicaPlan) * R) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.run_start, sizeof(int32_t) * R) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.run_len, sizeof(int32_t) * R) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); disp_free(w); delete d; return HFX_E_NOMEM; }
+  s->dispatch_ws = d;
+  *out = d;
+  return HFX_OK;
+}
+
+int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const int64_t *maturity, const hfx_dispatch_out *o,
+                        int32_t cap_max) {
+  hfx_dispatch_ws *d = nullptr;
+  int rc = disp_workspace(s, &d);
+  if (rc != HFX_OK) return rc;
+  const DispWork &w = d->w;
+  cudaStream_t st = s->stream;
+  const int R = s->p.n_replicas;
+  const int64_t n = t->n_rows;
+  DispArgs a;
+  a.replica_id = t->replica_id; a.class_id = t->class_id; a.state = t->state; a.prompt_len = t->prompt_len; a.gen = t->gen;
+  a.arrival = t->arrival_ns; a.req_id = t->req_id; a.weight = s->p.weight_max > 0 ? t->weight : nullptr;
+  a.n = n; a.now = now_ns; a.cap_max = cap_max; a.maturity = maturity; a.cfg = s->d_cfg;
+  a.assign = o->assign; a.queue_order = o->queue_order; a.n_queue = o->n_queue; a.inst_order = o->inst_order;
+  a.n_mature = o->n_mature; a.slack = o->slack_ns; a.budget = o->budget; a.e_d = o->e_d_ns; a.n_run = o->n_run;
+  a.sum_kv = o->sum_kv; a.adm_cost = o->adm_cost; a.adm_count = o->adm_count; a.maturity_next = o->maturity_next;
+  a.status = s->d_status;
+  if (cudaMemsetAsync(w.n_run, 0, sizeof(uint32_t) * R, st) != cudaSuccess ||
+      cudaMemsetAsync(w.sum_kv, 0, sizeof(unsigned long long) * R, st) != cudaSuccess ||
+      cudaMemsetAsync(w.mask_run, 0, sizeof(unsigned long long) * R, st) != cudaSuccess ||
+      cudaMemsetAsync(w.ctl, 0, 64, st) != cudaSuccess)
+    return HFX_E_CUDA;
+  const int tiles_max = (int)((s->max_rows + RADIX_TILE - 1) / RADIX_TILE);
+  const int tiles = n > 0 ? (int)((n + RADIX_TILE - 1) / RADIX_TILE) : 1;      // tiles the queue can fill in this call
+  {
+    KernelScope ks(s, KSLOT_DISPATCH);
+    int grid = (int)((n + DISP_THREADS - 1) / DISP_THREADS);
+    if (grid > s->n_sm * 8) grid = s->n_sm * 8;
+    if (grid < 1) grid = 1;
+    k_disp_scan<<<grid, DISP_THREADS, 0, st>>>(s->p, a, w);
+  }
+  int slot = 0;
+  auto pass = [&](int shift) {
+    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_hist<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.ctl + 1, shift, w.hist, tiles_max, w.ctl + 2); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_scatter<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.key[slot ^ 1], w.val[slot ^ 1], w.ctl + 1, shift, w.hist, tiles_max); }
+    slot ^= 1;
+  };
+  for (int shift = 0; shift < 32; shift += 8) pass(shift);            // by request id
+  {
+    KernelScope ks(s, KSLOT_DISPATCH);
+    k_disp_gather<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.rowkey, w.ctl + 1);
+  }
+  for (int shift = 0; shift < 48; shift += 8) pass(shift);            // by (priority, slack)
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_plan<<<(R + DISP_THREADS - 1) / DISP_THREADS, DISP_THREADS, 0, st>>>(s->p, a, w); }
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_tilesum<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.ctl + 3); }
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_prefix<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.prefix, w.prefix_cnt, o->queue_order, o->n_queue); }
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_chain<<<1, 1024, 12 * (size_t)R, st>>>(s->p, a, w); }
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_assign<<<R, DISP_THREADS, 0, st>>>(a, w, slot); }
+  return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
+}

@@ -59,7 +59,7 @@ static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
 #include <vector>
 
-enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT };
+enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT, KSLOT_DISPATCH };
 
 // tiling of the streaming passes: about this many tiles (2 per SM), each at most this many rows
 #define HFX_TILE_BLOCKS 296
@@ -105,6 +105,7 @@ struct hfx_sched {
   int front_enabled;
   size_t front_smem_cached;            // shared-memory size the capacity below was asked for
   int front_capacity;                  // blocks of the fused kernel that can be resident at once
+  void *dispatch_ws;                   // workspace of hfx_dispatch_step, allocated by its first call
 };
 
 // ---- latency predictor -------------------------------------------------------------------
@@ -343,6 +344,77 @@ __device__ __forceinline__ int32_t warp_incl_scan_i32(int32_t v, int lane) {
   return v;
 }
 
+// Compare-exchange of sort items, ascending: `hi` alone (items carry their tie-break in the low
+// bits) or the 96-bit pair (hi, lo).
+template <bool WIDE>
+__device__ __forceinline__ void cmp_swap(uint64_t *hi, uint32_t *lo, int i, int j) {
+  const uint64_t hi_i = hi[i], hi_j = hi[j];
+  if (WIDE) {
+    const uint32_t lo_i = lo[i], lo_j = lo[j];
+    if (hi_i > hi_j || (hi_i == hi_j && lo_i > lo_j)) { hi[i] = hi_j; hi[j] = hi_i; lo[i] = lo_j; lo[j] = lo_i; }
+  } else if (hi_i > hi_j) { hi[i] = hi_j; hi[j] = hi_i; }
+}
+
+// Bitonic sorting network with ascending comparators only (mirrored first sub-stage), so the virtual
+// +inf padding beyond n never moves: any n, in place.  Items are distinct, so the result is unique.
+// Each warp owns a contiguous chunk of E items; stages whose pairs stay inside a chunk need only a
+// warp barrier, the others a block barrier.  Callers synchronise the block before the call; the
+// block is synchronised on return.
+template <bool WIDE>
+__device__ void block_sort(uint64_t *hi, uint32_t *lo, int n) {
+  if (n > 1) {
+    int n_pad = 2;
+    while (n_pad < n) n_pad <<= 1;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    int E = n_pad / nwarp;
+    if (E < 64) E = 64;
+    if (E > n_pad) E = n_pad;
+    const int c0 = warp * E;
+    const bool has_chunk = c0 < n_pad;
+    const int half = n_pad >> 1;
+    bool local = true;    // the previous stage was chunk-local (or there was none)
+    for (int k = 2; k <= n_pad; k <<= 1) {
+      const int hk = k >> 1;
+      if (k <= E) {   // mirrored sub-stage of merge size k, inside the chunk
+        if (has_chunk)
+          for (int t = lane; t < (E >> 1); t += 32) {
+            const int blk = t / hk, off = t - blk * hk;
+            const int i = c0 + blk * k + off, j = c0 + blk * k + k - 1 - off;
+            if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
+          }
+        __syncwarp();
+      } else {
+        if (local) { __syncthreads(); local = false; }
+        for (int t = threadIdx.x; t < half; t += blockDim.x) {
+          const int blk = t / hk, off = t - blk * hk;
+          const int i = blk * k + off, j = blk * k + k - 1 - off;
+          if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
+        }
+        __syncthreads();
+      }
+      for (int j = k >> 2; j > 0; j >>= 1) {
+        if (2 * j <= E) {   // pairs (i, i+j) stay inside an aligned block of 2j <= E items
+          local = true;
+          if (has_chunk)
+            for (int t = lane; t < (E >> 1); t += 32) {
+              const int i = c0 + 2 * t - (t & (j - 1));
+              if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
+            }
+          __syncwarp();
+        } else {
+          if (local) { __syncthreads(); local = false; }
+          for (int t = threadIdx.x; t < half; t += blockDim.x) {
+            const int i = 2 * t - (t & (j - 1));
+            if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
+          }
+          __syncthreads();
+        }
+      }
+    }
+  }
+  __syncthreads();
+}
+
 // Brackets one kernel launch with events when profiling is on; counts the launch either way.
 struct KernelScope {
   hfx_sched *s; HfxBracket br; bool on; cudaStream_t st;
@@ -393,5 +465,8 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off);
 size_t hfx_regroup_smem(int R1, int tile_rows);
 int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n);
 int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o, uint32_t flags);
+int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const int64_t *maturity, const hfx_dispatch_out *o,
+                        int32_t cap_max);
+void hfx_dispatch_release(hfx_sched *s);
 int hfx_launch_sim(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
                    const hfx_sim_out *o);

@@ -22,77 +22,6 @@ struct BlockShared {
   int32_t adm_count, worked, n_act;
 };
 
-// Compare-exchange of sort items, ascending: `hi` alone (items carry their tie-break in the low
-// bits) or the 96-bit pair (hi, lo).
-template <bool WIDE>
-__device__ __forceinline__ void cmp_swap(uint64_t *hi, uint32_t *lo, int i, int j) {
-  const uint64_t hi_i = hi[i], hi_j = hi[j];
-  if (WIDE) {
-    const uint32_t lo_i = lo[i], lo_j = lo[j];
-    if (hi_i > hi_j || (hi_i == hi_j && lo_i > lo_j)) { hi[i] = hi_j; hi[j] = hi_i; lo[i] = lo_j; lo[j] = lo_i; }
-  } else if (hi_i > hi_j) { hi[i] = hi_j; hi[j] = hi_i; }
-}
-
-// Bitonic sorting network with ascending comparators only (mirrored first sub-stage), so the virtual
-// +inf padding beyond n never moves: any n, in place.  Items are distinct, so the result is unique.
-// Each warp owns a contiguous chunk of E items; stages whose pairs stay inside a chunk need only a
-// warp barrier, the others a block barrier.  Callers synchronise the block before the call; the
-// block is synchronised on return.
-template <bool WIDE>
-__device__ void block_sort(uint64_t *hi, uint32_t *lo, int n) {
-  if (n > 1) {
-    int n_pad = 2;
-    while (n_pad < n) n_pad <<= 1;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-    int E = n_pad / nwarp;
-    if (E < 64) E = 64;
-    if (E > n_pad) E = n_pad;
-    const int c0 = warp * E;
-    const bool has_chunk = c0 < n_pad;
-    const int half = n_pad >> 1;
-    bool local = true;    // the previous stage was chunk-local (or there was none)
-    for (int k = 2; k <= n_pad; k <<= 1) {
-      const int hk = k >> 1;
-      if (k <= E) {   // mirrored sub-stage of merge size k, inside the chunk
-        if (has_chunk)
-          for (int t = lane; t < (E >> 1); t += 32) {
-            const int blk = t / hk, off = t - blk * hk;
-            const int i = c0 + blk * k + off, j = c0 + blk * k + k - 1 - off;
-            if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
-          }
-        __syncwarp();
-      } else {
-        if (local) { __syncthreads(); local = false; }
-        for (int t = threadIdx.x; t < half; t += blockDim.x) {
-          const int blk = t / hk, off = t - blk * hk;
-          const int i = blk * k + off, j = blk * k + k - 1 - off;
-          if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
-        }
-        __syncthreads();
-      }
-      for (int j = k >> 2; j > 0; j >>= 1) {
-        if (2 * j <= E) {   // pairs (i, i+j) stay inside an aligned block of 2j <= E items
-          local = true;
-          if (has_chunk)
-            for (int t = lane; t < (E >> 1); t += 32) {
-              const int i = c0 + 2 * t - (t & (j - 1));
-              if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
-            }
-          __syncwarp();
-        } else {
-          if (local) { __syncthreads(); local = false; }
-          for (int t = threadIdx.x; t < half; t += blockDim.x) {
-            const int i = 2 * t - (t & (j - 1));
-            if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
-          }
-          __syncthreads();
-        }
-      }
-    }
-  }
-  __syncthreads();
-}
-
 // Distribution sort of distinct 64-bit items for small segments: items are binned by their offset
 // from the smallest item (a shift makes at most SORT_BINS bins, so bins are in key order), scattered
 // bin by bin, and ranked inside their bin by counting smaller items.  Writes the low 16 bits of the

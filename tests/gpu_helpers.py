@@ -85,3 +85,29 @@ def assert_sim_parity(wl, iters=None, traces=None):
     if len(traces) == T:
         assert st == oracle.sim(wl.copy(), iters=0)["status"] or True
     return res
+
+
+DISPATCH_KEYS = {"assign": "assign", "queue_order": "queue_order", "n_queue": "n_queue", "inst_order": "inst_order",
+                 "n_mature": "n_mature", "slack": "slack_ns", "budget": "budget", "e_d": "e_d_ns", "n_run": "n_run",
+                 "sum_kv": "sum_kv", "adm_cost": "adm_cost", "adm_count": "adm_count", "maturity_next": "maturity_next"}
+
+
+def assert_dispatch_parity(wl, now, sched=None, calls=1):
+    """hfx_dispatch_step against the oracle's dispatch on the same table, every output bit for bit."""
+    own = sched is None
+    sched = sched or make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    mat = torch.from_numpy(wl.maturity.copy()).cuda()
+    out = hfx.DispatchOut(wl.n_rows, wl.n_replicas)
+    c = oracle.dispatch(wl, now)
+    g = None
+    for _ in range(calls):
+        sched.dispatch_step(tab, now, mat, out)
+        st = sched.status()
+        g = out.to_numpy()
+        assert st == c["status"], (st, c["status"])
+        for ko, kg in DISPATCH_KEYS.items():
+            assert np.array_equal(g[kg], c[ko]), f"{kg} differs at {np.nonzero(g[kg] != c[ko])[0][:8]}: gpu {g[kg][np.nonzero(g[kg] != c[ko])[0][:4]]} oracle {c[ko][np.nonzero(g[kg] != c[ko])[0][:4]]}"
+    if own:
+        sched.close()
+    return g

@@ -369,3 +369,14 @@ def test_dispatch_batch_cap_stops_a_run_and_oversize_prompts_leave_the_queue():
     # instance 1 takes q2 and is full; instance 0 (budget 1281) takes q1 + q4 = 1016, q3 would make 1297
     assert list(o["assign"][80:86]) == [0, 1, -1, 0, -1, -1]
     assert list(o["adm_cost"]) == [1016, 1144, 0] and list(o["adm_count"]) == [2, 1, 0]
+
+
+def test_dispatch_entry_that_fits_nowhere_is_passed_over():
+    wl, now = _dispatch_hand_case()
+    wl.table["prompt_len"][80] = 3000
+    o = oracle.dispatch(wl, now)
+    assert o["slack"][80] == PINS["disp_slack_q1_long"]
+    assert list(o["queue_order"][:5]) == [80, 81, 83, 82, 84]
+    assert list(o["assign"][80:86]) == [-1, 1, 1, 1, -1, -1]
+    assert list(o["adm_cost"]) == [0, 1441, 0] and list(o["adm_count"]) == [0, 3, 0]
+    assert o["maturity_next"][1] - now == PINS["disp_mat1_delta_long"] and o["maturity_next"][0] == now - 5

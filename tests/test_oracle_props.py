@@ -283,7 +283,12 @@ def test_dispatch_invariants(seed):
     assert nm == mature.size and sorted(o["inst_order"][:nm].tolist()) == mature.tolist()
     mo = wl.maturity[o["inst_order"][:nm]]
     assert np.all(np.diff(mo) >= 0)
-    # consecutive runs of the queue, in instance order; each within budget and batch cap, each maximal
+    # consecutive runs of the queue's entries that fit some instance, in instance order; each run within
+    # budget and batch cap, each maximal; entries larger than every budget of the call are passed over
+    bmax = int(o["budget"][o["inst_order"][:nm]].max()) if nm else 0
+    fits = t["prompt_len"][queue] <= bmax
+    assert np.all(o["assign"][queue[~fits]] == -1)
+    queue = queue[fits]
     cursor = 0
     for r in o["inst_order"][:nm]:
         cnt, cost = int(o["adm_count"][r]), int(o["adm_cost"][r])
@@ -293,7 +298,7 @@ def test_dispatch_invariants(seed):
         cap = int(wl.replicas[r, 2])
         assert cap == 0 or cnt == 0 or o["n_run"][r] + cnt <= cap
         cursor += cnt
-        if cursor < nq:
+        if cursor < queue.size:
             nxt = int(t["prompt_len"][queue[cursor]])
             assert cost + nxt > o["budget"][r] or (cap != 0 and o["n_run"][r] + cnt + 1 > cap)
         assert (o["maturity_next"][r] > now) == (cnt > 0) or cnt == 0

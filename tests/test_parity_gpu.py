@@ -6,7 +6,7 @@ import torch
 import gen
 import oracle
 from helpers import MS, SEC, make_wl
-from gpu_helpers import assert_step_parity, assert_sim_parity, make_sched, run_sim_gpu
+from gpu_helpers import assert_dispatch_parity, assert_step_parity, assert_sim_parity, make_sched, run_sim_gpu
 
 pytestmark = pytest.mark.gpu
 MODES3 = (gen.COLOCATED, gen.PREFILL, gen.DECODE)
@@ -368,3 +368,54 @@ def test_scaler_tick_parity():
     _scale_parity(wl, int(wl.now.max()), np.full(9000, 5), window=2 * SEC)
     wl = gen.random_table(7, 0, 3)
     _scale_parity(wl, 5, np.full(3, 5))
+
+
+# ---- dispatching over the shared global queue -------------------------------------------------------
+def _colocated(wl):
+    wl.replicas[:, 0] = gen.COLOCATED
+    return wl
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_dispatch_random_tables(seed):
+    wl = gen.random_table(seed, 500 + 1777 * seed, 1 + (seed * 5) % 19, modes=(gen.COLOCATED,), tie_heavy=seed % 3 == 0,
+                          batch_cap=(0, 9)[seed % 2], weight_max=(0, 16)[seed % 4 == 1], token_cap=(4096, 700)[seed % 3 == 1],
+                          budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 2])
+    assert_dispatch_parity(wl, int(wl.now.max()), calls=2)
+
+
+def test_dispatch_hand_worked_case_and_degenerate_tables():
+    now = 1000 * MS
+    classes = [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)]
+    rows = [dict(state=1, replica_id=0, prompt_len=800, output_len=500, first_token_ns=now - 30 * MS) for _ in range(80)]
+    rows += [dict(replica_id=-1, class_id=0, prompt_len=1000, arrival_ns=now - 10 * MS),
+             dict(replica_id=-1, class_id=0, prompt_len=1144, arrival_ns=now - 50 * MS),
+             dict(replica_id=-1, class_id=1, prompt_len=281, arrival_ns=now - 900 * MS),
+             dict(replica_id=-1, class_id=0, prompt_len=16, arrival_ns=now - 1 * MS),
+             dict(replica_id=-1, class_id=1, prompt_len=2000, arrival_ns=now - 100 * MS),
+             dict(replica_id=-1, class_id=0, prompt_len=16, arrival_ns=now + 1)]
+    wl = make_wl(rows, classes, replicas=[(gen.COLOCATED, 8192, 0)] * 3, now=[now] * 3, maturity=[now - 5, now - 10, now + 1])
+    g = assert_dispatch_parity(wl, now)
+    assert list(g["assign"][80:86]) == [1, 1, 0, 0, -1, -1] and list(g["adm_cost"]) == [297, 2144, 0]
+    # nothing queued; nothing matured; an empty table; zero-token prompts against a zero budget
+    wl2 = wl.copy(); wl2.table["state"][80:] = 2
+    assert_dispatch_parity(wl2, now)
+    wl3 = wl.copy(); wl3.maturity[:] = now + 7
+    assert_dispatch_parity(wl3, now)
+    assert_dispatch_parity(make_wl([], classes, replicas=[(gen.COLOCATED, 8192, 0)] * 2, now=[now] * 2, maturity=[0, 0]), now)
+    wl4 = wl.copy(); wl4.table["prompt_len"][80:84] = 0; wl4.replicas[:, 1] = 80
+    assert_dispatch_parity(wl4, now)
+    # the most urgent entry is larger than every budget of the call: passed over, the rest is served
+    wl5 = wl.copy(); wl5.table["prompt_len"][80] = 3000
+    g = assert_dispatch_parity(wl5, now)
+    assert list(g["assign"][80:86]) == [-1, 1, 1, 1, -1, -1]
+
+
+def test_dispatch_shared_queue_workload():
+    # the shared-queue workload at reduced and at full size: many tiles, ragged tail, 1024 instances
+    wl = gen.config4(R=64, n=200_001, steps=1)
+    assert_dispatch_parity(wl, int(wl.now[0]))
+    wl = gen.config4(steps=1)
+    wl.maturity[::7] = wl.now[0] + 5            # some instances have not matured
+    g = assert_dispatch_parity(wl, int(wl.now[0]))
+    assert g["n_queue"][0] > 300_000 and g["adm_count"].sum() > 10_000
