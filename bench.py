@@ -278,6 +278,39 @@ def run_gpu(args):
                "mean_attainment": float((so["attained"] / 2048.0).mean()), "status": ssched.status()}
         ssched.close()
 
+    # ---- dispatching over the shared global queue of the same table (rank 0, outside the timed steps) --
+    disp = None
+    if rank == 0 and not args.no_dispatch:
+        restore()
+        dout = hfx.DispatchOut(n, R)
+        now_g = int(wl.now[0])
+        for _ in range(3):
+            sched.dispatch_step(tab, now_g, mat0, dout)
+        torch.cuda.synchronize()
+        d_evs = []
+        for _ in range(10):
+            flush.fill_(3)
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(stream); sched.dispatch_step(tab, now_g, mat0, dout); b.record(stream)
+            d_evs.append((a, b))
+        torch.cuda.synchronize()
+        d_ms = float(np.mean([a.elapsed_time(b) for a, b in d_evs]))
+        dn = dout.to_numpy()
+        disp = {"workload": "one hfx_dispatch_step over the same table: every matured instance takes its turn",
+                "ms": d_ms, "requests_per_sec": n / (d_ms * 1e-3), "queue_length": int(dn["n_queue"][0]),
+                "instances_matured": int(dn["n_mature"][0]), "requests_dispatched": int(dn["adm_count"].sum()),
+                "status": sched.status()}
+        if world == 1 and not args.no_cpu:
+            import oracle
+            oracle.build()
+            t0 = time.perf_counter()
+            k_d = 0
+            while time.perf_counter() - t0 < 3.0:
+                oracle.dispatch(wl, now_g)
+                k_d += 1
+            disp["cpu_oracle_ms"] = 1e3 * (time.perf_counter() - t0) / k_d
+            disp["cpu_oracle_calls"] = k_d
+
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only -----------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -326,7 +359,7 @@ def run_gpu(args):
                 "clocks": clk, "gpu_launches": launches, "device_status": status,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms_max},
-                "roofline": roof, "cpu_baseline": cpu, "sim": sim}
+                "roofline": roof, "cpu_baseline": cpu, "sim": sim, "dispatch": disp}
         print(json.dumps(line))
     sched.close()
     if world > 1:
@@ -345,6 +378,7 @@ def main():
     ap.add_argument("--sim-iters", type=int, default=10000)
     ap.add_argument("--no-sim", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-dispatch", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
