@@ -11,7 +11,7 @@
 //                   fit some instance; larger entries are passed over
 //   k_disp_chain    matured instances sorted by (maturity, index); one warp hands consecutive runs of
 //                   the queue to them, each run found by a search on the running totals
-//   k_disp_assign   the request -> instance binding of every dispatched row
+//   k_disp_assign   the request -> instance binding of every dispatched row, the new maturity times
 #include <new>
 #include <string.h>
 
@@ -28,7 +28,7 @@ struct DispWork {
   uint64_t *rowkey;          // [rows] the 48-bit key of a queue row, by row
   int64_t *prefix;           // [rows] running total of prompt lengths along the queue (entries that fit some instance)
   int32_t *prefix_cnt;       // [rows] running count of those entries
-  uint32_t *hist;            // [256][tiles] digit counts of the current pass, then their exclusive prefix
+  uint32_t *hist;            // [tiles][256] digit counts of the current pass
   int64_t *tile_sum;         // [2][tiles] totals of the prefix pass: tokens, entries
   uint32_t *n_run;           // [R]
   unsigned long long *sum_kv;    // [R]
@@ -123,74 +123,35 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, c
 }
 
 // ------------------------------------------------------------------------------------------------
-// Radix sort pass, 8 bits: k_radix_hist counts the digits of every tile (hist[digit][tile]); the
-// block that finishes last turns the whole array into its exclusive prefix, which is where each
-// tile's items of each digit go.  k_radix_scatter orders a tile by the digit (eight stable one-bit
-// splits of packed (digit, position) words in shared memory) and writes the items out.
-// The item count lives on the device (ctl[1]); tiles beyond it leave at once.
+// Radix sort pass, 8 bits.  k_radix_hist counts the digits of every tile (hist[tile][digit]).
+// k_radix_scatter first works out where its tile's items of each digit go -- thread d adds up digit
+// d's counts over all tiles (coalesced rows of the histogram), the part from earlier tiles and the
+// total, and a block scan of the totals gives the digit's start -- then orders the tile by the
+// digit (stable one-bit splits of packed (digit, position) words in shared memory) and writes the
+// items out.  The item count lives on the device (ctl[1]); tiles beyond it leave at once.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(DISP_THREADS) k_radix_hist(const uint64_t *__restrict__ keys, const unsigned long long *ctl_n,
-                                                             int shift, uint32_t *__restrict__ hist, int32_t tiles_max,
-                                                             unsigned long long *done) {
+                                                             int shift, uint32_t *__restrict__ hist) {
   __shared__ uint32_t s_h[256];
-  __shared__ uint32_t s_warp[32];
-  __shared__ uint32_t s_last, s_carry;
   const int64_t n = (int64_t)*ctl_n;
   const int32_t tiles = (int32_t)((n + RADIX_TILE - 1) / RADIX_TILE);
   const int tile = blockIdx.x;
-  if (tile < tiles) {
-    s_h[threadIdx.x] = 0;
-    __syncthreads();
-    const int64_t lo = (int64_t)tile * RADIX_TILE;
-    const int64_t hi = lo + RADIX_TILE < n ? lo + RADIX_TILE : n;
-    for (int64_t j = lo + threadIdx.x; j < hi; j += DISP_THREADS) atomicAdd(&s_h[(uint32_t)(keys[j] >> shift) & 255u], 1u);
-    __syncthreads();
-    hist[(size_t)threadIdx.x * tiles_max + tile] = s_h[threadIdx.x];
-  }
-  __threadfence();
+  if (tile >= tiles) return;
+  s_h[threadIdx.x] = 0;
   __syncthreads();
-  if (threadIdx.x == 0) s_last = atomicAdd(done, 1ull) == (unsigned long long)gridDim.x - 1 ? 1u : 0u;
+  const int64_t lo = (int64_t)tile * RADIX_TILE;
+  const int64_t hi = lo + RADIX_TILE < n ? lo + RADIX_TILE : n;
+  for (int64_t j = lo + threadIdx.x; j < hi; j += DISP_THREADS) atomicAdd(&s_h[(uint32_t)(keys[j] >> shift) & 255u], 1u);
   __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  // exclusive scan of hist[d][t], d-major, over the tiles in use (entries of unused tiles are skipped)
-  if (threadIdx.x == 0) { s_carry = 0; *done = 0; }
-  __syncthreads();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t total = (int64_t)256 * tiles;
-  for (int64_t base = 0; base < total; base += DISP_THREADS * 4) {
-    uint32_t v[4], sum = 0;
-#pragma unroll
-    for (int k = 0; k < 4; k++) {
-      const int64_t e = base + (int64_t)threadIdx.x * 4 + k;
-      v[k] = 0;
-      if (e < total) { const int64_t d = e / tiles, t = e - d * tiles; v[k] = __ldcg(hist + (size_t)d * tiles_max + t); }
-      sum += v[k];
-    }
-    uint32_t inc = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += x; }
-    if (lane == 31) s_warp[warp] = inc;
-    __syncthreads();
-    uint32_t run = s_carry + inc - sum;
-    for (int k = 0; k < warp; k++) run += s_warp[k];
-#pragma unroll
-    for (int k = 0; k < 4; k++) {
-      const int64_t e = base + (int64_t)threadIdx.x * 4 + k;
-      if (e < total) { const int64_t d = e / tiles, t = e - d * tiles; hist[(size_t)d * tiles_max + t] = run; }
-      run += v[k];
-    }
-    __syncthreads();
-    if (threadIdx.x == DISP_THREADS - 1) s_carry = run;
-    __syncthreads();
-  }
+  hist[(size_t)tile * 256 + threadIdx.x] = s_h[threadIdx.x];
 }
 
 __global__ void __launch_bounds__(DISP_THREADS) k_radix_scatter(const uint64_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in,
                                                                 uint64_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out,
                                                                 const unsigned long long *ctl_n, int shift,
-                                                                const uint32_t *__restrict__ hist, int32_t tiles_max) {
+                                                                const uint32_t *__restrict__ hist) {
   __shared__ uint64_t s_key[RADIX_TILE];
+  __shared__ uint32_t s_base[256];               // where the tile's items of each digit go
   __shared__ uint32_t s_val[RADIX_TILE];
   __shared__ uint32_t s_item[2][RADIX_TILE];     // digit << 16 | position in the tile
   __shared__ uint32_t s_start[257];              // where each digit starts in the ordered tile
@@ -202,6 +163,28 @@ __global__ void __launch_bounds__(DISP_THREADS) k_radix_scatter(const uint64_t *
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t lo = (int64_t)tile * RADIX_TILE;
   const int nt = (int)((lo + RADIX_TILE < n ? lo + RADIX_TILE : n) - lo);
+  {   // digit threadIdx.x: items in earlier tiles, items in all tiles; exclusive scan of the totals over the digits
+    uint32_t before = 0, total = 0;
+    const uint32_t *col = hist + threadIdx.x;
+    int t = 0;
+    for (; t + 8 <= tiles; t += 8) {
+      uint32_t x[8];
+#pragma unroll
+      for (int k = 0; k < 8; k++) x[k] = col[(size_t)(t + k) * 256];
+#pragma unroll
+      for (int k = 0; k < 8; k++) { total += x[k]; if (t + k < tile) before += x[k]; }
+    }
+    for (; t < tiles; t++) { const uint32_t x = col[(size_t)t * 256]; total += x; if (t < tile) before += x; }
+    uint32_t inc = total;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += y; }
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    uint32_t start = inc - total;
+    for (int k = 0; k < warp; k++) start += s_warp[k];
+    s_base[threadIdx.x] = start + before;
+    __syncthreads();
+  }
   for (int q = threadIdx.x; q < RADIX_TILE; q += DISP_THREADS) {
     uint32_t item = (256u << 16) | (uint32_t)q;           // padding sorts behind every digit
     if (q < nt) {
@@ -245,7 +228,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_radix_scatter(const uint64_t *
   for (int q = threadIdx.x; q < nt; q += DISP_THREADS) {
     const uint32_t item = s_item[src][q];
     const uint32_t d = item >> 16, from = item & 0xffffu;
-    const uint32_t pos = hist[(size_t)d * tiles_max + tile] + ((uint32_t)q - s_start[d]);
+    const uint32_t pos = s_base[d] + ((uint32_t)q - s_start[d]);
     keys_out[pos] = s_key[from];
     vals_out[pos] = s_val[from];
   }
@@ -293,14 +276,22 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_tilesum(const uint32_t *_
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  if (threadIdx.x == 0) {       // exclusive scan of the tile totals (a few hundred entries at most)
-    int64_t run = 0, runc = 0;
-    for (int32_t t = 0; t < tiles; t++) {
-      const int64_t x = __ldcg(tile_sum + t), y = __ldcg(tile_sum + tiles_max + t);
-      tile_sum[t] = run; tile_sum[tiles_max + t] = runc;
-      run += x; runc += y;
-    }
-    *done = 0;
+  // exclusive scan of the tile totals, DISP_THREADS tiles at a time with a carry
+  __shared__ int64_t s_carry[2];
+  if (threadIdx.x == 0) { s_carry[0] = 0; s_carry[1] = 0; *done = 0; }
+  __syncthreads();
+  for (int32_t t0 = 0; t0 < tiles; t0 += DISP_THREADS) {
+    const int32_t t = t0 + threadIdx.x;
+    const int64_t x = t < tiles ? __ldcg(tile_sum + t) : 0, y = t < tiles ? __ldcg(tile_sum + tiles_max + t) : 0;
+    const int64_t ix = warp_incl_scan_i64(x, lane), iy = warp_incl_scan_i64(y, lane);
+    if (lane == 31) { s_red[warp] = ix; s_redc[warp] = iy; }
+    __syncthreads();
+    int64_t rx = s_carry[0] + ix - x, ry = s_carry[1] + iy - y;
+    for (int k = 0; k < warp; k++) { rx += s_red[k]; ry += s_redc[k]; }
+    if (t < tiles) { tile_sum[t] = rx; tile_sum[tiles_max + t] = ry; }
+    __syncthreads();
+    if (threadIdx.x == DISP_THREADS - 1) { s_carry[0] = rx + x; s_carry[1] = ry + y; }
+    __syncthreads();
   }
 }
 
@@ -370,17 +361,55 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_plan(const HfxParams p, c
 
 // ------------------------------------------------------------------------------------------------
 // k_disp_chain: one block.  Dispatching step 1: the matured instances ordered by (maturity, index)
-// in shared memory.  Steps 3 and 4: the first warp walks them; each takes the longest run of queue
-// entries, from where the previous one stopped, whose total stays within its budget and batch room
-// (a gallop and a 32-way search on the running totals), then gets its new maturity time.
+// in shared memory.  Step 3: the first warp walks them; each takes the longest stretch of the queue,
+// from where the previous one stopped, whose entries stay within its budget and batch room (a
+// gallop and a 32-way search on the running totals).  The totals are read through a window in
+// shared memory that the whole block refills from the current position whenever a search reaches
+// its end; a run longer than the window finishes its search in global memory.
 // ------------------------------------------------------------------------------------------------
+#define CHAIN_WINDOW 2048
+
+// longest m in [lo0, hi0] with fits(m), given fits(lo0) (or lo0 = 0) and fits monotone; whole warp
+template <typename F>
+__device__ __forceinline__ int64_t warp_longest(int64_t lo0, const int64_t hi0, int lane, F fits) {
+  {   // short stretches first: lane l tries lo0 + l + 1
+    const int64_t m = lo0 + lane + 1;
+    const int f = __popc(__ballot_sync(0xffffffffu, m <= hi0 && fits(m)));      // the lanes that fit are a prefix
+    if (f < 32) return lo0 + f;
+    lo0 += 32;
+  }
+  int64_t lo = lo0, hi = hi0;
+  {   // gallop: lane l tries lo0 + 2^l
+    const int64_t m = lo0 + (INT64_C(1) << lane);
+    const bool ok = m <= hi0 && fits(m);
+    const int f = __popc(__ballot_sync(0xffffffffu, ok));      // the lanes that fit are a prefix
+    if (f > 0) lo = lo0 + (INT64_C(1) << (f - 1));
+    if (f < 32) { const int64_t t = lo0 + (INT64_C(1) << f) - 1; hi = t < hi ? t : hi; }
+  }
+  while (lo < hi) {
+    const int64_t step = (hi - lo + 31) / 32;
+    const int64_t cand = lo + (int64_t)(lane + 1) * step;
+    const bool ok = cand <= hi && fits(cand);
+    const int f = __popc(__ballot_sync(0xffffffffu, ok));
+    const int64_t nlo = lo + (int64_t)f * step;
+    int64_t nhi = lo + (int64_t)(f + 1) * step - 1;
+    if (nhi > hi) nhi = hi;
+    lo = nlo; hi = nhi;
+  }
+  return lo;
+}
+
 __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const DispArgs a, const DispWork w) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int R = p.n_replicas;
-  uint64_t *s_mat = reinterpret_cast<uint64_t *>(smem_raw);     // [R] maturity, biased to unsigned order
+  uint64_t *s_mat = reinterpret_cast<uint64_t *>(smem_raw);     // [R] maturity, biased to unsigned order; then the budgets
   uint32_t *s_id = reinterpret_cast<uint32_t *>(s_mat + R);     // [R]
-  __shared__ int32_t s_nm;
-  if (threadIdx.x == 0) s_nm = 0;
+  int32_t *s_room = reinterpret_cast<int32_t *>(s_id + R);      // [R] entries the batch cap still allows
+  __shared__ int64_t s_pre[CHAIN_WINDOW];
+  __shared__ int32_t s_cnt[CHAIN_WINDOW];
+  __shared__ int32_t s_nm, s_k, s_done;
+  __shared__ int64_t s_cursor, s_base, s_basec;
+  if (threadIdx.x == 0) { s_nm = 0; s_k = 0; s_done = 0; s_cursor = 0; s_base = 0; s_basec = 0; }
   __syncthreads();
   for (int r = threadIdx.x; r < R; r += blockDim.x)
     if (a.maturity[r] <= a.now) {
@@ -391,69 +420,70 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
   __syncthreads();
   const int nm = s_nm;
   block_sort<true>(s_mat, s_id, nm);
-  for (int k = threadIdx.x; k < nm; k += blockDim.x) a.inst_order[k] = (int32_t)s_id[k];
-  if (threadIdx.x == 0) *a.n_mature = nm;
-  if (threadIdx.x >= 32) return;
-  const int lane = threadIdx.x;
-  const int64_t nq = (int64_t)w.ctl[1];
-  int64_t cursor = 0, base = 0, base_cnt = 0;         // queue position; running totals before it
-  for (int k = 0; k < nm && cursor < nq; k++) {
+  int64_t *s_bud = reinterpret_cast<int64_t *>(s_mat);
+  for (int k = threadIdx.x; k < nm; k += blockDim.x) {
     const int r = (int)s_id[k];
-    const ReplicaPlan pl = w.plan[r];
-    const int64_t span = nq - cursor;
-    int64_t room = span;                              // entries the batch cap still allows
-    if (pl.batch_cap != 0) {
-      const int64_t left = (int64_t)pl.batch_cap - pl.n_run;
-      room = left < room ? (left > 0 ? left : 0) : room;
-    }
-    // longest stretch m in [0, span] of queue positions whose entries that count stay within the budget
-    // and the batch room (both running totals never decrease)
-    const int64_t limit = base + pl.budget, limit_cnt = base_cnt + room;
-    auto fits = [&](int64_t m) { return w.prefix[cursor + m - 1] <= limit && (int64_t)w.prefix_cnt[cursor + m - 1] <= limit_cnt; };
-    int64_t lo = 0, hi = span;                        // fits(lo); the answer lies in [lo, hi]
-    {   // gallop: lane l tries m = 2^l
-      const int64_t m = INT64_C(1) << lane;
-      const bool ok = m <= span && fits(m);
-      const uint32_t b = __ballot_sync(0xffffffffu, ok);
-      const int f = __popc(b);                        // the lanes that fit are a prefix
-      if (f > 0) lo = INT64_C(1) << (f - 1);
-      if (f < 32) { const int64_t t = (INT64_C(1) << f) - 1; hi = t < hi ? t : hi; }
-    }
-    while (lo < hi) {
-      const int64_t step = (hi - lo + 31) / 32;
-      const int64_t cand = lo + (int64_t)(lane + 1) * step;
-      const bool ok = cand <= hi && fits(cand);
-      const int f = __popc(__ballot_sync(0xffffffffu, ok));
-      const int64_t nlo = lo + (int64_t)f * step;
-      int64_t nhi = lo + (int64_t)(f + 1) * step - 1;
-      if (nhi > hi) nhi = hi;
-      lo = nlo; hi = nhi;
-    }
-    const int64_t m = lo;
-    if (m > 0) {
-      const int64_t cost = w.prefix[cursor + m - 1] - base;
-      const int64_t cnt = (int64_t)w.prefix_cnt[cursor + m - 1] - base_cnt;
-      if (lane == 0) {
-        w.run_start[r] = (int32_t)cursor;
-        w.run_len[r] = (int32_t)m;
-        if (cnt > 0) {
-          int64_t lp = 0;
-          a.adm_cost[r] = cost;
-          a.adm_count[r] = (int32_t)cnt;
-          a.maturity_next[r] = dev_maturity_next(p, pl, cnt, cost, 0, &lp);
+    a.inst_order[k] = r;
+    const ReplicaPlan *pl = w.plan + r;
+    s_bud[k] = pl->budget;
+    int64_t room = INT32_MAX;
+    if (pl->batch_cap != 0) { const int64_t left = (int64_t)pl->batch_cap - pl->n_run; room = left > 0 ? left : 0; }
+    s_room[k] = (int32_t)(room < INT32_MAX ? room : INT32_MAX);
+  }
+  if (threadIdx.x == 0) *a.n_mature = nm;
+  const int lane = threadIdx.x & 31;
+  const int64_t nq = (int64_t)w.ctl[1];
+  for (int guard = 0; guard < 2 * nm + 4; guard++) {      // every round finishes an instance or refills for one
+    __syncthreads();
+    if (s_done || s_k >= nm || s_cursor >= nq) break;
+    // refill the window from the current position
+    const int64_t w0 = s_cursor;
+    const int64_t wn = nq - w0 < CHAIN_WINDOW ? nq - w0 : CHAIN_WINDOW;
+    for (int i = threadIdx.x; i < wn; i += blockDim.x) { s_pre[i] = w.prefix[w0 + i]; s_cnt[i] = w.prefix_cnt[w0 + i]; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      int k = s_k;
+      int64_t cursor = s_cursor, base = s_base, base_cnt = s_basec;
+      for (; k < nm && cursor < nq; k++) {
+        const int64_t span = nq - cursor, avail = w0 + wn - cursor;
+        const int64_t limit = base + s_bud[k], limit_cnt = base_cnt + s_room[k];
+        const int64_t off = cursor - w0 - 1;
+        const int64_t hiw = span < avail ? span : avail;
+        int64_t m = warp_longest(0, hiw, lane, [&](int64_t x) { return s_pre[off + x] <= limit && (int64_t)s_cnt[off + x] <= limit_cnt; });
+        if (m == hiw && hiw < span) {          // the stretch may go on past the window
+          if (cursor != w0) break;              // refill from here and search again
+          m = warp_longest(m, span, lane, [&](int64_t x) {
+            return w.prefix[cursor + x - 1] <= limit && (int64_t)w.prefix_cnt[cursor + x - 1] <= limit_cnt; });
+        }
+        if (m > 0) {
+          int64_t e_pre, e_cnt;
+          if (m <= avail) { e_pre = s_pre[off + m]; e_cnt = s_cnt[off + m]; }
+          else { e_pre = w.prefix[cursor + m - 1]; e_cnt = w.prefix_cnt[cursor + m - 1]; }
+          if (lane == 0) {
+            const int r = (int)s_id[k];
+            w.run_start[r] = (int32_t)cursor;
+            w.run_len[r] = (int32_t)m;
+            a.adm_cost[r] = e_pre - base;
+            a.adm_count[r] = (int32_t)(e_cnt - base_cnt);
+          }
+          cursor += m; base = e_pre; base_cnt = e_cnt;
+          if (cursor >= w0 + wn) { k++; break; }      // the window is used up
         }
       }
-      cursor += m;
-      base += cost;
-      base_cnt += cnt;
+      if (lane == 0) { s_k = k; s_cursor = cursor; s_base = base; s_basec = base_cnt; }
     }
   }
 }
 
-// the request -> instance binding of every dispatched row: one block per instance
-__global__ void __launch_bounds__(DISP_THREADS) k_disp_assign(const DispArgs a, const DispWork w, int slot) {
+// the request -> instance binding of every dispatched row, and dispatching step 4 (the new maturity
+// time of an instance that took requests): one block per instance
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_assign(const HfxParams p, const DispArgs a, const DispWork w, int slot) {
   const int r = blockIdx.x;
   const int32_t m = w.run_len[r], s0 = w.run_start[r];
+  if (threadIdx.x == 0 && a.adm_count[r] > 0) {
+    int64_t lp = 0;
+    a.maturity_next[r] = dev_maturity_next(p, w.plan[r], a.adm_count[r], a.adm_cost[r], 0, &lp);
+  }
   const int64_t bmax = (int64_t)w.ctl[4];
   for (int32_t q = threadIdx.x; q < m; q += blockDim.x) {
     const uint32_t row = w.val[slot][s0 + q];
@@ -467,7 +497,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_assign(const DispArgs a, 
 struct hfx_dispatch_ws { DispWork w; int ready; };
 
 int hfx_dispatch_configure() {
-  if (cudaFuncSetAttribute(k_disp_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, 12 * DISP_MAX_INSTANCES) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_disp_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * DISP_MAX_INSTANCES) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }
@@ -552,8 +582,8 @@ int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const 
   }
   int slot = 0;
   auto pass = [&](int shift) {
-    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_hist<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.ctl + 1, shift, w.hist, tiles_max, w.ctl + 2); }
-    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_scatter<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.key[slot ^ 1], w.val[slot ^ 1], w.ctl + 1, shift, w.hist, tiles_max); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_hist<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.ctl + 1, shift, w.hist); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_scatter<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.key[slot ^ 1], w.val[slot ^ 1], w.ctl + 1, shift, w.hist); }
     slot ^= 1;
   };
   for (int shift = 0; shift < 32; shift += 8) pass(shift);            // by request id
@@ -565,7 +595,7 @@ int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const 
   { KernelScope ks(s, KSLOT_DISPATCH); k_disp_plan<<<(R + DISP_THREADS - 1) / DISP_THREADS, DISP_THREADS, 0, st>>>(s->p, a, w); }
   { KernelScope ks(s, KSLOT_DISPATCH); k_disp_tilesum<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.ctl + 3); }
   { KernelScope ks(s, KSLOT_DISPATCH); k_disp_prefix<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.prefix, w.prefix_cnt, o->queue_order, o->n_queue); }
-  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_chain<<<1, 1024, 12 * (size_t)R, st>>>(s->p, a, w); }
-  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_assign<<<R, DISP_THREADS, 0, st>>>(a, w, slot); }
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_chain<<<1, 1024, 16 * (size_t)R, st>>>(s->p, a, w); }
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_assign<<<R, DISP_THREADS, 0, st>>>(s->p, a, w, slot); }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }
