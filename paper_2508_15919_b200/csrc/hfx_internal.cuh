@@ -206,7 +206,7 @@ __device__ inline void dev_plan(const HfxParams &p, const hfx_replica_cfg &cfg, 
 
 // The same plan computed by a whole warp (all 32 lanes call with the same arguments and get the same
 // result).  The class minima are taken by lanes from a copy of the class tables in shared memory
-// (cls_ttft / cls_tpot, HFX_MAX_CLASSES entries each); the largest safe n comes from a 128-way search
+// (cls_ttft / cls_tpot, HFX_MAX_CLASSES entries each); the largest safe n comes from a 32-way search
 // on the bound itself, E_p(n) * (2 TPOT - E_d) <= TTFT * (TPOT - E_d), compared in 128 bits: for
 // integer E_p that is the same set of n as E_p(n) <= floor(TTFT (TPOT - E_d) / (2 TPOT - E_d)), and no
 // division is needed.
@@ -230,13 +230,9 @@ __device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t n
   if (!fits(0)) return 0;
   int64_t lo = 0, hi = cap;          // fits(lo); the answer lies in [lo, hi]
   while (lo < hi) {
-    const int64_t step = (int64_t)(((uint64_t)(hi - lo) + 127u) >> 7);
-    int m = 0;
-#pragma unroll
-    for (int j = 0; j < 4; j++) {    // candidate index j * 32 + lane: E_p is monotone, so the ones that fit are a prefix
-      const int64_t cand = lo + (int64_t)(j * 32 + lane + 1) * step;
-      m += __popc(__ballot_sync(0xffffffffu, cand <= hi && fits(cand)));
-    }
+    const int64_t step = (int64_t)(((uint64_t)(hi - lo) + 31u) >> 5);
+    const int64_t cand = lo + (int64_t)(lane + 1) * step;
+    const int m = __popc(__ballot_sync(0xffffffffu, cand <= hi && fits(cand)));     // E_p is monotone: the ones that fit are a prefix
     const int64_t nlo = lo + (int64_t)m * step;
     int64_t nhi = lo + (int64_t)(m + 1) * step - 1;
     if (nhi > hi) nhi = hi;
