@@ -38,7 +38,7 @@ KERNEL_BYTES_PER_ROW = {"k_front": 51, "k_count": 26, "k_colscan": 0, "k_regroup
 STEPS_PER_EPISODE = 10
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel on this workload,
 # taken from the ncu capture summarised under profiles/; absent = no capture of the current kernel
-NCU_TRAFFIC_BYTES = {"k_count": 27.28e6 + 0.01e6, "k_regroup": 46.71e6 + 3.30e6, "k_segment(small)": 18.67e6 + 1.68e6}
+NCU_TRAFFIC_BYTES = {"k_front": 44.70e6 + 4.27e6, "k_segment(small)": 18.09e6 + 1.09e6}
 
 
 def _peaks():
