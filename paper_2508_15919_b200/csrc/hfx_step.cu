@@ -1,6 +1,7 @@
 // hfx_sched_step: one scheduling iteration over the whole request table.
 //
-// Pipeline (all on one stream, no host synchronisation):
+// Pipeline (all on one stream, no host synchronisation).  The first four stages run as ONE cooperative
+// kernel, k_front, when every tile's block can be resident at once; otherwise as kernels of their own:
 //   k_count     per-tile histogram of replica_id (shared memory), one matrix row per tile
 //   k_colscan   column-wise exclusive scan of the tile histograms: where each tile's rows of each
 //               replica start inside the replica's range; per-replica totals
