@@ -419,3 +419,43 @@ def test_dispatch_shared_queue_workload():
     wl.maturity[::7] = wl.now[0] + 5            # some instances have not matured
     g = assert_dispatch_parity(wl, int(wl.now[0]))
     assert g["n_queue"][0] > 300_000 and g["adm_count"].sum() > 10_000
+
+
+def test_dispatch_argument_errors_and_bad_rows():
+    import paper_2508_15919_b200 as hfx
+    wl = gen.random_table(40, 300, 3, modes=(gen.COLOCATED,))
+    now = int(wl.now.max())
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    mat = torch.from_numpy(wl.maturity).cuda()
+    out = hfx.DispatchOut(300, 3)
+    bad = hfx.DispatchOut(300, 3)
+    bad.t["assign"] = torch.zeros(304, dtype=torch.int32, device="cuda")[1:]
+    with pytest.raises(hfx.HfxError) as e:
+        sched.dispatch_step(tab, now, mat, bad)
+    assert e.value.code == -2
+    bad = hfx.DispatchOut(300, 3)
+    bad.t["n_queue"] = None
+    with pytest.raises(hfx.HfxError) as e:
+        sched.dispatch_step(tab, now, mat, bad)
+    assert e.value.code == -1
+    big = hfx.DeviceTable.from_numpy(gen.random_table(41, 301, 3).table)
+    with pytest.raises(hfx.HfxError) as e:
+        sched.dispatch_step(big, now, mat, out)
+    assert e.value.code == -3
+    sched.dispatch_step(tab, now, mat, out)          # still usable
+    assert sched.status() == 0
+    sched.close()
+    # a scheduler with a P-stage or D-stage replica has no shared colocated queue to dispatch
+    wl2 = gen.random_table(42, 100, 2, modes=(gen.PREFILL,))
+    s2 = make_sched(wl2)
+    with pytest.raises(hfx.HfxError) as e:
+        s2.dispatch_step(hfx.DeviceTable.from_numpy(wl2.table), now, torch.from_numpy(wl2.maturity).cuda(), hfx.DispatchOut(100, 2))
+    assert e.value.code == -1
+    s2.close()
+    # rows with ids or lengths outside the domain are flagged and take no part
+    wl3 = gen.random_table(43, 2000, 5, modes=(gen.COLOCATED,))
+    wl3.table["class_id"][::97] = 200
+    wl3.table["prompt_len"][5::131] = -3
+    wl3.table["replica_id"][7::53] = 99
+    assert_dispatch_parity(wl3, int(wl3.now.max()))
