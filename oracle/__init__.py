@@ -99,6 +99,17 @@ class _DispatchOut(C.Structure):
     _fields_ = [(k, C.c_void_p) for k, _, _ in _DISPATCH_OUT]
 
 
+class _SloWindow(C.Structure):
+    _fields_ = [("w", C.c_int32), ("prio", C.c_void_p), ("ttft", C.c_void_p), ("tpot", C.c_void_p), ("queue", C.c_void_p)]
+
+
+SLO_BOUND_KEYS = ("ttft_min", "ttft_max", "ttft_min_relaxed", "tpot_min", "tpot_max", "tpot_min_relaxed")
+
+
+class _SloBounds(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in SLO_BOUND_KEYS]
+
+
 class _ScaleOut(C.Structure):
     _fields_ = [("counts", C.c_void_p), ("used_blocks", C.c_void_p), ("decision", C.c_void_p)]
 
@@ -130,6 +141,9 @@ def lib():
                               C.c_int32, C.POINTER(_SimOut)]
         L.ora_dispatch.restype = C.c_uint32
         L.ora_dispatch.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_DispatchOut)]
+        L.ora_slo_map.restype = C.c_uint32
+        L.ora_slo_map.argtypes = [C.c_int32, C.POINTER(_SloWindow), C.POINTER(_SloBounds), C.c_void_p, C.c_void_p,
+                                  C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ora_scale.restype = C.c_uint32
         L.ora_scale.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_ScaleParams),
                                 C.POINTER(_ScaleOut)]
@@ -236,6 +250,26 @@ def dispatch(wl, now: int) -> Dict[str, np.ndarray]:
             out[k] = out[k][:n]
     out["status"] = int(st)
     return out
+
+
+def slo_map(n_prio: int, window: Dict[str, np.ndarray], bounds: Dict[str, np.ndarray], last_queue: np.ndarray,
+            pending: np.ndarray, new_prio: np.ndarray) -> Dict[str, np.ndarray]:
+    """Priority-based SLO mapping: TTFT / TPOT targets of the requests `new_prio` (row order) from the
+    sliding window {prio, ttft, tpot, queue}; returns the targets and the updated last_queue."""
+    L = lib()
+    wp = np.ascontiguousarray(window["prio"], np.int32)
+    wt, wo, wq = (np.ascontiguousarray(window[k], np.int64) for k in ("ttft", "tpot", "queue"))
+    win = _SloWindow(int(wp.shape[0]), wp.ctypes.data, wt.ctypes.data, wo.ctypes.data, wq.ctypes.data)
+    barr = {k: np.ascontiguousarray(bounds[k], np.int64) for k in SLO_BOUND_KEYS}
+    bs = _SloBounds(*[barr[k].ctypes.data for k in SLO_BOUND_KEYS])
+    lq = np.ascontiguousarray(last_queue, np.int64).copy()
+    pend = np.ascontiguousarray(pending, np.int32)
+    npr = np.ascontiguousarray(new_prio, np.int32)
+    n = int(npr.shape[0])
+    ttft = np.zeros(max(n, 1), np.int64); tpot = np.zeros(max(n, 1), np.int64)
+    st = L.ora_slo_map(int(n_prio), C.byref(win), C.byref(bs), lq.ctypes.data, pend.ctypes.data, n, npr.ctypes.data,
+                       ttft.ctypes.data, tpot.ctypes.data)
+    return {"ttft_slo": ttft[:n], "tpot_slo": tpot[:n], "last_queue": lq, "status": int(st)}
 
 
 def scale_tick(wl, now: int, total_blocks: np.ndarray, **kw) -> Dict[str, np.ndarray]:

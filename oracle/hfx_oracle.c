@@ -793,3 +793,88 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
   free(n_run); free(sum_kv); free(min_tpot); free(q); free(inst);
   return status;
 }
+
+/* ==========================================================================
+ * Priority-based SLO mapping (Sec. 3.3.2, steps (1)-(5)): a request that
+ * carries only a priority p in [0, N) gets its TTFT and TPOT targets from the
+ * recent history.  The history is a sliding window of completed requests
+ * (priority, measured TTFT, measured TPOT, queueing delay).  With C_i the
+ * number of window records of priority i,
+ *     base = C_0 + ... + C_{p-1},   offset = floor((p + 1) * C_p / (N + 1)),
+ * and the provisional targets are the (base + offset)-th smallest TTFT and
+ * TPOT of the window (step 3).  Step 4 subtracts from the TTFT the queueing
+ * delay of the chosen reference record in excess of the queueing delay last
+ * seen for this priority, and remembers the reference's delay.  Step 5 clamps
+ * both targets into the priority's range; while requests of a higher priority
+ * are pending the strict lower bound applies, otherwise the relaxed one.
+ * Requests are served in row order, so the second request of a priority in
+ * one call sees the delay the first one left behind.
+ *
+ * reading: the two windows are ordered by value, ties by record position.
+ * reading: an index past the end of the window means its last record; with an
+ *   empty window the targets are the upper bounds of the range.
+ * reading: "higher-priority requests are pending" = some priority below p has
+ *   a positive pending count; the relaxed lower bound is a second per-priority
+ *   parameter.
+ * reading: window records and requests whose priority is outside [0, N) are
+ *   ignored (flagged); such a request gets 0, 0.
+ * ========================================================================== */
+typedef struct {
+  int32_t w;
+  const int32_t *prio;
+  const int64_t *ttft, *tpot, *queue;
+} ora_slo_window;
+
+typedef struct {
+  const int64_t *ttft_min, *ttft_max, *ttft_min_relaxed, *tpot_min, *tpot_max, *tpot_min_relaxed;
+} ora_slo_bounds;
+
+typedef struct { int64_t v; int32_t pos; } val_pos;
+static int cmp_val_pos(const void *pa, const void *pb) {
+  const val_pos *a = (const val_pos *)pa, *b = (const val_pos *)pb;
+  if (a->v != b->v) return a->v < b->v ? -1 : 1;
+  return a->pos < b->pos ? -1 : (a->pos > b->pos ? 1 : 0);
+}
+
+static int64_t clamp_i64(int64_t x, int64_t lo, int64_t hi) { return x < lo ? lo : (x > hi ? hi : x); }
+
+uint32_t ora_slo_map(int32_t n_prio, const ora_slo_window *win, const ora_slo_bounds *b, int64_t *last_queue,
+                     const int32_t *pending, int64_t n_new, const int32_t *new_prio, int64_t *ttft_out,
+                     int64_t *tpot_out) {
+  uint32_t status = 0;
+  val_pos *by_ttft = (val_pos *)malloc(sizeof(val_pos) * (size_t)(win->w + 1));
+  val_pos *by_tpot = (val_pos *)malloc(sizeof(val_pos) * (size_t)(win->w + 1));
+  int64_t *C = (int64_t *)calloc((size_t)n_prio + 1, sizeof(int64_t));
+  int32_t w = 0;
+  for (int32_t j = 0; j < win->w; j++) {
+    if (win->prio[j] < 0 || win->prio[j] >= n_prio) { status |= BAD_CLASS; continue; }
+    C[win->prio[j]] += 1;
+    by_ttft[w].v = win->ttft[j]; by_ttft[w].pos = j;
+    by_tpot[w].v = win->tpot[j]; by_tpot[w].pos = j;
+    w++;
+  }
+  qsort(by_ttft, (size_t)w, sizeof(val_pos), cmp_val_pos);
+  qsort(by_tpot, (size_t)w, sizeof(val_pos), cmp_val_pos);
+  for (int64_t r = 0; r < n_new; r++) {
+    const int32_t p = new_prio[r];
+    if (p < 0 || p >= n_prio) { status |= BAD_CLASS; ttft_out[r] = 0; tpot_out[r] = 0; continue; }
+    int64_t ttft = b->ttft_max[p], tpot = b->tpot_max[p];
+    if (w > 0) {
+      int64_t base = 0;
+      for (int32_t i = 0; i < p; i++) base += C[i];
+      const int64_t offset = ((int64_t)(p + 1) * C[p]) / (n_prio + 1);
+      int64_t idx = base + offset;
+      if (idx > w - 1) idx = w - 1;
+      const int64_t q_ref = win->queue[by_ttft[idx].pos];
+      ttft = by_ttft[idx].v - (q_ref - last_queue[p]);
+      last_queue[p] = q_ref;
+      tpot = by_tpot[idx].v;
+    }
+    int higher_pending = 0;
+    for (int32_t i = 0; i < p; i++) if (pending[i] > 0) higher_pending = 1;
+    ttft_out[r] = clamp_i64(ttft, higher_pending ? b->ttft_min[p] : b->ttft_min_relaxed[p], b->ttft_max[p]);
+    tpot_out[r] = clamp_i64(tpot, higher_pending ? b->tpot_min[p] : b->tpot_min_relaxed[p], b->tpot_max[p]);
+  }
+  free(by_ttft); free(by_tpot); free(C);
+  return status;
+}

@@ -380,3 +380,48 @@ def test_dispatch_entry_that_fits_nowhere_is_passed_over():
     assert list(o["assign"][80:86]) == [-1, 1, 1, 1, -1, -1]
     assert list(o["adm_cost"]) == [0, 1441, 0] and list(o["adm_count"]) == [0, 3, 0]
     assert o["maturity_next"][1] - now == PINS["disp_mat1_delta_long"] and o["maturity_next"][0] == now - 5
+
+
+# ---- priority-based SLO mapping -------------------------------------------------------------------------
+def _slo_hand_case():
+    win = {"prio": np.array([0, 1, 0, 2, 1, 2]), "ttft": np.array([100, 300, 150, 900, 250, 700]) * MS,
+           "tpot": np.array([20, 40, 25, 80, 35, 60]) * MS, "queue": np.array([10, 50, 30, 400, 20, 200]) * MS}
+    bounds = {"ttft_min": np.array([150, 200, 700]) * MS, "ttft_max": np.array([200, 1000, 5000]) * MS,
+              "ttft_min_relaxed": np.array([50, 100, 200]) * MS, "tpot_min": np.array([30, 30, 50]) * MS,
+              "tpot_max": np.array([30, 50, 100]) * MS, "tpot_min_relaxed": np.array([10, 20, 30]) * MS}
+    return win, bounds, np.array([10, 30, 100]) * MS, np.array([1, 2, 1, 0])
+
+
+def test_slo_mapping_hand_worked():
+    win, bounds, last, new = _slo_hand_case()
+    o = oracle.slo_map(3, win, bounds, last, np.array([0, 3, 0]), new)
+    assert o["status"] == 0
+    assert list(o["ttft_slo"]) == [PINS["slo_req0_ttft_ms"] * MS, PINS["slo_req1_ttft_ms_contended"] * MS,
+                                   PINS["slo_req2_ttft_ms"] * MS, PINS["slo_req3_ttft_ms"] * MS]
+    assert list(o["tpot_slo"]) == [40 * MS, 80 * MS, 40 * MS, 20 * MS]
+    assert list(o["last_queue"]) == [10 * MS, 50 * MS, 400 * MS]
+    o = oracle.slo_map(3, win, bounds, last, np.array([0, 0, 0]), new)
+    assert o["ttft_slo"][1] == PINS["slo_req1_ttft_ms_free"] * MS
+    # strict bounds when the highest priority is pending: p=1 TPOT 40 stays, p=2 TTFT 600 -> 700; p=0 never has a higher one
+    o = oracle.slo_map(3, win, bounds, last, np.array([5, 0, 0]), new)
+    assert list(o["ttft_slo"]) == [280 * MS, 700 * MS, 300 * MS, 100 * MS] and o["tpot_slo"][3] == 20 * MS
+    # an empty window: the loosest targets of each range; last_queue untouched
+    empty = {k: v[:0] for k, v in win.items()}
+    o = oracle.slo_map(3, empty, bounds, last, np.array([0, 0, 0]), new)
+    assert list(o["ttft_slo"]) == [1000 * MS, 5000 * MS, 1000 * MS, 200 * MS] and list(o["last_queue"]) == list(last)
+    # a priority outside [0, N): flagged, no targets
+    o = oracle.slo_map(3, win, bounds, last, np.array([0, 0, 0]), np.array([7, 0]))
+    assert o["status"] == 2 and o["ttft_slo"][0] == 0 and o["ttft_slo"][1] == 100 * MS
+
+
+def test_slo_mapping_quantiles_against_numpy():
+    # with one priority level the index is floor(C/2): the upper median of the window; ranges wide open
+    rng = np.random.default_rng(3)
+    for w in (1, 2, 7, 100, 1001):
+        win = {"prio": np.zeros(w, np.int64), "ttft": rng.integers(1, 10**9, w), "tpot": rng.integers(1, 10**8, w),
+               "queue": np.zeros(w, np.int64)}
+        big = np.array([1 << 60])
+        bounds = {"ttft_min": -big, "ttft_max": big, "ttft_min_relaxed": -big, "tpot_min": -big, "tpot_max": big,
+                  "tpot_min_relaxed": -big}
+        o = oracle.slo_map(1, win, bounds, np.array([0]), np.array([0]), np.array([0]))
+        assert o["ttft_slo"][0] == np.sort(win["ttft"])[w // 2] and o["tpot_slo"][0] == np.sort(win["tpot"])[w // 2]
