@@ -275,6 +275,48 @@ typedef struct hfx_dispatch_out {
 int hfx_dispatch_step(hfx_sched *s, const hfx_table *table, int64_t now_ns,
                       const int64_t *maturity_ns, const hfx_dispatch_out *out);
 
+/* Priority-based SLO mapping (Sec. 3.3.2 "Priority-Based SLO Mapping", its five
+ * steps): requests that carry only a priority p in [0, n_prio), 0 highest, get
+ * their TTFT and TPOT targets from recent history.  `win` is the sliding window
+ * of completed requests (device arrays of `w` records, w <= 4096, in any
+ * order): priority, measured TTFT, measured TPOT, queueing delay.  With C_i the
+ * window records of priority i, base = C_0 + ... + C_{p-1} and offset =
+ * floor((p + 1) C_p / (n_prio + 1)); the provisional targets are the
+ * (base + offset)-th smallest TTFT and TPOT of the window (ties by record
+ * position; an index past the end means the last record; an empty window gives
+ * the upper bounds of the priority's range).  The TTFT is then reduced by the
+ * reference record's queueing delay in excess of last_queue_ns[p] (device,
+ * [n_prio], in/out: it becomes the reference's delay), so within one call only
+ * the first request of a priority (lowest row) sees a correction.  Both targets
+ * are clamped into the priority's range; the lower bound is the strict one
+ * while some higher priority has pending[i] > 0 (device, [n_prio]), the relaxed
+ * one otherwise.  new_prio [n_new] and the outputs [n_new] are device arrays;
+ * a request or window record whose priority is outside [0, n_prio) is ignored
+ * and sets HFX_ST_BAD_CLASS (the request gets 0, 0).
+ * Errors: HFX_E_ARG (n_prio outside 1..64, w < 0, NULL), HFX_E_CAPACITY
+ * (w > 4096), HFX_E_ALIGN, HFX_E_CUDA. */
+typedef struct hfx_slo_window {
+  const int32_t *prio;      /* [w] */
+  const int64_t *ttft_ns;   /* [w] */
+  const int64_t *tpot_ns;   /* [w] */
+  const int64_t *queue_ns;  /* [w] */
+  int32_t w;
+  int32_t reserved;
+} hfx_slo_window;
+
+typedef struct hfx_slo_bounds {   /* device arrays of n_prio entries */
+  const int64_t *ttft_min_ns;
+  const int64_t *ttft_max_ns;
+  const int64_t *ttft_min_relaxed_ns;
+  const int64_t *tpot_min_ns;
+  const int64_t *tpot_max_ns;
+  const int64_t *tpot_min_relaxed_ns;
+} hfx_slo_bounds;
+
+int hfx_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const hfx_slo_bounds *bounds,
+                int64_t *last_queue_ns, const int32_t *pending, const int32_t *new_prio, int64_t n_new,
+                int64_t *ttft_slo_ns, int64_t *tpot_slo_ns);
+
 /* Trace-driven simulation (events are request arrivals and iteration
  * completions, Problem Definition; metrics are Eq. 2 and the TTFT / TPOT
  * definitions).  `table` holds n_traces traces back to back, trace j being
@@ -337,9 +379,9 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
  * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
  * 6 oversize path, 7 simulator, 8 scaler tick, 9 fused front end, 10 the kernels of
- * hfx_dispatch_step together; hfx_kernel_name gives the name of a slot (NULL past
- * the end). */
-#define HFX_N_KERNELS 11
+ * hfx_dispatch_step together, 11 those of hfx_slo_map; hfx_kernel_name gives the
+ * name of a slot (NULL past the end). */
+#define HFX_N_KERNELS 12
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
   int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */

@@ -21,9 +21,9 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step"]
+                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map"]
 NOALLOC_MAX_REPLICAS = 4096
-N_KERNELS = 11
+N_KERNELS = 12
 
 
 class HfxError(RuntimeError):
@@ -82,7 +82,7 @@ SIM_OUT_FIELDS = [("iters_executed", torch.int32), ("finished", torch.int32), ("
 
 
 class _Profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 11), ("launches", C.c_int64 * 11)]
+    _fields_ = [("ms", C.c_double * 12), ("launches", C.c_int64 * 12)]
 
 
 class _ScaleParams(C.Structure):
@@ -104,6 +104,18 @@ DISPATCH_OUT_FIELDS = [("assign", torch.int32, "n"), ("queue_order", torch.int32
                        ("budget", torch.int64, "R"), ("e_d_ns", torch.int64, "R"), ("n_run", torch.int32, "R"),
                        ("sum_kv", torch.int64, "R"), ("adm_cost", torch.int64, "R"), ("adm_count", torch.int32, "R"),
                        ("maturity_next", torch.int64, "R")]
+
+
+SLO_BOUND_FIELDS = ("ttft_min_ns", "ttft_max_ns", "ttft_min_relaxed_ns", "tpot_min_ns", "tpot_max_ns", "tpot_min_relaxed_ns")
+
+
+class _SloWindow(C.Structure):
+    _fields_ = [("prio", C.c_void_p), ("ttft_ns", C.c_void_p), ("tpot_ns", C.c_void_p), ("queue_ns", C.c_void_p),
+                ("w", C.c_int32), ("reserved", C.c_int32)]
+
+
+class _SloBounds(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in SLO_BOUND_FIELDS]
 
 
 class _DispatchOut(C.Structure):
@@ -130,6 +142,9 @@ def load_library():
     L.hfx_sched_step.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_ReplicaState), C.POINTER(_StepOut), C.c_uint32]
     L.hfx_dispatch_step.restype = C.c_int
     L.hfx_dispatch_step.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_DispatchOut)]
+    L.hfx_slo_map.restype = C.c_int
+    L.hfx_slo_map.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_SloWindow), C.POINTER(_SloBounds), C.c_void_p, C.c_void_p,
+                              C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
     L.hfx_sim_run.restype = C.c_int
     L.hfx_sim_run.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_void_p, C.c_int32, C.c_int32, C.POINTER(_SimOut)]
     L.hfx_sched_status.restype = C.c_int
@@ -323,6 +338,23 @@ class Scheduler:
         rc = self._L.hfx_dispatch_step(self._h, C.byref(ts), int(now_ns), _ptr(maturity), C.byref(os_))
         if rc != 0:
             raise HfxError(rc, "hfx_dispatch_step")
+
+    def slo_map(self, n_prio: int, window: Dict[str, torch.Tensor], bounds: Dict[str, torch.Tensor],
+                last_queue: torch.Tensor, pending: torch.Tensor, new_prio: torch.Tensor, ttft_out: torch.Tensor,
+                tpot_out: torch.Tensor):
+        """hfx_slo_map: window = {prio int32, ttft_ns, tpot_ns, queue_ns int64} device tensors of w records;
+        bounds = the six per-priority int64 device tensors of SLO_BOUND_FIELDS; last_queue int64 [n_prio]
+        (updated in place); pending int32 [n_prio]; new_prio int32 [n_new]; outputs int64 [n_new]."""
+        w = int(window["prio"].shape[0])
+        win = _SloWindow(_ptr(window["prio"]) if w else None, _ptr(window["ttft_ns"]) if w else None,
+                         _ptr(window["tpot_ns"]) if w else None, _ptr(window["queue_ns"]) if w else None, w, 0)
+        bs = _SloBounds(*[_ptr(bounds[k]) for k in SLO_BOUND_FIELDS])
+        n_new = int(new_prio.shape[0])
+        rc = self._L.hfx_slo_map(self._h, int(n_prio), C.byref(win), C.byref(bs), _ptr(last_queue), _ptr(pending),
+                                 _ptr(new_prio) if n_new else None, n_new, _ptr(ttft_out) if n_new else None,
+                                 _ptr(tpot_out) if n_new else None)
+        if rc != 0:
+            raise HfxError(rc, "hfx_slo_map")
 
     def scale_tick(self, table: DeviceTable, now_ns: int, total_blocks: torch.Tensor, counts: torch.Tensor,
                    used_blocks: torch.Tensor, decision: torch.Tensor, window_ns: int = 10_000_000_000,

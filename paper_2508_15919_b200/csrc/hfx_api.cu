@@ -8,6 +8,7 @@ int hfx_regroup_configure();
 int hfx_segment_configure();
 int hfx_sim_configure();
 int hfx_dispatch_configure();
+int hfx_slomap_configure();
 int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_trace_off, int32_t n_traces,
                           int32_t max_trace_rows, int32_t iters, const hfx_sim_out *o, uint32_t *d_work_counter);
 
@@ -67,7 +68,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     cudaGetLastError();
     return HFX_E_CUDA;
   }
-  if (hfx_regroup_configure() != HFX_OK || hfx_segment_configure() != HFX_OK || hfx_sim_configure() != HFX_OK || hfx_dispatch_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
+  if (hfx_regroup_configure() != HFX_OK || hfx_segment_configure() != HFX_OK || hfx_sim_configure() != HFX_OK || hfx_dispatch_configure() != HFX_OK || hfx_slomap_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
 
   hfx_sched_host *h = new (std::nothrow) hfx_sched_host();
   if (!h) return HFX_E_NOMEM;
@@ -117,6 +118,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   ok = ok && cudaMalloc(&s->d_rec, sizeof(HfxRec) * (size_t)max_rows) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_barrier, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_front_bar, 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_slo, hfx_slomap_workspace_bytes()) == cudaSuccess;
   s->front_enabled = 1; s->front_arrivals = 0; s->front_smem_cached = 0; s->front_capacity = 0;
   ok = ok && cudaMalloc(&h->d_trace_off, sizeof(int32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&h->d_work_counter, 256) == cudaSuccess;
@@ -159,7 +161,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   cudaFree(s->d_cfg); cudaFree(s->d_mode); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
   cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_mode);
-  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier); cudaFree(s->d_front_bar);
+  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier); cudaFree(s->d_front_bar); cudaFree(s->d_slo);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();
   if (s->brackets) {
@@ -221,6 +223,23 @@ extern "C" int hfx_dispatch_step(hfx_sched *s, const hfx_table *t, int64_t now_n
     if (h->h_cfg[r].token_cap > cap_max) cap_max = h->h_cfg[r].token_cap;
   }
   return hfx_launch_dispatch(s, t, now_ns, maturity_ns, o, cap_max);
+}
+
+extern "C" int hfx_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const hfx_slo_bounds *b,
+                           int64_t *last_queue_ns, const int32_t *pending, const int32_t *new_prio, int64_t n_new,
+                           int64_t *ttft_slo_ns, int64_t *tpot_slo_ns) {
+  if (!s || !win || !b || !last_queue_ns || !pending) return HFX_E_ARG;
+  if (n_prio < 1 || n_prio > HFX_MAX_CLASSES || win->w < 0 || n_new < 0) return HFX_E_ARG;
+  if (win->w > 4096) return HFX_E_CAPACITY;
+  if (win->w > 0 && (!win->prio || !win->ttft_ns || !win->tpot_ns || !win->queue_ns)) return HFX_E_ARG;
+  if (n_new > 0 && (!new_prio || !ttft_slo_ns || !tpot_slo_ns)) return HFX_E_ARG;
+  const void *bp[] = {b->ttft_min_ns, b->ttft_max_ns, b->ttft_min_relaxed_ns, b->tpot_min_ns, b->tpot_max_ns, b->tpot_min_relaxed_ns};
+  for (const void *p : bp) if (!p) return HFX_E_ARG;
+  const void *all[] = {win->prio, win->ttft_ns, win->tpot_ns, win->queue_ns, b->ttft_min_ns, b->ttft_max_ns, b->ttft_min_relaxed_ns,
+                       b->tpot_min_ns, b->tpot_max_ns, b->tpot_min_relaxed_ns, last_queue_ns, pending, new_prio, ttft_slo_ns,
+                       tpot_slo_ns};
+  for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
+  return hfx_launch_slo_map(s, n_prio, win, b, last_queue_ns, pending, new_prio, n_new, ttft_slo_ns, tpot_slo_ns);
 }
 
 extern "C" int hfx_sim_run(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
@@ -304,6 +323,6 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 
 extern "C" const char *hfx_kernel_name(int slot) {
   static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
-                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch"};
-  return (slot >= 0 && slot < 11) ? names[slot] : nullptr;
+                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch", "k_slo_map"};
+  return (slot >= 0 && slot < 12) ? names[slot] : nullptr;
 }

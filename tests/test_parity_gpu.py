@@ -459,3 +459,64 @@ def test_dispatch_argument_errors_and_bad_rows():
     wl3.table["prompt_len"][5::131] = -3
     wl3.table["replica_id"][7::53] = 99
     assert_dispatch_parity(wl3, int(wl3.now.max()))
+
+
+# ---- priority-based SLO mapping ---------------------------------------------------------------------------
+def _slo_parity(n_prio, win, bounds, last, pending, new, calls=2):
+    import paper_2508_15919_b200 as hfx
+    wl = gen.random_table(1, 16, 1)
+    sched = make_sched(wl)
+    dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a, dt)).cuda()
+    w = {"prio": dev(win["prio"], np.int32), "ttft_ns": dev(win["ttft"], np.int64), "tpot_ns": dev(win["tpot"], np.int64),
+         "queue_ns": dev(win["queue"], np.int64)}
+    b = {k + "_ns": dev(bounds[k], np.int64) for k in oracle.SLO_BOUND_KEYS}
+    lq = dev(last, np.int64)
+    lq_cpu = np.ascontiguousarray(last, np.int64)
+    pend = dev(pending, np.int32)
+    npr = dev(new, np.int32)
+    n = int(npr.shape[0])
+    t_out = torch.full((max(n, 1),), -7, dtype=torch.int64, device="cuda")
+    p_out = torch.full((max(n, 1),), -7, dtype=torch.int64, device="cuda")
+    for _ in range(calls):       # the second call starts from the delays the first one left behind
+        sched.slo_map(n_prio, w, b, lq, pend, npr, t_out, p_out)
+        st = sched.status()
+        c = oracle.slo_map(n_prio, win, bounds, lq_cpu, pending, new)
+        lq_cpu = c["last_queue"]
+        assert st == c["status"]
+        assert np.array_equal(t_out.cpu().numpy()[:n], c["ttft_slo"]), (t_out.cpu().numpy()[:8], c["ttft_slo"][:8])
+        assert np.array_equal(p_out.cpu().numpy()[:n], c["tpot_slo"])
+        assert np.array_equal(lq.cpu().numpy(), c["last_queue"])
+    sched.close()
+    return c
+
+
+def test_slo_mapping_hand_worked_and_edges():
+    win = {"prio": np.array([0, 1, 0, 2, 1, 2]), "ttft": np.array([100, 300, 150, 900, 250, 700]) * MS,
+           "tpot": np.array([20, 40, 25, 80, 35, 60]) * MS, "queue": np.array([10, 50, 30, 400, 20, 200]) * MS}
+    bounds = {"ttft_min": np.array([150, 200, 700]) * MS, "ttft_max": np.array([200, 1000, 5000]) * MS,
+              "ttft_min_relaxed": np.array([50, 100, 200]) * MS, "tpot_min": np.array([30, 30, 50]) * MS,
+              "tpot_max": np.array([30, 50, 100]) * MS, "tpot_min_relaxed": np.array([10, 20, 30]) * MS}
+    last = np.array([10, 30, 100]) * MS
+    c = _slo_parity(3, win, bounds, last, np.array([0, 3, 0]), np.array([1, 2, 1, 0]))
+    _slo_parity(3, win, bounds, last, np.array([0, 0, 0]), np.array([1, 2, 1, 0]))
+    _slo_parity(3, {k: v[:0] for k, v in win.items()}, bounds, last, np.array([0, 0, 0]), np.array([1, 2, 1, 0]))    # empty window
+    _slo_parity(3, win, bounds, last, np.array([1, 0, 0]), np.array([], np.int32))                                  # no requests
+    bad = dict(win); bad["prio"] = np.array([0, 9, 0, -1, 1, 2])
+    _slo_parity(3, bad, bounds, last, np.array([0, 0, 1]), np.array([1, 5, 2, -2, 0]))                              # bad priorities
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_slo_mapping_random(seed):
+    rng = np.random.default_rng(seed)
+    N = int(rng.integers(1, 65)) if seed else 64
+    w = [4096, 1, 37, 1000, 4095, 513][seed]
+    ties = seed % 2 == 1
+    win = {"prio": rng.integers(0, N, w), "ttft": rng.integers(1, 50 if ties else 10**10, w),
+           "tpot": rng.integers(1, 20 if ties else 10**9, w), "queue": rng.integers(0, 10**9, w)}
+    lo = rng.integers(0, 10**8, N)
+    bounds = {"ttft_min": lo + 10**8, "ttft_max": lo + 5 * 10**9, "ttft_min_relaxed": lo,
+              "tpot_min": lo // 10 + 10**7, "tpot_max": lo // 10 + 5 * 10**8, "tpot_min_relaxed": lo // 10}
+    last = rng.integers(0, 10**9, N)
+    pending = rng.integers(0, 2, N) * rng.integers(0, 2, N)
+    new = rng.integers(0, N, 10_000 + seed)
+    _slo_parity(N, win, bounds, last, pending, new)
