@@ -144,6 +144,9 @@ def lib():
         L.ora_slo_map.restype = C.c_uint32
         L.ora_slo_map.argtypes = [C.c_int32, C.POINTER(_SloWindow), C.POINTER(_SloBounds), C.c_void_p, C.c_void_p,
                                   C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ora_pd_migrate.restype = C.c_uint32
+        L.ora_pd_migrate.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                                     C.c_void_p]
         L.ora_scale.restype = C.c_uint32
         L.ora_scale.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_ScaleParams),
                                 C.POINTER(_ScaleOut)]
@@ -250,6 +253,19 @@ def dispatch(wl, now: int) -> Dict[str, np.ndarray]:
             out[k] = out[k][:n]
     out["status"] = int(st)
     return out
+
+
+def pd_migrate(wl, pair: np.ndarray, x0: int, x1: int) -> Dict[str, int]:
+    """Hand-off of prefilled requests from the P instances of wl to their partner D instances, in place
+    (wl.table["replica_id"], wl.table["state"], wl.now)."""
+    L = lib()
+    ctx = _Ctx(wl)
+    pr = np.ascontiguousarray(pair, np.int32)
+    moved = np.zeros(1, np.int32)
+    assert wl.table["replica_id"].flags["WRITEABLE"] and wl.now.flags["C_CONTIGUOUS"]
+    st = L.ora_pd_migrate(C.byref(ctx.cfg), C.byref(ctx.table), wl.now.ctypes.data, pr.ctypes.data, int(x0), int(x1),
+                          moved.ctypes.data)
+    return {"status": int(st), "moved": int(moved[0])}
 
 
 def slo_map(n_prio: int, window: Dict[str, np.ndarray], bounds: Dict[str, np.ndarray], last_queue: np.ndarray,

@@ -878,3 +878,58 @@ uint32_t ora_slo_map(int32_t n_prio, const ora_slo_window *win, const ora_slo_bo
   free(by_ttft); free(by_tpot); free(C);
   return status;
 }
+
+/* ==========================================================================
+ * Hand-off from the P stage to the D stage in the disaggregated mode
+ * (Sec. 3.3.1 "Disaggregated Mode": prefill and decode run on separate
+ * instance pools, the Migrator makes the D-stage decisions over the queue of
+ * prefilled requests; the Overview has the Migrator coordinate the KV-cache
+ * transfers).  Together with the per-replica step and its commit this couples
+ * the two stages: a request is prefilled on a P instance (step, commit: it is
+ * RUNNING there with its first-token time = the end of its prefill batch), its
+ * KV cache is transferred, and it joins the queue of its partner D instance.
+ *
+ * reading: every P instance r has one partner D instance pair[r].
+ * reading: the transfer of a request takes x0 + x1 * prompt_len ns and starts
+ *   when its prefill batch ends; the request can be handed over once the D
+ *   instance's clock has reached that time.  It then becomes QUEUED on the D
+ *   instance (prefilled: its first-token time stands).
+ * reading: a D instance with nothing in flight and nothing in its queue would
+ *   never move its clock; it is woken at the earliest time a transfer to it
+ *   completes.
+ * Requests that finished at their first token (output_len <= 1) are DONE on
+ * the P instance and stay there.
+ * ========================================================================== */
+uint32_t ora_pd_migrate(const ora_config *c, const ora_table *t, int64_t *now, const int32_t *pair, int64_t x0,
+                        int64_t x1, int32_t *n_moved) {
+  const int32_t R = c->n_replicas;
+  uint32_t status = 0;
+  int32_t *rid = (int32_t *)t->replica_id;      /* the binding is rewritten here */
+  int64_t *wake = (int64_t *)malloc(sizeof(int64_t) * (size_t)R);
+  int32_t *busy = (int32_t *)calloc((size_t)R, sizeof(int32_t));
+  int32_t moved = 0;
+  for (int32_t r = 0; r < R; r++) wake[r] = ORA_INF;
+  for (int64_t i = 0; i < t->n; i++) {
+    const int32_t r = rid[i];
+    if (r < 0 || r >= R) { status |= BAD_REPLICA; continue; }
+    if (!row_valid(c, t, i, &status)) continue;
+    if (c->replicas[r].mode != MODE_PREFILL || t->state[i] != ST_RUNNING) continue;
+    const int32_t d = pair[r];
+    if (d < 0 || d >= R || c->replicas[d].mode != MODE_DECODE) { status |= BAD_REPLICA; continue; }
+    const int64_t ready = t->first_token[i] + x0 + x1 * (int64_t)t->prompt_len[i];
+    if (ready <= now[d]) { rid[i] = d; t->state[i] = ST_QUEUED; moved++; }
+    else if (ready < wake[d]) wake[d] = ready;
+  }
+  for (int64_t i = 0; i < t->n; i++) {
+    const int32_t r = rid[i];
+    if (r < 0 || r >= R || c->replicas[r].mode != MODE_DECODE) continue;
+    uint32_t ignore = 0;
+    if (!row_valid(c, t, i, &ignore)) continue;
+    if (t->state[i] == ST_RUNNING || (t->state[i] == ST_QUEUED && t->arrival[i] <= now[r])) busy[r] = 1;
+  }
+  for (int32_t d = 0; d < R; d++)
+    if (c->replicas[d].mode == MODE_DECODE && !busy[d] && wake[d] != ORA_INF && wake[d] > now[d]) now[d] = wake[d];
+  if (n_moved) *n_moved = moved;
+  free(wake); free(busy);
+  return status;
+}

@@ -425,3 +425,39 @@ def test_slo_mapping_quantiles_against_numpy():
                   "tpot_min_relaxed": -big}
         o = oracle.slo_map(1, win, bounds, np.array([0]), np.array([0]), np.array([0]))
         assert o["ttft_slo"][0] == np.sort(win["ttft"])[w // 2] and o["tpot_slo"][0] == np.sort(win["tpot"])[w // 2]
+
+
+# ---- hand-off between the stages of the disaggregated mode ----------------------------------------------
+def test_pd_handoff_hand_worked():
+    cls = [(200 * MS, 30 * MS, 0)]
+    rows = [dict(replica_id=0, prompt_len=1000, output_len=3, arrival_ns=0),
+            dict(replica_id=0, prompt_len=64, output_len=1, arrival_ns=0)]          # finishes at its first token
+    wl = make_wl(rows, cls, replicas=[(gen.PREFILL, 32768, 0), (gen.DECODE, 32768, 8)], now=[0, 0], maturity=[0, 0])
+    pair = np.array([1, -1])
+    o = oracle.step(wl, commit=True)
+    assert o["budget"][0] == PINS["nsafe_idle"] and list(o["admit"]) == [1, 1]
+    ft = 5_000_000 + 40_000 * 1064 + 2 * 1064 * 1064          # both prompts form one prefill batch of 1064 tokens
+    assert wl.table["first_token_ns"][0] == ft and list(wl.table["state"]) == [gen.RUNNING, gen.DONE]
+    # the single-request figures of the pin file: the batch is request A alone
+    wl = make_wl(rows[:1], cls, replicas=[(gen.PREFILL, 32768, 0), (gen.DECODE, 32768, 8)], now=[0, 0], maturity=[0, 0])
+    oracle.step(wl, commit=True)
+    assert wl.table["first_token_ns"][0] == PINS["pd_first_token"] and wl.now[0] == PINS["pd_first_token"]
+    r = oracle.pd_migrate(wl, pair, 1_000_000, 1000)
+    assert r == {"status": 0, "moved": 0} and wl.table["replica_id"][0] == 0 and wl.table["state"][0] == gen.RUNNING
+    assert wl.now[1] == PINS["pd_ready"] and wl.now[0] == PINS["pd_first_token"]
+    r = oracle.pd_migrate(wl, pair, 1_000_000, 1000)
+    assert r["moved"] == 1 and wl.table["replica_id"][0] == 1 and wl.table["state"][0] == gen.QUEUED
+    o = oracle.step(wl, commit=True)
+    assert o["budget"][1] == 22_000_000 and o["admit"][0] == 1 and o["adm_cost"][1] == 120_000
+    assert wl.now[1] == PINS["pd_d_iteration_end"] and wl.table["gen"][0] == 1 and wl.table["state"][0] == gen.RUNNING
+    assert wl.table["first_token_ns"][0] == PINS["pd_first_token"] and wl.table["last_token_ns"][0] == PINS["pd_d_iteration_end"]
+    # a busy D instance is not woken, a request whose transfer is still under way stays on the P instance
+    rows = [dict(replica_id=0, state=gen.RUNNING, prompt_len=1000, output_len=9, first_token_ns=100 * MS),
+            dict(replica_id=1, state=gen.RUNNING, prompt_len=10, gen=2, output_len=99, first_token_ns=0),
+            dict(replica_id=0, state=gen.RUNNING, prompt_len=0, output_len=9, first_token_ns=9 * MS)]
+    wl = make_wl(rows, cls, replicas=[(gen.PREFILL, 32768, 0), (gen.DECODE, 32768, 8)], now=[200 * MS, 10 * MS], maturity=[0, 0])
+    r = oracle.pd_migrate(wl, pair, 1_000_000, 1000)
+    assert r["moved"] == 1 and list(wl.table["replica_id"]) == [0, 1, 1] and list(wl.now) == [200 * MS, 10 * MS]
+    # a partner that is not a D instance is an error of the data: flagged, nothing moves
+    r = oracle.pd_migrate(wl, np.array([0, -1]), 0, 0)
+    assert r["status"] == 1 and r["moved"] == 0
