@@ -311,6 +311,40 @@ def run_gpu(args):
             disp["cpu_oracle_ms"] = 1e3 * (time.perf_counter() - t0) / k_d
             disp["cpu_oracle_calls"] = k_d
 
+    # ---- the disaggregated mode end to end: committed steps coupled by the hand-off (rank 0) ----------
+    pd = None
+    if rank == 0 and not args.no_pd:
+        pw = gen.pd_pairs(7, 128, 8192)
+        psched = hfx.Scheduler(pw.model, pw.classes, pw.replicas, pw.n_rows)
+        ptab = hfx.DeviceTable.from_numpy(pw.table)
+        pnow = torch.from_numpy(pw.now.copy()).cuda(); pmat = torch.from_numpy(pw.maturity.copy()).cuda()
+        ppair = torch.from_numpy(gen.pd_partner_table(128)).cuda()
+        pout = hfx.StepOut(pw.n_rows, pw.n_replicas, optional=False)
+        pmoved = torch.zeros(4, dtype=torch.int32, device="cuda")
+        rounds_w, rounds_t = 10, 40
+        moved_total = 0
+        evs = []
+        for k in range(rounds_w + rounds_t):
+            flush.fill_(5)
+            a = torch.cuda.Event(enable_timing=True); m = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            psched.step(ptab, pnow, pmat, pout, commit=True)
+            m.record(stream)
+            psched.pd_migrate(ptab, pnow, pmat, ppair, 2_000_000, 500, pmoved)
+            b.record(stream)
+            if k >= rounds_w:
+                evs.append((a, m, b))
+        torch.cuda.synchronize()
+        step_ms_pd = float(np.mean([a.elapsed_time(m) for a, m, b in evs]))
+        mig_ms = float(np.mean([m.elapsed_time(b) for a, m, b in evs]))
+        pt = ptab.to_numpy()
+        pd = {"workload": "128 P + 128 D instances, 1,048,576 requests, %d rounds of (committed step, hand-off)" % (rounds_w + rounds_t),
+              "step_ms": step_ms_pd, "handoff_ms": mig_ms, "rounds_per_sec": 1e3 / (step_ms_pd + mig_ms),
+              "handoff_gbs": 15 * pw.n_rows / (mig_ms * 1e-3) / 1e9,
+              "requests_on_d_instances": int(np.count_nonzero(pt["replica_id"] >= 128)),
+              "requests_finished": int(np.count_nonzero(pt["state"] == 2)), "status": psched.status()}
+        psched.close()
+
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only -----------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -359,7 +393,7 @@ def run_gpu(args):
                 "clocks": clk, "gpu_launches": launches, "device_status": status,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms_max},
-                "roofline": roof, "cpu_baseline": cpu, "sim": sim, "dispatch": disp}
+                "roofline": roof, "cpu_baseline": cpu, "sim": sim, "dispatch": disp, "pd": pd}
         print(json.dumps(line))
     sched.close()
     if world > 1:
@@ -379,6 +413,7 @@ def main():
     ap.add_argument("--no-sim", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-dispatch", action="store_true")
+    ap.add_argument("--no-pd", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

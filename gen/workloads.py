@@ -377,6 +377,31 @@ def random_traces(seed: int, traces: int, rows_lo: int, rows_hi: int, iters: int
                     sim_iters=iters)
 
 
+def pd_pairs(seed: int, pairs: int, rows_per: int, rate: float = 40.0, token_cap: int = 8192, batch_cap: int = 64,
+             out_hi: int = 24, classes=None) -> Workload:
+    """Disaggregated deployment for the coupled P/D tests: `pairs` P instances (replicas 0 .. pairs-1) and
+    their partner D instances (replicas pairs .. 2 pairs-1).  Every request starts QUEUED on a P instance
+    (Poisson arrivals from time 0, short outputs so that requests finish within a few dozen rounds); all
+    clocks start at 0.  The partner table is `np.arange(pairs, 2 pairs)` for the P instances, -1 for the rest."""
+    rng = np.random.default_rng(seed)
+    classes = classes or CLASSES_PD
+    n = pairs * rows_per
+    tab = _empty_table(n)
+    tab["replica_id"][:] = rng.integers(0, pairs, n).astype(np.int32)
+    tab["class_id"][:] = rng.integers(0, len(classes), n).astype(np.uint8)
+    tab["prompt_len"][:] = _lognormal_int(rng, 5.5, 1.0, 1, token_cap // 2, n)
+    tab["output_len"][:] = rng.integers(1, out_hi + 1, n).astype(np.int32)
+    tab["arrival_ns"][:] = np.rint(np.sort(rng.exponential(1.0 / (rate * pairs), n).cumsum()) * SEC).astype(np.int64)
+    tab["req_id"][:] = rng.permutation(n).astype(np.int32)
+    reps = np.concatenate([_replicas(pairs, PREFILL, token_cap), _replicas(pairs, DECODE, token_cap, batch_cap)])
+    return Workload(f"pd{seed}", DEFAULT_MODEL, classes, reps, tab, np.zeros(2 * pairs, np.int64),
+                    np.zeros(2 * pairs, np.int64))
+
+
+def pd_partner_table(pairs: int) -> np.ndarray:
+    return np.concatenate([np.arange(pairs, 2 * pairs), -np.ones(pairs)]).astype(np.int32)
+
+
 def by_name(name: str, **kw) -> Workload:
     return {"config1": config1, "config2": config2, "config3": config3, "config4": config4,
             "config5": config5}[name](**kw)

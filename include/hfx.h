@@ -275,6 +275,28 @@ typedef struct hfx_dispatch_out {
 int hfx_dispatch_step(hfx_sched *s, const hfx_table *table, int64_t now_ns,
                       const int64_t *maturity_ns, const hfx_dispatch_out *out);
 
+/* Hand-off from the P stage to the D stage of the disaggregated mode
+ * (Sec. 3.3.1 "Disaggregated Mode": the Dispatcher serves the P instances, the
+ * Migrator the D instances over the queue of prefilled requests).  With
+ * hfx_sched_step + HFX_COMMIT on a scheduler that has HFX_PREFILL and
+ * HFX_DECODE replicas this couples the two stages: a committed P-stage step
+ * leaves an admitted request RUNNING on its P instance with first_token_ns =
+ * the end of its prefill batch; this call moves it to the partner D instance
+ * pair[r] (device, [n_replicas]; read for PREFILL replicas only) once its KV
+ * transfer, xfer_c0_ns + xfer_c1_ns * prompt_len after the first token, has
+ * ended by the partner's clock: replica_id := pair[r], state := HFX_QUEUED,
+ * first_token_ns stands, so the next step of the D instance sees it in its
+ * queue of prefilled requests.  A D instance with nothing in flight and
+ * nothing arrived in its queue is woken: its now_ns becomes the earliest end
+ * of a transfer to it.  `replica_id` must be table->replica_id (the column is
+ * written, which the const in hfx_table does not allow); state and now_ns are
+ * written too.  n_moved (device, [1]) may be NULL.  A partner that is not a
+ * DECODE replica sets HFX_ST_BAD_REPLICA and the row stays.
+ * Errors: HFX_E_ARG (NULL, negative transfer coefficients, replica_id not the
+ * table's column), HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_CUDA. */
+int hfx_pd_migrate(hfx_sched *s, const hfx_table *table, int32_t *replica_id, const hfx_replica_state *state,
+                   const int32_t *pair, int64_t xfer_c0_ns, int64_t xfer_c1_ns, int32_t *n_moved);
+
 /* Priority-based SLO mapping (Sec. 3.3.2 "Priority-Based SLO Mapping", its five
  * steps): requests that carry only a priority p in [0, n_prio), 0 highest, get
  * their TTFT and TPOT targets from recent history.  `win` is the sliding window
@@ -379,9 +401,9 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
  * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
  * 6 oversize path, 7 simulator, 8 scaler tick, 9 fused front end, 10 the kernels of
- * hfx_dispatch_step together, 11 those of hfx_slo_map; hfx_kernel_name gives the
- * name of a slot (NULL past the end). */
-#define HFX_N_KERNELS 12
+ * hfx_dispatch_step together, 11 those of hfx_slo_map, 12 those of hfx_pd_migrate;
+ * hfx_kernel_name gives the name of a slot (NULL past the end). */
+#define HFX_N_KERNELS 13
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
   int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */

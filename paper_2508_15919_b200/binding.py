@@ -21,9 +21,9 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map"]
+                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map", "hfx_pd_migrate"]
 NOALLOC_MAX_REPLICAS = 4096
-N_KERNELS = 12
+N_KERNELS = 13
 
 
 class HfxError(RuntimeError):
@@ -82,7 +82,7 @@ SIM_OUT_FIELDS = [("iters_executed", torch.int32), ("finished", torch.int32), ("
 
 
 class _Profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 12), ("launches", C.c_int64 * 12)]
+    _fields_ = [("ms", C.c_double * 13), ("launches", C.c_int64 * 13)]
 
 
 class _ScaleParams(C.Structure):
@@ -142,6 +142,9 @@ def load_library():
     L.hfx_sched_step.argtypes = [C.c_void_p, C.POINTER(_Table), C.POINTER(_ReplicaState), C.POINTER(_StepOut), C.c_uint32]
     L.hfx_dispatch_step.restype = C.c_int
     L.hfx_dispatch_step.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_DispatchOut)]
+    L.hfx_pd_migrate.restype = C.c_int
+    L.hfx_pd_migrate.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_void_p, C.POINTER(_ReplicaState), C.c_void_p, C.c_int64,
+                                 C.c_int64, C.c_void_p]
     L.hfx_slo_map.restype = C.c_int
     L.hfx_slo_map.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_SloWindow), C.POINTER(_SloBounds), C.c_void_p, C.c_void_p,
                               C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
@@ -338,6 +341,17 @@ class Scheduler:
         rc = self._L.hfx_dispatch_step(self._h, C.byref(ts), int(now_ns), _ptr(maturity), C.byref(os_))
         if rc != 0:
             raise HfxError(rc, "hfx_dispatch_step")
+
+    def pd_migrate(self, table: DeviceTable, now: torch.Tensor, maturity: torch.Tensor, pair: torch.Tensor,
+                   xfer_c0_ns: int, xfer_c1_ns: int, n_moved: Optional[torch.Tensor] = None):
+        """hfx_pd_migrate: hand prefilled requests over from the P instances to their partner D instances
+        (pair: int32 [n_replicas] on the device); table.replica_id, table.state and now are updated in place."""
+        ts = table.c_struct()
+        st = _ReplicaState(_ptr(now), _ptr(maturity))
+        rc = self._L.hfx_pd_migrate(self._h, C.byref(ts), _ptr(table.cols["replica_id"]), C.byref(st), _ptr(pair),
+                                    int(xfer_c0_ns), int(xfer_c1_ns), _ptr(n_moved))
+        if rc != 0:
+            raise HfxError(rc, "hfx_pd_migrate")
 
     def slo_map(self, n_prio: int, window: Dict[str, torch.Tensor], bounds: Dict[str, torch.Tensor],
                 last_queue: torch.Tensor, pending: torch.Tensor, new_prio: torch.Tensor, ttft_out: torch.Tensor,

@@ -119,6 +119,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   ok = ok && cudaMalloc(&s->d_barrier, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_front_bar, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_slo, hfx_slomap_workspace_bytes()) == cudaSuccess;
+  ok = ok && cudaMalloc(&s->d_pd, hfx_pd_workspace_bytes(n_replicas)) == cudaSuccess;
   s->front_enabled = 1; s->front_arrivals = 0; s->front_smem_cached = 0; s->front_capacity = 0;
   ok = ok && cudaMalloc(&h->d_trace_off, sizeof(int32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&h->d_work_counter, 256) == cudaSuccess;
@@ -161,7 +162,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   cudaFree(s->d_cfg); cudaFree(s->d_mode); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
   cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_mode);
-  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier); cudaFree(s->d_front_bar); cudaFree(s->d_slo);
+  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier); cudaFree(s->d_front_bar); cudaFree(s->d_slo); cudaFree(s->d_pd);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();
   if (s->brackets) {
@@ -223,6 +224,22 @@ extern "C" int hfx_dispatch_step(hfx_sched *s, const hfx_table *t, int64_t now_n
     if (h->h_cfg[r].token_cap > cap_max) cap_max = h->h_cfg[r].token_cap;
   }
   return hfx_launch_dispatch(s, t, now_ns, maturity_ns, o, cap_max);
+}
+
+extern "C" int hfx_pd_migrate(hfx_sched *s, const hfx_table *t, int32_t *replica_id, const hfx_replica_state *st,
+                              const int32_t *pair, int64_t xfer_c0_ns, int64_t xfer_c1_ns, int32_t *n_moved) {
+  if (!s || !t || !st || !st->now_ns || !pair) return HFX_E_ARG;
+  if (t->n_rows < 0 || xfer_c0_ns < 0 || xfer_c1_ns < 0 || xfer_c0_ns > (INT64_C(1) << 40) || xfer_c1_ns > (INT64_C(1) << 30)) return HFX_E_ARG;
+  if (t->n_rows > s->max_rows) return HFX_E_CAPACITY;
+  if (t->n_rows > 0) {
+    const void *need[] = {t->replica_id, t->class_id, t->state, t->prompt_len, t->gen, t->arrival_ns, t->first_token_ns};
+    for (const void *p : need) if (!p) return HFX_E_ARG;
+    if (replica_id != t->replica_id) return HFX_E_ARG;
+  }
+  const void *all[] = {t->replica_id, t->class_id, t->state, t->prompt_len, t->gen, t->arrival_ns, t->first_token_ns, st->now_ns,
+                       pair, n_moved};
+  for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
+  return hfx_launch_pd_migrate(s, t, replica_id, st->now_ns, pair, xfer_c0_ns, xfer_c1_ns, n_moved);
 }
 
 extern "C" int hfx_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const hfx_slo_bounds *b,
@@ -323,6 +340,6 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 
 extern "C" const char *hfx_kernel_name(int slot) {
   static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
-                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch", "k_slo_map"};
-  return (slot >= 0 && slot < 12) ? names[slot] : nullptr;
+                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch", "k_slo_map", "k_pd_migrate"};
+  return (slot >= 0 && slot < 13) ? names[slot] : nullptr;
 }

@@ -59,7 +59,7 @@ static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
 #include <vector>
 
-enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT, KSLOT_DISPATCH, KSLOT_SLOMAP };
+enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT, KSLOT_DISPATCH, KSLOT_SLOMAP, KSLOT_PD };
 
 // tiling of the streaming passes: about this many tiles (2 per SM), each at most this many rows
 #define HFX_TILE_BLOCKS 296
@@ -107,6 +107,7 @@ struct hfx_sched {
   int front_capacity;                  // blocks of the fused kernel that can be resident at once
   void *dispatch_ws;                   // workspace of hfx_dispatch_step, allocated by its first call
   void *d_slo;                         // per-priority table of hfx_slo_map
+  void *d_pd;                          // moved counter, wake-up times and busy flags of hfx_pd_migrate
 };
 
 // ---- latency predictor -------------------------------------------------------------------
@@ -468,5 +469,8 @@ void hfx_dispatch_release(hfx_sched *s);
 int hfx_launch_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const hfx_slo_bounds *b, int64_t *last_queue,
                        const int32_t *pending, const int32_t *new_prio, int64_t n_new, int64_t *ttft_out, int64_t *tpot_out);
 size_t hfx_slomap_workspace_bytes();
+int hfx_launch_pd_migrate(hfx_sched *s, const hfx_table *t, int32_t *replica_id, int64_t *now, const int32_t *pair, int64_t x0,
+                          int64_t x1, int32_t *n_moved);
+size_t hfx_pd_workspace_bytes(int n_replicas);
 int hfx_launch_sim(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
                    const hfx_sim_out *o);

@@ -520,3 +520,71 @@ def test_slo_mapping_random(seed):
     pending = rng.integers(0, 2, N) * rng.integers(0, 2, N)
     new = rng.integers(0, N, 10_000 + seed)
     _slo_parity(N, win, bounds, last, pending, new)
+
+
+# ---- the two stages of the disaggregated mode coupled by the hand-off --------------------------------------
+def _pd_coupled_parity(wl, pair, rounds, x0=2 * MS, x1=500):
+    """`rounds` times (committed step, hand-off) on both sides; the table, the clocks and the step's
+    outputs must agree after every call."""
+    import paper_2508_15919_b200 as hfx
+    cpu = wl.copy()
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    now = torch.from_numpy(wl.now.copy()).cuda(); mat = torch.from_numpy(wl.maturity.copy()).cuda()
+    prt = torch.from_numpy(pair).cuda()
+    out = hfx.StepOut(wl.n_rows, wl.n_replicas, optional=False)
+    moved = torch.zeros(4, dtype=torch.int32, device="cuda")
+    total_moved = 0
+    for k in range(rounds):
+        sched.step(tab, now, mat, out, commit=True)
+        c = oracle.step(cpu, commit=True)
+        g = out.to_numpy()
+        for ko, kg in (("order", "order"), ("admit", "admit"), ("budget", "budget"), ("adm_count", "adm_count"), ("slack", "slack_ns")):
+            assert np.array_equal(g[kg], c[ko]), (k, kg)
+        sched.pd_migrate(tab, now, mat, prt, x0, x1, moved)
+        st = sched.status()
+        r = oracle.pd_migrate(cpu, pair, x0, x1)
+        assert st == (c["status"] | r["status"]), (k, st, c["status"], r["status"])
+        assert int(moved[0].item()) == r["moved"], (k, int(moved[0].item()), r["moved"])
+        total_moved += r["moved"]
+        tg = tab.to_numpy()
+        for col in ("replica_id", "state", "gen", "first_token_ns", "last_token_ns", "finish_ns"):
+            assert np.array_equal(tg[col], cpu.table[col]), f"round {k}: column {col} differs at {np.nonzero(tg[col] != cpu.table[col])[0][:8]}"
+        assert np.array_equal(now.cpu().numpy(), cpu.now), f"round {k}: now"
+        assert np.array_equal(mat.cpu().numpy(), cpu.maturity), f"round {k}: maturity"
+    sched.close()
+    return cpu, total_moved
+
+
+@pytest.mark.parametrize("seed,pairs,rows_per", [(0, 1, 40), (1, 3, 200), (2, 16, 1500)])
+def test_pd_coupled_stages(seed, pairs, rows_per):
+    wl = gen.pd_pairs(seed, pairs, rows_per)
+    cpu, moved = _pd_coupled_parity(wl, gen.pd_partner_table(pairs), rounds=(60, 40, 25)[seed])
+    t = cpu.table
+    # requests went through both stages: some finished on a D instance, every first token precedes its last one
+    assert moved > 0 and np.count_nonzero((t["state"] == 2) & (t["replica_id"] >= pairs)) > 0
+    done = t["state"] == 2
+    assert np.all(t["first_token_ns"][done] <= t["finish_ns"][done]) and np.all(t["arrival_ns"][done] <= t["first_token_ns"][done])
+
+
+def test_pd_handoff_edges_and_errors():
+    import paper_2508_15919_b200 as hfx
+    # bad partners, rows with bad data, an empty table; argument errors
+    wl = gen.pd_pairs(5, 2, 300)
+    wl.table["class_id"][::41] = 99
+    pair = gen.pd_partner_table(2); pair[1] = 0          # instance 1's partner is a P instance: flagged, its rows stay
+    _pd_coupled_parity(wl, pair, rounds=12)
+    wl0 = gen.pd_pairs(6, 1, 8)
+    sched = make_sched(wl0)
+    tab = hfx.DeviceTable.from_numpy(wl0.table)
+    now = torch.from_numpy(wl0.now.copy()).cuda(); mat = torch.from_numpy(wl0.maturity.copy()).cuda()
+    prt = torch.from_numpy(gen.pd_partner_table(1)).cuda()
+    with pytest.raises(hfx.HfxError) as e:
+        sched.pd_migrate(tab, now, mat, prt, -1, 0)
+    assert e.value.code == -1
+    with pytest.raises(hfx.HfxError) as e:
+        sched.pd_migrate(tab, now, mat, prt[1:], 0, 0)
+    assert e.value.code == -2
+    sched.pd_migrate(tab, now, mat, prt, 0, 0)          # nothing is RUNNING on a P instance yet: a no-op
+    assert sched.status() == 0 and np.array_equal(tab.to_numpy()["replica_id"], wl0.table["replica_id"])
+    sched.close()
