@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
                                                      uint32_t *__restrict__ status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int cap = a.cap_rows;
-  int64_t *s_arr = reinterpret_cast<int64_t *>(smem_raw);              // arrival; later the TTFT, then the TPOT samples
+  int64_t *s_arr = reinterpret_cast<int64_t *>(smem_raw);              // arrival, the slack base once arrived; later the TTFT, then the TPOT samples
   int32_t *s_prompt = reinterpret_cast<int32_t *>(s_arr + cap);
   int32_t *s_fin = s_prompt + cap;                                     // iteration at which a running row emits its last token
   uint16_t *s_q = reinterpret_cast<uint16_t *>(s_fin + cap);           // visible queue (row indices, unordered)
@@ -165,6 +165,10 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           } else {
             const int slot = atomicAdd(&S.nq, 1);
             s_q[slot] = (uint16_t)i;
+            // from here on the row's arrival slot holds its slack base, ttft_slo + arrival - E_p(prompt_len):
+            // the slack at any later decision is the base minus the earliest start
+            const int64_t ttft = S.ttft[cls];
+            s_arr[i] = ttft > 0 ? ttft + s_arr[i] - dev_Ep(p, s_prompt[i]) : BASE_UNBOUNDED;
           }
         }
         if (local) atomicAdd(&S.arrived, local);
@@ -197,9 +201,9 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           for (int s = tid; s < nq; s += SIM_THREADS) {
             const int i = s_q[s];
             if ((int64_t)s_prompt[i] > budget) continue;
-            // slack of a queued request: ttft_slo - (start - arrival) - E_p(prompt_len)
-            const int64_t ttft = S.ttft[s_cls[i]];
-            const int64_t sl = ttft > 0 ? dev_clamp_slack(ttft + s_arr[i] - dev_Ep(p, s_prompt[i]) - start) : HFX_SLACK_MAX;
+            // slack of a queued request: ttft_slo - (start - arrival) - E_p(prompt_len) = base - start
+            const int64_t base = s_arr[i];
+            const int64_t sl = base != BASE_UNBOUNDED ? dev_clamp_slack(base - start) : HFX_SLACK_MAX;
             const uint64_t k = ((uint64_t)s_prio[i] << 40) | (uint64_t)(sl + (INT64_C(1) << 39));
             if (k < bk) { bk = k; bslot = s; bid = ~0u; }
             else if (k == bk) {      // equal keys are rare: only then fetch the request ids that break the tie
@@ -344,7 +348,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       }
       a.state[g] = (uint8_t)st;
       a.gen[g] = gen;
-      const int64_t arr = s_arr[i];
+      const int64_t arr = a.arrival[g];      // (the shared-memory slot holds the slack base of rows that arrived)
       const uint8_t cls = s_cls[i];
       int64_t ttft = -1;
       if (cls != ROW_INVALID) {
