@@ -338,11 +338,14 @@ def run_gpu(args):
         step_ms_pd = float(np.mean([a.elapsed_time(m) for a, m, b in evs]))
         mig_ms = float(np.mean([m.elapsed_time(b) for a, m, b in evs]))
         pt = ptab.to_numpy()
+        att = torch.zeros((len(pw.classes) + 1, 6), dtype=torch.int64, device="cuda")
+        psched.attainment(ptab, att)
+        att_tot = att.cpu().numpy()[-1]
         pd = {"workload": "128 P + 128 D instances, 1,048,576 requests, %d rounds of (committed step, hand-off)" % (rounds_w + rounds_t),
               "step_ms": step_ms_pd, "handoff_ms": mig_ms, "rounds_per_sec": 1e3 / (step_ms_pd + mig_ms),
               "handoff_gbs": 15 * pw.n_rows / (mig_ms * 1e-3) / 1e9,
               "requests_on_d_instances": int(np.count_nonzero(pt["replica_id"] >= 128)),
-              "requests_finished": int(np.count_nonzero(pt["state"] == 2)), "status": psched.status()}
+              "requests_finished": int(att_tot[1]), "requests_attained": int(att_tot[2]), "status": psched.status()}
         psched.close()
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only -----------------------------

@@ -297,6 +297,19 @@ int hfx_dispatch_step(hfx_sched *s, const hfx_table *table, int64_t now_ns,
 int hfx_pd_migrate(hfx_sched *s, const hfx_table *table, int32_t *replica_id, const hfx_replica_state *state,
                    const int32_t *pair, int64_t xfer_c0_ns, int64_t xfer_c1_ns, int32_t *n_moved);
 
+/* SLO attainment over the table (Problem Definition, Eq. 2: the fraction of
+ * requests that meet both their TTFT and their TPOT target; E2E = completion -
+ * arrival of the same section), per SLO class and in total.  `out` is a device
+ * array of (n_classes + 1) x 6 int64, row c = class c, the last row the totals:
+ * requests, DONE, attained, REJECTED, sum of TTFT (first_token - arrival over
+ * RUNNING and DONE requests), sum of E2E (finish - arrival over DONE ones).
+ * TPOT = floor((last_token - first_token) / (output_len - 1)), 0 for output_len
+ * <= 1; a target <= 0 is always met; a request that is not DONE is a miss, as
+ * Eq. 2 sums over all requests.  Rows with a class or a length outside the
+ * domain are left out and flagged.  Attainment = attained / requests.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_CUDA. */
+int hfx_attainment(hfx_sched *s, const hfx_table *table, int64_t *out);
+
 /* Priority-based SLO mapping (Sec. 3.3.2 "Priority-Based SLO Mapping", its five
  * steps): requests that carry only a priority p in [0, n_prio), 0 highest, get
  * their TTFT and TPOT targets from recent history.  `win` is the sliding window
@@ -401,9 +414,9 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
  * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
  * 6 oversize path, 7 simulator, 8 scaler tick, 9 fused front end, 10 the kernels of
- * hfx_dispatch_step together, 11 those of hfx_slo_map, 12 those of hfx_pd_migrate;
- * hfx_kernel_name gives the name of a slot (NULL past the end). */
-#define HFX_N_KERNELS 13
+ * hfx_dispatch_step together, 11 those of hfx_slo_map, 12 those of hfx_pd_migrate, 13
+ * hfx_attainment; hfx_kernel_name gives the name of a slot (NULL past the end). */
+#define HFX_N_KERNELS 14
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
   int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */

@@ -147,6 +147,8 @@ def lib():
         L.ora_pd_migrate.restype = C.c_uint32
         L.ora_pd_migrate.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
                                      C.c_void_p]
+        L.ora_attainment.restype = C.c_uint32
+        L.ora_attainment.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p]
         L.ora_scale.restype = C.c_uint32
         L.ora_scale.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_ScaleParams),
                                 C.POINTER(_ScaleOut)]
@@ -266,6 +268,16 @@ def pd_migrate(wl, pair: np.ndarray, x0: int, x1: int) -> Dict[str, int]:
     st = L.ora_pd_migrate(C.byref(ctx.cfg), C.byref(ctx.table), wl.now.ctypes.data, pr.ctypes.data, int(x0), int(x1),
                           moved.ctypes.data)
     return {"status": int(st), "moved": int(moved[0])}
+
+
+def attainment(wl) -> Dict[str, np.ndarray]:
+    """Eq. 2 over wl.table: int64 [n_classes + 1, 6] = requests, DONE, attained, REJECTED, sum of TTFT, sum of
+    E2E per class, totals in the last row."""
+    L = lib()
+    ctx = _Ctx(wl)
+    out = np.zeros((len(wl.classes) + 1, 6), np.int64)
+    st = L.ora_attainment(C.byref(ctx.cfg), C.byref(ctx.table), out.ctypes.data)
+    return {"counts": out, "status": int(st)}
 
 
 def slo_map(n_prio: int, window: Dict[str, np.ndarray], bounds: Dict[str, np.ndarray], last_queue: np.ndarray,

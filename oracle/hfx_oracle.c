@@ -933,3 +933,39 @@ uint32_t ora_pd_migrate(const ora_config *c, const ora_table *t, int64_t *now, c
   free(wake); free(busy);
   return status;
 }
+
+/* ==========================================================================
+ * SLO attainment over a request table (Problem Definition, Eq. 2: the
+ * fraction of requests that meet both their TTFT and their TPOT target), per
+ * SLO class and in total, with the sums behind the mean TTFT and the mean
+ * end-to-end time E2E = T_complete - T_arrival of the same section.
+ *   TTFT = first_token - arrival (requests RUNNING or DONE),
+ *   TPOT = floor((last_token - first_token) / (output_len - 1)), 0 for
+ *          output_len <= 1 (DONE requests),
+ * a target <= 0 is unbounded and always met; requests that are not DONE count
+ * as misses (Eq. 2 sums over all M requests).
+ * out[(c)*6 + k], c = class (row n_classes = total), k = 0 requests, 1 DONE,
+ * 2 attained, 3 REJECTED, 4 sum of TTFT, 5 sum of E2E over DONE requests.
+ * ========================================================================== */
+uint32_t ora_attainment(const ora_config *c, const ora_table *t, int64_t *out) {
+  uint32_t status = 0;
+  const int32_t K = c->n_classes;
+  for (int32_t k = 0; k < (K + 1) * 6; k++) out[k] = 0;
+  for (int64_t i = 0; i < t->n; i++) {
+    if (!row_valid(c, t, i, &status)) continue;
+    const int32_t cl = t->class_id[i];
+    const ora_class *k = &c->classes[cl];
+    int64_t v[6] = {1, 0, 0, 0, 0, 0};
+    if (t->state[i] == ST_REJECTED) v[3] = 1;
+    if (t->state[i] == ST_RUNNING || t->state[i] == ST_DONE) v[4] = t->first_token[i] - t->arrival[i];
+    if (t->state[i] == ST_DONE) {
+      const int64_t ttft = t->first_token[i] - t->arrival[i];
+      const int64_t tpot = t->output_len[i] > 1 ? (t->last_token[i] - t->first_token[i]) / (t->output_len[i] - 1) : 0;
+      v[1] = 1;
+      v[5] = t->finish[i] - t->arrival[i];
+      if ((k->ttft <= 0 || ttft <= k->ttft) && (k->tpot <= 0 || tpot <= k->tpot)) v[2] = 1;
+    }
+    for (int q = 0; q < 6; q++) { out[cl * 6 + q] += v[q]; out[K * 6 + q] += v[q]; }
+  }
+  return status;
+}

@@ -21,9 +21,9 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map", "hfx_pd_migrate"]
+                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map", "hfx_pd_migrate", "hfx_attainment"]
 NOALLOC_MAX_REPLICAS = 4096
-N_KERNELS = 13
+N_KERNELS = 14
 
 
 class HfxError(RuntimeError):
@@ -82,7 +82,7 @@ SIM_OUT_FIELDS = [("iters_executed", torch.int32), ("finished", torch.int32), ("
 
 
 class _Profile(C.Structure):
-    _fields_ = [("ms", C.c_double * 13), ("launches", C.c_int64 * 13)]
+    _fields_ = [("ms", C.c_double * 14), ("launches", C.c_int64 * 14)]
 
 
 class _ScaleParams(C.Structure):
@@ -145,6 +145,8 @@ def load_library():
     L.hfx_pd_migrate.restype = C.c_int
     L.hfx_pd_migrate.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_void_p, C.POINTER(_ReplicaState), C.c_void_p, C.c_int64,
                                  C.c_int64, C.c_void_p]
+    L.hfx_attainment.restype = C.c_int
+    L.hfx_attainment.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_void_p]
     L.hfx_slo_map.restype = C.c_int
     L.hfx_slo_map.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_SloWindow), C.POINTER(_SloBounds), C.c_void_p, C.c_void_p,
                               C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
@@ -352,6 +354,14 @@ class Scheduler:
                                     int(xfer_c0_ns), int(xfer_c1_ns), _ptr(n_moved))
         if rc != 0:
             raise HfxError(rc, "hfx_pd_migrate")
+
+    def attainment(self, table: DeviceTable, out: torch.Tensor):
+        """hfx_attainment: out int64 [n_classes + 1, 6] on the device (requests, DONE, attained, REJECTED,
+        sum of TTFT, sum of E2E per class; totals in the last row)."""
+        ts = table.c_struct()
+        rc = self._L.hfx_attainment(self._h, C.byref(ts), _ptr(out))
+        if rc != 0:
+            raise HfxError(rc, "hfx_attainment")
 
     def slo_map(self, n_prio: int, window: Dict[str, torch.Tensor], bounds: Dict[str, torch.Tensor],
                 last_queue: torch.Tensor, pending: torch.Tensor, new_prio: torch.Tensor, ttft_out: torch.Tensor,

@@ -242,6 +242,20 @@ extern "C" int hfx_pd_migrate(hfx_sched *s, const hfx_table *t, int32_t *replica
   return hfx_launch_pd_migrate(s, t, replica_id, st->now_ns, pair, xfer_c0_ns, xfer_c1_ns, n_moved);
 }
 
+extern "C" int hfx_attainment(hfx_sched *s, const hfx_table *t, int64_t *out) {
+  if (!s || !t || !out || t->n_rows < 0) return HFX_E_ARG;
+  if (t->n_rows > s->max_rows) return HFX_E_CAPACITY;
+  if (t->n_rows > 0) {
+    const void *need[] = {t->class_id, t->state, t->prompt_len, t->output_len, t->gen, t->arrival_ns, t->first_token_ns,
+                          t->last_token_ns, t->finish_ns};
+    for (const void *p : need) if (!p) return HFX_E_ARG;
+  }
+  const void *all[] = {t->class_id, t->state, t->prompt_len, t->output_len, t->gen, t->arrival_ns, t->first_token_ns,
+                       t->last_token_ns, t->finish_ns, out};
+  for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
+  return hfx_launch_attainment(s, t, out);
+}
+
 extern "C" int hfx_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const hfx_slo_bounds *b,
                            int64_t *last_queue_ns, const int32_t *pending, const int32_t *new_prio, int64_t n_new,
                            int64_t *ttft_slo_ns, int64_t *tpot_slo_ns) {
@@ -340,6 +354,6 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 
 extern "C" const char *hfx_kernel_name(int slot) {
   static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
-                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch", "k_slo_map", "k_pd_migrate"};
-  return (slot >= 0 && slot < 13) ? names[slot] : nullptr;
+                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch", "k_slo_map", "k_pd_migrate", "k_attainment"};
+  return (slot >= 0 && slot < 14) ? names[slot] : nullptr;
 }

@@ -59,7 +59,7 @@ static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
 #include <vector>
 
-enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT, KSLOT_DISPATCH, KSLOT_SLOMAP, KSLOT_PD };
+enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT, KSLOT_DISPATCH, KSLOT_SLOMAP, KSLOT_PD, KSLOT_METRICS };
 
 // tiling of the streaming passes: about this many tiles (2 per SM), each at most this many rows
 #define HFX_TILE_BLOCKS 296
@@ -472,5 +472,6 @@ size_t hfx_slomap_workspace_bytes();
 int hfx_launch_pd_migrate(hfx_sched *s, const hfx_table *t, int32_t *replica_id, int64_t *now, const int32_t *pair, int64_t x0,
                           int64_t x1, int32_t *n_moved);
 size_t hfx_pd_workspace_bytes(int n_replicas);
+int hfx_launch_attainment(hfx_sched *s, const hfx_table *t, int64_t *out);
 int hfx_launch_sim(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
                    const hfx_sim_out *o);

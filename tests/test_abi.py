@@ -34,7 +34,7 @@ def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(b._ReplicaCfg) == 12 and ctypes.sizeof(b._Options) == 16
     assert ctypes.sizeof(b._Table) == 8 + 12 * 8 and ctypes.sizeof(b._ReplicaState) == 16
     assert ctypes.sizeof(b._StepOut) == 15 * 8 and ctypes.sizeof(b._SimOut) == 9 * 8
-    assert ctypes.sizeof(b._Profile) == 208 and ctypes.sizeof(b._SloWindow) == 40 and ctypes.sizeof(b._SloBounds) == 48 and ctypes.sizeof(b._DispatchOut) == 13 * 8 and ctypes.sizeof(b._ScaleParams) == 40
+    assert ctypes.sizeof(b._Profile) == 224 and ctypes.sizeof(b._SloWindow) == 40 and ctypes.sizeof(b._SloBounds) == 48 and ctypes.sizeof(b._DispatchOut) == 13 * 8 and ctypes.sizeof(b._ScaleParams) == 40
     # field order of the header's structs
     src = open(os.path.join(ROOT, "include", "hfx.h")).read()
     for struct, cls in (("hfx_table", b._Table), ("hfx_step_out", b._StepOut), ("hfx_sim_out", b._SimOut),
@@ -49,7 +49,7 @@ def test_strerror_and_argument_checks_without_a_device():
     lib = hfx.load_library()
     assert lib.hfx_strerror(0) == b"ok" and b"aligned" in lib.hfx_strerror(-2)
     assert lib.hfx_strerror(-99) == b"unknown error"
-    assert lib.hfx_kernel_name(3) == b"k_regroup" and lib.hfx_kernel_name(9) == b"k_front" and lib.hfx_kernel_name(10) == b"k_dispatch" and lib.hfx_kernel_name(11) == b"k_slo_map" and lib.hfx_kernel_name(12) == b"k_pd_migrate" and lib.hfx_kernel_name(13) is None
+    assert lib.hfx_kernel_name(3) == b"k_regroup" and lib.hfx_kernel_name(9) == b"k_front" and lib.hfx_kernel_name(10) == b"k_dispatch" and lib.hfx_kernel_name(11) == b"k_slo_map" and lib.hfx_kernel_name(12) == b"k_pd_migrate" and lib.hfx_kernel_name(13) == b"k_attainment" and lib.hfx_kernel_name(14) is None
     import torch
     if not torch.cuda.is_available():
         # no device: the product path fails loudly, it never falls back to the CPU

@@ -461,3 +461,35 @@ def test_pd_handoff_hand_worked():
     # a partner that is not a D instance is an error of the data: flagged, nothing moves
     r = oracle.pd_migrate(wl, np.array([0, -1]), 0, 0)
     assert r["status"] == 1 and r["moved"] == 0
+
+
+# ---- SLO attainment (Eq. 2) -------------------------------------------------------------------------------
+def _attainment_hand_case():
+    cls = [(200 * MS, 30 * MS, 0), (1000 * MS, 0, 1)]
+    rows = [dict(state=gen.DONE, class_id=0, prompt_len=1000, output_len=101, gen=100, arrival_ns=0,
+                 first_token_ns=PINS["sim1_ttft"], last_token_ns=PINS["sim1_finish"], finish_ns=PINS["sim1_finish"]),
+            dict(state=gen.DONE, class_id=0, output_len=11, gen=10, arrival_ns=100 * MS, first_token_ns=350 * MS,
+                 last_token_ns=850 * MS, finish_ns=850 * MS),
+            dict(state=gen.RUNNING, class_id=0, output_len=50, gen=3, arrival_ns=5 * MS, first_token_ns=15 * MS, last_token_ns=99 * MS),
+            dict(state=gen.REJECTED, class_id=1, prompt_len=100000, arrival_ns=0),
+            dict(state=gen.DONE, class_id=1, output_len=1, arrival_ns=MS, first_token_ns=1000 * MS, last_token_ns=1000 * MS,
+                 finish_ns=1000 * MS),
+            dict(state=gen.QUEUED, class_id=1, arrival_ns=7 * MS)]
+    return make_wl(rows, cls, replicas=[(gen.COLOCATED, 8192, 0)])
+
+
+def test_attainment_hand_worked():
+    o = oracle.attainment(_attainment_hand_case())
+    c = o["counts"]
+    assert o["status"] == 0
+    assert list(c[0]) == [3, 2, 1, 0, PINS["att_A_ttft_sum"], PINS["att_A_e2e_sum"]]
+    assert list(c[1]) == [3, 1, 1, 1, PINS["att_B_ttft_sum"], 999 * MS]
+    assert list(c[2]) == [6, 3, 2, 1, PINS["att_A_ttft_sum"] + PINS["att_B_ttft_sum"], PINS["att_A_e2e_sum"] + 999 * MS]
+
+
+def test_attainment_agrees_with_the_simulator():
+    # the simulator reports finished / attained / rejected per trace; the table it leaves gives the same by Eq. 2
+    wl = gen.random_traces(3, 5, 30, 60, 400)
+    sim = oracle.sim(wl)
+    c = oracle.attainment(wl)["counts"][-1]
+    assert c[1] == sim["finished"].sum() and c[2] == sim["attained"].sum() and c[3] == sim["rejected"].sum()

@@ -588,3 +588,40 @@ def test_pd_handoff_edges_and_errors():
     sched.pd_migrate(tab, now, mat, prt, 0, 0)          # nothing is RUNNING on a P instance yet: a no-op
     assert sched.status() == 0 and np.array_equal(tab.to_numpy()["replica_id"], wl0.table["replica_id"])
     sched.close()
+
+
+# ---- SLO attainment (Eq. 2) ---------------------------------------------------------------------------------
+def _attainment_parity(wl):
+    import paper_2508_15919_b200 as hfx
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    out = torch.full((len(wl.classes) + 1, 6), -3, dtype=torch.int64, device="cuda")
+    for _ in range(2):          # twice: the output must not accumulate
+        sched.attainment(tab, out)
+    st = sched.status()
+    c = oracle.attainment(wl)
+    assert st == c["status"] and np.array_equal(out.cpu().numpy(), c["counts"]), (out.cpu().numpy(), c["counts"])
+    sched.close()
+    return c["counts"]
+
+
+def test_attainment_parity():
+    cls = [(200 * MS, 30 * MS, 0), (1000 * MS, 0, 1)]
+    rows = [dict(state=gen.DONE, class_id=0, prompt_len=1000, output_len=101, gen=100, first_token_ns=47 * MS, last_token_ns=859_099_000, finish_ns=859_099_000),
+            dict(state=gen.DONE, class_id=0, output_len=11, gen=10, arrival_ns=100 * MS, first_token_ns=350 * MS, last_token_ns=850 * MS, finish_ns=850 * MS),
+            dict(state=gen.RUNNING, class_id=0, output_len=50, gen=3, arrival_ns=5 * MS, first_token_ns=15 * MS, last_token_ns=99 * MS),
+            dict(state=gen.REJECTED, class_id=1, prompt_len=100000), dict(state=gen.QUEUED, class_id=1, arrival_ns=7 * MS),
+            dict(state=gen.DONE, class_id=1, output_len=1, arrival_ns=MS, first_token_ns=1000 * MS, last_token_ns=1000 * MS, finish_ns=1000 * MS)]
+    c = _attainment_parity(make_wl(rows, cls))
+    assert list(c[2][:4]) == [6, 3, 2, 1]
+    _attainment_parity(make_wl([], cls))
+    # the table a simulation leaves, and a committed shared-queue table with bad rows
+    wl = gen.random_traces(4, 40, 100, 300, 600)
+    oracle.sim(wl)
+    c = _attainment_parity(wl)
+    assert c[-1][1] > 0
+    wl = gen.config4(R=32, n=100_003, steps=3)
+    for _ in range(3):
+        oracle.step(wl, commit=True)
+    wl.table["class_id"][::997] = 77
+    _attainment_parity(wl)
