@@ -222,8 +222,21 @@ __device__ inline int64_t warp_min_over_mask(const int64_t *cls_v, uint64_t mask
   return m;
 }
 
+// What a caller that plans the same replica again and again keeps between its calls (one copy per lane
+// of the planning warp, all lanes equal): the class sets seen last with their minima, and the last
+// answer of the search, around which the next one starts.  None of it changes a result.
+struct PlanMemo {
+  uint64_t m_run, m_q;
+  int64_t min_tpot, min_ttft;
+  int64_t n_safe;           // < 0: none yet
+  int have_run, have_q;
+};
+__device__ __forceinline__ void plan_memo_reset(PlanMemo &m) { m.m_run = 0; m.m_q = 0; m.min_tpot = 0; m.min_ttft = 0; m.n_safe = -1; m.have_run = 0; m.have_q = 0; }
+
 // Largest n in [0, cap] with E_p(n) * den <= num (num = nh:nl as 128 bits, den > 0), 0 if none.
-__device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t nl, uint64_t den, int64_t cap, int lane) {
+// `hint` >= 0: a value the answer is probably close to (tried first: 32 neighbours in one round).
+__device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t nl, uint64_t den, int64_t cap, int lane,
+                                     int64_t hint = -1) {
   auto fits = [&](int64_t n) {
     const uint64_t ep = (uint64_t)dev_Ep(p, n);
     const uint64_t ph = __umul64hi(ep, den), pl = ep * den;
@@ -231,6 +244,16 @@ __device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t n
   };
   if (!fits(0)) return 0;
   int64_t lo = 0, hi = cap;          // fits(lo); the answer lies in [lo, hi]
+  if (hint >= 0) {
+    int64_t base = hint - 15;
+    if (base < 1) base = 1;
+    if (base > cap) base = cap;
+    const int64_t cand = base + lane;
+    const int f = __popc(__ballot_sync(0xffffffffu, cand <= cap && fits(cand)));    // a prefix of the lanes
+    if (f == 0) hi = base - 1;                    // the answer lies below the neighbourhood
+    else if (f == 32) lo = base + 31;             // at or above its top
+    else return base + f - 1;
+  }
   while (lo < hi) {
     const int64_t step = (int64_t)(((uint64_t)(hi - lo) + 31u) >> 5);
     const int64_t cand = lo + (int64_t)(lane + 1) * step;
@@ -245,11 +268,16 @@ __device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t n
 
 __device__ inline void warp_plan(const HfxParams &p, const int64_t *cls_ttft, const int64_t *cls_tpot,
                                  const hfx_replica_cfg &cfg, int64_t now, int64_t mat, int64_t n_run, int64_t sum_kv,
-                                 uint64_t mask_run, uint64_t mask_q, ReplicaPlan &pl, int lane) {
+                                 uint64_t mask_run, uint64_t mask_q, ReplicaPlan &pl, int lane, PlanMemo *memo = nullptr) {
   pl.now = now; pl.mat = mat; pl.start = now > mat ? now : mat;
   pl.mode = cfg.mode; pl.token_cap = cfg.token_cap; pl.batch_cap = cfg.batch_cap;
   pl.n_run = n_run; pl.sum_kv = sum_kv;
-  const int64_t min_tpot = warp_min_over_mask(cls_tpot, mask_run, lane);
+  int64_t min_tpot;
+  if (memo && memo->have_run && memo->m_run == mask_run) min_tpot = memo->min_tpot;
+  else {
+    min_tpot = warp_min_over_mask(cls_tpot, mask_run, lane);
+    if (memo) { memo->m_run = mask_run; memo->min_tpot = min_tpot; memo->have_run = 1; }
+  }
   const bool prefill = cfg.mode == HFX_PREFILL;
   pl.n_eff = prefill ? 0 : n_run;
   pl.kv_eff = prefill ? 0 : sum_kv;
@@ -269,15 +297,22 @@ __device__ inline void warp_plan(const HfxParams &p, const int64_t *cls_ttft, co
       int64_t n_safe;
       if (p.budget_mode == HFX_BUDGET_CAP_ONLY) n_safe = cfg.token_cap;
       else {
-        const int64_t min_ttft = warp_min_over_mask(cls_ttft, mask_q, lane);
+        int64_t min_ttft;
+        if (memo && memo->have_q && memo->m_q == mask_q) min_ttft = memo->min_ttft;
+        else {
+          min_ttft = warp_min_over_mask(cls_ttft, mask_q, lane);
+          if (memo) { memo->m_q = mask_q; memo->min_ttft = min_ttft; memo->have_q = 1; }
+        }
         const bool decoding = pl.n_eff > 0 && pl.tpot_eff < HFX_INF;
+        const int64_t hint = memo ? memo->n_safe : -1;
         if (min_ttft == HFX_INF) n_safe = cfg.token_cap;
-        else if (!decoding) n_safe = warp_nsafe(p, 0, (uint64_t)min_ttft, 2, cfg.token_cap, lane);     // 2 E_p <= TTFT
+        else if (!decoding) n_safe = warp_nsafe(p, 0, (uint64_t)min_ttft, 2, cfg.token_cap, lane, hint);     // 2 E_p <= TTFT
         else if (pl.tpot_eff <= pl.e_d) n_safe = 0;
         else {
           const uint64_t x = (uint64_t)min_ttft, y = (uint64_t)(pl.tpot_eff - pl.e_d);
-          n_safe = warp_nsafe(p, __umul64hi(x, y), x * y, (uint64_t)(2 * pl.tpot_eff - pl.e_d), cfg.token_cap, lane);
+          n_safe = warp_nsafe(p, __umul64hi(x, y), x * y, (uint64_t)(2 * pl.tpot_eff - pl.e_d), cfg.token_cap, lane, hint);
         }
+        if (memo) memo->n_safe = n_safe;
       }
       budget = n_safe < cap_left ? n_safe : cap_left;
     }

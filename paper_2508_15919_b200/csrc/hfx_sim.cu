@@ -144,6 +144,8 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     __syncthreads();
 
     int executed = 0;
+    PlanMemo memo;          // of the planning warp: the trace's replica is planned every iteration
+    plan_memo_reset(memo);
     uint16_t *run_cur = s_run, *run_nxt = s_run2;
     for (int it = 0; it < a.iters; it++) {
       // ---- 1. arrivals: rows [head, head + k) with arrival <= now join the queue -----------
@@ -183,7 +185,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
         const uint32_t q0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_q[lane] > 0);
         const uint32_t q1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && S.cnt_q[lane + 32] > 0);
         ReplicaPlan pl0;
-        warp_plan(p, S.ttft, S.tpot, cfg, S.now, S.mat, S.nr, S.sum_kv, ((uint64_t)r1 << 32) | r0, ((uint64_t)q1 << 32) | q0, pl0, lane);
+        warp_plan(p, S.ttft, S.tpot, cfg, S.now, S.mat, S.nr, S.sum_kv, ((uint64_t)r1 << 32) | r0, ((uint64_t)q1 << 32) | q0, pl0, lane, &memo);
         if (lane == 0) S.plan = pl0;
       }
       __syncthreads();
