@@ -110,6 +110,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     if (tid == 0) {
       S.now = 0; S.mat = 0; S.sum_kv = 0; S.head = 0; S.nq = 0; S.nr = 0; S.stop = 0;
       S.n_fin = 0; S.n_rej = 0; S.n_att = 0; S.n_a = 0; S.n_b = 0; S.zero_prompt = 0;
+      S.arrived = 0; S.no = 0; S.na = 0; S.nr_next = 0; S.d_kv = 0;
     }
     __syncthreads();
     for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; S.ttft[c] = c < p.n_classes ? p.ttft[c] : 0; S.tpot[c] = c < p.n_classes ? p.tpot[c] : 0; }
@@ -149,8 +150,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     uint16_t *run_cur = s_run, *run_nxt = s_run2;
     for (int it = 0; it < a.iters; it++) {
       // ---- 1. arrivals: rows [head, head + k) with arrival <= now join the queue -----------
-      if (tid == 0) { S.arrived = 0; S.no = 0; S.na = 0; S.nr_next = 0; S.d_kv = 0; }
-      __syncthreads();
+      // (the iteration's counters were cleared by the thread that closed the previous one)
       {
         const int64_t now = S.now;
         const int head = S.head;
@@ -252,16 +252,16 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       }
 
       // ---- 4. maturity and the iteration's clock -------------------------------------------
+      // every thread knows what was admitted, so every thread forms the iteration's two times itself; the
+      // new maturity (a division) is left to one thread, beside the commit
+      const int64_t t1 = S.now + (adm_cnt > 0 ? dev_Ep(p, adm_cost) : 0);
+      const int64_t t2 = t1 + (nr > 0 ? S.plan.e_d : 0);
       if (tid == 0) {
         int64_t lp = 0;
-        const int64_t mat_next = dev_maturity_next(p, S.plan, adm_cnt, adm_cost, 0, &lp);
-        const int worked = adm_cnt > 0 || nr > 0;
-        S.t1 = S.now + (adm_cnt > 0 ? lp : 0);
-        S.t2 = S.t1 + (nr > 0 ? S.plan.e_d : 0);
-        S.worked = worked; S.mat_next = mat_next; S.nq = nq; S.na = adm_cnt;
+        S.mat_next = dev_maturity_next(p, S.plan, adm_cnt, adm_cost, 0, &lp);
+        S.worked = adm_cnt > 0 || nr > 0;
+        S.nq = nq; S.na = adm_cnt;
       }
-      __syncthreads();
-      const int64_t t1 = S.t1, t2 = S.t2;
 
       // ---- 5. commit ---------------------------------------------------------------------------
       int64_t d_kv = 0;
@@ -312,6 +312,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
         S.sum_kv += S.d_kv;
         S.nr = S.nr_next;
         S.mat = S.mat_next;
+        S.arrived = 0; S.no = 0; S.na = 0; S.nr_next = 0; S.d_kv = 0;      // for the next iteration
         if (S.worked) S.now = t2;
         else {
           int64_t ev = HFX_INF;
