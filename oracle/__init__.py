@@ -51,7 +51,7 @@ class _Replica(C.Structure):
 class _Config(C.Structure):
     _fields_ = [("model", _Model), ("classes", C.POINTER(_Class)), ("n_classes", C.c_int32),
                 ("replicas", C.POINTER(_Replica)), ("n_replicas", C.c_int32),
-                ("budget_mode", C.c_int32), ("weight_max", C.c_int32)]
+                ("budget_mode", C.c_int32), ("weight_max", C.c_int32), ("first_fit", C.c_int32)]
 
 
 _TABLE_COLS = ["replica_id", "class_id", "state", "prompt_len", "output_len", "gen", "arrival_ns",
@@ -189,7 +189,7 @@ class _Ctx:
         reps = (_Replica * wl.n_replicas)(*[_Replica(int(r[0]), int(r[1]), int(r[2])) for r in wl.replicas])
         self.keep += [cls, reps]
         self.cfg = _Config(_model(wl.model), cls, len(wl.classes), reps, wl.n_replicas,
-                           int(wl.budget_mode), int(wl.weight_max))
+                           int(wl.budget_mode), int(wl.weight_max), int(bool(wl.meta.get("first_fit", False))))
         self.table = _Table()
         self.table.n = wl.n_rows
         for k in _TABLE_COLS:

@@ -50,6 +50,7 @@ typedef struct {
   int32_t n_replicas;
   int32_t budget_mode;
   int32_t weight_max;
+  int32_t first_fit;   /* admission variant, see step 6 */
 } ora_config;
 
 typedef struct {
@@ -302,7 +303,11 @@ static int step_replica(const ora_config *c, const ora_table *t, int32_t r, int3
   /* 6. admission (dispatching step 3): the most urgent requests that fit.
    *    reading: a request that could not fit even alone is skipped; among the
    *    rest admission is the longest prefix whose running totals stay within
-   *    the budget and the batch cap (totals keep growing after a failure). */
+   *    the budget and the batch cap (totals keep growing after a failure).
+   *    Variant (first_fit): the other reading of "requests that fit" -- every
+   *    request is tried in order against what is left of the budget and the
+   *    batch cap, taken if it fits and passed over if not, so a large request
+   *    never shuts out the smaller ones behind it. */
   int64_t s_cost = 0, s_count = 0, adm_cost = 0, adm_count = 0, adm_kv = 0;
   for (int64_t q = 0; q < m; q++) {
     int64_t j = tup[q].row, i = rows[j];
@@ -310,7 +315,16 @@ static int step_replica(const ora_config *c, const ora_table *t, int32_t r, int3
     if (o->admitted_rows) o->admitted_rows[order_base + q] = -1;
     uint8_t a = 0;
     if (phase[j] == PH_RUNNING) a = 1;
-    else if (phase[j] == PH_QUEUED && cost[j] <= budget) {
+    else if (c->first_fit) {
+      if (phase[j] == PH_QUEUED && adm_cost + cost[j] <= budget &&
+          (cfg->batch_cap == 0 || n_eff + adm_count + 1 <= cfg->batch_cap)) {
+        a = 1;
+        if (o->admitted_rows) o->admitted_rows[order_base + adm_count] = (int32_t)i;
+        adm_cost += cost[j];
+        adm_count += 1;
+        adm_kv += (int64_t)t->prompt_len[i] + t->gen[i];
+      }
+    } else if (phase[j] == PH_QUEUED && cost[j] <= budget) {
       s_cost += cost[j];
       s_count += 1;
       if (s_cost <= budget && (cfg->batch_cap == 0 || n_eff + s_count <= cfg->batch_cap)) {

@@ -339,3 +339,52 @@ def test_dispatch_single_instance_equals_the_per_replica_step_without_skips():
     queued = (wl.table["state"] == 0) & (wl.table["arrival_ns"] <= now)
     assert np.array_equal(d["assign"][queued] == 0, s["admit"][queued] == 1)
     assert np.array_equal(d["slack"][queued], s["slack"][queued])
+
+
+# ---- first-fit admission variant ---------------------------------------------------------------------------
+def test_first_fit_admission_hand_case_and_properties():
+    # budget 2144 (idle instance, TTFT 200 ms); queue in priority order: 1144, 1100 (does not fit behind the
+    # first), 900 (fits: 2044), 100 (fits exactly: 2144), 16 (nothing left).  The prefix rule stops at the second.
+    cls = [(200 * MS, 30 * MS, 0)]
+    rows = [dict(prompt_len=pl, arrival_ns=-(5 - k) * MS, req_id=k) for k, pl in enumerate([1144, 1100, 900, 100, 16])]
+    wl = make_wl(rows, cls, now=[0])
+    o = oracle.step(wl)
+    assert o["budget"][0] == 2144 and list(o["admit"]) == [1, 0, 0, 0, 0] and o["adm_cost"][0] == 1144
+    wl.meta["first_fit"] = True
+    o = oracle.step(wl)
+    assert list(o["order"]) == [0, 1, 2, 3, 4] and list(o["admit"]) == [1, 0, 1, 1, 0]
+    assert o["adm_cost"][0] == 2144 and o["adm_count"][0] == 3 and list(o["admitted_rows"][:4]) == [0, 2, 3, -1]
+    # batch cap 2: the third fitting request is refused
+    wl.replicas[0, 2] = 2
+    o = oracle.step(wl)
+    assert list(o["admit"]) == [1, 0, 1, 0, 0] and o["adm_count"][0] == 2
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_first_fit_invariants_and_dominance(seed):
+    wl = gen.random_table(seed, 400 + 57 * seed, 1 + seed % 5, modes=MODES3 if seed % 2 else (gen.COLOCATED,),
+                          batch_cap=(0, 9)[seed % 3 == 1], tie_heavy=seed % 4 == 3)
+    a = oracle.step(wl)
+    wf = wl.copy(); wf.meta["first_fit"] = True
+    b = oracle.step(wf)
+    t = wl.table
+    # same budgets, same order; first fit admits at least what the prefix rule admits, within the same limits
+    assert np.array_equal(a["budget"], b["budget"]) and np.array_equal(a["order"], b["order"])
+    assert np.all(b["admit"] >= a["admit"]) and np.all(b["adm_count"] >= a["adm_count"])
+    for r in range(wl.n_replicas):
+        seg = b["order"][b["seg_off"][r]:b["seg_off"][r + 1]]
+        mode, cap, bcap = wl.replicas[r]
+        queued = seg[(t["state"][seg] == 0) & (t["arrival_ns"][seg] <= wl.now[r]) & (t["class_id"][seg] < len(wl.classes))]
+        cost = t["prompt_len"][queued].astype(np.int64) if mode != gen.DECODE else None
+        if cost is None:
+            continue
+        adm = b["admit"][queued] == 1
+        assert cost[adm].sum() == b["adm_cost"][r] <= b["budget"][r]
+        # walking the order, a request is refused only if it does not fit what is left at its turn
+        used, cnt = 0, 0
+        n_eff = 0 if mode == gen.PREFILL else int(b["n_run"][r])
+        for k in range(queued.size):
+            fits = used + cost[k] <= b["budget"][r] and (bcap == 0 or n_eff + cnt + 1 <= bcap)
+            assert bool(adm[k]) == bool(fits)
+            if fits:
+                used += int(cost[k]); cnt += 1
