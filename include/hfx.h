@@ -75,6 +75,14 @@ extern "C" {
 #define HFX_BUDGET_SAFE      0  /* Eq. 3 (generalised to the quadratic E_p)   */
 #define HFX_BUDGET_CAP_ONLY  1  /* capacity caps only, no SLO-derived bound   */
 
+/* hfx_options.flags */
+#define HFX_OPT_FIRST_FIT 1u    /* admission by first fit: dispatching step 3 ("the most urgent
+                                   requests that fit") read as "try every request in priority
+                                   order against what is left of the budget and the batch cap,
+                                   take it if it fits, pass it over if not", instead of the
+                                   default longest prefix of the requests that fit alone; applies
+                                   to hfx_sched_step and hfx_sim_run                          */
+
 /* hfx_sched_step flags */
 #define HFX_COMMIT 1u           /* apply the admitted batch to the table      */
 
@@ -114,7 +122,7 @@ typedef struct hfx_options {
   int32_t  budget_mode; /* HFX_BUDGET_*                                       */
   int32_t  weight_max;  /* 0: prio = class prio; >0: prio = clamp(weight_max -
                            weight, 0, 62) and the table's `weight` is read    */
-  uint32_t flags;       /* reserved, 0                                        */
+  uint32_t flags;       /* HFX_OPT_* bits                                     */
   uint32_t reserved;
 } hfx_options;
 

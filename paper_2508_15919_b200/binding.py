@@ -296,7 +296,8 @@ class Scheduler:
     """hfx_sched_create / hfx_sched_step / hfx_sim_run / hfx_sched_status on torch tensors."""
 
     def __init__(self, model: Sequence[int], classes: Sequence[Sequence[int]], replicas, max_rows: int,
-                 budget_mode: int = BUDGET_SAFE, weight_max: int = 0, stream: Optional[torch.cuda.Stream] = None):
+                 budget_mode: int = BUDGET_SAFE, weight_max: int = 0, stream: Optional[torch.cuda.Stream] = None,
+                 first_fit: bool = False):
         L = load_library()
         self._L = L
         self._h = C.c_void_p()
@@ -304,7 +305,7 @@ class Scheduler:
         cls = (_SloClass * len(classes))(*[_SloClass(int(a), int(b), int(p), 0) for a, b, p in classes])
         reps_np = np.asarray(replicas, np.int32).reshape(-1, 3)
         reps = (_ReplicaCfg * reps_np.shape[0])(*[_ReplicaCfg(int(r[0]), int(r[1]), int(r[2])) for r in reps_np])
-        opts = _Options(int(budget_mode), int(weight_max), 0, 0)
+        opts = _Options(int(budget_mode), int(weight_max), 1 if first_fit else 0, 0)
         self.n_replicas = reps_np.shape[0]
         self.stream = stream
         if stream is not None:

@@ -59,7 +59,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     if (replicas[r].token_cap < 1 || replicas[r].token_cap > HFX_MAX_TOKENS || replicas[r].batch_cap < 0) return HFX_E_ARG;
   }
   if (opts->budget_mode != HFX_BUDGET_SAFE && opts->budget_mode != HFX_BUDGET_CAP_ONLY) return HFX_E_ARG;
-  if (opts->weight_max < 0 || opts->weight_max > (1 << 20) || opts->flags != 0) return HFX_E_ARG;
+  if (opts->weight_max < 0 || opts->weight_max > (1 << 20) || (opts->flags & ~HFX_OPT_FIRST_FIT) != 0) return HFX_E_ARG;
 
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return HFX_E_CUDA; }
@@ -83,6 +83,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   }
   s->p.n_classes = n_classes; s->p.n_replicas = n_replicas;
   s->p.budget_mode = opts->budget_mode; s->p.weight_max = opts->weight_max;
+  s->p.first_fit = (opts->flags & HFX_OPT_FIRST_FIT) ? 1 : 0;
   s->opts = *opts; s->max_rows = max_rows; s->n_sm = n_sm;
   s->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
   s->launches = 0;

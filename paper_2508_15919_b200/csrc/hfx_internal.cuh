@@ -42,6 +42,7 @@ struct HfxParams {
   int32_t n_replicas;
   int32_t budget_mode;
   int32_t weight_max;
+  int32_t first_fit;      // admission variant: every request is tried against what is left of the budget
 };
 
 // One row after regrouping by replica: everything the per-replica kernel needs, 32 bytes
@@ -446,6 +447,44 @@ __device__ void block_sort(uint64_t *hi, uint32_t *lo, int n) {
     }
   }
   __syncthreads();
+}
+
+// First-fit admission along an order of n places, by one warp (all 32 lanes call).  cost_of(q) is the
+// cost of the candidate at place q, or -1 where there is none; every candidate is tried in order against
+// what is left of `budget` and of `room` (how many more may be taken) and taken if it fits; decide(q, taken)
+// is called once for every place.  32 places at a time: the first lane that still fits starts a run, the
+// run ends at the first lane that no longer fits behind it (that lane is refused for good), the lanes after
+// it are tried again with what is left then.
+template <typename CostF, typename DecideF>
+__device__ __forceinline__ void warp_first_fit(int64_t n, int64_t budget, int64_t room, int lane, CostF cost_of, DecideF decide) {
+  int64_t used = 0, taken = 0;
+  for (int64_t base = 0; base < n; base += 32) {
+    const int64_t q = base + lane;
+    const int64_t c = q < n ? cost_of(q) : -1;
+    uint32_t pending = __ballot_sync(0xffffffffu, c >= 0);
+    bool mine = false;
+    while (pending) {
+      const int64_t rem = budget - used, left = room - taken;
+      const bool me = (pending >> lane) & 1u;
+      const uint32_t fit = left > 0 ? __ballot_sync(0xffffffffu, me && c <= rem) : 0u;
+      if (!fit) break;
+      const int l0 = __ffs(fit) - 1;
+      const bool in = me && lane >= l0;
+      const int64_t pre = warp_incl_scan_i64(in ? c : 0, lane);
+      const int32_t pcnt = warp_incl_scan_i32(in ? 1 : 0, lane);
+      const bool ok = in && pre <= rem && (int64_t)pcnt <= left;
+      const uint32_t bad = __ballot_sync(0xffffffffu, in && !ok);
+      const int l1 = bad ? __ffs(bad) - 1 : 32;            // the run is the pending lanes in [l0, l1)
+      const bool take = in && lane < l1;
+      if (take) mine = true;
+      const uint32_t tm = __ballot_sync(0xffffffffu, take);
+      const int last = 31 - __clz(tm);                      // tm has lane l0 at least
+      used += __shfl_sync(0xffffffffu, pre, last);
+      taken += __shfl_sync(0xffffffffu, pcnt, last);
+      pending = l1 >= 31 ? 0u : (pending & ~((2u << l1) - 1u));
+    }
+    if (q < n) decide(q, mine);
+  }
 }
 
 // Brackets one kernel launch with events when profiling is on; counts the launch either way.

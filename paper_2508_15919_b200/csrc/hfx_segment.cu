@@ -250,6 +250,19 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
                                               const HfxRec *seg, uint32_t b, uint32_t *s_lo, int n_sorted,
                                               BlockShared &sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  if (p.first_fit) {       // the first warp walks the order and marks what it takes (bit 17)
+    if (warp == 0) {
+      const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
+      warp_first_fit(n_sorted, pl.budget, room, lane,
+                     [&](int64_t q) -> int64_t {
+                       const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + (s_lo[q] & 0xffffu)) + 1);
+                       if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
+                       return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
+                     },
+                     [&](int64_t q, bool taken) { if (taken) s_lo[q] |= 0x20000u; });
+    }
+    __syncthreads();
+  }
   for (int tile = 0; tile < n_sorted; tile += blockDim.x) {
     const int q = tile + threadIdx.x;
     int64_t cost = 0, kv = 0;
@@ -263,7 +276,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
       if (kind == KIND_QUEUED) {
         kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
         const int64_t c = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-        if (c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
+        if (p.first_fit ? (s_lo[q] & 0x20000u) != 0 : c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
       }
       a.order[b + q] = row;
     }
@@ -282,7 +295,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
     sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
     bool adm = false;
-    if (cnt) adm = sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap);
+    if (cnt) adm = p.first_fit || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
     if (q < n_sorted) {
       if (kind == KIND_RUNNING || adm) a.admit[row] = 1;
       if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
@@ -612,6 +625,21 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
       __syncthreads();
     }
 
+    // ---- first-fit variant: the first warp walks the order and marks what it takes (bit 17) -----------
+    if (p.first_fit) {
+      if (warp == 0) {
+        const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
+        warp_first_fit(n_act, pl.budget, room, lane,
+                       [&](int64_t q) -> int64_t {
+                         const uint4 w1 = s_w1[s_lo[q] & 0xffffu];
+                         if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
+                         return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
+                       },
+                       [&](int64_t q, bool taken) { if (taken) s_lo[q] |= 0x20000u; });
+      }
+      __syncthreads();
+    }
+
     // ---- admission: each thread walks TINY_IPT consecutive places of the order ---------------------
     const int q0 = threadIdx.x * TINY_IPT;
     int64_t cost[TINY_IPT], kvs[TINY_IPT];
@@ -623,14 +651,15 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
       const int q = q0 + k;
       cost[k] = -1; kvs[k] = 0; rows[k] = -1; kinds[k] = KIND_DEAD;
       if (q < n_act) {
-        const int li = s_lo[q];
+        const int li = s_lo[q] & 0xffffu;
         const uint4 w1 = s_w1[li];
         rows[k] = s_row[li];
         kinds[k] = (w1.w >> 8) & 0xff;
         if (kinds[k] == KIND_QUEUED) {
           const int64_t kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
           const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-          if (cc <= pl.budget) { cost[k] = cc; kvs[k] = kv; my_cost += cc; my_cnt++; }
+          // what counts towards the totals: rows that fit alone, or (first fit) exactly the rows taken
+          if (p.first_fit ? (s_lo[q] & 0x20000u) != 0 : cc <= pl.budget) { cost[k] = cc; kvs[k] = kv; my_cost += cc; my_cnt++; }
         }
         a.order[b + q] = rows[k];
       }
@@ -651,7 +680,7 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
         bool adm = false;
         if (cost[k] >= 0) {
           run_c += cost[k]; run_n += 1;
-          adm = run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap);
+          adm = p.first_fit || (run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap));
           if (adm) { ac += cost[k]; ak += kvs[k]; an++; if (a.admitted_rows) a.admitted_rows[b + run_n - 1] = rows[k]; }
         }
         if (kinds[k] == KIND_RUNNING || adm) a.admit[rows[k]] = 1;
@@ -831,6 +860,19 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
 
     // admission walk by block 0 with a carried prefix, then commit by the whole grid
     if (blockIdx.x == 0) {
+      if (p.first_fit) {     // the first warp walks the order; lo (free now that the sort is over) says what it took
+        if (warp == 0) {
+          const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
+          warp_first_fit(n_act, pl.budget, room, lane,
+                         [&](int64_t q) -> int64_t {
+                           const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + idx[q]) + 1);
+                           if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
+                           return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
+                         },
+                         [&](int64_t q, bool taken) { lo[q] = taken ? 2u : 0u; });
+        }
+        __syncthreads();
+      }
       for (int64_t tile = 0; tile < n_act; tile += blockDim.x) {
         const int64_t q = tile + threadIdx.x;
         int64_t cost = 0, kv = 0;
@@ -844,7 +886,7 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
           if (kind == KIND_QUEUED) {
             kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
             const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-            if (cc <= pl.budget) { cost = cc; cnt = 1; } else kv = 0;
+            if (p.first_fit ? lo[q] == 2u : cc <= pl.budget) { cost = cc; cnt = 1; } else kv = 0;
           }
           a.order[b + q] = row;
         }
@@ -862,7 +904,7 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
         sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
         sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
         bool adm = false;
-        if (cnt) adm = sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap);
+        if (cnt) adm = p.first_fit || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
         if (q < n_act) {
           if (kind == KIND_RUNNING || adm) a.admit[row] = 1;
           if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;

@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           uint64_t bk = ~0ull; uint32_t bid = ~0u; int bslot = -1;
           for (int s = tid; s < nq; s += SIM_THREADS) {
             const int i = s_q[s];
-            if ((int64_t)s_prompt[i] > budget) continue;
+            if ((int64_t)s_prompt[i] > (p.first_fit ? budget - adm_cost : budget)) continue;      // first fit: against what is left
             // slack of a queued request: ttft_slo - (start - arrival) - E_p(prompt_len) = base - start
             const int64_t base = s_arr[i];
             const int64_t sl = base != BASE_UNBOUNDED ? dev_clamp_slack(base - start) : HFX_SLACK_MAX;

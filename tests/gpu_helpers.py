@@ -17,7 +17,7 @@ SIM_KEYS = {"iters_executed": "iters_executed", "finished": "finished", "rejecte
 
 def make_sched(wl, max_rows=None):
     return hfx.Scheduler(wl.model, wl.classes, wl.replicas, max_rows or max(wl.n_rows, 1),
-                         budget_mode=wl.budget_mode, weight_max=wl.weight_max)
+                         budget_mode=wl.budget_mode, weight_max=wl.weight_max, first_fit=bool(wl.meta.get("first_fit", False)))
 
 
 def assert_step_parity(wl, steps=1, commit=False, optional=True, sched=None):

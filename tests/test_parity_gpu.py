@@ -625,3 +625,26 @@ def test_attainment_parity():
         oracle.step(wl, commit=True)
     wl.table["class_id"][::997] = 77
     _attainment_parity(wl)
+
+
+# ---- first-fit admission variant -----------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(8))
+def test_first_fit_random_tables(seed):
+    wl = gen.random_table(50 + seed, 1500 + 1333 * seed, 1 + (seed * 3) % 11, modes=MODES3, tie_heavy=seed % 3 == 0,
+                          batch_cap=(0, 7)[seed % 2], weight_max=(0, 16)[seed % 4 == 1],
+                          budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 2], grouped=seed % 4 == 3)
+    wl.meta["first_fit"] = True
+    assert_step_parity(wl, steps=3, commit=True)
+
+
+def test_first_fit_all_segment_sizes_and_simulator():
+    for wl in (gen.config4(R=16, n=30_000, steps=3), gen.random_table(7, 9000, 1, tie_heavy=True),
+               gen.random_table(9, 40_001, 1), gen.config2(R=8, rows_per=2048, inflight=0.02)):
+        wl.meta["first_fit"] = True
+        assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_traces(11, 12, 60, 400, 500)
+    wl.meta["first_fit"] = True
+    assert_sim_parity(wl)
+    wl = gen.config1()
+    wl.meta["first_fit"] = True
+    assert_sim_parity(wl)
