@@ -257,7 +257,8 @@ typedef struct hfx_dispatch_out {
   int64_t *maturity_next;  /* [R] */
 } hfx_dispatch_out;
 
-/* The four dispatching steps of Sec. 3.3.1 (colocated mode) over a shared
+/* The four dispatching steps of Sec. 3.3.1 (colocated mode, and the P stage of
+ * the disaggregated mode) over a shared
  * global queue, for the decisions due at time now_ns: (1) the instances whose
  * maturity time (maturity_ns, device, [R]) has come take their turn once each,
  * earliest maturity first, ties in index order; (2) each gets its safe token
@@ -275,8 +276,11 @@ typedef struct hfx_dispatch_out {
  * than every instance's token_cap can never be served and is left out of the
  * queue.  The table is not changed; the caller binds the dispatched rows
  * (replica_id := assign) before the next hfx_sched_step.
- * Every replica of the scheduler must be HFX_COLOCATED, and there may be at
- * most 4096 of them.  The first call allocates the call's workspace (44 bytes
+ * HFX_PREFILL replicas take part the same way with the budget and maturity
+ * update of their stage (the "P-stage Dispatcher": no decode batch, maturity =
+ * end of the prefill batch); HFX_DECODE replicas are served from their own
+ * queue of prefilled requests by hfx_sched_step and take no part (budget 0).
+ * The scheduler may have at most 4096 replicas.  The first call allocates the call's workspace (44 bytes
  * per row of max_rows) with cudaMalloc, so it should not be made inside a
  * stream capture; hfx_sched_destroy frees it.
  * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_NOMEM, HFX_E_CUDA. */

@@ -674,6 +674,11 @@ uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const i
  *   it.  A prompt longer than every instance's token cap can never be served
  *   and is left out of the queue.
  * reading: instances tie on maturity in index order.
+ * The same four steps serve the P stage of the disaggregated mode ("P-stage
+ * Dispatcher"): a PREFILL instance takes part with the budget and the maturity
+ * update of its stage (no decode batch: E_d = 0, maturity = end of the prefill
+ * batch).  DECODE instances are served by the Migrator from the queue of
+ * prefilled requests (the per-replica step) and take no part here.
  * ========================================================================== */
 typedef struct {
   int32_t *assign;        /* [n] instance a queued row is dispatched to, else -1         */
@@ -712,7 +717,7 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
   int32_t cap_max = 0;
   for (int32_t r = 0; r < R; r++) {
     min_tpot[r] = ORA_INF;
-    if (c->replicas[r].token_cap > cap_max) cap_max = c->replicas[r].token_cap;
+    if (c->replicas[r].mode != MODE_DECODE && c->replicas[r].token_cap > cap_max) cap_max = c->replicas[r].token_cap;
   }
 
   /* in-flight requests: the running batch of each instance; the queue */
@@ -752,13 +757,18 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
   int32_t nm = 0;
   for (int32_t r = 0; r < R; r++) {
     const ora_replica *cfg = &c->replicas[r];
-    const int64_t e_d = n_run[r] > 0 ? ora_Ed(M, n_run[r], sum_kv[r]) : 0;
+    /* a P-stage instance starts from an empty instance: it has no decode batch */
+    const int64_t n_eff = cfg->mode == MODE_PREFILL ? 0 : n_run[r];
+    const int64_t tpot_eff = cfg->mode == MODE_PREFILL ? ORA_INF : min_tpot[r];
+    const int64_t e_d = n_eff > 0 ? ora_Ed(M, n_eff, sum_kv[r]) : 0;
     int64_t budget = 0;
-    if (maturity[r] <= now) {
+    if (cfg->mode == MODE_DECODE) {
+      /* takes no part: reported with the decode latency of its batch, budget 0 */
+    } else if (maturity[r] <= now) {
       int64_t n_safe;
       if (c->budget_mode == BUDGET_CAP_ONLY) n_safe = cfg->token_cap;
-      else n_safe = ora_nsafe(M, ora_epmax(min_ttft, n_run[r] > 0 && min_tpot[r] < ORA_INF, min_tpot[r], e_d), cfg->token_cap);
-      const int64_t cap_left = cfg->token_cap - n_run[r] > 0 ? cfg->token_cap - n_run[r] : 0;
+      else n_safe = ora_nsafe(M, ora_epmax(min_ttft, n_eff > 0 && tpot_eff < ORA_INF, tpot_eff, e_d), cfg->token_cap);
+      const int64_t cap_left = cfg->token_cap - n_eff > 0 ? cfg->token_cap - n_eff : 0;
       budget = n_safe < cap_left ? n_safe : cap_left;
       inst[nm].mat = maturity[r]; inst[nm].id = r; nm++;
     }
@@ -787,7 +797,7 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
       const int64_t i = q[cursor].row;
       if (t->prompt_len[i] > budget_max) { cursor++; continue; }   /* fits no instance in this call */
       if (cost + t->prompt_len[i] > o->budget[r]) break;
-      if (cfg->batch_cap != 0 && n_run[r] + count + 1 > cfg->batch_cap) break;
+      if (cfg->batch_cap != 0 && (cfg->mode == MODE_PREFILL ? 0 : n_run[r]) + count + 1 > cfg->batch_cap) break;
       cost += t->prompt_len[i];
       count += 1;
       o->assign[i] = r;
@@ -798,8 +808,9 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
     if (count > 0) {
       /* Maturity = E_p + k*E_d as in the per-instance step */
       const int64_t lp = ora_Ep(M, cost), e_d = o->e_d[r];
-      i128 kk = 0;
-      if (n_run[r] > 0 && min_tpot[r] < ORA_INF && min_tpot[r] > e_d) kk = ((i128)lp + (min_tpot[r] - e_d) - 1) / (min_tpot[r] - e_d);
+      i128 kk = 0;      /* a P-stage instance has E_d = 0 and no decode batch: maturity = end of the prefill batch */
+      if (cfg->mode != MODE_PREFILL && n_run[r] > 0 && min_tpot[r] < ORA_INF && min_tpot[r] > e_d)
+        kk = ((i128)lp + (min_tpot[r] - e_d) - 1) / (min_tpot[r] - e_d);
       i128 v = (i128)now + lp + kk * e_d;
       o->maturity_next[r] = v > ORA_TIME_MAX ? ORA_TIME_MAX : (int64_t)v;
     }

@@ -220,10 +220,8 @@ extern "C" int hfx_dispatch_step(hfx_sched *s, const hfx_table *t, int64_t now_n
                        o->e_d_ns, o->n_run, o->sum_kv, o->adm_cost, o->adm_count, o->maturity_next};
   for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
   int32_t cap_max = 0;
-  for (int r = 0; r < s->p.n_replicas; r++) {
-    if (h->h_cfg[r].mode != HFX_COLOCATED) return HFX_E_ARG;
-    if (h->h_cfg[r].token_cap > cap_max) cap_max = h->h_cfg[r].token_cap;
-  }
+  for (int r = 0; r < s->p.n_replicas; r++)
+    if (h->h_cfg[r].mode != HFX_DECODE && h->h_cfg[r].token_cap > cap_max) cap_max = h->h_cfg[r].token_cap;
   return hfx_launch_dispatch(s, t, now_ns, maturity_ns, o, cap_max);
 }
 

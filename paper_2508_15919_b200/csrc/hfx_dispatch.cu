@@ -1,5 +1,5 @@
 // hfx_dispatch_step: the four dispatching steps of Sec. 3.3.1 over a shared global queue, for every
-// instance whose maturity time has come, in maturity order.
+// colocated or P-stage instance whose maturity time has come, in maturity order.
 //
 //   k_disp_scan     one streaming pass over the table: the running batch of every instance (count,
 //                   context tokens, classes), and the visible queue: slack, priority key, and an
@@ -345,6 +345,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_plan(const HfxParams p, c
   if (r >= p.n_replicas) return;
   ReplicaPlan pl;
   dev_plan(p, a.cfg[r], a.now, a.maturity[r], (int64_t)w.n_run[r], (int64_t)w.sum_kv[r], w.mask_run[r], w.ctl[0], pl);
+  if (pl.mode == HFX_DECODE) pl.budget = 0;      // a D-stage instance is served by the per-replica step, not from this queue
   w.plan[r] = pl;
   a.budget[r] = pl.budget;
   a.e_d[r] = pl.e_d;
@@ -412,7 +413,7 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
   if (threadIdx.x == 0) { s_nm = 0; s_k = 0; s_done = 0; s_cursor = 0; s_base = 0; s_basec = 0; }
   __syncthreads();
   for (int r = threadIdx.x; r < R; r += blockDim.x)
-    if (a.maturity[r] <= a.now) {
+    if (a.maturity[r] <= a.now && a.cfg[r].mode != HFX_DECODE) {
       const int k = atomicAdd(&s_nm, 1);
       s_mat[k] = (uint64_t)a.maturity[r] ^ (1ull << 63);
       s_id[k] = (uint32_t)r;
@@ -427,7 +428,7 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
     const ReplicaPlan *pl = w.plan + r;
     s_bud[k] = pl->budget;
     int64_t room = INT32_MAX;
-    if (pl->batch_cap != 0) { const int64_t left = (int64_t)pl->batch_cap - pl->n_run; room = left > 0 ? left : 0; }
+    if (pl->batch_cap != 0) { const int64_t left = (int64_t)pl->batch_cap - pl->n_eff; room = left > 0 ? left : 0; }
     s_room[k] = (int32_t)(room < INT32_MAX ? room : INT32_MAX);
   }
   if (threadIdx.x == 0) *a.n_mature = nm;

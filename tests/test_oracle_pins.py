@@ -493,3 +493,18 @@ def test_attainment_agrees_with_the_simulator():
     sim = oracle.sim(wl)
     c = oracle.attainment(wl)["counts"][-1]
     assert c[1] == sim["finished"].sum() and c[2] == sim["attained"].sum() and c[3] == sim["rejected"].sum()
+
+
+def test_dispatch_serves_the_p_stage():
+    # the hand-worked case with instance 0 as a P-stage instance: its 80 resident requests do not decode there, so
+    # it has the budget of an empty instance (2144), no E_d, and matures when its prefill batch ends:
+    # E_p(297) = 17056418.  A D-stage instance takes no part.
+    wl, now = _dispatch_hand_case()
+    wl.replicas[0, 0] = gen.PREFILL
+    wl.replicas[2, 0] = gen.DECODE
+    wl.maturity[2] = now - 100
+    o = oracle.dispatch(wl, now)
+    assert list(o["inst_order"]) == [1, 0, -1] and o["n_mature"][0] == 2
+    assert list(o["budget"]) == [2144, 2144, 0] and list(o["e_d"]) == [0, 0, 0] and list(o["n_run"]) == [80, 0, 0]
+    assert list(o["assign"][80:86]) == [1, 1, 0, 0, -1, -1] and list(o["adm_cost"]) == [297, 2144, 0]
+    assert o["maturity_next"][0] - now == 17_056_418 and o["maturity_next"][2] == now - 100

@@ -446,13 +446,10 @@ def test_dispatch_argument_errors_and_bad_rows():
     sched.dispatch_step(tab, now, mat, out)          # still usable
     assert sched.status() == 0
     sched.close()
-    # a scheduler with a P-stage or D-stage replica has no shared colocated queue to dispatch
-    wl2 = gen.random_table(42, 100, 2, modes=(gen.PREFILL,))
-    s2 = make_sched(wl2)
-    with pytest.raises(hfx.HfxError) as e:
-        s2.dispatch_step(hfx.DeviceTable.from_numpy(wl2.table), now, torch.from_numpy(wl2.maturity).cuda(), hfx.DispatchOut(100, 2))
-    assert e.value.code == -1
-    s2.close()
+    # P-stage instances are served like colocated ones, D-stage instances take no part
+    for seed in (42, 44, 45):
+        wl2 = gen.random_table(seed, 3000, 7, modes=MODES3, batch_cap=(0, 5)[seed % 2])
+        assert_dispatch_parity(wl2, int(wl2.now.max()))
     # rows with ids or lengths outside the domain are flagged and take no part
     wl3 = gen.random_table(43, 2000, 5, modes=(gen.COLOCATED,))
     wl3.table["class_id"][::97] = 200
@@ -648,3 +645,46 @@ def test_first_fit_all_segment_sizes_and_simulator():
     wl = gen.config1()
     wl.meta["first_fit"] = True
     assert_sim_parity(wl)
+
+
+def test_disaggregated_pipeline_dispatch_step_handoff():
+    # the whole disaggregated flow on both sides: requests wait unbound in the global queue, the dispatcher hands
+    # them to matured P instances, the caller binds them, a committed step prefills and decodes, the hand-off moves
+    # prefilled requests to the D instances
+    import paper_2508_15919_b200 as hfx
+    pairs = 4
+    wl = gen.pd_pairs(21, pairs, 400)
+    wl.table["replica_id"][:] = -1
+    cpu = wl.copy()
+    pair = gen.pd_partner_table(pairs)
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    now = torch.from_numpy(wl.now.copy()).cuda(); mat = torch.from_numpy(wl.maturity.copy()).cuda()
+    prt = torch.from_numpy(pair).cuda()
+    dout = hfx.DispatchOut(wl.n_rows, wl.n_replicas)
+    sout = hfx.StepOut(wl.n_rows, wl.n_replicas, optional=False)
+    bound = 0
+    for k in range(30):
+        now_g = (k + 1) * 25 * MS          # the dispatcher's tick; an idle instance's clock catches up at its next step
+        sched.dispatch_step(tab, now_g, mat, dout)
+        d = oracle.dispatch(cpu, now_g)
+        g = dout.to_numpy()
+        assert np.array_equal(g["assign"], d["assign"]) and np.array_equal(g["maturity_next"], d["maturity_next"]), k
+        # bind: the dispatched requests now belong to their instance, which is busy until its new maturity
+        asg = dout.t["assign"][:wl.n_rows]
+        tab.cols["replica_id"].copy_(torch.where(asg >= 0, asg, tab.cols["replica_id"]))
+        sel = d["assign"] >= 0
+        cpu.table["replica_id"][sel] = d["assign"][sel]
+        bound += int(sel.sum())
+        sched.step(tab, now, mat, sout, commit=True)
+        c = oracle.step(cpu, commit=True)
+        sched.pd_migrate(tab, now, mat, prt, 2 * MS, 500)
+        r = oracle.pd_migrate(cpu, pair, 2 * MS, 500)
+        st = sched.status()
+        assert st == (d["status"] | c["status"] | r["status"]), (k, st)
+        tg = tab.to_numpy()
+        for col in ("replica_id", "state", "gen", "first_token_ns", "last_token_ns", "finish_ns"):
+            assert np.array_equal(tg[col], cpu.table[col]), f"round {k}: column {col}"
+        assert np.array_equal(now.cpu().numpy(), cpu.now) and np.array_equal(mat.cpu().numpy(), cpu.maturity), k
+    sched.close()
+    assert bound > 50 and np.count_nonzero((cpu.table["state"] == 2) & (cpu.table["replica_id"] >= pairs)) > 0
