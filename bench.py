@@ -314,7 +314,7 @@ def run_gpu(args):
     # ---- the disaggregated mode end to end: committed steps coupled by the hand-off (rank 0) ----------
     pd = None
     if rank == 0 and not args.no_pd:
-        pw = gen.pd_pairs(7, 128, 8192)
+        pw = gen.pd_pairs(7, 128, 8192, permute_ids=False)      # request ids in arrival order, as a front end assigns them
         psched = hfx.Scheduler(pw.model, pw.classes, pw.replicas, pw.n_rows)
         ptab = hfx.DeviceTable.from_numpy(pw.table)
         pnow = torch.from_numpy(pw.now.copy()).cuda(); pmat = torch.from_numpy(pw.maturity.copy()).cuda()

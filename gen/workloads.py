@@ -378,7 +378,7 @@ def random_traces(seed: int, traces: int, rows_lo: int, rows_hi: int, iters: int
 
 
 def pd_pairs(seed: int, pairs: int, rows_per: int, rate: float = 40.0, token_cap: int = 8192, batch_cap: int = 64,
-             out_hi: int = 24, classes=None) -> Workload:
+             out_hi: int = 24, classes=None, permute_ids: bool = True) -> Workload:
     """Disaggregated deployment for the coupled P/D tests: `pairs` P instances (replicas 0 .. pairs-1) and
     their partner D instances (replicas pairs .. 2 pairs-1).  Every request starts QUEUED on a P instance
     (Poisson arrivals from time 0, short outputs so that requests finish within a few dozen rounds); all
@@ -392,7 +392,8 @@ def pd_pairs(seed: int, pairs: int, rows_per: int, rate: float = 40.0, token_cap
     tab["prompt_len"][:] = _lognormal_int(rng, 5.5, 1.0, 1, token_cap // 2, n)
     tab["output_len"][:] = rng.integers(1, out_hi + 1, n).astype(np.int32)
     tab["arrival_ns"][:] = np.rint(np.sort(rng.exponential(1.0 / (rate * pairs), n).cumsum()) * SEC).astype(np.int64)
-    tab["req_id"][:] = rng.permutation(n).astype(np.int32)
+    if permute_ids:          # ids in arrival order otherwise (the table is sorted by arrival)
+        tab["req_id"][:] = rng.permutation(n).astype(np.int32)
     reps = np.concatenate([_replicas(pairs, PREFILL, token_cap), _replicas(pairs, DECODE, token_cap, batch_cap)])
     return Workload(f"pd{seed}", DEFAULT_MODEL, classes, reps, tab, np.zeros(2 * pairs, np.int64),
                     np.zeros(2 * pairs, np.int64))
