@@ -2,10 +2,11 @@
 // colocated or P-stage instance whose maturity time has come, in maturity order.
 //
 //   k_disp_scan     one streaming pass over the table: the running batch of every instance (count,
-//                   context tokens, classes), and the visible queue: slack, priority key, and an
-//                   unordered list of (request id, row) pairs
+//                   context tokens, classes), slack and priority key of the visible queue's rows
+//   k_disp_compact  the queue's rows in row order as (sort word, row) pairs
 //   radix passes    the queue ordered by (priority, slack, request id): a stable least-significant-
-//                   digit radix sort, 8 bits a pass, first on the request id, then on the 48-bit key
+//                   digit radix sort, 8 bits a pass, on the 48-bit key; before that on the request id,
+//                   unless the ids rise with the rows (then row order already is id order)
 //   k_disp_plan     E_d and the safe token budget (Eq. 3) of every instance; the largest budget
 //   k_disp_prefix   the queue's rows in order, and the running totals (tokens, entries) of those that
 //                   fit some instance; larger entries are passed over
@@ -21,6 +22,7 @@
 #define RADIX_ITEMS 8                               // items a thread holds in the scatter pass
 #define RADIX_TILE (DISP_THREADS * RADIX_ITEMS)     // 2048
 #define DISP_MAX_INSTANCES 4096                     // instances the chain kernel orders in shared memory
+#define DISP_SCAN_BLOCKS_MAX 4096                   // blocks of the scan / compaction pair
 
 struct DispWork {
   // queue, ping-pong
@@ -34,7 +36,8 @@ struct DispWork {
   unsigned long long *sum_kv;    // [R]
   unsigned long long *mask_run;  // [R]
   unsigned long long *ctl;   // [0] classes present in the queue  [1] queue length  [2], [3] last-block counters
-                             // [4] largest budget among the matured instances
+                             // [4] largest budget among the matured instances  [5] request ids do not rise with the rows
+  uint32_t *blk_cnt;         // [DISP_SCAN_BLOCKS_MAX] queue rows found by each block of the scan
   ReplicaPlan *plan;         // [R]
   int32_t *run_start;        // [R] where an instance's run starts in the queue
   int32_t *run_len;          // [R] queue positions the run covers (passed-over entries included)
@@ -52,6 +55,12 @@ struct DispArgs {
   uint32_t *status;
 };
 
+// rows per block of the scan / compaction pair: equal contiguous runs, whole warps
+__host__ __device__ inline int64_t disp_chunk(int64_t n, int blocks) {
+  int64_t c = (n + blocks - 1) / blocks;
+  return (c + 31) & ~INT64_C(31);
+}
+
 // ------------------------------------------------------------------------------------------------
 // k_disp_scan
 // ------------------------------------------------------------------------------------------------
@@ -66,12 +75,18 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, c
   const int lane = threadIdx.x & 31;
   uint32_t bad = 0;
   unsigned long long qmask = 0;
-  const int64_t n_round = (a.n + 31) & ~INT64_C(31);       // whole warps stay together for the ballot
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += (int64_t)gridDim.x * blockDim.x) {
+  __shared__ uint32_t s_count;
+  if (threadIdx.x == 0) s_count = 0;
+  __syncthreads();
+  // every block takes a contiguous run of rows, so that the compaction that follows keeps row order
+  const int64_t chunk = disp_chunk(a.n, gridDim.x);
+  const int64_t lo = (int64_t)blockIdx.x * chunk, hi = lo + chunk < a.n ? lo + chunk : a.n;
+  uint32_t mine = 0;
+  bool falls = false;
+  for (int64_t i = lo + threadIdx.x; i < hi; i += blockDim.x) {
     bool in_queue = false;
     uint64_t k48 = 0;
-    uint32_t uid = 0;
-    if (i < a.n) {
+    {
       const uint32_t cls = a.class_id[i], st = a.state[i];
       const int32_t prompt = a.prompt_len[i], gen = a.gen[i];
       bool ok = true;
@@ -94,32 +109,67 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, c
           const int64_t x = (int64_t)p.weight_max - a.weight[i];
           prio = (int)(x < 0 ? 0 : (x > 62 ? 62 : x));
         } else prio = s_prio[cls];
-        k48 = dev_key48(PH_QUEUED, prio, slack);
-        uid = (uint32_t)a.req_id[i] ^ 0x80000000u;         // signed order as unsigned
+        k48 = dev_key48(PH_QUEUED, prio, slack);           // never 0: the phase bits are set
         qmask |= 1ull << cls;
         in_queue = true;
       }
       a.slack[i] = slack;
       a.assign[i] = -1;
       a.queue_order[i] = -1;
-    }
-    // append to the queue list: one counter update per warp
-    const uint32_t m = __ballot_sync(0xffffffffu, in_queue);
-    if (m) {
-      unsigned long long base = 0;
-      if (lane == 0) base = atomicAdd(&w.ctl[1], (unsigned long long)__popc(m));
-      base = __shfl_sync(0xffffffffu, base, 0);
-      if (in_queue) {
-        const uint64_t pos = base + __popc(m & ((1u << lane) - 1u));
-        w.key[0][pos] = uid;
-        w.val[0][pos] = (uint32_t)i;
-        w.rowkey[i] = k48;
-      }
+      w.rowkey[i] = k48;
+      mine += in_queue ? 1u : 0u;
+      if (i + 1 < a.n && !(a.req_id[i] < a.req_id[i + 1])) falls = true;
     }
   }
   qmask = warp_or_u64(qmask);
   if (lane == 0 && qmask) atomicOr(&w.ctl[0], qmask);
   if (bad) atomicOr(a.status, bad);
+  if (falls) atomicExch(&w.ctl[5], 1ull);
+  mine = (uint32_t)warp_sum_i64(mine);
+  if (lane == 0 && mine) atomicAdd(&s_count, mine);
+  __syncthreads();
+  if (threadIdx.x == 0) w.blk_cnt[blockIdx.x] = s_count;
+}
+
+// k_disp_compact: the queue rows in row order, as (sort word, row) pairs.  A block starts where the blocks
+// before it end (it adds up their counts) and places its own rows by a block-wide prefix of the "in the
+// queue" flags.  When the request ids rise with the rows the pairs carry the 48-bit key at once (row
+// order is id order, and the radix passes keep it among equal keys); otherwise they carry the request id,
+// which is ordered first.
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_compact(const DispArgs a, const DispWork w) {
+  __shared__ uint32_t s_warp[DISP_THREADS / 32];
+  __shared__ unsigned long long s_base;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) s_base = 0;
+  __syncthreads();
+  {
+    unsigned long long part = 0;
+    for (int bb = threadIdx.x; bb < (int)blockIdx.x; bb += blockDim.x) part += w.blk_cnt[bb];
+    part = (unsigned long long)warp_sum_i64((int64_t)part);
+    if (lane == 0 && part) atomicAdd(&s_base, part);
+  }
+  __syncthreads();
+  unsigned long long run = s_base;
+  const bool by_id = w.ctl[5] != 0;
+  const int64_t chunk = disp_chunk(a.n, gridDim.x);
+  const int64_t lo = (int64_t)blockIdx.x * chunk, hi = lo + chunk < a.n ? lo + chunk : a.n;
+  for (int64_t i0 = lo; i0 < hi; i0 += blockDim.x) {
+    const int64_t i = i0 + threadIdx.x;
+    const uint64_t k48 = i < hi ? w.rowkey[i] : 0;
+    const uint32_t m = __ballot_sync(0xffffffffu, k48 != 0);
+    if (lane == 0) s_warp[warp] = __popc(m);
+    __syncthreads();
+    uint32_t before = 0, all = 0;
+    for (int k = 0; k < DISP_THREADS / 32; k++) { const uint32_t c = s_warp[k]; if (k < warp) before += c; all += c; }
+    if (k48 != 0) {
+      const unsigned long long pos = run + before + __popc(m & ((1u << lane) - 1u));
+      w.key[0][pos] = by_id ? (uint64_t)((uint32_t)a.req_id[i] ^ 0x80000000u) : k48;      // signed id order as unsigned
+      w.val[0][pos] = (uint32_t)i;
+    }
+    run += all;
+    __syncthreads();
+  }
+  if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) w.ctl[1] = run;      // the queue's length
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -131,8 +181,10 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, c
 // items out.  The item count lives on the device (ctl[1]); tiles beyond it leave at once.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(DISP_THREADS) k_radix_hist(const uint64_t *__restrict__ keys, const unsigned long long *ctl_n,
-                                                             int shift, uint32_t *__restrict__ hist) {
+                                                             int shift, uint32_t *__restrict__ hist,
+                                                             const unsigned long long *only_if) {
   __shared__ uint32_t s_h[256];
+  if (only_if && *only_if == 0) return;      // a pass on the request id, and the ids already rise with the rows
   const int64_t n = (int64_t)*ctl_n;
   const int32_t tiles = (int32_t)((n + RADIX_TILE - 1) / RADIX_TILE);
   const int tile = blockIdx.x;
@@ -149,8 +201,9 @@ __global__ void __launch_bounds__(DISP_THREADS) k_radix_hist(const uint64_t *__r
 __global__ void __launch_bounds__(DISP_THREADS) k_radix_scatter(const uint64_t *__restrict__ keys_in, const uint32_t *__restrict__ vals_in,
                                                                 uint64_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out,
                                                                 const unsigned long long *ctl_n, int shift,
-                                                                const uint32_t *__restrict__ hist) {
+                                                                const uint32_t *__restrict__ hist, const unsigned long long *only_if) {
   __shared__ uint64_t s_key[RADIX_TILE];
+  if (only_if && *only_if == 0) return;
   __shared__ uint32_t s_base[256];               // where the tile's items of each digit go
   __shared__ uint32_t s_val[RADIX_TILE];
   __shared__ uint32_t s_item[2][RADIX_TILE];     // digit << 16 | position in the tile
@@ -236,7 +289,9 @@ __global__ void __launch_bounds__(DISP_THREADS) k_radix_scatter(const uint64_t *
 
 // after the request-id passes: the 48-bit key of every queue entry, in the order reached so far
 __global__ void __launch_bounds__(DISP_THREADS) k_disp_gather(uint64_t *__restrict__ keys, const uint32_t *__restrict__ vals,
-                                                              const uint64_t *__restrict__ rowkey, const unsigned long long *ctl_n) {
+                                                              const uint64_t *__restrict__ rowkey, const unsigned long long *ctl_n,
+                                                              const unsigned long long *only_if) {
+  if (*only_if == 0) return;
   const int64_t n = (int64_t)*ctl_n;
   for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (int64_t)gridDim.x * blockDim.x)
     keys[j] = rowkey[vals[j]];
@@ -506,7 +561,7 @@ int hfx_dispatch_configure() {
 static void disp_free(DispWork &w) {
   cudaFree(w.key[0]); cudaFree(w.key[1]); cudaFree(w.val[0]); cudaFree(w.val[1]); cudaFree(w.rowkey); cudaFree(w.prefix);
   cudaFree(w.hist); cudaFree(w.tile_sum); cudaFree(w.n_run); cudaFree(w.sum_kv); cudaFree(w.mask_run); cudaFree(w.ctl);
-  cudaFree(w.plan); cudaFree(w.run_start); cudaFree(w.run_len); cudaFree(w.prefix_cnt);
+  cudaFree(w.plan); cudaFree(w.run_start); cudaFree(w.run_len); cudaFree(w.prefix_cnt); cudaFree(w.blk_cnt);
   cudaGetLastError();
 }
 
@@ -541,6 +596,7 @@ static int disp_workspace(hfx_sched *s, hfx_dispatch_ws **out) {
   ok = ok && cudaMalloc(&w.sum_kv, sizeof(unsigned long long) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.mask_run, sizeof(unsigned long long) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.ctl, 256) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.blk_cnt, sizeof(uint32_t) * DISP_SCAN_BLOCKS_MAX) == cudaSuccess;
   ok = ok && cudaMalloc(&w.plan, sizeof(ReplicaPlan) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.run_start, sizeof(int32_t) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.run_len, sizeof(int32_t) * R) == cudaSuccess;
@@ -578,21 +634,26 @@ int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const 
     KernelScope ks(s, KSLOT_DISPATCH);
     int grid = (int)((n + DISP_THREADS - 1) / DISP_THREADS);
     if (grid > s->n_sm * 8) grid = s->n_sm * 8;
+    if (grid > DISP_SCAN_BLOCKS_MAX) grid = DISP_SCAN_BLOCKS_MAX;
     if (grid < 1) grid = 1;
     k_disp_scan<<<grid, DISP_THREADS, 0, st>>>(s->p, a, w);
+    s->launches++;
+    k_disp_compact<<<grid, DISP_THREADS, 0, st>>>(a, w);
   }
   int slot = 0;
-  auto pass = [&](int shift) {
-    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_hist<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.ctl + 1, shift, w.hist); }
-    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_scatter<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.key[slot ^ 1], w.val[slot ^ 1], w.ctl + 1, shift, w.hist); }
+  auto pass = [&](int shift, const unsigned long long *only_if) {
+    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_hist<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.ctl + 1, shift, w.hist, only_if); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_scatter<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.key[slot ^ 1], w.val[slot ^ 1], w.ctl + 1, shift, w.hist, only_if); }
     slot ^= 1;
   };
-  for (int shift = 0; shift < 32; shift += 8) pass(shift);            // by request id
+  // by request id, only when the ids do not rise with the rows (the kernels leave at once otherwise; an even
+  // number of passes, so the pairs are back in the first buffer either way)
+  for (int shift = 0; shift < 32; shift += 8) pass(shift, w.ctl + 5);
   {
     KernelScope ks(s, KSLOT_DISPATCH);
-    k_disp_gather<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.rowkey, w.ctl + 1);
+    k_disp_gather<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.rowkey, w.ctl + 1, w.ctl + 5);
   }
-  for (int shift = 0; shift < 48; shift += 8) pass(shift);            // by (priority, slack)
+  for (int shift = 0; shift < 48; shift += 8) pass(shift, nullptr);   // by (priority, slack)
   { KernelScope ks(s, KSLOT_DISPATCH); k_disp_plan<<<(R + DISP_THREADS - 1) / DISP_THREADS, DISP_THREADS, 0, st>>>(s->p, a, w); }
   { KernelScope ks(s, KSLOT_DISPATCH); k_disp_tilesum<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.ctl + 3); }
   { KernelScope ks(s, KSLOT_DISPATCH); k_disp_prefix<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.prefix, w.prefix_cnt, o->queue_order, o->n_queue); }
