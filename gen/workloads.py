@@ -403,6 +403,44 @@ def pd_partner_table(pairs: int) -> np.ndarray:
     return np.concatenate([np.arange(pairs, 2 * pairs), -np.ones(pairs)]).astype(np.int32)
 
 
+def elastic(seed: int, R: int, n: int, rates=(10.0, 120.0), period: float = 2.0, token_cap: int = 8192,
+            batch_cap: int = 64, out_hi: int = 24, prompt_hi: int = 2000) -> Workload:
+    """Colocated fleet of up to R instances fed from one global queue, for the scaling loop: n requests, unbound
+    (replica_id -1), arriving as a two-state modulated Poisson process (quiet / burst, re-drawn every `period`
+    seconds) so that load rises above and falls below what a fixed fleet serves; short outputs, all clocks 0.
+    Prompts stay below the safe budget of an idle instance under the strictest TTFT (2144 tokens with the default
+    model), so every request can be dispatched at some time."""
+    rng = np.random.default_rng(seed)
+    tab = _empty_table(n)
+    tab["replica_id"][:] = -1
+    tab["class_id"][:] = rng.choice(4, n, p=[0.4, 0.3, 0.2, 0.1]).astype(np.uint8)
+    tab["prompt_len"][:] = _lognormal_int(rng, 6.0, 1.0, 16, prompt_hi, n)
+    tab["output_len"][:] = rng.integers(1, out_hi + 1, n).astype(np.int32)
+    tab["arrival_ns"][:] = _mmpp_arrivals(rng, n, rates, period)
+    tab["req_id"][:] = np.arange(n, dtype=np.int32)
+    return Workload(f"elastic{seed}", DEFAULT_MODEL, CLASSES_4, _replicas(R, COLOCATED, token_cap, batch_cap), tab,
+                    np.zeros(R, np.int64), np.zeros(R, np.int64))
+
+
+INST_OFF, INST_STARTING, INST_ACTIVE, INST_DRAINING = 0, 1, 2, 3
+T_NEVER = np.iinfo(np.int64).max
+
+
+def new_fleet(blocks_cap, active) -> Dict[str, np.ndarray]:
+    """Instance records for the scaling loop: the instances listed in `active` are ACTIVE since time 0 and due
+    for dispatching at once, the others are OFF (never due)."""
+    cap = np.ascontiguousarray(blocks_cap, np.int32)
+    R = cap.size
+    f = dict(inst_state=np.zeros(R, np.int32), ready=np.zeros(R, np.int64), billed=np.zeros(R, np.int64),
+             since=np.zeros(R, np.int64), total_blocks=np.zeros(R, np.int32), due=np.full(R, T_NEVER, np.int64),
+             blocks_cap=cap.copy())
+    a = np.asarray(list(active), np.int64)
+    f["inst_state"][a] = INST_ACTIVE
+    f["due"][a] = 0
+    f["total_blocks"][a] = cap[a]
+    return f
+
+
 def by_name(name: str, **kw) -> Workload:
     return {"config1": config1, "config2": config2, "config3": config3, "config4": config4,
             "config5": config5}[name](**kw)

@@ -51,7 +51,8 @@ class _Replica(C.Structure):
 class _Config(C.Structure):
     _fields_ = [("model", _Model), ("classes", C.POINTER(_Class)), ("n_classes", C.c_int32),
                 ("replicas", C.POINTER(_Replica)), ("n_replicas", C.c_int32),
-                ("budget_mode", C.c_int32), ("weight_max", C.c_int32), ("first_fit", C.c_int32)]
+                ("budget_mode", C.c_int32), ("weight_max", C.c_int32), ("first_fit", C.c_int32),
+                ("horizon", C.c_int64)]
 
 
 _TABLE_COLS = ["replica_id", "class_id", "state", "prompt_len", "output_len", "gen", "arrival_ns",
@@ -114,6 +115,16 @@ class _ScaleOut(C.Structure):
     _fields_ = [("counts", C.c_void_p), ("used_blocks", C.c_void_p), ("decision", C.c_void_p)]
 
 
+class _Fleet(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in ("inst_state", "ready", "billed", "since", "total_blocks", "due", "blocks_cap")]
+
+
+FLEET_DTYPES = dict(inst_state=np.int32, ready=np.int64, billed=np.int64, since=np.int64, total_blocks=np.int32,
+                    due=np.int64, blocks_cap=np.int32)
+INST_OFF, INST_STARTING, INST_ACTIVE, INST_DRAINING = 0, 1, 2, 3
+T_NEVER = np.iinfo(np.int64).max
+
+
 # defaults of the paper: 10 s window, eps_out 0.7, eps_in 1.1, eps_wait 1/4
 SCALE_DEFAULTS = dict(window=10_000_000_000, block_tokens=16, min_samples=10, eps_out=(7, 10), eps_in=(11, 10),
                       eps_wait=(1, 4))
@@ -149,6 +160,11 @@ def lib():
                                      C.c_void_p]
         L.ora_attainment.restype = C.c_uint32
         L.ora_attainment.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p]
+        L.ora_dispatch_bind.restype = None
+        L.ora_dispatch_bind.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64] + [C.c_void_p] * 4
+        L.ora_scale_apply.restype = None
+        L.ora_scale_apply.argtypes = [C.POINTER(_Config), C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(_Fleet),
+                                      C.c_void_p, C.c_void_p, C.c_void_p]
         L.ora_scale.restype = C.c_uint32
         L.ora_scale.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64, C.c_void_p, C.POINTER(_ScaleParams),
                                 C.POINTER(_ScaleOut)]
@@ -189,7 +205,8 @@ class _Ctx:
         reps = (_Replica * wl.n_replicas)(*[_Replica(int(r[0]), int(r[1]), int(r[2])) for r in wl.replicas])
         self.keep += [cls, reps]
         self.cfg = _Config(_model(wl.model), cls, len(wl.classes), reps, wl.n_replicas,
-                           int(wl.budget_mode), int(wl.weight_max), int(bool(wl.meta.get("first_fit", False))))
+                           int(wl.budget_mode), int(wl.weight_max), int(bool(wl.meta.get("first_fit", False))),
+                           int(wl.meta.get("horizon", np.iinfo(np.int64).max)))
         self.table = _Table()
         self.table.n = wl.n_rows
         for k in _TABLE_COLS:
@@ -257,6 +274,17 @@ def dispatch(wl, now: int) -> Dict[str, np.ndarray]:
     return out
 
 
+def dispatch_bind(wl, now: int, d: Dict[str, np.ndarray]) -> None:
+    """Bind the requests that dispatch() assigned (d = its result) to their instances, in place
+    (wl.table["replica_id"], wl.now)."""
+    L = lib()
+    ctx = _Ctx(wl)
+    asg = np.ascontiguousarray(d["assign"], np.int32); cnt = np.ascontiguousarray(d["adm_count"], np.int32)
+    assert asg.size == wl.n_rows and cnt.size == wl.n_replicas and wl.now.dtype == np.int64
+    L.ora_dispatch_bind(C.byref(ctx.cfg), C.byref(ctx.table), int(now), asg.ctypes.data, cnt.ctypes.data,
+                        wl.table["replica_id"].ctypes.data, wl.now.ctypes.data)
+
+
 def pd_migrate(wl, pair: np.ndarray, x0: int, x1: int) -> Dict[str, int]:
     """Hand-off of prefilled requests from the P instances of wl to their partner D instances, in place
     (wl.table["replica_id"], wl.table["state"], wl.now)."""
@@ -298,6 +326,25 @@ def slo_map(n_prio: int, window: Dict[str, np.ndarray], bounds: Dict[str, np.nda
     st = L.ora_slo_map(int(n_prio), C.byref(win), C.byref(bs), lq.ctypes.data, pend.ctypes.data, n, npr.ctypes.data,
                        ttft.ctypes.data, tpot.ctypes.data)
     return {"ttft_slo": ttft[:n], "tpot_slo": tpot[:n], "last_queue": lq, "status": int(st)}
+
+
+def scale_apply(wl, now: int, decision: np.ndarray, used_blocks: np.ndarray, cold_start, fleet: Dict[str, np.ndarray]) -> np.ndarray:
+    """Carry out one tick's decisions on `fleet` (dict of the FLEET_DTYPES arrays, updated in place); of wl the
+    replica modes are read and the clocks wl.now / wl.maturity of an instance that comes up are advanced.  Returns
+    the cost per pool (instance-time charged so far, Eq. 1 without UnitCost)."""
+    L = lib()
+    ctx = _Ctx(wl)
+    for k, dt in FLEET_DTYPES.items():
+        assert fleet[k].dtype == dt and fleet[k].flags["C_CONTIGUOUS"] and fleet[k].shape == (wl.n_replicas,), k
+    fl = _Fleet(*[fleet[k].ctypes.data for k in FLEET_DTYPES])
+    dec = np.ascontiguousarray(decision, np.int32); used = np.ascontiguousarray(used_blocks, np.int64)
+    cold = np.ascontiguousarray(cold_start, np.int64)
+    assert dec.size == 6 and used.size == wl.n_replicas and cold.size == 3
+    cost = np.zeros(3, np.int64)
+    assert wl.now.dtype == np.int64 and wl.maturity.dtype == np.int64
+    L.ora_scale_apply(C.byref(ctx.cfg), int(now), dec.ctypes.data, used.ctypes.data, cold.ctypes.data, C.byref(fl),
+                      wl.now.ctypes.data, wl.maturity.ctypes.data, cost.ctypes.data)
+    return cost
 
 
 def scale_tick(wl, now: int, total_blocks: np.ndarray, **kw) -> Dict[str, np.ndarray]:

@@ -51,6 +51,7 @@ typedef struct {
   int32_t budget_mode;
   int32_t weight_max;
   int32_t first_fit;   /* admission variant, see step 6 */
+  int64_t horizon;     /* a committed step leaves a replica whose clock is past it untouched, see step 8 */
 } ora_config;
 
 typedef struct {
@@ -371,8 +372,13 @@ static int step_replica(const ora_config *c, const ora_table *t, int32_t r, int3
   /* 8. commit: the iteration happens.  Colocated: the new prefill batch runs
    *    first (prefill preempts ongoing decoding), then one decode iteration of
    *    the batch that was running. */
+  /*    reading (coupling replicas to a global clock): the events of the paper
+   *    happen in one global time; when a caller advances many replicas in
+   *    rounds, a replica whose own clock is already past the round's horizon
+   *    has nothing due yet and sits the commit out (its decisions are still
+   *    reported).  The horizon is "never" unless the caller sets one. */
   int result = CM_WORKED;
-  if (flags & FLAG_COMMIT) {
+  if ((flags & FLAG_COMMIT) && now <= c->horizon) {
     int worked;
     int64_t t1 = now, t2 = now;
     if (cfg->mode == MODE_COLOCATED) {
@@ -585,7 +591,10 @@ uint32_t ora_sim(const ora_config *c, const ora_table *t, const int32_t *trace_o
  * reading: waiting time is measured against the TTFT SLO, requests without one are left out of N;
  * each ratio waiting/SLO is taken in 16.16 fixed point (floor), saturated at 2^15; thresholds are
  * rationals num/den compared by cross-multiplication; an instance with total_blocks <= 0 is not
- * active; ties for the smallest f3 go to the lowest instance id. */
+ * active; ties for the smallest f3 go to the lowest instance id.
+ * reading: a QUEUED request with replica_id -1 waits in the global queue, bound to no instance yet; the
+ * global queue feeds the colocated instances and the P stage, so such a request counts as an arrival
+ * and as a waiting request for both of those pools (and holds no KV block anywhere). */
 typedef struct {
   int64_t window;
   int32_t block_tokens, min_samples;
@@ -607,6 +616,22 @@ uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const i
   const int64_t B = sp->block_tokens;
   for (int64_t i = 0; i < t->n; i++) {
     const int32_t r = t->replica_id[i];
+    if (r == -1 && t->state[i] == ST_QUEUED) {
+      /* still in the global queue: it feeds the colocated pool and the P stage, so it counts for both */
+      if (!row_valid(c, t, i, &status)) continue;
+      const ora_class *k = &c->classes[t->class_id[i]];
+      for (int pool = 0; pool < 2; pool++) {
+        int64_t *cnt = o->counts + 4 * pool;
+        if (t->arrival[i] > now - sp->window && t->arrival[i] <= now) cnt[0] += 1;
+        if (t->arrival[i] <= now && k->ttft > 0) {
+          i128 q = ((i128)(now - t->arrival[i]) << 16) / k->ttft;
+          if (q > ((i128)1 << 31)) q = (i128)1 << 31;
+          cnt[2] += 1;
+          cnt[3] += (int64_t)q;
+        }
+      }
+      continue;
+    }
     if (r < 0 || r >= R) { status |= BAD_REPLICA; continue; }
     if (!row_valid(c, t, i, &status)) continue;
     int64_t *cnt = o->counts + 4 * c->replicas[r].mode;
@@ -993,4 +1018,102 @@ uint32_t ora_attainment(const ora_config *c, const ora_table *t, int64_t *out) {
     for (int q = 0; q < 6; q++) { out[cl * 6 + q] += v[q]; out[K * 6 + q] += v[q]; }
   }
   return status;
+}
+
+/* ==========================================================================
+ * Carrying out the Scaler's decisions: the life of an instance and the cost of
+ * the fleet (Sec. 3.3.3 "Scaling Mechanism and Policy" for the decisions, the
+ * Problem Definition's Eq. 1 for the cost; the time to bring an instance up is
+ * a constant per pool, the quantity the paper's scaling-time table measures).
+ * An instance is OFF (0), STARTING (1: decided, not yet serving), ACTIVE (2)
+ * or DRAINING (3: chosen for removal, finishing what it holds).  At a tick at
+ * time `now`, in this order:
+ *   1. every instance that is not OFF is charged for (since, now];
+ *   2. a STARTING instance whose ready time has come turns ACTIVE: its clock
+ *      and its maturity (the per-instance arrays of the scheduling step) are
+ *      brought up to the ready time, it serves nothing earlier;
+ *   3. a DRAINING instance that holds no KV block any more turns OFF;
+ *   4. per pool, the decision of this tick: scale out -> the pool gets one
+ *      more instance; scale in -> the named instance starts DRAINING;
+ *   5. due[r], the maturity the dispatcher sees, is the instance's maturity
+ *      if it is ACTIVE and "never" otherwise (only ACTIVE instances are given
+ *      new requests); total_blocks (what the next tick reads) is the capacity
+ *      of an ACTIVE instance and 0 for every other one; cost[pool] = sum of
+ *      charged time.
+ * reading: Eq. 1's "active time" runs from the decision to start an instance
+ *   until it is turned off: starting up and draining hold the device too.
+ * reading: while an instance of the pool is STARTING a further scale-out does
+ *   nothing (the capacity already on its way is not ordered twice).  Otherwise
+ *   a DRAINING instance of the pool, lowest id first, is taken back into
+ *   service at once (no start-up), else the lowest-id OFF instance of the pool
+ *   starts and is ready at now + cold_start[pool]; with none left, nothing.
+ * reading: a scale-in that names an instance which is not ACTIVE, or of
+ *   another pool, does nothing.  Role switching between pools is not modelled.
+ * ========================================================================== */
+#define INST_OFF 0
+#define INST_STARTING 1
+#define INST_ACTIVE 2
+#define INST_DRAINING 3
+#define T_NEVER INT64_MAX
+
+typedef struct {
+  int32_t *inst_state;       /* [R] */
+  int64_t *ready;            /* [R] */
+  int64_t *billed;           /* [R] */
+  int64_t *since;            /* [R] */
+  int32_t *total_blocks;     /* [R] out */
+  int64_t *due;              /* [R] out */
+  const int32_t *blocks_cap; /* [R] */
+} ora_fleet;
+
+void ora_scale_apply(const ora_config *c, int64_t now, const int32_t *decision, const int64_t *used_blocks,
+                     const int64_t *cold_start, const ora_fleet *f, int64_t *clock, int64_t *maturity, int64_t *cost) {
+  const int32_t R = c->n_replicas;
+  for (int32_t r = 0; r < R; r++) {
+    if (f->inst_state[r] != INST_OFF && now > f->since[r]) { f->billed[r] += now - f->since[r]; f->since[r] = now; }
+    if (f->inst_state[r] == INST_STARTING && f->ready[r] <= now) {
+      f->inst_state[r] = INST_ACTIVE;
+      if (clock[r] < f->ready[r]) clock[r] = f->ready[r];
+      if (maturity[r] < f->ready[r]) maturity[r] = f->ready[r];
+    }
+    if (f->inst_state[r] == INST_DRAINING && used_blocks[r] == 0) f->inst_state[r] = INST_OFF;
+  }
+  for (int pool = 0; pool < 3; pool++) {
+    const int action = decision[2 * pool], victim = decision[2 * pool + 1];
+    if (action > 0) {
+      int32_t first[4] = {-1, -1, -1, -1};      /* lowest id of the pool in each state */
+      for (int32_t r = R - 1; r >= 0; r--)
+        if (c->replicas[r].mode == pool) first[f->inst_state[r]] = r;
+      if (first[INST_STARTING] >= 0) {
+        /* capacity is already on its way */
+      } else if (first[INST_DRAINING] >= 0) {
+        f->inst_state[first[INST_DRAINING]] = INST_ACTIVE;
+      } else if (first[INST_OFF] >= 0) {
+        const int32_t r = first[INST_OFF];
+        f->inst_state[r] = INST_STARTING; f->ready[r] = now + cold_start[pool]; f->since[r] = now;
+      }
+    } else if (action < 0 && victim >= 0 && victim < R && c->replicas[victim].mode == pool &&
+               f->inst_state[victim] == INST_ACTIVE) {
+      f->inst_state[victim] = INST_DRAINING;
+    }
+  }
+  cost[0] = cost[1] = cost[2] = 0;
+  for (int32_t r = 0; r < R; r++) {
+    const int on = f->inst_state[r] == INST_ACTIVE;
+    f->total_blocks[r] = on ? f->blocks_cap[r] : 0;
+    f->due[r] = on ? maturity[r] : T_NEVER;
+    cost[c->replicas[r].mode] += f->billed[r];
+  }
+}
+
+/* Binding what a dispatching call decided (Sec. 3.3.1, step "dispatch them"): each request the call
+ * assigned now belongs to its instance (replica_id), and an instance that was given requests cannot
+ * have started them before the call was made: its clock is brought up to `now` if it was behind
+ * (an idle instance's clock stands where its last iteration ended). */
+void ora_dispatch_bind(const ora_config *c, const ora_table *t, int64_t now, const int32_t *assign,
+                       const int32_t *adm_count, int32_t *replica_id, int64_t *clock) {
+  for (int64_t i = 0; i < t->n; i++)
+    if (assign[i] >= 0) replica_id[i] = assign[i];
+  for (int32_t r = 0; r < c->n_replicas; r++)
+    if (adm_count[r] > 0 && clock[r] < now) clock[r] = now;
 }

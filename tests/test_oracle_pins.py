@@ -508,3 +508,67 @@ def test_dispatch_serves_the_p_stage():
     assert list(o["budget"]) == [2144, 2144, 0] and list(o["e_d"]) == [0, 0, 0] and list(o["n_run"]) == [80, 0, 0]
     assert list(o["assign"][80:86]) == [1, 1, 0, 0, -1, -1] and list(o["adm_cost"]) == [297, 2144, 0]
     assert o["maturity_next"][0] - now == 17_056_418 and o["maturity_next"][2] == now - 100
+
+
+def test_scale_apply_hand_worked():
+    S = 1_000_000_000
+    rows = [dict(replica_id=0, prompt_len=1, output_len=1)]
+    wl = make_wl(rows, [(200 * MS, 30 * MS, 0)], replicas=[(gen.COLOCATED, 4096, 0)] * 4 + [(gen.PREFILL, 4096, 0)],
+                 now=[0] * 5, maturity=[0] * 5)
+    f = gen.new_fleet([100] * 5, [0, 1, 4])
+    NEVER = gen.T_NEVER
+    hold = [0, -1]
+
+    def tick(t, dec0, used, dec1=hold):
+        return oracle.scale_apply(wl, t * S, np.array([dec0, dec1, hold]), np.array(used), [2 * S, 5 * S, 7 * S], f)
+
+    cost = tick(10, [1, -1], [50, 20, 0, 0, 10])
+    assert list(f["inst_state"]) == [2, 2, 1, 0, 2] and f["ready"][2] == 12 * S and list(cost) == [20 * S, 10 * S, 0]
+    assert list(f["total_blocks"]) == [100, 100, 0, 0, 100] and list(f["due"]) == [0, 0, NEVER, NEVER, 0]
+    cost = tick(11, [1, -1], [50, 20, 0, 0, 10])
+    assert list(f["inst_state"]) == [2, 2, 1, 0, 2] and cost[0] == 23 * S
+    wl.maturity[0] = 14 * S                                              # instance 0 is busy until 14 s
+    cost = tick(13, hold, [50, 20, 0, 0, 10], dec1=[1, -1])
+    assert list(f["inst_state"]) == [2, 2, 2, 0, 2] and f["total_blocks"][2] == 100
+    assert list(f["due"]) == [14 * S, 0, 12 * S, NEVER, 0] and list(wl.now) == [0, 0, 12 * S, 0, 0] and wl.maturity[2] == 12 * S
+    assert cost[0] == PINS["fleet_cost_s_t13"] * S and cost[1] == 13 * S
+    cost = tick(20, [-1, 1], [50, 20, 5, 0, 10])
+    assert list(f["inst_state"]) == [2, 3, 2, 0, 2] and f["due"][1] == NEVER and f["total_blocks"][1] == 0 and cost[0] == 50 * S
+    cost = tick(21, hold, [50, 20, 5, 0, 10])
+    assert f["inst_state"][1] == 3 and cost[0] == 53 * S
+    wl.maturity[1] = 25 * S
+    cost = tick(22, [1, -1], [50, 7, 5, 0, 10])
+    assert list(f["inst_state"]) == [2, 2, 2, 0, 2] and f["due"][1] == 25 * S and cost[0] == PINS["fleet_cost_s_t22"] * S
+    cost = tick(30, [-1, 0], [9, 7, 5, 0, 10])
+    assert f["inst_state"][0] == 3 and cost[0] == 80 * S
+    cost = tick(31, hold, [0, 7, 5, 0, 10])
+    assert f["inst_state"][0] == 0 and f["due"][0] == NEVER and cost[0] == PINS["fleet_cost_s_t31"] * S
+    cost = tick(40, [1, -1], [0, 7, 5, 0, 10])
+    assert list(f["inst_state"]) == [1, 2, 2, 0, 2] and f["ready"][0] == 42 * S and f["billed"][0] == 31 * S and cost[0] == 101 * S
+    cost = tick(41, [-1, 0], [0, 7, 5, 0, 10], dec1=[-1, 0])          # the second names an instance of another pool
+    assert list(f["inst_state"]) == [1, 2, 2, 0, 2]
+    assert cost[0] == PINS["fleet_cost_s_t41"] * S and cost[1] == PINS["fleet_prefill_cost_s_t41"] * S and cost[2] == 0
+    assert list(f["billed"]) == [32 * S, 41 * S, 31 * S, 0, 41 * S]
+    # an instance whose clock is already past its ready time keeps it
+    wl.now[0] = 50 * S; wl.maturity[0] = 55 * S
+    tick(43, hold, [0, 7, 5, 0, 10])
+    assert f["inst_state"][0] == 2 and wl.now[0] == 50 * S and f["due"][0] == 55 * S
+
+
+def test_horizon_gate_and_binding():
+    # a replica whose clock is past the horizon reports its decisions and changes nothing
+    rows = [dict(replica_id=0, prompt_len=1000, output_len=3, arrival_ns=0), dict(replica_id=1, prompt_len=1000, output_len=3, arrival_ns=0)]
+    wl = make_wl(rows, [(200 * MS, 30 * MS, 0)], replicas=[(gen.COLOCATED, 32768, 0)] * 2, now=[10 * MS, 30 * MS], maturity=[0, 0])
+    wl.meta["horizon"] = 20 * MS
+    o = oracle.step(wl, commit=True)
+    assert list(o["admit"]) == [1, 1]
+    assert list(wl.table["state"]) == [gen.RUNNING, gen.QUEUED] and list(wl.now) == [10 * MS + PINS["pd_first_token"], 30 * MS]
+    assert wl.table["first_token_ns"][0] == 10 * MS + PINS["pd_first_token"] and wl.maturity[1] == 0
+    wl.meta["horizon"] = 30 * MS                      # a clock exactly at the horizon still acts
+    oracle.step(wl, commit=True)
+    assert wl.table["state"][1] == gen.RUNNING and wl.now[1] == 30 * MS + PINS["pd_first_token"]
+    # binding: the request moves to its instance, whose clock cannot stay behind the time of the call
+    wl = make_wl([dict(replica_id=-1, prompt_len=10, output_len=3), dict(replica_id=-1, prompt_len=10, output_len=3)],
+                 [(200 * MS, 30 * MS, 0)], replicas=[(gen.COLOCATED, 32768, 0)] * 3, now=[5, 500, 7], maturity=[0, 0, 0])
+    oracle.dispatch_bind(wl, 100, dict(assign=np.array([1, -1], np.int32), adm_count=np.array([1, 1, 0], np.int32)))
+    assert list(wl.table["replica_id"]) == [1, -1] and list(wl.now) == [100, 500, 7]

@@ -388,3 +388,40 @@ def test_first_fit_invariants_and_dominance(seed):
             assert bool(adm[k]) == bool(fits)
             if fits:
                 used += int(cost[k]); cnt += 1
+
+
+def test_scaling_loop_invariants():
+    # global queue -> dispatcher -> instances, with the Scaler switching instances on and off between ticks
+    from elastic_loop import oracle_round
+    R = 8
+    wl = gen.elastic(1, R, 1500)
+    f = gen.new_fleet([2000] * R, [0, 1])
+    on_max, on_later_min, prev_cost, seen = 2, R, 0, set()
+    for k in range(330):
+        before = f["inst_state"].copy()
+        o = oracle_round(wl, f, k)
+        st, d = f["inst_state"], o["dispatch"]
+        sel = d["assign"] >= 0
+        assert np.all(st[d["assign"][sel]] == gen.INST_ACTIVE)                   # only ACTIVE instances are given work
+        assert np.all(wl.now[np.unique(d["assign"][sel])] >= o["now"])           # and not before the call was made
+        assert np.count_nonzero(st == gen.INST_STARTING) <= 1                    # capacity is not ordered twice
+        assert np.array_equal(f["due"] == gen.T_NEVER, st != gen.INST_ACTIVE)
+        assert np.array_equal(f["total_blocks"], np.where(st == gen.INST_ACTIVE, 2000, 0))
+        assert o["cost"][0] == f["billed"].sum() and o["cost"][0] >= prev_cost and np.all(f["billed"] <= o["now"])
+        assert o["cost"][0] - prev_cost <= R * 50 * MS                            # at most every instance for one tick
+        for r in range(R):                                                        # the life cycle has no other edges
+            assert (before[r], st[r]) in {(0, 0), (0, 1), (1, 1), (1, 2), (2, 2), (2, 3), (3, 3), (3, 2), (3, 0)}, (k, r)
+            seen.add((before[r], st[r]))
+        off = np.flatnonzero(st == gen.INST_OFF)
+        assert not np.any(np.isin(wl.table["replica_id"], off) & np.isin(wl.table["state"], (gen.QUEUED, gen.RUNNING)))
+        prev_cost = o["cost"][0]
+        n_on = int(np.count_nonzero(st != gen.INST_OFF))
+        on_max = max(on_max, n_on)
+        if on_max >= 6:
+            on_later_min = min(on_later_min, n_on)
+    assert on_max >= 6 and on_later_min <= 3, (on_max, on_later_min)             # the fleet grew with the burst and shrank after it
+    assert {(0, 1), (1, 2), (2, 3), (3, 0)} <= seen
+    assert np.count_nonzero(wl.table["state"] == gen.DONE) > 700
+    # every instance's clock stays within one iteration of the global clock once it has work
+    busy = np.isin(np.arange(R), wl.table["replica_id"][wl.table["state"] == gen.RUNNING])
+    assert np.all(wl.now[busy] <= o["now"] + 1100 * MS)      # one iteration: a prefill batch up to the token cap, then a decode iteration
