@@ -287,6 +287,16 @@ typedef struct hfx_dispatch_out {
 int hfx_dispatch_step(hfx_sched *s, const hfx_table *table, int64_t now_ns,
                       const int64_t *maturity_ns, const hfx_dispatch_out *out);
 
+/* Binding what a dispatching call decided (Sec. 3.3.1, "dispatch them"): replica_id[i] = assign[i] for
+ * every request that hfx_dispatch_step assigned (out->assign, out->adm_count as it wrote them), and the
+ * clock now_ns[r] of an instance that was given requests is raised to now_ns if it was behind (an idle
+ * instance's clock stands where its last iteration ended; it cannot start the requests before the call
+ * that dispatched them).  replica_id must be table->replica_id (passed separately because the table
+ * is otherwise read-only here); device pointers; asynchronous on the scheduler's stream.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY, HFX_E_CUDA. */
+int hfx_dispatch_bind(hfx_sched *s, const hfx_table *table, int32_t *replica_id, int64_t now_ns,
+                      const hfx_dispatch_out *out, int64_t *clock_ns);
+
 /* Hand-off from the P stage to the D stage of the disaggregated mode
  * (Sec. 3.3.1 "Disaggregated Mode": the Dispatcher serves the P instances, the
  * Migrator the D instances over the queue of prefilled requests).  With
@@ -410,6 +420,46 @@ typedef struct hfx_scale_out {
 int hfx_scale_tick(hfx_sched *s, const hfx_table *table, int64_t now_ns, const int32_t *total_blocks,
                    const hfx_scale_params *params, const hfx_scale_out *out);
 
+/* Carrying out the decisions of a Scaler tick: the life of an instance and the cost of the fleet
+ * (Sec. 3.3.3 for the decisions, Eq. 1 of the Problem Definition for the cost; the time to bring an
+ * instance up is a constant per pool).  An instance is HFX_INST_OFF, STARTING (decided, not yet
+ * serving), ACTIVE or DRAINING (chosen for removal, finishing what it holds).  At time now_ns, in
+ * this order:
+ *   1. every instance that is not OFF is charged for (since_ns, now_ns];
+ *   2. a STARTING instance whose ready_ns has come turns ACTIVE; its clock and maturity in `state`
+ *      (the arrays hfx_sched_step works on) are raised to ready_ns: it serves nothing earlier;
+ *   3. a DRAINING instance with used_blocks == 0 turns OFF;
+ *   4. per pool (0 colocated, 1 prefill, 2 decode) the decision {action, instance}: scale out (+1)
+ *      does nothing while an instance of the pool is STARTING; else the lowest-id DRAINING instance
+ *      of the pool is taken back (ACTIVE at once); else the lowest-id OFF one turns STARTING with
+ *      ready_ns = now_ns + cold_start_ns[pool]; else nothing.  Scale in (-1) turns the named
+ *      instance DRAINING if it is ACTIVE and of this pool, and does nothing otherwise;
+ *   5. due_ns[r] = maturity of an ACTIVE instance, INT64_MAX for any other (the maturity array to
+ *      give hfx_dispatch_step: only ACTIVE instances receive requests); total_blocks[r] =
+ *      blocks_cap[r] if ACTIVE else 0 (the input of the next hfx_scale_tick); cost_ns[pool] = sum of
+ *      billed_ns, Eq. 1 up to the factor UnitCost.
+ * `decision` ([3][2]) and `used_blocks` ([n_replicas]) are what hfx_scale_tick wrote; all arrays are
+ * device pointers of n_replicas entries owned by the caller (cost_ns: 3), cold_start_ns is a HOST
+ * array of 3 values >= 0.  An inst_state outside 0..3 is read as OFF.  Role switching between pools
+ * is not modelled.  Asynchronous on the scheduler's stream.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CUDA. */
+#define HFX_INST_OFF 0
+#define HFX_INST_STARTING 1
+#define HFX_INST_ACTIVE 2
+#define HFX_INST_DRAINING 3
+typedef struct hfx_fleet {
+  int32_t *inst_state;        /* read and written */
+  int64_t *ready_ns;          /* written when an instance starts */
+  int64_t *billed_ns;         /* read and written: time charged so far */
+  int64_t *since_ns;          /* read and written: time up to which billed_ns is settled */
+  int32_t *total_blocks;      /* written */
+  int64_t *due_ns;            /* written */
+  const int32_t *blocks_cap;  /* KV blocks of the instance when it is on */
+} hfx_fleet;
+int hfx_scale_apply(hfx_sched *s, int64_t now_ns, const int32_t *decision, const int64_t *used_blocks,
+                    const int64_t *cold_start_ns, const hfx_fleet *fleet, const hfx_replica_state *state,
+                    int64_t *cost_ns);
+
 /* Synchronise the scheduler's stream and return the sticky status word
  * (HFX_ST_* bits) in *status_word (host pointer); the word is then cleared.
  * Returns HFX_E_TIMEOUT if HFX_ST_TIMEOUT was set, HFX_E_CUDA if the stream
@@ -425,8 +475,8 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * stream, adds the elapsed times of all brackets recorded since the last call
  * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
  * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
- * 6 oversize path, 7 simulator, 8 scaler tick, 9 fused front end, 10 the kernels of
- * hfx_dispatch_step together, 11 those of hfx_slo_map, 12 those of hfx_pd_migrate, 13
+ * 6 oversize path, 7 simulator, 8 scaler tick and hfx_scale_apply, 9 fused front end, 10 the kernels of
+ * hfx_dispatch_step and hfx_dispatch_bind together, 11 those of hfx_slo_map, 12 those of hfx_pd_migrate, 13
  * hfx_attainment; hfx_kernel_name gives the name of a slot (NULL past the end). */
 #define HFX_N_KERNELS 14
 typedef struct hfx_profile {
@@ -442,6 +492,13 @@ int hfx_sched_set_profiling(hfx_sched *s, int on);
  * to.  Results are identical either way.  Host call, takes effect at the next
  * hfx_sched_step.  The paper has no counterpart (an execution switch). */
 int hfx_sched_set_fused_front(hfx_sched *s, int on);
+/* Commit horizon, for callers that advance many instances in rounds of one global clock (the events of
+ * the Problem Definition happen in one global time): in the following steps with HFX_COMMIT an
+ * instance whose clock now_ns[r] is past horizon_ns has nothing due yet and sits the commit out --
+ * its decisions are reported as usual, its rows, clock and maturity stay as they are.  A clock equal
+ * to the horizon still acts.  The default, INT64_MAX, gates nothing.  Host call, takes effect at the
+ * next hfx_sched_step; the simulator is not affected. */
+int hfx_sched_set_horizon(hfx_sched *s, int64_t horizon_ns);
 int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out);
 const char *hfx_kernel_name(int slot);
 

@@ -21,7 +21,8 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
-                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map", "hfx_pd_migrate", "hfx_attainment"]
+                    "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map", "hfx_pd_migrate", "hfx_attainment",
+                    "hfx_sched_set_horizon", "hfx_scale_apply", "hfx_dispatch_bind"]
 NOALLOC_MAX_REPLICAS = 4096
 N_KERNELS = 14
 
@@ -160,6 +161,13 @@ def load_library():
     L.hfx_sched_destroy.argtypes = [C.c_void_p]
     L.hfx_sched_set_profiling.restype = C.c_int
     L.hfx_sched_set_profiling.argtypes = [C.c_void_p, C.c_int]
+    L.hfx_sched_set_horizon.restype = C.c_int
+    L.hfx_sched_set_horizon.argtypes = [C.c_void_p, C.c_int64]
+    L.hfx_scale_apply.restype = C.c_int
+    L.hfx_scale_apply.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(C.c_int64), C.POINTER(_Fleet),
+                                  C.POINTER(_ReplicaState), C.c_void_p]
+    L.hfx_dispatch_bind.restype = C.c_int
+    L.hfx_dispatch_bind.argtypes = [C.c_void_p, C.POINTER(_Table), C.c_void_p, C.c_int64, C.POINTER(_DispatchOut), C.c_void_p]
     L.hfx_sched_set_fused_front.restype = C.c_int
     L.hfx_sched_set_fused_front.argtypes = [C.c_void_p, C.c_int]
     L.hfx_sched_get_profile.restype = C.c_int
@@ -255,6 +263,28 @@ class StepOut:
         return out
 
 
+FLEET_FIELDS = [("inst_state", torch.int32), ("ready", torch.int64), ("billed", torch.int64), ("since", torch.int64),
+                ("total_blocks", torch.int32), ("due", torch.int64), ("blocks_cap", torch.int32)]
+INST_OFF, INST_STARTING, INST_ACTIVE, INST_DRAINING = 0, 1, 2, 3
+
+
+class _Fleet(C.Structure):
+    _fields_ = [(k, C.c_void_p) for k in ("inst_state", "ready_ns", "billed_ns", "since_ns", "total_blocks", "due_ns", "blocks_cap")]
+
+
+class Fleet:
+    """Instance records of hfx_scale_apply on the device (fields as FLEET_FIELDS, one entry per instance)."""
+
+    def __init__(self, arrays: Dict[str, np.ndarray], device="cuda"):
+        self.t = {k: torch.from_numpy(np.ascontiguousarray(arrays[k])).to(dtype=dt, device=device) for k, dt in FLEET_FIELDS}
+
+    def c_struct(self) -> _Fleet:
+        return _Fleet(*[_ptr(self.t[k]) for k, _ in FLEET_FIELDS])
+
+    def to_numpy(self) -> Dict[str, np.ndarray]:
+        return {k: v.cpu().numpy() for k, v in self.t.items()}
+
+
 class DispatchOut:
     """Output buffers of hfx_dispatch_step (allocated once, reused)."""
 
@@ -344,6 +374,29 @@ class Scheduler:
         rc = self._L.hfx_dispatch_step(self._h, C.byref(ts), int(now_ns), _ptr(maturity), C.byref(os_))
         if rc != 0:
             raise HfxError(rc, "hfx_dispatch_step")
+
+    def dispatch_bind(self, table: DeviceTable, now_ns: int, out: DispatchOut, now: torch.Tensor):
+        """hfx_dispatch_bind: bind what dispatch_step assigned (table.replica_id, the instance clocks `now`)."""
+        ts, os_ = table.c_struct(), out.c_struct()
+        rc = self._L.hfx_dispatch_bind(self._h, C.byref(ts), _ptr(table.cols["replica_id"]), int(now_ns), C.byref(os_), _ptr(now))
+        if rc != 0:
+            raise HfxError(rc, "hfx_dispatch_bind")
+
+    def scale_apply(self, now_ns: int, decision: torch.Tensor, used_blocks: torch.Tensor, cold_start_ns, fleet: "Fleet",
+                    now: torch.Tensor, maturity: torch.Tensor, cost: torch.Tensor):
+        """hfx_scale_apply: carry out one tick's decisions on `fleet`; cost int64 [3] on the device."""
+        cold = (C.c_int64 * 3)(*[int(x) for x in cold_start_ns])
+        fs = fleet.c_struct()
+        st = _ReplicaState(_ptr(now), _ptr(maturity))
+        rc = self._L.hfx_scale_apply(self._h, int(now_ns), _ptr(decision), _ptr(used_blocks), cold, C.byref(fs), C.byref(st), _ptr(cost))
+        if rc != 0:
+            raise HfxError(rc, "hfx_scale_apply")
+
+    def set_horizon(self, horizon_ns: Optional[int]):
+        """hfx_sched_set_horizon (None: no horizon)."""
+        rc = self._L.hfx_sched_set_horizon(self._h, int(np.iinfo(np.int64).max if horizon_ns is None else horizon_ns))
+        if rc != 0:
+            raise HfxError(rc, "hfx_sched_set_horizon")
 
     def pd_migrate(self, table: DeviceTable, now: torch.Tensor, maturity: torch.Tensor, pair: torch.Tensor,
                    xfer_c0_ns: int, xfer_c1_ns: int, n_moved: Optional[torch.Tensor] = None):

@@ -121,6 +121,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   ok = ok && cudaMalloc(&s->d_front_bar, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_slo, hfx_slomap_workspace_bytes()) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_pd, hfx_pd_workspace_bytes(n_replicas)) == cudaSuccess;
+  s->horizon = INT64_MAX;
   s->front_enabled = 1; s->front_arrivals = 0; s->front_smem_cached = 0; s->front_capacity = 0;
   ok = ok && cudaMalloc(&h->d_trace_off, sizeof(int32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&h->d_work_counter, 256) == cudaSuccess;
@@ -332,6 +333,33 @@ extern "C" int hfx_sched_set_fused_front(hfx_sched *s, int on) {
   if (!s) return HFX_E_ARG;
   s->front_enabled = on ? 1 : 0;
   return HFX_OK;
+}
+
+extern "C" int hfx_sched_set_horizon(hfx_sched *s, int64_t horizon_ns) {
+  if (!s) return HFX_E_ARG;
+  s->horizon = horizon_ns;
+  return HFX_OK;
+}
+
+extern "C" int hfx_scale_apply(hfx_sched *s, int64_t now_ns, const int32_t *decision, const int64_t *used_blocks,
+                               const int64_t *cold_start_ns, const hfx_fleet *f, const hfx_replica_state *st, int64_t *cost_ns) {
+  if (!s || !decision || !used_blocks || !cold_start_ns || !f || !st || !st->now_ns || !st->maturity_ns || !cost_ns) return HFX_E_ARG;
+  if (!f->inst_state || !f->ready_ns || !f->billed_ns || !f->since_ns || !f->total_blocks || !f->due_ns || !f->blocks_cap) return HFX_E_ARG;
+  for (int q = 0; q < 3; q++) if (cold_start_ns[q] < 0 || cold_start_ns[q] > (INT64_C(1) << 50)) return HFX_E_ARG;
+  const void *all[] = {decision, used_blocks, f->inst_state, f->ready_ns, f->billed_ns, f->since_ns, f->total_blocks, f->due_ns,
+                       f->blocks_cap, st->now_ns, st->maturity_ns, cost_ns};
+  for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
+  return hfx_launch_fleet_apply(s, now_ns, decision, used_blocks, cold_start_ns, f, st->now_ns, st->maturity_ns, cost_ns);
+}
+
+extern "C" int hfx_dispatch_bind(hfx_sched *s, const hfx_table *t, int32_t *replica_id, int64_t now_ns,
+                                 const hfx_dispatch_out *o, int64_t *clock_ns) {
+  if (!s || !t || !o || !o->assign || !o->adm_count || !clock_ns || t->n_rows < 0) return HFX_E_ARG;
+  if (t->n_rows > s->max_rows) return HFX_E_CAPACITY;
+  if (t->n_rows > 0 && (!replica_id || replica_id != t->replica_id)) return HFX_E_ARG;
+  const void *all[] = {replica_id, o->assign, o->adm_count, clock_ns};
+  for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
+  return hfx_launch_dispatch_bind(s, t->n_rows, now_ns, o->assign, o->adm_count, replica_id, clock_ns);
 }
 
 extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {

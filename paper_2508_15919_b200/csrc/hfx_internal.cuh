@@ -103,6 +103,7 @@ struct hfx_sched {
   // fused front end (count + column scan + offsets + regroup as one cooperative kernel)
   unsigned long long *d_front_bar;     // arrivals at its grid barriers, only ever grows
   unsigned long long front_arrivals;   // host copy of what that word holds once every launch so far is done
+  int64_t horizon;          // commit horizon of the following steps (INT64_MAX: none)
   int front_enabled;
   size_t front_smem_cached;            // shared-memory size the capacity below was asked for
   int front_capacity;                  // blocks of the fused kernel that can be resident at once
@@ -529,6 +530,7 @@ struct SegArgs {
   int64_t *budget; int64_t *e_d; int32_t *n_run; int64_t *sum_kv; int64_t *adm_cost; int32_t *adm_count;
   int64_t *maturity_next;
   uint32_t flags;
+  int64_t horizon;           // a replica whose clock is past it sits the commit out
 };
 
 // host-side launchers implemented in the .cu files
@@ -547,5 +549,9 @@ int hfx_launch_pd_migrate(hfx_sched *s, const hfx_table *t, int32_t *replica_id,
                           int64_t x1, int32_t *n_moved);
 size_t hfx_pd_workspace_bytes(int n_replicas);
 int hfx_launch_attainment(hfx_sched *s, const hfx_table *t, int64_t *out);
+int hfx_launch_fleet_apply(hfx_sched *s, int64_t now, const int32_t *decision, const int64_t *used_blocks,
+                           const int64_t *cold, const hfx_fleet *f, int64_t *clock, int64_t *maturity, int64_t *cost);
+int hfx_launch_dispatch_bind(hfx_sched *s, int64_t n, int64_t now, const int32_t *assign, const int32_t *adm_count,
+                             int32_t *replica_id, int64_t *clock);
 int hfx_launch_sim(hfx_sched *s, const hfx_table *t, const int32_t *trace_off, int32_t n_traces, int32_t iters,
                    const hfx_sim_out *o);

@@ -51,11 +51,23 @@ __global__ void __launch_bounds__(SCALE_THREADS) k_scale(const HfxParams p, cons
   for (int k = 0; k < 12; k++) cnt[k] = 0;
 
   auto row = [&](int32_t rid, uint32_t cls, uint32_t st, int32_t prompt, int32_t gen, int64_t arrival, int64_t finish) {
-    if (rid < 0 || rid >= R) { bad |= HFX_ST_BAD_REPLICA; return; }
+    const bool unbound = rid == -1 && st == HFX_QUEUED;     // still in the global queue
+    if (!unbound && (rid < 0 || rid >= R)) { bad |= HFX_ST_BAD_REPLICA; return; }
     bool ok = true;
     if (cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
     if (prompt < 0 || prompt > HFX_MAX_TOKENS || gen < 0 || gen > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }
     if (!ok) return;
+    if (unbound) {
+      // the global queue feeds the colocated pool and the P stage: the request counts for both, holds no block
+      const unsigned long long c0 = arrival > lo_t && arrival <= now ? 1 : 0;
+      const int64_t ttft = s_ttft[cls];
+      const bool waits = arrival <= now && ttft > 0;
+      const unsigned long long c3 = waits ? ratio_q16(now - arrival, ttft) : 0;
+      cnt[0] += c0; cnt[4] += c0;
+      cnt[2] += waits; cnt[6] += waits;
+      cnt[3] += c3; cnt[7] += c3;
+      return;
+    }
     const int pool = __ldg(a.mode + rid);
     unsigned long long c0 = 0, c1 = 0, c2 = 0, c3 = 0;
     if (arrival > lo_t && arrival <= now) c0 = 1;

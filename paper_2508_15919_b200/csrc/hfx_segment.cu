@@ -136,7 +136,7 @@ __device__ __forceinline__ void write_replica_outputs(const SegArgs &a, int r, c
   a.adm_cost[r] = adm_cost;
   a.adm_count[r] = adm_count;
   a.maturity_next[r] = mat_next;
-  if (a.flags & HFX_COMMIT) {
+  if ((a.flags & HFX_COMMIT) && pl.now <= a.horizon) {
     int64_t now_next = pl.now;
     if (worked) now_next = t2;
     else {   // idle: jump to the next event, if any
@@ -408,7 +408,7 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
       sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
     }
     __syncthreads();
-    const bool commit = real && (a.flags & HFX_COMMIT);
+    const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
     const int worked = sh.worked;
     const int64_t mat_next = sh.red_c[0];
     if (commit && !worked && ordered) {
@@ -702,7 +702,7 @@ __global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_s
       sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
     }
     __syncthreads();
-    const bool commit = real && (a.flags & HFX_COMMIT);
+    const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
     const int worked = sh.worked;
     const int64_t mat_next = sh.red_c[0];
     if (commit && !worked && ordered) {
@@ -947,7 +947,7 @@ __global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a,
     {
       const int64_t t1 = mail[0], t2 = mail[1];
       const int worked = (int)mail[2], adm_count = (int)mail[3];
-      const bool commit = real && (a.flags & HFX_COMMIT);
+      const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
       if (a.admitted_rows)
         for (int64_t q = adm_count + gtid; q < n; q += gsize) a.admitted_rows[b + q] = -1;
       if (commit)

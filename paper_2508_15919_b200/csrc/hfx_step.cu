@@ -45,7 +45,7 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
   sa.slack = o->slack_ns; sa.pred_tpot = o->pred_tpot_ns; sa.key = o->key; sa.order = o->order; sa.admit = o->admit;
   sa.admitted_rows = o->admitted_rows; sa.budget = o->budget; sa.e_d = o->e_d_ns; sa.n_run = o->n_run;
   sa.sum_kv = o->sum_kv; sa.adm_cost = o->adm_cost; sa.adm_count = o->adm_count; sa.maturity_next = o->maturity_next;
-  sa.flags = flags;
+  sa.flags = flags; sa.horizon = s->horizon;
   rc = hfx_launch_segments(s, sa, t->n_rows);
   s->step_parity ^= 1u;
   if (rc != HFX_OK) return rc;

@@ -26,6 +26,7 @@ def assert_step_parity(wl, steps=1, commit=False, optional=True, sched=None):
     cpu = wl.copy()
     own = sched is None
     sched = sched or make_sched(wl)
+    sched.set_horizon(wl.meta.get("horizon"))
     tab = hfx.DeviceTable.from_numpy(wl.table)
     now = torch.from_numpy(wl.now.copy()).cuda()
     mat = torch.from_numpy(wl.maturity.copy()).cuda()

@@ -368,6 +368,11 @@ def test_scaler_tick_parity():
     _scale_parity(wl, int(wl.now.max()), np.full(9000, 5), window=2 * SEC)
     wl = gen.random_table(7, 0, 3)
     _scale_parity(wl, 5, np.full(3, 5))
+    # requests still in the global queue (QUEUED, bound to no instance) count for the colocated pool and the P stage
+    wl = gen.random_table(8, 30_001, 12, modes=MODES3, future=0.1, done=0.3)
+    wl.table["replica_id"][::3] = -1
+    c = _scale_parity(wl, int(wl.now.max()), np.full(12, 500), window=2 * SEC, min_samples=1)
+    assert c["counts"][0][2] > 1000 and c["counts"][1][2] > 1000 and c["status"] != 0
 
 
 # ---- dispatching over the shared global queue -------------------------------------------------------
@@ -688,3 +693,158 @@ def test_disaggregated_pipeline_dispatch_step_handoff():
         assert np.array_equal(now.cpu().numpy(), cpu.now) and np.array_equal(mat.cpu().numpy(), cpu.maturity), k
     sched.close()
     assert bound > 50 and np.count_nonzero((cpu.table["state"] == 2) & (cpu.table["replica_id"] >= pairs)) > 0
+
+
+# ---- rounds on a global clock: commit horizon, binding, the Scaler's decisions carried out -----------------
+def test_commit_horizon_all_segment_sizes():
+    # replicas whose clock is past the horizon report their decisions and change nothing; small, medium and
+    # oversize segments, all three modes, both front ends
+    for seed, n, R, kw in ((1, 6000, 37, dict(modes=MODES3)), (2, 30_000, 4, dict(modes=MODES3, grouped=True)),
+                           (3, 16384 + 16385 + 3000, 3, dict(grouped=True, modes=MODES3))):
+        wl = gen.random_table(seed, n, R, **kw)
+        wl.now[::2] += 20 * MS
+        wl.meta["horizon"] = int(wl.now.min()) + 10 * MS
+        assert np.any(wl.now > wl.meta["horizon"]) and np.any(wl.now <= wl.meta["horizon"])
+        assert_step_parity(wl, steps=3, commit=True)
+    wl = gen.config2(R=16, rows_per=700)
+    wl.now[::3] += 5 * SEC
+    wl.meta["horizon"] = int(wl.now.min()) + SEC
+    assert_step_parity(wl, steps=2, commit=True)
+    wl.meta["horizon"] = -1                       # nobody acts
+    assert_step_parity(wl, steps=1, commit=True)
+
+
+def test_dispatch_bind_parity_and_errors():
+    import paper_2508_15919_b200 as hfx
+    wl = _colocated(gen.random_table(4, 5000, 9, modes=(gen.COLOCATED,)))
+    wl.table["replica_id"][wl.table["state"] == gen.QUEUED] = -1
+    now_g = int(wl.now.max())
+    wl.now[::2] -= 3 * SEC                         # clocks behind the call are raised, the others stay
+    cpu = wl.copy()
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    now = torch.from_numpy(wl.now.copy()).cuda(); mat = torch.from_numpy(wl.maturity.copy()).cuda()
+    dout = hfx.DispatchOut(wl.n_rows, wl.n_replicas)
+    sched.dispatch_step(tab, now_g, mat, dout)
+    d = oracle.dispatch(cpu, now_g)
+    assert np.array_equal(dout.to_numpy()["assign"], d["assign"]) and (d["assign"] >= 0).sum() > 5
+    sched.dispatch_bind(tab, now_g, dout, now)
+    oracle.dispatch_bind(cpu, now_g, d)
+    assert np.array_equal(tab.to_numpy()["replica_id"], cpu.table["replica_id"]) and np.array_equal(now.cpu().numpy(), cpu.now)
+    assert np.any(cpu.now != wl.now)
+    import ctypes as C
+    other = hfx.DeviceTable.from_numpy(wl.table)   # replica_id must be the table's own column
+    ts, os_ = tab.c_struct(), dout.c_struct()
+    assert sched._L.hfx_dispatch_bind(sched._h, C.byref(ts), other.cols["replica_id"].data_ptr(), now_g, C.byref(os_), now.data_ptr()) != 0
+    assert sched._L.hfx_dispatch_bind(sched._h, C.byref(ts), tab.cols["replica_id"].data_ptr(), now_g, C.byref(os_), None) != 0
+    sched.close()
+
+
+def _fleet_parity(seed, R, modes, rounds=6):
+    import paper_2508_15919_b200 as hfx
+    rng = np.random.default_rng(seed)
+    wl = gen.random_table(seed, 10, R, modes=modes)
+    cpu = wl.copy()
+    f = gen.new_fleet(rng.integers(1, 4000, R), rng.choice(R, max(1, R // 3), replace=False))
+    f["inst_state"][:] = rng.integers(0, 4, R)                # every state from the start
+    f["ready"][:] = rng.integers(0, 3 * SEC, R); f["since"][:] = rng.integers(0, SEC, R); f["billed"][:] = rng.integers(0, SEC, R)
+    sched = make_sched(wl)
+    fl = hfx.Fleet(f)
+    now = torch.from_numpy(wl.now.copy()).cuda(); mat = torch.from_numpy(wl.maturity.copy()).cuda()
+    cost = torch.full((3,), -1, dtype=torch.int64, device="cuda")
+    cold = [300 * MS, 2 * SEC, 0]
+    t = 0
+    for k in range(rounds):
+        t += int(rng.integers(0, SEC))
+        dec = np.stack([rng.integers(-1, 2, 3), rng.integers(-2, R + 2, 3)], axis=1).astype(np.int32)
+        used = (rng.integers(0, 50, R) * rng.integers(0, 2, R)).astype(np.int64)
+        sched.scale_apply(t, torch.from_numpy(dec).cuda(), torch.from_numpy(used).cuda(), cold, fl, now, mat, cost)
+        c = oracle.scale_apply(cpu, t, dec, used, cold, f)
+        g = fl.to_numpy()
+        for key in f:
+            assert np.array_equal(g[key], f[key]), (seed, k, key, np.flatnonzero(g[key] != f[key])[:8])
+        assert np.array_equal(cost.cpu().numpy(), c), (k, cost.cpu().numpy(), c)
+        assert np.array_equal(now.cpu().numpy(), cpu.now) and np.array_equal(mat.cpu().numpy(), cpu.maturity)
+    assert sched.status() == 0
+    sched.close()
+    return f
+
+
+def test_scale_apply_parity():
+    _fleet_parity(0, 1, (gen.COLOCATED,))
+    _fleet_parity(1, 7, (gen.COLOCATED,), rounds=20)
+    _fleet_parity(2, 40, MODES3, rounds=20)
+    _fleet_parity(3, 1025, MODES3)                # more instances than the block has threads
+    _fleet_parity(4, 5000, MODES3)
+
+
+def test_scale_apply_hand_worked_sequence():
+    # the hand-worked sequence of the pin file (costs 29, 56, 83, 104 instance-seconds) through the library
+    import paper_2508_15919_b200 as hfx
+    S = SEC
+    wl = gen.random_table(0, 4, 5, modes=(gen.COLOCATED,))
+    wl.replicas[4, 0] = gen.PREFILL
+    wl.now[:] = 0; wl.maturity[:] = 0
+    sched = make_sched(wl)
+    fl = hfx.Fleet(gen.new_fleet([100] * 5, [0, 1, 4]))
+    now = torch.zeros(5, dtype=torch.int64, device="cuda"); mat = torch.zeros(5, dtype=torch.int64, device="cuda")
+    cost = torch.zeros(3, dtype=torch.int64, device="cuda")
+    hold = [0, -1]
+    seq = [(10, [1, -1], hold, [50, 20, 0, 0, 10]), (11, [1, -1], hold, [50, 20, 0, 0, 10]), (13, hold, [1, -1], [50, 20, 0, 0, 10]),
+           (20, [-1, 1], hold, [50, 20, 5, 0, 10]), (21, hold, hold, [50, 20, 5, 0, 10]), (22, [1, -1], hold, [50, 7, 5, 0, 10]),
+           (30, [-1, 0], hold, [9, 7, 5, 0, 10]), (31, hold, hold, [0, 7, 5, 0, 10]), (40, [1, -1], hold, [0, 7, 5, 0, 10]),
+           (41, [-1, 0], [-1, 0], [0, 7, 5, 0, 10])]
+    costs = {}
+    for t, d0, d1, used in seq:
+        sched.scale_apply(t * S, torch.tensor([d0, d1, hold], dtype=torch.int32, device="cuda"),
+                          torch.tensor(used, dtype=torch.int64, device="cuda"), [2 * S, 5 * S, 7 * S], fl, now, mat, cost)
+        costs[t] = cost.cpu().numpy().copy()
+    assert [int(costs[t][0]) // S for t in (13, 22, 31, 41)] == [29, 56, 83, 104] and int(costs[41][1]) == 41 * S
+    g = fl.to_numpy()
+    assert list(g["inst_state"]) == [1, 2, 2, 0, 2] and list(g["billed"]) == [32 * S, 41 * S, 31 * S, 0, 41 * S]
+    assert now.cpu().numpy()[2] == 12 * S
+    sched.close()
+
+
+def test_scaling_loop_round_by_round():
+    # the whole loop: instances advance to the tick under the horizon, the Scaler ticks, its decisions are carried
+    # out, the dispatcher serves the ACTIVE instances that are due, the requests are bound -- compared after each round
+    import paper_2508_15919_b200 as hfx
+    from elastic_loop import COLD, SCALE_KW, SUBSTEPS, oracle_round
+    R = 8
+    wl = gen.elastic(1, R, 1500)
+    cpu = wl.copy()
+    f = gen.new_fleet([2000] * R, [0, 1])
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    fl = hfx.Fleet(f)
+    now = torch.from_numpy(wl.now.copy()).cuda(); mat = torch.from_numpy(wl.maturity.copy()).cuda()
+    sout = hfx.StepOut(wl.n_rows, R, optional=False)
+    dout = hfx.DispatchOut(wl.n_rows, R)
+    counts = torch.zeros((3, 4), dtype=torch.int64, device="cuda"); used = torch.zeros(R, dtype=torch.int64, device="cuda")
+    dec = torch.zeros((3, 2), dtype=torch.int32, device="cuda"); cost = torch.zeros(3, dtype=torch.int64, device="cuda")
+    on_max = 0
+    for k in range(330):
+        o = oracle_round(cpu, f, k)
+        sched.set_horizon(o["now"])
+        for _ in range(SUBSTEPS):
+            sched.step(tab, now, mat, sout, commit=True)
+        sched.scale_tick(tab, o["now"], fl.t["total_blocks"], counts, used, dec, window_ns=SCALE_KW["window"],
+                         min_samples=SCALE_KW["min_samples"])
+        sched.scale_apply(o["now"], dec, used, COLD, fl, now, mat, cost)
+        sched.dispatch_step(tab, o["now"], fl.t["due"], dout)
+        sched.dispatch_bind(tab, o["now"], dout, now)
+        assert sched.status() == o["status"], k
+        assert np.array_equal(counts.cpu().numpy(), o["tick"]["counts"]) and np.array_equal(dec.cpu().numpy(), o["tick"]["decision"]), k
+        assert np.array_equal(dout.to_numpy()["assign"], o["dispatch"]["assign"]), k
+        g = fl.to_numpy()
+        for key in f:
+            assert np.array_equal(g[key], f[key]), (k, key)
+        assert np.array_equal(cost.cpu().numpy(), o["cost"]), k
+        tg = tab.to_numpy()
+        for col in ("replica_id", "state", "gen", "first_token_ns", "last_token_ns", "finish_ns"):
+            assert np.array_equal(tg[col], cpu.table[col]), f"round {k}: column {col}"
+        assert np.array_equal(now.cpu().numpy(), cpu.now) and np.array_equal(mat.cpu().numpy(), cpu.maturity), k
+        on_max = max(on_max, int(np.count_nonzero(f["inst_state"] != gen.INST_OFF)))
+    sched.close()
+    assert on_max >= 6 and np.count_nonzero(cpu.table["state"] == gen.DONE) > 700
