@@ -348,6 +348,53 @@ def run_gpu(args):
               "requests_finished": int(att_tot[1]), "requests_attained": int(att_tot[2]), "status": psched.status()}
         psched.close()
 
+    # ---- the scaling loop: global queue, dispatcher, instances under a horizon, Scaler tick and its decisions ----
+    elastic = None
+    if rank == 0 and not args.no_elastic:
+        ER, EN, TICK, SUB = 1024, 1 << 20, 50_000_000, 6
+        ew = gen.elastic(11, ER, EN, rates=(2000.0, 30000.0))
+        esched = hfx.Scheduler(ew.model, ew.classes, ew.replicas, ew.n_rows)
+        etab = hfx.DeviceTable.from_numpy(ew.table)
+        efl = hfx.Fleet(gen.new_fleet([4096] * ER, range(64)))
+        enow = torch.from_numpy(ew.now.copy()).cuda(); emat = torch.from_numpy(ew.maturity.copy()).cuda()
+        eout = hfx.StepOut(EN, ER, optional=False); edout = hfx.DispatchOut(EN, ER)
+        ecnt = torch.zeros((3, 4), dtype=torch.int64, device="cuda"); eused = torch.zeros(ER, dtype=torch.int64, device="cuda")
+        edec = torch.zeros((3, 2), dtype=torch.int32, device="cuda"); ecost = torch.zeros(3, dtype=torch.int64, device="cuda")
+        cold = [300_000_000] * 3
+        rounds_w, rounds_t = 20, 60
+        evs, on_max = [], 0
+        for k in range(rounds_w + rounds_t):
+            now_g = (k + 1) * TICK
+            flush.fill_(7)
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            esched.set_horizon(now_g)
+            e[0].record(stream)
+            for _ in range(SUB):
+                esched.step(etab, enow, emat, eout, commit=True)
+            e[1].record(stream)
+            esched.scale_tick(etab, now_g, efl.t["total_blocks"], ecnt, eused, edec, window_ns=2_000_000_000)
+            esched.scale_apply(now_g, edec, eused, cold, efl, enow, emat, ecost)
+            e[2].record(stream)
+            esched.dispatch_step(etab, now_g, efl.t["due"], edout)
+            esched.dispatch_bind(etab, now_g, edout, enow)
+            e[3].record(stream)
+            if k >= rounds_w:
+                evs.append(e)
+            if k % 10 == 9:
+                on_max = max(on_max, int((efl.t["inst_state"] != 0).sum().item()))
+        torch.cuda.synchronize()
+        seg = [float(np.mean([e[i].elapsed_time(e[i + 1]) for e in evs])) for i in range(3)]
+        est = etab.to_numpy()
+        elastic = {"workload": "up to %d colocated instances (64 on at the start), %d requests in one global queue, %d rounds of a %d ms "
+                               "tick: %d committed steps under the horizon, Scaler tick + its decisions, dispatch + binding"
+                               % (ER, EN, rounds_w + rounds_t, TICK // 1_000_000, SUB),
+                   "steps_ms": seg[0], "scaler_ms": seg[1], "dispatch_ms": seg[2], "rounds_per_sec": 1e3 / sum(seg),
+                   "instances_on_max": on_max, "instances_on_end": int((efl.t["inst_state"] != 0).sum().item()),
+                   "cost_instance_seconds": float(ecost.cpu().numpy()[0]) / 1e9,
+                   "requests_bound": int(np.count_nonzero(est["replica_id"] >= 0)),
+                   "requests_finished": int(np.count_nonzero(est["state"] == gen.DONE)), "status": esched.status()}
+        esched.close()
+
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only -----------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -396,7 +443,7 @@ def run_gpu(args):
                 "clocks": clk, "gpu_launches": launches, "device_status": status,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms_max},
-                "roofline": roof, "cpu_baseline": cpu, "sim": sim, "dispatch": disp, "pd": pd}
+                "roofline": roof, "cpu_baseline": cpu, "sim": sim, "dispatch": disp, "pd": pd, "elastic": elastic}
         print(json.dumps(line))
     sched.close()
     if world > 1:
@@ -417,6 +464,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-dispatch", action="store_true")
     ap.add_argument("--no-pd", action="store_true")
+    ap.add_argument("--no-elastic", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

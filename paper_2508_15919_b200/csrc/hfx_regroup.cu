@@ -122,7 +122,7 @@ __device__ __forceinline__ void count_tile(const HfxParams &p, const CountArgs &
   for (int i = threadIdx.x; i < 2 * R1; i += blockDim.x) {
     const uint32_t c = s_hist[i];
     row[i] = c;
-    if (i < R1) mx = c > mx ? c : mx;
+    if (i < R) mx = c > mx ? c : mx;      // rows bound to no replica are ranked by a scan, whatever their number
   }
   const int small_groups = __syncthreads_and(mx <= GROUP_MAX);
   if (threadIdx.x == 0) {
@@ -474,6 +474,7 @@ __device__ __forceinline__ void regroup_tile(const HfxParams &p, const RegroupAr
   const int64_t v0 = lo >> 2;
   const size_t mrow = (size_t)blockIdx.x * 2 * R1;
 
+  bool tail_scan = false;
   if (mode != TILE_ANY) {
     // ---- A: histogram of the tile; active flag of every position ------------------------------------
     for (int v = tid; v < nvec; v += blockDim.x) {
@@ -512,8 +513,8 @@ __device__ __forceinline__ void regroup_tile(const HfxParams &p, const RegroupAr
       if (tid == 0) s_off[R1] = (uint32_t)nt;
     }
     __syncthreads();
-    if (mode == TILE_SORTED) {
-      // ---- C0: s_P := number of active rows before each position (exclusive scan, in place) -----------
+    // exclusive scan of s_P[0 .. nt) in place, the total in s_P[nt]
+    auto scan_P = [&]() {
       const int per = (nt + blockDim.x - 1) / blockDim.x;
       const int i0 = tid * per < nt ? tid * per : nt, i1 = (i0 + per < nt) ? i0 + per : nt;
       uint32_t sum = 0;
@@ -534,13 +535,26 @@ __device__ __forceinline__ void regroup_tile(const HfxParams &p, const RegroupAr
       for (int i = i0; i < i1; i++) { const uint32_t f = s_P[i]; s_P[i] = (uint16_t)run; run += f; }
       if (i1 == nt && i0 < nt) s_P[nt] = (uint16_t)run;
       if (nt == 0 && tid == 0) s_P[0] = 0;
+    };
+    if (mode == TILE_SORTED) {
+      // ---- C0: s_P := number of active rows before each position ----------------------------------------
+      scan_P();
     } else {
       // ---- C1: tile rows grouped by replica (counting sort of local indices, class in bit 15) ---------
+      tail_scan = s_off[R1] - s_off[R] > GROUP_MAX;
       for (int i = tid; i < R1; i += blockDim.x) s_cnt[i] = 0;
       __syncthreads();
       for (int i = tid; i < nt; i += blockDim.x) {
         const int b = bucket_of(__ldg(a.replica_id + lo + i), R);
+        if (b == R && tail_scan) continue;
         s_stage[s_off[b] + atomicAdd(&s_cnt[b], 1u)] = (uint16_t)(i | (s_P[i] ? 0x8000 : 0));
+      }
+      if (tail_scan) {
+        // ---- C2: many rows bound to no replica (none of them active): s_P := how many precede each position
+        __syncthreads();
+        for (int i = tid; i < nt; i += blockDim.x) s_P[i] = bucket_of(__ldg(a.replica_id + lo + i), R) == R;
+        __syncthreads();
+        scan_P();
       }
     }
   }
@@ -560,6 +574,8 @@ __device__ __forceinline__ void regroup_tile(const HfxParams &p, const RegroupAr
       const uint32_t o = s_off[bkt];
       const uint32_t ra = (uint32_t)s_P[il] - (uint32_t)s_P[o];
       rank = act ? ra : (uint32_t)il - o - ra;
+    } else if (mode == TILE_GROUPS && bkt == R && tail_scan) {
+      rank = s_P[il];
     } else if (mode == TILE_GROUPS) {
       rank = 0;
       const uint32_t g0 = s_off[bkt], g1 = s_off[bkt + 1];

@@ -848,3 +848,20 @@ def test_scaling_loop_round_by_round():
         on_max = max(on_max, int(np.count_nonzero(f["inst_state"] != gen.INST_OFF)))
     sched.close()
     assert on_max >= 6 and np.count_nonzero(cpu.table["state"] == gen.DONE) > 700
+
+
+@pytest.mark.parametrize("R,permute", [(64, False), (64, True), (4, False)])
+def test_tables_that_are_mostly_global_queue(R, permute):
+    # most rows bound to no instance (they wait in the global queue), a few bound ones in between: tiles with one
+    # large group of unbound rows; ids rising (the step stays ordered) or permuted; with 4 instances the bound
+    # groups of a tile are large too
+    rng = np.random.default_rng(R + permute)
+    wl = gen.elastic(3, R, 50_000)
+    idx = rng.choice(20_000, 3000, replace=False)
+    wl.table["replica_id"][idx] = rng.integers(0, R, 3000)
+    wl.table["replica_id"][49_990:] = R + 5                      # and a few that are simply out of range
+    wl.now[:] = int(np.sort(wl.table["arrival_ns"])[10_000])
+    if permute:
+        wl.table["req_id"][:] = rng.permutation(wl.n_rows).astype(np.int32)
+    g = assert_step_parity(wl, steps=2, commit=True)
+    assert g["adm_count"].sum() > 0
