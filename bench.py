@@ -352,7 +352,7 @@ def run_gpu(args):
     elastic = None
     if rank == 0 and not args.no_elastic:
         ER, EN, TICK, SUB = 1024, 1 << 20, 50_000_000, 6
-        ew = gen.elastic(11, ER, EN, rates=(2000.0, 30000.0))
+        ew = gen.elastic(11, ER, EN, rates=(800.0, 2400.0))       # about 14 requests/s saturate one instance
         esched = hfx.Scheduler(ew.model, ew.classes, ew.replicas, ew.n_rows)
         etab = hfx.DeviceTable.from_numpy(ew.table)
         efl = hfx.Fleet(gen.new_fleet([4096] * ER, range(64)))
@@ -361,9 +361,9 @@ def run_gpu(args):
         ecnt = torch.zeros((3, 4), dtype=torch.int64, device="cuda"); eused = torch.zeros(ER, dtype=torch.int64, device="cuda")
         edec = torch.zeros((3, 2), dtype=torch.int32, device="cuda"); ecost = torch.zeros(3, dtype=torch.int64, device="cuda")
         cold = [300_000_000] * 3
-        rounds_w, rounds_t = 20, 60
+        rounds_w, rounds_t, rounds_all = 20, 60, 600       # the rounds after the timed ones carry the fleet through two bursts
         evs, on_max = [], 0
-        for k in range(rounds_w + rounds_t):
+        for k in range(rounds_all):
             now_g = (k + 1) * TICK
             flush.fill_(7)
             e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
@@ -378,22 +378,38 @@ def run_gpu(args):
             esched.dispatch_step(etab, now_g, efl.t["due"], edout)
             esched.dispatch_bind(etab, now_g, edout, enow)
             e[3].record(stream)
-            if k >= rounds_w:
+            if rounds_w <= k < rounds_w + rounds_t:
                 evs.append(e)
             if k % 10 == 9:
                 on_max = max(on_max, int((efl.t["inst_state"] != 0).sum().item()))
         torch.cuda.synchronize()
         seg = [float(np.mean([e[i].elapsed_time(e[i + 1]) for e in evs])) for i in range(3)]
         est = etab.to_numpy()
-        elastic = {"workload": "up to %d colocated instances (64 on at the start), %d requests in one global queue, %d rounds of a %d ms "
-                               "tick: %d committed steps under the horizon, Scaler tick + its decisions, dispatch + binding"
-                               % (ER, EN, rounds_w + rounds_t, TICK // 1_000_000, SUB),
+        eatt = torch.zeros((len(ew.classes) + 1, 6), dtype=torch.int64, device="cuda")
+        esched.attainment(etab, eatt)
+        eatt_tot = eatt.cpu().numpy()[-1]
+        arrived = int(np.count_nonzero(ew.table["arrival_ns"] <= rounds_all * TICK))
+        elastic = {"workload": "up to %d colocated instances (64 on at the start), a trace of %d requests in one global queue, its first %d rounds of a %d ms "
+                               "tick (%d timed): %d committed steps under the horizon, Scaler tick + its decisions, dispatch + binding"
+                               % (ER, EN, rounds_all, TICK // 1_000_000, rounds_t, SUB),
                    "steps_ms": seg[0], "scaler_ms": seg[1], "dispatch_ms": seg[2], "rounds_per_sec": 1e3 / sum(seg),
                    "instances_on_max": on_max, "instances_on_end": int((efl.t["inst_state"] != 0).sum().item()),
                    "cost_instance_seconds": float(ecost.cpu().numpy()[0]) / 1e9,
                    "requests_bound": int(np.count_nonzero(est["replica_id"] >= 0)),
-                   "requests_finished": int(np.count_nonzero(est["state"] == gen.DONE)), "status": esched.status()}
+                   "requests_arrived": arrived, "requests_finished": int(eatt_tot[1]), "requests_attained": int(eatt_tot[2]),
+                   "status": esched.status()}
         esched.close()
+        if world == 1 and not args.no_cpu:
+            # the same round on the oracle, one host core (test infrastructure timed as a baseline, two rounds)
+            import oracle
+            oracle.build()
+            from oracle import elastic_loop
+            cw_e = ew.copy()
+            cf = gen.new_fleet([4096] * ER, range(64))
+            t0 = time.perf_counter()
+            for k in range(2):
+                elastic_loop.oracle_round(cw_e, cf, k)
+            elastic["cpu_oracle_round_ms"] = 1e3 * (time.perf_counter() - t0) / 2
 
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only -----------------------------
     cpu = None

@@ -1,10 +1,8 @@
-"""The scaling loop both test suites drive: per tick of the global clock, the instances advance up to the tick
-(committed steps under a horizon), the Scaler inspects queue and instances, its decisions are carried out, the
+"""Test infrastructure, like the rest of this package.  The scaling loop both test suites drive: per tick of
+the global clock, the instances advance up to the tick (committed steps under a horizon), the Scaler inspects queue and instances, its decisions are carried out, the
 dispatcher serves the instances that are due and the dispatched requests are bound.  This module runs it on the
 oracle; the GPU parity test runs the same sequence through the library and compares after every call."""
-import numpy as np
-
-import oracle
+from . import dispatch, dispatch_bind, scale_apply, scale_tick, step
 
 MS = 1_000_000
 TICK = 50 * MS
@@ -18,12 +16,12 @@ def oracle_round(wl, fleet, k):
     wl.meta["horizon"] = now_g
     status = 0
     for _ in range(SUBSTEPS):
-        status |= oracle.step(wl, commit=True)["status"]
-    t = oracle.scale_tick(wl, now_g, fleet["total_blocks"], **SCALE_KW)
-    cost = oracle.scale_apply(wl, now_g, t["decision"], t["used_blocks"], COLD, fleet)
+        status |= step(wl, commit=True)["status"]
+    t = scale_tick(wl, now_g, fleet["total_blocks"], **SCALE_KW)
+    cost = scale_apply(wl, now_g, t["decision"], t["used_blocks"], COLD, fleet)
     step_mat = wl.maturity
     wl.maturity = fleet["due"]
-    d = oracle.dispatch(wl, now_g)
+    d = dispatch(wl, now_g)
     wl.maturity = step_mat
-    oracle.dispatch_bind(wl, now_g, d)
+    dispatch_bind(wl, now_g, d)
     return dict(now=now_g, tick=t, cost=cost, dispatch=d, status=status | t["status"] | d["status"])

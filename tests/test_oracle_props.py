@@ -392,7 +392,7 @@ def test_first_fit_invariants_and_dominance(seed):
 
 def test_scaling_loop_invariants():
     # global queue -> dispatcher -> instances, with the Scaler switching instances on and off between ticks
-    from elastic_loop import oracle_round
+    from oracle.elastic_loop import oracle_round
     R = 8
     wl = gen.elastic(1, R, 1500)
     f = gen.new_fleet([2000] * R, [0, 1])

@@ -810,7 +810,7 @@ def test_scaling_loop_round_by_round():
     # the whole loop: instances advance to the tick under the horizon, the Scaler ticks, its decisions are carried
     # out, the dispatcher serves the ACTIVE instances that are due, the requests are bound -- compared after each round
     import paper_2508_15919_b200 as hfx
-    from elastic_loop import COLD, SCALE_KW, SUBSTEPS, oracle_round
+    from oracle.elastic_loop import COLD, SCALE_KW, SUBSTEPS, oracle_round
     R = 8
     wl = gen.elastic(1, R, 1500)
     cpu = wl.copy()
