@@ -361,7 +361,8 @@ def run_gpu(args):
         ecnt = torch.zeros((3, 4), dtype=torch.int64, device="cuda"); eused = torch.zeros(ER, dtype=torch.int64, device="cuda")
         edec = torch.zeros((3, 2), dtype=torch.int32, device="cuda"); ecost = torch.zeros(3, dtype=torch.int64, device="cuda")
         cold = [300_000_000] * 3
-        rounds_w, rounds_t, rounds_all = 20, 60, 600       # the rounds after the timed ones carry the fleet through two bursts
+        rounds_all = max(3, args.elastic_rounds)
+        rounds_w = min(20, rounds_all // 3); rounds_t = min(60, rounds_all - rounds_w)      # the rounds after the timed ones carry the fleet through two bursts
         evs, on_max = [], 0
         for k in range(rounds_all):
             now_g = (k + 1) * TICK
@@ -481,6 +482,7 @@ def main():
     ap.add_argument("--no-dispatch", action="store_true")
     ap.add_argument("--no-pd", action="store_true")
     ap.add_argument("--no-elastic", action="store_true")
+    ap.add_argument("--elastic-rounds", type=int, default=600, help="rounds of the scaling loop (the first 20 warm up, the next 60 are timed)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
