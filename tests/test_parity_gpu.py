@@ -865,3 +865,45 @@ def test_tables_that_are_mostly_global_queue(R, permute):
         wl.table["req_id"][:] = rng.permutation(wl.n_rows).astype(np.int32)
     g = assert_step_parity(wl, steps=2, commit=True)
     assert g["adm_count"].sum() > 0
+
+
+def test_dispatch_with_instances_that_are_never_due():
+    # the maturity array of a fleet: instances that are not ACTIVE are due "never"
+    wl = _colocated(gen.random_table(11, 6000, 12, modes=(gen.COLOCATED,)))
+    now = int(wl.now.max())
+    wl.maturity[:] = gen.T_NEVER
+    g = assert_dispatch_parity(wl, now)
+    assert g["n_mature"][0] == 0 and (g["assign"] >= 0).sum() == 0
+    wl.maturity[::3] = now - 5
+    g = assert_dispatch_parity(wl, now)
+    assert g["n_mature"][0] == 4 and (g["assign"] >= 0).sum() > 0 and set(np.unique(g["assign"])) <= {-1, 0, 3, 6, 9}
+
+
+def test_scale_apply_and_horizon_argument_errors():
+    import ctypes as C
+    import paper_2508_15919_b200 as hfx
+    from paper_2508_15919_b200.binding import _Fleet, _ReplicaState
+    wl = gen.random_table(0, 10, 4)
+    sched = make_sched(wl)
+    fl = hfx.Fleet(gen.new_fleet([10] * 4, [0]))
+    now = torch.zeros(4, dtype=torch.int64, device="cuda"); mat = torch.zeros(4, dtype=torch.int64, device="cuda")
+    dec = torch.zeros((3, 2), dtype=torch.int32, device="cuda"); used = torch.zeros(4, dtype=torch.int64, device="cuda")
+    cost = torch.zeros(4, dtype=torch.int64, device="cuda")
+    L, h = sched._L, sched._h
+    good = (C.c_int64 * 3)(1, 1, 1)
+    fs = fl.c_struct(); st = _ReplicaState(now.data_ptr(), mat.data_ptr())
+
+    def call(decision=dec.data_ptr(), usedp=used.data_ptr(), cold=good, fleet=fs, state=st, costp=cost.data_ptr()):
+        return L.hfx_scale_apply(h, 5, decision, usedp, cold, C.byref(fleet), C.byref(state), costp)
+
+    assert call() == 0
+    assert call(decision=None) != 0 and call(usedp=None) != 0 and call(costp=None) != 0
+    assert call(cold=(C.c_int64 * 3)(1, -1, 1)) != 0
+    assert call(costp=cost.data_ptr() + 8) != 0                         # misaligned
+    holes = fl.c_struct(); holes.due_ns = None
+    assert call(fleet=holes) != 0
+    assert call(state=_ReplicaState(now.data_ptr(), None)) != 0
+    assert L.hfx_scale_apply(None, 5, dec.data_ptr(), used.data_ptr(), good, C.byref(fs), C.byref(st), cost.data_ptr()) != 0
+    assert L.hfx_sched_set_horizon(None, 5) != 0
+    assert sched.status() == 0
+    sched.close()
