@@ -398,6 +398,10 @@ int hfx_sim_run(hfx_sched *s, const hfx_table *table, const int32_t *trace_off,
  *        in 16.16 fixed point (floor), saturated at 2^15,
  *   f3 = used_blocks / total_blocks per instance: ceil((prompt_len + gen) / block_tokens) of every
  *        in-flight request plus ceil(prompt_len / block_tokens) of every visible queued one.
+ * A QUEUED request with replica_id -1 is still in the global queue, bound to no instance: the global
+ * queue feeds the colocated instances and the P stage, so it counts as an arrival and as a waiting
+ * request for pools 0 and 1 and holds no KV block (any other row with a replica_id outside
+ * [0, n_replicas) is skipped and sets HFX_ST_BAD_REPLICA).
  * Decision per pool: scale out (+1) if f1 < eps_out or f2 > eps_wait; else scale in (-1) if
  * f1 > eps_in and more than one instance of the pool is active (total_blocks > 0), removing the
  * active instance with the smallest f3 (lowest id on ties); else hold (0).  Thresholds are the
