@@ -423,6 +423,13 @@ typedef struct hfx_scale_out {
 
 int hfx_scale_tick(hfx_sched *s, const hfx_table *table, int64_t now_ns, const int32_t *total_blocks,
                    const hfx_scale_params *params, const hfx_scale_out *out);
+/* The decision of a tick alone, from counters that are already there: out->counts and out->used_blocks are
+ * READ (as hfx_scale_tick writes them, or sums of what it wrote for the shards of a table: a Scaler that
+ * watches instances on several GPUs adds up their counters first -- integer sums, the decision is the same
+ * on every rank), out->decision is written.  window_ns and block_tokens of `params` are not used.
+ * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CUDA. */
+int hfx_scale_decide(hfx_sched *s, const int32_t *total_blocks, const hfx_scale_params *params,
+                     const hfx_scale_out *out);
 
 /* Carrying out the decisions of a Scaler tick: the life of an instance and the cost of the fleet
  * (Sec. 3.3.3 for the decisions, Eq. 1 of the Problem Definition for the cost; the time to bring an

@@ -160,6 +160,8 @@ def lib():
                                      C.c_void_p]
         L.ora_attainment.restype = C.c_uint32
         L.ora_attainment.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_void_p]
+        L.ora_scale_decide.restype = None
+        L.ora_scale_decide.argtypes = [C.POINTER(_Config), C.c_void_p, C.POINTER(_ScaleParams), C.POINTER(_ScaleOut)]
         L.ora_dispatch_bind.restype = None
         L.ora_dispatch_bind.argtypes = [C.POINTER(_Config), C.POINTER(_Table), C.c_int64] + [C.c_void_p] * 4
         L.ora_scale_apply.restype = None
@@ -345,6 +347,23 @@ def scale_apply(wl, now: int, decision: np.ndarray, used_blocks: np.ndarray, col
     L.ora_scale_apply(C.byref(ctx.cfg), int(now), dec.ctypes.data, used.ctypes.data, cold.ctypes.data, C.byref(fl),
                       wl.now.ctypes.data, wl.maturity.ctypes.data, cost.ctypes.data)
     return cost
+
+
+def scale_decide(wl, total_blocks: np.ndarray, counts: np.ndarray, used_blocks: np.ndarray, **kw) -> np.ndarray:
+    """The threshold decision per pool from counters and used blocks that are already there (summed over the
+    shards of a table, for instance).  Returns decision int32 [3, 2]."""
+    L = lib()
+    ctx = _Ctx(wl)
+    prm = dict(SCALE_DEFAULTS); prm.update(kw)
+    sp = _ScaleParams(int(prm["window"]), int(prm["block_tokens"]), int(prm["min_samples"]), *prm["eps_out"],
+                      *prm["eps_in"], *prm["eps_wait"])
+    cnt = np.ascontiguousarray(counts, np.int64).reshape(3, 4); used = np.ascontiguousarray(used_blocks, np.int64)
+    tb = np.ascontiguousarray(total_blocks, np.int32)
+    assert used.size == wl.n_replicas and tb.size == wl.n_replicas
+    dec = np.zeros((3, 2), np.int32)
+    so = _ScaleOut(cnt.ctypes.data, used.ctypes.data, dec.ctypes.data)
+    L.ora_scale_decide(C.byref(ctx.cfg), tb.ctypes.data, C.byref(sp), C.byref(so))
+    return dec
 
 
 def scale_tick(wl, now: int, total_blocks: np.ndarray, **kw) -> Dict[str, np.ndarray]:

@@ -607,6 +607,31 @@ typedef struct {
   int32_t *decision;     /* [3][2]: per pool action (+1 out, -1 in, 0 hold), instance to remove or -1 */
 } ora_scale_out;
 
+/* The decision alone, from counters and used blocks that are already there (a Scaler that watches
+ * several shards of the table sums their counters first; integer sums, so the result is the same). */
+void ora_scale_decide(const ora_config *c, const int32_t *total_blocks, const ora_scale_params *sp, const ora_scale_out *o) {
+  const int32_t R = c->n_replicas;
+  for (int pool = 0; pool < 3; pool++) {
+    const int64_t *cnt = o->counts + 4 * pool;
+    int32_t n_active = 0, victim = -1;
+    for (int32_t r = 0; r < R; r++) {
+      if (c->replicas[r].mode != pool || total_blocks[r] <= 0) continue;
+      n_active++;
+      /* smallest used/total: compare by cross-multiplication */
+      if (victim < 0 || (i128)o->used_blocks[r] * total_blocks[victim] < (i128)o->used_blocks[victim] * total_blocks[r]) victim = r;
+    }
+    const int f1_valid = cnt[0] >= sp->min_samples;
+    int action = 0;
+    if ((f1_valid && (i128)sp->eps_out_den * cnt[1] < (i128)sp->eps_out_num * cnt[0]) ||
+        (cnt[2] > 0 && (i128)sp->eps_wait_den * cnt[3] > ((i128)sp->eps_wait_num * cnt[2] << 16)))
+      action = 1;
+    else if (f1_valid && (i128)sp->eps_in_den * cnt[1] > (i128)sp->eps_in_num * cnt[0] && n_active > 1)
+      action = -1;
+    o->decision[2 * pool] = action;
+    o->decision[2 * pool + 1] = action == -1 ? victim : -1;
+  }
+}
+
 uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const int32_t *total_blocks,
                    const ora_scale_params *sp, const ora_scale_out *o) {
   const int32_t R = c->n_replicas;
@@ -650,25 +675,7 @@ uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const i
       }
     }
   }
-  for (int pool = 0; pool < 3; pool++) {
-    const int64_t *cnt = o->counts + 4 * pool;
-    int32_t n_active = 0, victim = -1;
-    for (int32_t r = 0; r < R; r++) {
-      if (c->replicas[r].mode != pool || total_blocks[r] <= 0) continue;
-      n_active++;
-      /* smallest used/total: compare by cross-multiplication */
-      if (victim < 0 || (i128)o->used_blocks[r] * total_blocks[victim] < (i128)o->used_blocks[victim] * total_blocks[r]) victim = r;
-    }
-    const int f1_valid = cnt[0] >= sp->min_samples;
-    int action = 0;
-    if ((f1_valid && (i128)sp->eps_out_den * cnt[1] < (i128)sp->eps_out_num * cnt[0]) ||
-        (cnt[2] > 0 && (i128)sp->eps_wait_den * cnt[3] > ((i128)sp->eps_wait_num * cnt[2] << 16)))
-      action = 1;
-    else if (f1_valid && (i128)sp->eps_in_den * cnt[1] > (i128)sp->eps_in_num * cnt[0] && n_active > 1)
-      action = -1;
-    o->decision[2 * pool] = action;
-    o->decision[2 * pool + 1] = action == -1 ? victim : -1;
-  }
+  ora_scale_decide(c, total_blocks, sp, o);
   return status;
 }
 

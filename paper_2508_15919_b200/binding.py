@@ -22,7 +22,7 @@ E_ARG, E_ALIGN, E_CAPACITY, E_CUDA, E_TIMEOUT, E_NOMEM = -1, -2, -3, -4, -5, -6
 EXPORTED_SYMBOLS = ["hfx_sched_create", "hfx_sched_step", "hfx_sim_run", "hfx_sched_status",
                     "hfx_sched_launch_count", "hfx_sched_destroy", "hfx_strerror", "hfx_sched_set_profiling",
                     "hfx_sched_get_profile", "hfx_sched_set_fused_front", "hfx_kernel_name", "hfx_count_rows_noalloc", "hfx_scale_tick", "hfx_dispatch_step", "hfx_slo_map", "hfx_pd_migrate", "hfx_attainment",
-                    "hfx_sched_set_horizon", "hfx_scale_apply", "hfx_dispatch_bind"]
+                    "hfx_sched_set_horizon", "hfx_scale_apply", "hfx_dispatch_bind", "hfx_scale_decide"]
 NOALLOC_MAX_REPLICAS = 4096
 N_KERNELS = 14
 
@@ -163,6 +163,8 @@ def load_library():
     L.hfx_sched_set_profiling.argtypes = [C.c_void_p, C.c_int]
     L.hfx_sched_set_horizon.restype = C.c_int
     L.hfx_sched_set_horizon.argtypes = [C.c_void_p, C.c_int64]
+    L.hfx_scale_decide.restype = C.c_int
+    L.hfx_scale_decide.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(_ScaleParams), C.POINTER(_ScaleOut)]
     L.hfx_scale_apply.restype = C.c_int
     L.hfx_scale_apply.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(C.c_int64), C.POINTER(_Fleet),
                                   C.POINTER(_ReplicaState), C.c_void_p]
@@ -444,6 +446,15 @@ class Scheduler:
         rc = self._L.hfx_scale_tick(self._h, C.byref(ts), int(now_ns), total_blocks.data_ptr(), C.byref(sp), C.byref(so))
         if rc != 0:
             raise HfxError(rc, "hfx_scale_tick")
+
+    def scale_decide(self, total_blocks: torch.Tensor, counts: torch.Tensor, used_blocks: torch.Tensor, decision: torch.Tensor,
+                     min_samples: int = 10, eps_out=(7, 10), eps_in=(11, 10), eps_wait=(1, 4)):
+        """hfx_scale_decide: the decision from counters that are already there (counts and used_blocks are read)."""
+        sp = _ScaleParams(1, 1, int(min_samples), *eps_out, *eps_in, *eps_wait)
+        so = _ScaleOut(counts.data_ptr(), used_blocks.data_ptr(), decision.data_ptr())
+        rc = self._L.hfx_scale_decide(self._h, total_blocks.data_ptr(), C.byref(sp), C.byref(so))
+        if rc != 0:
+            raise HfxError(rc, "hfx_scale_decide")
 
     def status(self) -> int:
         w = C.c_uint32(0)

@@ -223,3 +223,22 @@ extern "C" int hfx_scale_tick(hfx_sched *s, const hfx_table *t, int64_t now_ns, 
   }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }
+
+extern "C" int hfx_scale_decide(hfx_sched *s, const int32_t *total_blocks, const hfx_scale_params *sp, const hfx_scale_out *o) {
+  if (!s || !total_blocks || !sp || !o || !o->counts || !o->used_blocks || !o->decision) return HFX_E_ARG;
+  if (sp->eps_out_num <= 0 || sp->eps_out_den <= 0 || sp->eps_in_num <= 0 || sp->eps_in_den <= 0 || sp->eps_wait_num <= 0 ||
+      sp->eps_wait_den <= 0)
+    return HFX_E_ARG;
+  const void *all[] = {total_blocks, o->counts, o->used_blocks, o->decision};
+  for (const void *q : all) if (misaligned16(q)) return HFX_E_ALIGN;
+  ScaleArgs a = {};
+  a.mode = s->d_mode; a.total_blocks = total_blocks;
+  a.counts = reinterpret_cast<unsigned long long *>(o->counts);
+  a.used_blocks = reinterpret_cast<unsigned long long *>(o->used_blocks);
+  a.decision = o->decision; a.status = s->d_status; a.sp = *sp;
+  {
+    KernelScope ks(s, KSLOT_SCALE);
+    k_scale_decide<<<1, 1024, 0, s->stream>>>(s->p, a);
+  }
+  return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
+}

@@ -2,7 +2,8 @@
 
 Replicas are independent units of the scheduler step, so a table is split by contiguous replica
 ranges and every rank runs the whole path on its own rows; no collective touches the data path.
-The only communication is the reduction of timings and counts for reporting.
+The only communication is the reduction of timings and counts for reporting -- and, for a Scaler that
+watches instances on several GPUs, the sum of the tick's counters (scaler_exchange).
 """
 from __future__ import annotations
 
@@ -41,3 +42,15 @@ def reduce_report(step_ms: float, rows: int, group=None) -> Tuple[float, int]:
     dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
     dist.all_reduce(r, op=dist.ReduceOp.SUM, group=group)
     return float(t.item()), int(r.item())
+
+
+def scaler_exchange(counts, used_blocks, group=None) -> None:
+    """Sum, in place and over all ranks, what hfx_scale_tick counted on each rank's shard of the table (counts
+    int64 [3, 4]; used_blocks int64 [n_replicas] with global instance ids, zero for instances whose rows live on
+    another rank).  Afterwards hfx_scale_decide gives the same decision on every rank.  Integer sums: the order
+    of the reduction cannot change the result.  CPU tensors go over gloo, CUDA tensors over NCCL."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return
+    dist.all_reduce(counts, op=dist.ReduceOp.SUM, group=group)
+    dist.all_reduce(used_blocks, op=dist.ReduceOp.SUM, group=group)

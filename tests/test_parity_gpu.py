@@ -907,3 +907,44 @@ def test_scale_apply_and_horizon_argument_errors():
     assert L.hfx_sched_set_horizon(None, 5) != 0
     assert sched.status() == 0
     sched.close()
+
+
+def test_scale_decide_from_summed_counters():
+    # the decision alone: from the tick's own counters it repeats the tick's decision; from counters of two shards
+    # of the table, summed, it gives the decision of the whole table; and from arbitrary counters the oracle's
+    import paper_2508_15919_b200 as hfx
+    rng = np.random.default_rng(12)
+    R = 23
+    wl = gen.random_table(12, 40_000, R, modes=MODES3, future=0.1, done=0.4)
+    wl.table["finish_ns"][:] = wl.now.max() - rng.integers(0, 3 * SEC, wl.n_rows)
+    wl.table["replica_id"][::6] = -1
+    now = int(wl.now.max())
+    tb_np = (rng.integers(1, 900, R) * (rng.random(R) < 0.8)).astype(np.int32)
+    kw = dict(window=2 * SEC, min_samples=1, eps_in=(1, 50), eps_wait=(50, 1))
+    full = oracle.scale_tick(wl, now, tb_np, **kw)
+    sched = make_sched(wl)
+    tb = torch.from_numpy(tb_np).cuda()
+    tot_c = torch.zeros((3, 4), dtype=torch.int64, device="cuda"); tot_u = torch.zeros(R, dtype=torch.int64, device="cuda")
+    for half in range(2):
+        part = {k: np.ascontiguousarray(v[half::2]) for k, v in wl.table.items()}
+        tab = hfx.DeviceTable.from_numpy(part)
+        c = torch.zeros((3, 4), dtype=torch.int64, device="cuda"); u = torch.zeros(R, dtype=torch.int64, device="cuda")
+        d = torch.zeros((3, 2), dtype=torch.int32, device="cuda")
+        sched.scale_tick(tab, now, tb, c, u, d, window_ns=kw["window"], min_samples=1, eps_in=kw["eps_in"], eps_wait=kw["eps_wait"])
+        tot_c += c; tot_u += u
+    assert np.array_equal(tot_c.cpu().numpy(), full["counts"]) and np.array_equal(tot_u.cpu().numpy(), full["used_blocks"])
+    dec = torch.full((3, 2), 9, dtype=torch.int32, device="cuda")
+    sched.scale_decide(tb, tot_c, tot_u, dec, min_samples=1, eps_in=kw["eps_in"], eps_wait=kw["eps_wait"])
+    assert np.array_equal(dec.cpu().numpy(), full["decision"])
+    seen = set()
+    for k in range(40):
+        cnt = rng.integers(0, 60, (3, 4)).astype(np.int64); cnt[:, 3] = cnt[:, 2] * rng.integers(0, 1 << 15, 3)
+        used = (rng.integers(0, 400, R) * rng.integers(0, 2, R)).astype(np.int64)
+        kk = dict(min_samples=int(rng.integers(0, 30)), eps_out=(int(rng.integers(1, 20)), 10), eps_in=(int(rng.integers(1, 20)), 10),
+                  eps_wait=(1, int(rng.integers(1, 8))))
+        sched.scale_decide(tb, torch.from_numpy(cnt).cuda(), torch.from_numpy(used).cuda(), dec, **kk)
+        want = oracle.scale_decide(wl, tb_np, cnt, used, **kk)
+        assert np.array_equal(dec.cpu().numpy(), want), (k, dec.cpu().numpy(), want)
+        seen |= set(want[:, 0].tolist())
+    assert seen == {-1, 0, 1} and sched.status() != 0      # the shards held rows with ids out of range too
+    sched.close()
