@@ -850,8 +850,8 @@ def test_scaling_loop_round_by_round():
     assert on_max >= 6 and np.count_nonzero(cpu.table["state"] == gen.DONE) > 700
 
 
-@pytest.mark.parametrize("R,permute", [(64, False), (64, True), (4, False)])
-def test_tables_that_are_mostly_global_queue(R, permute):
+@pytest.mark.parametrize("R,permute,fused", [(64, False, True), (64, True, True), (4, False, True), (64, False, False), (4, False, False)])
+def test_tables_that_are_mostly_global_queue(R, permute, fused):
     # most rows bound to no instance (they wait in the global queue), a few bound ones in between: tiles with one
     # large group of unbound rows; ids rising (the step stays ordered) or permuted; with 4 instances the bound
     # groups of a tile are large too
@@ -863,7 +863,10 @@ def test_tables_that_are_mostly_global_queue(R, permute):
     wl.now[:] = int(np.sort(wl.table["arrival_ns"])[10_000])
     if permute:
         wl.table["req_id"][:] = rng.permutation(wl.n_rows).astype(np.int32)
-    g = assert_step_parity(wl, steps=2, commit=True)
+    sched = make_sched(wl)
+    sched.set_fused_front(fused)
+    g = assert_step_parity(wl, steps=2, commit=True, sched=sched)
+    sched.close()
     assert g["adm_count"].sum() > 0
 
 
