@@ -55,7 +55,9 @@ extern "C" {
 #define HFX_E_NOMEM      -6   /* workspace allocation failed                 */
 
 /* bits of the sticky device status word */
-#define HFX_ST_BAD_REPLICA  1u  /* replica_id outside [0, n_replicas)         */
+#define HFX_ST_BAD_REPLICA  1u  /* replica_id outside [0, n_replicas); not raised for -1
+                                   on a QUEUED row: that request is still in the global
+                                   queue, bound to no instance yet                     */
 #define HFX_ST_BAD_CLASS    2u  /* class_id >= n_classes                      */
 #define HFX_ST_BAD_LEN      4u  /* prompt_len or gen outside [0, 2^24]        */
 #define HFX_ST_TIMEOUT      8u  /* a device-side wait gave up                 */
@@ -133,7 +135,8 @@ typedef struct hfx_options {
  * `finish_ns` unless HFX_COMMIT is given or the call is hfx_sim_run. */
 typedef struct hfx_table {
   int64_t        n_rows;
-  const int32_t *replica_id;     /* instance the request is bound to          */
+  const int32_t *replica_id;     /* instance the request is bound to; -1 on a
+                                    QUEUED row: still in the global queue     */
   const uint8_t *class_id;       /* index into the SLO class table            */
   uint8_t       *state;          /* HFX_QUEUED .. HFX_REJECTED (written by
                                     COMMIT and by hfx_sim_run)                */

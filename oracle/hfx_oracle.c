@@ -448,7 +448,10 @@ uint32_t ora_step(const ora_config *c, const ora_table *t, int64_t *now, int64_t
   int64_t *cnt = (int64_t *)calloc((size_t)R + 2, sizeof(int64_t));
   for (int64_t i = 0; i < t->n; i++) {
     int32_t r = t->replica_id[i];
-    if (r < 0 || r >= R) { status |= BAD_REPLICA; r = R; }
+    /* reading: replica_id -1 on a QUEUED request means "still in the global queue" (the dispatcher has not
+     * bound it yet): no replica looks at it, it is listed behind the last replica, and it is no error */
+    if (r == -1 && t->state[i] == ST_QUEUED) r = R;
+    else if (r < 0 || r >= R) { status |= BAD_REPLICA; r = R; }
     cnt[r + 1]++;
   }
   for (int32_t r = 0; r <= R; r++) cnt[r + 1] += cnt[r];
@@ -968,6 +971,7 @@ uint32_t ora_pd_migrate(const ora_config *c, const ora_table *t, int64_t *now, c
   for (int32_t r = 0; r < R; r++) wake[r] = ORA_INF;
   for (int64_t i = 0; i < t->n; i++) {
     const int32_t r = rid[i];
+    if (r == -1 && t->state[i] == ST_QUEUED) continue;      /* still in the global queue */
     if (r < 0 || r >= R) { status |= BAD_REPLICA; continue; }
     if (!row_valid(c, t, i, &status)) continue;
     if (c->replicas[r].mode != MODE_PREFILL || t->state[i] != ST_RUNNING) continue;

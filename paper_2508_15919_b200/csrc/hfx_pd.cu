@@ -24,6 +24,7 @@ __global__ void __launch_bounds__(PD_THREADS) k_pd_rows(const HfxParams p, const
   uint32_t bad = 0;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < a.n; i += (int64_t)gridDim.x * blockDim.x) {
     const int32_t r = a.replica_id[i];
+    if (r == -1 && a.state[i] == HFX_QUEUED) continue;       // still in the global queue
     if (r < 0 || r >= R) { bad |= HFX_ST_BAD_REPLICA; continue; }
     const uint32_t cls = a.class_id[i], st = a.state[i];
     const int32_t prompt = a.prompt_len[i], gen = a.gen[i];

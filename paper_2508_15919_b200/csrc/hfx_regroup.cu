@@ -32,7 +32,10 @@ __device__ __forceinline__ int bucket_of(int rid, int R) { return (rid < 0 || ri
 // Kind of a row (KIND_*), with ROWFLAG_BADREP for a row bound to no replica; raises status bits.
 __device__ __forceinline__ uint32_t classify_row(const HfxParams &p, int32_t rid, uint32_t cls, uint32_t st, int32_t prompt,
                                                  int32_t gen, int64_t arrival, const int64_t *now, uint32_t &bad) {
-  if (rid < 0 || rid >= p.n_replicas) { bad |= HFX_ST_BAD_REPLICA; return KIND_DEAD | ROWFLAG_BADREP; }
+  if (rid < 0 || rid >= p.n_replicas) {
+    if (!(rid == -1 && st == HFX_QUEUED)) bad |= HFX_ST_BAD_REPLICA;      // -1 on a QUEUED row: still in the global queue, no error
+    return KIND_DEAD | ROWFLAG_BADREP;
+  }
   bool ok = true;
   if (cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
   if (prompt < 0 || prompt > HFX_MAX_TOKENS || gen < 0 || gen > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }

@@ -572,3 +572,21 @@ def test_horizon_gate_and_binding():
                  [(200 * MS, 30 * MS, 0)], replicas=[(gen.COLOCATED, 32768, 0)] * 3, now=[5, 500, 7], maturity=[0, 0, 0])
     oracle.dispatch_bind(wl, 100, dict(assign=np.array([1, -1], np.int32), adm_count=np.array([1, 1, 0], np.int32)))
     assert list(wl.table["replica_id"]) == [1, -1] and list(wl.now) == [100, 500, 7]
+
+
+def test_unbound_queued_rows_are_the_global_queue_not_an_error():
+    rows = [dict(prompt_len=100, req_id=0, output_len=5), dict(prompt_len=100, req_id=1, replica_id=-1, output_len=5),
+            dict(prompt_len=100, req_id=2, replica_id=-1, output_len=5), dict(prompt_len=100, req_id=3, output_len=5)]
+    wl = make_wl(rows, C200, now=[MS])
+    o = oracle.step(wl, commit=True)
+    assert o["status"] == 0 and list(o["seg_off"]) == [0, 2] and list(o["order"]) == [0, 3, 1, 2]
+    assert list(o["admit"]) == [1, 0, 0, 1] and list(wl.table["state"]) == [gen.RUNNING, gen.QUEUED, gen.QUEUED, gen.RUNNING]
+    # the same id on a request that is running somewhere is bad data; so is any other id out of range
+    wl.table["replica_id"][0] = -1
+    assert oracle.step(wl)["status"] == 1
+    wl.table["replica_id"][0] = 0; wl.table["replica_id"][1] = -2
+    assert oracle.step(wl)["status"] == 1
+    # the hand-off between the stages leaves the global queue alone too
+    wl = make_wl(rows[:2], [(200 * MS, 30 * MS, 0)], replicas=[(gen.PREFILL, 32768, 0), (gen.DECODE, 32768, 8)], now=[0, 0], maturity=[0, 0])
+    r = oracle.pd_migrate(wl, np.array([1, -1]), 1_000_000, 1000)
+    assert r == {"status": 0, "moved": 0}

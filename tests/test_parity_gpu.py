@@ -188,6 +188,16 @@ def test_bad_rows_are_flagged_not_fatal():
     sched = make_sched(wl)
     assert sched.status() == 0
     sched.close()
+    # -1 on a QUEUED row is the global queue, not an error: a table whose only oddity is that raises nothing
+    wl = gen.random_table(15, 3000, 5, modes=MODES3)
+    q = np.flatnonzero(wl.table["state"] == gen.QUEUED)
+    wl.table["replica_id"][q[::3]] = -1
+    cpu = wl.copy()
+    assert oracle.step(cpu)["status"] == 0
+    assert_step_parity(wl, steps=2, commit=True)
+    wl.table["replica_id"][np.flatnonzero(wl.table["state"] == gen.RUNNING)[:1]] = -1
+    assert oracle.step(wl.copy())["status"] == 1
+    assert_step_parity(wl, steps=1)
 
 
 def test_ties_in_every_key_field():
