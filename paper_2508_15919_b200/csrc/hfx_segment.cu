@@ -315,6 +315,92 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
   }
 }
 
+// The sorting network of block_sort for items of one 64-bit word (ordered steps), with the items held in
+// registers: thread t of the 1024 owns the items IPT*t .. IPT*t + IPT-1 (IPT * 1024 = the padded length).
+// Every pair of the network is (i, i ^ mask): mask = k-1 in the mirrored first sub-stage of merge size k,
+// a single bit j afterwards; the lower index keeps the smaller item.  Masks below IPT stay inside a
+// thread (no memory traffic), thread distances below 32 go through warp shuffles, the rest (15 of the
+// 105 sub-stages at 16384 items) through shared memory, striped by item slot so that neither side has
+// bank conflicts.  `hi` holds the items on entry and is the exchange buffer afterwards; on return
+// pos_out[i] is the low 16 bits (the item's tie-break position) of the i-th smallest item.
+// The block is synchronised on entry by the caller; the caller synchronises before reading pos_out.
+__device__ __forceinline__ void cx64(uint64_t &a, uint64_t &b) {
+  const uint64_t lo = a < b ? a : b, hi = a < b ? b : a;
+  a = lo; b = hi;
+}
+
+template <int IPT>
+__device__ void block_sort_reg(uint64_t *hi, uint32_t *pos_out, int n) {
+  const int t = threadIdx.x;
+  uint64_t v[IPT];
+#pragma unroll
+  for (int e = 0; e < IPT; e++) { const int i = t * IPT + e; v[e] = i < n ? hi[i] : ~UINT64_C(0); }
+  __syncthreads();
+  // merge sizes up to IPT: inside the thread
+#pragma unroll
+  for (int k = 2; k <= IPT; k <<= 1) {
+#pragma unroll
+    for (int e = 0; e < IPT; e++) if (e < (e ^ (k - 1))) cx64(v[e], v[e ^ (k - 1)]);
+#pragma unroll
+    for (int j = k >> 2; j > 0; j >>= 1)
+#pragma unroll
+      for (int e = 0; e < IPT; e++) if (!(e & j)) cx64(v[e], v[e | j]);
+  }
+  // merge sizes kt * IPT: kt threads per merged run
+  for (int kt = 2; kt <= 1024; kt <<= 1) {
+    {   // mirrored sub-stage: partner thread t ^ (kt-1), partner slot IPT-1-e
+      const int mt = kt - 1;
+      const bool lower = (t & (kt >> 1)) == 0;
+      if (mt < 32) {
+#pragma unroll
+        for (int e = 0; e < (IPT + 1) / 2; e++) {
+          const int f = IPT - 1 - e;
+          const uint64_t pa = __shfl_xor_sync(0xffffffffu, v[f], mt);     // the partner's slot f pairs with my slot e
+          const uint64_t pb = __shfl_xor_sync(0xffffffffu, v[e], mt);     // and its slot e with my slot f
+          v[e] = lower ? (v[e] < pa ? v[e] : pa) : (v[e] < pa ? pa : v[e]);
+          if (f != e) v[f] = lower ? (v[f] < pb ? v[f] : pb) : (v[f] < pb ? pb : v[f]);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < IPT; e++) hi[e * 1024 + t] = v[e];
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < IPT; e++) {
+          const uint64_t w = hi[(IPT - 1 - e) * 1024 + (t ^ mt)];
+          v[e] = lower ? (v[e] < w ? v[e] : w) : (v[e] < w ? w : v[e]);
+        }
+        __syncthreads();
+      }
+    }
+    for (int jt = kt >> 2; jt > 0; jt >>= 1) {     // partner thread t ^ jt, same slot
+      const bool lower = (t & jt) == 0;
+      if (jt < 32) {
+#pragma unroll
+        for (int e = 0; e < IPT; e++) {
+          const uint64_t w = __shfl_xor_sync(0xffffffffu, v[e], jt);
+          v[e] = lower ? (v[e] < w ? v[e] : w) : (v[e] < w ? w : v[e]);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < IPT; e++) hi[e * 1024 + t] = v[e];
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < IPT; e++) {
+          const uint64_t w = hi[e * 1024 + (t ^ jt)];
+          v[e] = lower ? (v[e] < w ? v[e] : w) : (v[e] < w ? w : v[e]);
+        }
+        __syncthreads();
+      }
+    }
+#pragma unroll
+    for (int j = IPT >> 1; j > 0; j >>= 1)          // the remaining distances are inside the thread
+#pragma unroll
+      for (int e = 0; e < IPT; e++) if (!(e & j)) cx64(v[e], v[e | j]);
+  }
+#pragma unroll
+  for (int e = 0; e < IPT; e++) { const int i = t * IPT + e; if (i < n) pos_out[i] = (uint32_t)(v[e] & 0xffffu); }
+}
+
 __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegArgs a, const SegCtx c, int seg_min,
                                                   int seg_cap, int bucket) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -388,8 +474,16 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
     __syncthreads();
     if (ordered) {
       if (!(bucket && n_act > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_act, sh))) {
-        block_sort<false>(s_hi, nullptr, n_act);
-        for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+        if (blockDim.x == 1024 && n_act > 512) {      // items in registers: 1, 2, 4, 8 or 16 per thread
+          if (n_act <= 1024) block_sort_reg<1>(s_hi, s_lo, n_act);
+          else if (n_act <= 2048) block_sort_reg<2>(s_hi, s_lo, n_act);
+          else if (n_act <= 4096) block_sort_reg<4>(s_hi, s_lo, n_act);
+          else if (n_act <= 8192) block_sort_reg<8>(s_hi, s_lo, n_act);
+          else block_sort_reg<16>(s_hi, s_lo, n_act);
+        } else {
+          block_sort<false>(s_hi, nullptr, n_act);
+          for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+        }
       }
     } else {
       block_sort<true>(s_hi, s_lo, n_act);
