@@ -263,7 +263,18 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     }
     __syncthreads();
   }
-  for (int tile = 0; tile < n_sorted; tile += blockDim.x) {
+  // The order begins with the requests in flight (phase 0 sorts first): they are listed and marked, no
+  // prefix is needed for them.  Whole tiles of them are passed here; the scan starts at the tile that
+  // reaches the queue.
+  const int n_front = (int)((pl.n_run < n_sorted ? pl.n_run : n_sorted) / blockDim.x) * blockDim.x;
+  for (int q = threadIdx.x; q < n_front; q += blockDim.x) {
+    const uint32_t li = s_lo[q] & 0xffffu;
+    const int32_t row = (int32_t)__ldg(reinterpret_cast<const uint4 *>(seg + li)).w;
+    a.order[b + q] = row;
+    a.admit[row] = 1;
+    s_lo[q] = li;
+  }
+  for (int tile = n_front; tile < n_sorted; tile += blockDim.x) {
     const int q = tile + threadIdx.x;
     int64_t cost = 0, kv = 0;
     int32_t cnt = 0, row = -1, kind = KIND_DEAD;
@@ -279,6 +290,13 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
         if (p.first_fit ? (s_lo[q] & 0x20000u) != 0 : c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
       }
       a.order[b + q] = row;
+    }
+    if (!__syncthreads_or(cnt)) {      // no candidate in this tile (a spent budget, requests in flight): nothing to add up
+      if (q < n_sorted) {
+        if (kind == KIND_RUNNING) a.admit[row] = 1;
+        s_lo[q] &= 0xffffu;
+      }
+      continue;
     }
     // block-wide inclusive scan of (cost, cnt) with carry
     int64_t sc = warp_incl_scan_i64(cost, lane);
@@ -307,11 +325,23 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)warp_sum_i64(an);
     __syncthreads();     // everyone has read red_a / red_b / carry
     if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_c[warp] = an; }
-    if (threadIdx.x == blockDim.x - 1) { sh.carry_cost = sc; sh.carry_count = sn; }
+    if (threadIdx.x == blockDim.x - 1) { sh.carry_cost = sc; sh.carry_count = sn; sh.carry_act = kind == KIND_QUEUED; }
     __syncthreads();
     if (threadIdx.x == 0)
       for (int k = 0; k < nwarp; k++) { sh.adm_cost += sh.red_a[k]; sh.adm_kv += sh.red_b[k]; sh.adm_count += (int32_t)sh.red_c[k]; }
     __syncthreads();
+    // Admission along the order is closed under prefixes: once the running cost is over the budget, or the
+    // batch is full, nothing behind is admitted; and once the order has reached the queue, nothing behind is
+    // in flight.  The rest of the order then only has to be written out.
+    if (!p.first_fit && sh.carry_act &&
+        (sh.carry_cost > pl.budget || (pl.batch_cap != 0 && pl.n_eff + sh.carry_count >= pl.batch_cap))) {
+      for (int q = tile + blockDim.x + threadIdx.x; q < n_sorted; q += blockDim.x) {
+        const uint32_t li = s_lo[q] & 0xffffu;
+        a.order[b + q] = (int32_t)__ldg(reinterpret_cast<const uint4 *>(seg + li)).w;
+        s_lo[q] = li;
+      }
+      break;
+    }
   }
 }
 
