@@ -431,6 +431,22 @@ __device__ void block_sort_reg(uint64_t *hi, uint32_t *pos_out, int n) {
   for (int e = 0; e < IPT; e++) { const int i = t * IPT + e; if (i < n) pos_out[i] = (uint32_t)(v[e] & 0xffffu); }
 }
 
+// Sort n distinct 64-bit items (block-synchronised on entry) and write their low 16 bits, in ascending item
+// order, to pos_out; the caller synchronises before reading pos_out.  1024-thread blocks keep the items in
+// registers (1, 2, 4, 8 or 16 per thread) for more than 512 items.
+__device__ __forceinline__ void sort64_positions(uint64_t *hi, uint32_t *pos_out, int n) {
+  if (blockDim.x == 1024 && n > 512) {
+    if (n <= 1024) block_sort_reg<1>(hi, pos_out, n);
+    else if (n <= 2048) block_sort_reg<2>(hi, pos_out, n);
+    else if (n <= 4096) block_sort_reg<4>(hi, pos_out, n);
+    else if (n <= 8192) block_sort_reg<8>(hi, pos_out, n);
+    else block_sort_reg<16>(hi, pos_out, n);
+  } else {
+    block_sort<false>(hi, nullptr, n);
+    for (int q = threadIdx.x; q < n; q += blockDim.x) pos_out[q] = (uint32_t)(hi[q] & 0xffffu);
+  }
+}
+
 __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegArgs a, const SegCtx c, int seg_min,
                                                   int seg_cap, int bucket) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -468,8 +484,7 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
       }
       __syncthreads();
       if (!(bucket && n_in > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_in, sh))) {
-        block_sort<false>(s_hi, nullptr, n_in);
-        for (int q = threadIdx.x; q < n_in; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
+        sort64_positions(s_hi, s_lo, n_in);
         __syncthreads();
       }
       for (int q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = sin[s_lo[q]].row;
@@ -504,16 +519,7 @@ __global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegAr
     __syncthreads();
     if (ordered) {
       if (!(bucket && n_act > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_act, sh))) {
-        if (blockDim.x == 1024 && n_act > 512) {      // items in registers: 1, 2, 4, 8 or 16 per thread
-          if (n_act <= 1024) block_sort_reg<1>(s_hi, s_lo, n_act);
-          else if (n_act <= 2048) block_sort_reg<2>(s_hi, s_lo, n_act);
-          else if (n_act <= 4096) block_sort_reg<4>(s_hi, s_lo, n_act);
-          else if (n_act <= 8192) block_sort_reg<8>(s_hi, s_lo, n_act);
-          else block_sort_reg<16>(s_hi, s_lo, n_act);
-        } else {
-          block_sort<false>(s_hi, nullptr, n_act);
-          for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] = (uint32_t)(s_hi[q] & 0xffffu);
-        }
+        sort64_positions(s_hi, s_lo, n_act);
       }
     } else {
       block_sort<true>(s_hi, s_lo, n_act);
