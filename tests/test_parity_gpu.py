@@ -961,3 +961,16 @@ def test_scale_decide_from_summed_counters():
         seen |= set(want[:, 0].tolist())
     assert seen == {-1, 0, 1} and sched.status() != 0      # the shards held rows with ids out of range too
     sched.close()
+
+
+@pytest.mark.parametrize("n", [770, 1024, 1025, 2048, 2049, 4096, 4097, 8192, 8193, 12_345, 16_384])
+def test_medium_segment_sizes_around_the_register_sort_shapes(n):
+    # one replica whose rows are nearly all active: 1, 2, 4, 8 or 16 items per thread in the sorting network, at
+    # and around each boundary; ids in row order (ordered step) and permuted (inactive rows sorted too), ties
+    for permute, tie in ((False, False), (True, True)):
+        wl = gen.random_table(n, n, 1, modes=(gen.COLOCATED,), permute_ids=permute, tie_heavy=tie, inflight=0.2, done=0.0, future=0.0)
+        assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_table(n + 1, n, 1, modes=(gen.DECODE,), permute_ids=False, inflight=0.6, done=0.01, future=0.01, batch_cap=40)
+    assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_table(n + 2, n, 1, modes=(gen.COLOCATED,), permute_ids=True, inflight=0.05, done=0.45, future=0.45)     # mostly inactive
+    assert_step_parity(wl, steps=1, commit=True)
