@@ -412,6 +412,38 @@ def run_gpu(args):
                 elastic_loop.oracle_round(cw_e, cf, k)
             elastic["cpu_oracle_round_ms"] = 1e3 * (time.perf_counter() - t0) / 2
 
+    # ---- the other step configurations (parity cases, not the benchmark line): time of one step each ----------
+    others = None
+    if rank == 0 and not args.no_other_configs:
+        others = {}
+        for name, ow in (("config2", gen.config2()), ("config3", gen.config3())):
+            osched = hfx.Scheduler(ow.model, ow.classes, ow.replicas, ow.n_rows, budget_mode=ow.budget_mode, weight_max=ow.weight_max)
+            otab = hfx.DeviceTable.from_numpy(ow.table)
+            onow = torch.from_numpy(ow.now.copy()).cuda(); omat = torch.from_numpy(ow.maturity.copy()).cuda()
+            oout = hfx.StepOut(ow.n_rows, ow.n_replicas, optional=False)
+            for _ in range(3):
+                osched.step(otab, onow, omat, oout)
+            torch.cuda.synchronize()
+            oevs = []
+            for _ in range(10):
+                flush.fill_(9)
+                a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+                a.record(stream); osched.step(otab, onow, omat, oout); b.record(stream)
+                oevs.append((a, b))
+            torch.cuda.synchronize()
+            o_ms = float(np.mean([a.elapsed_time(b) for a, b in oevs]))
+            osched.get_profile(); osched.set_profiling(True)
+            for _ in range(5):
+                osched.step(otab, onow, omat, oout)
+            oprof = osched.get_profile()
+            others[name] = {"rows": ow.n_rows, "replicas": ow.n_replicas, "ms_per_step": o_ms,
+                            "requests_per_sec": ow.n_rows / (o_ms * 1e-3),
+                            "algorithmic_gbs": 51 * ow.n_rows / (o_ms * 1e-3) / 1e9,
+                            "kernel_us": {k: 1e3 * v["ms"] / v["launches"] for k, v in oprof.items()},
+                            "status": osched.status()}
+            osched.close()
+            del otab, oout
+
     # ---- CPU baseline: the oracle on a bounded sample, rank 0 at N = 1 only -----------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -460,7 +492,7 @@ def run_gpu(args):
                 "clocks": clk, "gpu_launches": launches, "device_status": status,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                         "ms_per_step": e2e_ms_max},
-                "roofline": roof, "cpu_baseline": cpu, "sim": sim, "dispatch": disp, "pd": pd, "elastic": elastic}
+                "roofline": roof, "cpu_baseline": cpu, "sim": sim, "dispatch": disp, "pd": pd, "elastic": elastic, "other_configs": others}
         print(json.dumps(line))
     sched.close()
     if world > 1:
@@ -482,6 +514,7 @@ def main():
     ap.add_argument("--no-dispatch", action="store_true")
     ap.add_argument("--no-pd", action="store_true")
     ap.add_argument("--no-elastic", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true")
     ap.add_argument("--elastic-rounds", type=int, default=600, help="rounds of the scaling loop (the first 20 warm up, the next 60 are timed)")
     args = ap.parse_args()
     if args.impl == "reference":
