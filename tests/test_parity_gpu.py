@@ -816,13 +816,15 @@ def test_scale_apply_hand_worked_sequence():
     sched.close()
 
 
-def test_scaling_loop_round_by_round():
+@pytest.mark.parametrize("first_fit,rounds", [(False, 330), (True, 120)])
+def test_scaling_loop_round_by_round(first_fit, rounds):
     # the whole loop: instances advance to the tick under the horizon, the Scaler ticks, its decisions are carried
     # out, the dispatcher serves the ACTIVE instances that are due, the requests are bound -- compared after each round
     import paper_2508_15919_b200 as hfx
     from oracle.elastic_loop import COLD, SCALE_KW, SUBSTEPS, oracle_round
     R = 8
     wl = gen.elastic(1, R, 1500)
+    wl.meta["first_fit"] = first_fit
     cpu = wl.copy()
     f = gen.new_fleet([2000] * R, [0, 1])
     sched = make_sched(wl)
@@ -834,7 +836,7 @@ def test_scaling_loop_round_by_round():
     counts = torch.zeros((3, 4), dtype=torch.int64, device="cuda"); used = torch.zeros(R, dtype=torch.int64, device="cuda")
     dec = torch.zeros((3, 2), dtype=torch.int32, device="cuda"); cost = torch.zeros(3, dtype=torch.int64, device="cuda")
     on_max = 0
-    for k in range(330):
+    for k in range(rounds):
         o = oracle_round(cpu, f, k)
         sched.set_horizon(o["now"])
         for _ in range(SUBSTEPS):
@@ -857,7 +859,10 @@ def test_scaling_loop_round_by_round():
         assert np.array_equal(now.cpu().numpy(), cpu.now) and np.array_equal(mat.cpu().numpy(), cpu.maturity), k
         on_max = max(on_max, int(np.count_nonzero(f["inst_state"] != gen.INST_OFF)))
     sched.close()
-    assert on_max >= 6 and np.count_nonzero(cpu.table["state"] == gen.DONE) > 700
+    if rounds >= 330:
+        assert on_max >= 6 and np.count_nonzero(cpu.table["state"] == gen.DONE) > 700
+    else:
+        assert on_max >= 3 and np.count_nonzero(cpu.table["state"] == gen.DONE) > 50
 
 
 @pytest.mark.parametrize("R,permute,fused", [(64, False, True), (64, True, True), (4, False, True), (64, False, False), (4, False, False)])
