@@ -225,6 +225,40 @@ def test_prefill_and_decode_stage_budgets():
     assert o["maturity_next"][0] == MS + 8_000_000 + 2 * 100_000 + 20 * 2500
 
 
+def test_decode_stage_queued_slack_hand_worked():
+    """D stage, prefilled request waiting in the queue: slack = first token + (gen+1) TPOT - earliest start -
+    predicted TPOT of the enlarged batch, with the earliest start at the maturity time while the instance is busy."""
+    cls = [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)]
+    rows = [dict(state=gen.RUNNING, prompt_len=900, gen=100, first_token_ns=20 * MS, arrival_ns=5 * MS, class_id=1, req_id=7),
+            dict(prompt_len=500, gen=3, first_token_ns=60 * MS, arrival_ns=10 * MS, class_id=0, req_id=1),
+            dict(prompt_len=2000, gen=0, first_token_ns=90 * MS, arrival_ns=40 * MS, class_id=1, req_id=2)]
+    wl = make_wl(rows, cls, replicas=[(gen.DECODE, 32768, 0)], now=[100 * MS], maturity=[130 * MS])
+    o = oracle.step(wl)
+    assert o["e_d"][0] == PINS["dq_ed"] and o["n_run"][0] == 1 and o["sum_kv"][0] == 1000
+    assert o["slack"][0] == PINS["dq_slack_R0"] and o["pred_tpot"][0] == PINS["dq_ed"]
+    assert o["slack"][1] == PINS["dq_slack_Q1"] and o["pred_tpot"][1] == PINS["dq_ptpot_Q1"]
+    assert o["slack"][2] == PINS["dq_slack_Q2"] and o["pred_tpot"][2] == PINS["dq_ptpot_Q2"]
+    assert o["pred_ttft"][1] == PINS["dq_pttft_Q1"] and o["pred_ttft"][2] == 50 * MS
+    assert o["key"][1] == PINS["dq_key_Q1"] and o["key"][2] == PINS["dq_key_Q2"]
+    assert list(o["order"]) == [0, 1, 2]
+    # busy until maturity: no decision, the maturity time stands
+    assert o["budget"][0] == 0 and o["adm_count"][0] == 0 and o["maturity_next"][0] == 130 * MS
+    assert list(o["admit"]) == [1, 0, 0]
+    # the same instance once matured: the earliest start is now
+    wl = make_wl(rows, cls, replicas=[(gen.DECODE, 32768, 0)], now=[100 * MS], maturity=[90 * MS])
+    o = oracle.step(wl)
+    assert o["slack"][1] == PINS["dq_slack_Q1_matured"] and o["slack"][2] == PINS["dq_slack_Q2_matured"]
+    assert o["slack"][0] == PINS["dq_slack_R0"]
+    assert o["budget"][0] == PINS["dq_budget_matured"] and o["adm_count"][0] == 2
+    assert o["adm_cost"][0] == PINS["dq_adm_cost_matured"] and o["maturity_next"][0] == PINS["dq_maturity_matured"]
+    assert list(o["admit"]) == [1, 1, 1]
+    # a class without a TPOT bound: the slack saturates high and the request goes last in its priority
+    cls2 = cls + [(0, 0, 0)]
+    rows2 = rows + [dict(prompt_len=10, gen=0, first_token_ns=1, arrival_ns=0, class_id=2, req_id=0)]
+    o = oracle.step(make_wl(rows2, cls2, replicas=[(gen.DECODE, 32768, 0)], now=[100 * MS], maturity=[130 * MS]))
+    assert o["slack"][3] == oracle.SLACK_MAX and list(o["order"]) == [0, 1, 3, 2]
+
+
 def test_cap_only_mode_and_batch_cap():
     rows = [dict(prompt_len=3000, req_id=i, arrival_ns=i) for i in range(5)]
     wl = make_wl(rows, C200, replicas=[(gen.COLOCATED, 8192, 2)], now=[MS], budget_mode=gen.BUDGET_CAP_ONLY)

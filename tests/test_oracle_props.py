@@ -77,6 +77,19 @@ def test_step_invariants(wl):
                         if ttft[c] > 0 else oracle.SLACK_MAX)
                 assert o["slack"][i] == want
                 assert o["pred_ttft"][i] == start - t["arrival_ns"][i] + oracle.Ep(wl.model, int(t["prompt_len"][i]))
+        else:
+            # D stage: a prefilled request's slack runs from its token deadline, first token + (gen+1) TPOT,
+            # to the earliest start, net of the step latency the enlarged batch is predicted to have
+            start = max(wl.now[r], wl.maturity[r])
+            d0, d1, d2 = wl.model[3:]
+            for i in rows[visible][:20]:
+                c = t["class_id"][i]
+                kv_i = int(t["prompt_len"][i]) + int(t["gen"][i])
+                ptpot = d0 + d1 * (nrun + 1) + d2 * (int(o["sum_kv"][r]) + kv_i)
+                want = (int(t["first_token_ns"][i]) + (int(t["gen"][i]) + 1) * int(tpot[c]) - int(start) - ptpot
+                        if tpot[c] > 0 else oracle.SLACK_MAX)
+                assert o["slack"][i] == want and o["pred_tpot"][i] == ptpot
+                assert o["pred_ttft"][i] == t["first_token_ns"][i] - t["arrival_ns"][i]
 
 
 @pytest.mark.parametrize("seed", range(6))
