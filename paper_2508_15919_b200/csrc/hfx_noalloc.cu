@@ -76,7 +76,7 @@ extern "C" int hfx_count_rows_noalloc(const int32_t *replica_id, int64_t n_rows,
                                       int32_t *seg_off, uint32_t *n_bad, void *cuda_stream) {
   if (n_replicas < 1 || n_rows < 0 || !seg_off || (n_rows > 0 && !replica_id)) return HFX_E_ARG;
   if (n_replicas > HFX_NOALLOC_MAX_REPLICAS || n_rows > (INT64_C(1) << 27)) return HFX_E_CAPACITY;
-  if ((reinterpret_cast<uintptr_t>(replica_id) | reinterpret_cast<uintptr_t>(seg_off)) & 3u) return HFX_E_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(replica_id) | reinterpret_cast<uintptr_t>(seg_off) | reinterpret_cast<uintptr_t>(n_bad)) & 3u) return HFX_E_ALIGN;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return HFX_E_CUDA; }
   if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return HFX_E_CAPACITY;

@@ -40,3 +40,16 @@ def permute_rows(wl, perm):
     for k in out.table:
         out.table[k] = np.ascontiguousarray(out.table[k][perm])
     return out
+
+
+def oracle_sim_config5_range(args):
+    """Worker of a process pool (importable under `spawn`): the single-threaded oracle on traces
+    [first, first + count) of config 5, drawn afresh from their seeds (a subset of the batch equals
+    the same slice of the full batch).  Returns the per-trace metrics and the table columns the
+    simulator writes."""
+    first, count, iters = args
+    import oracle
+    wl = gen.config5(traces=count, first_trace=first, iters=iters)
+    res = oracle.sim(wl)
+    cols = {k: wl.table[k] for k in ("state", "gen", "first_token_ns", "last_token_ns", "finish_ns")}
+    return first, count, res, cols

@@ -56,10 +56,31 @@ def test_config5_subset_of_traces():
 
 
 def test_config5_full_batch_sampled_traces():
-    # the whole 4096-trace batch in one call (the launch the benchmark times); four traces spread over
-    # the batch are checked against the oracle, the rest through properties that hold for every trace
+    # the whole 4096-trace batch in one call (the launch the benchmark times); 256 traces spread evenly
+    # over the batch (every 16th) are compared with the oracle, which runs as a pool of single-threaded
+    # worker processes over disjoint trace ranges; the rest through properties that hold for every trace
+    import multiprocessing as mp
+    import os
+    from gpu_helpers import SIM_KEYS, STATE_COLS
+    from helpers import oracle_sim_config5_range
     wl = gen.config5()
-    res = assert_sim_parity(wl, traces=[0, 1365, 2730, 4095])
+    T = wl.trace_off.shape[0] - 1
+    picked = list(range(0, T, 16))
+    workers = max(1, min(len(picked), (os.cpu_count() or 1) - 1, 64))
+    # the pool is started with `spawn`: this process may hold a CUDA context already, and a forked child of it hangs
+    with mp.get_context("spawn").Pool(workers) as pool:
+        pending = pool.map_async(oracle_sim_config5_range, [(j, 1, wl.sim_iters) for j in picked], chunksize=1)
+        res, cols, st = run_sim_gpu(wl)
+        done = pending.get(timeout=900)
+    print(f"oracle: {len(picked)} traces on {workers} worker processes of {os.cpu_count()} cores")
+    assert st == 0
+    for first, count, c, ccols in done:
+        a, b = wl.trace_off[first], wl.trace_off[first + count]
+        for ko, kg in SIM_KEYS.items():
+            assert np.array_equal(res[kg][first:first + count], c[ko][:count]), f"trace {first}: {kg}"
+        for k in STATE_COLS:
+            assert np.array_equal(cols[k][a:b], ccols[k]), f"trace {first}: column {k}"
+        assert c["status"] == 0
     assert np.all(res["iters_executed"] <= wl.sim_iters) and np.all(res["iters_executed"] > 0)
     assert np.all(res["attained"] <= res["finished"]) and np.all(res["finished"] + res["rejected"] <= 2048)
     assert np.all(res["ttft_p50_ns"] <= res["ttft_p99_ns"]) and np.all(res["tpot_p50_ns"] <= res["tpot_p99_ns"])

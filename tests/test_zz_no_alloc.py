@@ -39,7 +39,11 @@ def test_two_calls_in_a_row_match_the_step():
         hfx.count_rows_noalloc(rid, wl.n_replicas, seg, bad)
         torch.cuda.synchronize()
         assert np.array_equal(seg.cpu().numpy(), ref)
+        # and against the definition: rows per replica, as an exclusive prefix
         rid_np = wl.table["replica_id"]
+        valid = rid_np[(rid_np >= 0) & (rid_np < wl.n_replicas)]
+        want = np.concatenate([[0], np.cumsum(np.bincount(valid, minlength=wl.n_replicas))]).astype(np.int32)
+        assert np.array_equal(seg.cpu().numpy(), want)
         assert int(bad.item()) == int(((rid_np < 0) | (rid_np >= wl.n_replicas)).sum())
 
 
@@ -52,3 +56,18 @@ def test_limits_are_rejected():
     with pytest.raises(hfx.HfxError) as e:
         hfx.count_rows_noalloc(rid, hfx.NOALLOC_MAX_REPLICAS + 1, torch.zeros(hfx.NOALLOC_MAX_REPLICAS + 2, dtype=torch.int32, device="cuda"))
     assert e.value.code == -3
+
+
+def test_empty_table_and_misaligned_counter():
+    # no rows: every offset is 0 (the kernels still clear what the previous call left)
+    seg = torch.full((6,), -7, dtype=torch.int32, device="cuda")
+    bad = torch.full((1,), 9, dtype=torch.int32, device="cuda")
+    hfx.count_rows_noalloc(torch.zeros(0, dtype=torch.int32, device="cuda"), 5, seg, bad)
+    torch.cuda.synchronize()
+    assert seg.cpu().tolist() == [0] * 6 and int(bad.item()) == 0
+    # a counter address that is not 4-byte aligned is an argument error; nothing is launched
+    raw = torch.zeros(8, dtype=torch.uint8, device="cuda")
+    rid = torch.zeros(16, dtype=torch.int32, device="cuda")
+    with pytest.raises(hfx.HfxError) as e:
+        hfx.count_rows_noalloc(rid, 5, seg, raw[1:5])
+    assert e.value.code == -2
