@@ -9,8 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhfx.so")
-SOURCES = ["hfx_api.cu", "hfx_step.cu", "hfx_regroup.cu", "hfx_segment.cu", "hfx_sim.cu", "hfx_scale.cu", "hfx_dispatch.cu", "hfx_slomap.cu", "hfx_pd.cu", "hfx_metrics.cu", "hfx_fleet.cu", "hfx_noalloc.cu"]
-HEADERS = [os.path.join(CSRC, "hfx_internal.cuh"), os.path.join(ROOT, "include", "hfx.h")]
+SOURCES = ["hfx_api.cu", "hfx_step.cu", "hfx_front.cu", "hfx_regroup.cu", "hfx_segment.cu", "hfx_sim.cu", "hfx_scale.cu", "hfx_dispatch.cu", "hfx_slomap.cu", "hfx_pd.cu", "hfx_metrics.cu", "hfx_fleet.cu", "hfx_noalloc.cu"]
+HEADERS = [os.path.join(CSRC, "hfx_internal.cuh"), os.path.join(CSRC, "hfx_rows.cuh"), os.path.join(ROOT, "include", "hfx.h")]
 
 
 def _stale() -> bool:

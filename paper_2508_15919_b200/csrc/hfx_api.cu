@@ -4,7 +4,7 @@
 
 #include "hfx_internal.cuh"
 
-int hfx_regroup_configure();
+int hfx_front_configure();
 int hfx_segment_configure();
 int hfx_sim_configure();
 int hfx_dispatch_configure();
@@ -68,7 +68,7 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     cudaGetLastError();
     return HFX_E_CUDA;
   }
-  if (hfx_regroup_configure() != HFX_OK || hfx_segment_configure() != HFX_OK || hfx_sim_configure() != HFX_OK || hfx_dispatch_configure() != HFX_OK || hfx_slomap_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
+  if (hfx_front_configure() != HFX_OK || hfx_segment_configure() != HFX_OK || hfx_sim_configure() != HFX_OK || hfx_dispatch_configure() != HFX_OK || hfx_slomap_configure() != HFX_OK) { cudaGetLastError(); return HFX_E_CUDA; }
 
   hfx_sched_host *h = new (std::nothrow) hfx_sched_host();
   if (!h) return HFX_E_NOMEM;
@@ -92,9 +92,6 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
 
   const size_t R2 = (size_t)n_replicas + 2;
   bool ok = true;
-  ok = ok && cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking) == cudaSuccess;
-  ok = ok && cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) == cudaSuccess;
-  ok = ok && cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_cfg, sizeof(hfx_replica_cfg) * n_replicas) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_status, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_mode, (size_t)n_replicas + 16) == cudaSuccess;
@@ -105,24 +102,26 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
   ok = ok && cudaMalloc(&s->d_rowflag, (size_t)max_rows + 16) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_flags, 256) == cudaSuccess;
   {
+    // the tile front end: slabs for every tile of the largest table, one matrix row per tile
     int32_t tile_rows = 0, n_tiles = 0;
-    hfx_tile_shape(max_rows, &tile_rows, &n_tiles);
-    if (n_tiles < HFX_TILE_BLOCKS) n_tiles = HFX_TILE_BLOCKS;
-    s->tile_blocks_max = 0;
-    if (n_replicas <= HFX_TILE_REPLICAS_MAX && 2 * (int64_t)n_tiles * (n_replicas + 1) <= HFX_TILE_MATRIX_MAX) {
-      const size_t cells = (size_t)n_tiles * ((size_t)n_replicas + 1);
-      ok = ok && cudaMalloc(&s->d_tile_hist, sizeof(uint32_t) * 2 * cells) == cudaSuccess;
-      ok = ok && cudaMalloc(&s->d_tile_mode, (size_t)n_tiles + 16) == cudaSuccess;
-      s->tile_blocks_max = n_tiles;
+    hfx_front_shape(s, max_rows, &tile_rows, &n_tiles);
+    if (n_tiles < n_sm + 1) n_tiles = n_sm + 1;      // smaller tables have lower tiles, about one per SM
+    s->tiles_max = 0;
+    if (n_replicas <= HFX_TILE_REPLICAS_MAX && (int64_t)n_tiles * (n_replicas + 1) <= HFX_TILE_MATRIX_MAX) {
+      const size_t slots = (size_t)max_rows + HFX_TILE_ROWS_MAX;
+      ok = ok && cudaMalloc(&s->d_M, sizeof(uint2) * (size_t)n_tiles * ((size_t)n_replicas + 1)) == cudaSuccess;
+      ok = ok && cudaMalloc(&s->d_slab_rec, sizeof(uint4) * slots) == cudaSuccess;
+      ok = ok && cudaMalloc(&s->d_slab_idx, sizeof(uint16_t) * slots) == cudaSuccess;
+      ok = ok && cudaMalloc(&s->d_tot, sizeof(unsigned long long) * 2 * R2) == cudaSuccess;
+      ok = ok && cudaMemset(s->d_tot, 0, sizeof(unsigned long long) * 2 * R2) == cudaSuccess;
+      s->tiles_max = n_tiles;
     }
   }
   ok = ok && cudaMalloc(&s->d_rec, sizeof(HfxRec) * (size_t)max_rows) == cudaSuccess;
-  ok = ok && cudaMalloc(&s->d_barrier, 256) == cudaSuccess;
-  ok = ok && cudaMalloc(&s->d_front_bar, 256) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_slo, hfx_slomap_workspace_bytes()) == cudaSuccess;
   ok = ok && cudaMalloc(&s->d_pd, hfx_pd_workspace_bytes(n_replicas)) == cudaSuccess;
   s->horizon = INT64_MAX;
-  s->front_enabled = 1; s->front_arrivals = 0; s->front_smem_cached = 0; s->front_capacity = 0;
+  s->front_enabled = 1; s->tot_parity = 0;
   ok = ok && cudaMalloc(&h->d_trace_off, sizeof(int32_t) * R2) == cudaSuccess;
   ok = ok && cudaMalloc(&h->d_work_counter, 256) == cudaSuccess;
   if (ok && max_rows > 16384) {   // scratch of the global sort: only tables that can hold an oversize segment
@@ -135,13 +134,12 @@ extern "C" int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
     memcpy(h->h_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas);
     ok = ok && cudaMemcpy(s->d_cfg, replicas, sizeof(hfx_replica_cfg) * n_replicas, cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemset(s->d_status, 0, 256) == cudaSuccess;
-    ok = ok && cudaMemset(s->d_front_bar, 0, 256) == cudaSuccess;
     {
       std::vector<uint8_t> modes((size_t)n_replicas);
       for (int r = 0; r < n_replicas; r++) modes[r] = (uint8_t)replicas[r].mode;
       ok = ok && cudaMemcpy(s->d_mode, modes.data(), (size_t)n_replicas, cudaMemcpyHostToDevice) == cudaSuccess;
     }
-    const uint32_t init_flags[4] = {1u, 1u, 0u, 0u};
+    const uint32_t init_flags[8] = {0u, 0u, 0u, 0u, 1u, 1u, 0u, 0u};
     ok = ok && cudaMemcpy(s->d_flags, init_flags, sizeof(init_flags), cudaMemcpyHostToDevice) == cudaSuccess;
   }
   if (!ok) {
@@ -158,13 +156,11 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   hfx_sched_host *h = reinterpret_cast<hfx_sched_host *>(s);
   cudaStreamSynchronize(s->stream);
   hfx_dispatch_release(s);
-  if (s->side) { cudaStreamSynchronize(s->side); cudaStreamDestroy(s->side); }
-  if (s->ev_fork) cudaEventDestroy(s->ev_fork);
-  if (s->ev_join) cudaEventDestroy(s->ev_join);
   cudaFree(s->d_cfg); cudaFree(s->d_mode); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
-  cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_tile_hist); cudaFree(s->d_rec);
-  cudaFree(s->d_act_count); cudaFree(s->d_rowflag); cudaFree(s->d_tile_mode);
-  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_barrier); cudaFree(s->d_front_bar); cudaFree(s->d_slo); cudaFree(s->d_pd);
+  cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_rec);
+  cudaFree(s->d_act_count); cudaFree(s->d_rowflag);
+  cudaFree(s->d_M); cudaFree(s->d_slab_rec); cudaFree(s->d_slab_idx); cudaFree(s->d_tot);
+  cudaFree(s->d_big_hi); cudaFree(s->d_big_lo); cudaFree(s->d_slo); cudaFree(s->d_pd);
   cudaFree(h->d_trace_off); cudaFree(h->d_work_counter);
   cudaGetLastError();
   if (s->brackets) {
@@ -380,7 +376,7 @@ extern "C" int hfx_sched_get_profile(hfx_sched *s, hfx_profile *out) {
 }
 
 extern "C" const char *hfx_kernel_name(int slot) {
-  static const char *names[] = {"k_count", "k_colscan", "k_offsets", "k_regroup", "k_segment(small)", "k_segment(medium)",
-                                "k_big", "k_sim", "k_scale", "k_front", "k_dispatch", "k_slo_map", "k_pd_migrate", "k_attainment"};
+  static const char *names[] = {"k_count", "(unused)", "k_offsets", "k_regroup_atomic", "k_replicas", "(unused)",
+                                "(unused)", "k_sim", "k_scale", "k_front", "k_dispatch", "k_slo_map", "k_pd_migrate", "k_attainment"};
   return (slot >= 0 && slot < 14) ? names[slot] : nullptr;
 }

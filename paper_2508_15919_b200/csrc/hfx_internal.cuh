@@ -58,15 +58,27 @@ struct __align__(32) HfxRec {
 };
 static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
+// Compact record of an ACTIVE row as the tile front end leaves it (16 bytes, a uint4):
+//   x, y  slack base (int64, as HfxRec::base)
+//   z     prompt_len<25> | kind<1> (KIND_RUNNING / KIND_QUEUED) | prio<6>
+//   w     gen<25> | class<6>
+// The row index travels beside it (16-bit index inside the tile); req_id and output_len are fetched
+// from the table by the few paths that need them.
+#define CREC_LEN_MASK 0x1ffffffu
+#define CREC_KIND_SHIFT 25
+#define CREC_PRIO_SHIFT 26
+#define CREC_CLS_SHIFT 25
+#define HFX_FRONT_SMEM (220 * 1024)      // dynamic shared memory the tile kernel may use
+
 #include <vector>
 
 enum { KSLOT_COUNT = 0, KSLOT_COLSCAN, KSLOT_OFFSETS, KSLOT_REGROUP, KSLOT_SEG_SMALL, KSLOT_SEG_MED, KSLOT_BIG, KSLOT_SIM, KSLOT_SCALE, KSLOT_FRONT, KSLOT_DISPATCH, KSLOT_SLOMAP, KSLOT_PD, KSLOT_METRICS };
 
-// tiling of the streaming passes: about this many tiles (2 per SM), each at most this many rows
-#define HFX_TILE_BLOCKS 296
+// tiling of the front end: one tile per block, at most 8192 rows (16-bit indices inside a tile)
 #define HFX_TILE_ROWS_MAX 8192
-#define HFX_TILE_MATRIX_MAX (INT64_C(8) << 20)   // entries of the tile-histogram matrix (32 MiB)
-#define HFX_TILE_REPLICAS_MAX 4095               // replicas whose counters fit in shared memory
+#define HFX_TILE_MATRIX_MAX (INT64_C(8) << 20)   // entries of the tile matrix (64 MiB)
+#define HFX_TILE_REPLICAS_MAX 4095               // replicas whose counters fit in shared memory (12-bit bucket ids)
+#define HFX_COUNT_TILE_ROWS 4096                 // rows per block of the counting pass of the fallback front end
 
 struct HfxBracket { cudaEvent_t a, b; int slot; };
 
@@ -76,8 +88,6 @@ struct hfx_sched {
   int64_t max_rows;
   int n_sm;
   cudaStream_t stream;
-  cudaStream_t side;        // second stream: the (usually empty) kernels of larger replicas run beside the main one
-  cudaEvent_t ev_fork, ev_join;
   int64_t launches;
   int profiling;
   std::vector<HfxBracket> *brackets;
@@ -85,28 +95,25 @@ struct hfx_sched {
   hfx_replica_cfg *d_cfg;   // [R]
   uint8_t *d_mode;          // [R] replica modes, one byte each
   uint32_t *d_status;       // sticky status word
-  uint32_t *d_seg_count;    // [R+2] rows per replica (+ the bad-replica bucket R)
-  uint32_t *d_act_count;    // [R+2] active rows (in flight or in the visible queue) per replica
-  uint32_t *d_seg_begin;    // [R+2] exclusive prefix of d_seg_count
-  uint32_t *d_cursor;       // [2][R+2] fill cursors of the atomic regroup (active, inactive)
-  uint32_t *d_tile_hist;    // [tile_blocks_max][2][R+1] per-tile histograms: all rows, active rows
-                            // (nullptr: atomic mode only)
-  uint8_t *d_tile_mode;     // [tile_blocks_max] how ranks inside a tile are found (TILE_*)
+  uint32_t *d_seg_count;    // [R+2] rows per replica (+ the bad-replica bucket R)      (fallback front end)
+  uint32_t *d_act_count;    // [R+2] active rows (in flight or in the visible queue) per replica    (fallback)
+  uint32_t *d_seg_begin;    // [R+2] exclusive prefix of d_seg_count                      (fallback)
+  uint32_t *d_cursor;       // [2][R+2] fill cursors of the fallback regroup (active, inactive)
   uint8_t *d_rowflag;       // [max_rows] kind of every row (KIND_*), ROWFLAG_BADREP for a bad replica id
-  int32_t tile_blocks_max;
-  uint32_t step_parity;     // which of the two `ordered` words this step uses
-  uint32_t *d_flags;        // [0],[1] "ordered" (by step parity), [2] largest sort size of a replica
-  HfxRec *d_rec;            // [max_rows]
+  uint32_t *d_flags;        // [0] "ordered" of the fallback front end (never), [4],[5] "ordered" of the tile front end by parity
+  HfxRec *d_rec;            // [max_rows] contiguous records: written by the fallback regroup, or gathered from the
+                            // slabs by the blocks of larger replicas
   uint64_t *d_big_hi;       // sort scratch of oversize segments
   uint32_t *d_big_lo;
-  uint32_t *d_barrier;      // grid barrier words of the oversize path
-  // fused front end (count + column scan + offsets + regroup as one cooperative kernel)
-  unsigned long long *d_front_bar;     // arrivals at its grid barriers, only ever grows
-  unsigned long long front_arrivals;   // host copy of what that word holds once every launch so far is done
+  // tile front end (see hfx_front.cu)
+  uint4 *d_slab_rec;        // [tiles_max * tile_rows] records of active rows, tile-major
+  uint16_t *d_slab_idx;     // [tiles_max * tile_rows] local row indices, tile-major, grouped by replica
+  uint2 *d_M;               // [tiles_max][R+1] where each replica's rows sit in a tile's slabs
+  unsigned long long *d_tot;// [2][R+2] rows | active rows << 32 per replica, by parity
+  int32_t tiles_max;        // matrix rows allocated (0: fallback front end only)
+  uint32_t tot_parity;      // which half of d_tot / which "ordered" word the next tile front end uses
   int64_t horizon;          // commit horizon of the following steps (INT64_MAX: none)
-  int front_enabled;
-  size_t front_smem_cached;            // shared-memory size the capacity below was asked for
-  int front_capacity;                  // blocks of the fused kernel that can be resident at once
+  int front_enabled;        // 0: use the fallback front end (global counters) even where the tile front end fits
   void *dispatch_ws;                   // workspace of hfx_dispatch_step, allocated by its first call
   void *d_slo;                         // per-priority table of hfx_slo_map
   void *d_pd;                          // moved counter, wake-up times and busy flags of hfx_pd_migrate
@@ -507,6 +514,7 @@ struct KernelScope {
 };
 
 // ---- kernel argument blocks ------------------------------------------------------------------
+// the fallback front end (global counters; tables with more replicas than the tile front end takes)
 struct RegroupArgs {
   const int32_t *replica_id; const uint8_t *class_id; const uint8_t *state; const int32_t *prompt_len;
   const int32_t *output_len; const int32_t *gen; const int64_t *arrival; const int64_t *first_token;
@@ -514,19 +522,33 @@ struct RegroupArgs {
   const int64_t *now; const int64_t *mat; const hfx_replica_cfg *cfg; const uint8_t *mode;
   int64_t *pred_ttft;    // optional output
   int64_t n;
-  // outputs of inactive rows, written by the regroup itself when the step is "ordered"
+  // per-row outputs written by the regroup itself
   int64_t *slack; int64_t *pred_tpot; uint64_t *key; int32_t *order; uint8_t *admit; int32_t *admitted_rows;
   uint32_t commit;
 };
 
+// the tile front end
+struct FrontArgs {
+  const int32_t *replica_id; const uint8_t *class_id; const uint8_t *state; const int32_t *prompt_len; const int32_t *gen;
+  const int64_t *arrival; const int64_t *first_token; const int32_t *req_id; const int32_t *weight;
+  const int64_t *now; const int64_t *mat; const uint8_t *mode;
+  int64_t n; int32_t tile_rows; int32_t n_tiles;
+  // per-row outputs, written in row order
+  int64_t *slack; int64_t *pred_ttft; int64_t *pred_tpot; uint64_t *key; uint8_t *admit; uint8_t *rowflag;
+  // the slabs
+  uint4 *slab_rec; uint16_t *slab_idx; uint2 *M; unsigned long long *tot; unsigned long long *tot_next;
+  uint32_t *ordered; uint32_t *ordered_next; uint32_t *status;
+};
+
 struct SegArgs {
-  const int64_t *arrival;   // read-only table column (next arrival of an idle replica)
+  // read-only table columns (fetched by row where a path needs them)
+  const int64_t *arrival; const int32_t *req_id; const int32_t *output_len;
   // table columns written by COMMIT
   uint8_t *state; int32_t *gen; int64_t *first_token; int64_t *last_token; int64_t *finish;
   // replica state
   int64_t *now; int64_t *mat; const hfx_replica_cfg *cfg;
   // outputs
-  int64_t *slack; int64_t *pred_tpot; uint64_t *key; int32_t *order; uint8_t *admit; int32_t *admitted_rows;
+  int64_t *slack; int64_t *pred_tpot; uint64_t *key; int32_t *order; int32_t *seg_off; uint8_t *admit; int32_t *admitted_rows;
   int64_t *budget; int64_t *e_d; int32_t *n_run; int64_t *sum_kv; int64_t *adm_cost; int32_t *adm_count;
   int64_t *maturity_next;
   uint32_t flags;
@@ -534,10 +556,10 @@ struct SegArgs {
 };
 
 // host-side launchers implemented in the .cu files
-void hfx_tile_shape(int64_t n, int32_t *tile_rows, int32_t *n_tiles);
+void hfx_front_shape(const hfx_sched *s, int64_t n, int32_t *tile_rows, int32_t *n_tiles);
+int hfx_launch_front(hfx_sched *s, const FrontArgs &fa);
 int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off);
-size_t hfx_regroup_smem(int R1, int tile_rows);
-int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n);
+int hfx_launch_replicas(hfx_sched *s, const SegArgs &sa, int64_t n, bool slabs);
 int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o, uint32_t flags);
 int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const int64_t *maturity, const hfx_dispatch_out *o,
                         int32_t cap_max);

@@ -1,15 +1,31 @@
-// Per-replica work after the regroup: aggregates of the running batch, E_d, the safe budget
-// (Eq. 3), final slack and key, the sort, segmented-scan admission, maturity, commit.
-//   k_segment  one block per replica whose rows fit in shared memory (two size classes)
-//   k_big      cooperative kernel for larger replicas (global sort with bounded grid barriers)
+// Per-replica work of a step, one persistent kernel (k_replicas, one block of 1024 threads per SM):
+// the replica's rows are gathered from the tile slabs in tile order (= row order), then aggregates of
+// the running batch, E_d, the safe budget (Eq. 3), final slack and key, the sort, segmented-scan
+// admission, maturity, commit.  Three size classes share the kernel:
+//   small    (<= SEG_TINY items to sort)  a group of 128 threads per replica, eight groups per block, each on
+//                                         its own hardware barrier; records staged in shared memory
+//   medium   (<= SEG_MED items)           the whole block; records gathered into a contiguous scratch range
+//   oversize                              the whole block with a sorting network in global memory; slow, it
+//                                         only exists so that any table is handled
+// No block ever waits for another: the only cross-block data are the slabs and totals that the front end
+// finished before this kernel reads them.
+#include <string.h>
+
 #include "hfx_internal.cuh"
 
-#define SEG_SMALL 2048    // rows a small-segment block sorts in shared memory
-#define SEG_MED 16384     // rows a medium-segment block sorts in shared memory
-#define THREADS_SMALL 256
-#define TINY_BLOCKS_PER_SM 4
-#define THREADS_MED 1024
-#define SMEM_SMALL (SEG_SMALL * 20 + (2 * 1024 + 8) * 4)   // sort items, their order, scatter buffer, bins
+#define SEG_TINY 768      // items a 128-thread group sorts
+#define SEG_MED 16384     // items a block sorts in shared memory
+#define REP_THREADS 1024
+#define REP_GROUPS 8
+#define GROUP_THREADS 128
+#define TINY_IPT ((SEG_TINY + GROUP_THREADS - 1) / GROUP_THREADS)     // items per thread
+#define TINY_BINS 1024    // bins of the distribution sort (16-bit counters, two to a word)
+#define TINY_BIN_MAX 48
+#define TINY_CLASSES 128  // (phase, priority) classes of the sort items of active rows: phase<1> | prio<6>
+#define GROUP_TPT 2       // tiles per thread and round when a group gathers
+#define LIST_MAX 2048     // inactive rows a replica's own threads list while they gather; longer lists are shared by the grid
+#define SMEM_MED (SEG_MED * 12)
+#define SMEM_GROUP (SMEM_MED / REP_GROUPS)
 
 struct BlockShared {
   int64_t red_a[32], red_b[32], red_c[32];
@@ -22,68 +38,89 @@ struct BlockShared {
   int32_t adm_count, worked, n_act;
 };
 
-// Distribution sort of distinct 64-bit items for small segments: items are binned by their offset
-// from the smallest item (a shift makes at most SORT_BINS bins, so bins are in key order), scattered
-// bin by bin, and ranked inside their bin by counting smaller items.  Writes the low 16 bits of the
-// items, in ascending item order, to s_lo.  Returns false (uniformly, nothing written) when a bin is
-// too crowded for the counting to pay; the caller then runs the sorting network instead.
-// Needs blockDim.x <= SORT_BINS and SORT_BINS % blockDim.x == 0.  Block-synchronised on entry by the
-// caller and on return.
-#define SORT_BINS 1024
-#define SORT_BIN_MAX 48
-__device__ bool block_bucket_order(const uint64_t *s_hi, uint64_t *s_tmp, uint32_t *s_lo, uint32_t *s_bin,
-                                   uint32_t *s_cur, int n, BlockShared &sh) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  uint64_t mn = ~0ull, mx = 0;
-  for (int q = threadIdx.x; q < n; q += blockDim.x) { const uint64_t v = s_hi[q]; mn = v < mn ? v : mn; mx = v > mx ? v : mx; }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const uint64_t a = __shfl_xor_sync(0xffffffffu, mn, o), b = __shfl_xor_sync(0xffffffffu, mx, o);
-    mn = a < mn ? a : mn; mx = b > mx ? b : mx;
+// where the kernel finds the rows of a replica
+struct SegCtx {
+  // tile front end: slabs
+  const uint4 *slab_rec; const uint16_t *slab_idx; const uint2 *M; const unsigned long long *tot;
+  int32_t tile_rows, n_tiles;
+  // fallback front end: contiguous records, counts and range starts
+  const uint32_t *seg_count; const uint32_t *act_count; const uint32_t *seg_begin;
+  HfxRec *rec;            // contiguous records (fallback: input; slabs: scratch of the larger replicas)
+  const uint32_t *ordered; const uint8_t *rowflag;
+  uint64_t *big_hi; uint32_t *big_lo; uint32_t *big_idx;
+  int32_t slabs;
+};
+
+// A set of threads of the block that synchronise on a hardware barrier of their own (0 = the whole block).
+struct Grp {
+  int tid, n, bar;
+  __device__ __forceinline__ void sync() const { asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(n) : "memory"); }
+  __device__ __forceinline__ int any(int pred) const {
+    int r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.s32 p, %3, 0;\n\tbar.red.or.pred q, %1, %2, p;\n\tselp.s32 %0, 1, 0, q;\n\t}"
+                 : "=r"(r) : "r"(bar), "r"(n), "r"(pred) : "memory");
+    return r;
   }
-  if (lane == 0) { sh.red_m0[warp] = mn; sh.red_m1[warp] = mx; }
-  for (int i = threadIdx.x; i <= SORT_BINS; i += blockDim.x) s_bin[i] = 0;
-  __syncthreads();
-  for (int k = 0; k < nwarp; k++) { const uint64_t a = sh.red_m0[k], b = sh.red_m1[k]; mn = a < mn ? a : mn; mx = b > mx ? b : mx; }
-  const uint64_t range = mx - mn;
-  int sft = 0;
-  if (range >> 10) sft = 64 - __clzll((long long)range) - 10;     // (range >> sft) < SORT_BINS
-  for (int q = threadIdx.x; q < n; q += blockDim.x) atomicAdd(&s_bin[(uint32_t)((s_hi[q] - mn) >> sft)], 1u);
-  __syncthreads();
-  // exclusive scan of the bin counts; the largest bin
-  const int per = SORT_BINS / blockDim.x;
-  const int i0 = threadIdx.x * per;
-  uint32_t sum = 0, big = 0;
-  for (int i = 0; i < per; i++) { const uint32_t c = s_bin[i0 + i]; sum += c; big = c > big ? c : big; }
-  uint32_t v = sum;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) { const uint32_t x = __shfl_xor_sync(0xffffffffu, big, o); big = x > big ? x : big; }
-  if (lane == 31) sh.red_n[warp] = (int32_t)v;
-  if (lane == 0) sh.red_a[warp] = big;
-  __syncthreads();
-  uint32_t pre = 0, bigall = 0;
-  for (int k = 0; k < nwarp; k++) { if (k < warp) pre += (uint32_t)sh.red_n[k]; const uint32_t x = (uint32_t)sh.red_a[k]; bigall = x > bigall ? x : bigall; }
-  if (bigall > SORT_BIN_MAX) { __syncthreads(); return false; }
-  uint32_t run = pre + v - sum;
-  for (int i = 0; i < per; i++) { const uint32_t c = s_bin[i0 + i]; s_bin[i0 + i] = run; s_cur[i0 + i] = run; run += c; }
-  __syncthreads();
-  for (int q = threadIdx.x; q < n; q += blockDim.x) {
-    const uint64_t x = s_hi[q];
-    s_tmp[atomicAdd(&s_cur[(uint32_t)((x - mn) >> sft)], 1u)] = x;
+};
+
+// ---- sorting networks ---------------------------------------------------------------------------
+// Bitonic network with ascending comparators only (mirrored first sub-stage), so the virtual +inf
+// padding beyond n never moves: any n, in place.  Items are distinct, so the result is unique.  Each
+// warp owns a contiguous chunk of E items; stages whose pairs stay inside a chunk need only a warp
+// barrier.  Callers synchronise the group before the call; it is synchronised on return.
+template <bool WIDE>
+__device__ void group_sort(uint64_t *hi, uint32_t *lo, int n, const Grp &G) {
+  if (n > 1) {
+    int n_pad = 2;
+    while (n_pad < n) n_pad <<= 1;
+    const int lane = G.tid & 31, warp = G.tid >> 5, nwarp = G.n >> 5;
+    int E = n_pad / nwarp;
+    if (E < 64) E = 64;
+    if (E > n_pad) E = n_pad;
+    const int c0 = warp * E;
+    const bool has_chunk = c0 < n_pad;
+    const int half = n_pad >> 1;
+    bool local = true;    // the previous stage was chunk-local (or there was none)
+    for (int k = 2; k <= n_pad; k <<= 1) {
+      const int hk = k >> 1;
+      if (k <= E) {   // mirrored sub-stage of merge size k, inside the chunk
+        if (has_chunk)
+          for (int t = lane; t < (E >> 1); t += 32) {
+            const int blk = t / hk, off = t - blk * hk;
+            const int i = c0 + blk * k + off, j = c0 + blk * k + k - 1 - off;
+            if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
+          }
+        __syncwarp();
+      } else {
+        if (local) { G.sync(); local = false; }
+        for (int t = G.tid; t < half; t += G.n) {
+          const int blk = t / hk, off = t - blk * hk;
+          const int i = blk * k + off, j = blk * k + k - 1 - off;
+          if (j < n) cmp_swap<WIDE>(hi, lo, i, j);
+        }
+        G.sync();
+      }
+      for (int j = k >> 2; j > 0; j >>= 1) {
+        if (2 * j <= E) {   // pairs (i, i+j) stay inside an aligned block of 2j <= E items
+          local = true;
+          if (has_chunk)
+            for (int t = lane; t < (E >> 1); t += 32) {
+              const int i = c0 + 2 * t - (t & (j - 1));
+              if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
+            }
+          __syncwarp();
+        } else {
+          if (local) { G.sync(); local = false; }
+          for (int t = G.tid; t < half; t += G.n) {
+            const int i = 2 * t - (t & (j - 1));
+            if (i + j < n) cmp_swap<WIDE>(hi, lo, i, i + j);
+          }
+          G.sync();
+        }
+      }
+    }
   }
-  __syncthreads();
-  for (int e = threadIdx.x; e < n; e += blockDim.x) {
-    const uint64_t x = s_tmp[e];
-    const uint32_t b = (uint32_t)((x - mn) >> sft);
-    const uint32_t g0 = s_bin[b], g1 = s_cur[b];
-    uint32_t rank = 0;
-    for (uint32_t g = g0; g < g1; g++) rank += s_tmp[g] < x ? 1u : 0u;
-    s_lo[g0 + rank] = (uint32_t)(x & 0xffffu);
-  }
-  __syncthreads();
-  return true;
+  G.sync();
 }
 
 // what a record says about its row once the replica's plan is known
@@ -178,15 +215,15 @@ __device__ __forceinline__ void commit_row(const SegArgs &a, const ReplicaPlan &
   }
 }
 
-// where a kernel finds the regrouped table
-struct SegCtx {
-  const HfxRec *rec; const uint32_t *seg_begin; const uint32_t *tot_act; const uint32_t *flags;
-  const uint8_t *rowflag; uint32_t parity;
-};
+// does the commit of this row read its output length?  (rows in flight that advance, and admitted rows)
+__device__ __forceinline__ bool commit_needs_out_len(const ReplicaPlan &pl, int kind, bool adm, int worked) {
+  if (kind == KIND_RUNNING) return !(pl.mode == HFX_PREFILL || (pl.mode == HFX_DECODE && !worked));
+  return kind == KIND_QUEUED && adm;
+}
 
 // Earliest arrival among a replica's rows that have not arrived yet, for the clock jump of an idle
-// replica in an ordered step: the regroup has listed the replica's inactive rows in
-// order[b + n_act .. b + n); their kind bytes say which of them are still to come.
+// replica: the replica's inactive rows are listed in order[b + n_act .. b + n); their kind bytes say
+// which of them are still to come.
 __device__ __forceinline__ int64_t next_arrival_listed(const SegArgs &a, const SegCtx &c, uint32_t b, int64_t n_act, int64_t n,
                                                        int64_t first, int64_t stride) {
   int64_t v = HFX_INF;
@@ -197,15 +234,516 @@ __device__ __forceinline__ int64_t next_arrival_listed(const SegArgs &a, const S
   return v;
 }
 
-// aggregates of a replica's active records into the block's plan (all threads call; result in
-// sh.plan; sh.next_arrival is left at "none")
+// minimum of v over the group into sh.next_arrival (all threads of the group call)
+__device__ __forceinline__ void group_min_arrival(int64_t v, BlockShared &sh, const Grp &G) {
+  const int lane = G.tid & 31, warp = G.tid >> 5, nwarp = G.n >> 5;
+  v = warp_min_i64(v);
+  G.sync();
+  if (lane == 0) sh.red_c[warp] = v;
+  G.sync();
+  if (G.tid == 0) {
+    int64_t m = sh.next_arrival;
+    for (int k = 0; k < nwarp; k++) m = sh.red_c[k] < m ? sh.red_c[k] : m;
+    sh.next_arrival = m;
+  }
+  G.sync();
+}
+
+// ---- gathering a replica's rows from the tile slabs -------------------------------------------------
+// Replica r's chunks are taken in tile order, TPT * G.n tiles per round: a thread reads the chunk
+// descriptors of TPT neighbouring tiles, an exclusive scan over the round's tiles gives each chunk's
+// place inside the replica (row order, since tiles and the rows inside a chunk are in row order); then
+// the round's rows are spread evenly over the threads, each finding its chunk by a binary search over the
+// round's prefixes, a few rows at a time so that their loads are in flight together.
+// emit_act(pos, rec, row) is called once for the pos-th active row, emit_in(pos, row) for the pos-th
+// inactive row (only if list_in; active rows only if take_act).
+// Shared memory: GatherTiles for TPT * G.n tiles.  The slabs were written by the previous kernel: L2 loads.
+struct GatherTiles {
+  uint32_t *pa, *pi;          // [n] active / inactive rows of the replica in the round's earlier tiles
+  uint16_t *oa, *oall, *ca;   // [n] chunk descriptor: first record, first row index, active rows
+  uint32_t *scan;             // [2 * warps + 2]
+};
+__host__ __device__ constexpr size_t gather_tiles_bytes(int n_tiles, int n_threads) { return (size_t)n_tiles * 14 + 4 * (2 * (size_t)(n_threads / 32) + 2); }
+__device__ __forceinline__ GatherTiles gather_tiles_at(unsigned char *smem, int n_tiles, int n_threads) {
+  GatherTiles g;
+  g.pa = reinterpret_cast<uint32_t *>(smem); g.pi = g.pa + n_tiles; g.scan = g.pi + n_tiles;
+  g.oa = reinterpret_cast<uint16_t *>(g.scan + 2 * (n_threads / 32) + 2); g.oall = g.oa + n_tiles; g.ca = g.oall + n_tiles;
+  return g;
+}
+
+template <int NT, int TPT, class ActF, class InF>      // NT = G.n threads, TPT tiles per thread and round; NT * TPT a power of two
+__device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, const Grp &G, const GatherTiles &gt, bool take_act,
+                                               bool list_in, ActF emit_act, InF emit_in) {
+  const int lane = G.tid & 31, w = G.tid >> 5, nw = G.n >> 5;
+  constexpr int round_tiles = NT * TPT;
+  uint32_t base_a = 0, base_i = 0;
+  for (int t0 = 0; t0 < c.n_tiles; t0 += round_tiles) {
+    uint32_t ca[TPT], ci[TPT], oa[TPT], oall[TPT];
+    uint32_t sa = 0, si = 0;
+#pragma unroll
+    for (int e = 0; e < TPT; e++) {
+      const int t = t0 + G.tid * TPT + e;
+      ca[e] = 0; ci[e] = 0; oa[e] = 0; oall[e] = 0;
+      if (t < c.n_tiles) {
+        const uint2 m = __ldcg(c.M + (size_t)t * R1 + r);
+        oall[e] = m.x & 0xffffu; oa[e] = m.y & 0xffffu; ca[e] = m.y >> 16; ci[e] = (m.x >> 16) - ca[e];
+      }
+      sa += ca[e]; si += ci[e];
+    }
+    const uint32_t mine_a = sa, mine_i = si;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t x = __shfl_up_sync(0xffffffffu, sa, o), y = __shfl_up_sync(0xffffffffu, si, o);
+      if (lane >= o) { sa += x; si += y; }
+    }
+    if (t0 > 0) G.sync();      // the previous round still reads the tile arrays
+    if (lane == 31) { gt.scan[2 * w] = sa; gt.scan[2 * w + 1] = si; }
+    G.sync();
+    uint32_t pa = sa - mine_a, pi = si - mine_i, ta = 0, ti = 0;
+    for (int k = 0; k < nw; k++) {
+      const uint32_t x = gt.scan[2 * k], y = gt.scan[2 * k + 1];
+      if (k < w) { pa += x; pi += y; }
+      ta += x; ti += y;
+    }
+#pragma unroll
+    for (int e = 0; e < TPT; e++) {
+      const int lt = G.tid * TPT + e;
+      const bool in = t0 + lt < c.n_tiles;
+      gt.pa[lt] = in ? pa : 0xffffffffu; gt.pi[lt] = in ? pi : 0xffffffffu;
+      gt.oa[lt] = (uint16_t)oa[e]; gt.oall[lt] = (uint16_t)oall[e]; gt.ca[lt] = (uint16_t)ca[e];
+      pa += ca[e]; pi += ci[e];
+    }
+    G.sync();
+    // the chunk that holds the q-th row of the round: the last tile whose prefix is <= q
+    auto chunk_of = [&](const uint32_t *pre, uint32_t q) -> int {
+      int lo = 0;
+#pragma unroll
+      for (int s = round_tiles >> 1; s > 0; s >>= 1) if (pre[lo + s] <= q) lo += s;
+      return lo;
+    };
+    if (take_act)
+      for (uint32_t q0 = G.tid; q0 < ta; q0 += 3 * G.n) {
+        uint4 rec[3];
+        int32_t row[3];
+#pragma unroll
+        for (int e = 0; e < 3; e++) {
+          const uint32_t q = q0 + e * G.n;
+          if (q < ta) {
+            const int lt = chunk_of(gt.pa, q);
+            const uint32_t k = q - gt.pa[lt];
+            const size_t tb = (size_t)(t0 + lt) * c.tile_rows;
+            rec[e] = __ldcg(c.slab_rec + tb + gt.oa[lt] + k);
+            row[e] = (int32_t)(tb + __ldcg(c.slab_idx + tb + gt.oall[lt] + k));
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 3; e++) { const uint32_t q = q0 + e * G.n; if (q < ta) emit_act(base_a + q, rec[e], row[e]); }
+      }
+    if (list_in)
+      for (uint32_t q0 = G.tid; q0 < ti; q0 += 4 * G.n) {
+        int32_t row[4];
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+          const uint32_t q = q0 + e * G.n;
+          if (q < ti) {
+            const int lt = chunk_of(gt.pi, q);
+            const uint32_t k = q - gt.pi[lt];
+            const size_t tb = (size_t)(t0 + lt) * c.tile_rows;
+            row[e] = (int32_t)(tb + __ldcg(c.slab_idx + tb + gt.oall[lt] + gt.ca[lt] + k));
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; e++) { const uint32_t q = q0 + e * G.n; if (q < ti) emit_in(base_i + q, row[e]); }
+      }
+    base_a += ta; base_i += ti;
+  }
+}
+
+// First-fit admission along the order by the first warp of G; marks what it takes in bit 17 of s_lo.
+template <class CostF>
+__device__ __forceinline__ void first_fit_marks(const ReplicaPlan &pl, uint32_t *s_lo, int n_sorted, const Grp &G, CostF cost_of) {
+  if ((G.tid >> 5) == 0) {
+    const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
+    warp_first_fit(n_sorted, pl.budget, room, G.tid & 31, cost_of, [&](int64_t q, bool taken) { if (taken) s_lo[q] |= 0x20000u; });
+  }
+  G.sync();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Small replicas: one group of 128 threads.  What later passes need of the replica's active rows
+// (slack base, record words, row) is staged once in shared memory; sort items live in registers
+// until they are scattered into their bins.
+// ------------------------------------------------------------------------------------------------
+#define SMALL_SMEM (SEG_TINY * 24 + (TINY_BINS + 4) * 4 + TINY_CLASSES * 8)
+static_assert(SMALL_SMEM <= SMEM_GROUP, "a group's arrays fit its share of the block's shared memory");
+
+__device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx &c, const Grp &G, int r, uint32_t b, int n,
+                              int n_act, bool ordered, bool list_in, unsigned char *smem, BlockShared &sh,
+                              const int64_t *s_cls_ttft, const int64_t *s_cls_tpot) {
+  uint64_t *s_bk = reinterpret_cast<uint64_t *>(smem);                     // [SEG_TINY] slack base of every active row; then the sort items, binned
+  uint2 *s_zw = reinterpret_cast<uint2 *>(s_bk + SEG_TINY);                // [SEG_TINY] record words z, w; bit 31 of w: admitted
+  int32_t *s_row = reinterpret_cast<int32_t *>(s_zw + SEG_TINY);           // [SEG_TINY]
+  uint32_t *s_lo = reinterpret_cast<uint32_t *>(s_row + SEG_TINY);         // [SEG_TINY] order (+ tie-break words)
+  uint32_t *s_bin = s_lo + SEG_TINY;                                       // [TINY_BINS / 2 + 4] bin counts, then bin starts; two 16-bit values to a word
+  uint32_t *s_cur = s_bin + TINY_BINS / 2 + 4;                             // [TINY_BINS / 2] fill cursors, then bin ends
+  uint2 *s_cinfo = reinterpret_cast<uint2 *>(s_cur + TINY_BINS / 2);       // [TINY_CLASSES] per class: smallest sub-key; first bin | shift << 16
+  // over s_lo .. s_cur while the gather runs: the round's tile descriptors
+  const GatherTiles gt = gather_tiles_at(reinterpret_cast<unsigned char *>(s_lo), GROUP_THREADS * GROUP_TPT, GROUP_THREADS);
+  // over s_lo until the ranks are written: per class the smallest and largest sub-key and the number of items
+  uint32_t *s_cmin = s_lo, *s_cmax = s_lo + TINY_CLASSES, *s_ccnt = s_lo + 2 * TINY_CLASSES;
+  const int R = p.n_replicas, R1 = R + 1;
+  const int lane = G.tid & 31, warp = G.tid >> 5, nwarp = G.n >> 5;
+  const int n_in = n - n_act;
+  const bool real = r < R;    // bucket R holds rows bound to no replica
+  const HfxRec *seg = c.rec + b;   // (fallback layout only)
+
+  // the replica's state, asked for early by the planning warp and used after the gather
+  hfx_replica_cfg cfg; cfg.mode = HFX_COLOCATED; cfg.token_cap = 1; cfg.batch_cap = 0;
+  int64_t now = 0, mat = 0;
+  if (warp == 0 && real) { cfg = a.cfg[r]; now = a.now[r]; mat = a.mat[r]; }
+
+  // ---- a step that is not ordered: the inactive rows, listed by req_id behind the active ones --------
+  if (!ordered && n_in > 0) {
+    if (c.slabs)
+      gather_replica<GROUP_THREADS, GROUP_TPT>(c, R1, r, G, gt, false, true, [](uint32_t, const uint4, int32_t) {},
+                                               [&](uint32_t pos, int32_t row) { s_row[pos] = row; });
+    else
+      for (int q = G.tid; q < n_in; q += G.n) s_row[q] = (int32_t)__ldg(reinterpret_cast<const uint4 *>(seg + n_act + q)).w;
+    G.sync();
+    for (int q = G.tid; q < n_in; q += G.n) s_bk[q] = ((uint64_t)((uint32_t)__ldg(a.req_id + s_row[q]) ^ 0x80000000u) << 16) | (uint32_t)q;
+    G.sync();
+    group_sort<false>(s_bk, nullptr, n_in, G);
+    for (int q = G.tid; q < n_in; q += G.n) a.order[b + n_act + q] = s_row[s_bk[q] & 0xffffu];
+    G.sync();
+  }
+
+  // ---- gather: base, record words and row of the active rows; the inactive rows' places; aggregates ----
+  uint32_t n_run = 0;
+  int64_t sum_kv = 0;
+  uint64_t m_run = 0, m_q = 0;
+  auto take = [&](uint32_t pos, const uint4 rec, int32_t row) {
+    s_bk[pos] = ((uint64_t)rec.y << 32) | rec.x; s_zw[pos] = make_uint2(rec.z, rec.w); s_row[pos] = row;
+    const uint32_t cls = rec.w >> CREC_CLS_SHIFT;
+    if (((rec.z >> CREC_KIND_SHIFT) & 1u) == KIND_RUNNING) {
+      n_run++; sum_kv += (int64_t)(rec.z & CREC_LEN_MASK) + (rec.w & CREC_LEN_MASK); m_run |= 1ull << cls;
+    } else m_q |= 1ull << cls;
+  };
+  if (c.slabs) {
+    gather_replica<GROUP_THREADS, GROUP_TPT>(c, R1, r, G, gt, true, ordered && list_in, take,
+                                             [&](uint32_t pos, int32_t row) { a.order[b + n_act + pos] = row; });
+  } else {
+    for (int q = G.tid; q < n_act; q += G.n) {
+      const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
+      const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
+      uint4 rec;
+      rec.x = w0.x; rec.y = w0.y;
+      rec.z = w1.x | (((w1.w >> 8) & 1u) << CREC_KIND_SHIFT) | (((w1.w >> 16) & 0x3fu) << CREC_PRIO_SHIFT);
+      rec.w = w1.y | ((w1.w & 0x3fu) << CREC_CLS_SHIFT);
+      take((uint32_t)q, rec, (int32_t)w0.w);
+    }
+  }
+
+  // ---- aggregates -> plan ----------------------------------------------------------------------------
+  n_run = __reduce_add_sync(0xffffffffu, n_run);
+  sum_kv = warp_sum_i64(sum_kv);
+  m_run = ((uint64_t)__reduce_or_sync(0xffffffffu, (uint32_t)(m_run >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)m_run);
+  m_q = ((uint64_t)__reduce_or_sync(0xffffffffu, (uint32_t)(m_q >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)m_q);
+  G.sync();       // the gather is over: its tile descriptors may be overwritten
+  if (lane == 0) { sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_m0[warp] = m_run; sh.red_m1[warp] = m_q; }
+  for (int i = G.tid; i < TINY_BINS / 2 + 2; i += G.n) s_bin[i] = 0;
+  for (int i = G.tid; i < TINY_CLASSES; i += G.n) { s_cmin[i] = 0xffffffffu; s_cmax[i] = 0; s_ccnt[i] = 0; }
+  G.sync();
+  if (warp == 0) {     // the whole first warp finishes the reduction and plans
+    int64_t nr = 0, kv = 0;
+    uint64_t mr = 0, mq = 0;
+    for (int k = 0; k < nwarp; k++) { nr += sh.red_a[k]; kv += sh.red_b[k]; mr |= sh.red_m0[k]; mq |= sh.red_m1[k]; }
+    ReplicaPlan pl0;
+    warp_plan(p, s_cls_ttft, s_cls_tpot, cfg, now, mat, nr, kv, mr, mq, pl0, lane);
+    if (lane == 0) { sh.plan = pl0; sh.next_arrival = HFX_INF; }
+  }
+  G.sync();
+  const ReplicaPlan pl = sh.plan;
+
+  // ---- keys (in registers); per class their range ---------------------------------------------------
+  uint64_t item[TINY_IPT];
+#pragma unroll
+  for (int k = 0; k < TINY_IPT; k++) {
+    const int q = G.tid + k * GROUP_THREADS;
+    item[k] = ~0ull;
+    if (q < n_act) {
+      const int64_t base = (int64_t)s_bk[q];
+      const uint2 zw = s_zw[q];
+      const int kind = (zw.x >> CREC_KIND_SHIFT) & 1, prio = zw.x >> CREC_PRIO_SHIFT;
+      const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)(zw.x & CREC_LEN_MASK), (int32_t)(zw.y & CREC_LEN_MASK));
+      if (ordered) {
+        item[k] = (e.k48 << 16) | (uint32_t)q;     // rows were gathered in req_id order: position breaks ties
+        const uint32_t cl = (uint32_t)(item[k] >> 56), sub = (uint32_t)(item[k] >> 24);
+        atomicMin(&s_cmin[cl], sub); atomicMax(&s_cmax[cl], sub); atomicAdd(&s_ccnt[cl], 1u);
+      } else {
+        const uint32_t uid = (uint32_t)__ldg(a.req_id + s_row[q]) ^ 0x80000000u;
+        s_bk[q] = (e.k48 << 16) | (uid >> 16);
+        s_lo[q] = (uid << 16) | (uint32_t)q;
+      }
+      if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the front end wrote the slack of the other queued rows)
+        const int32_t row = s_row[q];
+        a.slack[row] = e.slack;
+        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+      }
+      if (a.pred_tpot) a.pred_tpot[s_row[q]] = e.pred_tpot;
+    }
+  }
+
+  // ---- sort --------------------------------------------------------------------------------------------
+  // Distribution sort.  The top 8 bits of an item are its class (phase, priority); inside a class items are
+  // spread over the class's share of the bins by their sub-key (slack >> 8) between the class's smallest and
+  // largest, so bins stay in item order; an item's place inside its bin comes from counting the smaller
+  // items of the bin.
+  bool sorted_done = false;
+  if (ordered && n_act > 0) {
+    G.sync();
+    if (warp == 0) {     // bins per class in proportion to its items (a power of two), the shift that fits its range
+      uint32_t nb[TINY_CLASSES / 32], sft[TINY_CLASSES / 32], lo_[TINY_CLASSES / 32];
+      uint32_t sum = 0;
+#pragma unroll
+      for (int e = 0; e < TINY_CLASSES / 32; e++) {
+        const int cl = lane * (TINY_CLASSES / 32) + e;
+        const uint32_t cnt = s_ccnt[cl], lo = s_cmin[cl], hi = s_cmax[cl];
+        uint32_t want = cnt * (TINY_BINS - TINY_CLASSES) / (uint32_t)n_act;      // the shares add up to at most TINY_BINS - TINY_CLASSES
+        nb[e] = cnt ? (want > 1 ? 1u << (31 - __clz(want)) : 1u) : 0u;
+        const uint32_t range = cnt ? hi - lo : 0u;
+        const int bits = 32 - __clz(range), lg = 31 - __clz(nb[e] | 1u);
+        sft[e] = bits > lg ? (uint32_t)(bits - lg) : 0u;       // (range >> sft) < nb
+        lo_[e] = lo;
+        sum += nb[e];
+      }
+      uint32_t v = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+      uint32_t run = v - sum;
+#pragma unroll
+      for (int e = 0; e < TINY_CLASSES / 32; e++) { s_cinfo[lane * (TINY_CLASSES / 32) + e] = make_uint2(lo_[e], run | (sft[e] << 16)); run += nb[e]; }
+    }
+    G.sync();
+    auto bin_of = [&](uint64_t x) -> uint32_t {
+      const uint2 ci = s_cinfo[(uint32_t)(x >> 56)];
+      return (ci.y & 0xffffu) + (((uint32_t)(x >> 24) - ci.x) >> (ci.y >> 16));
+    };
+    uint32_t bins[TINY_IPT];
+#pragma unroll
+    for (int k = 0; k < TINY_IPT; k++) {
+      bins[k] = 0;
+      if (G.tid + k * GROUP_THREADS < n_act) { bins[k] = bin_of(item[k]); atomicAdd(&s_bin[bins[k] >> 1], 1u << ((bins[k] & 1u) * 16)); }
+    }
+    G.sync();
+    {   // exclusive scan of the 1024 bin counts: 8 per thread; the largest bin
+      const uint4 wd = reinterpret_cast<const uint4 *>(s_bin)[G.tid];
+      const uint32_t ww[4] = {wd.x, wd.y, wd.z, wd.w};
+      uint32_t cnt[8], sum = 0, big = 0;
+#pragma unroll
+      for (int i = 0; i < 4; i++) { cnt[2 * i] = ww[i] & 0xffffu; cnt[2 * i + 1] = ww[i] >> 16; }
+#pragma unroll
+      for (int i = 0; i < 8; i++) { sum += cnt[i]; big = cnt[i] > big ? cnt[i] : big; }
+      uint32_t v = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+      big = __reduce_max_sync(0xffffffffu, big);
+      if (lane == 31) sh.red_n[warp] = (int32_t)v;
+      if (lane == 0) sh.red_n[8 + warp] = (int32_t)big;
+      G.sync();
+      uint32_t run = v - sum, bigall = 0;
+      for (int k = 0; k < nwarp; k++) { if (k < warp) run += (uint32_t)sh.red_n[k]; const uint32_t x = (uint32_t)sh.red_n[8 + k]; bigall = x > bigall ? x : bigall; }
+      if (bigall <= TINY_BIN_MAX) {
+        uint32_t st[8];
+#pragma unroll
+        for (int i = 0; i < 8; i++) { st[i] = run; run += cnt[i]; }
+        const uint4 o4 = make_uint4(st[0] | (st[1] << 16), st[2] | (st[3] << 16), st[4] | (st[5] << 16), st[6] | (st[7] << 16));
+        reinterpret_cast<uint4 *>(s_bin)[G.tid] = o4;
+        reinterpret_cast<uint4 *>(s_cur)[G.tid] = o4;
+        sorted_done = true;
+      }
+    }
+    G.sync();
+    if (sorted_done) {
+#pragma unroll
+      for (int k = 0; k < TINY_IPT; k++)
+        if (G.tid + k * GROUP_THREADS < n_act) {
+          const uint32_t sh16 = (bins[k] & 1u) * 16;
+          const uint32_t pos = (atomicAdd(&s_cur[bins[k] >> 1], 1u << sh16) >> sh16) & 0xffffu;
+          s_bk[pos] = item[k];
+        }
+      G.sync();
+#pragma unroll
+      for (int k = 0; k < TINY_IPT; k++) {
+        const int e = G.tid + k * GROUP_THREADS;
+        if (e < n_act) {
+          const uint64_t x = s_bk[e];
+          const uint32_t bi = bin_of(x), sh16 = (bi & 1u) * 16;
+          const uint32_t g0 = (s_bin[bi >> 1] >> sh16) & 0xffffu, g1 = (s_cur[bi >> 1] >> sh16) & 0xffffu;
+          uint32_t rank = 0;
+          for (uint32_t g = g0; g < g1; g++) rank += s_bk[g] < x ? 1u : 0u;
+          s_lo[g0 + rank] = (uint32_t)(x & 0xffffu);      // (the class ranges that s_lo overlays were last read when the bins were laid out)
+        }
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < TINY_IPT; k++) { const int q = G.tid + k * GROUP_THREADS; if (q < n_act) s_bk[q] = item[k]; }
+    }
+  }
+  G.sync();
+  if (!sorted_done) {
+    if (ordered) {
+      group_sort<false>(s_bk, nullptr, n_act, G);
+      for (int q = G.tid; q < n_act; q += G.n) s_lo[q] = (uint32_t)(s_bk[q] & 0xffffu);
+    } else {
+      group_sort<true>(s_bk, s_lo, n_act, G);
+      for (int q = G.tid; q < n_act; q += G.n) s_lo[q] &= 0xffffu;
+    }
+    G.sync();
+  }
+
+  auto cost_at = [&](uint32_t li, int64_t &kv) -> int64_t {      // cost of the queued row at record li, -1 if it is in flight
+    const uint2 zw = s_zw[li];
+    if (((zw.x >> CREC_KIND_SHIFT) & 1u) != KIND_QUEUED) return -1;
+    kv = (int64_t)(zw.x & CREC_LEN_MASK) + (zw.y & CREC_LEN_MASK);
+    return pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(zw.x & CREC_LEN_MASK);
+  };
+
+  // ---- first-fit variant: the first warp walks the order and marks what it takes (bit 17) -----------
+  if (p.first_fit)
+    first_fit_marks(pl, s_lo, n_act, G, [&](int64_t q) -> int64_t { int64_t kv; return cost_at(s_lo[q] & 0xffffu, kv); });
+
+  // ---- admission: each thread walks TINY_IPT consecutive places of the order ---------------------
+  const int q0 = G.tid * TINY_IPT;
+  uint32_t cand[TINY_IPT];      // record position of the candidate at each of my places | 0x80000000, or 0
+  uint64_t mine = 0;            // cost | count << 48 of the candidates of this thread (costs stay below 2^44 in total)
+#pragma unroll
+  for (int k = 0; k < TINY_IPT; k++) {
+    const int q = q0 + k;
+    cand[k] = 0;
+    if (q < n_act) {
+      const uint32_t li = s_lo[q] & 0xffffu;
+      int64_t kv = 0;
+      const int64_t cc = cost_at(li, kv);
+      // what counts towards the totals: rows that fit alone, or (first fit) exactly the rows taken
+      if (cc >= 0 && (p.first_fit ? (s_lo[q] & 0x20000u) != 0 : cc <= pl.budget)) { cand[k] = li | 0x80000000u; mine += (uint64_t)cc + (1ull << 48); }
+      a.order[b + q] = s_row[li];
+    }
+  }
+  uint64_t sc = (uint64_t)warp_incl_scan_i64((int64_t)mine, lane);
+  if (lane == 31) sh.red_m0[warp] = sc;
+  G.sync();
+  uint64_t run = sc - mine;
+  for (int k = 0; k < warp; k++) run += sh.red_m0[k];
+  int64_t run_c = (int64_t)(run & ((1ull << 48) - 1));
+  int32_t run_n = (int32_t)(run >> 48);
+  int64_t ac = 0, ak = 0;
+  int32_t an = 0;
+#pragma unroll
+  for (int k = 0; k < TINY_IPT; k++) {
+    if (cand[k]) {
+      const uint32_t li = cand[k] & 0xffffu;
+      int64_t kv = 0;
+      const int64_t cc = cost_at(li, kv);
+      run_c += cc; run_n += 1;
+      if (p.first_fit || (run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap))) {
+        ac += cc; ak += kv; an++;
+        const int32_t row = s_row[li];
+        a.admit[row] = 1;
+        if (a.admitted_rows) a.admitted_rows[b + run_n - 1] = row;
+        s_zw[li].y |= 0x80000000u;
+      }
+    }
+  }
+
+  // ---- totals, maturity, replica outputs, commit ---------------------------------------------------------
+  ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)__reduce_add_sync(0xffffffffu, (uint32_t)an);
+  if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_n[warp] = an; }
+  G.sync();
+  if (G.tid == 0) {
+    int64_t adm_cost = 0, adm_kv = 0; int32_t adm_count = 0;
+    for (int k = 0; k < nwarp; k++) { adm_cost += sh.red_a[k]; adm_kv += sh.red_b[k]; adm_count += sh.red_n[k]; }
+    int64_t lp = 0;
+    const int64_t mat_next = dev_maturity_next(p, pl, adm_count, adm_cost, adm_kv, &lp);
+    int worked; int64_t t1, t2;
+    iteration_clock(pl, adm_count, lp, mat_next, worked, t1, t2);
+    sh.adm_cost = adm_cost; sh.adm_count = adm_count;
+    sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
+  }
+  G.sync();
+  const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
+  const int worked = sh.worked;
+  const int64_t mat_next = sh.red_c[0];
+  if (commit && !worked) {
+    // idle replica: its next arrival is looked up among its listed inactive rows (unless the grid lists them later)
+    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, G.tid, G.n) : HFX_INF, sh, G);
+  }
+  if (G.tid == 0 && real)
+    write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
+  if (a.admitted_rows)
+    for (int q = sh.adm_count + G.tid; q < n; q += G.n) a.admitted_rows[b + q] = -1;
+  if (commit) {      // every thread its own rows: the output lengths it needs are asked for together
+    const int64_t t1 = sh.t1, t2 = sh.t2;
+    int32_t out_len[TINY_IPT];
+#pragma unroll
+    for (int k = 0; k < TINY_IPT; k++) {
+      const int q = G.tid + k * GROUP_THREADS;
+      out_len[k] = 0;
+      if (q < n_act) {
+        const uint2 zw = s_zw[q];
+        if (commit_needs_out_len(pl, (zw.x >> CREC_KIND_SHIFT) & 1, (zw.y >> 31) != 0, worked)) out_len[k] = __ldg(a.output_len + s_row[q]);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < TINY_IPT; k++) {
+      const int q = G.tid + k * GROUP_THREADS;
+      if (q < n_act) {
+        const uint2 zw = s_zw[q];
+        commit_row(a, pl, (zw.x >> CREC_KIND_SHIFT) & 1, (zw.y >> 31) != 0, worked, t1, t2, s_row[q], (int32_t)(zw.x & CREC_LEN_MASK),
+                   (int32_t)(zw.y & CREC_LEN_MASK), out_len[k]);
+      }
+    }
+  }
+  G.sync();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Larger replicas: the whole block.  Their records are first gathered into the contiguous scratch range
+// [b, b + n) of c.rec (32-byte records, active rows first), which the passes below read by position.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_rec(const HfxRec *rec, int half) { return *(reinterpret_cast<const uint4 *>(rec) + half); }
+
+__device__ void gather_to_records(const SegArgs &a, const SegCtx &c, int R1, int r, uint32_t b, int64_t n_act, bool ordered,
+                                  bool list_in, unsigned char *smem) {
+  const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
+  HfxRec *seg = c.rec + b;
+  gather_replica<REP_THREADS, 1>(c, R1, r, B, gather_tiles_at(smem, REP_THREADS, REP_THREADS), true, list_in || !ordered,
+                 [&](uint32_t pos, const uint4 rec, int32_t row) {
+                   uint4 w0, w1;
+                   w0.x = rec.x; w0.y = rec.y; w0.z = ordered ? 0u : (uint32_t)__ldg(a.req_id + row); w0.w = (uint32_t)row;
+                   w1.x = rec.z & CREC_LEN_MASK; w1.y = rec.w & CREC_LEN_MASK; w1.z = 0;
+                   w1.w = (rec.w >> CREC_CLS_SHIFT) | (((rec.z >> CREC_KIND_SHIFT) & 1u) << 8) | ((rec.z >> CREC_PRIO_SHIFT) << 16);
+                   uint4 *dst = reinterpret_cast<uint4 *>(seg + pos);
+                   dst[0] = w0; dst[1] = w1;
+                 },
+                 [&](uint32_t pos, int32_t row) {
+                   if (ordered) a.order[b + n_act + pos] = row;
+                   else {
+                     uint4 *dst = reinterpret_cast<uint4 *>(seg + n_act + pos);
+                     dst[0] = make_uint4(0u, 0u, (uint32_t)__ldg(a.req_id + row), (uint32_t)row);
+                     dst[1] = make_uint4(0u, 0u, 0u, KIND_DEAD << 8);
+                   }
+                 });
+  __syncthreads();
+}
+
+// aggregates of a replica's active records into the block's plan (all threads call; result in sh.plan)
 __device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &a, const HfxRec *seg, int64_t n_act, int r,
                                              bool real, BlockShared &sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   int64_t n_run = 0, sum_kv = 0;
   uint64_t m_run = 0, m_q = 0;
   for (int64_t q = threadIdx.x; q < n_act; q += blockDim.x) {
-    const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);   // prompt, gen, output_len, bytes
+    const uint4 w1 = ld_rec(seg + q, 1);   // prompt, gen, -, bytes
     const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
     if (kind == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
     else m_q |= 1ull << cls;
@@ -227,22 +765,6 @@ __device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &
   __syncthreads();
 }
 
-// block-wide minimum into sh.next_arrival (all threads call)
-__device__ __forceinline__ void block_min_arrival(int64_t v, BlockShared &sh) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  v = warp_min_i64(v);
-  __syncthreads();
-  if (lane == 0) sh.red_c[warp] = v;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int64_t m = sh.next_arrival;
-    for (int k = 0; k < nwarp; k++) m = sh.red_c[k] < m ? sh.red_c[k] : m;
-    sh.next_arrival = m;
-  }
-  __syncthreads();
-}
-
-
 // Block-wide admission over the sorted items s_lo[0..n_sorted) (low 16 bits = position of the
 // record inside the segment): writes order, admit and the compacted admitted list, keeps each
 // decision in bit 16 of s_lo, accumulates the totals in sh.
@@ -250,28 +772,21 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
                                               const HfxRec *seg, uint32_t b, uint32_t *s_lo, int n_sorted,
                                               BlockShared &sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  if (p.first_fit) {       // the first warp walks the order and marks what it takes (bit 17)
-    if (warp == 0) {
-      const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
-      warp_first_fit(n_sorted, pl.budget, room, lane,
-                     [&](int64_t q) -> int64_t {
-                       const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + (s_lo[q] & 0xffffu)) + 1);
-                       if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
-                       return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
-                     },
-                     [&](int64_t q, bool taken) { if (taken) s_lo[q] |= 0x20000u; });
-    }
-    __syncthreads();
+  if (p.first_fit) {
+    const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
+    first_fit_marks(pl, s_lo, n_sorted, B, [&](int64_t q) -> int64_t {
+      const uint4 w1 = ld_rec(seg + (s_lo[q] & 0xffffu), 1);
+      if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
+      return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
+    });
   }
-  // The order begins with the requests in flight (phase 0 sorts first): they are listed and marked, no
+  // The order begins with the requests in flight (phase 0 sorts first): they are only listed, no
   // prefix is needed for them.  Whole tiles of them are passed here; the scan starts at the tile that
   // reaches the queue.
   const int n_front = (int)((pl.n_run < n_sorted ? pl.n_run : n_sorted) / blockDim.x) * blockDim.x;
   for (int q = threadIdx.x; q < n_front; q += blockDim.x) {
     const uint32_t li = s_lo[q] & 0xffffu;
-    const int32_t row = (int32_t)__ldg(reinterpret_cast<const uint4 *>(seg + li)).w;
-    a.order[b + q] = row;
-    a.admit[row] = 1;
+    a.order[b + q] = (int32_t)ld_rec(seg + li, 0).w;
     s_lo[q] = li;
   }
   for (int tile = n_front; tile < n_sorted; tile += blockDim.x) {
@@ -280,8 +795,8 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     int32_t cnt = 0, row = -1, kind = KIND_DEAD;
     if (q < n_sorted) {
       const int li = s_lo[q] & 0xffff;
-      const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
-      const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
+      const uint4 w0 = ld_rec(seg + li, 0);
+      const uint4 w1 = ld_rec(seg + li, 1);
       row = (int32_t)w0.w;
       kind = (w1.w >> 8) & 0xff;
       if (kind == KIND_QUEUED) {
@@ -292,10 +807,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
       a.order[b + q] = row;
     }
     if (!__syncthreads_or(cnt)) {      // no candidate in this tile (a spent budget, requests in flight): nothing to add up
-      if (q < n_sorted) {
-        if (kind == KIND_RUNNING) a.admit[row] = 1;
-        s_lo[q] &= 0xffffu;
-      }
+      if (q < n_sorted) s_lo[q] &= 0xffffu;
       continue;
     }
     // block-wide inclusive scan of (cost, cnt) with carry
@@ -315,7 +827,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     bool adm = false;
     if (cnt) adm = p.first_fit || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
     if (q < n_sorted) {
-      if (kind == KIND_RUNNING || adm) a.admit[row] = 1;
+      if (adm) a.admit[row] = 1;
       if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
       s_lo[q] = (s_lo[q] & 0xffffu) | (adm ? 0x10000u : 0u);
     }
@@ -337,7 +849,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
         (sh.carry_cost > pl.budget || (pl.batch_cap != 0 && pl.n_eff + sh.carry_count >= pl.batch_cap))) {
       for (int q = tile + blockDim.x + threadIdx.x; q < n_sorted; q += blockDim.x) {
         const uint32_t li = s_lo[q] & 0xffffu;
-        a.order[b + q] = (int32_t)__ldg(reinterpret_cast<const uint4 *>(seg + li)).w;
+        a.order[b + q] = (int32_t)ld_rec(seg + li, 0).w;
         s_lo[q] = li;
       }
       break;
@@ -345,7 +857,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
   }
 }
 
-// The sorting network of block_sort for items of one 64-bit word (ordered steps), with the items held in
+// The sorting network for items of one 64-bit word (ordered steps), with the items held in
 // registers: thread t of the 1024 owns the items IPT*t .. IPT*t + IPT-1 (IPT * 1024 = the padded length).
 // Every pair of the network is (i, i ^ mask): mask = k-1 in the mirrored first sub-stage of merge size k,
 // a single bit j afterwards; the lower index keeps the smaller item.  Masks below IPT stay inside a
@@ -432,463 +944,117 @@ __device__ void block_sort_reg(uint64_t *hi, uint32_t *pos_out, int n) {
 }
 
 // Sort n distinct 64-bit items (block-synchronised on entry) and write their low 16 bits, in ascending item
-// order, to pos_out; the caller synchronises before reading pos_out.  1024-thread blocks keep the items in
-// registers (1, 2, 4, 8 or 16 per thread) for more than 512 items.
+// order, to pos_out; the caller synchronises before reading pos_out.
 __device__ __forceinline__ void sort64_positions(uint64_t *hi, uint32_t *pos_out, int n) {
-  if (blockDim.x == 1024 && n > 512) {
+  if (n > 512) {
     if (n <= 1024) block_sort_reg<1>(hi, pos_out, n);
     else if (n <= 2048) block_sort_reg<2>(hi, pos_out, n);
     else if (n <= 4096) block_sort_reg<4>(hi, pos_out, n);
     else if (n <= 8192) block_sort_reg<8>(hi, pos_out, n);
     else block_sort_reg<16>(hi, pos_out, n);
   } else {
-    block_sort<false>(hi, nullptr, n);
+    const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
+    group_sort<false>(hi, nullptr, n, B);
     for (int q = threadIdx.x; q < n; q += blockDim.x) pos_out[q] = (uint32_t)(hi[q] & 0xffffu);
   }
 }
 
-__global__ void __launch_bounds__(1024) k_segment(const HfxParams p, const SegArgs a, const SegCtx c, int seg_min,
-                                                  int seg_cap, int bucket) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint64_t *s_hi = reinterpret_cast<uint64_t *>(smem_raw);
-  uint32_t *s_lo = reinterpret_cast<uint32_t *>(smem_raw + (size_t)seg_cap * 8);
-  // only with `bucket`: scratch of the distribution sort
-  uint64_t *s_tmp = reinterpret_cast<uint64_t *>(smem_raw + (size_t)seg_cap * 12);
-  uint32_t *s_bin = reinterpret_cast<uint32_t *>(smem_raw + (size_t)seg_cap * 20);
-  uint32_t *s_cur = s_bin + SORT_BINS + 4;
-  __shared__ BlockShared sh;
+__device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCtx &c, int r, uint32_t b, int n, int n_act,
+                               bool ordered, bool list_in, unsigned char *smem, BlockShared &sh) {
+  uint64_t *s_hi = reinterpret_cast<uint64_t *>(smem);
+  uint32_t *s_lo = reinterpret_cast<uint32_t *>(smem + (size_t)SEG_MED * 8);
   const int R = p.n_replicas;
-  if (c.flags[2] < (uint32_t)seg_min) return;     // no replica of this kernel's size class exists
-  const bool ordered = c.flags[c.parity] != 0;
+  const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
+  const int n_in = n - n_act;
+  const HfxRec *seg = c.rec + b;
+  const bool real = r < R;    // bucket R holds rows bound to no replica
+  if (c.slabs) gather_to_records(a, c, R + 1, r, b, n_act, ordered, list_in, smem);
 
-  for (int r = blockIdx.x; r <= R; r += gridDim.x) {
-    const uint32_t b = c.seg_begin[r];
-    const int n = (int)(c.seg_begin[r + 1] - b);
-    const int n_act = (int)c.tot_act[r];
-    const int n_in = n - n_act;
-    const int need = ordered ? n_act : (n_act > n_in ? n_act : n_in);
-    if (need < seg_min || need > seg_cap) continue;
-    if (r == R && n == 0) continue;
-    const HfxRec *seg = c.rec + b;
-    const bool real = r < R;    // bucket R holds rows bound to no replica
-
-    // ---- inactive rows of a step that is not ordered: listed by req_id behind the active ones ----
-    if (!ordered && n_in > 0) {
-      const HfxRec *sin = seg + n_act;
-      int64_t next_arr = HFX_INF;
-      for (int q = threadIdx.x; q < n_in; q += blockDim.x) {
-        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
-        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
-        if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); next_arr = arr < next_arr ? arr : next_arr; }
-        s_hi[q] = ((uint64_t)(w0.z ^ 0x80000000u) << 16) | (uint32_t)q;     // signed req_id order, then position
-      }
-      __syncthreads();
-      if (!(bucket && n_in > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_in, sh))) {
-        sort64_positions(s_hi, s_lo, n_in);
-        __syncthreads();
-      }
-      for (int q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = sin[s_lo[q]].row;
-      __syncthreads();
-      segment_plan(p, a, seg, n_act, r, real, sh);
-      block_min_arrival(next_arr, sh);
-    } else {
-      segment_plan(p, a, seg, n_act, r, real, sh);
-    }
-    const ReplicaPlan pl = sh.plan;
-
-    // ---- sort items of the active rows ---------------------------------------------------------------
-    for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
-      const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
-      const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
-      const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
-      const int32_t row = (int32_t)w0.w;
-      const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
-      const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
-      if (ordered) s_hi[q] = (e.k48 << 16) | (uint32_t)q;     // records are in req_id order: position breaks ties
-      else {
-        const uint32_t uid = w0.z ^ 0x80000000u;               // signed req_id order as unsigned
-        s_hi[q] = (e.k48 << 16) | (uid >> 16);
-        s_lo[q] = (uid << 16) | (uint32_t)q;
-      }
-      if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the regroup wrote the slack of the other queued rows)
-        a.slack[row] = e.slack;
-        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
-      }
-      if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-    }
+  // ---- inactive rows of a step that is not ordered: listed by req_id behind the active ones ----
+  if (!ordered && n_in > 0) {
+    const HfxRec *sin = seg + n_act;
+    for (int q = threadIdx.x; q < n_in; q += blockDim.x)
+      s_hi[q] = ((uint64_t)(ld_rec(sin + q, 0).z ^ 0x80000000u) << 16) | (uint32_t)q;     // signed req_id order, then position
     __syncthreads();
-    if (ordered) {
-      if (!(bucket && n_act > 64 && block_bucket_order(s_hi, s_tmp, s_lo, s_bin, s_cur, n_act, sh))) {
-        sort64_positions(s_hi, s_lo, n_act);
-      }
-    } else {
-      block_sort<true>(s_hi, s_lo, n_act);
-      for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] &= 0xffffu;
-    }
+    sort64_positions(s_hi, s_lo, n_in);
     __syncthreads();
-
-    segment_admit(p, a, pl, seg, b, s_lo, n_act, sh);
-
-    // ---- maturity, iteration clock ------------------------------------------------------------------
-    if (threadIdx.x == 0) {
-      int64_t lp = 0;
-      const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
-      int worked; int64_t t1, t2;
-      iteration_clock(pl, sh.adm_count, lp, mat_next, worked, t1, t2);
-      sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
-    }
-    __syncthreads();
-    const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
-    const int worked = sh.worked;
-    const int64_t mat_next = sh.red_c[0];
-    if (commit && !worked && ordered) {
-      // idle replica of an ordered step: its next arrival is looked up among its listed inactive rows
-      block_min_arrival(next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x), sh);
-    }
-    if (threadIdx.x == 0 && real)
-      write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
-
-    // ---- padding of the compacted list, commit ----------------------------------------------------
-    if (a.admitted_rows)
-      for (int q = sh.adm_count + threadIdx.x; q < n; q += blockDim.x) a.admitted_rows[b + q] = -1;
-    if (commit) {
-      const int64_t t1 = sh.t1, t2 = sh.t2;
-      for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
-        const uint32_t lo = s_lo[q];
-        const int li = lo & 0xffff;
-        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
-        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
-        commit_row(a, pl, (w1.w >> 8) & 0xff, (lo & 0x10000u) != 0, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x,
-                   (int32_t)w1.y, (int32_t)w1.z);
-      }
-    }
+    for (int q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = (int32_t)ld_rec(sin + s_lo[q], 0).w;
     __syncthreads();
   }
-}
+  segment_plan(p, a, seg, n_act, r, real, sh);
+  const ReplicaPlan pl = sh.plan;
 
-// ------------------------------------------------------------------------------------------------
-// k_segment_small: replicas with at most SEG_TINY items to sort.  What later passes need of the
-// replica's active records (lengths, kind, row) is staged once into shared memory; sort items live
-// in registers until they are scattered into their bins.
-// ------------------------------------------------------------------------------------------------
-#define SEG_TINY 768
-#define TINY_IPT ((SEG_TINY + THREADS_SMALL - 1) / THREADS_SMALL)     // items per thread
-#define TINY_BINS 512
-#define TINY_BIN_MAX 48
-#define SMEM_TINY (SEG_TINY * (16 + 4 + 8 + 4) + (2 * TINY_BINS + 8) * 4)
-
-__global__ void __launch_bounds__(THREADS_SMALL, TINY_BLOCKS_PER_SM) k_segment_small(const HfxParams p, const SegArgs a, const SegCtx c) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint4 *s_w1 = reinterpret_cast<uint4 *>(smem_raw);                                   // [SEG_TINY] prompt, gen, output_len, bytes
-  uint64_t *s_key = reinterpret_cast<uint64_t *>(smem_raw + (size_t)SEG_TINY * 16);    // [SEG_TINY] sort items, binned
-  int32_t *s_row = reinterpret_cast<int32_t *>(s_key + SEG_TINY);                      // [SEG_TINY]
-  uint32_t *s_lo = reinterpret_cast<uint32_t *>(s_row + SEG_TINY);                     // [SEG_TINY] order (+ tie-break words)
-  uint32_t *s_bin = s_lo + SEG_TINY;                                                   // [TINY_BINS + 4]
-  uint32_t *s_cur = s_bin + TINY_BINS + 4;                                             // [TINY_BINS]
-  __shared__ BlockShared sh;
-  __shared__ int64_t s_cls_ttft[HFX_MAX_CLASSES], s_cls_tpot[HFX_MAX_CLASSES];     // class tables for the planning warp
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  const int R = p.n_replicas;
-  const bool ordered = c.flags[c.parity] != 0;
-  for (int k = threadIdx.x; k < HFX_MAX_CLASSES; k += blockDim.x) {
-    s_cls_ttft[k] = k < p.n_classes ? p.ttft[k] : 0;
-    s_cls_tpot[k] = k < p.n_classes ? p.tpot[k] : 0;
+  // ---- sort items of the active rows ---------------------------------------------------------------
+  for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
+    const uint4 w0 = ld_rec(seg + q, 0);
+    const uint4 w1 = ld_rec(seg + q, 1);
+    const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
+    const int32_t row = (int32_t)w0.w;
+    const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
+    const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+    if (ordered) s_hi[q] = (e.k48 << 16) | (uint32_t)q;     // records are in req_id order: position breaks ties
+    else {
+      const uint32_t uid = w0.z ^ 0x80000000u;               // signed req_id order as unsigned
+      s_hi[q] = (e.k48 << 16) | (uid >> 16);
+      s_lo[q] = (uid << 16) | (uint32_t)q;
+    }
+    if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the front end wrote the slack of the other queued rows)
+      a.slack[row] = e.slack;
+      if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
+    }
+    if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
   }
-
-  for (int r = blockIdx.x; r <= R; r += gridDim.x) {
-    const uint32_t b = c.seg_begin[r];
-    const int n = (int)(c.seg_begin[r + 1] - b);
-    const int n_act = (int)c.tot_act[r];
-    const int n_in = n - n_act;
-    const int need = ordered ? n_act : (n_act > n_in ? n_act : n_in);
-    if (need > SEG_TINY) continue;
-    if (r == R && n == 0) continue;
-    const HfxRec *seg = c.rec + b;
-    const bool real = r < R;    // bucket R holds rows bound to no replica
-
-    int64_t next_arr = HFX_INF;
-    if (!ordered && n_in > 0) {
-      // inactive rows of a step that is not ordered: listed by req_id behind the active ones
-      const HfxRec *sin = seg + n_act;
-      for (int q = threadIdx.x; q < n_in; q += blockDim.x) {
-        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
-        const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
-        if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); next_arr = arr < next_arr ? arr : next_arr; }
-        s_key[q] = ((uint64_t)(w0.z ^ 0x80000000u) << 16) | (uint32_t)q;
-      }
-      __syncthreads();
-      block_sort<false>(s_key, nullptr, n_in);
-      for (int q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = sin[s_key[q] & 0xffffu].row;
-      __syncthreads();
-    }
-
-    // ---- stage what later passes need of the active records; aggregates --------------------------
-    uint4 w0r[TINY_IPT];
-    {
-      int64_t n_run = 0, sum_kv = 0;
-      uint64_t m_run = 0, m_q = 0;
-#pragma unroll
-      for (int k = 0; k < TINY_IPT; k++) {
-        const int q = threadIdx.x + k * THREADS_SMALL;
-        if (q < n_act) {
-          w0r[k] = __ldg(reinterpret_cast<const uint4 *>(seg + q));
-          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
-          s_w1[q] = w1;
-          s_row[q] = (int32_t)w0r[k].w;
-          const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
-          if (kind == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
-          else m_q |= 1ull << cls;
-        }
-      }
-      n_run = warp_sum_i64(n_run); sum_kv = warp_sum_i64(sum_kv); next_arr = warp_min_i64(next_arr);
-      m_run = warp_or_u64(m_run); m_q = warp_or_u64(m_q);
-      if (lane == 0) { sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_c[warp] = next_arr; sh.red_m0[warp] = m_run; sh.red_m1[warp] = m_q; }
-      for (int i = threadIdx.x; i <= TINY_BINS; i += blockDim.x) s_bin[i] = 0;
-      __syncthreads();
-      if (warp == 0) {     // the whole first warp finishes the reduction and plans
-        const bool has = lane < nwarp;
-        n_run = warp_sum_i64(has ? sh.red_a[lane] : 0); sum_kv = warp_sum_i64(has ? sh.red_b[lane] : 0);
-        next_arr = warp_min_i64(has ? sh.red_c[lane] : HFX_INF);
-        m_run = warp_or_u64(has ? sh.red_m0[lane] : 0); m_q = warp_or_u64(has ? sh.red_m1[lane] : 0);
-        hfx_replica_cfg cfg; cfg.mode = HFX_COLOCATED; cfg.token_cap = 1; cfg.batch_cap = 0;
-        int64_t now = 0, mat = 0;
-        if (real) { cfg = a.cfg[r]; now = a.now[r]; mat = a.mat[r]; }
-        ReplicaPlan pl0;
-        warp_plan(p, s_cls_ttft, s_cls_tpot, cfg, now, mat, n_run, sum_kv, m_run, m_q, pl0, lane);
-        if (lane == 0) { sh.plan = pl0; sh.next_arrival = next_arr; }
-      }
-      __syncthreads();
-    }
-    const ReplicaPlan pl = sh.plan;
-
-    // ---- keys (in registers), their range ---------------------------------------------------------
-    uint64_t item[TINY_IPT];
-    uint64_t mn = ~0ull, mx = 0;
-#pragma unroll
-    for (int k = 0; k < TINY_IPT; k++) {
-      const int q = threadIdx.x + k * THREADS_SMALL;
-      item[k] = ~0ull;
-      if (q < n_act) {
-        const uint4 w0 = w0r[k], w1 = s_w1[q];
-        const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
-        const int32_t row = (int32_t)w0.w;
-        const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
-        const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
-        if (ordered) {
-          item[k] = (e.k48 << 16) | (uint32_t)q;     // records are in req_id order: position breaks ties
-          mn = item[k] < mn ? item[k] : mn; mx = item[k] > mx ? item[k] : mx;
-        } else {
-          const uint32_t uid = w0.z ^ 0x80000000u;
-          s_key[q] = (e.k48 << 16) | (uid >> 16);
-          s_lo[q] = (uid << 16) | (uint32_t)q;
-        }
-        if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the regroup wrote the slack of the other queued rows)
-          a.slack[row] = e.slack;
-          if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
-        }
-        if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-      }
-    }
-    bool sorted_done = false;
-    if (ordered && n_act > 0) {
-      // ---- distribution sort: bins by offset from the smallest item, rank inside the bin by counting ----
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const uint64_t x = __shfl_xor_sync(0xffffffffu, mn, o), y = __shfl_xor_sync(0xffffffffu, mx, o);
-        mn = x < mn ? x : mn; mx = y > mx ? y : mx;
-      }
-      if (lane == 0) { sh.red_m0[warp] = mn; sh.red_m1[warp] = mx; }
-      __syncthreads();
-      for (int k = 0; k < nwarp; k++) { const uint64_t x = sh.red_m0[k], y = sh.red_m1[k]; mn = x < mn ? x : mn; mx = y > mx ? y : mx; }
-      const uint64_t range = mx - mn;
-      int sft = 0;
-      if (range >= TINY_BINS) sft = 64 - __clzll((long long)range) - 9;     // (range >> sft) < TINY_BINS
-#pragma unroll
-      for (int k = 0; k < TINY_IPT; k++)
-        if (threadIdx.x + k * THREADS_SMALL < n_act) atomicAdd(&s_bin[(uint32_t)((item[k] - mn) >> sft)], 1u);
-      __syncthreads();
-      if (warp == 0) {     // exclusive scan of the bin counts by one warp; the largest bin
-        const int per = TINY_BINS / 32;
-        uint32_t cnt[TINY_BINS / 32];
-        uint32_t sum = 0, big = 0;
-#pragma unroll
-        for (int i = 0; i < per; i++) { cnt[i] = s_bin[lane * per + i]; sum += cnt[i]; big = cnt[i] > big ? cnt[i] : big; }
-        uint32_t v = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) { const uint32_t x = __shfl_xor_sync(0xffffffffu, big, o); big = x > big ? x : big; }
-        uint32_t run = v - sum;
-#pragma unroll
-        for (int i = 0; i < per; i++) { s_bin[lane * per + i] = run; s_cur[lane * per + i] = run; run += cnt[i]; }
-        if (lane == 0) sh.red_n[0] = (int32_t)big;
-      }
-      __syncthreads();
-      if (sh.red_n[0] <= TINY_BIN_MAX) {
-#pragma unroll
-        for (int k = 0; k < TINY_IPT; k++)
-          if (threadIdx.x + k * THREADS_SMALL < n_act) s_key[atomicAdd(&s_cur[(uint32_t)((item[k] - mn) >> sft)], 1u)] = item[k];
-        __syncthreads();
-        for (int e = threadIdx.x; e < n_act; e += blockDim.x) {
-          const uint64_t x = s_key[e];
-          const uint32_t bi = (uint32_t)((x - mn) >> sft);
-          const uint32_t g0 = s_bin[bi], g1 = s_cur[bi];
-          uint32_t rank = 0;
-          for (uint32_t g = g0; g < g1; g++) rank += s_key[g] < x ? 1u : 0u;
-          s_lo[g0 + rank] = (uint32_t)(x & 0xffffu);
-        }
-        sorted_done = true;
-      } else {
-#pragma unroll
-        for (int k = 0; k < TINY_IPT; k++) { const int q = threadIdx.x + k * THREADS_SMALL; if (q < n_act) s_key[q] = item[k]; }
-      }
-    }
-    __syncthreads();
-    if (!sorted_done) {
-      if (ordered) {
-        block_sort<false>(s_key, nullptr, n_act);
-        for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] = (uint32_t)(s_key[q] & 0xffffu);
-      } else {
-        block_sort<true>(s_key, s_lo, n_act);
-        for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] &= 0xffffu;
-      }
-      __syncthreads();
-    }
-
-    // ---- first-fit variant: the first warp walks the order and marks what it takes (bit 17) -----------
-    if (p.first_fit) {
-      if (warp == 0) {
-        const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
-        warp_first_fit(n_act, pl.budget, room, lane,
-                       [&](int64_t q) -> int64_t {
-                         const uint4 w1 = s_w1[s_lo[q] & 0xffffu];
-                         if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
-                         return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
-                       },
-                       [&](int64_t q, bool taken) { if (taken) s_lo[q] |= 0x20000u; });
-      }
-      __syncthreads();
-    }
-
-    // ---- admission: each thread walks TINY_IPT consecutive places of the order ---------------------
-    const int q0 = threadIdx.x * TINY_IPT;
-    int64_t cost[TINY_IPT], kvs[TINY_IPT];
-    int32_t rows[TINY_IPT], kinds[TINY_IPT];
-    int64_t my_cost = 0;
-    int32_t my_cnt = 0;
-#pragma unroll
-    for (int k = 0; k < TINY_IPT; k++) {
-      const int q = q0 + k;
-      cost[k] = -1; kvs[k] = 0; rows[k] = -1; kinds[k] = KIND_DEAD;
-      if (q < n_act) {
-        const int li = s_lo[q] & 0xffffu;
-        const uint4 w1 = s_w1[li];
-        rows[k] = s_row[li];
-        kinds[k] = (w1.w >> 8) & 0xff;
-        if (kinds[k] == KIND_QUEUED) {
-          const int64_t kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
-          const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-          // what counts towards the totals: rows that fit alone, or (first fit) exactly the rows taken
-          if (p.first_fit ? (s_lo[q] & 0x20000u) != 0 : cc <= pl.budget) { cost[k] = cc; kvs[k] = kv; my_cost += cc; my_cnt++; }
-        }
-        a.order[b + q] = rows[k];
-      }
-    }
-    int64_t sc = warp_incl_scan_i64(my_cost, lane);
-    int32_t sn = warp_incl_scan_i32(my_cnt, lane);
-    if (lane == 31) { sh.red_a[warp] = sc; sh.red_n[warp] = sn; }
-    __syncthreads();
-    int64_t run_c = sc - my_cost;
-    int32_t run_n = sn - my_cnt;
-    for (int k = 0; k < warp; k++) { run_c += sh.red_a[k]; run_n += sh.red_n[k]; }
-    int64_t ac = 0, ak = 0;
-    int32_t an = 0;
-#pragma unroll
-    for (int k = 0; k < TINY_IPT; k++) {
-      const int q = q0 + k;
-      if (q < n_act) {
-        bool adm = false;
-        if (cost[k] >= 0) {
-          run_c += cost[k]; run_n += 1;
-          adm = p.first_fit || (run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap));
-          if (adm) { ac += cost[k]; ak += kvs[k]; an++; if (a.admitted_rows) a.admitted_rows[b + run_n - 1] = rows[k]; }
-        }
-        if (kinds[k] == KIND_RUNNING || adm) a.admit[rows[k]] = 1;
-        s_lo[q] = (s_lo[q] & 0xffffu) | (adm ? 0x10000u : 0u);
-      }
-    }
-    ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)warp_sum_i64(an);
-    __syncthreads();
-    if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_n[warp] = an; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int64_t adm_cost = 0, adm_kv = 0; int32_t adm_count = 0;
-      for (int k = 0; k < nwarp; k++) { adm_cost += sh.red_a[k]; adm_kv += sh.red_b[k]; adm_count += sh.red_n[k]; }
-      int64_t lp = 0;
-      const int64_t mat_next = dev_maturity_next(p, pl, adm_count, adm_cost, adm_kv, &lp);
-      int worked; int64_t t1, t2;
-      iteration_clock(pl, adm_count, lp, mat_next, worked, t1, t2);
-      sh.adm_cost = adm_cost; sh.adm_count = adm_count;
-      sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
-    }
-    __syncthreads();
-    const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
-    const int worked = sh.worked;
-    const int64_t mat_next = sh.red_c[0];
-    if (commit && !worked && ordered) {
-      // idle replica of an ordered step: its next arrival is looked up among its listed inactive rows
-      block_min_arrival(next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x), sh);
-    }
-    if (threadIdx.x == 0 && real)
-      write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
-    if (a.admitted_rows)
-      for (int q = sh.adm_count + threadIdx.x; q < n; q += blockDim.x) a.admitted_rows[b + q] = -1;
-    if (commit) {
-      const int64_t t1 = sh.t1, t2 = sh.t2;
-      for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
-        const uint32_t lo = s_lo[q];
-        const int li = lo & 0xffff;
-        const uint4 w1 = s_w1[li];
-        commit_row(a, pl, (w1.w >> 8) & 0xff, (lo & 0x10000u) != 0, worked, t1, t2, s_row[li], (int32_t)w1.x,
-                   (int32_t)w1.y, (int32_t)w1.z);
-      }
-    }
-    __syncthreads();
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Oversize replicas (more items than a block can sort in shared memory): one cooperative kernel.
-// All blocks walk the replicas in the same order and share the work of each oversize one: keys
-// spread over the grid, a global bitonic network with bounded grid barriers, admission by block 0
-// walking the order with a carried prefix, commit by the grid.  Slow but exact; it only exists so
-// that any table is handled.
-// ------------------------------------------------------------------------------------------------
-
-// Bounded grid barrier (all blocks of a cooperative launch are resident).  Returns false if the
-// wait ran out; the caller then leaves, and HFX_ST_TIMEOUT is raised.
-__device__ bool grid_barrier(uint32_t *bar, uint32_t *status, uint32_t &epoch) {
-  __shared__ int ok_s;
   __syncthreads();
-  epoch++;
+  if (ordered) sort64_positions(s_hi, s_lo, n_act);
+  else {
+    group_sort<true>(s_hi, s_lo, n_act, B);
+    for (int q = threadIdx.x; q < n_act; q += blockDim.x) s_lo[q] &= 0xffffu;
+  }
+  __syncthreads();
+
+  segment_admit(p, a, pl, seg, b, s_lo, n_act, sh);
+
+  // ---- maturity, iteration clock ------------------------------------------------------------------
   if (threadIdx.x == 0) {
-    __threadfence();
-    const uint32_t target = epoch * gridDim.x;
-    atomicAdd(bar, 1u);
-    int ok = 0;
-    for (long long spin = 0; spin < (1ll << 26); spin++) {
-      if (*((volatile uint32_t *)bar) >= target) { ok = 1; break; }
-      if (*((volatile uint32_t *)status) & HFX_ST_TIMEOUT) break;
-      __nanosleep(64);
-    }
-    if (!ok) atomicOr(status, HFX_ST_TIMEOUT);
-    __threadfence();
-    ok_s = ok;
+    int64_t lp = 0;
+    const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
+    int worked; int64_t t1, t2;
+    iteration_clock(pl, sh.adm_count, lp, mat_next, worked, t1, t2);
+    sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
   }
   __syncthreads();
-  return ok_s != 0;
+  const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
+  const int worked = sh.worked;
+  const int64_t mat_next = sh.red_c[0];
+  if (commit && !worked)      // idle replica: its next arrival is looked up among its listed inactive rows
+    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x) : HFX_INF, sh, B);
+  if (threadIdx.x == 0 && real)
+    write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
+
+  // ---- padding of the compacted list, commit ----------------------------------------------------
+  if (a.admitted_rows)
+    for (int q = sh.adm_count + threadIdx.x; q < n; q += blockDim.x) a.admitted_rows[b + q] = -1;
+  if (commit) {
+    const int64_t t1 = sh.t1, t2 = sh.t2;
+    for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
+      const uint32_t lo = s_lo[q];
+      const int li = lo & 0xffff;
+      const uint4 w0 = ld_rec(seg + li, 0);
+      const uint4 w1 = ld_rec(seg + li, 1);
+      const int kind = (w1.w >> 8) & 0xff;
+      const bool adm = (lo & 0x10000u) != 0;
+      const int32_t out_len = commit_needs_out_len(pl, kind, adm, worked) ? __ldg(a.output_len + (int32_t)w0.w) : 0;
+      commit_row(a, pl, kind, adm, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x, (int32_t)w1.y, out_len);
+    }
+  }
+  __syncthreads();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Oversize replicas (more items than a block sorts in shared memory): the block runs the sorting
+// network in global memory (items in c.big_hi / big_lo, the record positions travelling in big_idx),
+// then admission with a carried prefix.  Slow but exact.
+// ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void global_cmp_swap(uint64_t *hi, uint32_t *lo, uint32_t *idx, int64_t i, int64_t j) {
   const uint64_t hi_i = hi[i], hi_j = hi[j];
   const uint32_t lo_i = lo[i], lo_j = lo[j];
@@ -898,253 +1064,340 @@ __device__ __forceinline__ void global_cmp_swap(uint64_t *hi, uint32_t *lo, uint
   }
 }
 
-// Global bitonic network over n items (hi, lo) with idx travelling along: ascending comparators,
-// virtual padding.  The items must be visible grid-wide on entry (a grid barrier precedes it).
-__device__ bool grid_sort(uint64_t *hi, uint32_t *lo, uint32_t *idx, int64_t n, uint32_t *bar, uint32_t *status,
-                          uint32_t &epoch) {
-  const int64_t gtid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t gsize = (int64_t)gridDim.x * blockDim.x;
+// Bitonic network over n items (hi, lo) in global memory with idx travelling along: ascending comparators,
+// virtual padding.  Block-synchronised on entry by the caller and on return.
+__device__ void block_global_sort(uint64_t *hi, uint32_t *lo, uint32_t *idx, int64_t n) {
   int64_t n_pad = 1;
   while (n_pad < n) n_pad <<= 1;
   const int64_t half = n_pad >> 1;
   for (int64_t k = 2; k <= n_pad; k <<= 1) {
     const int64_t hk = k >> 1;
-    for (int64_t t = gtid; t < half; t += gsize) {
+    for (int64_t t = threadIdx.x; t < half; t += blockDim.x) {
       const int64_t blk = t / hk, off = t - blk * hk;
       const int64_t i = blk * k + off, j = blk * k + k - 1 - off;
       if (j < n) global_cmp_swap(hi, lo, idx, i, j);
     }
-    if (!grid_barrier(bar, status, epoch)) return false;
+    __syncthreads();
     for (int64_t j = k >> 2; j > 0; j >>= 1) {
-      for (int64_t t = gtid; t < half; t += gsize) {
+      for (int64_t t = threadIdx.x; t < half; t += blockDim.x) {
         const int64_t i = 2 * t - (t & (j - 1));
         if (i + j < n) global_cmp_swap(hi, lo, idx, i, i + j);
       }
-      if (!grid_barrier(bar, status, epoch)) return false;
+      __syncthreads();
     }
   }
-  return true;
 }
 
-__global__ void __launch_bounds__(512) k_big(const HfxParams p, const SegArgs a, const SegCtx c,
-                                             uint64_t *__restrict__ g_hi, uint32_t *__restrict__ g_lo,
-                                             uint32_t *__restrict__ g_idx, uint32_t *bar, uint32_t *status) {
-  __shared__ BlockShared sh;
-  if (c.flags[2] <= SEG_MED) return;
-  const bool ordered = c.flags[c.parity] != 0;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+__device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const SegCtx &c, int r, uint32_t b, int64_t n, int64_t n_act,
+                                 bool ordered, bool list_in, unsigned char *smem, BlockShared &sh) {
   const int R = p.n_replicas;
-  uint32_t epoch = 0;
-  const int64_t gtid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t gsize = (int64_t)gridDim.x * blockDim.x;
-  volatile int64_t *mail = reinterpret_cast<volatile int64_t *>(bar + 4);
+  const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const int64_t n_in = n - n_act;
+  const HfxRec *seg = c.rec + b;
+  const bool real = r < R;
+  if (c.slabs) gather_to_records(a, c, R + 1, r, b, n_act, ordered, list_in, smem);
 
-  for (int r = 0; r <= R; r++) {
-    const uint32_t b = c.seg_begin[r];
-    const int64_t n = (int64_t)(c.seg_begin[r + 1] - b);
-    const int64_t n_act = c.tot_act[r], n_in = n - n_act;
-    const int64_t need = ordered ? n_act : (n_act > n_in ? n_act : n_in);
-    if (need <= SEG_MED) continue;
-    const HfxRec *seg = c.rec + b;
-    const bool real = r < R;
+  // ---- inactive rows of a step that is not ordered: by req_id behind the active ones -----------
+  if (!ordered && n_in > 0) {
+    const HfxRec *sin = seg + n_act;
+    uint64_t *hi = c.big_hi + b + n_act;
+    uint32_t *lo = c.big_lo + b + n_act, *idx = c.big_idx + b + n_act;
+    for (int64_t q = threadIdx.x; q < n_in; q += blockDim.x) { hi[q] = ld_rec(sin + q, 0).z ^ 0x80000000u; lo[q] = 0; idx[q] = (uint32_t)q; }
+    __syncthreads();
+    block_global_sort(hi, lo, idx, n_in);
+    for (int64_t q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = (int32_t)ld_rec(sin + idx[q], 0).w;
+    __syncthreads();
+  }
 
-    // ---- inactive rows of a step that is not ordered: by req_id behind the active ones -----------
-    if (!ordered && n_in > 0) {
-      const HfxRec *sin = seg + n_act;
-      uint64_t *hi = g_hi + b + n_act;
-      uint32_t *lo = g_lo + b + n_act, *idx = g_idx + b + n_act;
-      for (int64_t q = gtid; q < n_in; q += gsize) {
-        const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
-        hi[q] = w0.z ^ 0x80000000u; lo[q] = 0; idx[q] = (uint32_t)q;
-      }
-      if (!grid_barrier(bar, status, epoch)) return;
-      if (!grid_sort(hi, lo, idx, n_in, bar, status, epoch)) return;
-      for (int64_t q = gtid; q < n_in; q += gsize) a.order[b + n_act + q] = sin[idx[q]].row;
+  segment_plan(p, a, seg, n_act, r, real, sh);
+  const ReplicaPlan pl = sh.plan;
+  uint64_t *hi = c.big_hi + b;
+  uint32_t *lo = c.big_lo + b, *idx = c.big_idx + b;
+
+  for (int64_t q = threadIdx.x; q < n_act; q += blockDim.x) {
+    const uint4 w0 = ld_rec(seg + q, 0);
+    const uint4 w1 = ld_rec(seg + q, 1);
+    const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
+    const int32_t row = (int32_t)w0.w;
+    const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
+    const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+    hi[q] = e.k48;
+    lo[q] = ordered ? (uint32_t)q : (w0.z ^ 0x80000000u);     // ties: position (rows in req_id order) or the request id
+    idx[q] = (uint32_t)q;
+    if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {
+      a.slack[row] = e.slack;
+      if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
     }
+    if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
+  }
+  __syncthreads();
+  block_global_sort(hi, lo, idx, n_act);
 
-    // every block computes the aggregates redundantly (reads come from L2 after the first)
-    segment_plan(p, a, seg, n_act, r, real, sh);
-    const ReplicaPlan pl = sh.plan;
-    uint64_t *hi = g_hi + b;
-    uint32_t *lo = g_lo + b, *idx = g_idx + b;
+  // admission walk with a carried prefix
+  if (p.first_fit) {     // the first warp walks the order; lo (free now that the sort is over) says what it took
+    if (warp == 0) {
+      const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
+      warp_first_fit(n_act, pl.budget, room, lane,
+                     [&](int64_t q) -> int64_t {
+                       const uint4 w1 = ld_rec(seg + idx[q], 1);
+                       if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
+                       return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
+                     },
+                     [&](int64_t q, bool taken) { lo[q] = taken ? 2u : 0u; });
+    }
+    __syncthreads();
+  }
+  for (int64_t tile = 0; tile < n_act; tile += blockDim.x) {
+    const int64_t q = tile + threadIdx.x;
+    int64_t cost = 0, kv = 0;
+    int32_t cnt = 0, row = -1, kind = KIND_DEAD;
+    if (q < n_act) {
+      const uint32_t li = idx[q];
+      const uint4 w0 = ld_rec(seg + li, 0);
+      const uint4 w1 = ld_rec(seg + li, 1);
+      row = (int32_t)w0.w;
+      kind = (w1.w >> 8) & 0xff;
+      if (kind == KIND_QUEUED) {
+        kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
+        const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
+        if (p.first_fit ? lo[q] == 2u : cc <= pl.budget) { cost = cc; cnt = 1; } else kv = 0;
+      }
+      a.order[b + q] = row;
+    }
+    int64_t sc = warp_incl_scan_i64(cost, lane);
+    int32_t sn = warp_incl_scan_i32(cnt, lane);
+    if (lane == 31) { sh.red_a[warp] = sc; sh.red_b[warp] = sn; }
+    __syncthreads();
+    if (warp == 0) {
+      int64_t x = lane < nwarp ? sh.red_a[lane] : 0;
+      int32_t y = lane < nwarp ? (int32_t)sh.red_b[lane] : 0;
+      x = warp_incl_scan_i64(x, lane); y = warp_incl_scan_i32(y, lane);
+      sh.red_a[lane] = x; sh.red_b[lane] = y;
+    }
+    __syncthreads();
+    sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
+    sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
+    bool adm = false;
+    if (cnt) adm = p.first_fit || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
+    if (q < n_act) {
+      if (adm) a.admit[row] = 1;
+      if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
+      lo[q] = adm ? 1u : 0u;      // the sort is over: lo now carries the decision
+    }
+    int64_t ac = adm ? cost : 0, ak = adm ? kv : 0;
+    int32_t an = adm ? 1 : 0;
+    ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)warp_sum_i64(an);
+    __syncthreads();
+    if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_c[warp] = an; }
+    if (threadIdx.x == blockDim.x - 1) { sh.carry_cost = sc; sh.carry_count = sn; }
+    __syncthreads();
+    if (threadIdx.x == 0)
+      for (int k = 0; k < nwarp; k++) { sh.adm_cost += sh.red_a[k]; sh.adm_kv += sh.red_b[k]; sh.adm_count += (int32_t)sh.red_c[k]; }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    int64_t lp = 0;
+    const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
+    int worked; int64_t t1, t2;
+    iteration_clock(pl, sh.adm_count, lp, mat_next, worked, t1, t2);
+    sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
+  }
+  __syncthreads();
+  const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
+  const int worked = sh.worked;
+  const int64_t mat_next = sh.red_c[0];
+  if (commit && !worked)
+    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x) : HFX_INF, sh, B);
+  if (threadIdx.x == 0 && real)
+    write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
+  if (a.admitted_rows)
+    for (int64_t q = sh.adm_count + threadIdx.x; q < n; q += blockDim.x) a.admitted_rows[b + q] = -1;
+  if (commit) {
+    const int64_t t1 = sh.t1, t2 = sh.t2;
+    for (int64_t q = threadIdx.x; q < n_act; q += blockDim.x) {
+      const uint32_t li = idx[q];
+      const uint4 w0 = ld_rec(seg + li, 0);
+      const uint4 w1 = ld_rec(seg + li, 1);
+      const int kind = (w1.w >> 8) & 0xff;
+      const bool adm = lo[q] != 0;
+      const int32_t out_len = commit_needs_out_len(pl, kind, adm, worked) ? __ldg(a.output_len + (int32_t)w0.w) : 0;
+      commit_row(a, pl, kind, adm, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x, (int32_t)w1.y, out_len);
+    }
+  }
+  __syncthreads();
+}
 
-    // keys of the active rows, spread over the grid
-    for (int64_t q = gtid; q < n_act; q += gsize) {
-      const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
-      const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
-      const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
-      const int32_t row = (int32_t)w0.w;
-      const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
-      const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
-      hi[q] = e.k48;
-      lo[q] = w0.z ^ 0x80000000u;
-      idx[q] = (uint32_t)q;
-      if (kind == KIND_RUNNING || pl.mode == HFX_DECODE) {    // (the regroup wrote the slack of the other queued rows)
-        a.slack[row] = e.slack;
-        if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | e.k48;
-      }
-      if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
-    }
-    if (!grid_barrier(bar, status, epoch)) return;
-    if (!grid_sort(hi, lo, idx, n_act, bar, status, epoch)) return;
+// ------------------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, const SegArgs a, const SegCtx c) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ BlockShared sh_g[REP_GROUPS];
+  __shared__ int64_t s_cls_ttft[HFX_MAX_CLASSES], s_cls_tpot[HFX_MAX_CLASSES];     // class tables for the planning warps
+  __shared__ uint32_t s_scan[2 * 32 + 2];      // (also the scratch of the block-wide scans below)
+  __shared__ uint32_t s_long[(HFX_TILE_REPLICAS_MAX + 1 + 31) / 32 + 1];           // replicas whose inactive rows the grid lists together
+  uint32_t *s_begin = reinterpret_cast<uint32_t *>(smem_raw + SMEM_MED);           // [R+2] range starts (slabs only)
+  const int R = p.n_replicas, R1 = R + 1;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (int k = tid; k < HFX_MAX_CLASSES; k += blockDim.x) {
+    s_cls_ttft[k] = k < p.n_classes ? p.ttft[k] : 0;
+    s_cls_tpot[k] = k < p.n_classes ? p.tpot[k] : 0;
+  }
+  for (int k = tid; k < (int)(sizeof(s_long) / sizeof(uint32_t)); k += blockDim.x) s_long[k] = 0;
 
-    // admission walk by block 0 with a carried prefix, then commit by the whole grid
-    if (blockIdx.x == 0) {
-      if (p.first_fit) {     // the first warp walks the order; lo (free now that the sort is over) says what it took
-        if (warp == 0) {
-          const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
-          warp_first_fit(n_act, pl.budget, room, lane,
-                         [&](int64_t q) -> int64_t {
-                           const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + idx[q]) + 1);
-                           if (((w1.w >> 8) & 0xff) != KIND_QUEUED) return -1;
-                           return pl.mode == HFX_DECODE ? p.d1 + p.d2 * ((int64_t)(int32_t)w1.x + (int32_t)w1.y) : (int64_t)(int32_t)w1.x;
-                         },
-                         [&](int64_t q, bool taken) { lo[q] = taken ? 2u : 0u; });
+  // everything below reads what the front end wrote
+  cudaGridDependencySynchronize();
+
+  const bool ordered = c.slabs ? __ldcg(c.ordered) != 0 : false;
+  const uint32_t *begin = c.seg_begin;
+  int larger = 1, longer = 0;       // does any replica need the whole block?  does any list of inactive rows need the grid?
+  __syncthreads();
+  if (c.slabs) {
+    // range starts: exclusive prefix of the rows per replica, every block its own copy
+    const int per = (R1 + blockDim.x - 1) / blockDim.x;
+    const int i0 = tid * per < R1 ? tid * per : R1, i1 = (i0 + per < R1) ? i0 + per : R1;
+    uint32_t sum = 0;
+    larger = 0;
+    for (int i = i0; i < i1; i++) {
+      const unsigned long long t = __ldcg(c.tot + i);
+      const uint32_t n_all = (uint32_t)t, n_act = (uint32_t)(t >> 32), n_in = n_all - n_act;
+      sum += n_all;
+      if ((ordered ? n_act : (n_act > n_in ? n_act : n_in)) > SEG_TINY) larger = 1;
+      if (ordered && n_in > LIST_MAX) { atomicOr(&s_long[i >> 5], 1u << (i & 31)); longer = 1; }
+    }
+    uint32_t v = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+    if (lane == 31) s_scan[warp] = v;
+    larger = __syncthreads_or(larger);
+    longer = __syncthreads_or(longer);
+    if (warp == 0) {      // the warps' totals, scanned by the first warp
+      uint32_t w = s_scan[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, w, o); if (lane >= o) w += x; }
+      s_scan[32 + lane] = w;
+    }
+    __syncthreads();
+    uint32_t run = v - sum + (warp ? s_scan[32 + warp - 1] : 0u);
+    for (int i = i0; i < i1; i++) {
+      s_begin[i] = run;
+      if (blockIdx.x == 0) a.seg_off[i] = (int32_t)run;
+      run += (uint32_t)__ldcg(c.tot + i);
+    }
+    if (tid == 0) s_begin[R1] = s_scan[63];
+    begin = s_begin;
+    __syncthreads();
+  }
+  auto counts = [&](int r, uint32_t &n_all, uint32_t &n_act) {
+    if (c.slabs) { const unsigned long long t = __ldcg(c.tot + r); n_all = (uint32_t)t; n_act = (uint32_t)(t >> 32); }
+    else { n_all = c.seg_count[r]; n_act = c.act_count[r]; }
+  };
+  auto need_of = [&](uint32_t n_all, uint32_t n_act) -> uint32_t {
+    const uint32_t n_in = n_all - n_act;
+    return ordered ? n_act : (n_act > n_in ? n_act : n_in);
+  };
+
+  // ---- small replicas: four groups of 256 threads, each on a barrier of its own ---------------------
+  {
+    const int g = tid / GROUP_THREADS;
+    const Grp G = {tid - g * GROUP_THREADS, GROUP_THREADS, g + 1};
+    for (int r = blockIdx.x * REP_GROUPS + g; r <= R; r += gridDim.x * REP_GROUPS) {
+      uint32_t n_all, n_act;
+      counts(r, n_all, n_act);
+      if (need_of(n_all, n_act) > SEG_TINY) continue;
+      if (r == R && n_all == 0) continue;
+      const bool list_in = !ordered || n_all - n_act <= LIST_MAX;
+      small_replica(p, a, c, G, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw + (size_t)g * SMEM_GROUP, sh_g[g],
+                    s_cls_ttft, s_cls_tpot);
+    }
+  }
+  __syncthreads();
+
+  // ---- larger replicas: the whole block -------------------------------------------------------------
+  if (larger)
+  for (int r = blockIdx.x; r <= R; r += gridDim.x) {
+    uint32_t n_all, n_act;
+    counts(r, n_all, n_act);
+    const uint32_t need = need_of(n_all, n_act);
+    if (need <= SEG_TINY) continue;
+    const bool list_in = !ordered || n_all - n_act <= LIST_MAX;
+    if (need <= SEG_MED) medium_replica(p, a, c, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw, sh_g[0]);
+    else oversize_replica(p, a, c, r, begin[r], n_all, n_act, ordered, list_in, smem_raw, sh_g[0]);
+  }
+
+  // ---- long lists of inactive rows (ordered steps): every block lists a range of tiles ----------------
+  if (longer) {
+    const int per = (c.n_tiles + gridDim.x - 1) / gridDim.x;
+    const int tA = blockIdx.x * per < c.n_tiles ? blockIdx.x * per : c.n_tiles;
+    const int tB = tA + per < c.n_tiles ? tA + per : c.n_tiles;
+    for (int wd = 0; wd * 32 < R1; wd++) {
+      uint32_t word = s_long[wd];
+      while (word) {
+        const int r = wd * 32 + __ffs(word) - 1;
+        word &= word - 1;
+        // inactive rows of replica r in the tiles before mine
+        uint32_t pre = 0;
+        for (int t = tid; t < tA; t += blockDim.x) { const uint2 m = __ldcg(c.M + (size_t)t * R1 + r); pre += (m.x >> 16) - (m.y >> 16); }
+        pre = (uint32_t)warp_sum_i64(pre);
+        __syncthreads();
+        if (lane == 0) s_scan[warp] = pre;
+        __syncthreads();
+        pre = 0;
+        for (int k = 0; k < 32; k++) pre += s_scan[k];
+        const uint32_t dst = begin[r] + (uint32_t)(__ldcg(c.tot + r) >> 32) + pre;
+        uint32_t done = 0;
+        for (int t = tA; t < tB; t++) {
+          const uint2 m = __ldcg(c.M + (size_t)t * R1 + r);
+          const uint32_t ca = m.y >> 16, ci = (m.x >> 16) - ca, src = (m.x & 0xffffu) + ca;
+          const size_t tb = (size_t)t * c.tile_rows;
+          for (uint32_t k = tid; k < ci; k += blockDim.x) a.order[dst + done + k] = (int32_t)(tb + __ldcg(c.slab_idx + tb + src + k));
+          done += ci;
         }
-        __syncthreads();
-      }
-      for (int64_t tile = 0; tile < n_act; tile += blockDim.x) {
-        const int64_t q = tile + threadIdx.x;
-        int64_t cost = 0, kv = 0;
-        int32_t cnt = 0, row = -1, kind = KIND_DEAD;
-        if (q < n_act) {
-          const uint32_t li = idx[q];
-          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
-          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
-          row = (int32_t)w0.w;
-          kind = (w1.w >> 8) & 0xff;
-          if (kind == KIND_QUEUED) {
-            kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
-            const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-            if (p.first_fit ? lo[q] == 2u : cc <= pl.budget) { cost = cc; cnt = 1; } else kv = 0;
-          }
-          a.order[b + q] = row;
-        }
-        int64_t sc = warp_incl_scan_i64(cost, lane);
-        int32_t sn = warp_incl_scan_i32(cnt, lane);
-        if (lane == 31) { sh.red_a[warp] = sc; sh.red_b[warp] = sn; }
-        __syncthreads();
-        if (warp == 0) {
-          int64_t x = lane < nwarp ? sh.red_a[lane] : 0;
-          int32_t y = lane < nwarp ? (int32_t)sh.red_b[lane] : 0;
-          x = warp_incl_scan_i64(x, lane); y = warp_incl_scan_i32(y, lane);
-          sh.red_a[lane] = x; sh.red_b[lane] = y;
-        }
-        __syncthreads();
-        sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
-        sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
-        bool adm = false;
-        if (cnt) adm = p.first_fit || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
-        if (q < n_act) {
-          if (kind == KIND_RUNNING || adm) a.admit[row] = 1;
-          if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
-          lo[q] = adm ? 1u : 0u;      // the sort is over: lo now carries the decision
-        }
-        int64_t ac = adm ? cost : 0, ak = adm ? kv : 0;
-        int32_t an = adm ? 1 : 0;
-        ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)warp_sum_i64(an);
-        __syncthreads();
-        if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_c[warp] = an; }
-        if (threadIdx.x == blockDim.x - 1) { sh.carry_cost = sc; sh.carry_count = sn; }
-        __syncthreads();
-        if (threadIdx.x == 0)
-          for (int k = 0; k < nwarp; k++) { sh.adm_cost += sh.red_a[k]; sh.adm_kv += sh.red_b[k]; sh.adm_count += (int32_t)sh.red_c[k]; }
-        __syncthreads();
-      }
-      // the replica's next arrival, should it turn out idle
-      int64_t v = HFX_INF;
-      if (ordered) {
-        v = next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x);
-      } else {
-        const HfxRec *sin = seg + n_act;
-        for (int64_t q = threadIdx.x; q < n_in; q += blockDim.x) {
-          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(sin + q));
-          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(sin + q) + 1);
-          if (((w1.w >> 8) & 0xff) == KIND_FUTURE) { const int64_t arr = (int64_t)(((uint64_t)w0.y << 32) | w0.x); v = arr < v ? arr : v; }
-        }
-      }
-      block_min_arrival(v, sh);
-      if (threadIdx.x == 0) {
-        int64_t lp = 0;
-        const int64_t mat_next = dev_maturity_next(p, pl, sh.adm_count, sh.adm_cost, sh.adm_kv, &lp);
-        int worked; int64_t t1, t2;
-        iteration_clock(pl, sh.adm_count, lp, mat_next, worked, t1, t2);
-        mail[0] = t1; mail[1] = t2; mail[2] = worked; mail[3] = sh.adm_count;   // for the other blocks
-        if (real) write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, t2, sh.next_arrival);
       }
     }
-    if (!grid_barrier(bar, status, epoch)) return;
-    {
-      const int64_t t1 = mail[0], t2 = mail[1];
-      const int worked = (int)mail[2], adm_count = (int)mail[3];
-      const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
-      if (a.admitted_rows)
-        for (int64_t q = adm_count + gtid; q < n; q += gsize) a.admitted_rows[b + q] = -1;
-      if (commit)
-        for (int64_t q = gtid; q < n_act; q += gsize) {
-          const uint32_t li = idx[q];
-          const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + li));
-          const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + li) + 1);
-          commit_row(a, pl, (w1.w >> 8) & 0xff, lo[q] != 0, worked, t1, t2, (int32_t)w0.w, (int32_t)w1.x, (int32_t)w1.y,
-                     (int32_t)w1.z);
-        }
-    }
-    if (!grid_barrier(bar, status, epoch)) return;
   }
 }
 
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
-int hfx_launch_segments(hfx_sched *s, const SegArgs &sa, int64_t n) {
+int hfx_launch_replicas(hfx_sched *s, const SegArgs &sa, int64_t n, bool slabs) {
   const int R1 = s->p.n_replicas + 1;
-  cudaStream_t stream = s->stream;
   SegCtx c;
-  c.rec = s->d_rec; c.seg_begin = s->d_seg_begin; c.tot_act = s->d_act_count; c.flags = s->d_flags;
-  c.rowflag = s->d_rowflag; c.parity = s->step_parity;
-  // Replicas too large for the small kernel are rare; their kernels (which leave at once when there is
-  // nothing for them) run on a second stream beside the small-replica kernel, forked and joined by events.
-  const bool larger = n > SEG_TINY;
-  const bool beside = larger && !s->profiling;
-  cudaStream_t st2 = beside ? s->side : stream;
-  if (beside) {
-    if (cudaEventRecord(s->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(s->side, s->ev_fork, 0) != cudaSuccess)
-      return HFX_E_CUDA;
+  memset(&c, 0, sizeof(c));
+  c.slabs = slabs ? 1 : 0;
+  c.rec = s->d_rec; c.rowflag = s->d_rowflag;
+  c.big_hi = s->d_big_hi; c.big_lo = s->d_big_lo; c.big_idx = s->d_big_lo ? s->d_big_lo + s->max_rows : nullptr;
+  if (slabs) {
+    const uint32_t par = s->tot_parity;
+    c.slab_rec = s->d_slab_rec; c.slab_idx = s->d_slab_idx; c.M = s->d_M;
+    c.tot = s->d_tot + (size_t)par * (R1 + 1);
+    c.ordered = s->d_flags + 4 + par;
+    hfx_front_shape(s, n, &c.tile_rows, &c.n_tiles);
+  } else {
+    c.seg_count = s->d_seg_count; c.act_count = s->d_act_count; c.seg_begin = s->d_seg_begin;
+    c.ordered = s->d_flags;
   }
-  if (!beside) {
-    KernelScope ks(s, KSLOT_SEG_SMALL);
-    const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
-    k_segment_small<<<grid, THREADS_SMALL, SMEM_TINY, stream>>>(s->p, sa, c);
-  }
-  if (larger) {
-    KernelScope ks(s, KSLOT_SEG_MED, st2);
-    const int grid = R1 < s->n_sm ? R1 : s->n_sm;
-    k_segment<<<grid, THREADS_MED, SEG_MED * 12, st2>>>(s->p, sa, c, SEG_TINY + 1, SEG_MED, 0);
-  }
-  if (n > SEG_MED) {
-    uint32_t *big_idx = reinterpret_cast<uint32_t *>(s->d_big_lo + s->max_rows);
-    if (cudaMemsetAsync(s->d_barrier, 0, 64, st2) != cudaSuccess) return HFX_E_CUDA;
-    void *args[] = {(void *)&s->p, (void *)&sa, (void *)&c, (void *)&s->d_big_hi, (void *)&s->d_big_lo, (void *)&big_idx,
-                    (void *)&s->d_barrier, (void *)&s->d_status};
-    KernelScope ks(s, KSLOT_BIG, st2);
-    if (cudaLaunchCooperativeKernel((void *)k_big, dim3(s->n_sm), dim3(512), args, 0, st2) != cudaSuccess)
-      return HFX_E_CUDA;
-  }
-  if (beside) {
-    {
-      KernelScope ks(s, KSLOT_SEG_SMALL);
-      const int grid = R1 < s->n_sm * 16 ? R1 : s->n_sm * 16;
-      k_segment_small<<<grid, THREADS_SMALL, SMEM_TINY, stream>>>(s->p, sa, c);
-    }
-    if (cudaEventRecord(s->ev_join, s->side) != cudaSuccess || cudaStreamWaitEvent(stream, s->ev_join, 0) != cudaSuccess)
-      return HFX_E_CUDA;
-  }
+  // one block per SM; the fallback layout has nothing that every block shares, so it needs no more blocks than replicas
+  const int grid = slabs ? s->n_sm : (R1 < s->n_sm ? R1 : s->n_sm);
+  const size_t smem = SMEM_MED + (slabs ? sizeof(uint32_t) * ((size_t)R1 + 2) : 0);
+  KernelScope ks(s, KSLOT_SEG_SMALL);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(REP_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = s->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = (slabs && !s->profiling) ? 1 : 0;      // the kernel may be set up while the tile front end drains
+  if (cudaLaunchKernelEx(&cfg, k_replicas, s->p, sa, c) != cudaSuccess) return HFX_E_CUDA;
   return HFX_OK;
 }
 
 int hfx_segment_configure() {
-  if (cudaFuncSetAttribute(k_segment, cudaFuncAttributeMaxDynamicSharedMemorySize, SEG_MED * 12) != cudaSuccess ||
-      cudaFuncSetAttribute(k_segment_small, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_TINY) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_replicas, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           SMEM_MED + sizeof(uint32_t) * (HFX_TILE_REPLICAS_MAX + 3)) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }
