@@ -129,18 +129,21 @@ __global__ void __launch_bounds__(FRONT_THREADS, 1) k_front(const HfxParams p, c
       int prio;
       if (p.weight_max > 0) prio = weight >= p.weight_max ? 0 : (weight <= p.weight_max - 62 ? 62 : p.weight_max - weight);
       else prio = s_prio[cls];
-      const int64_t base = row_base(p, s_ttft[cls], s_tpot[cls], kind, mode, prompt, gen, arrival, first_token);
-      s_rec[il] = make_uint4((uint32_t)(uint64_t)base, (uint32_t)((uint64_t)base >> 32),
-                             (uint32_t)prompt | (kind << CREC_KIND_SHIFT) | ((uint32_t)prio << CREC_PRIO_SHIFT),
-                             (uint32_t)gen | (cls << CREC_CLS_SHIFT));
+      int64_t base = row_base(p, s_ttft[cls], s_tpot[cls], kind, mode, prompt, gen, arrival, first_token);
       if (kind == KIND_QUEUED && mode != HFX_DECODE) {
+        // the slack of such a row needs nothing from the running batch: it is final here, and the record carries
+        // the row's final key in place of the base
         const int64_t start = s_start[bkt];
         slack = base == BASE_UNBOUNDED ? HFX_SLACK_MAX : base - start;
+        base = (int64_t)dev_key48(PH_QUEUED, prio, slack);
         if (EXTRA) {
-          k48 = dev_key48(PH_QUEUED, prio, slack);
+          k48 = (uint64_t)base;
           pttft = (start - arrival) + dev_Ep_prompt(p, prompt);
         }
       } else if (EXTRA) pttft = first_token - arrival;
+      s_rec[il] = make_uint4((uint32_t)(uint64_t)base, (uint32_t)((uint64_t)base >> 32),
+                             (uint32_t)prompt | (kind << CREC_KIND_SHIFT) | ((uint32_t)prio << CREC_PRIO_SHIFT),
+                             (uint32_t)gen | (cls << CREC_CLS_SHIFT));
     }
     const uint32_t g = 2u * (uint32_t)bkt + (act ? 0u : 1u);
     s_bkt[il] = (uint32_t)bkt | (act ? 0x8000u : 0u) | (atomicAdd(&s_cnt[g], 1u) << 16);

@@ -48,7 +48,8 @@ struct HfxParams {
 // One row after regrouping by replica: everything the per-replica kernel needs, 32 bytes
 // (one L2 sector), so that kernel never goes back to the table for reads.
 struct __align__(32) HfxRec {
-  int64_t base;      // slack before the per-replica shift (see ReplicaPlan); arrival for KIND_FUTURE
+  int64_t base;      // slack before the per-replica shift (see ReplicaPlan); the final 48-bit key for a queued row on a
+                     // colocated / prefill replica; arrival for KIND_FUTURE
   int32_t req_id;
   int32_t row;
   int32_t prompt;
@@ -59,7 +60,8 @@ struct __align__(32) HfxRec {
 static_assert(sizeof(HfxRec) == 32, "record is one 32-byte sector");
 
 // Compact record of an ACTIVE row as the tile front end leaves it (16 bytes, a uint4):
-//   x, y  slack base (int64, as HfxRec::base)
+//   x, y  slack base (int64, as HfxRec::base); for a queued row on a colocated / prefill replica the row's final
+//         48-bit key (phase | prio | clamped slack) instead, which needs nothing from the running batch
 //   z     prompt_len<25> | kind<1> (KIND_RUNNING / KIND_QUEUED) | prio<6>
 //   w     gen<25> | class<6>
 // The row index travels beside it (16-bit index inside the tile); req_id and output_len are fetched

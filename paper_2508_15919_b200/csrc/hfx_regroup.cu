@@ -191,6 +191,7 @@ __global__ void __launch_bounds__(256) k_regroup_atomic(const HfxParams p, const
     if (r.kind == KIND_QUEUED && mode != HFX_DECODE) {
       slack = r.base == BASE_UNBOUNDED ? HFX_SLACK_MAX : r.base - start;
       k48 = dev_key48(PH_QUEUED, r.prio, slack);
+      r.base = (int64_t)k48;      // final here: the record carries the row's key in place of the base
     }
     a.slack[i] = slack;
     a.admit[i] = in.kind == KIND_RUNNING;

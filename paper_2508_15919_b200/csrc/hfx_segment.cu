@@ -262,16 +262,18 @@ struct GatherTiles {
   uint32_t *pa, *pi;          // [n] active / inactive rows of the replica in the round's earlier tiles
   uint16_t *oa, *oall, *ca;   // [n] chunk descriptor: first record, first row index, active rows
   uint32_t *scan;             // [2 * warps + 2]
+  uint8_t *own_a, *own_i;     // optional (small replicas, n <= 256): the tile of every active / inactive row of the round
 };
 __host__ __device__ constexpr size_t gather_tiles_bytes(int n_tiles, int n_threads) { return (size_t)n_tiles * 14 + 4 * (2 * (size_t)(n_threads / 32) + 2); }
 __device__ __forceinline__ GatherTiles gather_tiles_at(unsigned char *smem, int n_tiles, int n_threads) {
   GatherTiles g;
   g.pa = reinterpret_cast<uint32_t *>(smem); g.pi = g.pa + n_tiles; g.scan = g.pi + n_tiles;
   g.oa = reinterpret_cast<uint16_t *>(g.scan + 2 * (n_threads / 32) + 2); g.oall = g.oa + n_tiles; g.ca = g.oall + n_tiles;
+  g.own_a = nullptr; g.own_i = nullptr;
   return g;
 }
 
-template <int NT, int TPT, class ActF, class InF>      // NT = G.n threads, TPT tiles per thread and round; NT * TPT a power of two
+template <int NT, int TPT, bool OWNER, class ActF, class InF>      // NT = G.n threads, TPT tiles per thread and round; NT * TPT a power of two
 __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, const Grp &G, const GatherTiles &gt, bool take_act,
                                                bool list_in, ActF emit_act, InF emit_in) {
   const int lane = G.tid & 31, w = G.tid >> 5, nw = G.n >> 5;
@@ -311,6 +313,10 @@ __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, c
       const bool in = t0 + lt < c.n_tiles;
       gt.pa[lt] = in ? pa : 0xffffffffu; gt.pi[lt] = in ? pi : 0xffffffffu;
       gt.oa[lt] = (uint16_t)oa[e]; gt.oall[lt] = (uint16_t)oall[e]; gt.ca[lt] = (uint16_t)ca[e];
+      if (OWNER) {      // which tile every row of the round comes from (rows are few: a small replica)
+        if (take_act) for (uint32_t k = 0; k < ca[e]; k++) gt.own_a[pa + k] = (uint8_t)lt;
+        if (list_in) for (uint32_t k = 0; k < ci[e]; k++) gt.own_i[pi + k] = (uint8_t)lt;
+      }
       pa += ca[e]; pi += ci[e];
     }
     G.sync();
@@ -329,7 +335,7 @@ __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, c
         for (int e = 0; e < 3; e++) {
           const uint32_t q = q0 + e * G.n;
           if (q < ta) {
-            const int lt = chunk_of(gt.pa, q);
+            const int lt = OWNER ? (int)gt.own_a[q] : chunk_of(gt.pa, q);
             const uint32_t k = q - gt.pa[lt];
             const size_t tb = (size_t)(t0 + lt) * c.tile_rows;
             rec[e] = __ldcg(c.slab_rec + tb + gt.oa[lt] + k);
@@ -346,7 +352,7 @@ __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, c
         for (int e = 0; e < 4; e++) {
           const uint32_t q = q0 + e * G.n;
           if (q < ti) {
-            const int lt = chunk_of(gt.pi, q);
+            const int lt = OWNER ? (int)gt.own_i[q] : chunk_of(gt.pi, q);
             const uint32_t k = q - gt.pi[lt];
             const size_t tb = (size_t)(t0 + lt) * c.tile_rows;
             row[e] = (int32_t)(tb + __ldcg(c.slab_idx + tb + gt.oall[lt] + gt.ca[lt] + k));
@@ -388,7 +394,11 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
   uint32_t *s_cur = s_bin + TINY_BINS / 2 + 4;                             // [TINY_BINS / 2] fill cursors, then bin ends
   uint2 *s_cinfo = reinterpret_cast<uint2 *>(s_cur + TINY_BINS / 2);       // [TINY_CLASSES] per class: smallest sub-key; first bin | shift << 16
   // over s_lo .. s_cur while the gather runs: the round's tile descriptors
-  const GatherTiles gt = gather_tiles_at(reinterpret_cast<unsigned char *>(s_lo), GROUP_THREADS * GROUP_TPT, GROUP_THREADS);
+  GatherTiles gt = gather_tiles_at(reinterpret_cast<unsigned char *>(s_lo), GROUP_THREADS * GROUP_TPT, GROUP_THREADS);
+  gt.own_a = reinterpret_cast<uint8_t *>(s_lo) + ((gather_tiles_bytes(GROUP_THREADS * GROUP_TPT, GROUP_THREADS) + 15) & ~(size_t)15);
+  gt.own_i = gt.own_a + SEG_TINY;
+  static_assert(((gather_tiles_bytes(GROUP_THREADS * GROUP_TPT, GROUP_THREADS) + 15) & ~(size_t)15) + SEG_TINY + LIST_MAX <=
+                (size_t)SEG_TINY * 4 + (TINY_BINS + 4) * 4, "the gather's scratch fits over the order and bin arrays");
   // over s_lo until the ranks are written: per class the smallest and largest sub-key and the number of items
   uint32_t *s_cmin = s_lo, *s_cmax = s_lo + TINY_CLASSES, *s_ccnt = s_lo + 2 * TINY_CLASSES;
   const int R = p.n_replicas, R1 = R + 1;
@@ -405,7 +415,7 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
   // ---- a step that is not ordered: the inactive rows, listed by req_id behind the active ones --------
   if (!ordered && n_in > 0) {
     if (c.slabs)
-      gather_replica<GROUP_THREADS, GROUP_TPT>(c, R1, r, G, gt, false, true, [](uint32_t, const uint4, int32_t) {},
+      gather_replica<GROUP_THREADS, GROUP_TPT, true>(c, R1, r, G, gt, false, true, [](uint32_t, const uint4, int32_t) {},
                                                [&](uint32_t pos, int32_t row) { s_row[pos] = row; });
     else
       for (int q = G.tid; q < n_in; q += G.n) s_row[q] = (int32_t)__ldg(reinterpret_cast<const uint4 *>(seg + n_act + q)).w;
@@ -429,7 +439,7 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
     } else m_q |= 1ull << cls;
   };
   if (c.slabs) {
-    gather_replica<GROUP_THREADS, GROUP_TPT>(c, R1, r, G, gt, true, ordered && list_in, take,
+    gather_replica<GROUP_THREADS, GROUP_TPT, true>(c, R1, r, G, gt, true, ordered && list_in, take,
                                              [&](uint32_t pos, int32_t row) { a.order[b + n_act + pos] = row; });
   } else {
     for (int q = G.tid; q < n_act; q += G.n) {
@@ -466,15 +476,22 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
 
   // ---- keys (in registers); per class their range ---------------------------------------------------
   uint64_t item[TINY_IPT];
+  int32_t out_len[TINY_IPT];       // of my rows in flight, asked for now and used by the commit
+  const bool will_commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
 #pragma unroll
   for (int k = 0; k < TINY_IPT; k++) {
     const int q = G.tid + k * GROUP_THREADS;
     item[k] = ~0ull;
+    out_len[k] = 0;
     if (q < n_act) {
+      if (will_commit && ((s_zw[q].x >> CREC_KIND_SHIFT) & 1u) == KIND_RUNNING) out_len[k] = __ldg(a.output_len + s_row[q]);
       const int64_t base = (int64_t)s_bk[q];
       const uint2 zw = s_zw[q];
       const int kind = (zw.x >> CREC_KIND_SHIFT) & 1, prio = zw.x >> CREC_PRIO_SHIFT;
-      const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)(zw.x & CREC_LEN_MASK), (int32_t)(zw.y & CREC_LEN_MASK));
+      const bool given = kind == KIND_QUEUED && pl.mode != HFX_DECODE;      // the front end has put the row's final key in place of the base
+      RowEval e;
+      if (given) { e.k48 = (uint64_t)base; e.slack = 0; e.pred_tpot = a.pred_tpot ? pl.tpot_q0 + p.d2 * ((int64_t)(zw.x & CREC_LEN_MASK) + (zw.y & CREC_LEN_MASK)) : 0; }
+      else e = eval_row(p, pl, base, kind, prio, (int32_t)(zw.x & CREC_LEN_MASK), (int32_t)(zw.y & CREC_LEN_MASK));
       if (ordered) {
         item[k] = (e.k48 << 16) | (uint32_t)q;     // rows were gathered in req_id order: position breaks ties
         const uint32_t cl = (uint32_t)(item[k] >> 56), sub = (uint32_t)(item[k] >> 24);
@@ -681,25 +698,17 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
     write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
   if (a.admitted_rows)
     for (int q = sh.adm_count + G.tid; q < n; q += G.n) a.admitted_rows[b + q] = -1;
-  if (commit) {      // every thread its own rows: the output lengths it needs are asked for together
+  if (commit) {      // every thread its own rows; an admitted row's output length is fetched now (there are few)
     const int64_t t1 = sh.t1, t2 = sh.t2;
-    int32_t out_len[TINY_IPT];
-#pragma unroll
-    for (int k = 0; k < TINY_IPT; k++) {
-      const int q = G.tid + k * GROUP_THREADS;
-      out_len[k] = 0;
-      if (q < n_act) {
-        const uint2 zw = s_zw[q];
-        if (commit_needs_out_len(pl, (zw.x >> CREC_KIND_SHIFT) & 1, (zw.y >> 31) != 0, worked)) out_len[k] = __ldg(a.output_len + s_row[q]);
-      }
-    }
 #pragma unroll
     for (int k = 0; k < TINY_IPT; k++) {
       const int q = G.tid + k * GROUP_THREADS;
       if (q < n_act) {
         const uint2 zw = s_zw[q];
-        commit_row(a, pl, (zw.x >> CREC_KIND_SHIFT) & 1, (zw.y >> 31) != 0, worked, t1, t2, s_row[q], (int32_t)(zw.x & CREC_LEN_MASK),
-                   (int32_t)(zw.y & CREC_LEN_MASK), out_len[k]);
+        const int kind = (zw.x >> CREC_KIND_SHIFT) & 1;
+        const bool adm = (zw.y >> 31) != 0;
+        const int32_t ol = adm ? __ldg(a.output_len + s_row[q]) : out_len[k];
+        commit_row(a, pl, kind, adm, worked, t1, t2, s_row[q], (int32_t)(zw.x & CREC_LEN_MASK), (int32_t)(zw.y & CREC_LEN_MASK), ol);
       }
     }
   }
@@ -716,7 +725,7 @@ __device__ void gather_to_records(const SegArgs &a, const SegCtx &c, int R1, int
                                   bool list_in, unsigned char *smem) {
   const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
   HfxRec *seg = c.rec + b;
-  gather_replica<REP_THREADS, 1>(c, R1, r, B, gather_tiles_at(smem, REP_THREADS, REP_THREADS), true, list_in || !ordered,
+  gather_replica<REP_THREADS, 1, false>(c, R1, r, B, gather_tiles_at(smem, REP_THREADS, REP_THREADS), true, list_in || !ordered,
                  [&](uint32_t pos, const uint4 rec, int32_t row) {
                    uint4 w0, w1;
                    w0.x = rec.x; w0.y = rec.y; w0.z = ordered ? 0u : (uint32_t)__ldg(a.req_id + row); w0.w = (uint32_t)row;
@@ -968,6 +977,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
   const int n_in = n - n_act;
   const HfxRec *seg = c.rec + b;
   const bool real = r < R;    // bucket R holds rows bound to no replica
+  // ---- gather into contiguous records -----------------------------------------------------------------
   if (c.slabs) gather_to_records(a, c, R + 1, r, b, n_act, ordered, list_in, smem);
 
   // ---- inactive rows of a step that is not ordered: listed by req_id behind the active ones ----
@@ -981,6 +991,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
     for (int q = threadIdx.x; q < n_in; q += blockDim.x) a.order[b + n_act + q] = (int32_t)ld_rec(sin + s_lo[q], 0).w;
     __syncthreads();
   }
+  // ---- aggregates, plan ---------------------------------------------------------------------------------
   segment_plan(p, a, seg, n_act, r, real, sh);
   const ReplicaPlan pl = sh.plan;
 
@@ -991,7 +1002,8 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
     const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
     const int32_t row = (int32_t)w0.w;
     const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
-    const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+    RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+    if (kind == KIND_QUEUED && pl.mode != HFX_DECODE) e.k48 = (uint64_t)base;      // the front end has put the row's final key in place of the base
     if (ordered) s_hi[q] = (e.k48 << 16) | (uint32_t)q;     // records are in req_id order: position breaks ties
     else {
       const uint32_t uid = w0.z ^ 0x80000000u;               // signed req_id order as unsigned
@@ -1005,6 +1017,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
     if (a.pred_tpot) a.pred_tpot[row] = e.pred_tpot;
   }
   __syncthreads();
+  // ---- sort ------------------------------------------------------------------------------------------------
   if (ordered) sort64_positions(s_hi, s_lo, n_act);
   else {
     group_sort<true>(s_hi, s_lo, n_act, B);
@@ -1012,6 +1025,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
   }
   __syncthreads();
 
+  // ---- admission -------------------------------------------------------------------------------------------
   segment_admit(p, a, pl, seg, b, s_lo, n_act, sh);
 
   // ---- maturity, iteration clock ------------------------------------------------------------------
@@ -1121,7 +1135,8 @@ __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const Seg
     const int64_t base = (int64_t)(((uint64_t)w0.y << 32) | w0.x);
     const int32_t row = (int32_t)w0.w;
     const int kind = (w1.w >> 8) & 0xff, prio = (w1.w >> 16) & 0xff;
-    const RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+    RowEval e = eval_row(p, pl, base, kind, prio, (int32_t)w1.x, (int32_t)w1.y);
+    if (kind == KIND_QUEUED && pl.mode != HFX_DECODE) e.k48 = (uint64_t)base;      // the front end has put the row's final key in place of the base
     hi[q] = e.k48;
     lo[q] = ordered ? (uint32_t)q : (w0.z ^ 0x80000000u);     // ties: position (rows in req_id order) or the request id
     idx[q] = (uint32_t)q;
@@ -1298,7 +1313,7 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
     return ordered ? n_act : (n_act > n_in ? n_act : n_in);
   };
 
-  // ---- small replicas: four groups of 256 threads, each on a barrier of its own ---------------------
+  // ---- small replicas: eight groups of 128 threads, each on a barrier of its own ---------------------
   {
     const int g = tid / GROUP_THREADS;
     const Grp G = {tid - g * GROUP_THREADS, GROUP_THREADS, g + 1};
