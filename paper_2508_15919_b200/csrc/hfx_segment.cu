@@ -327,7 +327,9 @@ __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, c
       for (int s = round_tiles >> 1; s > 0; s >>= 1) if (pre[lo + s] <= q) lo += s;
       return lo;
     };
-    if (take_act)
+    if (take_act) {
+      int lt_c = 0;            // the chunk of my previous row and where it ends: my rows rise, so large chunks are searched once
+      uint32_t lim_c = 0;
       for (uint32_t q0 = G.tid; q0 < ta; q0 += 3 * G.n) {
         uint4 rec[3];
         int32_t row[3];
@@ -335,7 +337,8 @@ __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, c
         for (int e = 0; e < 3; e++) {
           const uint32_t q = q0 + e * G.n;
           if (q < ta) {
-            const int lt = OWNER ? (int)gt.own_a[q] : chunk_of(gt.pa, q);
+            if (!OWNER && q >= lim_c) { lt_c = chunk_of(gt.pa, q); lim_c = gt.pa[lt_c] + gt.ca[lt_c]; }
+            const int lt = OWNER ? (int)gt.own_a[q] : lt_c;
             const uint32_t k = q - gt.pa[lt];
             const size_t tb = (size_t)(t0 + lt) * c.tile_rows;
             rec[e] = __ldcg(c.slab_rec + tb + gt.oa[lt] + k);
@@ -345,6 +348,7 @@ __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, c
 #pragma unroll
         for (int e = 0; e < 3; e++) { const uint32_t q = q0 + e * G.n; if (q < ta) emit_act(base_a + q, rec[e], row[e]); }
       }
+    }
     if (list_in)
       for (uint32_t q0 = G.tid; q0 < ti; q0 += 4 * G.n) {
         int32_t row[4];
@@ -751,6 +755,7 @@ __device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   int64_t n_run = 0, sum_kv = 0;
   uint64_t m_run = 0, m_q = 0;
+#pragma unroll 4
   for (int64_t q = threadIdx.x; q < n_act; q += blockDim.x) {
     const uint4 w1 = ld_rec(seg + q, 1);   // prompt, gen, -, bytes
     const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
@@ -996,6 +1001,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
   const ReplicaPlan pl = sh.plan;
 
   // ---- sort items of the active rows ---------------------------------------------------------------
+#pragma unroll 4
   for (int q = threadIdx.x; q < n_act; q += blockDim.x) {
     const uint4 w0 = ld_rec(seg + q, 0);
     const uint4 w1 = ld_rec(seg + q, 1);
