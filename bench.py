@@ -31,14 +31,40 @@ import gen  # noqa: E402
 
 METRIC = "requests_scheduled_per_sec_per_hfx_sched_step"
 UNIT = "requests/s"
-ALGO_BYTES_PER_ROW = 51            # 38 B read (incl. priority weight) + 13 B written per row and step
-# algorithmic bytes per row of each kernel (what that kernel must move once)
-KERNEL_BYTES_PER_ROW = {"k_front": 51, "k_count": 26, "k_colscan": 0, "k_regroup": 51, "k_segment(small)": 13,
-                        "k_segment(medium)": 13, "k_big": 13}
+ALGO_BYTES_PER_ROW = 51            # 38 B read (incl. priority weight) + 13 B written (slack 8, order 4, admit 1) per row and step
+# what each kernel itself moves of those bytes (they add up to the step's 51): the tile front end reads the
+# columns and writes slack and admit, the replica kernel writes the order
+KERNEL_BYTES_PER_ROW = {"k_front": 47, "k_replicas": 4, "k_count": 22, "k_offsets": 0, "k_regroup_atomic": 25}
 STEPS_PER_EPISODE = 10
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel on this workload,
-# taken from the ncu capture summarised under profiles/; absent = no capture of the current kernel
-NCU_TRAFFIC_BYTES = {"k_front": 44.70e6 + 4.27e6, "k_segment(small)": 18.09e6 + 1.09e6}
+KERNEL_SOURCES = ["hfx_front.cu", "hfx_segment.cu", "hfx_step.cu", "hfx_regroup.cu", "hfx_rows.cuh", "hfx_internal.cuh"]
+PROFILE = os.path.join(ROOT, "profiles", "step_config4_k_front_k_replicas.md")
+
+
+def _kernel_source_hash():
+    """Identifies the kernels a profile was taken on: a hash of the step's CUDA sources."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2508_15919_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def _profile_counters():
+    """Per-kernel ncu counters of the committed profile summary (lines `<!-- bench: kernel=.. key=value .. -->`),
+    or {} when the summary was taken on other kernel sources than the ones in the tree."""
+    import re
+    out = {}
+    if not os.path.exists(PROFILE):
+        return out
+    src = _kernel_source_hash()
+    with open(PROFILE) as f:
+        for m in re.finditer(r"<!-- bench: (.*?) -->", f.read()):
+            kv = dict(x.split("=", 1) for x in m.group(1).split())
+            if kv.get("src") != src:
+                continue
+            out[kv["kernel"]] = {"traffic": float(kv["dram_bytes"]), "warp_inst": float(kv["warp_inst"]), "rows": float(kv["rows"])}
+    return out
 
 
 def _peaks():
@@ -416,7 +442,11 @@ def run_gpu(args):
     others = None
     if rank == 0 and not args.no_other_configs:
         others = {}
-        for name, ow in (("config2", gen.config2()), ("config3", gen.config3())):
+        peak_o, _ = _peaks()
+        perm4 = gen.config4()
+        perm4.table["req_id"] = np.random.default_rng(1).permutation(perm4.n_rows).astype(np.int32)      # ids not in row order: the general path
+        for name, ow in (("config1", gen.config1()), ("config2", gen.config2()), ("config3", gen.config3()),
+                         ("config4_permuted_req_id", perm4)):
             osched = hfx.Scheduler(ow.model, ow.classes, ow.replicas, ow.n_rows, budget_mode=ow.budget_mode, weight_max=ow.weight_max)
             otab = hfx.DeviceTable.from_numpy(ow.table)
             onow = torch.from_numpy(ow.now.copy()).cuda(); omat = torch.from_numpy(ow.maturity.copy()).cuda()
@@ -436,10 +466,13 @@ def run_gpu(args):
             for _ in range(5):
                 osched.step(otab, onow, omat, oout)
             oprof = osched.get_profile()
+            bpr = 51 if ow.weight_max > 0 else 47
+            gbs = bpr * ow.n_rows / (o_ms * 1e-3) / 1e9
             others[name] = {"rows": ow.n_rows, "replicas": ow.n_replicas, "ms_per_step": o_ms,
                             "requests_per_sec": ow.n_rows / (o_ms * 1e-3),
-                            "algorithmic_gbs": 51 * ow.n_rows / (o_ms * 1e-3) / 1e9,
+                            "algorithmic_bytes_per_row": bpr, "algorithmic_gbs": gbs, "frac": gbs / peak_o,
                             "kernel_us": {k: 1e3 * v["ms"] / v["launches"] for k, v in oprof.items()},
+                            "note": "one step without commit, L2 flushed before it" + ("; launch-latency bound at this size" if ow.n_rows < 100000 else ""),
                             "status": osched.status()}
             osched.close()
             del otab, oout
@@ -466,21 +499,36 @@ def run_gpu(args):
 
     if rank == 0:
         peak, peak_kind = _peaks()
-        dom = max(prof.items(), key=lambda kv: kv[1]["ms"])[0] if prof else None
+        counters = _profile_counters()
         roof = None
-        if dom:
-            per_launch_ms = prof[dom]["ms"] / prof[dom]["launches"]
-            bpr = KERNEL_BYTES_PER_ROW.get(dom, ALGO_BYTES_PER_ROW)
-            achieved = bpr * n / (per_launch_ms * 1e-3) / 1e9
-            step_gbs = ALGO_BYTES_PER_ROW * n / (step_ms_max * 1e-3) / 1e9
+        if prof:
+            step_bytes = ALGO_BYTES_PER_ROW * n
+            step_gbs = step_bytes / (step_ms_max * 1e-3) / 1e9
             tot = sum(x["ms"] for x in prof.values())
-            roof = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES.get(dom),
-                    "algorithmic_bytes_per_launch": bpr * n, "ms_per_launch": per_launch_ms,
-                    "step": {"algorithmic_bytes": ALGO_BYTES_PER_ROW * n, "achieved": step_gbs,
-                             "frac": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / 8000.0},
-                    "kernels": {k: {"ms_per_launch": v["ms"] / v["launches"], "launches": v["launches"],
-                                    "share": v["ms"] / tot} for k, v in prof.items()}}
+            kern = {}
+            for k, v in prof.items():
+                ms_l = v["ms"] / v["launches"]
+                bpr = KERNEL_BYTES_PER_ROW.get(k, 0)
+                cnt = counters.get(k)
+                kern[k] = {"ms_per_launch": ms_l, "launches": v["launches"], "share": v["ms"] / tot,
+                           "algorithmic_bytes_per_row": bpr, "algorithmic_bytes_per_launch": bpr * n,
+                           "achieved": bpr * n / (ms_l * 1e-3) / 1e9, "frac": bpr * n / (ms_l * 1e-3) / 1e9 / peak,
+                           "traffic": cnt["traffic"] * n / cnt["rows"] if cnt else None,
+                           "warp_instructions_per_row": cnt["warp_inst"] / cnt["rows"] if cnt else None}
+            traffic = sum(kv["traffic"] for kv in kern.values()) if kern and all(kv["traffic"] is not None for kv in kern.values()) else None
+            dom = max(prof.items(), key=lambda kv: kv[1]["ms"])[0]
+            # the headline is the whole step: every kernel of it runs once per step, and their algorithmic bytes add up to the step's
+            roof = {"bound": "hbm", "kernel": "hfx_sched_step = " + " + ".join(sorted(prof)), "dominant_kernel": dom,
+                    "achieved": step_gbs, "peak": peak, "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": "of " + peak_kind,
+                    "frac_of_nominal_8TBs": step_gbs / 8000.0, "traffic": traffic,
+                    "traffic_source": ("profiles/step_config4_k_front_k_replicas.md (ncu dram__bytes_read.sum + dram__bytes_write.sum, "
+                                       "taken on these kernel sources: hash %s)" % _kernel_source_hash()) if traffic is not None
+                                      else "none: the committed profile was taken on other kernel sources",
+                    "algorithmic_bytes_per_launch": step_bytes, "ms_per_launch": step_ms_max,
+                    "what_bounds_it": "instruction issue and dependent phases, not bytes: see warp_instructions_per_row and profiles/",
+                    "kernels": kern,
+                    "kernel_times_note": "per-kernel times come from event brackets inside the library in a second pass over the same steps; "
+                                         "the brackets keep the second kernel from being set up while the first drains, so their sum exceeds ms_per_step"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "int64", "data": "synthetic",

@@ -51,7 +51,7 @@ extern "C" {
 #define HFX_E_ALIGN      -2   /* a device pointer is not 16-byte aligned     */
 #define HFX_E_CAPACITY   -3   /* more rows / replicas than created for       */
 #define HFX_E_CUDA       -4   /* a CUDA runtime call failed (no device, ...) */
-#define HFX_E_TIMEOUT    -5   /* a bounded device-side wait ran out          */
+#define HFX_E_TIMEOUT    -5   /* reserved: no kernel of this version waits on another block, so none can run out */
 #define HFX_E_NOMEM      -6   /* workspace allocation failed                 */
 
 /* bits of the sticky device status word */
@@ -60,7 +60,7 @@ extern "C" {
                                    queue, bound to no instance yet                     */
 #define HFX_ST_BAD_CLASS    2u  /* class_id >= n_classes                      */
 #define HFX_ST_BAD_LEN      4u  /* prompt_len or gen outside [0, 2^24]        */
-#define HFX_ST_TIMEOUT      8u  /* a device-side wait gave up                 */
+#define HFX_ST_TIMEOUT      8u  /* reserved (see HFX_E_TIMEOUT)               */
 
 /* request states (column `state`) */
 #define HFX_QUEUED    0
@@ -216,9 +216,10 @@ typedef struct hfx_sim_out {
 
 /* Create a scheduler.  `model`, `classes[n_classes]`, `replicas[n_replicas]`
  * and `opts` are host pointers, copied.  `max_rows` bounds n_rows of later
- * calls and sizes the workspace (about 50 bytes per row of device memory, plus
- * per-replica tables of a few KB per replica for up to 4095 replicas).  `cuda_stream` is a cudaStream_t (NULL = the
- * default stream).  Errors: HFX_E_ARG (NULL pointer, value outside the domain
+ * calls and sizes the workspace (about 51 bytes per row of device memory, 67
+ * for tables of more than 16384 rows, plus 8 bytes per replica and tile of the
+ * table -- a tile is about 1/148 of the rows, at most 8192 -- for up to 4095
+ * replicas).  `cuda_stream` is a cudaStream_t (NULL = the default stream).  Errors: HFX_E_ARG (NULL pointer, value outside the domain
  * above), HFX_E_CUDA, HFX_E_NOMEM.  On error *out is NULL. */
 int hfx_sched_create(hfx_sched **out, const hfx_latency_model *model,
                      const hfx_slo_class *classes, int n_classes,
@@ -387,8 +388,12 @@ int hfx_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const h
  * columns are overwritten) and runs `iters` iterations of step + commit, or
  * until nothing is left to happen.  Written: state, gen, first_token_ns,
  * last_token_ns, finish_ns and `out`.
+ * A trace of up to 10240 rows is kept in shared memory; a longer one (at most 65535 rows) works in a scratch
+ * buffer in device memory (19 bytes per row for two traces per SM), which the first call that needs it
+ * allocates with cudaMalloc after synchronising the stream, so such a call should not be made inside a stream
+ * capture; hfx_sched_destroy frees it.
  * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY (n_traces > n_replicas, or a
- * trace longer than 4096 rows), HFX_E_CUDA. */
+ * trace longer than 65535 rows), HFX_E_NOMEM, HFX_E_CUDA. */
 int hfx_sim_run(hfx_sched *s, const hfx_table *table, const int32_t *trace_off,
                 int32_t n_traces, int32_t iters, const hfx_sim_out *out);
 
@@ -476,8 +481,7 @@ int hfx_scale_apply(hfx_sched *s, int64_t now_ns, const int32_t *decision, const
 
 /* Synchronise the scheduler's stream and return the sticky status word
  * (HFX_ST_* bits) in *status_word (host pointer); the word is then cleared.
- * Returns HFX_E_TIMEOUT if HFX_ST_TIMEOUT was set, HFX_E_CUDA if the stream
- * reports an error, else HFX_OK. */
+ * Returns HFX_E_CUDA if the stream reports an error, else HFX_OK. */
 int hfx_sched_status(hfx_sched *s, uint32_t *status_word);
 
 /* Number of kernels the library has launched on behalf of `s` so far. */
@@ -487,23 +491,22 @@ int64_t hfx_sched_launch_count(const hfx_sched *s);
  * profiling is on, every kernel the library launches is bracketed by CUDA
  * events on the scheduler's stream.  hfx_sched_get_profile synchronises the
  * stream, adds the elapsed times of all brackets recorded since the last call
- * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 1 column
- * scan, 2 offsets, 3 regroup, 4 segment (small), 5 segment (medium),
- * 6 oversize path, 7 simulator, 8 scaler tick and hfx_scale_apply, 9 fused front end, 10 the kernels of
- * hfx_dispatch_step and hfx_dispatch_bind together, 11 those of hfx_slo_map, 12 those of hfx_pd_migrate, 13
- * hfx_attainment; hfx_kernel_name gives the name of a slot (NULL past the end). */
+ * to *out (host pointer) and forgets them.  Kernel slots: 0 count, 2 offsets and 3 regroup (the fallback
+ * front end), 4 the per-replica kernel k_replicas, 7 simulator, 8 scaler tick and hfx_scale_apply, 9 the tile
+ * front end k_front, 10 the kernels of hfx_dispatch_step and hfx_dispatch_bind together, 11 those of hfx_slo_map,
+ * 12 those of hfx_pd_migrate, 13 hfx_attainment (1, 5, 6 unused); hfx_kernel_name gives the name of a slot
+ * (NULL past the end).  While profiling is on the per-replica kernel is not set up ahead of the front end's end
+ * (the brackets sit between them), so a step takes a little longer than without. */
 #define HFX_N_KERNELS 14
 typedef struct hfx_profile {
   double  ms[HFX_N_KERNELS];        /* total device time per kernel slot      */
   int64_t launches[HFX_N_KERNELS];  /* launches per kernel slot               */
 } hfx_profile;
 int hfx_sched_set_profiling(hfx_sched *s, int on);
-/* The front end of a step (row kinds and per-tile counts, their column scan,
- * the offsets, the regroup into per-replica ranges) normally runs as one
- * cooperative kernel, k_front, when every tile's block can be resident at once
- * (slot 9); `on` = 0 makes the following steps use the separate kernels k_count,
- * k_colscan and k_regroup instead, which is also what larger tables fall back
- * to.  Results are identical either way.  Host call, takes effect at the next
+/* The front end of a step normally is the tile kernel k_front (one pass over the table, one block per tile;
+ * slot 9), for schedulers of at most 4095 replicas whose tile matrix fits the workspace; `on` = 0 makes the
+ * following steps use the fallback front end instead (three kernels with global counters, slots 0, 2, 3), which
+ * is what larger schedulers always use.  Results are identical either way.  Host call, takes effect at the next
  * hfx_sched_step.  The paper has no counterpart (an execution switch). */
 int hfx_sched_set_fused_front(hfx_sched *s, int on);
 /* Commit horizon, for callers that advance many instances in rounds of one global clock (the events of

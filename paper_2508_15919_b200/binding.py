@@ -469,8 +469,8 @@ class Scheduler:
             raise HfxError(rc, "hfx_sched_set_profiling")
 
     def set_fused_front(self, on: bool):
-        """Run the front end of the following steps as one cooperative kernel (default) or as
-        separate kernels; the results are the same."""
+        """Run the front end of the following steps as the tile kernel (default) or as the fallback
+        kernels with global counters; the results are the same."""
         rc = self._L.hfx_sched_set_fused_front(self._h, int(on))
         if rc != 0:
             raise HfxError(rc, "hfx_sched_set_fused_front")

@@ -12,7 +12,7 @@ int hfx_slomap_configure();
 int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_trace_off, int32_t n_traces,
                           int32_t max_trace_rows, int32_t iters, const hfx_sim_out *o, uint32_t *d_work_counter);
 
-#define SIM_MAX_ROWS 4096
+#define SIM_MAX_ROWS 65535      // rows of a trace are numbered with 16 bits inside the simulator
 
 struct hfx_sched_host {
   hfx_sched core;
@@ -156,6 +156,7 @@ extern "C" void hfx_sched_destroy(hfx_sched *s) {
   hfx_sched_host *h = reinterpret_cast<hfx_sched_host *>(s);
   cudaStreamSynchronize(s->stream);
   hfx_dispatch_release(s);
+  hfx_sim_release(s);
   cudaFree(s->d_cfg); cudaFree(s->d_mode); cudaFree(s->d_status); cudaFree(s->d_seg_count); cudaFree(s->d_seg_begin);
   cudaFree(s->d_cursor); cudaFree(s->d_flags); cudaFree(s->d_rec);
   cudaFree(s->d_act_count); cudaFree(s->d_rowflag);

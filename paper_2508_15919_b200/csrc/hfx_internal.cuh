@@ -117,6 +117,8 @@ struct hfx_sched {
   int64_t horizon;          // commit horizon of the following steps (INT64_MAX: none)
   int front_enabled;        // 0: use the fallback front end (global counters) even where the tile front end fits
   void *dispatch_ws;                   // workspace of hfx_dispatch_step, allocated by its first call
+  unsigned char *d_sim_scratch;        // rows of long traces in hfx_sim_run (allocated by the first call that needs it)
+  size_t sim_scratch_bytes;
   void *d_slo;                         // per-priority table of hfx_slo_map
   void *d_pd;                          // moved counter, wake-up times and busy flags of hfx_pd_migrate
 };
@@ -566,6 +568,7 @@ int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *s
 int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const int64_t *maturity, const hfx_dispatch_out *o,
                         int32_t cap_max);
 void hfx_dispatch_release(hfx_sched *s);
+void hfx_sim_release(hfx_sched *s);
 int hfx_launch_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const hfx_slo_bounds *b, int64_t *last_queue,
                        const int32_t *pending, const int32_t *new_prio, int64_t n_new, int64_t *ttft_out, int64_t *tpot_out);
 size_t hfx_slomap_workspace_bytes();

@@ -11,15 +11,25 @@
 //   - admission extracts the most urgent eligible request repeatedly (block-wide arg-min on
 //     (prio, clamp(slack), req_id)) and stops at the first one that does not fit, which is
 //     exactly the prefix-closed rule of the sorted formulation.
+// Shared memory is what bounds the number of resident traces, so a row takes 19 bytes: one 8-byte slot
+// (arrival, then the slack base while queued, then the finish iteration while running), a word (prompt
+// length and priority), a byte (class and state) and three list entries; the rows admitted in an
+// iteration are parked in the part of the queue array that their extraction frees.
 #include "hfx_internal.cuh"
 
 #define SIM_THREADS 128
 #define SIM_WARPS (SIM_THREADS / 32)
-#define SIM_MAX_ROWS 4096
-#define SIM_BYTES_PER_ROW 28
+#define SIM_SMEM_ROWS 10240          // longest trace whose rows are kept in shared memory (19 bytes each); longer ones work in global scratch
+#define SIM_BYTES_PER_ROW 19
 #define SIM_OUTLEN_CAP (1 << 30)   // output lengths are clamped here when the finish iteration is formed
 
-#define ROW_INVALID 0xff
+// the byte of a row: class<6> | state<2>; the word of a row: prompt_len<25> | prio<6>, prio 63 marks a row with bad data
+#define ROW_CLS(x) ((x) & 0x3fu)
+#define ROW_STATE(x) ((x) >> 6)
+#define ROW_BYTE(cls, st) ((uint8_t)((cls) | ((st) << 6)))
+#define ROW_PROMPT(w) ((int32_t)((w) & 0x1ffffffu))
+#define ROW_PRIO(w) ((w) >> 25)
+#define ROW_INVALID_PRIO 63u
 
 struct SimArgs {
   const uint8_t *class_id; const int32_t *prompt_len; const int32_t *output_len; const int64_t *arrival;
@@ -38,7 +48,7 @@ struct SimShared {
   int64_t t1, t2, lp, mat_next;
   int64_t d_kv;                 // change of sum_kv collected during commit
   int32_t cnt_run[HFX_MAX_CLASSES], cnt_q[HFX_MAX_CLASSES];
-  int32_t head, nq, nr, nr_next, na, no, arrived;
+  int32_t head, head_prev, nq, nr, nr_next, na, no, arrived;
   int32_t worked, stop, trace, zero_prompt;
   // arg-min scratch, double buffered
   uint64_t best_key[2][SIM_WARPS];
@@ -79,20 +89,20 @@ __device__ __forceinline__ int64_t nearest_rank(const int64_t *sorted, int n, in
   return sorted[k - 1];
 }
 
+// SCRATCH: the per-row arrays of a block live in its part of a global scratch buffer instead of shared memory (traces
+// too long for it); the code is the same.
+template <bool SCRATCH>
 __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const SimArgs a, uint32_t *__restrict__ work_counter,
-                                                     uint32_t *__restrict__ status) {
+                                                     uint32_t *__restrict__ status, unsigned char *__restrict__ scratch) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int cap = a.cap_rows;
-  int64_t *s_arr = reinterpret_cast<int64_t *>(smem_raw);              // arrival, the slack base once arrived; later the TTFT, then the TPOT samples
-  int32_t *s_prompt = reinterpret_cast<int32_t *>(s_arr + cap);
-  int32_t *s_fin = s_prompt + cap;                                     // iteration at which a running row emits its last token
-  uint16_t *s_q = reinterpret_cast<uint16_t *>(s_fin + cap);           // visible queue (row indices, unordered)
+  unsigned char *rows_mem = SCRATCH ? scratch + (size_t)blockIdx.x * cap * SIM_BYTES_PER_ROW : smem_raw;
+  int64_t *s_arr = reinterpret_cast<int64_t *>(rows_mem);              // arrival; the slack base once arrived; the finish iteration once running; later the TTFT, then the TPOT samples
+  uint32_t *s_word = reinterpret_cast<uint32_t *>(s_arr + cap);        // prompt_len | prio << 25
+  uint16_t *s_q = reinterpret_cast<uint16_t *>(s_word + cap);          // visible queue (row indices, unordered); behind it the rows admitted in this iteration
   uint16_t *s_run = s_q + cap;                                         // running batch, ping
   uint16_t *s_run2 = s_run + cap;                                      // running batch, pong
-  uint16_t *s_adm = s_run2 + cap;                                      // admitted this iteration; oversize rows from the top
-  uint8_t *s_cls = reinterpret_cast<uint8_t *>(s_adm + cap);
-  uint8_t *s_prio = s_cls + cap;
-  uint8_t *s_state = s_prio + cap;
+  uint8_t *s_byte = reinterpret_cast<uint8_t *>(s_run2 + cap);         // class | state << 6
   __shared__ SimShared S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -108,7 +118,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
 
     // ---- stage the trace ----------------------------------------------------------------
     if (tid == 0) {
-      S.now = 0; S.mat = 0; S.sum_kv = 0; S.head = 0; S.nq = 0; S.nr = 0; S.stop = 0;
+      S.now = 0; S.mat = 0; S.sum_kv = 0; S.head = 0; S.head_prev = 0; S.nq = 0; S.nr = 0; S.stop = 0;
       S.n_fin = 0; S.n_rej = 0; S.n_att = 0; S.n_a = 0; S.n_b = 0; S.zero_prompt = 0;
       S.arrived = 0; S.no = 0; S.na = 0; S.nr_next = 0; S.d_kv = 0;
     }
@@ -124,19 +134,16 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       if (cls >= (uint32_t)p.n_classes) { bad |= HFX_ST_BAD_CLASS; ok = false; }
       if (prompt < 0 || prompt > HFX_MAX_TOKENS) { bad |= HFX_ST_BAD_LEN; ok = false; }
       s_arr[i] = arr;
-      s_prompt[i] = prompt;
       if (prompt == 0) S.zero_prompt = 1;   // a zero-token prompt fits a zero budget
-      s_fin[i] = -1;
-      s_cls[i] = ok ? (uint8_t)cls : ROW_INVALID;
-      s_state[i] = HFX_QUEUED;
-      int prio = 63;
+      uint32_t prio = ROW_INVALID_PRIO;
       if (ok) {
         if (p.weight_max > 0) {
           const int64_t w = (int64_t)p.weight_max - a.weight[g];
-          prio = (int)(w < 0 ? 0 : (w > 62 ? 62 : w));
+          prio = (uint32_t)(w < 0 ? 0 : (w > 62 ? 62 : w));
         } else prio = p.prio[cls];
       }
-      s_prio[i] = (uint8_t)prio;
+      s_word[i] = (ok ? (uint32_t)prompt : 0u) | (prio << 25);
+      s_byte[i] = ROW_BYTE(ok ? cls : 0u, HFX_QUEUED);
       a.first_token[g] = -1; a.last_token[g] = -1; a.finish[g] = -1;
     }
     if (bad) atomicOr(status, bad);
@@ -157,20 +164,21 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
         int local = 0;
         for (int i = head + tid; i < m && s_arr[i] <= now; i += SIM_THREADS) {
           local++;
-          const uint8_t cls = s_cls[i];
-          if (cls == ROW_INVALID) continue;
+          const uint32_t w = s_word[i];
+          if (ROW_PRIO(w) == ROW_INVALID_PRIO) continue;
+          const uint32_t cls = ROW_CLS(s_byte[i]);
           atomicAdd(&S.cnt_q[cls], 1);
-          if (s_prompt[i] > cfg.token_cap) {
-            // can never be served: visible for this one iteration, rejected at its commit
-            const int slot = atomicAdd(&S.no, 1);
-            s_adm[cap - 1 - slot] = (uint16_t)i;
+          if (ROW_PROMPT(w) > cfg.token_cap) {
+            // can never be served: visible for this one iteration, rejected at its commit (which looks through
+            // the rows that arrived in the iteration again)
+            atomicAdd(&S.no, 1);
           } else {
             const int slot = atomicAdd(&S.nq, 1);
             s_q[slot] = (uint16_t)i;
-            // from here on the row's arrival slot holds its slack base, ttft_slo + arrival - E_p(prompt_len):
+            // from here on the row's slot holds its slack base, ttft_slo + arrival - E_p(prompt_len):
             // the slack at any later decision is the base minus the earliest start
             const int64_t ttft = S.ttft[cls];
-            s_arr[i] = ttft > 0 ? ttft + s_arr[i] - dev_Ep(p, s_prompt[i]) : BASE_UNBOUNDED;
+            s_arr[i] = ttft > 0 ? ttft + s_arr[i] - dev_Ep(p, ROW_PROMPT(w)) : BASE_UNBOUNDED;
           }
         }
         if (local) atomicAdd(&S.arrived, local);
@@ -179,7 +187,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
 
       // ---- 2. plan: E_d of the running batch and the safe budget (the first warp) ----------------
       if (warp == 0) {
-        if (lane == 0) S.head += S.arrived;
+        if (lane == 0) { S.head_prev = S.head; S.head += S.arrived; }
         const uint32_t r0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_run[lane] > 0);
         const uint32_t r1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && S.cnt_run[lane + 32] > 0);
         const uint32_t q0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_q[lane] > 0);
@@ -202,11 +210,12 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           uint64_t bk = ~0ull; uint32_t bid = ~0u; int bslot = -1;
           for (int s = tid; s < nq; s += SIM_THREADS) {
             const int i = s_q[s];
-            if ((int64_t)s_prompt[i] > (p.first_fit ? budget - adm_cost : budget)) continue;      // first fit: against what is left
+            const uint32_t wd = s_word[i];
+            if ((int64_t)ROW_PROMPT(wd) > (p.first_fit ? budget - adm_cost : budget)) continue;      // first fit: against what is left
             // slack of a queued request: ttft_slo - (start - arrival) - E_p(prompt_len) = base - start
             const int64_t base = s_arr[i];
             const int64_t sl = base != BASE_UNBOUNDED ? dev_clamp_slack(base - start) : HFX_SLACK_MAX;
-            const uint64_t k = ((uint64_t)s_prio[i] << 40) | (uint64_t)(sl + (INT64_C(1) << 39));
+            const uint64_t k = ((uint64_t)ROW_PRIO(wd) << 40) | (uint64_t)(sl + (INT64_C(1) << 39));
             if (k < bk) { bk = k; bslot = s; bid = ~0u; }
             else if (k == bk) {      // equal keys are rare: only then fetch the request ids that break the tie
               if (bid == ~0u) bid = (uint32_t)__ldg(a.req_id + b + s_q[bslot]) ^ 0x80000000u;
@@ -241,15 +250,18 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           buf ^= 1;
           if (bslot < 0) break;                       // no eligible request left
           const int i = s_q[bslot];
-          s_cost += s_prompt[i]; s_cnt += 1;
+          const int32_t pr_i = ROW_PROMPT(s_word[i]);
+          s_cost += pr_i; s_cnt += 1;
           if (!(s_cost <= budget && (cfg.batch_cap == 0 || nr + s_cnt <= cfg.batch_cap))) break;
-          adm_cost += s_prompt[i]; adm_cnt += 1;
+          adm_cost += pr_i; adm_cnt += 1;
           __syncthreads();                            // everyone has read s_q[bslot]
-          if (tid == 0) { s_adm[adm_cnt - 1] = (uint16_t)i; s_q[bslot] = s_q[nq - 1]; }
+          // the queue shrinks by one; the place it frees behind its end takes the admitted row
+          if (tid == 0) { s_q[bslot] = s_q[nq - 1]; s_q[nq - 1] = (uint16_t)i; }
           nq -= 1;
           __syncthreads();
         }
       }
+      const int nq_adm = nq;      // the rows admitted in this iteration are s_q[nq_adm .. nq_adm + adm_cnt), last admitted first
 
       // ---- 4. maturity and the iteration's clock -------------------------------------------
       // every thread knows what was admitted, so every thread forms the iteration's two times itself; the
@@ -268,12 +280,13 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       // running batch: one more token each; a request finishes when gen + 1 reaches output_len
       for (int s = tid; s < nr; s += SIM_THREADS) {
         const int i = run_cur[s];
-        if (it >= s_fin[i]) {       // gen + 1 reaches output_len in this iteration
-          s_state[i] = HFX_DONE;
+        if (it >= (int32_t)s_arr[i]) {       // gen + 1 reaches output_len in this iteration
+          const uint32_t cls = ROW_CLS(s_byte[i]);
+          s_byte[i] = ROW_BYTE(cls, HFX_DONE);
           a.finish[(int64_t)b + i] = t2;
-          atomicSub(&S.cnt_run[s_cls[i]], 1);
+          atomicSub(&S.cnt_run[cls], 1);
           const int32_t outlen = __ldg(a.output_len + b + i);
-          d_kv -= (int64_t)s_prompt[i] + outlen - 2;       // leaves with the context it had before this step
+          d_kv -= (int64_t)ROW_PROMPT(s_word[i]) + outlen - 2;       // leaves with the context it had before this step
         } else {
           run_nxt[atomicAdd(&S.nr_next, 1)] = (uint16_t)i;
           d_kv += 1;
@@ -281,28 +294,31 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       }
       // admitted requests: first token at t1
       for (int s = tid; s < adm_cnt; s += SIM_THREADS) {
-        const int i = s_adm[s];
+        const int i = s_q[nq_adm + s];
         a.first_token[(int64_t)b + i] = t1;
         const int32_t outlen = __ldg(a.output_len + b + i);
-        s_fin[i] = it + (outlen < SIM_OUTLEN_CAP ? outlen : SIM_OUTLEN_CAP) - 1;
-        atomicSub(&S.cnt_q[s_cls[i]], 1);
+        s_arr[i] = it + (outlen < SIM_OUTLEN_CAP ? outlen : SIM_OUTLEN_CAP) - 1;      // the slot now holds the finish iteration
+        const uint32_t cls = ROW_CLS(s_byte[i]);
+        atomicSub(&S.cnt_q[cls], 1);
         if (outlen <= 1) {
-          s_state[i] = HFX_DONE;
+          s_byte[i] = ROW_BYTE(cls, HFX_DONE);
           a.finish[(int64_t)b + i] = t1;
         } else {
-          s_state[i] = HFX_RUNNING;
+          s_byte[i] = ROW_BYTE(cls, HFX_RUNNING);
           run_nxt[atomicAdd(&S.nr_next, 1)] = (uint16_t)i;
-          atomicAdd(&S.cnt_run[s_cls[i]], 1);
-          d_kv += s_prompt[i];
+          atomicAdd(&S.cnt_run[cls], 1);
+          d_kv += ROW_PROMPT(s_word[i]);
         }
       }
-      // oversize prompts seen for the first time
-      {
-        const int no = S.no;
-        for (int s = tid; s < no; s += SIM_THREADS) {
-          const int i = s_adm[cap - 1 - s];
-          s_state[i] = HFX_REJECTED;
-          atomicSub(&S.cnt_q[s_cls[i]], 1);
+      // oversize prompts seen for the first time: among the rows that arrived in this iteration
+      if (S.no > 0) {
+        for (int i = S.head_prev + tid; i < S.head; i += SIM_THREADS) {
+          const uint32_t w = s_word[i];
+          if (ROW_PRIO(w) != ROW_INVALID_PRIO && ROW_PROMPT(w) > cfg.token_cap) {
+            const uint32_t cls = ROW_CLS(s_byte[i]);
+            s_byte[i] = ROW_BYTE(cls, HFX_REJECTED);
+            atomicSub(&S.cnt_q[cls], 1);
+          }
         }
       }
       d_kv = warp_sum_i64(d_kv);
@@ -318,7 +334,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           int64_t ev = HFX_INF;
           if (S.plan.mat > S.plan.now) ev = S.plan.mat;
           int h = S.head;
-          while (h < m && s_cls[h] == ROW_INVALID) h++;     // rows with bad data never arrive
+          while (h < m && ROW_PRIO(s_word[h]) == ROW_INVALID_PRIO) h++;     // rows with bad data never arrive
           if (h < m && s_arr[h] < ev) ev = s_arr[h];
           if (ev == HFX_INF) S.stop = 1; else S.now = ev;
         }
@@ -335,7 +351,9 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     int fin = 0, rej = 0, att = 0;
     for (int i = tid; i < m; i += SIM_THREADS) {
       const int64_t g = (int64_t)b + i;
-      const int st = s_state[i];
+      const int st = ROW_STATE(s_byte[i]);
+      const bool valid = ROW_PRIO(s_word[i]) != ROW_INVALID_PRIO;
+      const uint32_t cls = ROW_CLS(s_byte[i]);
       const int32_t outlen = a.output_len[g];
       int32_t gen = 0;
       int64_t first = -1, last = -1;
@@ -343,7 +361,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
         first = a.first_token[g];
         if (st == HFX_DONE) { gen = outlen > 1 ? outlen - 1 : 0; last = a.finish[g]; }
         else {
-          const int admit_it = s_fin[i] - (outlen < SIM_OUTLEN_CAP ? outlen : SIM_OUTLEN_CAP) + 1;
+          const int admit_it = (int32_t)s_arr[i] - (outlen < SIM_OUTLEN_CAP ? outlen : SIM_OUTLEN_CAP) + 1;
           gen = executed - 1 - admit_it;
           last = gen > 0 ? now_final : first;
         }
@@ -351,10 +369,9 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       }
       a.state[g] = (uint8_t)st;
       a.gen[g] = gen;
-      const int64_t arr = a.arrival[g];      // (the shared-memory slot holds the slack base of rows that arrived)
-      const uint8_t cls = s_cls[i];
+      const int64_t arr = a.arrival[g];      // (the shared-memory slot holds other things by now)
       int64_t ttft = -1;
-      if (cls != ROW_INVALID) {
+      if (valid) {
         if (st == HFX_REJECTED) rej++;
         if (st == HFX_RUNNING || st == HFX_DONE) ttft = first - arr;
         if (st == HFX_DONE) {
@@ -380,7 +397,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     for (int i = tid; i < m; i += SIM_THREADS) {
       const int64_t g = (int64_t)b + i;
       int64_t tpot = -1;
-      if (s_state[i] == HFX_DONE && s_cls[i] != ROW_INVALID) {
+      if (ROW_STATE(s_byte[i]) == HFX_DONE && ROW_PRIO(s_word[i]) != ROW_INVALID_PRIO) {
         const int32_t outlen = a.output_len[g];
         if (outlen > 1) tpot = (a.finish[g] - a.first_token[g]) / (outlen - 1);
       }
@@ -406,9 +423,14 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
 }
 
 int hfx_sim_configure() {
-  if (cudaFuncSetAttribute(k_sim, cudaFuncAttributeMaxDynamicSharedMemorySize, SIM_MAX_ROWS * SIM_BYTES_PER_ROW) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_sim<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SIM_SMEM_ROWS * SIM_BYTES_PER_ROW) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
+}
+
+void hfx_sim_release(hfx_sched *s) {
+  cudaFree(s->d_sim_scratch);
+  s->d_sim_scratch = nullptr; s->sim_scratch_bytes = 0;
 }
 
 // `trace_off` is already on the device (copied by the caller of this launcher); max_rows is the
@@ -427,16 +449,30 @@ int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_tra
   a.iters_executed = o->iters_executed; a.finished = o->finished; a.rejected = o->rejected; a.attained = o->attained;
   a.ttft_p50 = o->ttft_p50_ns; a.ttft_p99 = o->ttft_p99_ns; a.tpot_p50 = o->tpot_p50_ns; a.tpot_p99 = o->tpot_p99_ns;
   a.now_out = o->now_ns;
-  const size_t smem = (size_t)cap * SIM_BYTES_PER_ROW;
+  const size_t rows_bytes = (size_t)cap * SIM_BYTES_PER_ROW;
   if (cudaMemsetAsync(d_work_counter, 0, sizeof(uint32_t), s->stream) != cudaSuccess) return HFX_E_CUDA;
-  int per_sm = (int)((224 * 1024) / (smem + 2560));
-  if (per_sm < 1) per_sm = 1;
-  if (per_sm > 8) per_sm = 8;
-  int grid = s->n_sm * per_sm;
-  if (grid > n_traces) grid = n_traces;
-  {
+  if (cap <= SIM_SMEM_ROWS) {
+    int per_sm = (int)((224 * 1024) / (rows_bytes + 3072));
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm > 8) per_sm = 8;
+    int grid = s->n_sm * per_sm;
+    if (grid > n_traces) grid = n_traces;
     KernelScope ks(s, KSLOT_SIM);
-    k_sim<<<grid, SIM_THREADS, smem, s->stream>>>(s->p, a, d_work_counter, s->d_status);
+    k_sim<false><<<grid, SIM_THREADS, rows_bytes, s->stream>>>(s->p, a, d_work_counter, s->d_status, nullptr);
+  } else {
+    // long traces: the rows of every resident block in a scratch buffer (two blocks per SM), allocated when first needed
+    int grid = s->n_sm * 2;
+    if (grid > n_traces) grid = n_traces;
+    const size_t need = rows_bytes * (size_t)grid;
+    if (s->sim_scratch_bytes < need) {
+      if (cudaStreamSynchronize(s->stream) != cudaSuccess) return HFX_E_CUDA;
+      cudaFree(s->d_sim_scratch);
+      s->d_sim_scratch = nullptr; s->sim_scratch_bytes = 0;
+      if (cudaMalloc(&s->d_sim_scratch, need) != cudaSuccess) { cudaGetLastError(); return HFX_E_NOMEM; }
+      s->sim_scratch_bytes = need;
+    }
+    KernelScope ks(s, KSLOT_SIM);
+    k_sim<true><<<grid, SIM_THREADS, 0, s->stream>>>(s->p, a, d_work_counter, s->d_status, s->d_sim_scratch);
   }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }

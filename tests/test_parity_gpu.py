@@ -293,6 +293,27 @@ def test_simulator_iteration_limits():
         assert_sim_parity(wl, iters=iters)
 
 
+def test_simulator_traces_beyond_shared_memory():
+    # 20,000 rows do not fit a block's shared memory: the trace's rows work in device scratch (same code)
+    wl = gen.random_traces(23, 2, 20_000, 20_000, iters=1200, rate=400.0, out_hi=64)
+    assert_sim_parity(wl)
+    # 9,000 rows: still in shared memory, one trace per SM
+    wl = gen.random_traces(24, 2, 9000, 9000, iters=1500, rate=300.0, out_hi=64)
+    assert_sim_parity(wl)
+
+
+def test_simulator_trace_length_limit():
+    # rows of a trace are numbered with 16 bits inside the simulator: 65,536 rows are refused before anything is launched
+    import paper_2508_15919_b200 as hfx
+    wl = gen.random_traces(25, 1, 65_536, 65_536, iters=1)
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    with pytest.raises(hfx.HfxError) as e:
+        sched.sim_run(tab, wl.trace_off, 1, hfx.SimOut(1))
+    assert e.value.code == -3
+    sched.close()
+
+
 def test_simulator_long_trace_and_weights():
     wl = gen.random_traces(21, 3, 3000, 4096, iters=6000, rate=60.0)
     wl.weight_max = 8
