@@ -49,7 +49,7 @@ def test_strerror_and_argument_checks_without_a_device():
     lib = hfx.load_library()
     assert lib.hfx_strerror(0) == b"ok" and b"aligned" in lib.hfx_strerror(-2)
     assert lib.hfx_strerror(-99) == b"unknown error"
-    assert lib.hfx_kernel_name(3) == b"k_regroup" and lib.hfx_kernel_name(9) == b"k_front" and lib.hfx_kernel_name(10) == b"k_dispatch" and lib.hfx_kernel_name(11) == b"k_slo_map" and lib.hfx_kernel_name(12) == b"k_pd_migrate" and lib.hfx_kernel_name(13) == b"k_attainment" and lib.hfx_kernel_name(14) is None
+    assert lib.hfx_kernel_name(3) == b"k_regroup_atomic" and lib.hfx_kernel_name(4) == b"k_replicas" and lib.hfx_kernel_name(9) == b"k_front" and lib.hfx_kernel_name(10) == b"k_dispatch" and lib.hfx_kernel_name(11) == b"k_slo_map" and lib.hfx_kernel_name(12) == b"k_pd_migrate" and lib.hfx_kernel_name(13) == b"k_attainment" and lib.hfx_kernel_name(14) is None
     import torch
     if not torch.cuda.is_available():
         # no device: the product path fails loudly, it never falls back to the CPU
