@@ -273,9 +273,20 @@ __device__ __forceinline__ GatherTiles gather_tiles_at(unsigned char *smem, int 
   return g;
 }
 
-template <int NT, int TPT, bool OWNER, class ActF, class InF>      // NT = G.n threads, TPT tiles per thread and round; NT * TPT a power of two
+__device__ __forceinline__ void cp_async8(void *smem_dst, const void *gmem_src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// where an asynchronous gather puts the active rows (shared memory): slack base, record words z and w, row index
+struct GatherDst { uint64_t *bk; uint2 *zw; int32_t *row; };
+
+// ASYNC: the records of the active rows are copied global -> shared memory without passing through registers (two
+// 8-byte cp.async per row, all of a round in flight together; the caller waits for them with cp_async_wait_all and
+// a barrier) and emit_act is not called.
+template <int NT, int TPT, bool OWNER, bool ASYNC, class ActF, class InF>      // NT = G.n threads, TPT tiles per thread and round; NT * TPT a power of two
 __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, const Grp &G, const GatherTiles &gt, bool take_act,
-                                               bool list_in, ActF emit_act, InF emit_in) {
+                                               bool list_in, ActF emit_act, InF emit_in, const GatherDst dst = GatherDst()) {
   const int lane = G.tid & 31, w = G.tid >> 5, nw = G.n >> 5;
   constexpr int round_tiles = NT * TPT;
   uint32_t base_a = 0, base_i = 0;
@@ -327,7 +338,28 @@ __device__ __forceinline__ void gather_replica(const SegCtx &c, int R1, int r, c
       for (int s = round_tiles >> 1; s > 0; s >>= 1) if (pre[lo + s] <= q) lo += s;
       return lo;
     };
-    if (take_act) {
+    if (ASYNC && take_act) {
+      for (uint32_t q = G.tid; q < ta; q += G.n) {
+        const int lt = OWNER ? (int)gt.own_a[q] : chunk_of(gt.pa, q);
+        const uint4 *src = c.slab_rec + (size_t)(t0 + lt) * c.tile_rows + gt.oa[lt] + (q - gt.pa[lt]);
+        cp_async8(&dst.bk[base_a + q], src);
+        cp_async8(&dst.zw[base_a + q], reinterpret_cast<const uint2 *>(src) + 1);
+      }
+      for (uint32_t q0 = G.tid; q0 < ta; q0 += 4 * G.n) {      // their row indices, four loads in flight per thread
+        int32_t row[4];
+#pragma unroll
+        for (int e = 0; e < 4; e++) {
+          const uint32_t q = q0 + e * G.n;
+          if (q < ta) {
+            const int lt = OWNER ? (int)gt.own_a[q] : chunk_of(gt.pa, q);
+            const size_t tb = (size_t)(t0 + lt) * c.tile_rows;
+            row[e] = (int32_t)(tb + __ldcg(c.slab_idx + tb + gt.oall[lt] + (q - gt.pa[lt])));
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; e++) { const uint32_t q = q0 + e * G.n; if (q < ta) dst.row[base_a + q] = row[e]; }
+      }
+    } else if (take_act) {
       int lt_c = 0;            // the chunk of my previous row and where it ends: my rows rise, so large chunks are searched once
       uint32_t lim_c = 0;
       for (uint32_t q0 = G.tid; q0 < ta; q0 += 3 * G.n) {
@@ -387,6 +419,7 @@ __device__ __forceinline__ void first_fit_marks(const ReplicaPlan &pl, uint32_t 
 #define SMALL_SMEM (SEG_TINY * 24 + (TINY_BINS + 4) * 4 + TINY_CLASSES * 8)
 static_assert(SMALL_SMEM <= SMEM_GROUP, "a group's arrays fit its share of the block's shared memory");
 
+template <bool SLABS, bool FF>
 __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx &c, const Grp &G, int r, uint32_t b, int n,
                               int n_act, bool ordered, bool list_in, unsigned char *smem, BlockShared &sh,
                               const int64_t *s_cls_ttft, const int64_t *s_cls_tpot) {
@@ -418,9 +451,9 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
 
   // ---- a step that is not ordered: the inactive rows, listed by req_id behind the active ones --------
   if (!ordered && n_in > 0) {
-    if (c.slabs)
-      gather_replica<GROUP_THREADS, GROUP_TPT, true>(c, R1, r, G, gt, false, true, [](uint32_t, const uint4, int32_t) {},
-                                               [&](uint32_t pos, int32_t row) { s_row[pos] = row; });
+    if (SLABS)
+      gather_replica<GROUP_THREADS, GROUP_TPT, true, false>(c, R1, r, G, gt, false, true, [](uint32_t, const uint4, int32_t) {},
+                                                            [&](uint32_t pos, int32_t row) { s_row[pos] = row; });
     else
       for (int q = G.tid; q < n_in; q += G.n) s_row[q] = (int32_t)__ldg(reinterpret_cast<const uint4 *>(seg + n_act + q)).w;
     G.sync();
@@ -431,38 +464,42 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
     G.sync();
   }
 
-  // ---- gather: base, record words and row of the active rows; the inactive rows' places; aggregates ----
-  uint32_t n_run = 0;
-  int64_t sum_kv = 0;
-  uint64_t m_run = 0, m_q = 0;
-  auto take = [&](uint32_t pos, const uint4 rec, int32_t row) {
-    s_bk[pos] = ((uint64_t)rec.y << 32) | rec.x; s_zw[pos] = make_uint2(rec.z, rec.w); s_row[pos] = row;
-    const uint32_t cls = rec.w >> CREC_CLS_SHIFT;
-    if (((rec.z >> CREC_KIND_SHIFT) & 1u) == KIND_RUNNING) {
-      n_run++; sum_kv += (int64_t)(rec.z & CREC_LEN_MASK) + (rec.w & CREC_LEN_MASK); m_run |= 1ull << cls;
-    } else m_q |= 1ull << cls;
-  };
-  if (c.slabs) {
-    gather_replica<GROUP_THREADS, GROUP_TPT, true>(c, R1, r, G, gt, true, ordered && list_in, take,
-                                             [&](uint32_t pos, int32_t row) { a.order[b + n_act + pos] = row; });
+  // ---- gather: base, record words and row of the active rows; the inactive rows' places ----------------------
+  if (SLABS) {
+    GatherDst dst; dst.bk = s_bk; dst.zw = s_zw; dst.row = s_row;
+    gather_replica<GROUP_THREADS, GROUP_TPT, true, true>(c, R1, r, G, gt, true, ordered && list_in, [](uint32_t, const uint4, int32_t) {},
+                                                         [&](uint32_t pos, int32_t row) { a.order[b + n_act + pos] = row; }, dst);
+    cp_async_wait_all();
   } else {
     for (int q = G.tid; q < n_act; q += G.n) {
       const uint4 w0 = __ldg(reinterpret_cast<const uint4 *>(seg + q));
       const uint4 w1 = __ldg(reinterpret_cast<const uint4 *>(seg + q) + 1);
-      uint4 rec;
-      rec.x = w0.x; rec.y = w0.y;
-      rec.z = w1.x | (((w1.w >> 8) & 1u) << CREC_KIND_SHIFT) | (((w1.w >> 16) & 0x3fu) << CREC_PRIO_SHIFT);
-      rec.w = w1.y | ((w1.w & 0x3fu) << CREC_CLS_SHIFT);
-      take((uint32_t)q, rec, (int32_t)w0.w);
+      s_bk[q] = ((uint64_t)w0.y << 32) | w0.x;
+      s_zw[q] = make_uint2(w1.x | (((w1.w >> 8) & 1u) << CREC_KIND_SHIFT) | (((w1.w >> 16) & 0x3fu) << CREC_PRIO_SHIFT),
+                           w1.y | ((w1.w & 0x3fu) << CREC_CLS_SHIFT));
+      s_row[q] = (int32_t)w0.w;
     }
   }
+  G.sync();       // the gather is over: its tile descriptors may be overwritten
 
   // ---- aggregates -> plan ----------------------------------------------------------------------------
+  uint32_t n_run = 0;
+  int64_t sum_kv = 0;
+  uint64_t m_run = 0, m_q = 0;
+#pragma unroll
+  for (int k = 0; k < TINY_IPT; k++) {
+    const int q = G.tid + k * GROUP_THREADS;
+    if (q < n_act) {
+      const uint2 zw = s_zw[q];
+      const uint32_t cls = zw.y >> CREC_CLS_SHIFT;
+      if (((zw.x >> CREC_KIND_SHIFT) & 1u) == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(zw.x & CREC_LEN_MASK) + (zw.y & CREC_LEN_MASK); m_run |= 1ull << cls; }
+      else m_q |= 1ull << cls;
+    }
+  }
   n_run = __reduce_add_sync(0xffffffffu, n_run);
   sum_kv = warp_sum_i64(sum_kv);
   m_run = ((uint64_t)__reduce_or_sync(0xffffffffu, (uint32_t)(m_run >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)m_run);
   m_q = ((uint64_t)__reduce_or_sync(0xffffffffu, (uint32_t)(m_q >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)m_q);
-  G.sync();       // the gather is over: its tile descriptors may be overwritten
   if (lane == 0) { sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_m0[warp] = m_run; sh.red_m1[warp] = m_q; }
   for (int i = G.tid; i < TINY_BINS / 2 + 2; i += G.n) s_bin[i] = 0;
   for (int i = G.tid; i < TINY_CLASSES; i += G.n) { s_cmin[i] = 0xffffffffu; s_cmax[i] = 0; s_ccnt[i] = 0; }
@@ -630,7 +667,7 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
   };
 
   // ---- first-fit variant: the first warp walks the order and marks what it takes (bit 17) -----------
-  if (p.first_fit)
+  if (FF)
     first_fit_marks(pl, s_lo, n_act, G, [&](int64_t q) -> int64_t { int64_t kv; return cost_at(s_lo[q] & 0xffffu, kv); });
 
   // ---- admission: each thread walks TINY_IPT consecutive places of the order ---------------------
@@ -646,7 +683,7 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
       int64_t kv = 0;
       const int64_t cc = cost_at(li, kv);
       // what counts towards the totals: rows that fit alone, or (first fit) exactly the rows taken
-      if (cc >= 0 && (p.first_fit ? (s_lo[q] & 0x20000u) != 0 : cc <= pl.budget)) { cand[k] = li | 0x80000000u; mine += (uint64_t)cc + (1ull << 48); }
+      if (cc >= 0 && (FF ? (s_lo[q] & 0x20000u) != 0 : cc <= pl.budget)) { cand[k] = li | 0x80000000u; mine += (uint64_t)cc + (1ull << 48); }
       a.order[b + q] = s_row[li];
     }
   }
@@ -666,7 +703,7 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
       int64_t kv = 0;
       const int64_t cc = cost_at(li, kv);
       run_c += cc; run_n += 1;
-      if (p.first_fit || (run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap))) {
+      if (FF || (run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap))) {
         ac += cc; ak += kv; an++;
         const int32_t row = s_row[li];
         a.admit[row] = 1;
@@ -729,7 +766,7 @@ __device__ void gather_to_records(const SegArgs &a, const SegCtx &c, int R1, int
                                   bool list_in, unsigned char *smem) {
   const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
   HfxRec *seg = c.rec + b;
-  gather_replica<REP_THREADS, 1, false>(c, R1, r, B, gather_tiles_at(smem, REP_THREADS, REP_THREADS), true, list_in || !ordered,
+  gather_replica<REP_THREADS, 1, false, false>(c, R1, r, B, gather_tiles_at(smem, REP_THREADS, REP_THREADS), true, list_in || !ordered,
                  [&](uint32_t pos, const uint4 rec, int32_t row) {
                    uint4 w0, w1;
                    w0.x = rec.x; w0.y = rec.y; w0.z = ordered ? 0u : (uint32_t)__ldg(a.req_id + row); w0.w = (uint32_t)row;
@@ -782,11 +819,12 @@ __device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &
 // Block-wide admission over the sorted items s_lo[0..n_sorted) (low 16 bits = position of the
 // record inside the segment): writes order, admit and the compacted admitted list, keeps each
 // decision in bit 16 of s_lo, accumulates the totals in sh.
+template <bool FF>
 __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs &a, const ReplicaPlan &pl,
                                               const HfxRec *seg, uint32_t b, uint32_t *s_lo, int n_sorted,
                                               BlockShared &sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  if (p.first_fit) {
+  if (FF) {
     const Grp B = {(int)threadIdx.x, (int)blockDim.x, 0};
     first_fit_marks(pl, s_lo, n_sorted, B, [&](int64_t q) -> int64_t {
       const uint4 w1 = ld_rec(seg + (s_lo[q] & 0xffffu), 1);
@@ -816,7 +854,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
       if (kind == KIND_QUEUED) {
         kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
         const int64_t c = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-        if (p.first_fit ? (s_lo[q] & 0x20000u) != 0 : c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
+        if (FF ? (s_lo[q] & 0x20000u) != 0 : c <= pl.budget) { cost = c; cnt = 1; } else kv = 0;
       }
       a.order[b + q] = row;
     }
@@ -839,7 +877,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
     sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
     bool adm = false;
-    if (cnt) adm = p.first_fit || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
+    if (cnt) adm = FF || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
     if (q < n_sorted) {
       if (adm) a.admit[row] = 1;
       if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
@@ -859,7 +897,7 @@ __device__ __forceinline__ void segment_admit(const HfxParams &p, const SegArgs 
     // Admission along the order is closed under prefixes: once the running cost is over the budget, or the
     // batch is full, nothing behind is admitted; and once the order has reached the queue, nothing behind is
     // in flight.  The rest of the order then only has to be written out.
-    if (!p.first_fit && sh.carry_act &&
+    if (!FF && sh.carry_act &&
         (sh.carry_cost > pl.budget || (pl.batch_cap != 0 && pl.n_eff + sh.carry_count >= pl.batch_cap))) {
       for (int q = tile + blockDim.x + threadIdx.x; q < n_sorted; q += blockDim.x) {
         const uint32_t li = s_lo[q] & 0xffffu;
@@ -973,6 +1011,7 @@ __device__ __forceinline__ void sort64_positions(uint64_t *hi, uint32_t *pos_out
   }
 }
 
+template <bool SLABS, bool FF>
 __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCtx &c, int r, uint32_t b, int n, int n_act,
                                bool ordered, bool list_in, unsigned char *smem, BlockShared &sh) {
   uint64_t *s_hi = reinterpret_cast<uint64_t *>(smem);
@@ -983,7 +1022,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
   const HfxRec *seg = c.rec + b;
   const bool real = r < R;    // bucket R holds rows bound to no replica
   // ---- gather into contiguous records -----------------------------------------------------------------
-  if (c.slabs) gather_to_records(a, c, R + 1, r, b, n_act, ordered, list_in, smem);
+  if (SLABS) gather_to_records(a, c, R + 1, r, b, n_act, ordered, list_in, smem);
 
   // ---- inactive rows of a step that is not ordered: listed by req_id behind the active ones ----
   if (!ordered && n_in > 0) {
@@ -1032,7 +1071,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
   __syncthreads();
 
   // ---- admission -------------------------------------------------------------------------------------------
-  segment_admit(p, a, pl, seg, b, s_lo, n_act, sh);
+  segment_admit<FF>(p, a, pl, seg, b, s_lo, n_act, sh);
 
   // ---- maturity, iteration clock ------------------------------------------------------------------
   if (threadIdx.x == 0) {
@@ -1108,6 +1147,7 @@ __device__ void block_global_sort(uint64_t *hi, uint32_t *lo, uint32_t *idx, int
   }
 }
 
+template <bool SLABS, bool FF>
 __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const SegCtx &c, int r, uint32_t b, int64_t n, int64_t n_act,
                                  bool ordered, bool list_in, unsigned char *smem, BlockShared &sh) {
   const int R = p.n_replicas;
@@ -1116,7 +1156,7 @@ __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const Seg
   const int64_t n_in = n - n_act;
   const HfxRec *seg = c.rec + b;
   const bool real = r < R;
-  if (c.slabs) gather_to_records(a, c, R + 1, r, b, n_act, ordered, list_in, smem);
+  if (SLABS) gather_to_records(a, c, R + 1, r, b, n_act, ordered, list_in, smem);
 
   // ---- inactive rows of a step that is not ordered: by req_id behind the active ones -----------
   if (!ordered && n_in > 0) {
@@ -1156,7 +1196,7 @@ __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const Seg
   block_global_sort(hi, lo, idx, n_act);
 
   // admission walk with a carried prefix
-  if (p.first_fit) {     // the first warp walks the order; lo (free now that the sort is over) says what it took
+  if (FF) {     // the first warp walks the order; lo (free now that the sort is over) says what it took
     if (warp == 0) {
       const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
       warp_first_fit(n_act, pl.budget, room, lane,
@@ -1182,7 +1222,7 @@ __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const Seg
       if (kind == KIND_QUEUED) {
         kv = (int64_t)(int32_t)w1.x + (int32_t)w1.y;
         const int64_t cc = pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(int32_t)w1.x;
-        if (p.first_fit ? lo[q] == 2u : cc <= pl.budget) { cost = cc; cnt = 1; } else kv = 0;
+        if (FF ? lo[q] == 2u : cc <= pl.budget) { cost = cc; cnt = 1; } else kv = 0;
       }
       a.order[b + q] = row;
     }
@@ -1200,7 +1240,7 @@ __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const Seg
     sc += sh.carry_cost + (warp ? sh.red_a[warp - 1] : 0);
     sn += sh.carry_count + (warp ? (int32_t)sh.red_b[warp - 1] : 0);
     bool adm = false;
-    if (cnt) adm = p.first_fit || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
+    if (cnt) adm = FF || (sc <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + sn <= pl.batch_cap));
     if (q < n_act) {
       if (adm) a.admit[row] = 1;
       if (adm && a.admitted_rows) a.admitted_rows[b + sn - 1] = row;
@@ -1252,6 +1292,7 @@ __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const Seg
 // ------------------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------------------
+template <bool SLABS, bool FF>
 __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, const SegArgs a, const SegCtx c) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ BlockShared sh_g[REP_GROUPS];
@@ -1270,11 +1311,11 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
   // everything below reads what the front end wrote
   cudaGridDependencySynchronize();
 
-  const bool ordered = c.slabs ? __ldcg(c.ordered) != 0 : false;
+  const bool ordered = SLABS ? __ldcg(c.ordered) != 0 : false;
   const uint32_t *begin = c.seg_begin;
   int larger = 1, longer = 0;       // does any replica need the whole block?  does any list of inactive rows need the grid?
   __syncthreads();
-  if (c.slabs) {
+  if (SLABS) {
     // range starts: exclusive prefix of the rows per replica, every block its own copy
     const int per = (R1 + blockDim.x - 1) / blockDim.x;
     const int i0 = tid * per < R1 ? tid * per : R1, i1 = (i0 + per < R1) ? i0 + per : R1;
@@ -1311,7 +1352,7 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
     __syncthreads();
   }
   auto counts = [&](int r, uint32_t &n_all, uint32_t &n_act) {
-    if (c.slabs) { const unsigned long long t = __ldcg(c.tot + r); n_all = (uint32_t)t; n_act = (uint32_t)(t >> 32); }
+    if (SLABS) { const unsigned long long t = __ldcg(c.tot + r); n_all = (uint32_t)t; n_act = (uint32_t)(t >> 32); }
     else { n_all = c.seg_count[r]; n_act = c.act_count[r]; }
   };
   auto need_of = [&](uint32_t n_all, uint32_t n_act) -> uint32_t {
@@ -1329,7 +1370,7 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
       if (need_of(n_all, n_act) > SEG_TINY) continue;
       if (r == R && n_all == 0) continue;
       const bool list_in = !ordered || n_all - n_act <= LIST_MAX;
-      small_replica(p, a, c, G, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw + (size_t)g * SMEM_GROUP, sh_g[g],
+      small_replica<SLABS, FF>(p, a, c, G, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw + (size_t)g * SMEM_GROUP, sh_g[g],
                     s_cls_ttft, s_cls_tpot);
     }
   }
@@ -1343,8 +1384,8 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
     const uint32_t need = need_of(n_all, n_act);
     if (need <= SEG_TINY) continue;
     const bool list_in = !ordered || n_all - n_act <= LIST_MAX;
-    if (need <= SEG_MED) medium_replica(p, a, c, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw, sh_g[0]);
-    else oversize_replica(p, a, c, r, begin[r], n_all, n_act, ordered, list_in, smem_raw, sh_g[0]);
+    if (need <= SEG_MED) medium_replica<SLABS, FF>(p, a, c, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw, sh_g[0]);
+    else oversize_replica<SLABS, FF>(p, a, c, r, begin[r], n_all, n_act, ordered, list_in, smem_raw, sh_g[0]);
   }
 
   // ---- long lists of inactive rows (ordered steps): every block lists a range of tiles ----------------
@@ -1412,13 +1453,18 @@ int hfx_launch_replicas(hfx_sched *s, const SegArgs &sa, int64_t n, bool slabs) 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = (slabs && !s->profiling) ? 1 : 0;      // the kernel may be set up while the tile front end drains
-  if (cudaLaunchKernelEx(&cfg, k_replicas, s->p, sa, c) != cudaSuccess) return HFX_E_CUDA;
-  return HFX_OK;
+  cudaError_t e;
+  if (slabs) e = s->p.first_fit ? cudaLaunchKernelEx(&cfg, k_replicas<true, true>, s->p, sa, c) : cudaLaunchKernelEx(&cfg, k_replicas<true, false>, s->p, sa, c);
+  else e = s->p.first_fit ? cudaLaunchKernelEx(&cfg, k_replicas<false, true>, s->p, sa, c) : cudaLaunchKernelEx(&cfg, k_replicas<false, false>, s->p, sa, c);
+  return e == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }
 
 int hfx_segment_configure() {
-  if (cudaFuncSetAttribute(k_replicas, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           SMEM_MED + sizeof(uint32_t) * (HFX_TILE_REPLICAS_MAX + 3)) != cudaSuccess)
+  const int smem = (int)(SMEM_MED + sizeof(uint32_t) * (HFX_TILE_REPLICAS_MAX + 3));
+  if (cudaFuncSetAttribute(k_replicas<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaFuncSetAttribute(k_replicas<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaFuncSetAttribute(k_replicas<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaFuncSetAttribute(k_replicas<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }
