@@ -126,10 +126,16 @@ class ClockSampler:
 
 
 def _workload(rank: int, args):
+    if args.workload == "config2":        # (profiling aid: the bench line is config 4)
+        return gen.config2(seed=2 + rank, inflight=0.02)
+    if args.workload == "config3":
+        return gen.config3(seed=3 + rank)
     return gen.config4(seed=4 + rank, R=args.replicas, n=args.rows, steps=STEPS_PER_EPISODE)
 
 
-def _workload_name(n, R):
+def _workload_name(n, R, which="config4"):
+    if which != "config4":
+        return "%s: %d requests over %d replicas (see gen/workloads.py); not the benchmark configuration" % (which, n, R)
     return ("config4: shared queue, %d requests over %d replicas (rows interleaved), 5 SLO tiers, priority "
             "weights, Pareto prompts, committed steps with in-flight state carried over" % (n, R))
 
@@ -189,6 +195,8 @@ def run_gpu(args):
     wl = _workload(rank, args)
     n, R = wl.n_rows, wl.n_replicas
     sched = hfx.Scheduler(wl.model, wl.classes, wl.replicas, n, budget_mode=wl.budget_mode, weight_max=wl.weight_max)
+    if args.front == "fallback":
+        sched.set_fused_front(False)
     tab = hfx.DeviceTable.from_numpy(wl.table)
     init = {k: v.clone() for k, v in tab.cols.items()}
     now0 = torch.from_numpy(wl.now).cuda(); mat0 = torch.from_numpy(wl.maturity).cuda()
@@ -532,7 +540,7 @@ def run_gpu(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-                "config": {"workload": _workload_name(n, R),
+                "config": {"workload": _workload_name(n, R, args.workload), "front_end": args.front,
                            "rows_per_gpu": n, "replicas_per_gpu": R, "parallelism": "replica shards, no collective",
                            "l2": "flushed between steps (256 MiB write, outside the per-step events)",
                            "episode": "table restored every %d steps, outside the events" % STEPS_PER_EPISODE,
@@ -557,6 +565,9 @@ def main():
     ap.add_argument("--replicas", type=int, default=1024)
     ap.add_argument("--sim-traces", type=int, default=4096)
     ap.add_argument("--sim-iters", type=int, default=10000)
+    ap.add_argument("--workload", default="config4", choices=["config4", "config2", "config3"],
+                    help="step configuration to time (profiling aid; the benchmark line is config4)")
+    ap.add_argument("--front", default="tile", choices=["tile", "fallback"], help="front end of the step (profiling aid)")
     ap.add_argument("--no-sim", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-dispatch", action="store_true")
