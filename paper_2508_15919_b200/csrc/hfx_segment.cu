@@ -411,6 +411,34 @@ __device__ __forceinline__ void first_fit_marks(const ReplicaPlan &pl, uint32_t 
   G.sync();
 }
 
+// Distribution sort, bin layout (one warp; all 32 lanes call): every (phase, priority) class gets a share of the
+// n_bins bins in proportion to its items (a power of two; the shares add up to at most n_bins - TINY_CLASSES) and
+// the shift that maps its range of sub-keys onto its bins.  cinfo[class] = (smallest sub-key, first bin | shift << 16).
+template <int N_BINS>
+__device__ __forceinline__ void layout_class_bins(const uint32_t *s_ccnt, const uint32_t *s_cmin, const uint32_t *s_cmax, uint2 *s_cinfo,
+                                                  uint32_t n_items, int lane) {
+  uint32_t nb[TINY_CLASSES / 32], sft[TINY_CLASSES / 32], lo_[TINY_CLASSES / 32];
+  uint32_t sum = 0;
+#pragma unroll
+  for (int e = 0; e < TINY_CLASSES / 32; e++) {
+    const int cl = lane * (TINY_CLASSES / 32) + e;
+    const uint32_t cnt = s_ccnt[cl], lo = s_cmin[cl], hi = s_cmax[cl];
+    uint32_t want = cnt * (uint32_t)(N_BINS - TINY_CLASSES) / n_items;
+    nb[e] = cnt ? (want > 1 ? 1u << (31 - __clz(want)) : 1u) : 0u;
+    const uint32_t range = cnt ? hi - lo : 0u;
+    const int bits = 32 - __clz(range), lg = 31 - __clz(nb[e] | 1u);
+    sft[e] = bits > lg ? (uint32_t)(bits - lg) : 0u;       // (range >> sft) < nb
+    lo_[e] = lo;
+    sum += nb[e];
+  }
+  uint32_t v = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+  uint32_t run = v - sum;
+#pragma unroll
+  for (int e = 0; e < TINY_CLASSES / 32; e++) { s_cinfo[lane * (TINY_CLASSES / 32) + e] = make_uint2(lo_[e], run | (sft[e] << 16)); run += nb[e]; }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Small replicas: one group of 128 threads.  What later passes need of the replica's active rows
 // (slack base, record words, row) is staged once in shared memory; sort items live in registers
@@ -559,28 +587,7 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
   bool sorted_done = false;
   if (ordered && n_act > 0) {
     G.sync();
-    if (warp == 0) {     // bins per class in proportion to its items (a power of two), the shift that fits its range
-      uint32_t nb[TINY_CLASSES / 32], sft[TINY_CLASSES / 32], lo_[TINY_CLASSES / 32];
-      uint32_t sum = 0;
-#pragma unroll
-      for (int e = 0; e < TINY_CLASSES / 32; e++) {
-        const int cl = lane * (TINY_CLASSES / 32) + e;
-        const uint32_t cnt = s_ccnt[cl], lo = s_cmin[cl], hi = s_cmax[cl];
-        uint32_t want = cnt * (TINY_BINS - TINY_CLASSES) / (uint32_t)n_act;      // the shares add up to at most TINY_BINS - TINY_CLASSES
-        nb[e] = cnt ? (want > 1 ? 1u << (31 - __clz(want)) : 1u) : 0u;
-        const uint32_t range = cnt ? hi - lo : 0u;
-        const int bits = 32 - __clz(range), lg = 31 - __clz(nb[e] | 1u);
-        sft[e] = bits > lg ? (uint32_t)(bits - lg) : 0u;       // (range >> sft) < nb
-        lo_[e] = lo;
-        sum += nb[e];
-      }
-      uint32_t v = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
-      uint32_t run = v - sum;
-#pragma unroll
-      for (int e = 0; e < TINY_CLASSES / 32; e++) { s_cinfo[lane * (TINY_CLASSES / 32) + e] = make_uint2(lo_[e], run | (sft[e] << 16)); run += nb[e]; }
-    }
+    if (warp == 0) layout_class_bins<TINY_BINS>(s_ccnt, s_cmin, s_cmax, s_cinfo, (uint32_t)n_act, lane);
     G.sync();
     auto bin_of = [&](uint64_t x) -> uint32_t {
       const uint2 ci = s_cinfo[(uint32_t)(x >> 56)];
@@ -786,19 +793,10 @@ __device__ void gather_to_records(const SegArgs &a, const SegCtx &c, int R1, int
   __syncthreads();
 }
 
-// aggregates of a replica's active records into the block's plan (all threads call; result in sh.plan)
-__device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &a, const HfxRec *seg, int64_t n_act, int r,
-                                             bool real, BlockShared &sh) {
+// the block's partial aggregates of a replica's active rows -> its plan (all threads call; result in sh.plan)
+__device__ __forceinline__ void block_plan(const HfxParams &p, const SegArgs &a, int r, bool real, BlockShared &sh,
+                                           int64_t n_run, int64_t sum_kv, uint64_t m_run, uint64_t m_q) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  int64_t n_run = 0, sum_kv = 0;
-  uint64_t m_run = 0, m_q = 0;
-#pragma unroll 4
-  for (int64_t q = threadIdx.x; q < n_act; q += blockDim.x) {
-    const uint4 w1 = ld_rec(seg + q, 1);   // prompt, gen, -, bytes
-    const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
-    if (kind == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
-    else m_q |= 1ull << cls;
-  }
   n_run = warp_sum_i64(n_run); sum_kv = warp_sum_i64(sum_kv);
   m_run = warp_or_u64(m_run); m_q = warp_or_u64(m_q);
   if (lane == 0) { sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_m0[warp] = m_run; sh.red_m1[warp] = m_q; }
@@ -814,6 +812,21 @@ __device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &
     sh.adm_cost = 0; sh.adm_kv = 0; sh.adm_count = 0;
   }
   __syncthreads();
+}
+
+// aggregates of a replica's active records into the block's plan (all threads call; result in sh.plan)
+__device__ __forceinline__ void segment_plan(const HfxParams &p, const SegArgs &a, const HfxRec *seg, int64_t n_act, int r,
+                                             bool real, BlockShared &sh) {
+  int64_t n_run = 0, sum_kv = 0;
+  uint64_t m_run = 0, m_q = 0;
+#pragma unroll 4
+  for (int64_t q = threadIdx.x; q < n_act; q += blockDim.x) {
+    const uint4 w1 = ld_rec(seg + q, 1);   // prompt, gen, -, bytes
+    const int kind = (w1.w >> 8) & 0xff, cls = w1.w & 0xff;
+    if (kind == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(int32_t)w1.x + (int32_t)w1.y; m_run |= 1ull << cls; }
+    else m_q |= 1ull << cls;
+  }
+  block_plan(p, a, r, real, sh, n_run, sum_kv, m_run, m_q);
 }
 
 // Block-wide admission over the sorted items s_lo[0..n_sorted) (low 16 bits = position of the
@@ -1110,6 +1123,334 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
 }
 
 // ------------------------------------------------------------------------------------------------
+// Larger replicas of an ordered step on the slab layout: the whole block with a distribution sort.
+// The replica's scratch range of c.rec (32 bytes per row, of which 20 per active row are used) holds three
+// arrays by position q in row order: slack base, then sort item (8 bytes); record words z, w (8); row (4).
+// Every pass reads them front to back; shared memory holds the binned items (afterwards the record words), the
+// order as 16-bit positions and the bin counters.
+// ------------------------------------------------------------------------------------------------
+#define MED_BINS 8192     // bins of the block's distribution sort (16-bit counters, two to a word)
+#define MED_BIN_MAX 160   // fuller bins send the replica to the sorting network
+static_assert((size_t)SEG_MED * 10 + MED_BINS * 4 <= SMEM_MED, "items, order and bins of a medium replica fit the block's shared memory");
+static_assert(MED_BINS / 8 == REP_THREADS, "every thread scans eight bins");
+
+template <bool FF>
+__device__ void medium_ordered(const HfxParams &p, const SegArgs &a, const SegCtx &c, int r, uint32_t b, int n, int n_act,
+                               bool list_in, unsigned char *smem, BlockShared &sh, uint64_t *s_cinfo,
+                               const int64_t *s_cls_ttft, const int64_t *s_cls_tpot) {
+  uint64_t *s_item = reinterpret_cast<uint64_t *>(smem);                          // [SEG_MED] items by bin
+  uint2 *s_zw = reinterpret_cast<uint2 *>(smem);                                  // [SEG_MED] afterwards: record words by position; bit 31 of x: taken by first fit, of y: admitted
+  uint16_t *s_ord = reinterpret_cast<uint16_t *>(smem + (size_t)SEG_MED * 8);     // [SEG_MED] position of the i-th row of the order
+  uint32_t *s_bin = reinterpret_cast<uint32_t *>(smem + (size_t)SEG_MED * 10);    // [MED_BINS / 2] bin counts, then bin starts
+  uint32_t *s_cur = s_bin + MED_BINS / 2;                                         // [MED_BINS / 2] fill cursors, then bin ends
+  uint32_t *s_lo = reinterpret_cast<uint32_t *>(s_ord);                           // (sorting network only: 32-bit positions over order and bins)
+  // until the bins are laid out: per class the smallest and largest of the slack's upper 32 bits and of its low 8 bits, the items
+  uint32_t *s_cmin = reinterpret_cast<uint32_t *>(s_ord), *s_cmax = s_cmin + TINY_CLASSES, *s_lmin = s_cmax + TINY_CLASSES,
+           *s_lmax = s_lmin + TINY_CLASSES, *s_ccnt = s_lmax + TINY_CLASSES;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int R = p.n_replicas;
+  const bool real = r < R;    // bucket R holds rows bound to no replica
+  const Grp B = {tid, REP_THREADS, 0};
+  unsigned char *g = reinterpret_cast<unsigned char *>(c.rec + b);
+  uint64_t *g_item = reinterpret_cast<uint64_t *>(g);
+  uint2 *g_zw = reinterpret_cast<uint2 *>(g + (size_t)n_act * 8);
+  int32_t *g_row = reinterpret_cast<int32_t *>(g + (size_t)n_act * 16);
+
+  // ---- gather into the scratch arrays; the inactive rows go straight to their places -------------------
+  gather_replica<REP_THREADS, 1, false, false>(c, R + 1, r, B, gather_tiles_at(smem, REP_THREADS, REP_THREADS), true, list_in,
+                 [&](uint32_t pos, const uint4 rec, int32_t row) {
+                   g_item[pos] = ((uint64_t)rec.y << 32) | rec.x; g_zw[pos] = make_uint2(rec.z, rec.w); g_row[pos] = row;
+                 },
+                 [&](uint32_t pos, int32_t row) { a.order[b + n_act + pos] = row; });
+  __syncthreads();
+
+  // ---- aggregates, plan ---------------------------------------------------------------------------------
+  {
+    int64_t n_run = 0, sum_kv = 0;
+    uint64_t m_run = 0, m_q = 0;
+#pragma unroll 4
+    for (int q = tid; q < n_act; q += REP_THREADS) {
+      const uint2 zw = g_zw[q];
+      const uint32_t cls = zw.y >> CREC_CLS_SHIFT;
+      if (((zw.x >> CREC_KIND_SHIFT) & 1u) == KIND_RUNNING) { n_run++; sum_kv += (int64_t)(zw.x & CREC_LEN_MASK) + (zw.y & CREC_LEN_MASK); m_run |= 1ull << cls; }
+      else m_q |= 1ull << cls;
+    }
+    for (int i = tid; i < MED_BINS / 2; i += REP_THREADS) s_bin[i] = 0;
+    for (int i = tid; i < TINY_CLASSES; i += REP_THREADS) { s_cmin[i] = 0xffffffffu; s_cmax[i] = 0; s_lmin[i] = 0xffu; s_lmax[i] = 0; s_ccnt[i] = 0; }
+    n_run = warp_sum_i64(n_run); sum_kv = warp_sum_i64(sum_kv);
+    m_run = warp_or_u64(m_run); m_q = warp_or_u64(m_q);
+    if (lane == 0) { sh.red_a[warp] = n_run; sh.red_b[warp] = sum_kv; sh.red_m0[warp] = m_run; sh.red_m1[warp] = m_q; }
+    __syncthreads();
+    if (warp == 0) {     // the first warp finishes the reduction and plans
+      n_run = warp_sum_i64(sh.red_a[lane]); sum_kv = warp_sum_i64(sh.red_b[lane]);
+      m_run = warp_or_u64(sh.red_m0[lane]); m_q = warp_or_u64(sh.red_m1[lane]);
+      hfx_replica_cfg cfg; cfg.mode = HFX_COLOCATED; cfg.token_cap = 1; cfg.batch_cap = 0;
+      int64_t now = 0, mat = 0;
+      if (real) { cfg = a.cfg[r]; now = a.now[r]; mat = a.mat[r]; }
+      ReplicaPlan pl0;
+      warp_plan(p, s_cls_ttft, s_cls_tpot, cfg, now, mat, n_run, sum_kv, m_run, m_q, pl0, lane);
+      if (lane == 0) { sh.plan = pl0; sh.next_arrival = HFX_INF; }
+    }
+    __syncthreads();
+  }
+  const ReplicaPlan pl = sh.plan;
+
+  // ---- sort items (into the scratch, over the bases); per class their range ------------------------
+  {
+    const int n_rounds = (n_act + REP_THREADS - 1) / REP_THREADS;
+    int64_t base_n = 0; uint2 zw_n = make_uint2(0u, 0u); int32_t row_n = 0;      // the next round's row, asked for a round ahead
+    if (tid < n_act) { base_n = (int64_t)g_item[tid]; zw_n = g_zw[tid]; row_n = g_row[tid]; }
+    for (int q0 = 0; q0 < n_act; q0 += REP_THREADS) {
+      if (q0 + (tid & ~31) >= n_act) break;      // (whole warps leave)
+      const int q = q0 + tid;
+      const bool in = q < n_act;
+      const int64_t base = base_n; const uint2 zw = zw_n; const int32_t row = row_n;
+      if (q + REP_THREADS < n_act) { base_n = (int64_t)g_item[q + REP_THREADS]; zw_n = g_zw[q + REP_THREADS]; row_n = g_row[q + REP_THREADS]; }
+      uint64_t item = ~0ull;
+      if (in) {
+        const int kind = (zw.x >> CREC_KIND_SHIFT) & 1, prio = zw.x >> CREC_PRIO_SHIFT;
+        const bool given = kind == KIND_QUEUED && pl.mode != HFX_DECODE;      // the front end has put the row's final key in place of the base
+        RowEval ev;
+        if (given) { ev.k48 = (uint64_t)base; ev.slack = 0; ev.pred_tpot = a.pred_tpot ? pl.tpot_q0 + p.d2 * ((int64_t)(zw.x & CREC_LEN_MASK) + (zw.y & CREC_LEN_MASK)) : 0; }
+        else ev = eval_row(p, pl, base, kind, prio, (int32_t)(zw.x & CREC_LEN_MASK), (int32_t)(zw.y & CREC_LEN_MASK));
+        item = (ev.k48 << 16) | (uint32_t)q;     // rows were gathered in req_id order: position breaks ties
+        g_item[q] = item;
+        if (!given) {    // (the front end wrote the slack of the other queued rows)
+          a.slack[row] = ev.slack;
+          if (a.key) a.key[row] = ((uint64_t)(r & 0xffff) << 48) | ev.k48;
+        }
+        if (a.pred_tpot) a.pred_tpot[row] = ev.pred_tpot;
+      }
+      // Ranges of the slacks per class, from a sample: in every round one warp in n_rounds looks (a different one each
+      // round, so the sample is spread over the replica's rows).  The warp's rows of one class update the class's range
+      // together.  The smallest upper part joined to the smallest low part is a lower bound of the sampled slacks of
+      // the class, likewise an upper bound; both are exact when they are all equal (requests without a bound).
+      if ((warp + (q0 >> 10)) % n_rounds == 0) {
+        const uint32_t cl = in ? (uint32_t)(item >> 56) : 0xffu, up = (uint32_t)(item >> 24), low = (uint32_t)(item >> 16) & 0xffu;
+        const uint32_t same = __match_any_sync(0xffffffffu, cl);
+        const uint32_t mn = __reduce_min_sync(same, up), mx = __reduce_max_sync(same, up);
+        const uint32_t mn_low = __reduce_min_sync(same, low), mx_low = __reduce_max_sync(same, low);
+        if (in && lane == __ffs(same) - 1) {
+          atomicMin(&s_cmin[cl], mn); atomicMax(&s_cmax[cl], mx); atomicMin(&s_lmin[cl], mn_low); atomicMax(&s_lmax[cl], mx_low);
+          atomicAdd(&s_ccnt[cl], (uint32_t)__popc(same));
+        }
+      }
+    }
+  }
+  __syncthreads();
+
+  // ---- sort: bins by class and sub-key, places inside a bin by counting ------------------------------
+  // An item's place in its class's order is (slack - smallest slack of the class) << 16 | position, at most
+  // (range of slacks) << 16 | (n_act - 1); the class's bins divide that evenly, so equal slacks spread by position.
+  // Every class has a bin, sampled or not; what falls outside the sampled range goes to the class's first or last
+  // bin, which keeps the bins in item order.
+  if (warp == 0) {
+    uint32_t cnt[TINY_CLASSES / 32], seen = 0;
+#pragma unroll
+    for (int e = 0; e < TINY_CLASSES / 32; e++) { cnt[e] = s_ccnt[lane * (TINY_CLASSES / 32) + e]; seen += cnt[e]; }
+    seen = __reduce_add_sync(0xffffffffu, seen);
+    uint32_t lg[TINY_CLASSES / 32], sum = 0;
+#pragma unroll
+    for (int e = 0; e < TINY_CLASSES / 32; e++) {
+      const uint32_t want = seen ? cnt[e] * (uint32_t)(MED_BINS - TINY_CLASSES) / seen : 0u;      // the shares add up to at most MED_BINS - TINY_CLASSES, plus one bin per class
+      lg[e] = want > 1 ? 31 - __clz(want) : 0;
+      sum += 1u << lg[e];
+    }
+    uint32_t v = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+    uint32_t run = v - sum;
+#pragma unroll
+    for (int e = 0; e < TINY_CLASSES / 32; e++) {
+      const int cl = lane * (TINY_CLASSES / 32) + e;
+      unsigned long long lo = 0, range = 0;
+      if (cnt[e]) {
+        lo = ((unsigned long long)s_cmin[cl] << 8) | s_lmin[cl];
+        range = (((((unsigned long long)s_cmax[cl] << 8) | s_lmax[cl]) - lo) << 16) | (unsigned long long)(n_act - 1);
+      }
+      const int bits = 64 - __clzll((long long)range);
+      const unsigned long long sft = bits > (int)lg[e] ? (unsigned long long)(bits - (int)lg[e]) : 0ull;       // (range >> sft) < number of bins
+      s_cinfo[cl] = lo | ((unsigned long long)run << 40) | (sft << 53) | ((unsigned long long)lg[e] << 59);
+      run += 1u << lg[e];
+    }
+  }
+  __syncthreads();
+  auto bin_of = [&](uint64_t x) -> uint32_t {
+    const uint64_t ci = s_cinfo[(uint32_t)(x >> 56)];
+    const uint64_t v = x & ((1ull << 56) - 1), lo = (ci & ((1ull << 40) - 1)) << 16;
+    const uint32_t last = (1u << ((uint32_t)(ci >> 59) & 15u)) - 1u;
+    const uint64_t d = v > lo ? (v - lo) >> ((uint32_t)(ci >> 53) & 63u) : 0ull;
+    return ((uint32_t)(ci >> 40) & 0x1fffu) + (d < last ? (uint32_t)d : last);
+  };
+#pragma unroll 4
+  for (int q = tid; q < n_act; q += REP_THREADS) {
+    const uint32_t bi = bin_of(g_item[q]);
+    atomicAdd(&s_bin[bi >> 1], 1u << ((bi & 1u) * 16));
+  }
+  __syncthreads();
+  bool binned = false;
+  {   // exclusive scan of the bin counts, eight per thread; the fullest bin
+    const uint4 wd = reinterpret_cast<const uint4 *>(s_bin)[tid];
+    const uint32_t ww[4] = {wd.x, wd.y, wd.z, wd.w};
+    uint32_t cnt[8], sum = 0, big = 0;
+#pragma unroll
+    for (int i = 0; i < 4; i++) { cnt[2 * i] = ww[i] & 0xffffu; cnt[2 * i + 1] = ww[i] >> 16; }
+#pragma unroll
+    for (int i = 0; i < 8; i++) { sum += cnt[i]; big = cnt[i] > big ? cnt[i] : big; }
+    uint32_t v = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const uint32_t w = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += w; }
+    big = __reduce_max_sync(0xffffffffu, big);
+    if (lane == 31) sh.red_n[warp] = (int32_t)v;
+    if (lane == 0) sh.red_a[warp] = (int64_t)big;
+    __syncthreads();
+    uint32_t run = v - sum, bigall = 0;
+    for (int k = 0; k < REP_THREADS / 32; k++) { if (k < warp) run += (uint32_t)sh.red_n[k]; const uint32_t x = (uint32_t)sh.red_a[k]; bigall = x > bigall ? x : bigall; }
+    if (bigall <= MED_BIN_MAX) {
+      uint32_t st[8];
+#pragma unroll
+      for (int i = 0; i < 8; i++) { st[i] = run; run += cnt[i]; }
+      const uint4 o4 = make_uint4(st[0] | (st[1] << 16), st[2] | (st[3] << 16), st[4] | (st[5] << 16), st[6] | (st[7] << 16));
+      reinterpret_cast<uint4 *>(s_bin)[tid] = o4;
+      reinterpret_cast<uint4 *>(s_cur)[tid] = o4;
+      binned = true;
+    }
+  }
+  __syncthreads();
+  if (binned) {
+#pragma unroll 4
+    for (int q = tid; q < n_act; q += REP_THREADS) {
+      const uint64_t x = g_item[q];
+      const uint32_t bi = bin_of(x), sh16 = (bi & 1u) * 16;
+      const uint32_t pos = (atomicAdd(&s_cur[bi >> 1], 1u << sh16) >> sh16) & 0xffffu;
+      s_item[pos] = x;
+    }
+    __syncthreads();
+    for (int e = tid; e < n_act; e += REP_THREADS) {
+      const uint64_t x = s_item[e];
+      const uint32_t bi = bin_of(x), sh16 = (bi & 1u) * 16;
+      const uint32_t g0 = (s_bin[bi >> 1] >> sh16) & 0xffffu, g1 = (s_cur[bi >> 1] >> sh16) & 0xffffu;
+      uint32_t rank = 0;
+      for (uint32_t k = g0; k < g1; k++) rank += s_item[k] < x ? 1u : 0u;
+      s_ord[g0 + rank] = (uint16_t)(x & 0xffffu);      // (the class ranges that s_ord overlays were last read when the bins were laid out)
+    }
+  } else {      // a bin is too full: the sorting network
+    for (int q = tid; q < n_act; q += REP_THREADS) s_item[q] = g_item[q];
+    __syncthreads();
+    sort64_positions(s_item, s_lo, n_act);
+    __syncthreads();
+    for (int q0 = 0; q0 < n_act; q0 += REP_THREADS) {      // 32-bit positions -> 16-bit, in place: a chunk's writes land on words already read
+      const int q = q0 + tid;
+      const uint32_t v = q < n_act ? s_lo[q] : 0u;
+      __syncthreads();
+      if (q < n_act) s_ord[q] = (uint16_t)v;
+    }
+  }
+  __syncthreads();
+
+  // ---- the order; the record words by position, over the items -----------------------------------------
+#pragma unroll 4
+  for (int q = tid; q < n_act; q += REP_THREADS) {
+    a.order[b + q] = g_row[s_ord[q]];
+    const uint2 zw = g_zw[q];
+    s_zw[q] = make_uint2(zw.x & ((1u << CREC_PRIO_SHIFT) - 1u), zw.y);      // (the priority has served; its bits make room for the marks)
+  }
+  __syncthreads();
+
+  auto cost_at = [&](uint32_t li, int64_t &kv) -> int64_t {      // cost of the queued row at position li, -1 if it is in flight
+    const uint2 zw = s_zw[li];
+    if (((zw.x >> CREC_KIND_SHIFT) & 1u) != KIND_QUEUED) return -1;
+    kv = (int64_t)(zw.x & CREC_LEN_MASK) + (zw.y & CREC_LEN_MASK);
+    return pl.mode == HFX_DECODE ? p.d1 + p.d2 * kv : (int64_t)(zw.x & CREC_LEN_MASK);
+  };
+  if (FF) {     // first fit: the first warp walks the order and marks what it takes
+    if (warp == 0) {
+      const int64_t room = pl.batch_cap == 0 ? HFX_INF : (pl.batch_cap > pl.n_eff ? pl.batch_cap - pl.n_eff : 0);
+      warp_first_fit(n_act, pl.budget, room, lane, [&](int64_t q) -> int64_t { int64_t kv; return cost_at(s_ord[q], kv); },
+                     [&](int64_t q, bool taken) { if (taken) s_zw[s_ord[q]].x |= 0x80000000u; });
+    }
+    __syncthreads();
+  }
+
+  // ---- admission: every thread walks consecutive places of the order, twice -------------------------------
+  const int ipt = (n_act + REP_THREADS - 1) / REP_THREADS;
+  const int qa = tid * ipt < n_act ? tid * ipt : n_act, qb = qa + ipt < n_act ? qa + ipt : n_act;
+  int64_t my_cost = 0;
+  int32_t my_cnt = 0;
+  for (int q = qa; q < qb; q++) {      // what counts towards the running totals: rows that fit alone, or (first fit) exactly the rows taken
+    const uint32_t li = s_ord[q];
+    int64_t kv = 0;
+    const int64_t cc = cost_at(li, kv);
+    if (cc >= 0 && (FF ? (s_zw[li].x >> 31) != 0 : cc <= pl.budget)) { my_cost += cc; my_cnt++; }
+  }
+  int64_t run_c = warp_incl_scan_i64(my_cost, lane);
+  int32_t run_n = warp_incl_scan_i32(my_cnt, lane);
+  if (lane == 31) { sh.red_a[warp] = run_c; sh.red_n[warp] = run_n; }
+  __syncthreads();
+  run_c -= my_cost; run_n -= my_cnt;
+  for (int k = 0; k < warp; k++) { run_c += sh.red_a[k]; run_n += sh.red_n[k]; }
+  int64_t ac = 0, ak = 0;
+  int32_t an = 0;
+  if (my_cnt)
+    for (int q = qa; q < qb; q++) {
+      const uint32_t li = s_ord[q];
+      int64_t kv = 0;
+      const int64_t cc = cost_at(li, kv);
+      if (cc >= 0 && (FF ? (s_zw[li].x >> 31) != 0 : cc <= pl.budget)) {
+        run_c += cc; run_n += 1;
+        if (FF || (run_c <= pl.budget && (pl.batch_cap == 0 || pl.n_eff + run_n <= pl.batch_cap))) {
+          ac += cc; ak += kv; an++;
+          const int32_t row = g_row[li];
+          a.admit[row] = 1;
+          if (a.admitted_rows) a.admitted_rows[b + run_n - 1] = row;
+          s_zw[li].y |= 0x80000000u;
+        }
+      }
+    }
+  __syncthreads();      // (the scan's partial sums have been read)
+
+  // ---- totals, maturity, iteration clock ---------------------------------------------------------
+  ac = warp_sum_i64(ac); ak = warp_sum_i64(ak); an = (int32_t)__reduce_add_sync(0xffffffffu, (uint32_t)an);
+  if (lane == 0) { sh.red_a[warp] = ac; sh.red_b[warp] = ak; sh.red_n[warp] = an; }
+  __syncthreads();
+  if (tid == 0) {
+    int64_t adm_cost = 0, adm_kv = 0; int32_t adm_count = 0;
+    for (int k = 0; k < REP_THREADS / 32; k++) { adm_cost += sh.red_a[k]; adm_kv += sh.red_b[k]; adm_count += sh.red_n[k]; }
+    int64_t lp = 0;
+    const int64_t mat_next = dev_maturity_next(p, pl, adm_count, adm_cost, adm_kv, &lp);
+    int worked; int64_t t1, t2;
+    iteration_clock(pl, adm_count, lp, mat_next, worked, t1, t2);
+    sh.adm_cost = adm_cost; sh.adm_count = adm_count;
+    sh.worked = worked; sh.t1 = t1; sh.t2 = t2; sh.red_c[0] = mat_next;
+  }
+  __syncthreads();
+  const bool commit = real && (a.flags & HFX_COMMIT) && pl.now <= a.horizon;
+  const int worked = sh.worked;
+  const int64_t mat_next = sh.red_c[0];
+  if (commit && !worked)      // idle replica: its next arrival is looked up among its listed inactive rows
+    group_min_arrival(list_in ? next_arrival_listed(a, c, b, n_act, n, tid, REP_THREADS) : HFX_INF, sh, B);
+  if (tid == 0 && real)
+    write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
+
+  // ---- padding of the compacted list, commit ----------------------------------------------------
+  if (a.admitted_rows)
+    for (int q = sh.adm_count + tid; q < n; q += REP_THREADS) a.admitted_rows[b + q] = -1;
+  if (commit) {
+    const int64_t t1 = sh.t1, t2 = sh.t2;
+#pragma unroll 2
+    for (int q = tid; q < n_act; q += REP_THREADS) {
+      const uint2 zw = s_zw[q];
+      const int kind = (zw.x >> CREC_KIND_SHIFT) & 1;
+      const bool adm = (zw.y >> 31) != 0;
+      const int32_t row = g_row[q];
+      const int32_t out_len = commit_needs_out_len(pl, kind, adm, worked) ? __ldg(a.output_len + row) : 0;
+      commit_row(a, pl, kind, adm, worked, t1, t2, row, (int32_t)(zw.x & CREC_LEN_MASK), (int32_t)(zw.y & CREC_LEN_MASK), out_len);
+    }
+  }
+  __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
 // Oversize replicas (more items than a block sorts in shared memory): the block runs the sorting
 // network in global memory (items in c.big_hi / big_lo, the record positions travelling in big_idx),
 // then admission with a carried prefix.  Slow but exact.
@@ -1298,6 +1639,7 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
   __shared__ BlockShared sh_g[REP_GROUPS];
   __shared__ int64_t s_cls_ttft[HFX_MAX_CLASSES], s_cls_tpot[HFX_MAX_CLASSES];     // class tables for the planning warps
   __shared__ uint32_t s_scan[2 * 32 + 2];      // (also the scratch of the block-wide scans below)
+  __shared__ uint64_t s_cinfo_med[TINY_CLASSES];  // bin layout of a medium replica's distribution sort: smallest slack<40> | first bin<13> | shift<6> | log2 bins<4>
   __shared__ uint32_t s_long[(HFX_TILE_REPLICAS_MAX + 1 + 31) / 32 + 1];           // replicas whose inactive rows the grid lists together
   uint32_t *s_begin = reinterpret_cast<uint32_t *>(smem_raw + SMEM_MED);           // [R+2] range starts (slabs only)
   const int R = p.n_replicas, R1 = R + 1;
@@ -1384,7 +1726,8 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
     const uint32_t need = need_of(n_all, n_act);
     if (need <= SEG_TINY) continue;
     const bool list_in = !ordered || n_all - n_act <= LIST_MAX;
-    if (need <= SEG_MED) medium_replica<SLABS, FF>(p, a, c, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw, sh_g[0]);
+    if (SLABS && ordered && need <= SEG_MED) medium_ordered<FF>(p, a, c, r, begin[r], (int)n_all, (int)n_act, list_in, smem_raw, sh_g[0], s_cinfo_med, s_cls_ttft, s_cls_tpot);
+    else if (need <= SEG_MED) medium_replica<SLABS, FF>(p, a, c, r, begin[r], (int)n_all, (int)n_act, ordered, list_in, smem_raw, sh_g[0]);
     else oversize_replica<SLABS, FF>(p, a, c, r, begin[r], n_all, n_act, ordered, list_in, smem_raw, sh_g[0]);
   }
 
