@@ -90,8 +90,8 @@ class _ScaleParams(C.Structure):
                 ("eps_in_den", C.c_int32), ("eps_wait_num", C.c_int32), ("eps_wait_den", C.c_int32)]
 
 
-_DISPATCH_OUT = [("assign", np.int32, "n"), ("queue_order", np.int32, "n"), ("n_queue", np.int32, "1"),
-                 ("inst_order", np.int32, "R"), ("n_mature", np.int32, "1"), ("slack", np.int64, "n"),
+_DISPATCH_OUT = [("assign", np.int32, "n"), ("queue_order", np.int32, "n"), ("n_queue", np.int32, "2"),
+                 ("inst_order", np.int32, "R"), ("n_mature", np.int32, "2"), ("slack", np.int64, "n"),
                  ("budget", np.int64, "R"), ("e_d", np.int64, "R"), ("n_run", np.int32, "R"), ("sum_kv", np.int64, "R"),
                  ("adm_cost", np.int64, "R"), ("adm_count", np.int32, "R"), ("maturity_next", np.int64, "R")]
 
@@ -258,14 +258,16 @@ def sim(wl, iters: Optional[int] = None, j0: int = 0, j1: Optional[int] = None) 
 
 def dispatch(wl, now: int) -> Dict[str, np.ndarray]:
     """The dispatching steps over the shared global queue at time `now`: every instance of wl whose
-    maturity (wl.maturity) has come takes its turn once, in maturity order.  Nothing in wl changes."""
+    maturity (wl.maturity) has come takes its turn once, in maturity order; then the same steps for the
+    D-stage instances over the queue of prefilled requests.  n_queue and n_mature hold two numbers each
+    (the first stage's, the D stage's).  Nothing in wl changes."""
     L = lib()
     ctx = _Ctx(wl)
     n, R = wl.n_rows, wl.n_replicas
     out = {}
     so = _DispatchOut()
     for k, dt, dim in _DISPATCH_OUT:
-        out[k] = np.zeros({"n": max(n, 1), "R": R, "1": 1}[dim], dt)
+        out[k] = np.zeros({"n": max(n, 1), "R": R, "2": 2}[dim], dt)
         setattr(so, k, out[k].ctypes.data)
     mat = np.ascontiguousarray(wl.maturity, np.int64)
     st = L.ora_dispatch(C.byref(ctx.cfg), C.byref(ctx.table), int(now), mat.ctypes.data, C.byref(so))

@@ -712,15 +712,31 @@ uint32_t ora_scale(const ora_config *c, const ora_table *t, int64_t now, const i
  * The same four steps serve the P stage of the disaggregated mode ("P-stage
  * Dispatcher"): a PREFILL instance takes part with the budget and the maturity
  * update of its stage (no decode batch: E_d = 0, maturity = end of the prefill
- * batch).  DECODE instances are served by the Migrator from the queue of
- * prefilled requests (the per-replica step) and take no part here.
+ * batch).
+ * The D stage ("D-stage Migrator") runs the four steps once more in the same
+ * call, for the DECODE instances over the queue of prefilled requests:
+ * reading: a prefilled request is one in flight on a PREFILL instance whose
+ *   first token has been produced by `now` (the end of its prefill batch); what
+ *   the KV transfer adds is not modelled by this call.
+ * reading: that queue is ordered by (priority, slack, req_id) with slack =
+ *   first_token + (gen + 1) TPOT - now - E_d(1, prompt + gen): the time to the
+ *   request's next-token deadline, net of a decode iteration on its own.
+ * reading: step 2 as in the per-instance step of a DECODE replica: the budget
+ *   is a time, T - E_d(running batch), T the strictest TPOT in flight on the
+ *   instance, or, when it has none, of the queue of prefilled requests; a
+ *   request costs d1 + d2 (prompt + gen) of it.  Step 3 hands the queue out as
+ *   in the P stage (in order, stop at the first entry that does not fit, pass
+ *   over what exceeds every D budget of the call).  Step 4: a matured instance
+ *   with a batch gets maturity = now + E_d of the enlarged batch.
+ * The caller binds a dispatched prefilled request by replica_id := assign; it
+ * stays in flight, now on the D instance.
  * ========================================================================== */
 typedef struct {
   int32_t *assign;        /* [n] instance a queued row is dispatched to, else -1         */
   int32_t *queue_order;   /* [n] rows of the queue, most urgent first; -1 past n_queue   */
-  int32_t *n_queue;       /* [1]                                                         */
-  int32_t *inst_order;    /* [R] matured instances in dispatch order; -1 past n_mature   */
-  int32_t *n_mature;      /* [1]                                                         */
+  int32_t *n_queue;       /* [2] global queue; queue of prefilled requests (listed behind it in queue_order) */
+  int32_t *inst_order;    /* [R] matured instances in dispatch order, colocated / P stage first, then D stage; -1 behind */
+  int32_t *n_mature;      /* [2] colocated and P-stage instances; D-stage instances      */
   int64_t *slack;         /* [n] slack of queue rows, 0 elsewhere                        */
   int64_t *budget;        /* [R] safe token budget (0 for an instance not matured)       */
   int64_t *e_d;           /* [R] */
@@ -786,7 +802,7 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
   }
   qsort(q, (size_t)nq, sizeof(sort_tuple), cmp_tuple);
   for (int64_t j = 0; j < nq; j++) o->queue_order[j] = (int32_t)q[j].row;
-  *o->n_queue = (int32_t)nq;
+  o->n_queue[0] = (int32_t)nq;
 
   /* step 2 for every instance that has matured; step 1: their order */
   int32_t nm = 0;
@@ -818,7 +834,7 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
   }
   qsort(inst, (size_t)nm, sizeof(inst_tuple), cmp_inst);
   for (int32_t k = 0; k < nm; k++) o->inst_order[k] = inst[k].id;
-  *o->n_mature = nm;
+  o->n_mature[0] = nm;
 
   /* steps 3 and 4, instance by instance */
   int64_t budget_max = 0;
@@ -850,6 +866,77 @@ uint32_t ora_dispatch(const ora_config *c, const ora_table *t, int64_t now, cons
       o->maturity_next[r] = v > ORA_TIME_MAX ? ORA_TIME_MAX : (int64_t)v;
     }
   }
+
+  /* ---- the D stage: the same four steps, by the Migrator (Sec. 3.3.1, "D-stage Migrator") ---- */
+  /* the queue of prefilled requests, priority-ordered */
+  sort_tuple *dq = (sort_tuple *)malloc(sizeof(sort_tuple) * (size_t)(n + 1));
+  int64_t ndq = 0, min_tpot_dq = ORA_INF;
+  for (int64_t i = 0; i < n; i++) {
+    uint32_t again = 0;
+    if (!row_valid(c, t, i, &again) || t->state[i] != ST_RUNNING) continue;
+    const int32_t r = t->replica_id[i];
+    if (r < 0 || r >= R || c->replicas[r].mode != MODE_PREFILL || t->first_token[i] > now) continue;
+    const ora_class *k = &c->classes[t->class_id[i]];
+    const int64_t kv_i = (int64_t)t->prompt_len[i] + t->gen[i];
+    const int64_t sl = k->tpot > 0 ? t->first_token[i] + ((int64_t)t->gen[i] + 1) * k->tpot - now - ora_Ed(M, 1, kv_i) : ORA_SLACK_MAX;
+    int32_t prio;
+    if (c->weight_max > 0) {
+      int64_t pw = (int64_t)c->weight_max - t->weight[i];
+      prio = (int32_t)(pw < 0 ? 0 : (pw > 62 ? 62 : pw));
+    } else prio = k->prio;
+    o->slack[i] = sl;
+    dq[ndq].phase = PH_QUEUED; dq[ndq].prio = prio; dq[ndq].cslack = clamp_slack(sl);
+    dq[ndq].req_id = t->req_id[i]; dq[ndq].row = i;
+    ndq++;
+    if (k->tpot > 0 && k->tpot < min_tpot_dq) min_tpot_dq = k->tpot;
+  }
+  qsort(dq, (size_t)ndq, sizeof(sort_tuple), cmp_tuple);
+  for (int64_t j = 0; j < ndq; j++) o->queue_order[nq + j] = (int32_t)dq[j].row;
+  o->n_queue[1] = (int32_t)ndq;
+
+  /* step 1: the D-stage instances that have matured, earliest first; step 2: their budget, a time */
+  int32_t nmd = 0;
+  int64_t dbudget_max = 0;
+  for (int32_t r = 0; r < R; r++) {
+    if (c->replicas[r].mode != MODE_DECODE || maturity[r] > now) continue;
+    const int64_t T = (n_run[r] > 0 && min_tpot[r] < ORA_INF) ? min_tpot[r] : min_tpot_dq;
+    int64_t budget;
+    if (c->budget_mode == BUDGET_CAP_ONLY || T == ORA_INF) budget = ORA_INF;
+    else {
+      const int64_t room = T - ora_Ed(M, n_run[r], sum_kv[r]);
+      budget = room > 0 ? room : 0;
+    }
+    o->budget[r] = budget;
+    if (budget > dbudget_max) dbudget_max = budget;
+    inst[nmd].mat = maturity[r]; inst[nmd].id = r; nmd++;
+  }
+  qsort(inst, (size_t)nmd, sizeof(inst_tuple), cmp_inst);
+  for (int32_t k = 0; k < nmd; k++) o->inst_order[nm + k] = inst[k].id;
+  o->n_mature[1] = nmd;
+
+  /* steps 3 and 4, instance by instance */
+  cursor = 0;
+  for (int32_t k = 0; k < nmd; k++) {
+    const int32_t r = inst[k].id;
+    const ora_replica *cfg = &c->replicas[r];
+    int64_t cost = 0, count = 0, adm_kv = 0;
+    while (cursor < ndq) {
+      const int64_t i = dq[cursor].row;
+      const int64_t kv_i = (int64_t)t->prompt_len[i] + t->gen[i];
+      const int64_t c_i = M->d1 + M->d2 * kv_i;
+      if (c_i > dbudget_max) { cursor++; continue; }          /* fits no instance in this call */
+      if (c_i > o->budget[r] - cost) break;
+      if (cfg->batch_cap != 0 && n_run[r] + count + 1 > cfg->batch_cap) break;
+      cost += c_i; count += 1; adm_kv += kv_i;
+      o->assign[i] = r;
+      cursor++;
+    }
+    o->adm_cost[r] = cost;
+    o->adm_count[r] = (int32_t)count;
+    /* maturity = end of the next decoding iteration of the enlarged batch */
+    if (n_run[r] + count > 0) o->maturity_next[r] = now + ora_Ed(M, n_run[r] + count, sum_kv[r] + adm_kv);
+  }
+  free(dq);
   free(n_run); free(sum_kv); free(min_tpot); free(q); free(inst);
   return status;
 }

@@ -532,16 +532,80 @@ def test_attainment_agrees_with_the_simulator():
 def test_dispatch_serves_the_p_stage():
     # the hand-worked case with instance 0 as a P-stage instance: its 80 resident requests do not decode there, so
     # it has the budget of an empty instance (2144), no E_d, and matures when its prefill batch ends:
-    # E_p(297) = 17056418.  A D-stage instance takes no part.
+    # E_p(297) = 17056418.
     wl, now = _dispatch_hand_case()
     wl.replicas[0, 0] = gen.PREFILL
     wl.replicas[2, 0] = gen.DECODE
     wl.maturity[2] = now - 100
     o = oracle.dispatch(wl, now)
-    assert list(o["inst_order"]) == [1, 0, -1] and o["n_mature"][0] == 2
-    assert list(o["budget"]) == [2144, 2144, 0] and list(o["e_d"]) == [0, 0, 0] and list(o["n_run"]) == [80, 0, 0]
-    assert list(o["assign"][80:86]) == [1, 1, 0, 0, -1, -1] and list(o["adm_cost"]) == [297, 2144, 0]
-    assert o["maturity_next"][0] - now == 17_056_418 and o["maturity_next"][2] == now - 100
+    assert list(o["inst_order"]) == [1, 0, 2] and list(o["n_mature"]) == [2, 1]
+    assert list(o["budget"][:2]) == [2144, 2144] and list(o["e_d"]) == [0, 0, 0] and list(o["n_run"]) == [80, 0, 0]
+    assert list(o["assign"][80:86]) == [1, 1, 0, 0, -1, -1] and list(o["adm_cost"][:2]) == [297, 2144]
+    assert o["maturity_next"][0] - now == 17_056_418
+    # The D stage in the same call (Sec. 3.3.1, "D-stage Migrator"): the 80 residents got their first token 30 ms ago
+    # and are the queue of prefilled requests; TPOT 30 ms, 800 tokens of context each.  Slack = (now - 30 ms) + 30 ms
+    # - now - E_d(1, 800) = -(8000000 + 100000 + 16000); all equal, so they queue by request id behind the 5
+    # entries of the global queue.  The idle D instance 2 takes the strictest TPOT of that queue: budget = 30 ms -
+    # E_d(0, 0) = 22000000 ns; a request costs d1 + d2 * 800 = 116000 ns, all 80 fit (9280000); its maturity is
+    # the end of the first decode iteration of the 80: E_d(80, 64000).
+    assert list(o["n_queue"]) == [5, 80] and list(o["queue_order"][5:85]) == list(range(80)) and o["queue_order"][85] == -1
+    assert np.all(o["slack"][:80] == -8_116_000)
+    assert o["budget"][2] == 22_000_000 and o["adm_cost"][2] == 80 * 116_000 and o["adm_count"][2] == 80
+    assert np.all(o["assign"][:80] == 2)
+    assert o["maturity_next"][2] - now == PINS["Ed_80_64000"] == 17_280_000
+
+
+def _migrator_hand_case():
+    # model with a decode iteration of 8 ms + 2 ms per request + 2 us per token of context
+    now = 1000 * MS
+    model = (5_000_000, 40_000, 2, 8_000_000, 2_000_000, 2_000)
+    classes = [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)]
+    rows = [dict(state=1, replica_id=2, class_id=1, prompt_len=1000, gen=10, output_len=500, first_token_ns=now - 600 * MS),   # in flight on D instance 2
+            dict(state=1, replica_id=2, class_id=1, prompt_len=1000, gen=10, output_len=500, first_token_ns=now - 600 * MS),
+            dict(state=1, replica_id=0, class_id=1, prompt_len=7000, gen=0, output_len=50, first_token_ns=now - 20 * MS),      # A  row 2
+            dict(state=1, replica_id=0, class_id=0, prompt_len=500, gen=0, output_len=50, first_token_ns=now - 25 * MS),       # B  row 3
+            dict(state=1, replica_id=0, class_id=0, prompt_len=4000, gen=0, output_len=50, first_token_ns=now - 1 * MS),       # C  row 4
+            dict(state=1, replica_id=0, class_id=0, prompt_len=100, gen=0, output_len=50, first_token_ns=now + 1)]             # its prefill batch has not ended
+    wl = make_wl(rows, classes, replicas=[(gen.PREFILL, 8192, 0), (gen.DECODE, 8192, 0), (gen.DECODE, 8192, 3)],
+                 now=[now] * 3, maturity=[now + 1, now - 5 * MS, now - 10 * MS], model=model)
+    return wl, now
+
+
+def test_migrator_selects_the_d_instance_hand_worked():
+    # Sec. 3.3.1, "Disaggregated Mode": the four steps once more for the D stage.  E_d(n, kv) = 8 ms + 2 ms n + 2 us kv.
+    # Queue of prefilled requests (first token produced): slack = first_token + TPOT - now - E_d(1, kv)
+    #   A (class 1, 50 ms, 7000 tokens)  30 ms - 24 ms =  6 ms   cost 2 ms + 14 ms = 16 ms
+    #   B (class 0, 30 ms,  500 tokens)   5 ms - 11 ms = -6 ms   cost 2 ms +  1 ms =  3 ms
+    #   C (class 0, 30 ms, 4000 tokens)  29 ms - 18 ms = 11 ms   cost 2 ms +  8 ms = 10 ms
+    # order: priority 0 first (B, C), then A.  Instance 2 matured first (10 ms ago): two requests in flight with
+    # 2020 tokens, E_d = 8 + 4 + 4.04 = 16.04 ms, strictest TPOT in flight 50 ms: budget 33.96 ms; its batch cap of 3
+    # leaves room for one request: it takes B and stops at C.  Instance 1 is idle: strictest TPOT of the queue as
+    # the call began (30 ms) minus E_d(0, 0) = 22 ms; it takes C (10 ms), A (16 ms more) does not fit and waits.
+    wl, now = _migrator_hand_case()
+    o = oracle.dispatch(wl, now)
+    assert o["status"] == 0
+    assert list(o["n_queue"]) == [0, 3] and list(o["queue_order"][:4]) == [3, 4, 2, -1]
+    assert o["slack"][2] == PINS["mig_slack_A"] and o["slack"][3] == PINS["mig_slack_B"] and o["slack"][4] == PINS["mig_slack_C"]
+    assert o["slack"][5] == 0 and o["slack"][0] == 0
+    assert list(o["n_mature"]) == [0, 2] and list(o["inst_order"]) == [2, 1, -1]
+    assert list(o["n_run"]) == [4, 0, 2] and list(o["e_d"]) == [0, 0, PINS["mig_ed_inst2"]]
+    assert list(o["budget"]) == [0, PINS["mig_budget_inst1"], PINS["mig_budget_inst2"]]
+    assert list(o["assign"]) == [-1, -1, -1, 2, 1, -1]
+    assert list(o["adm_cost"]) == [0, PINS["mig_cost_C"], PINS["mig_cost_B"]] and list(o["adm_count"]) == [0, 1, 1]
+    assert o["maturity_next"][2] - now == PINS["mig_mat_inst2"] and o["maturity_next"][1] - now == PINS["mig_mat_inst1"]
+    assert o["maturity_next"][0] == now + 1
+    # a D instance before its maturity takes no part; the other then takes its share: room for B only stands, so
+    # with instance 2 protected instance 1 takes B and C (13 ms) and A (29 ms) still does not fit
+    wl.maturity[2] = now + 1
+    o = oracle.dispatch(wl, now)
+    assert list(o["n_mature"]) == [0, 1] and list(o["inst_order"]) == [1, -1, -1] and o["budget"][2] == 0
+    assert list(o["assign"]) == [-1, -1, -1, 1, 1, -1] and o["adm_cost"][1] == 13_000_000
+    assert o["maturity_next"][1] - now == 8_000_000 + 2 * 2_000_000 + 2_000 * 4500 and o["maturity_next"][2] == now + 1
+    # binding: a dispatched prefilled request stays in flight, now on its D instance
+    wl.maturity[2] = now - 10 * MS
+    o = oracle.dispatch(wl, now)
+    oracle.dispatch_bind(wl, now, o)
+    assert list(wl.table["replica_id"]) == [2, 2, 0, 2, 1, 0] and list(wl.table["state"]) == [1] * 6
 
 
 def test_scale_apply_hand_worked():

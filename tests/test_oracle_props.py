@@ -438,3 +438,124 @@ def test_scaling_loop_invariants():
     # every instance's clock stays within one iteration of the global clock once it has work
     busy = np.isin(np.arange(R), wl.table["replica_id"][wl.table["state"] == gen.RUNNING])
     assert np.all(wl.now[busy] <= o["now"] + 1100 * MS)      # one iteration: a prefill batch up to the token cap, then a decode iteration
+
+
+# ---- the D stage of the dispatching call (the Migrator) ----------------------------------------------
+def _migrator_case(seed, **kw):
+    modes = (gen.PREFILL, gen.DECODE, gen.DECODE, gen.COLOCATED, gen.DECODE)[: 2 + seed % 4]
+    wl = gen.random_table(200 + seed, 80 + 41 * seed, len(modes), modes=modes, inflight=0.7, **kw)
+    wl.replicas[:, 0] = modes          # (the generator draws the modes; here every instance has the one listed)
+    now = int(wl.now.max())
+    t = wl.table
+    run_on_p = (t["state"] == gen.RUNNING) & (wl.replicas[np.clip(t["replica_id"], 0, wl.n_replicas - 1), 0] == gen.PREFILL)
+    # prefill batches that ended up to 40 ms ago, a few that have not ended yet
+    rng = np.random.default_rng(seed)
+    t["first_token_ns"][run_on_p] = now - rng.integers(-3 * MS, 40 * MS, int(run_on_p.sum()))
+    wl.maturity[:] = now - rng.integers(-2 * MS, 20 * MS, wl.n_replicas)
+    return wl, now
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_migrator_invariants(seed):
+    wl, now = _migrator_case(seed, batch_cap=(0, 6)[seed % 3 == 1], tie_heavy=seed % 4 == 2,
+                             budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 3])
+    o = oracle.dispatch(wl, now)
+    t, R, M = wl.table, wl.n_replicas, wl.model
+    nq, ndq = int(o["n_queue"][0]), int(o["n_queue"][1])
+    nm, nmd = int(o["n_mature"][0]), int(o["n_mature"][1])
+    mode = wl.replicas[:, 0]
+    ok = (t["class_id"] < len(wl.classes)) & (t["replica_id"] >= 0) & (t["replica_id"] < R)
+    on_p = ok & (mode[np.clip(t["replica_id"], 0, R - 1)] == gen.PREFILL)
+    pre = (t["state"] == gen.RUNNING) & on_p & (t["first_token_ns"] <= now)
+    dqueue = o["queue_order"][nq:nq + ndq]
+    assert sorted(dqueue.tolist()) == np.nonzero(pre)[0].tolist() and np.all(o["queue_order"][nq + ndq:] == -1)
+    # its order: (priority, clamped slack, request id), the slack being the time to the next-token deadline net
+    # of a decode iteration of the request alone
+    kv = t["prompt_len"].astype(np.int64) + t["gen"]
+    keys = []
+    for i in dqueue:
+        ttft, tpot, prio = wl.classes[t["class_id"][i]]
+        sl = int(t["first_token_ns"][i]) + (int(t["gen"][i]) + 1) * tpot - now - oracle.Ed(M, 1, int(kv[i])) if tpot > 0 else oracle.SLACK_MAX
+        assert o["slack"][i] == sl
+        keys.append((prio, min(max(sl, oracle.SLACK_MIN), oracle.SLACK_MAX), int(t["req_id"][i])))
+    assert keys == sorted(keys)
+    # D instances take their turn in maturity order behind the instances of the first stage
+    dmat = np.nonzero((mode == gen.DECODE) & (wl.maturity <= now))[0]
+    dorder = o["inst_order"][nm:nm + nmd]
+    assert sorted(dorder.tolist()) == dmat.tolist() and np.all(np.diff(wl.maturity[dorder]) >= 0)
+    assert np.all(o["inst_order"][nm + nmd:] == -1)
+    # budgets: a time, from the strictest TPOT in flight or, for an idle instance, of the queue of prefilled requests
+    tpot_of = np.array([c[1] for c in wl.classes], np.int64)
+    qt = tpot_of[t["class_id"][dqueue]]
+    tq = int(qt[qt > 0].min()) if np.any(qt > 0) else oracle.INF
+    for r in dorder:
+        mine = ok & (t["state"] == gen.RUNNING) & (t["replica_id"] == r)
+        rt = tpot_of[t["class_id"][mine]]
+        T = int(rt[rt > 0].min()) if np.any(rt > 0) else tq
+        if wl.budget_mode == gen.BUDGET_CAP_ONLY or T == oracle.INF:
+            assert o["budget"][r] == oracle.INF
+        else:
+            assert o["budget"][r] == max(T - oracle.Ed(M, int(mine.sum()), int(kv[mine].sum())), 0)
+    # consecutive runs of the entries that fit some D instance; within budget and batch room; maximal
+    cost_of = M[4] + M[5] * kv
+    bmax = int(o["budget"][dorder].max()) if nmd else 0
+    fits = cost_of[dqueue] <= bmax
+    assert np.all(o["assign"][dqueue[~fits]] == -1)
+    queue = dqueue[fits]
+    cursor = 0
+    for r in dorder:
+        cnt, cost = int(o["adm_count"][r]), int(o["adm_cost"][r])
+        rows = queue[cursor:cursor + cnt]
+        assert np.all(o["assign"][rows] == r) and int(cost_of[rows].sum()) == cost and cost <= o["budget"][r]
+        cap = int(wl.replicas[r, 2])
+        assert cap == 0 or cnt == 0 or o["n_run"][r] + cnt <= cap
+        cursor += cnt
+        if cursor < queue.size:
+            assert cost + int(cost_of[queue[cursor]]) > o["budget"][r] or (cap != 0 and o["n_run"][r] + cnt + 1 > cap)
+        if o["n_run"][r] + cnt > 0:
+            assert o["maturity_next"][r] == now + oracle.Ed(M, int(o["n_run"][r]) + cnt, int(o["sum_kv"][r]) + int(kv[rows].sum()))
+        else:
+            assert o["maturity_next"][r] == wl.maturity[r]
+    assert np.all(o["assign"][queue[cursor:]] == -1)
+    for r in np.nonzero((mode == gen.DECODE) & (wl.maturity > now))[0]:
+        assert o["budget"][r] == 0 and o["adm_count"][r] == 0 and o["maturity_next"][r] == wl.maturity[r]
+    assert np.count_nonzero(o["assign"] >= 0) == int(o["adm_count"].sum())
+
+
+def test_migrator_single_instance_equals_the_per_replica_decode_step():
+    # One matured D instance and prefilled requests that each fit alone: handing them to that instance's own queue
+    # (what the partner-table hand-off does) and running the per-replica step must admit the same requests with
+    # the same budget, cost and maturity -- the two slacks differ by a constant, the order does not.
+    for seed in range(6):
+        wl = gen.random_table(300 + seed, 200, 2, modes=(gen.PREFILL, gen.DECODE), inflight=0.8, done=0.0, future=0.0, batch_cap=(0, 25)[seed % 2])
+        wl.replicas[:, 0] = (gen.PREFILL, gen.DECODE)
+        if seed in (0, 4):
+            wl.model = wl.model[:4] + (400_000, 200)                    # dearer decode steps: the budget ends the run
+        now = int(wl.now.max())
+        wl.now[:] = now
+        wl.maturity[:] = [now + 1, now - 1]
+        t = wl.table
+        on_p = t["replica_id"] == 0
+        t["state"][on_p] = gen.RUNNING
+        t["first_token_ns"][on_p] = now - 5 * MS
+        t["gen"][on_p] = 0
+        t["state"][(t["replica_id"] == 1) & (t["state"] == gen.QUEUED)] = gen.DONE      # the D instance has no queue of its own
+        if seed >= 4:
+            t["state"][t["replica_id"] == 1] = gen.DONE                 # an idle D instance: the queue's strictest TPOT
+        d = oracle.dispatch(wl, now)
+        assert d["n_queue"][1] == int(on_p.sum()) and d["n_mature"][1] == 1
+        w2 = wl.copy()
+        w2.table["replica_id"][on_p] = 1
+        w2.table["state"][on_p] = gen.QUEUED
+        s = oracle.step(w2)
+        assert d["budget"][1] == s["budget"][1] and d["e_d"][1] == s["e_d"][1]
+        cost_of = wl.model[4] + wl.model[5] * (t["prompt_len"].astype(np.int64) + t["gen"])
+        if np.all(cost_of[on_p] <= d["budget"][1]):                     # nothing is skipped by either
+            nq = int(d["n_queue"][0])
+            order_d = d["queue_order"][nq:nq + int(on_p.sum())]
+            order_s = [i for i in s["order"] if on_p[i]]
+            assert order_d.tolist() == order_s
+            assert np.array_equal(np.nonzero(d["assign"] == 1)[0], np.nonzero(s["admit"].astype(bool) & on_p)[0])
+            assert d["adm_cost"][1] == s["adm_cost"][1] and d["adm_count"][1] == s["adm_count"][1]
+            assert d["maturity_next"][1] == s["maturity_next"][1]
+            assert seed not in (0, 4) or 0 < d["adm_count"][1] < d["n_queue"][1]

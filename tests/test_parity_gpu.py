@@ -1021,3 +1021,23 @@ def test_medium_segment_sizes_around_the_register_sort_shapes(n):
     assert_step_parity(wl, steps=2, commit=True)
     wl = gen.random_table(n + 2, n, 1, modes=(gen.COLOCATED,), permute_ids=True, inflight=0.05, done=0.45, future=0.45)     # mostly inactive
     assert_step_parity(wl, steps=1, commit=True)
+
+
+@pytest.mark.parametrize("n", [3000, 16384])
+def test_medium_replica_with_crowded_and_outlying_slacks(n):
+    # The distribution sort of a larger replica spreads a class over its bins by slack: queued requests that arrived
+    # within nanoseconds of each other crowd one bin (the sorting network takes over), a few far outliers stretch the
+    # range, and arrivals outside the sampled range go to the end bins.  Ids in row order: an ordered step.
+    wl = gen.random_table(900 + n % 7, n, 1, modes=(gen.COLOCATED,), permute_ids=False, inflight=0.3, done=0.0, future=0.0)
+    t = wl.table
+    q = np.nonzero(t["state"] == gen.QUEUED)[0]
+    now = int(wl.now[0])
+    t["arrival_ns"][q] = now - 10**9 - (np.arange(len(q)) % 1500)            # crowded: 1500 distinct slacks a nanosecond apart
+    t["arrival_ns"][q[::97]] = now - 10**9 * (2 + np.arange(len(q[::97])) % 300)   # outliers up to 300 s back
+    t["arrival_ns"][q[5]] = now - 500 * 10**9
+    assert_step_parity(wl, steps=2, commit=True)
+    wl = gen.random_table(901 + n % 7, n, 1, modes=(gen.DECODE,), permute_ids=False, inflight=0.7, done=0.0, future=0.0)
+    t = wl.table
+    r = np.nonzero(t["state"] == gen.RUNNING)[0]
+    t["last_token_ns"][r] = int(wl.now[0]) - (np.arange(len(r)) % 7)         # requests in flight with seven distinct slacks per class
+    assert_step_parity(wl, steps=2, commit=True)
