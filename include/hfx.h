@@ -246,17 +246,18 @@ int hfx_sched_step(hfx_sched *s, const hfx_table *table,
 /* Outputs of hfx_dispatch_step; every member is a device pointer.  n = rows of
  * the table, R = replicas of the scheduler. */
 typedef struct hfx_dispatch_out {
-  int32_t *assign;         /* [n] instance a queued row is dispatched to, else -1 */
-  int32_t *queue_order;    /* [n] rows of the queue, most urgent first; -1 past n_queue */
-  int32_t *n_queue;        /* [1] */
-  int32_t *inst_order;     /* [R] matured instances in dispatch order; -1 past n_mature */
-  int32_t *n_mature;       /* [1] */
-  int64_t *slack_ns;       /* [n] slack of queue rows, 0 elsewhere */
-  int64_t *budget;         /* [R] safe token budget; 0 for an instance not matured */
+  int32_t *assign;         /* [n] instance a queued row (or, D stage, a prefilled request) is dispatched to, else -1 */
+  int32_t *queue_order;    /* [n] rows of the global queue, most urgent first, then the rows of the queue of
+                              prefilled requests; -1 behind them */
+  int32_t *n_queue;        /* [2] length of the global queue; of the queue of prefilled requests */
+  int32_t *inst_order;     /* [R] matured instances in dispatch order: colocated and P stage, then D stage; -1 behind */
+  int32_t *n_mature;       /* [2] matured colocated and P-stage instances; matured D-stage instances */
+  int64_t *slack_ns;       /* [n] slack of the rows of either queue, 0 elsewhere */
+  int64_t *budget;         /* [R] safe budget: tokens (colocated, P stage), ns (D stage); 0 for an instance not matured */
   int64_t *e_d_ns;         /* [R] */
   int32_t *n_run;          /* [R] */
   int64_t *sum_kv;         /* [R] */
-  int64_t *adm_cost;       /* [R] tokens dispatched to the instance */
+  int64_t *adm_cost;       /* [R] what was dispatched to the instance, in the unit of its budget */
   int32_t *adm_count;      /* [R] requests dispatched to the instance */
   int64_t *maturity_next;  /* [R] */
 } hfx_dispatch_out;
@@ -282,8 +283,23 @@ typedef struct hfx_dispatch_out {
  * (replica_id := assign) before the next hfx_sched_step.
  * HFX_PREFILL replicas take part the same way with the budget and maturity
  * update of their stage (the "P-stage Dispatcher": no decode batch, maturity =
- * end of the prefill batch); HFX_DECODE replicas are served from their own
- * queue of prefilled requests by hfx_sched_step and take no part (budget 0).
+ * end of the prefill batch).
+ * On a scheduler with HFX_DECODE replicas the same call then runs the four
+ * steps for the D stage (Sec. 3.3.1, "D-stage Migrator"): (1) the DECODE
+ * instances whose maturity has come, earliest first; (2) each gets a budget in
+ * time, T - E_d(its running batch), T the strictest TPOT among its in-flight
+ * requests or, when it has none, in the queue of prefilled requests as the
+ * call begins (unbounded when no TPOT applies or in HFX_BUDGET_CAP_ONLY mode);
+ * (3) the queue of prefilled requests -- every RUNNING row on an HFX_PREFILL
+ * replica whose first_token_ns has come (the end of its prefill batch; a KV
+ * transfer time is not modelled here), ordered by (priority, slack, req_id)
+ * with slack = first_token + (gen + 1) TPOT - now - E_d(1, prompt_len + gen)
+ * -- is handed out as above, an entry costing d1 + d2 (prompt_len + gen) of
+ * the budget; (4) a matured instance that then has a batch gets maturity =
+ * now + E_d of the enlarged batch.  A dispatched prefilled request stays
+ * RUNNING; binding it (replica_id := assign) puts it in flight on the D
+ * instance.  DECODE replicas also keep their own queue (QUEUED rows bound to
+ * them, e.g. by hfx_pd_migrate), which hfx_sched_step serves.
  * The scheduler may have at most 4096 replicas.  The first call allocates the call's workspace (44 bytes
  * per row of max_rows) with cudaMalloc, so it should not be made inside a
  * stream capture; hfx_sched_destroy frees it.

@@ -100,8 +100,8 @@ class _SimOut(C.Structure):
     _fields_ = [(k, C.c_void_p) for k, _ in SIM_OUT_FIELDS]
 
 
-DISPATCH_OUT_FIELDS = [("assign", torch.int32, "n"), ("queue_order", torch.int32, "n"), ("n_queue", torch.int32, "1"),
-                       ("inst_order", torch.int32, "R"), ("n_mature", torch.int32, "1"), ("slack_ns", torch.int64, "n"),
+DISPATCH_OUT_FIELDS = [("assign", torch.int32, "n"), ("queue_order", torch.int32, "n"), ("n_queue", torch.int32, "2"),
+                       ("inst_order", torch.int32, "R"), ("n_mature", torch.int32, "2"), ("slack_ns", torch.int64, "n"),
                        ("budget", torch.int64, "R"), ("e_d_ns", torch.int64, "R"), ("n_run", torch.int32, "R"),
                        ("sum_kv", torch.int64, "R"), ("adm_cost", torch.int64, "R"), ("adm_count", torch.int32, "R"),
                        ("maturity_next", torch.int64, "R")]
@@ -291,7 +291,7 @@ class DispatchOut:
     """Output buffers of hfx_dispatch_step (allocated once, reused)."""
 
     def __init__(self, n_rows: int, n_replicas: int, device="cuda"):
-        self.t = {k: torch.zeros({"n": max(n_rows, 1), "R": n_replicas, "1": 4}[dim], dtype=dt, device=device)
+        self.t = {k: torch.zeros({"n": max(n_rows, 1), "R": n_replicas, "2": 4}[dim], dtype=dt, device=device)
                   for k, dt, dim in DISPATCH_OUT_FIELDS}
         self.n_rows = n_rows
 
@@ -305,7 +305,7 @@ class DispatchOut:
         out = {}
         for k, _, dim in DISPATCH_OUT_FIELDS:
             a = self.t[k].cpu().numpy()
-            out[k] = a[:self.n_rows] if dim == "n" else (a[:1] if dim == "1" else a)
+            out[k] = a[:self.n_rows] if dim == "n" else (a[:2] if dim == "2" else a)
         return out
 
 

@@ -218,9 +218,14 @@ extern "C" int hfx_dispatch_step(hfx_sched *s, const hfx_table *t, int64_t now_n
                        o->e_d_ns, o->n_run, o->sum_kv, o->adm_cost, o->adm_count, o->maturity_next};
   for (const void *p : all) if (misaligned(p)) return HFX_E_ALIGN;
   int32_t cap_max = 0;
-  for (int r = 0; r < s->p.n_replicas; r++)
+  bool d_stage = false;      // the scheduler has D-stage instances: the Migrator's stage runs too
+  for (int r = 0; r < s->p.n_replicas; r++) {
     if (h->h_cfg[r].mode != HFX_DECODE && h->h_cfg[r].token_cap > cap_max) cap_max = h->h_cfg[r].token_cap;
-  return hfx_launch_dispatch(s, t, now_ns, maturity_ns, o, cap_max);
+    d_stage = d_stage || h->h_cfg[r].mode == HFX_DECODE;
+  }
+  if (d_stage && t->n_rows > 0 && !t->first_token_ns) return HFX_E_ARG;
+  if (misaligned(t->first_token_ns)) return HFX_E_ALIGN;
+  return hfx_launch_dispatch(s, t, now_ns, maturity_ns, o, cap_max, d_stage);
 }
 
 extern "C" int hfx_pd_migrate(hfx_sched *s, const hfx_table *t, int32_t *replica_id, const hfx_replica_state *st,

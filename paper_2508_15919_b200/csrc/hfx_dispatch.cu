@@ -1,5 +1,8 @@
 // hfx_dispatch_step: the four dispatching steps of Sec. 3.3.1 over a shared global queue, for every
-// colocated or P-stage instance whose maturity time has come, in maturity order.
+// colocated or P-stage instance whose maturity time has come, in maturity order; then, on a scheduler with
+// D-stage instances, the same steps once more for the D stage (the Migrator): the queue of prefilled
+// requests, the D instances in maturity order, budgets and costs in time.  One scan of the table finds both
+// queues; the kernels from the compaction on run once per stage (stage 0, then stage 1 on the same buffers).
 //
 //   k_disp_scan     one streaming pass over the table: the running batch of every instance (count,
 //                   context tokens, classes), slack and priority key of the visible queue's rows
@@ -35,9 +38,10 @@ struct DispWork {
   uint32_t *n_run;           // [R]
   unsigned long long *sum_kv;    // [R]
   unsigned long long *mask_run;  // [R]
-  unsigned long long *ctl;   // [0] classes present in the queue  [1] queue length  [2], [3] last-block counters
-                             // [4] largest budget among the matured instances  [5] request ids do not rise with the rows
-  uint32_t *blk_cnt;         // [DISP_SCAN_BLOCKS_MAX] queue rows found by each block of the scan
+  unsigned long long *ctl;   // per stage, 8 words each: [0] classes present in the queue  [1] queue length  [2], [3] last-block
+                             // counters  [4] largest budget among the matured instances;  [5] (first stage's only) request
+                             // ids do not rise with the rows
+  uint32_t *blk_cnt;         // [2][DISP_SCAN_BLOCKS_MAX] queue rows of each stage found by each block of the scan
   ReplicaPlan *plan;         // [R]
   int32_t *run_start;        // [R] where an instance's run starts in the queue
   int32_t *run_len;          // [R] queue positions the run covers (passed-over entries included)
@@ -46,13 +50,26 @@ struct DispWork {
 
 struct DispArgs {
   const int32_t *replica_id; const uint8_t *class_id; const uint8_t *state; const int32_t *prompt_len; const int32_t *gen;
-  const int64_t *arrival; const int32_t *req_id; const int32_t *weight;
+  const int64_t *arrival; const int32_t *req_id; const int32_t *weight; const int64_t *first_token;
   int64_t n; int64_t now; int32_t cap_max;
-  const int64_t *maturity; const hfx_replica_cfg *cfg;
+  int32_t d_stage;           // the scheduler has D-stage instances: the Migrator's stage runs too
+  const int64_t *maturity; const hfx_replica_cfg *cfg; const uint8_t *mode;
   // outputs
   int32_t *assign; int32_t *queue_order; int32_t *n_queue; int32_t *inst_order; int32_t *n_mature; int64_t *slack;
   int64_t *budget; int64_t *e_d; int32_t *n_run; int64_t *sum_kv; int64_t *adm_cost; int32_t *adm_count; int64_t *maturity_next;
   uint32_t *status;
+};
+
+#define DQ_TAG (UINT64_C(1) << 63)      // on a row's key: the row belongs to the queue of prefilled requests
+#define KEY48 ((UINT64_C(1) << 48) - 1)
+
+// what a queue entry takes of an instance's budget: prompt tokens (first stage), decode time d1 + d2 kv (D stage)
+struct DispCost {
+  const int32_t *prompt_len, *gen; int64_t d1, d2; int32_t stage;
+  __device__ __forceinline__ int64_t of(uint32_t row) const {
+    const int64_t x = prompt_len[row];
+    return stage ? d1 + d2 * (x + gen[row]) : x;
+  }
 };
 
 // rows per block of the scan / compaction pair: equal contiguous runs, whole warps
@@ -65,23 +82,24 @@ __host__ __device__ inline int64_t disp_chunk(int64_t n, int blocks) {
 // k_disp_scan
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, const DispArgs a, const DispWork w) {
-  __shared__ int64_t s_ttft[HFX_MAX_CLASSES];
+  __shared__ int64_t s_ttft[HFX_MAX_CLASSES], s_tpot[HFX_MAX_CLASSES];
   __shared__ uint8_t s_prio[HFX_MAX_CLASSES];
   for (int c = threadIdx.x; c < HFX_MAX_CLASSES; c += blockDim.x) {
     s_ttft[c] = c < p.n_classes ? p.ttft[c] : 0;
+    s_tpot[c] = c < p.n_classes ? p.tpot[c] : 0;
     s_prio[c] = c < p.n_classes ? p.prio[c] : 63;
   }
   __syncthreads();
   const int lane = threadIdx.x & 31;
   uint32_t bad = 0;
-  unsigned long long qmask = 0;
-  __shared__ uint32_t s_count;
-  if (threadIdx.x == 0) s_count = 0;
+  unsigned long long qmask = 0, dmask = 0;
+  __shared__ uint32_t s_count, s_dcount;
+  if (threadIdx.x == 0) { s_count = 0; s_dcount = 0; }
   __syncthreads();
   // every block takes a contiguous run of rows, so that the compaction that follows keeps row order
   const int64_t chunk = disp_chunk(a.n, gridDim.x);
   const int64_t lo = (int64_t)blockIdx.x * chunk, hi = lo + chunk < a.n ? lo + chunk : a.n;
-  uint32_t mine = 0;
+  uint32_t mine = 0, dmine = 0;
   bool falls = false;
   for (int64_t i = lo + threadIdx.x; i < hi; i += blockDim.x) {
     bool in_queue = false;
@@ -100,6 +118,22 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, c
           atomicAdd(&w.n_run[r], 1u);
           atomicAdd(&w.sum_kv[r], (unsigned long long)((int64_t)prompt + gen));
           atomicOr(&w.mask_run[r], 1ull << cls);
+          // a prefilled request: in flight on a P-stage instance, its first token produced by now
+          if (a.d_stage && a.mode[r] == HFX_PREFILL) {
+            const int64_t ft = a.first_token[i];
+            if (ft <= a.now) {
+              const int64_t tpot = s_tpot[cls];
+              slack = tpot > 0 ? ft + ((int64_t)gen + 1) * tpot - a.now - dev_Ed(p, 1, (int64_t)prompt + gen) : HFX_SLACK_MAX;
+              int prio;
+              if (p.weight_max > 0) {
+                const int64_t x = (int64_t)p.weight_max - a.weight[i];
+                prio = (int)(x < 0 ? 0 : (x > 62 ? 62 : x));
+              } else prio = s_prio[cls];
+              k48 = dev_key48(PH_QUEUED, prio, slack) | DQ_TAG;
+              dmask |= 1ull << cls;
+              dmine += 1u;
+            }
+          }
         }
       } else if (ok && st == HFX_QUEUED && a.arrival[i] <= a.now && prompt <= a.cap_max) {
         const int64_t ttft = s_ttft[cls];
@@ -123,12 +157,18 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, c
   }
   qmask = warp_or_u64(qmask);
   if (lane == 0 && qmask) atomicOr(&w.ctl[0], qmask);
+  if (a.d_stage) {
+    dmask = warp_or_u64(dmask);
+    if (lane == 0 && dmask) atomicOr(&w.ctl[8], dmask);
+    dmine = (uint32_t)warp_sum_i64(dmine);
+    if (lane == 0 && dmine) atomicAdd(&s_dcount, dmine);
+  }
   if (bad) atomicOr(a.status, bad);
   if (falls) atomicExch(&w.ctl[5], 1ull);
   mine = (uint32_t)warp_sum_i64(mine);
   if (lane == 0 && mine) atomicAdd(&s_count, mine);
   __syncthreads();
-  if (threadIdx.x == 0) w.blk_cnt[blockIdx.x] = s_count;
+  if (threadIdx.x == 0) { w.blk_cnt[blockIdx.x] = s_count; w.blk_cnt[DISP_SCAN_BLOCKS_MAX + blockIdx.x] = s_dcount; }
 }
 
 // k_disp_compact: the queue rows in row order, as (sort word, row) pairs.  A block starts where the blocks
@@ -136,7 +176,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_scan(const HfxParams p, c
 // queue" flags.  When the request ids rise with the rows the pairs carry the 48-bit key at once (row
 // order is id order, and the radix passes keep it among equal keys); otherwise they carry the request id,
 // which is ordered first.
-__global__ void __launch_bounds__(DISP_THREADS) k_disp_compact(const DispArgs a, const DispWork w) {
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_compact(const DispArgs a, const DispWork w, const int stage) {
   __shared__ uint32_t s_warp[DISP_THREADS / 32];
   __shared__ unsigned long long s_base;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -144,7 +184,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_compact(const DispArgs a,
   __syncthreads();
   {
     unsigned long long part = 0;
-    for (int bb = threadIdx.x; bb < (int)blockIdx.x; bb += blockDim.x) part += w.blk_cnt[bb];
+    for (int bb = threadIdx.x; bb < (int)blockIdx.x; bb += blockDim.x) part += w.blk_cnt[stage * DISP_SCAN_BLOCKS_MAX + bb];
     part = (unsigned long long)warp_sum_i64((int64_t)part);
     if (lane == 0 && part) atomicAdd(&s_base, part);
   }
@@ -155,7 +195,8 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_compact(const DispArgs a,
   const int64_t lo = (int64_t)blockIdx.x * chunk, hi = lo + chunk < a.n ? lo + chunk : a.n;
   for (int64_t i0 = lo; i0 < hi; i0 += blockDim.x) {
     const int64_t i = i0 + threadIdx.x;
-    const uint64_t k48 = i < hi ? w.rowkey[i] : 0;
+    uint64_t k48 = i < hi ? w.rowkey[i] : 0;
+    k48 = (k48 != 0 && (int)(k48 >> 63) == stage) ? (k48 & KEY48) : 0;      // this stage's queue only
     const uint32_t m = __ballot_sync(0xffffffffu, k48 != 0);
     if (lane == 0) s_warp[warp] = __popc(m);
     __syncthreads();
@@ -169,7 +210,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_compact(const DispArgs a,
     run += all;
     __syncthreads();
   }
-  if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) w.ctl[1] = run;      // the queue's length
+  if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) w.ctl[8 * stage + 1] = run;      // the queue's length
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -294,14 +335,14 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_gather(uint64_t *__restri
   if (*only_if == 0) return;
   const int64_t n = (int64_t)*ctl_n;
   for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += (int64_t)gridDim.x * blockDim.x)
-    keys[j] = rowkey[vals[j]];
+    keys[j] = rowkey[vals[j]] & KEY48;
 }
 
 // ------------------------------------------------------------------------------------------------
 // Running total of prompt lengths along the ordered queue: per-tile totals, the last block scans
 // them; then every tile scans its own items on top of its offset and lists the queue's rows.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(DISP_THREADS) k_disp_tilesum(const uint32_t *__restrict__ vals, const int32_t *__restrict__ prompt_len,
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_tilesum(const uint32_t *__restrict__ vals, const DispCost cost,
                                                                const unsigned long long *ctl, int64_t *__restrict__ tile_sum,
                                                                int32_t tiles_max, unsigned long long *done) {
   __shared__ int64_t s_red[32], s_redc[32];
@@ -314,7 +355,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_tilesum(const uint32_t *_
     const int64_t lo = (int64_t)blockIdx.x * RADIX_TILE;
     const int64_t hi = lo + RADIX_TILE < n ? lo + RADIX_TILE : n;
     int64_t s = 0, c = 0;
-    for (int64_t j = lo + threadIdx.x; j < hi; j += DISP_THREADS) { const int64_t x = prompt_len[vals[j]]; if (x <= bmax) { s += x; c += 1; } }
+    for (int64_t j = lo + threadIdx.x; j < hi; j += DISP_THREADS) { const int64_t x = cost.of(vals[j]); if (x <= bmax) { s += x; c += 1; } }
     s = warp_sum_i64(s); c = warp_sum_i64(c);
     if (lane == 0) { s_red[warp] = s; s_redc[warp] = c; }
     __syncthreads();
@@ -350,11 +391,11 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_tilesum(const uint32_t *_
   }
 }
 
-__global__ void __launch_bounds__(DISP_THREADS) k_disp_prefix(const uint32_t *__restrict__ vals, const int32_t *__restrict__ prompt_len,
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_prefix(const uint32_t *__restrict__ vals, const DispCost cost,
                                                               const unsigned long long *ctl, const int64_t *__restrict__ tile_sum,
                                                               int32_t tiles_max, int64_t *__restrict__ prefix,
                                                               int32_t *__restrict__ prefix_cnt, int32_t *__restrict__ queue_order,
-                                                              int32_t *__restrict__ n_queue) {
+                                                              int32_t *__restrict__ n_queue, const unsigned long long *listed_before) {
   __shared__ int64_t s_warp[32];
   __shared__ int32_t s_warpc[32];
   const int64_t n = (int64_t)ctl[1];
@@ -362,6 +403,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_prefix(const uint32_t *__
   const int32_t tiles = (int32_t)((n + RADIX_TILE - 1) / RADIX_TILE);
   if (blockIdx.x == 0 && threadIdx.x == 0) *n_queue = (int32_t)n;
   if ((int)blockIdx.x >= tiles) return;
+  const int64_t q0 = listed_before ? (int64_t)*listed_before : 0;      // the D stage's queue is listed behind the first stage's
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t lo = (int64_t)blockIdx.x * RADIX_TILE + (int64_t)threadIdx.x * RADIX_ITEMS;
   int64_t c[RADIX_ITEMS], sum = 0;
@@ -371,9 +413,9 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_prefix(const uint32_t *__
     c[k] = 0; e[k] = 0;
     if (lo + k < n) {
       const uint32_t row = vals[lo + k];
-      const int64_t x = prompt_len[row];
+      const int64_t x = cost.of(row);
       if (x <= bmax) { c[k] = x; e[k] = 1; }      // larger than every budget of this call: passed over
-      queue_order[lo + k] = (int32_t)row;
+      queue_order[q0 + lo + k] = (int32_t)row;
     }
     sum += c[k]; cnt += e[k];
   }
@@ -395,12 +437,21 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_prefix(const uint32_t *__
 // k_disp_plan: dispatching step 2 for every instance (E_d of its running batch, the safe budget from
 // the strictest TTFT in the queue and the strictest TPOT in flight); resets the per-instance results.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(DISP_THREADS) k_disp_plan(const HfxParams p, const DispArgs a, const DispWork w) {
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_plan(const HfxParams p, const DispArgs a, const DispWork w, const int stage) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r >= p.n_replicas) return;
   ReplicaPlan pl;
+  if (stage) {     // the D stage: the time budget of a DECODE instance, from its batch or the queue of prefilled requests
+    if (a.cfg[r].mode != HFX_DECODE) return;
+    dev_plan(p, a.cfg[r], a.now, a.maturity[r], (int64_t)w.n_run[r], (int64_t)w.sum_kv[r], w.mask_run[r], w.ctl[8], pl);
+    w.plan[r] = pl;
+    a.budget[r] = pl.budget;
+    if (pl.now >= pl.mat && pl.budget > 0) atomicMax(&w.ctl[8 + 4], (unsigned long long)pl.budget);
+    return;
+  }
+  if (r == 0) { a.n_queue[1] = 0; a.n_mature[1] = 0; }
   dev_plan(p, a.cfg[r], a.now, a.maturity[r], (int64_t)w.n_run[r], (int64_t)w.sum_kv[r], w.mask_run[r], w.ctl[0], pl);
-  if (pl.mode == HFX_DECODE) pl.budget = 0;      // a D-stage instance is served by the per-replica step, not from this queue
+  if (pl.mode == HFX_DECODE) pl.budget = 0;      // a D-stage instance takes nothing from this queue
   w.plan[r] = pl;
   a.budget[r] = pl.budget;
   a.e_d[r] = pl.e_d;
@@ -455,7 +506,7 @@ __device__ __forceinline__ int64_t warp_longest(int64_t lo0, const int64_t hi0, 
   return lo;
 }
 
-__global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const DispArgs a, const DispWork w) {
+__global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const DispArgs a, const DispWork w, const int stage) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int R = p.n_replicas;
   uint64_t *s_mat = reinterpret_cast<uint64_t *>(smem_raw);     // [R] maturity, biased to unsigned order; then the budgets
@@ -468,7 +519,7 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
   if (threadIdx.x == 0) { s_nm = 0; s_k = 0; s_done = 0; s_cursor = 0; s_base = 0; s_basec = 0; }
   __syncthreads();
   for (int r = threadIdx.x; r < R; r += blockDim.x)
-    if (a.maturity[r] <= a.now && a.cfg[r].mode != HFX_DECODE) {
+    if (a.maturity[r] <= a.now && (a.cfg[r].mode == HFX_DECODE) == (stage != 0)) {
       const int k = atomicAdd(&s_nm, 1);
       s_mat[k] = (uint64_t)a.maturity[r] ^ (1ull << 63);
       s_id[k] = (uint32_t)r;
@@ -477,18 +528,19 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
   const int nm = s_nm;
   block_sort<true>(s_mat, s_id, nm);
   int64_t *s_bud = reinterpret_cast<int64_t *>(s_mat);
+  const int listed = stage ? a.n_mature[0] : 0;      // the D instances are listed behind the first stage's
   for (int k = threadIdx.x; k < nm; k += blockDim.x) {
     const int r = (int)s_id[k];
-    a.inst_order[k] = r;
+    a.inst_order[listed + k] = r;
     const ReplicaPlan *pl = w.plan + r;
     s_bud[k] = pl->budget;
     int64_t room = INT32_MAX;
     if (pl->batch_cap != 0) { const int64_t left = (int64_t)pl->batch_cap - pl->n_eff; room = left > 0 ? left : 0; }
     s_room[k] = (int32_t)(room < INT32_MAX ? room : INT32_MAX);
   }
-  if (threadIdx.x == 0) *a.n_mature = nm;
+  if (threadIdx.x == 0) a.n_mature[stage] = nm;
   const int lane = threadIdx.x & 31;
-  const int64_t nq = (int64_t)w.ctl[1];
+  const int64_t nq = (int64_t)w.ctl[8 * stage + 1];
   for (int guard = 0; guard < 2 * nm + 4; guard++) {      // every round finishes an instance or refills for one
     __syncthreads();
     if (s_done || s_k >= nm || s_cursor >= nq) break;
@@ -502,7 +554,8 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
       int64_t cursor = s_cursor, base = s_base, base_cnt = s_basec;
       for (; k < nm && cursor < nq; k++) {
         const int64_t span = nq - cursor, avail = w0 + wn - cursor;
-        const int64_t limit = base + s_bud[k], limit_cnt = base_cnt + s_room[k];
+        const int64_t limit = s_bud[k] > INT64_MAX - base ? INT64_MAX : base + s_bud[k];      // (a D-stage budget may be unbounded)
+        const int64_t limit_cnt = base_cnt + s_room[k];
         const int64_t off = cursor - w0 - 1;
         const int64_t hiw = span < avail ? span : avail;
         int64_t m = warp_longest(0, hiw, lane, [&](int64_t x) { return s_pre[off + x] <= limit && (int64_t)s_cnt[off + x] <= limit_cnt; });
@@ -533,17 +586,34 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
 
 // the request -> instance binding of every dispatched row, and dispatching step 4 (the new maturity
 // time of an instance that took requests): one block per instance
-__global__ void __launch_bounds__(DISP_THREADS) k_disp_assign(const HfxParams p, const DispArgs a, const DispWork w, int slot) {
+__global__ void __launch_bounds__(DISP_THREADS) k_disp_assign(const HfxParams p, const DispArgs a, const DispWork w, int slot,
+                                                              const DispCost cost, const int stage) {
   const int r = blockIdx.x;
+  if ((a.cfg[r].mode == HFX_DECODE) != (stage != 0)) return;      // the other stage's instance
   const int32_t m = w.run_len[r], s0 = w.run_start[r];
-  if (threadIdx.x == 0 && a.adm_count[r] > 0) {
-    int64_t lp = 0;
-    a.maturity_next[r] = dev_maturity_next(p, w.plan[r], a.adm_count[r], a.adm_cost[r], 0, &lp);
-  }
-  const int64_t bmax = (int64_t)w.ctl[4];
+  const int64_t bmax = (int64_t)w.ctl[8 * stage + 4];
+  int64_t kv = 0;
   for (int32_t q = threadIdx.x; q < m; q += blockDim.x) {
     const uint32_t row = w.val[slot][s0 + q];
-    if (a.prompt_len[row] <= bmax) a.assign[row] = r;       // the others were passed over
+    if (cost.of(row) <= bmax) {       // the others were passed over
+      a.assign[row] = r;
+      kv += (int64_t)a.prompt_len[row] + a.gen[row];
+    }
+  }
+  if (stage) {      // maturity = end of the next decode iteration of the enlarged batch: the context the run brings
+    __shared__ int64_t s_kv[DISP_THREADS / 32];
+    kv = warp_sum_i64(kv);
+    if ((threadIdx.x & 31) == 0) s_kv[threadIdx.x >> 5] = kv;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      kv = 0;
+      for (int k = 0; k < DISP_THREADS / 32; k++) kv += s_kv[k];
+      int64_t lp = 0;
+      a.maturity_next[r] = dev_maturity_next(p, w.plan[r], a.adm_count[r], a.adm_cost[r], kv, &lp);
+    }
+  } else if (threadIdx.x == 0 && a.adm_count[r] > 0) {
+    int64_t lp = 0;
+    a.maturity_next[r] = dev_maturity_next(p, w.plan[r], a.adm_count[r], a.adm_cost[r], 0, &lp);
   }
 }
 
@@ -596,7 +666,7 @@ static int disp_workspace(hfx_sched *s, hfx_dispatch_ws **out) {
   ok = ok && cudaMalloc(&w.sum_kv, sizeof(unsigned long long) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.mask_run, sizeof(unsigned long long) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.ctl, 256) == cudaSuccess;
-  ok = ok && cudaMalloc(&w.blk_cnt, sizeof(uint32_t) * DISP_SCAN_BLOCKS_MAX) == cudaSuccess;
+  ok = ok && cudaMalloc(&w.blk_cnt, sizeof(uint32_t) * 2 * DISP_SCAN_BLOCKS_MAX) == cudaSuccess;
   ok = ok && cudaMalloc(&w.plan, sizeof(ReplicaPlan) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.run_start, sizeof(int32_t) * R) == cudaSuccess;
   ok = ok && cudaMalloc(&w.run_len, sizeof(int32_t) * R) == cudaSuccess;
@@ -607,7 +677,7 @@ static int disp_workspace(hfx_sched *s, hfx_dispatch_ws **out) {
 }
 
 int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const int64_t *maturity, const hfx_dispatch_out *o,
-                        int32_t cap_max) {
+                        int32_t cap_max, bool d_stage) {
   hfx_dispatch_ws *d = nullptr;
   int rc = disp_workspace(s, &d);
   if (rc != HFX_OK) return rc;
@@ -618,6 +688,7 @@ int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const 
   DispArgs a;
   a.replica_id = t->replica_id; a.class_id = t->class_id; a.state = t->state; a.prompt_len = t->prompt_len; a.gen = t->gen;
   a.arrival = t->arrival_ns; a.req_id = t->req_id; a.weight = s->p.weight_max > 0 ? t->weight : nullptr;
+  a.first_token = t->first_token_ns; a.d_stage = d_stage ? 1 : 0; a.mode = s->d_mode;
   a.n = n; a.now = now_ns; a.cap_max = cap_max; a.maturity = maturity; a.cfg = s->d_cfg;
   a.assign = o->assign; a.queue_order = o->queue_order; a.n_queue = o->n_queue; a.inst_order = o->inst_order;
   a.n_mature = o->n_mature; a.slack = o->slack_ns; a.budget = o->budget; a.e_d = o->e_d_ns; a.n_run = o->n_run;
@@ -626,38 +697,39 @@ int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const 
   if (cudaMemsetAsync(w.n_run, 0, sizeof(uint32_t) * R, st) != cudaSuccess ||
       cudaMemsetAsync(w.sum_kv, 0, sizeof(unsigned long long) * R, st) != cudaSuccess ||
       cudaMemsetAsync(w.mask_run, 0, sizeof(unsigned long long) * R, st) != cudaSuccess ||
-      cudaMemsetAsync(w.ctl, 0, 64, st) != cudaSuccess)
+      cudaMemsetAsync(w.ctl, 0, 128, st) != cudaSuccess)
     return HFX_E_CUDA;
   const int tiles_max = (int)((s->max_rows + RADIX_TILE - 1) / RADIX_TILE);
   const int tiles = n > 0 ? (int)((n + RADIX_TILE - 1) / RADIX_TILE) : 1;      // tiles the queue can fill in this call
-  {
-    KernelScope ks(s, KSLOT_DISPATCH);
-    int grid = (int)((n + DISP_THREADS - 1) / DISP_THREADS);
-    if (grid > s->n_sm * 8) grid = s->n_sm * 8;
-    if (grid > DISP_SCAN_BLOCKS_MAX) grid = DISP_SCAN_BLOCKS_MAX;
-    if (grid < 1) grid = 1;
-    k_disp_scan<<<grid, DISP_THREADS, 0, st>>>(s->p, a, w);
-    s->launches++;
-    k_disp_compact<<<grid, DISP_THREADS, 0, st>>>(a, w);
+  int grid = (int)((n + DISP_THREADS - 1) / DISP_THREADS);
+  if (grid > s->n_sm * 8) grid = s->n_sm * 8;
+  if (grid > DISP_SCAN_BLOCKS_MAX) grid = DISP_SCAN_BLOCKS_MAX;
+  if (grid < 1) grid = 1;
+  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_scan<<<grid, DISP_THREADS, 0, st>>>(s->p, a, w); }
+  for (int stage = 0; stage < (d_stage ? 2 : 1); stage++) {
+    unsigned long long *ctl = w.ctl + 8 * stage;
+    DispCost cost;
+    cost.prompt_len = t->prompt_len; cost.gen = t->gen; cost.d1 = s->p.d1; cost.d2 = s->p.d2; cost.stage = stage;
+    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_compact<<<grid, DISP_THREADS, 0, st>>>(a, w, stage); }
+    int slot = 0;
+    auto pass = [&](int shift, const unsigned long long *only_if) {
+      { KernelScope ks(s, KSLOT_DISPATCH); k_radix_hist<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], ctl + 1, shift, w.hist, only_if); }
+      { KernelScope ks(s, KSLOT_DISPATCH); k_radix_scatter<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.key[slot ^ 1], w.val[slot ^ 1], ctl + 1, shift, w.hist, only_if); }
+      slot ^= 1;
+    };
+    // by request id, only when the ids do not rise with the rows (the kernels leave at once otherwise; an even
+    // number of passes, so the pairs are back in the first buffer either way)
+    for (int shift = 0; shift < 32; shift += 8) pass(shift, w.ctl + 5);
+    {
+      KernelScope ks(s, KSLOT_DISPATCH);
+      k_disp_gather<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.rowkey, ctl + 1, w.ctl + 5);
+    }
+    for (int shift = 0; shift < 48; shift += 8) pass(shift, nullptr);   // by (priority, slack)
+    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_plan<<<(R + DISP_THREADS - 1) / DISP_THREADS, DISP_THREADS, 0, st>>>(s->p, a, w, stage); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_tilesum<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], cost, ctl, w.tile_sum, tiles_max, ctl + 3); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_prefix<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], cost, ctl, w.tile_sum, tiles_max, w.prefix, w.prefix_cnt, o->queue_order, o->n_queue + stage, stage ? w.ctl + 1 : nullptr); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_chain<<<1, 1024, 16 * (size_t)R, st>>>(s->p, a, w, stage); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_assign<<<R, DISP_THREADS, 0, st>>>(s->p, a, w, slot, cost, stage); }
   }
-  int slot = 0;
-  auto pass = [&](int shift, const unsigned long long *only_if) {
-    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_hist<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.ctl + 1, shift, w.hist, only_if); }
-    { KernelScope ks(s, KSLOT_DISPATCH); k_radix_scatter<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.key[slot ^ 1], w.val[slot ^ 1], w.ctl + 1, shift, w.hist, only_if); }
-    slot ^= 1;
-  };
-  // by request id, only when the ids do not rise with the rows (the kernels leave at once otherwise; an even
-  // number of passes, so the pairs are back in the first buffer either way)
-  for (int shift = 0; shift < 32; shift += 8) pass(shift, w.ctl + 5);
-  {
-    KernelScope ks(s, KSLOT_DISPATCH);
-    k_disp_gather<<<tiles, DISP_THREADS, 0, st>>>(w.key[slot], w.val[slot], w.rowkey, w.ctl + 1, w.ctl + 5);
-  }
-  for (int shift = 0; shift < 48; shift += 8) pass(shift, nullptr);   // by (priority, slack)
-  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_plan<<<(R + DISP_THREADS - 1) / DISP_THREADS, DISP_THREADS, 0, st>>>(s->p, a, w); }
-  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_tilesum<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.ctl + 3); }
-  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_prefix<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], t->prompt_len, w.ctl, w.tile_sum, tiles_max, w.prefix, w.prefix_cnt, o->queue_order, o->n_queue); }
-  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_chain<<<1, 1024, 16 * (size_t)R, st>>>(s->p, a, w); }
-  { KernelScope ks(s, KSLOT_DISPATCH); k_disp_assign<<<R, DISP_THREADS, 0, st>>>(s->p, a, w, slot); }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }

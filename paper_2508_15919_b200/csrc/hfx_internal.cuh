@@ -566,7 +566,7 @@ int hfx_launch_regroup(hfx_sched *s, const RegroupArgs &ra, int32_t *seg_off);
 int hfx_launch_replicas(hfx_sched *s, const SegArgs &sa, int64_t n, bool slabs);
 int hfx_launch_step(hfx_sched *s, const hfx_table *t, const hfx_replica_state *st, const hfx_step_out *o, uint32_t flags);
 int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const int64_t *maturity, const hfx_dispatch_out *o,
-                        int32_t cap_max);
+                        int32_t cap_max, bool d_stage);
 void hfx_dispatch_release(hfx_sched *s);
 void hfx_sim_release(hfx_sched *s);
 int hfx_launch_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const hfx_slo_bounds *b, int64_t *last_queue,

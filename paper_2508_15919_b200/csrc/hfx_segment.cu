@@ -234,6 +234,23 @@ __device__ __forceinline__ int64_t next_arrival_listed(const SegArgs &a, const S
   return v;
 }
 
+// The same when the inactive rows are not listed yet (a long list that the grid writes at the end of the kernel):
+// read from the slabs, a warp of the group per tile, its lanes over the replica's inactive rows of that tile.
+__device__ __forceinline__ int64_t next_arrival_slabs(const SegArgs &a, const SegCtx &c, int R1, int r, const Grp &G) {
+  const int lane = G.tid & 31, warp = G.tid >> 5, nwarp = G.n >> 5;
+  int64_t v = HFX_INF;
+  for (int t = warp; t < c.n_tiles; t += nwarp) {
+    const uint2 m = __ldcg(c.M + (size_t)t * R1 + r);
+    const uint32_t ca = m.y >> 16, ci = (m.x >> 16) - ca, src = (m.x & 0xffffu) + ca;
+    const size_t tb = (size_t)t * c.tile_rows;
+    for (uint32_t k = lane; k < ci; k += 32) {
+      const size_t row = tb + __ldcg(c.slab_idx + tb + src + k);
+      if (c.rowflag[row] == KIND_FUTURE) { const int64_t x = a.arrival[row]; v = x < v ? x : v; }
+    }
+  }
+  return v;
+}
+
 // minimum of v over the group into sh.next_arrival (all threads of the group call)
 __device__ __forceinline__ void group_min_arrival(int64_t v, BlockShared &sh, const Grp &G) {
   const int lane = G.tid & 31, warp = G.tid >> 5, nwarp = G.n >> 5;
@@ -740,7 +757,7 @@ __device__ void small_replica(const HfxParams &p, const SegArgs &a, const SegCtx
   const int64_t mat_next = sh.red_c[0];
   if (commit && !worked) {
     // idle replica: its next arrival is looked up among its listed inactive rows (unless the grid lists them later)
-    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, G.tid, G.n) : HFX_INF, sh, G);
+    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, G.tid, G.n) : next_arrival_slabs(a, c, R1, r, G), sh, G);
   }
   if (G.tid == 0 && real)
     write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
@@ -1099,7 +1116,7 @@ __device__ void medium_replica(const HfxParams &p, const SegArgs &a, const SegCt
   const int worked = sh.worked;
   const int64_t mat_next = sh.red_c[0];
   if (commit && !worked)      // idle replica: its next arrival is looked up among its listed inactive rows
-    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x) : HFX_INF, sh, B);
+    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x) : next_arrival_slabs(a, c, p.n_replicas + 1, r, B), sh, B);
   if (threadIdx.x == 0 && real)
     write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
 
@@ -1428,7 +1445,7 @@ __device__ void medium_ordered(const HfxParams &p, const SegArgs &a, const SegCt
   const int worked = sh.worked;
   const int64_t mat_next = sh.red_c[0];
   if (commit && !worked)      // idle replica: its next arrival is looked up among its listed inactive rows
-    group_min_arrival(list_in ? next_arrival_listed(a, c, b, n_act, n, tid, REP_THREADS) : HFX_INF, sh, B);
+    group_min_arrival(list_in ? next_arrival_listed(a, c, b, n_act, n, tid, REP_THREADS) : next_arrival_slabs(a, c, R + 1, r, B), sh, B);
   if (tid == 0 && real)
     write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
 
@@ -1610,7 +1627,7 @@ __device__ void oversize_replica(const HfxParams &p, const SegArgs &a, const Seg
   const int worked = sh.worked;
   const int64_t mat_next = sh.red_c[0];
   if (commit && !worked)
-    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x) : HFX_INF, sh, B);
+    group_min_arrival(list_in || !ordered ? next_arrival_listed(a, c, b, n_act, n, threadIdx.x, blockDim.x) : next_arrival_slabs(a, c, p.n_replicas + 1, r, B), sh, B);
   if (threadIdx.x == 0 && real)
     write_replica_outputs(a, r, pl, sh.adm_cost, sh.adm_count, mat_next, worked, sh.t2, sh.next_arrival);
   if (a.admitted_rows)

@@ -8,7 +8,7 @@ import pytest
 
 import gen
 import oracle
-from helpers import MS, load_pins, make_wl
+from helpers import MS, load_pins, make_wl, migrator_hand_case
 
 PINS = load_pins()
 M = gen.DEFAULT_MODEL
@@ -555,33 +555,17 @@ def test_dispatch_serves_the_p_stage():
     assert o["maturity_next"][2] - now == PINS["Ed_80_64000"] == 17_280_000
 
 
-def _migrator_hand_case():
-    # model with a decode iteration of 8 ms + 2 ms per request + 2 us per token of context
-    now = 1000 * MS
-    model = (5_000_000, 40_000, 2, 8_000_000, 2_000_000, 2_000)
-    classes = [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)]
-    rows = [dict(state=1, replica_id=2, class_id=1, prompt_len=1000, gen=10, output_len=500, first_token_ns=now - 600 * MS),   # in flight on D instance 2
-            dict(state=1, replica_id=2, class_id=1, prompt_len=1000, gen=10, output_len=500, first_token_ns=now - 600 * MS),
-            dict(state=1, replica_id=0, class_id=1, prompt_len=7000, gen=0, output_len=50, first_token_ns=now - 20 * MS),      # A  row 2
-            dict(state=1, replica_id=0, class_id=0, prompt_len=500, gen=0, output_len=50, first_token_ns=now - 25 * MS),       # B  row 3
-            dict(state=1, replica_id=0, class_id=0, prompt_len=4000, gen=0, output_len=50, first_token_ns=now - 1 * MS),       # C  row 4
-            dict(state=1, replica_id=0, class_id=0, prompt_len=100, gen=0, output_len=50, first_token_ns=now + 1)]             # its prefill batch has not ended
-    wl = make_wl(rows, classes, replicas=[(gen.PREFILL, 8192, 0), (gen.DECODE, 8192, 0), (gen.DECODE, 8192, 3)],
-                 now=[now] * 3, maturity=[now + 1, now - 5 * MS, now - 10 * MS], model=model)
-    return wl, now
-
-
 def test_migrator_selects_the_d_instance_hand_worked():
-    # Sec. 3.3.1, "Disaggregated Mode": the four steps once more for the D stage.  E_d(n, kv) = 8 ms + 2 ms n + 2 us kv.
+    # Sec. 3.3.1, "Disaggregated Mode": the four steps once more for the D stage.  E_d(n, kv) = 8 ms + 2 ms n + 0.2 us kv.
     # Queue of prefilled requests (first token produced): slack = first_token + TPOT - now - E_d(1, kv)
-    #   A (class 1, 50 ms, 7000 tokens)  30 ms - 24 ms =  6 ms   cost 2 ms + 14 ms = 16 ms
-    #   B (class 0, 30 ms,  500 tokens)   5 ms - 11 ms = -6 ms   cost 2 ms +  1 ms =  3 ms
-    #   C (class 0, 30 ms, 4000 tokens)  29 ms - 18 ms = 11 ms   cost 2 ms +  8 ms = 10 ms
+    #   A (class 1, 50 ms, 70000 tokens) 30 ms - 24 ms =  6 ms   cost 2 ms + 14 ms = 16 ms
+    #   B (class 0, 30 ms,  5000 tokens)  5 ms - 11 ms = -6 ms   cost 2 ms +  1 ms =  3 ms
+    #   C (class 0, 30 ms, 40000 tokens) 29 ms - 18 ms = 11 ms   cost 2 ms +  8 ms = 10 ms
     # order: priority 0 first (B, C), then A.  Instance 2 matured first (10 ms ago): two requests in flight with
-    # 2020 tokens, E_d = 8 + 4 + 4.04 = 16.04 ms, strictest TPOT in flight 50 ms: budget 33.96 ms; its batch cap of 3
+    # 20200 tokens, E_d = 8 + 4 + 4.04 = 16.04 ms, strictest TPOT in flight 50 ms: budget 33.96 ms; its batch cap of 3
     # leaves room for one request: it takes B and stops at C.  Instance 1 is idle: strictest TPOT of the queue as
     # the call began (30 ms) minus E_d(0, 0) = 22 ms; it takes C (10 ms), A (16 ms more) does not fit and waits.
-    wl, now = _migrator_hand_case()
+    wl, now = migrator_hand_case()
     o = oracle.dispatch(wl, now)
     assert o["status"] == 0
     assert list(o["n_queue"]) == [0, 3] and list(o["queue_order"][:4]) == [3, 4, 2, -1]
@@ -600,7 +584,7 @@ def test_migrator_selects_the_d_instance_hand_worked():
     o = oracle.dispatch(wl, now)
     assert list(o["n_mature"]) == [0, 1] and list(o["inst_order"]) == [1, -1, -1] and o["budget"][2] == 0
     assert list(o["assign"]) == [-1, -1, -1, 1, 1, -1] and o["adm_cost"][1] == 13_000_000
-    assert o["maturity_next"][1] - now == 8_000_000 + 2 * 2_000_000 + 2_000 * 4500 and o["maturity_next"][2] == now + 1
+    assert o["maturity_next"][1] - now == 8_000_000 + 2 * 2_000_000 + 200 * 45_000 and o["maturity_next"][2] == now + 1
     # binding: a dispatched prefilled request stays in flight, now on its D instance
     wl.maturity[2] = now - 10 * MS
     o = oracle.dispatch(wl, now)

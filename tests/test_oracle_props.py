@@ -6,7 +6,7 @@ import pytest
 
 import gen
 import oracle
-from helpers import MS, SEC, make_wl, permute_rows
+from helpers import MS, SEC, make_wl, permute_rows, migrator_case
 
 MODES3 = (gen.COLOCATED, gen.PREFILL, gen.DECODE)
 
@@ -441,23 +441,9 @@ def test_scaling_loop_invariants():
 
 
 # ---- the D stage of the dispatching call (the Migrator) ----------------------------------------------
-def _migrator_case(seed, **kw):
-    modes = (gen.PREFILL, gen.DECODE, gen.DECODE, gen.COLOCATED, gen.DECODE)[: 2 + seed % 4]
-    wl = gen.random_table(200 + seed, 80 + 41 * seed, len(modes), modes=modes, inflight=0.7, **kw)
-    wl.replicas[:, 0] = modes          # (the generator draws the modes; here every instance has the one listed)
-    now = int(wl.now.max())
-    t = wl.table
-    run_on_p = (t["state"] == gen.RUNNING) & (wl.replicas[np.clip(t["replica_id"], 0, wl.n_replicas - 1), 0] == gen.PREFILL)
-    # prefill batches that ended up to 40 ms ago, a few that have not ended yet
-    rng = np.random.default_rng(seed)
-    t["first_token_ns"][run_on_p] = now - rng.integers(-3 * MS, 40 * MS, int(run_on_p.sum()))
-    wl.maturity[:] = now - rng.integers(-2 * MS, 20 * MS, wl.n_replicas)
-    return wl, now
-
-
 @pytest.mark.parametrize("seed", range(12))
 def test_migrator_invariants(seed):
-    wl, now = _migrator_case(seed, batch_cap=(0, 6)[seed % 3 == 1], tie_heavy=seed % 4 == 2,
+    wl, now = migrator_case(seed, batch_cap=(0, 6)[seed % 3 == 1], tie_heavy=seed % 4 == 2,
                              budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 3])
     o = oracle.dispatch(wl, now)
     t, R, M = wl.table, wl.n_replicas, wl.model

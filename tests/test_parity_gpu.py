@@ -503,7 +503,7 @@ def test_dispatch_argument_errors_and_bad_rows():
     sched.dispatch_step(tab, now, mat, out)          # still usable
     assert sched.status() == 0
     sched.close()
-    # P-stage instances are served like colocated ones, D-stage instances take no part
+    # P-stage instances are served like colocated ones, D-stage instances by the second stage of the call
     for seed in (42, 44, 45):
         wl2 = gen.random_table(seed, 3000, 7, modes=MODES3, batch_cap=(0, 5)[seed % 2])
         assert_dispatch_parity(wl2, int(wl2.now.max()))
@@ -513,6 +513,57 @@ def test_dispatch_argument_errors_and_bad_rows():
     wl3.table["prompt_len"][5::131] = -3
     wl3.table["replica_id"][7::53] = 99
     assert_dispatch_parity(wl3, int(wl3.now.max()))
+
+
+def test_migrator_selects_d_instances():
+    # the D stage of the dispatching call (Sec. 3.3.1, "D-stage Migrator"): the hand-worked case, then seeded tables
+    from helpers import migrator_case, migrator_hand_case
+    wl, now = migrator_hand_case()
+    g = assert_dispatch_parity(wl, now, calls=2)
+    assert list(g["assign"]) == [-1, -1, -1, 2, 1, -1] and list(g["n_queue"]) == [0, 3] and list(g["inst_order"]) == [2, 1, -1]
+    for seed in range(12):
+        wl, now = migrator_case(seed, batch_cap=(0, 6)[seed % 3 == 1], tie_heavy=seed % 4 == 2,
+                                budget_mode=(gen.BUDGET_SAFE, gen.BUDGET_CAP_ONLY)[seed % 5 == 3], permute_ids=seed % 2 == 0)
+        assert_dispatch_parity(wl, now)
+    # D instances only (no P stage: the queue of prefilled requests is empty, the budgets and maturities stand)
+    wl = gen.random_table(77, 5000, 4, modes=(gen.DECODE,), inflight=0.5)
+    assert_dispatch_parity(wl, int(wl.now.max()))
+
+
+def test_migrator_many_tiles_and_binding():
+    # a table whose two queues span many tiles; both stages dispatch; binding puts the prefilled requests in flight
+    # on their D instances, and the per-replica step that follows agrees with the oracle's
+    import paper_2508_15919_b200 as hfx
+    R = 48
+    wl = gen.random_table(88, 150_001, R, modes=MODES3, inflight=0.6, permute_ids=False)
+    wl.replicas[:, 0] = np.arange(R) % 3                      # colocated, P, D in turn
+    now = int(wl.now.max())
+    wl.now[:] = now
+    t = wl.table
+    on_p = (t["state"] == gen.RUNNING) & (wl.replicas[np.clip(t["replica_id"], 0, R - 1), 0] == gen.PREFILL)
+    rng = np.random.default_rng(5)
+    t["first_token_ns"][on_p] = now - rng.integers(-2 * MS, 30 * MS, int(on_p.sum()))
+    on_d = np.nonzero((t["state"] == gen.RUNNING) & (wl.replicas[np.clip(t["replica_id"], 0, R - 1), 0] == gen.DECODE))[0]
+    t["state"][on_d[on_d % 100 != 0]] = gen.DONE            # small decode batches: the D instances have room
+    wl.maturity[:] = now - rng.integers(-1 * MS, 10 * MS, R)
+    g = assert_dispatch_parity(wl, now)
+    assert g["n_queue"][0] > 10_000 and g["n_queue"][1] > 10_000 and g["n_mature"][1] > 0
+    d_inst = np.nonzero(wl.replicas[:, 0] == gen.DECODE)[0]
+    assert g["adm_count"][d_inst].sum() > 0 and set(np.unique(g["assign"][on_p])) <= set(d_inst.tolist()) | {-1}
+    # bind on both sides, then one per-replica step
+    sched = make_sched(wl)
+    tab = hfx.DeviceTable.from_numpy(wl.table)
+    out = hfx.DispatchOut(wl.n_rows, R)
+    mat = torch.from_numpy(wl.maturity.copy()).cuda()
+    clock = torch.from_numpy(wl.now.copy()).cuda()
+    sched.dispatch_step(tab, now, mat, out)
+    sched.dispatch_bind(tab, now, out, clock)
+    c = oracle.dispatch(wl, now)
+    oracle.dispatch_bind(wl, now, c)
+    assert np.array_equal(tab.to_numpy()["replica_id"], wl.table["replica_id"]) and np.array_equal(clock.cpu().numpy(), wl.now)
+    sched.close()
+    wl.maturity[:] = c["maturity_next"]
+    assert_step_parity(wl, steps=2, commit=True)
 
 
 # ---- priority-based SLO mapping ---------------------------------------------------------------------------
@@ -1041,3 +1092,35 @@ def test_medium_replica_with_crowded_and_outlying_slacks(n):
     r = np.nonzero(t["state"] == gen.RUNNING)[0]
     t["last_token_ns"][r] = int(wl.now[0]) - (np.arange(len(r)) % 7)         # requests in flight with seven distinct slacks per class
     assert_step_parity(wl, steps=2, commit=True)
+
+
+@pytest.mark.parametrize("grouped", [False, True])
+def test_idle_replica_with_a_long_list_of_inactive_rows_jumps_to_its_next_arrival(grouped):
+    # An ordered step (ids in row order) leaves lists of more than 2048 inactive rows to the end of the kernel; an idle
+    # replica that commits must still find the earliest arrival among them for its clock jump.  Replica 0: nothing
+    # in flight, nothing arrived, 3000 finished requests and a few that arrive later; replica 1: busy; replica 2:
+    # idle with a short list.  Interleaved rows and rows grouped by replica; small and whole-block replicas.
+    for n_busy in (300, 2500):
+        wl = gen.random_table(70 + n_busy % 7, 3000 + n_busy + 200, 3, modes=(gen.COLOCATED, gen.COLOCATED, gen.DECODE),
+                              permute_ids=False, grouped=grouped, inflight=0.4, done=0.0, future=0.0)
+        wl.replicas[:, 0] = (gen.COLOCATED, gen.COLOCATED, gen.DECODE)
+        t = wl.table
+        now = int(wl.now.max())
+        wl.now[:] = now
+        wl.maturity[:] = now - 1
+        rid = np.zeros(wl.n_rows, np.int32)
+        rid[3000:3000 + n_busy] = 1
+        rid[3000 + n_busy:] = 2
+        if not grouped:
+            rid = rid[np.random.default_rng(n_busy).permutation(wl.n_rows)]
+        t["replica_id"][:] = rid
+        r0 = np.nonzero(rid == 0)[0]
+        t["state"][r0] = gen.DONE
+        late = r0[::211]
+        t["state"][late] = gen.QUEUED
+        t["arrival_ns"][late] = now + 5 * MS + (np.arange(late.size) * 7919) % (50 * MS)
+        r2 = np.nonzero(rid == 2)[0]
+        t["state"][r2] = gen.DONE
+        t["state"][r2[:3]] = gen.QUEUED
+        t["arrival_ns"][r2[:3]] = now + 9 * MS
+        assert_step_parity(wl, steps=3, commit=True)
