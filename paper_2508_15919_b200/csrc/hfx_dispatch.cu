@@ -14,7 +14,8 @@
 //   k_disp_prefix   the queue's rows in order, and the running totals (tokens, entries) of those that
 //                   fit some instance; larger entries are passed over
 //   k_disp_chain    matured instances sorted by (maturity, index); one warp hands consecutive runs of
-//                   the queue to them, each run found by a search on the running totals
+//                   the queue to them, each run found by a probe of the next 32 entries of the running totals
+//                   (a search for the longer ones) and only noted; all threads then write what each took
 //   k_disp_assign   the request -> instance binding of every dispatched row, the new maturity times
 #include <new>
 #include <string.h>
@@ -512,8 +513,10 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
   uint64_t *s_mat = reinterpret_cast<uint64_t *>(smem_raw);     // [R] maturity, biased to unsigned order; then the budgets
   uint32_t *s_id = reinterpret_cast<uint32_t *>(s_mat + R);     // [R]
   int32_t *s_room = reinterpret_cast<int32_t *>(s_id + R);      // [R] entries the batch cap still allows
-  __shared__ int64_t s_pre[CHAIN_WINDOW];
-  __shared__ int32_t s_cnt[CHAIN_WINDOW];
+  int32_t *s_rs = s_room + R;                                   // [R] where the k-th instance's run starts in the queue
+  int32_t *s_rl = s_rs + R;                                     // [R] and how many positions it covers
+  __shared__ int64_t s_pre[CHAIN_WINDOW + 32];                  // running totals of the window; behind them entries that fit nothing
+  __shared__ int32_t s_cnt[CHAIN_WINDOW + 32];
   __shared__ int32_t s_nm, s_k, s_done;
   __shared__ int64_t s_cursor, s_base, s_basec;
   if (threadIdx.x == 0) { s_nm = 0; s_k = 0; s_done = 0; s_cursor = 0; s_base = 0; s_basec = 0; }
@@ -533,10 +536,11 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
     const int r = (int)s_id[k];
     a.inst_order[listed + k] = r;
     const ReplicaPlan *pl = w.plan + r;
-    s_bud[k] = pl->budget;
+    s_bud[k] = pl->budget < (INT64_C(1) << 62) ? pl->budget : (INT64_C(1) << 62);     // (a D-stage budget may be unbounded; the totals stay far below)
     int64_t room = INT32_MAX;
     if (pl->batch_cap != 0) { const int64_t left = (int64_t)pl->batch_cap - pl->n_eff; room = left > 0 ? left : 0; }
     s_room[k] = (int32_t)(room < INT32_MAX ? room : INT32_MAX);
+    s_rs[k] = 0; s_rl[k] = 0;
   }
   if (threadIdx.x == 0) a.n_mature[stage] = nm;
   const int lane = threadIdx.x & 31;
@@ -548,14 +552,32 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
     const int64_t w0 = s_cursor;
     const int64_t wn = nq - w0 < CHAIN_WINDOW ? nq - w0 : CHAIN_WINDOW;
     for (int i = threadIdx.x; i < wn; i += blockDim.x) { s_pre[i] = w.prefix[w0 + i]; s_cnt[i] = w.prefix_cnt[w0 + i]; }
+    if (threadIdx.x < 32) { s_pre[wn + threadIdx.x] = INT64_MAX; s_cnt[wn + threadIdx.x] = INT32_MAX; }
     __syncthreads();
     if (threadIdx.x < 32) {
       int k = s_k;
       int64_t cursor = s_cursor, base = s_base, base_cnt = s_basec;
+      const bool last_window = w0 + wn >= nq;
       for (; k < nm && cursor < nq; k++) {
+        const int64_t limit = base + s_bud[k], limit_cnt = base_cnt + s_room[k];
+        const int i0 = (int)(cursor - w0);
+        {   // most runs are short: one probe of the next 32 entries settles them (the entries that fit are a prefix)
+          const int64_t pre = s_pre[i0 + lane];
+          const int32_t cn = s_cnt[i0 + lane];
+          const int f = __popc(__ballot_sync(0xffffffffu, pre <= limit && (int64_t)cn <= limit_cnt));
+          if (f < 32 && (i0 + f < (int)wn || last_window)) {      // the first entry that does not fit was looked at, or the queue ends
+            if (f > 0) {
+              s_rs[k] = (int32_t)cursor; s_rl[k] = f;
+              base = __shfl_sync(0xffffffffu, pre, f - 1);
+              base_cnt = __shfl_sync(0xffffffffu, cn, f - 1);
+              cursor += f;
+              if (cursor >= w0 + wn) { k++; break; }      // the window is used up
+            }
+            continue;
+          }
+        }
+        // longer runs, and runs that may leave the window: a gallop and a 32-way search on the running totals
         const int64_t span = nq - cursor, avail = w0 + wn - cursor;
-        const int64_t limit = s_bud[k] > INT64_MAX - base ? INT64_MAX : base + s_bud[k];      // (a D-stage budget may be unbounded)
-        const int64_t limit_cnt = base_cnt + s_room[k];
         const int64_t off = cursor - w0 - 1;
         const int64_t hiw = span < avail ? span : avail;
         int64_t m = warp_longest(0, hiw, lane, [&](int64_t x) { return s_pre[off + x] <= limit && (int64_t)s_cnt[off + x] <= limit_cnt; });
@@ -568,18 +590,27 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
           int64_t e_pre, e_cnt;
           if (m <= avail) { e_pre = s_pre[off + m]; e_cnt = s_cnt[off + m]; }
           else { e_pre = w.prefix[cursor + m - 1]; e_cnt = w.prefix_cnt[cursor + m - 1]; }
-          if (lane == 0) {
-            const int r = (int)s_id[k];
-            w.run_start[r] = (int32_t)cursor;
-            w.run_len[r] = (int32_t)m;
-            a.adm_cost[r] = e_pre - base;
-            a.adm_count[r] = (int32_t)(e_cnt - base_cnt);
-          }
+          s_rs[k] = (int32_t)cursor; s_rl[k] = (int32_t)m;
           cursor += m; base = e_pre; base_cnt = e_cnt;
           if (cursor >= w0 + wn) { k++; break; }      // the window is used up
         }
       }
       if (lane == 0) { s_k = k; s_cursor = cursor; s_base = base; s_basec = base_cnt; }
+    }
+  }
+  __syncthreads();
+  // what every instance took, from the running totals at the ends of its run
+  for (int k = threadIdx.x; k < nm; k += blockDim.x) {
+    const int32_t m = s_rl[k];
+    if (m > 0) {
+      const int32_t st = s_rs[k];
+      const int r = (int)s_id[k];
+      const int64_t b0 = st > 0 ? w.prefix[st - 1] : 0, b1 = w.prefix[st + m - 1];
+      const int32_t c0 = st > 0 ? w.prefix_cnt[st - 1] : 0, c1 = w.prefix_cnt[st + m - 1];
+      w.run_start[r] = st;
+      w.run_len[r] = m;
+      a.adm_cost[r] = b1 - b0;
+      a.adm_count[r] = c1 - c0;
     }
   }
 }
@@ -623,7 +654,7 @@ __global__ void __launch_bounds__(DISP_THREADS) k_disp_assign(const HfxParams p,
 struct hfx_dispatch_ws { DispWork w; int ready; };
 
 int hfx_dispatch_configure() {
-  if (cudaFuncSetAttribute(k_disp_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * DISP_MAX_INSTANCES) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_disp_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, 24 * DISP_MAX_INSTANCES) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }
@@ -728,7 +759,7 @@ int hfx_launch_dispatch(hfx_sched *s, const hfx_table *t, int64_t now_ns, const 
     { KernelScope ks(s, KSLOT_DISPATCH); k_disp_plan<<<(R + DISP_THREADS - 1) / DISP_THREADS, DISP_THREADS, 0, st>>>(s->p, a, w, stage); }
     { KernelScope ks(s, KSLOT_DISPATCH); k_disp_tilesum<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], cost, ctl, w.tile_sum, tiles_max, ctl + 3); }
     { KernelScope ks(s, KSLOT_DISPATCH); k_disp_prefix<<<tiles, DISP_THREADS, 0, st>>>(w.val[slot], cost, ctl, w.tile_sum, tiles_max, w.prefix, w.prefix_cnt, o->queue_order, o->n_queue + stage, stage ? w.ctl + 1 : nullptr); }
-    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_chain<<<1, 1024, 16 * (size_t)R, st>>>(s->p, a, w, stage); }
+    { KernelScope ks(s, KSLOT_DISPATCH); k_disp_chain<<<1, 1024, 24 * (size_t)R, st>>>(s->p, a, w, stage); }
     { KernelScope ks(s, KSLOT_DISPATCH); k_disp_assign<<<R, DISP_THREADS, 0, st>>>(s->p, a, w, slot, cost, stage); }
   }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
