@@ -18,7 +18,9 @@
 
 #define FRONT_THREADS 1024
 #define FRONT_PER 8                 // rows per thread in the scans over tile positions: T <= 8192
-#define FRONT_GROUP_MAX 64          // largest group that is put in row order by counting
+#define FRONT_GROUP_MAX 1024        // largest group that is put in row order by counting (a row costs its group's size; the network over the
+                                    // whole tile that larger groups need costs as much as groups of about a thousand rows)
+#define FRONT_TAIL_MAX 64           // more rows bound to no replica than this are ranked by a scan
 #define FRONT_ROW_BYTES 24          // shared memory per row of the tile
 #define FRONT_REP_BYTES 31          // shared memory per replica
 
@@ -241,7 +243,7 @@ __global__ void __launch_bounds__(FRONT_THREADS, 1) k_front(const HfxParams p, c
       run += (cA + cI) | (cA << 16);
     }
   }
-  const bool tail_scan = s_cnt[2 * R + 1] > FRONT_GROUP_MAX;    // many rows bound to no replica: ranked by a scan
+  const bool tail_scan = s_cnt[2 * R + 1] > FRONT_TAIL_MAX;    // many rows bound to no replica: ranked by a scan
   const int any_big = __syncthreads_or(big);          // (also publishes s_base / s_offact)
   uint16_t *fin = s_fin;
 

@@ -235,17 +235,33 @@ __device__ __forceinline__ int64_t next_arrival_listed(const SegArgs &a, const S
 }
 
 // The same when the inactive rows are not listed yet (a long list that the grid writes at the end of the kernel):
-// read from the slabs, a warp of the group per tile, its lanes over the replica's inactive rows of that tile.
+// read from the slabs.  The warps of the group share the tiles; a warp reads the descriptors of 32 of its tiles at
+// once (a lane each), then walks them one by one, its lanes over the replica's inactive rows of the tile, the row
+// kind and the arrival of a row asked for together.  All threads of the group call.
 __device__ __forceinline__ int64_t next_arrival_slabs(const SegArgs &a, const SegCtx &c, int R1, int r, const Grp &G) {
   const int lane = G.tid & 31, warp = G.tid >> 5, nwarp = G.n >> 5;
   int64_t v = HFX_INF;
-  for (int t = warp; t < c.n_tiles; t += nwarp) {
-    const uint2 m = __ldcg(c.M + (size_t)t * R1 + r);
-    const uint32_t ca = m.y >> 16, ci = (m.x >> 16) - ca, src = (m.x & 0xffffu) + ca;
-    const size_t tb = (size_t)t * c.tile_rows;
-    for (uint32_t k = lane; k < ci; k += 32) {
-      const size_t row = tb + __ldcg(c.slab_idx + tb + src + k);
-      if (c.rowflag[row] == KIND_FUTURE) { const int64_t x = a.arrival[row]; v = x < v ? x : v; }
+  for (int t0 = warp; t0 < c.n_tiles; t0 += 32 * nwarp) {      // this warp's tiles t0, t0 + nwarp, ...: 32 at a time
+    const int t = t0 + lane * nwarp;
+    uint32_t ci = 0, src = 0;
+    if (t < c.n_tiles) {
+      const uint2 m = __ldcg(c.M + (size_t)t * R1 + r);
+      const uint32_t ca = m.y >> 16;
+      ci = (m.x >> 16) - ca; src = (m.x & 0xffffu) + ca;
+    }
+    uint32_t some = __ballot_sync(0xffffffffu, ci != 0);
+    while (some) {
+      const int l = __ffs(some) - 1;
+      some &= some - 1;
+      const uint32_t src_l = __shfl_sync(0xffffffffu, src, l), ci_l = __shfl_sync(0xffffffffu, ci, l);
+      const size_t tb = (size_t)(t0 + l * nwarp) * c.tile_rows;
+#pragma unroll 2
+      for (uint32_t k = lane; k < ci_l; k += 32) {
+        const size_t row = tb + __ldcg(c.slab_idx + tb + src_l + k);
+        const uint8_t kind = c.rowflag[row];
+        const int64_t x = a.arrival[row];
+        if (kind == KIND_FUTURE && x < v) v = x;
+      }
     }
   }
   return v;
@@ -1723,7 +1739,7 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
   {
     const int g = tid / GROUP_THREADS;
     const Grp G = {tid - g * GROUP_THREADS, GROUP_THREADS, g + 1};
-    for (int r = blockIdx.x * REP_GROUPS + g; r <= R; r += gridDim.x * REP_GROUPS) {
+    for (int r = g * gridDim.x + blockIdx.x; r <= R; r += gridDim.x * REP_GROUPS) {      // consecutive replicas on different SMs: few replicas still use them all
       uint32_t n_all, n_act;
       counts(r, n_all, n_act);
       if (need_of(n_all, n_act) > SEG_TINY) continue;
@@ -1749,32 +1765,39 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
   }
 
   // ---- long lists of inactive rows (ordered steps): every block lists a range of tiles ----------------
+  // The replicas with a long list are collected in shared memory; a thread per replica adds up the replica's
+  // inactive rows in the tiles before the block's, then a warp per replica copies the rows of the block's tiles.
   if (longer) {
+    __syncthreads();      // the larger replicas are done with the block's shared memory
+    uint16_t *s_lr = reinterpret_cast<uint16_t *>(smem_raw);                                   // [R1] the replicas
+    uint32_t *s_lpre = reinterpret_cast<uint32_t *>(smem_raw + (((size_t)R1 * 2 + 15) & ~(size_t)15));   // [R1] rows in earlier tiles
+    if (tid == 0) s_scan[0] = 0;
+    __syncthreads();
+    for (int r = tid; r < R1; r += blockDim.x)
+      if ((s_long[r >> 5] >> (r & 31)) & 1u) s_lr[atomicAdd(&s_scan[0], 1u)] = (uint16_t)r;
+    __syncthreads();
+    const int n_long = (int)s_scan[0];
     const int per = (c.n_tiles + gridDim.x - 1) / gridDim.x;
     const int tA = blockIdx.x * per < c.n_tiles ? blockIdx.x * per : c.n_tiles;
     const int tB = tA + per < c.n_tiles ? tA + per : c.n_tiles;
-    for (int wd = 0; wd * 32 < R1; wd++) {
-      uint32_t word = s_long[wd];
-      while (word) {
-        const int r = wd * 32 + __ffs(word) - 1;
-        word &= word - 1;
-        // inactive rows of replica r in the tiles before mine
+    if (tA < tB) {
+      for (int j = tid; j < n_long; j += blockDim.x) {
+        const int r = s_lr[j];
         uint32_t pre = 0;
-        for (int t = tid; t < tA; t += blockDim.x) { const uint2 m = __ldcg(c.M + (size_t)t * R1 + r); pre += (m.x >> 16) - (m.y >> 16); }
-        pre = (uint32_t)warp_sum_i64(pre);
-        __syncthreads();
-        if (lane == 0) s_scan[warp] = pre;
-        __syncthreads();
-        pre = 0;
-        for (int k = 0; k < 32; k++) pre += s_scan[k];
-        const uint32_t dst = begin[r] + (uint32_t)(__ldcg(c.tot + r) >> 32) + pre;
-        uint32_t done = 0;
+#pragma unroll 8
+        for (int t = 0; t < tA; t++) { const uint2 m = __ldcg(c.M + (size_t)t * R1 + r); pre += (m.x >> 16) - (m.y >> 16); }
+        s_lpre[j] = pre;
+      }
+      __syncthreads();
+      for (int j = warp; j < n_long; j += (int)(blockDim.x >> 5)) {
+        const int r = s_lr[j];
+        uint32_t dst = begin[r] + (uint32_t)(__ldcg(c.tot + r) >> 32) + s_lpre[j];
         for (int t = tA; t < tB; t++) {
           const uint2 m = __ldcg(c.M + (size_t)t * R1 + r);
           const uint32_t ca = m.y >> 16, ci = (m.x >> 16) - ca, src = (m.x & 0xffffu) + ca;
           const size_t tb = (size_t)t * c.tile_rows;
-          for (uint32_t k = tid; k < ci; k += blockDim.x) a.order[dst + done + k] = (int32_t)(tb + __ldcg(c.slab_idx + tb + src + k));
-          done += ci;
+          for (uint32_t k = lane; k < ci; k += 32) a.order[dst + k] = (int32_t)(tb + __ldcg(c.slab_idx + tb + src + k));
+          dst += ci;
         }
       }
     }
