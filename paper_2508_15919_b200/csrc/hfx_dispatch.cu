@@ -561,16 +561,27 @@ __global__ void __launch_bounds__(1024) k_disp_chain(const HfxParams p, const Di
       for (; k < nm && cursor < nq; k++) {
         const int64_t limit = base + s_bud[k], limit_cnt = base_cnt + s_room[k];
         const int i0 = (int)(cursor - w0);
-        {   // most runs are short: one probe of the next 32 entries settles them (the entries that fit are a prefix)
-          const int64_t pre = s_pre[i0 + lane];
-          const int32_t cn = s_cnt[i0 + lane];
-          const int f = __popc(__ballot_sync(0xffffffffu, pre <= limit && (int64_t)cn <= limit_cnt));
-          if (f < 32 && (i0 + f < (int)wn || last_window)) {      // the first entry that does not fit was looked at, or the queue ends
+        {   // most runs are short: probes of the next 32 entries, up to eight in a row, settle them (the entries that
+            // fit are a prefix); the first entry that does not fit must have been looked at, or the queue must end
+          int i1 = i0;
+          int64_t e_pre = base, e_cnt = base_cnt;
+          bool settled = false;
+          for (int it = 0; it < 8; it++) {
+            const int64_t pre = s_pre[i1 + lane];
+            const int32_t cn = s_cnt[i1 + lane];
+            const int f = __popc(__ballot_sync(0xffffffffu, pre <= limit && (int64_t)cn <= limit_cnt));
             if (f > 0) {
-              s_rs[k] = (int32_t)cursor; s_rl[k] = f;
-              base = __shfl_sync(0xffffffffu, pre, f - 1);
-              base_cnt = __shfl_sync(0xffffffffu, cn, f - 1);
-              cursor += f;
+              e_pre = __shfl_sync(0xffffffffu, pre, f - 1);
+              e_cnt = __shfl_sync(0xffffffffu, cn, f - 1);
+              i1 += f;
+            }
+            if (f < 32) { settled = i1 < (int)wn || last_window; break; }
+            if (i1 >= (int)wn && !last_window) break;      // the window is used up and the queue goes on: the search below decides
+          }
+          if (settled) {
+            if (i1 > i0) {
+              s_rs[k] = (int32_t)cursor; s_rl[k] = i1 - i0;
+              cursor += i1 - i0; base = e_pre; base_cnt = e_cnt;
               if (cursor >= w0 + wn) { k++; break; }      // the window is used up
             }
             continue;
