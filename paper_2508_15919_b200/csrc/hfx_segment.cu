@@ -1789,14 +1789,19 @@ __global__ void __launch_bounds__(REP_THREADS, 1) k_replicas(const HfxParams p, 
         s_lpre[j] = pre;
       }
       __syncthreads();
-      for (int j = warp; j < n_long; j += (int)(blockDim.x >> 5)) {
+      // many long lists: a warp per replica; few (one bucket of unbound rows, say): the whole block on each
+      const bool by_warp = n_long >= (int)(blockDim.x >> 5);
+      const int first = by_warp ? warp : 0, step = by_warp ? (int)(blockDim.x >> 5) : 1;
+      const uint32_t k0 = by_warp ? (uint32_t)lane : (uint32_t)tid, kstep = by_warp ? 32u : blockDim.x;
+      for (int j = first; j < n_long; j += step) {
         const int r = s_lr[j];
         uint32_t dst = begin[r] + (uint32_t)(__ldcg(c.tot + r) >> 32) + s_lpre[j];
         for (int t = tA; t < tB; t++) {
           const uint2 m = __ldcg(c.M + (size_t)t * R1 + r);
           const uint32_t ca = m.y >> 16, ci = (m.x >> 16) - ca, src = (m.x & 0xffffu) + ca;
           const size_t tb = (size_t)t * c.tile_rows;
-          for (uint32_t k = lane; k < ci; k += 32) a.order[dst + k] = (int32_t)(tb + __ldcg(c.slab_idx + tb + src + k));
+#pragma unroll 4
+          for (uint32_t k = k0; k < ci; k += kstep) a.order[dst + k] = (int32_t)(tb + __ldcg(c.slab_idx + tb + src + k));
           dst += ci;
         }
       }
