@@ -242,21 +242,25 @@ struct PlanMemo {
   uint64_t m_run, m_q;
   int64_t min_tpot, min_ttft;
   int64_t n_safe;           // < 0: none yet
+  int64_t need;             // > 0: the caller only wants the budget if at least this many tokens are safe (the shortest
+                            // prompt it could admit); otherwise the budget it gets is 0.  <= 0: always the exact budget
   int have_run, have_q;
 };
-__device__ __forceinline__ void plan_memo_reset(PlanMemo &m) { m.m_run = 0; m.m_q = 0; m.min_tpot = 0; m.min_ttft = 0; m.n_safe = -1; m.have_run = 0; m.have_q = 0; }
+__device__ __forceinline__ void plan_memo_reset(PlanMemo &m) { m.m_run = 0; m.m_q = 0; m.min_tpot = 0; m.min_ttft = 0; m.n_safe = -1; m.need = 0; m.have_run = 0; m.have_q = 0; }
 
 // Largest n in [0, cap] with E_p(n) * den <= num (num = nh:nl as 128 bits, den > 0), 0 if none.
 // `hint` >= 0: a value the answer is probably close to (tried first: 32 neighbours in one round).
+// `need` > 0: return -1 at once when fewer than `need` tokens are safe.
 __device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t nl, uint64_t den, int64_t cap, int lane,
-                                     int64_t hint = -1) {
+                                     int64_t hint = -1, int64_t need = 0) {
   auto fits = [&](int64_t n) {
     const uint64_t ep = (uint64_t)dev_Ep(p, n);
     const uint64_t ph = __umul64hi(ep, den), pl = ep * den;
     return ph < nh || (ph == nh && pl <= nl);
   };
-  if (!fits(0)) return 0;
-  int64_t lo = 0, hi = cap;          // fits(lo); the answer lies in [lo, hi]
+  if (need > 0) { if (need > cap || !fits(need)) return -1; }
+  else if (!fits(0)) return 0;
+  int64_t lo = need > 0 ? need : 0, hi = cap;          // fits(lo); the answer lies in [lo, hi]
   if (hint >= 0) {
     int64_t base = hint - 15;
     if (base < 1) base = 1;
@@ -264,7 +268,7 @@ __device__ inline int64_t warp_nsafe(const HfxParams &p, uint64_t nh, uint64_t n
     const int64_t cand = base + lane;
     const int f = __popc(__ballot_sync(0xffffffffu, cand <= cap && fits(cand)));    // a prefix of the lanes
     if (f == 0) hi = base - 1;                    // the answer lies below the neighbourhood
-    else if (f == 32) lo = base + 31;             // at or above its top
+    else if (f == 32) lo = base + 31 > lo ? base + 31 : lo;      // at or above its top
     else return base + f - 1;
   }
   while (lo < hi) {
@@ -317,15 +321,16 @@ __device__ inline void warp_plan(const HfxParams &p, const int64_t *cls_ttft, co
           if (memo) { memo->m_q = mask_q; memo->min_ttft = min_ttft; memo->have_q = 1; }
         }
         const bool decoding = pl.n_eff > 0 && pl.tpot_eff < HFX_INF;
-        const int64_t hint = memo ? memo->n_safe : -1;
+        const int64_t hint = memo ? memo->n_safe : -1, need = memo ? memo->need : 0;
         if (min_ttft == HFX_INF) n_safe = cfg.token_cap;
-        else if (!decoding) n_safe = warp_nsafe(p, 0, (uint64_t)min_ttft, 2, cfg.token_cap, lane, hint);     // 2 E_p <= TTFT
+        else if (!decoding) n_safe = warp_nsafe(p, 0, (uint64_t)min_ttft, 2, cfg.token_cap, lane, hint, need);     // 2 E_p <= TTFT
         else if (pl.tpot_eff <= pl.e_d) n_safe = 0;
         else {
           const uint64_t x = (uint64_t)min_ttft, y = (uint64_t)(pl.tpot_eff - pl.e_d);
-          n_safe = warp_nsafe(p, __umul64hi(x, y), x * y, (uint64_t)(2 * pl.tpot_eff - pl.e_d), cfg.token_cap, lane, hint);
+          n_safe = warp_nsafe(p, __umul64hi(x, y), x * y, (uint64_t)(2 * pl.tpot_eff - pl.e_d), cfg.token_cap, lane, hint, need);
         }
-        if (memo) memo->n_safe = n_safe;
+        if (n_safe < 0) n_safe = 0;      // fewer than `need` tokens are safe: the caller admits nothing
+        else if (memo) memo->n_safe = n_safe;
       }
       budget = n_safe < cap_left ? n_safe : cap_left;
     }

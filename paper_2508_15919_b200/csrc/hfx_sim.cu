@@ -11,16 +11,21 @@
 //   - admission extracts the most urgent eligible request repeatedly (block-wide arg-min on
 //     (prio, clamp(slack), req_id)) and stops at the first one that does not fit, which is
 //     exactly the prefix-closed rule of the sorted formulation.
-// Shared memory is what bounds the number of resident traces, so a row takes 19 bytes: one 8-byte slot
+// Shared memory is what bounds the number of resident traces, so a row takes 15 bytes: one 8-byte slot
 // (arrival, then the slack base while queued, then the finish iteration while running), a word (prompt
-// length and priority), a byte (class and state) and three list entries; the rows admitted in an
-// iteration are parked in the part of the queue array that their extraction frees.
+// length and priority), a byte (class and state) and one list entry (the queue from the front of the list array, the running batch
+// from its back: a row is in one of them at most); the rows
+// admitted in an iteration are parked in the part of the queue array that their extraction frees, and the
+// running list is kept in place (a finished request's place is filled from the tail).  A scan of the queue is
+// only made when the budget reaches the shortest queued prompt (a bound kept beside the queue).
 #include "hfx_internal.cuh"
 
 #define SIM_THREADS 128
 #define SIM_WARPS (SIM_THREADS / 32)
-#define SIM_SMEM_ROWS 10240          // longest trace whose rows are kept in shared memory (19 bytes each); longer ones work in global scratch
-#define SIM_BYTES_PER_ROW 19
+#define SIM_SMEM_ROWS 10240          // longest trace whose rows are kept in shared memory (15 bytes each); longer ones work in global scratch
+#define SIM_BYTES_PER_ROW 15
+#define SIM_CLASS_BYTES(nc) ((((size_t)(nc) * 24) + 15) & ~(size_t)15)     // per-class tables in dynamic shared memory: TTFT, TPOT, two counters
+#define SIM_HOLES 32                 // finished requests of one iteration whose places in the running list are noted
 #define SIM_OUTLEN_CAP (1 << 30)   // output lengths are clamped here when the finish iteration is formed
 
 // the byte of a row: class<6> | state<2>; the word of a row: prompt_len<25> | prio<6>, prio 63 marks a row with bad data
@@ -47,17 +52,19 @@ struct SimShared {
   int64_t now, mat, sum_kv;
   int64_t t1, t2, lp, mat_next;
   int64_t d_kv;                 // change of sum_kv collected during commit
-  int32_t cnt_run[HFX_MAX_CLASSES], cnt_q[HFX_MAX_CLASSES];
-  int32_t head, head_prev, nq, nr, nr_next, na, no, arrived;
+  int32_t head, head_prev, nq, nr, na, no, arrived;
   int32_t worked, stop, trace, zero_prompt;
+  int32_t min_prompt;           // a lower bound of the shortest prompt in the queue: lowered by every arrival, made exact by
+                                // every scan of the queue (an admission can only raise the true value)
+  int32_t best_min[2][SIM_WARPS];
+  int32_t n_holes;              // requests of the running list that finished in this iteration
+  uint16_t holes[SIM_HOLES];    // their places in the list (the first SIM_HOLES of them)
   // arg-min scratch, double buffered
   uint64_t best_key[2][SIM_WARPS];
   uint32_t best_id[2][SIM_WARPS];
   int32_t best_slot[2][SIM_WARPS];
   // end-of-trace counters
   int32_t n_fin, n_rej, n_att, n_a, n_b;
-  int64_t ttft[HFX_MAX_CLASSES];   // TTFT SLO per class
-  int64_t tpot[HFX_MAX_CLASSES];   // TPOT SLO per class
 };
 
 __device__ __forceinline__ void sort_i64(int64_t *v, int n) {
@@ -96,13 +103,19 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
                                                      uint32_t *__restrict__ status, unsigned char *__restrict__ scratch) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int cap = a.cap_rows;
-  unsigned char *rows_mem = SCRATCH ? scratch + (size_t)blockIdx.x * cap * SIM_BYTES_PER_ROW : smem_raw;
+  // per class, in front of the rows: TTFT and TPOT bounds, requests in flight, requests in the queue
+  const int nc = p.n_classes;
+  int64_t *c_ttft = reinterpret_cast<int64_t *>(smem_raw), *c_tpot = c_ttft + nc;
+  int32_t *c_run = reinterpret_cast<int32_t *>(c_tpot + nc), *c_q = c_run + nc;
+  unsigned char *rows_mem = SCRATCH ? scratch + (size_t)blockIdx.x * cap * SIM_BYTES_PER_ROW : smem_raw + SIM_CLASS_BYTES(nc);
   int64_t *s_arr = reinterpret_cast<int64_t *>(rows_mem);              // arrival; the slack base once arrived; the finish iteration once running; later the TTFT, then the TPOT samples
   uint32_t *s_word = reinterpret_cast<uint32_t *>(s_arr + cap);        // prompt_len | prio << 25
-  uint16_t *s_q = reinterpret_cast<uint16_t *>(s_word + cap);          // visible queue (row indices, unordered); behind it the rows admitted in this iteration
-  uint16_t *s_run = s_q + cap;                                         // running batch, ping
-  uint16_t *s_run2 = s_run + cap;                                      // running batch, pong
-  uint8_t *s_byte = reinterpret_cast<uint8_t *>(s_run2 + cap);         // class | state << 6
+  // One list array for both lists (a row is in one of them at most): from the front the visible queue (row indices,
+  // unordered) and behind it the rows admitted in this iteration; from the back the running batch (RUN(s), unordered;
+  // 0xffff: a request that just finished)
+  uint16_t *s_q = reinterpret_cast<uint16_t *>(s_word + cap);
+  uint8_t *s_byte = reinterpret_cast<uint8_t *>(s_q + cap);            // class | state << 6
+#define RUN(s) s_q[cap - 1 - (s)]
   __shared__ SimShared S;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -119,11 +132,11 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     // ---- stage the trace ----------------------------------------------------------------
     if (tid == 0) {
       S.now = 0; S.mat = 0; S.sum_kv = 0; S.head = 0; S.head_prev = 0; S.nq = 0; S.nr = 0; S.stop = 0;
-      S.n_fin = 0; S.n_rej = 0; S.n_att = 0; S.n_a = 0; S.n_b = 0; S.zero_prompt = 0;
-      S.arrived = 0; S.no = 0; S.na = 0; S.nr_next = 0; S.d_kv = 0;
+      S.n_fin = 0; S.n_rej = 0; S.n_att = 0; S.n_a = 0; S.n_b = 0; S.zero_prompt = 0; S.min_prompt = INT32_MAX; S.n_holes = 0;
+      S.arrived = 0; S.no = 0; S.na = 0; S.d_kv = 0;
     }
     __syncthreads();
-    for (int c = tid; c < HFX_MAX_CLASSES; c += SIM_THREADS) { S.cnt_run[c] = 0; S.cnt_q[c] = 0; S.ttft[c] = c < p.n_classes ? p.ttft[c] : 0; S.tpot[c] = c < p.n_classes ? p.tpot[c] : 0; }
+    for (int c = tid; c < nc; c += SIM_THREADS) { c_run[c] = 0; c_q[c] = 0; c_ttft[c] = p.ttft[c]; c_tpot[c] = p.tpot[c]; }
     uint32_t bad = 0;
     for (int i = tid; i < m; i += SIM_THREADS) {
       const int64_t g = (int64_t)b + i;
@@ -154,7 +167,6 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
     int executed = 0;
     PlanMemo memo;          // of the planning warp: the trace's replica is planned every iteration
     plan_memo_reset(memo);
-    uint16_t *run_cur = s_run, *run_nxt = s_run2;
     for (int it = 0; it < a.iters; it++) {
       // ---- 1. arrivals: rows [head, head + k) with arrival <= now join the queue -----------
       // (the iteration's counters were cleared by the thread that closed the previous one)
@@ -167,7 +179,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           const uint32_t w = s_word[i];
           if (ROW_PRIO(w) == ROW_INVALID_PRIO) continue;
           const uint32_t cls = ROW_CLS(s_byte[i]);
-          atomicAdd(&S.cnt_q[cls], 1);
+          atomicAdd(&c_q[cls], 1);
           if (ROW_PROMPT(w) > cfg.token_cap) {
             // can never be served: visible for this one iteration, rejected at its commit (which looks through
             // the rows that arrived in the iteration again)
@@ -175,9 +187,10 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           } else {
             const int slot = atomicAdd(&S.nq, 1);
             s_q[slot] = (uint16_t)i;
+            atomicMin(&S.min_prompt, (int32_t)ROW_PROMPT(w));
             // from here on the row's slot holds its slack base, ttft_slo + arrival - E_p(prompt_len):
             // the slack at any later decision is the base minus the earliest start
-            const int64_t ttft = S.ttft[cls];
+            const int64_t ttft = c_ttft[cls];
             s_arr[i] = ttft > 0 ? ttft + s_arr[i] - dev_Ep(p, ROW_PROMPT(w)) : BASE_UNBOUNDED;
           }
         }
@@ -188,29 +201,35 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       // ---- 2. plan: E_d of the running batch and the safe budget (the first warp) ----------------
       if (warp == 0) {
         if (lane == 0) { S.head_prev = S.head; S.head += S.arrived; }
-        const uint32_t r0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_run[lane] > 0);
-        const uint32_t r1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && S.cnt_run[lane + 32] > 0);
-        const uint32_t q0 = __ballot_sync(0xffffffffu, lane < p.n_classes && S.cnt_q[lane] > 0);
-        const uint32_t q1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && S.cnt_q[lane + 32] > 0);
+        const uint32_t r0 = __ballot_sync(0xffffffffu, lane < p.n_classes && c_run[lane] > 0);
+        const uint32_t r1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && c_run[lane + 32] > 0);
+        const uint32_t q0 = __ballot_sync(0xffffffffu, lane < p.n_classes && c_q[lane] > 0);
+        const uint32_t q1 = __ballot_sync(0xffffffffu, lane + 32 < p.n_classes && c_q[lane + 32] > 0);
         ReplicaPlan pl0;
-        warp_plan(p, S.ttft, S.tpot, cfg, S.now, S.mat, S.nr, S.sum_kv, ((uint64_t)r1 << 32) | r0, ((uint64_t)q1 << 32) | q0, pl0, lane, &memo);
+        // the budget only matters if it reaches the shortest queued prompt (a queue without requests admits nothing)
+        memo.need = S.zero_prompt ? 0 : (S.nq > 0 ? (int64_t)S.min_prompt : (int64_t)cfg.token_cap + 1);
+        warp_plan(p, c_ttft, c_tpot, cfg, S.now, S.mat, S.nr, S.sum_kv, ((uint64_t)r1 << 32) | r0, ((uint64_t)q1 << 32) | q0, pl0, lane, &memo);
         if (lane == 0) S.plan = pl0;
       }
       __syncthreads();
       const int64_t budget = S.plan.budget, start = S.plan.start;
       const int nr = S.nr;
+      const int32_t min_prompt = S.min_prompt;
 
       // ---- 3. admission: extract the most urgent request that fits alone, until one fails ----
       int64_t s_cost = 0, adm_cost = 0;
       int s_cnt = 0, adm_cnt = 0;
       int nq = S.nq;
-      if (budget > 0 || S.zero_prompt) {
+      // (a budget below the shortest queued prompt admits nothing: the scan of the queue would come back empty)
+      if ((budget > 0 || S.zero_prompt) && (int64_t)min_prompt <= budget) {
         int buf = 0;
         for (;;) {
           uint64_t bk = ~0ull; uint32_t bid = ~0u; int bslot = -1;
+          int32_t lmin = INT32_MAX;
           for (int s = tid; s < nq; s += SIM_THREADS) {
             const int i = s_q[s];
             const uint32_t wd = s_word[i];
+            lmin = (int32_t)ROW_PROMPT(wd) < lmin ? (int32_t)ROW_PROMPT(wd) : lmin;
             if ((int64_t)ROW_PROMPT(wd) > (p.first_fit ? budget - adm_cost : budget)) continue;      // first fit: against what is left
             // slack of a queued request: ttft_slo - (start - arrival) - E_p(prompt_len) = base - start
             const int64_t base = s_arr[i];
@@ -234,8 +253,15 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
             }
             if (k2 < bk || (k2 == bk && i2 < bid)) { bk = k2; bid = i2; bslot = s2; }
           }
-          if (lane == 0) { S.best_key[buf][warp] = bk; S.best_id[buf][warp] = bid; S.best_slot[buf][warp] = bslot; }
+          lmin = __reduce_min_sync(0xffffffffu, lmin);
+          if (lane == 0) { S.best_key[buf][warp] = bk; S.best_id[buf][warp] = bid; S.best_slot[buf][warp] = bslot; S.best_min[buf][warp] = lmin; }
           __syncthreads();
+          if (tid == 0) {      // the shortest prompt of the queue as it stood for this scan
+            int32_t mn = S.best_min[buf][0];
+#pragma unroll
+            for (int w = 1; w < SIM_WARPS; w++) mn = S.best_min[buf][w] < mn ? S.best_min[buf][w] : mn;
+            S.min_prompt = mn;
+          }
           bk = S.best_key[buf][0]; bid = S.best_id[buf][0]; bslot = S.best_slot[buf][0];
 #pragma unroll
           for (int w = 1; w < SIM_WARPS; w++) {
@@ -279,18 +305,18 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       int64_t d_kv = 0;
       // running batch: one more token each; a request finishes when gen + 1 reaches output_len
       for (int s = tid; s < nr; s += SIM_THREADS) {
-        const int i = run_cur[s];
+        const int i = RUN(s);
         if (it >= (int32_t)s_arr[i]) {       // gen + 1 reaches output_len in this iteration
+          RUN(s) = 0xffffu;                // its place is free
+          const int h = atomicAdd(&S.n_holes, 1);
+          if (h < SIM_HOLES) S.holes[h] = (uint16_t)s;
           const uint32_t cls = ROW_CLS(s_byte[i]);
           s_byte[i] = ROW_BYTE(cls, HFX_DONE);
           a.finish[(int64_t)b + i] = t2;
-          atomicSub(&S.cnt_run[cls], 1);
+          atomicSub(&c_run[cls], 1);
           const int32_t outlen = __ldg(a.output_len + b + i);
           d_kv -= (int64_t)ROW_PROMPT(s_word[i]) + outlen - 2;       // leaves with the context it had before this step
-        } else {
-          run_nxt[atomicAdd(&S.nr_next, 1)] = (uint16_t)i;
-          d_kv += 1;
-        }
+        } else d_kv += 1;
       }
       // admitted requests: first token at t1
       for (int s = tid; s < adm_cnt; s += SIM_THREADS) {
@@ -299,14 +325,13 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
         const int32_t outlen = __ldg(a.output_len + b + i);
         s_arr[i] = it + (outlen < SIM_OUTLEN_CAP ? outlen : SIM_OUTLEN_CAP) - 1;      // the slot now holds the finish iteration
         const uint32_t cls = ROW_CLS(s_byte[i]);
-        atomicSub(&S.cnt_q[cls], 1);
+        atomicSub(&c_q[cls], 1);
         if (outlen <= 1) {
           s_byte[i] = ROW_BYTE(cls, HFX_DONE);
           a.finish[(int64_t)b + i] = t1;
         } else {
-          s_byte[i] = ROW_BYTE(cls, HFX_RUNNING);
-          run_nxt[atomicAdd(&S.nr_next, 1)] = (uint16_t)i;
-          atomicAdd(&S.cnt_run[cls], 1);
+          s_byte[i] = ROW_BYTE(cls, HFX_RUNNING);      // (joins the running list below)
+          atomicAdd(&c_run[cls], 1);
           d_kv += ROW_PROMPT(s_word[i]);
         }
       }
@@ -317,7 +342,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           if (ROW_PRIO(w) != ROW_INVALID_PRIO && ROW_PROMPT(w) > cfg.token_cap) {
             const uint32_t cls = ROW_CLS(s_byte[i]);
             s_byte[i] = ROW_BYTE(cls, HFX_REJECTED);
-            atomicSub(&S.cnt_q[cls], 1);
+            atomicSub(&c_q[cls], 1);
           }
         }
       }
@@ -326,9 +351,45 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
       __syncthreads();
       if (tid == 0) {
         S.sum_kv += S.d_kv;
-        S.nr = S.nr_next;
+        {   // the running list, in place: free places below the new length are filled from the tail, then the
+            // admitted requests that go on decoding join (the list has no order)
+          int n = S.nr;
+          const int k = S.n_holes;
+          if (k > 0) {
+            if (k <= SIM_HOLES) {
+              for (int e = 1; e < k; e++) {      // the noted places in ascending order (k is small)
+                const uint16_t x = S.holes[e];
+                int f = e - 1;
+                while (f >= 0 && S.holes[f] > x) { S.holes[f + 1] = S.holes[f]; f--; }
+                S.holes[f + 1] = x;
+              }
+              int tail = n - 1;
+              for (int e = 0; e < k; e++) {
+                const int h = S.holes[e];
+                while (tail > h && RUN(tail) == 0xffffu) tail--;
+                if (h >= tail) break;          // this place and the ones after it lie beyond the new length
+                RUN(h) = RUN(tail); tail--;
+              }
+            } else {                             // many at once: one pass from both ends
+              int lo = 0, hi = n - 1;
+              for (;;) {
+                while (lo < hi && RUN(lo) != 0xffffu) lo++;
+                while (hi > lo && RUN(hi) == 0xffffu) hi--;
+                if (lo >= hi) break;
+                RUN(lo) = RUN(hi); RUN(hi) = 0xffffu;
+              }
+            }
+            n -= k;
+          }
+          const int na = S.na, q0 = S.nq;
+          for (int e = na - 1; e >= 0; e--) {      // from the last parked row down: the list grows towards them and may take
+            const int i = s_q[q0 + e];              // the place of a row already read, never of one still to be read
+            if ((s_byte[i] >> 6) == HFX_RUNNING) RUN(n++) = (uint16_t)i;
+          }
+          S.nr = n;
+        }
         S.mat = S.mat_next;
-        S.arrived = 0; S.no = 0; S.na = 0; S.nr_next = 0; S.d_kv = 0;      // for the next iteration
+        S.arrived = 0; S.no = 0; S.na = 0; S.n_holes = 0; S.d_kv = 0;      // for the next iteration
         if (S.worked) S.now = t2;
         else {
           int64_t ev = HFX_INF;
@@ -339,7 +400,6 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
           if (ev == HFX_INF) S.stop = 1; else S.now = ev;
         }
       }
-      { uint16_t *x = run_cur; run_cur = run_nxt; run_nxt = x; }
       __syncthreads();
       if (S.stop) break;
       executed++;
@@ -423,7 +483,7 @@ __global__ void __launch_bounds__(SIM_THREADS) k_sim(const HfxParams p, const Si
 }
 
 int hfx_sim_configure() {
-  if (cudaFuncSetAttribute(k_sim<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SIM_SMEM_ROWS * SIM_BYTES_PER_ROW) != cudaSuccess)
+  if (cudaFuncSetAttribute(k_sim<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SIM_SMEM_ROWS * SIM_BYTES_PER_ROW + (int)SIM_CLASS_BYTES(HFX_MAX_CLASSES)) != cudaSuccess)
     return HFX_E_CUDA;
   return HFX_OK;
 }
@@ -449,16 +509,16 @@ int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_tra
   a.iters_executed = o->iters_executed; a.finished = o->finished; a.rejected = o->rejected; a.attained = o->attained;
   a.ttft_p50 = o->ttft_p50_ns; a.ttft_p99 = o->ttft_p99_ns; a.tpot_p50 = o->tpot_p50_ns; a.tpot_p99 = o->tpot_p99_ns;
   a.now_out = o->now_ns;
-  const size_t rows_bytes = (size_t)cap * SIM_BYTES_PER_ROW;
+  const size_t rows_bytes = (size_t)cap * SIM_BYTES_PER_ROW, class_bytes = SIM_CLASS_BYTES(s->p.n_classes);
   if (cudaMemsetAsync(d_work_counter, 0, sizeof(uint32_t), s->stream) != cudaSuccess) return HFX_E_CUDA;
   if (cap <= SIM_SMEM_ROWS) {
-    int per_sm = (int)((224 * 1024) / (rows_bytes + 3072));
+    int per_sm = (int)((224 * 1024) / (rows_bytes + class_bytes + 1792));      // (static shared memory and the per-block reserve)
     if (per_sm < 1) per_sm = 1;
     if (per_sm > 8) per_sm = 8;
     int grid = s->n_sm * per_sm;
     if (grid > n_traces) grid = n_traces;
     KernelScope ks(s, KSLOT_SIM);
-    k_sim<false><<<grid, SIM_THREADS, rows_bytes, s->stream>>>(s->p, a, d_work_counter, s->d_status, nullptr);
+    k_sim<false><<<grid, SIM_THREADS, rows_bytes + class_bytes, s->stream>>>(s->p, a, d_work_counter, s->d_status, nullptr);
   } else {
     // long traces: the rows of every resident block in a scratch buffer (two blocks per SM), allocated when first needed
     int grid = s->n_sm * 2;
@@ -472,7 +532,7 @@ int hfx_launch_sim_kernel(hfx_sched *s, const hfx_table *t, const int32_t *d_tra
       s->sim_scratch_bytes = need;
     }
     KernelScope ks(s, KSLOT_SIM);
-    k_sim<true><<<grid, SIM_THREADS, 0, s->stream>>>(s->p, a, d_work_counter, s->d_status, s->d_sim_scratch);
+    k_sim<true><<<grid, SIM_THREADS, class_bytes, s->stream>>>(s->p, a, d_work_counter, s->d_status, s->d_sim_scratch);
   }
   return cudaGetLastError() == cudaSuccess ? HFX_OK : HFX_E_CUDA;
 }

@@ -1124,3 +1124,19 @@ def test_idle_replica_with_a_long_list_of_inactive_rows_jumps_to_its_next_arriva
         t["state"][r2[:3]] = gen.QUEUED
         t["arrival_ns"][r2[:3]] = now + 9 * MS
         assert_step_parity(wl, steps=3, commit=True)
+
+
+@pytest.mark.parametrize("m", [16, 64, 2048])
+def test_simulator_every_row_live_at_once(m):
+    # The queue and the running batch share one list array of the trace's length (a multiple of 16 here, so the array
+    # has no spare entry): every request arrives at time 0, prompts are short so that several are admitted per
+    # iteration, outputs are long so that nothing finishes while the queue drains, then they finish in bunches.
+    rng = np.random.default_rng(m)
+    rows = [dict(prompt_len=int(rng.integers(1, 40)), output_len=int(rng.integers(150, 170)), arrival_ns=0, req_id=i,
+                 class_id=int(rng.integers(0, 2))) for i in range(m)]
+    late = np.sort(rng.integers(0, 40 * MS, m))                  # a second trace (rows in arrival order), short outputs: places free up all the time
+    rows += [dict(prompt_len=int(rng.integers(1, 40)), output_len=int(rng.integers(2, 5)), arrival_ns=int(late[i]), req_id=m + i)
+             for i in range(m)]
+    wl = make_wl(rows, [(200 * MS, 30 * MS, 0), (1000 * MS, 50 * MS, 1)], replicas=[(gen.COLOCATED, 8192, 0)] * 2, now=[0, 0],
+                 maturity=[0, 0], trace_off=[0, m, 2 * m], sim_iters=600)
+    assert_sim_parity(wl)
