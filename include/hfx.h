@@ -405,7 +405,7 @@ int hfx_slo_map(hfx_sched *s, int32_t n_prio, const hfx_slo_window *win, const h
  * until nothing is left to happen.  Written: state, gen, first_token_ns,
  * last_token_ns, finish_ns and `out`.
  * A trace of up to 10240 rows is kept in shared memory; a longer one (at most 65535 rows) works in a scratch
- * buffer in device memory (19 bytes per row for two traces per SM), which the first call that needs it
+ * buffer in device memory (15 bytes per row for two traces per SM), which the first call that needs it
  * allocates with cudaMalloc after synchronising the stream, so such a call should not be made inside a stream
  * capture; hfx_sched_destroy frees it.
  * Errors: HFX_E_ARG, HFX_E_ALIGN, HFX_E_CAPACITY (n_traces > n_replicas, or a
